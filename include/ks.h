@@ -1,0 +1,194 @@
+/*
+ * ks.h -- C ABI of libks: execution-free CUTLASS kernel selection on one sm_100a GPU.
+ *
+ * The library evaluates, for every (GEMM problem p, candidate configuration c) pair, the
+ * statically computable hardware-aware feature map x = phi(p, c, h) of the paper's section
+ * "From CUTLASS Candidates to Hardware-Aware Features" (Table "Feature groups" and the
+ * sub-sections Structural Core, Work Decomposition and Wave Quantization, Memory Behavior,
+ * Resource Pressure and Occupancy, Pipeline Balance), scores x with a learned ranker
+ * f_theta (section "Learning to Rank Candidates": Model A, an additive tree ensemble, or
+ * Model B, a feed-forward ranker) and returns, per problem, the k best candidates -- the
+ * decision rule c^(p) = argmax_{c in C(p)} f_theta(x(p, c, h)) (Eq. "selection"), widened
+ * from the single argmax to a top-k shortlist.
+ *
+ * Conventions
+ *   - Every call returns a ks_status (KS_OK == 0). Nothing aborts, throws or prints.
+ *   - Pointers named d_* are DEVICE pointers on the context's CUDA device, h_* are HOST
+ *     pointers; the caller owns every data buffer, the library owns only ks_ctx / ks_model.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream). Batch
+ *     calls only enqueue work on that stream; they do not synchronise.
+ *   - A context is bound to one device and is not thread-safe: use one per host thread.
+ *   - All structs are plain little-endian PODs with exactly the fields shown.
+ */
+#ifndef KS_H_
+#define KS_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define KS_F 63          /* number of features (columns 0..62 of a feature row)            */
+#define KS_F_PAD 64      /* a feature row is 64 fp32; column 63 is always 0                */
+#define KS_MAX_K 32      /* largest k accepted by ks_select / ks_select_one                */
+#define KS_MAX_DEPTH 15  /* deepest tree accepted (a leaf index must fit 16 bits)          */
+#define KS_MAX_DIM (1u << 19) /* largest M, N or K for which all int64 products are exact  */
+#define KS_MLP_MAX_LAYERS 6
+#define KS_MLP_MAX_WIDTH 1024
+
+typedef int ks_status;
+enum {
+  KS_OK = 0,
+  KS_ERR_INVALID_ARG = 1, /* null pointer, size out of range, malformed model              */
+  KS_ERR_UNSUPPORTED = 2, /* valid request this build has no kernel for                    */
+  KS_ERR_CUDA = 3,        /* a CUDA runtime call failed; see ks_last_cuda_error            */
+  KS_ERR_TIMEOUT = 4,     /* a bounded device-side wait gave up (status word set)          */
+  KS_ERR_OOM = 5          /* device or host allocation failed                              */
+};
+
+/* GEMM instance p = (M, N, K, layout) (section "Problem and Candidate Sets"), extended with
+ * the operand / output types and the epilogue-fusion kind of the transfer studies. */
+typedef struct {
+  uint32_t m, n, k;   /* 1 .. KS_MAX_DIM                                                   */
+  uint8_t layout;     /* 0 TN, 1 TT, 2 NN, 3 NT (order of Table "Configuration knobs")     */
+  uint8_t dtype_ab;   /* 0 fp16, 1 bf16, 2 fp8_e4m3, 3 tf32                                */
+  uint8_t dtype_d;    /* 0 fp16, 1 bf16, 2 fp8_e4m3, 3 fp32                                */
+  uint8_t epi_flags;  /* bit0 bias; bits1-2 activation: 0 none, 1 ReLU, 2 GELU             */
+} ks_problem;         /* 16 bytes, 16-byte aligned in arrays                               */
+
+/* One CUTLASS configuration c (Table "Configuration knobs"). All extents >= 1. */
+typedef struct {
+  uint16_t tile_m, tile_n, tile_k; /* thread-block tile T_M x T_N x T_K                    */
+  uint16_t instr_n;                /* instruction tile N extent                            */
+  uint8_t stages;                  /* mainloop pipeline stages S                           */
+  uint8_t cluster_m, cluster_n;    /* cluster shape c_M x c_N                              */
+  uint8_t kernel_sched;            /* 0 WS, 1 Pingpong, 2 Cooperative, 3 TMA-basic         */
+  uint8_t epi_sched;               /* 0 NoSmem, 1 TMA, 2 TMA-Cooperative                   */
+  uint8_t tile_sched;              /* 0 Persistent, 1 Stream-K                             */
+  uint8_t instr_m, instr_k;        /* instruction tile M and K extents                     */
+} ks_candidate;                    /* 16 bytes, 16-byte aligned in arrays                  */
+
+/* Hardware descriptor h (section "Structural Core": SM count, shared-memory and register
+ * capacities, LLC capacity, memory bandwidth, compute-engine peak). Plain data: the values
+ * describe the target the candidates would run on, not the GPU libks itself runs on. */
+typedef struct {
+  uint32_t num_sms;            /* S_SM                                                     */
+  uint32_t smem_per_sm;        /* C_smem, bytes                                            */
+  uint32_t smem_per_cta_max;   /* largest footprint one CTA may request, bytes             */
+  uint32_t smem_reserved;      /* bytes added to every footprint                           */
+  uint32_t regs_per_sm;        /* C_reg, 32-bit registers                                  */
+  uint32_t max_threads_per_sm;
+  uint32_t max_ctas_per_sm;
+  uint32_t reserved0;          /* must be 0                                                */
+  uint64_t l2_bytes;           /* LLC capacity                                             */
+  uint64_t tma_bytes_per_us;   /* aggregate load bandwidth BW_TMA, bytes per microsecond   */
+  uint64_t tc_flops_per_us_per_sm[4]; /* per-SM tensor rate by dtype_ab, flop per us       */
+} ks_gpu_desc;                 /* 80 bytes                                                 */
+
+/* Interchange form of one tree node. Node 0 of a tree is its root. An internal node sends
+ * a row to `left` when x[feat] < thr (strict, fp32) and to `left + 1` otherwise; a leaf has
+ * feat == 0xFFFF and carries its value in thr_or_leaf. Indices are relative to the tree. */
+typedef struct {
+  float thr_or_leaf;
+  uint16_t feat;   /* 0 .. KS_F-1, or 0xFFFF for a leaf                                    */
+  uint16_t pad;    /* must be 0                                                            */
+  int32_t left;    /* index of the left child (right child = left + 1); 0 for a leaf       */
+} ks_node_host;    /* 12 bytes                                                             */
+
+typedef struct ks_ctx ks_ctx;
+typedef struct ks_model ks_model;
+
+/* ---- context ------------------------------------------------------------------------- */
+
+/* Create a context on CUDA device `cuda_device` for the target described by *desc (copied).
+ * Fails with KS_ERR_INVALID_ARG on a null pointer or a descriptor with a zero capacity or
+ * rate, KS_ERR_CUDA / KS_ERR_OOM if the device cannot be used. */
+ks_status ks_create(ks_ctx** out_ctx, int cuda_device, const ks_gpu_desc* desc);
+ks_status ks_destroy(ks_ctx* ctx);
+/* Text of the last CUDA error seen by this context ("" if none). Owned by the context. */
+const char* ks_last_cuda_error(const ks_ctx* ctx);
+
+/* ---- models -------------------------------------------------------------------------- */
+
+/* Model A (section "Model A (gradient-boosted ranker)"): f(x) = base_score + sum_m h_m(x).
+ * h_nodes holds the trees back to back, tree t in [h_tree_offsets[t], h_tree_offsets[t+1]).
+ * All structural validation happens here, on the host: feature ids < KS_F, children inside
+ * the tree and after their parent, finite thresholds and leaves, depth <= KS_MAX_DEPTH,
+ * every node reachable exactly once. The trees are repacked into a private device layout;
+ * the host arrays may be freed on return. Synchronous. */
+ks_status ks_model_create_gbdt(ks_ctx* ctx, int n_trees, const int64_t* h_tree_offsets,
+                               const ks_node_host* h_nodes, float base_score,
+                               ks_model** out_model);
+
+/* Model B (section "Model B (feed-forward ranker)") with the standardisation folded in:
+ * x'_j = (x_j - mu_j) / sigma_j for j < 63 with a non-finite x_j replaced by 0 first,
+ * x'_63 = 0, rounded to bf16; every hidden layer is h = ReLU(W h_prev + b) with fp32
+ * accumulation, rounded to bf16; the last layer (width 1) is s = w . h + b in fp32.
+ * h_widths = {64, w_1, ..., w_{L-1}, 1} (n_layers = L weight matrices, 2 <= L <=
+ * KS_MLP_MAX_LAYERS; hidden widths multiples of 64, <= KS_MLP_MAX_WIDTH). h_w_bf16[l] is
+ * row-major [out, in] bf16 bit patterns, h_bias[l] is [out] fp32; h_mu / h_sigma are [64]
+ * fp32 with sigma != 0. Synchronous. */
+ks_status ks_model_create_mlp(ks_ctx* ctx, int n_layers, const int* h_widths,
+                              const uint16_t* const* h_w_bf16, const float* const* h_bias,
+                              const float* h_mu, const float* h_sigma, ks_model** out_model);
+
+ks_status ks_model_destroy(ks_model* model);
+
+/* ---- the three calls of the selection path -------------------------------------------- */
+
+/* Candidate sets: with d_seg_offsets == NULL every problem is ranked against the whole pool
+ * d_c[0..C) (dense P x C; pairs = P*C, pair (i, j) is row i*C + j). Otherwise problem i is
+ * ranked against d_c[d_seg_index[j]] for j in [d_seg_offsets[i], d_seg_offsets[i+1])
+ * (d_seg_offsets has P+1 non-decreasing entries starting at 0; row j belongs to pair j). */
+
+/* x = phi(p, c, h) for every pair (Table "Feature groups"; the column list is
+ * ks_feature_name). Writes pairs x 64 fp32, row-major. `pairs` must equal P*C or
+ * seg_offsets[P] (the caller states it so that no device read is needed on the host). */
+ks_status ks_featurize(ks_ctx* ctx, const ks_problem* d_p, int P, const ks_candidate* d_c,
+                       int C, const int64_t* d_seg_offsets, const int32_t* d_seg_index,
+                       int64_t pairs, float* d_features, void* stream);
+
+/* s = f_theta(x) for `rows` feature rows (row-major [rows, 64] fp32). For a tree model,
+ * d_leaf_idx (nullable, [rows, n_trees] uint16) receives the tree-relative node index of
+ * the leaf each tree ends in. Must be NULL for an MLP. */
+ks_status ks_score(ks_ctx* ctx, const float* d_features, int64_t rows, const ks_model* model,
+                   float* d_scores, uint16_t* d_leaf_idx, void* stream);
+
+/* Fused featurize + score + per-problem top-k (Eq. "selection" as a shortlist): for problem
+ * i the k best pairs of its candidate set ordered by (score descending, pool index
+ * ascending). d_topk_idx [P, k] receives pool indices (-1 where the set has fewer than k
+ * members), d_topk_score [P, k] the scores (-inf there). 1 <= k <= KS_MAX_K. The feature
+ * matrix and the scores are never written to memory. `pairs` as in ks_featurize. */
+ks_status ks_select(ks_ctx* ctx, const ks_problem* d_p, int P, const ks_candidate* d_c, int C,
+                    const int64_t* d_seg_offsets, const int32_t* d_seg_index, int64_t pairs,
+                    const ks_model* model, int k, int32_t* d_topk_idx, float* d_topk_score,
+                    void* stream);
+
+/* Latency form of ks_select for one problem passed by value against the dense pool
+ * d_c[0..C): h_topk_idx / h_topk_score ([k], host memory, pinned for best latency) are
+ * valid when the call returns (it synchronises `stream`). */
+ks_status ks_select_one(ks_ctx* ctx, ks_problem p, const ks_candidate* d_c, int C,
+                        const ks_model* model, int k, int32_t* h_topk_idx,
+                        float* h_topk_score, void* stream);
+
+/* ks_select for callers whose inputs live in HOST memory: copies problems, candidates and
+ * segment arrays to the device, runs ks_select, copies the [P, k] results back and
+ * synchronises. Device staging comes from the context's workspace (grown on demand). */
+ks_status ks_select_host(ks_ctx* ctx, const ks_problem* h_p, int P, const ks_candidate* h_c,
+                         int C, const int64_t* h_seg_offsets, const int32_t* h_seg_index,
+                         int64_t pairs, const ks_model* model, int k, int32_t* h_topk_idx,
+                         float* h_topk_score, void* stream);
+
+/* ---- introspection -------------------------------------------------------------------- */
+
+const char* ks_status_string(ks_status s);
+int ks_feature_count(void);             /* KS_F                                            */
+const char* ks_feature_name(int index); /* NULL if index is outside 0..KS_F-1              */
+/* Number of kernels libks launched on behalf of this context since creation. */
+int64_t ks_launch_count(const ks_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KS_H_ */

@@ -1,0 +1,392 @@
+// ks_oracle.cpp -- plain CPU oracle of the execution-free selection path.
+//
+// TEST INFRASTRUCTURE, NOT PRODUCT CODE. Only the test-suite, the smoke check and the
+// benchmark's CPU-baseline leg may build, load or call this file. It shares no code, header
+// or table with the CUDA library: the record layouts below are re-declared here on purpose.
+//
+// What it is: the definitions of the paper written out one pair at a time -- scalar feature
+// formulas, a recursive tree walk, a scalar MLP, a full sort per problem. No blocking, no
+// fusion, no hoisting. Integer quantities are exact in int64; every float feature is a short
+// fixed sequence of individually rounded binary32 operations (build with
+// -O2 -ffp-contract=off on x86-64/SSE so that no FMA contraction or x87 excess precision
+// can change a bit).
+//
+// Pins (tests marked "not gpu"): hand-worked examples from the equations, the invariants the
+// equations imply (waves*SMs*b_eff >= tiles, eta in (0,1], T_K cancelling in the tile
+// intensity, f_fill*S == min(S, n_K), footprint linear in S ...), closed forms (square GEMM
+// intensity 2s/(3b)), brute-force nested-if evaluation of tiny ensembles, torch CPU linear
+// layers for the MLP, and numpy sorting for the top-k.
+// Parity unpinned (the paper names the quantity but prints no formula; the readings are this
+// build's own and are listed in the design notes): B_epi, T_block / n_consumer per schedule,
+// the register estimate behind b_reg, Q_epilogue, the cache-fraction, cluster-fit and
+// cluster-traffic columns.
+
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <limits>
+#include <vector>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+namespace {
+
+struct OProblem {
+  uint32_t m, n, k;
+  uint8_t layout, dtype_ab, dtype_d, epi_flags;
+};
+struct OCandidate {
+  uint16_t tile_m, tile_n, tile_k, instr_n;
+  uint8_t stages, cluster_m, cluster_n, kernel_sched, epi_sched, tile_sched, instr_m, instr_k;
+};
+struct OGpuDesc {
+  uint32_t num_sms, smem_per_sm, smem_per_cta_max, smem_reserved, regs_per_sm,
+      max_threads_per_sm, max_ctas_per_sm, reserved0;
+  uint64_t l2_bytes, tma_bytes_per_us, tc_flops_per_us_per_sm[4];
+};
+struct ONode {
+  float v;
+  uint16_t feat;
+  uint16_t pad;
+  int32_t left;
+};
+static_assert(sizeof(OProblem) == 16 && sizeof(OCandidate) == 16 && sizeof(OGpuDesc) == 80 &&
+                  sizeof(ONode) == 12,
+              "record layout");
+
+constexpr int NF = 63;   // features
+constexpr int ROW = 64;  // floats per feature row
+
+inline int64_t cdiv(int64_t a, int64_t b) { return (a + b - 1) / b; }
+// int64 -> binary32, round to nearest even (cvtsi2ss).
+inline float F(int64_t i) { return static_cast<float>(i); }
+
+// Section "Structural Core": log2 of a problem dimension.
+inline float log2_dim(uint32_t v) { return static_cast<float>(std::log2(static_cast<double>(v))); }
+
+// x = phi(p, c, h): Table "Feature groups", one column per quantity.
+void featurize_pair(const OProblem& p, const OCandidate& c, const OGpuDesc& h, float* x) {
+  static const int64_t kBytesAB[4] = {2, 2, 1, 4};  // fp16, bf16, fp8_e4m3, tf32
+  static const int64_t kBytesD[4] = {2, 2, 1, 4};   // fp16, bf16, fp8_e4m3, fp32
+  // (consumer warpgroups in the mainloop, threads per block) per kernel schedule:
+  // WS, Pingpong, Cooperative, TMA-basic.
+  static const int64_t kCons[4] = {1, 1, 2, 1};
+  static const int64_t kBlock[4] = {256, 384, 384, 128};
+
+  const int64_t M = p.m, N = p.n, K = p.k;
+  const int64_t bA = kBytesAB[p.dtype_ab & 3], bB = bA, bD = kBytesD[p.dtype_d & 3];
+  const int64_t TM = c.tile_m, TN = c.tile_n, TK = c.tile_k, S = c.stages;
+  const int64_t cM = c.cluster_m, cN = c.cluster_n;
+  const int ks = c.kernel_sched & 3;
+  const int64_t n_cons = kCons[ks], T_block = kBlock[ks];
+  const bool has_bias = (p.epi_flags & 1) != 0;
+  const int act = (p.epi_flags >> 1) & 3;
+
+  // ---- Structural core --------------------------------------------------------------
+  x[0] = log2_dim(p.m);
+  x[1] = log2_dim(p.n);
+  x[2] = log2_dim(p.k);
+  x[3] = F(p.layout == 2 || p.layout == 3);  // A column-major (NN, NT)
+  x[4] = F(p.layout == 1 || p.layout == 3);  // B row-major (TT, NT)
+  x[5] = F(p.dtype_ab);
+  x[6] = F(bA);
+  x[7] = F(bD);
+  x[8] = F(has_bias ? 1 : 0);
+  x[9] = F(act);
+  x[10] = F(TM);
+  x[11] = F(TN);
+  x[12] = F(TK);
+  x[13] = F(c.instr_m);
+  x[14] = F(c.instr_n);
+  x[15] = F(c.instr_k);
+  x[16] = F(S);
+  x[17] = F(c.kernel_sched);
+  x[18] = F(c.epi_sched);
+  x[19] = F(c.tile_sched);
+  x[20] = F(cM);
+  x[21] = F(cN);
+  x[22] = F(cM * cN);
+
+  // ---- Resource pressure and occupancy (needed first: b_res feeds the wave count) ------
+  const int64_t B_stage = TK * (TM * bA + TN * bB);  // B_stage = T_M T_K b_A + T_N T_K b_B
+  const int64_t smem_main = S * B_stage;
+  const int64_t E = (ks == 2) ? 128 : 64;
+  const int64_t B_epi =
+      (c.epi_sched == 0) ? 0 : 2 * std::min<int64_t>(TM, E) * std::min<int64_t>(TN, 32) * bD;
+  const int64_t both = smem_main + B_epi + h.smem_reserved;
+  // Warp-specialised (and the non-specialised basic) mainloop may overlap epilogue storage
+  // with the mainloop buffers; cooperative and ping-pong hold both at once.
+  const int64_t B_smem =
+      (ks == 0 || ks == 3) ? std::max(smem_main, B_epi) + h.smem_reserved : both;
+  const float f_smem = F(B_smem) / F(h.smem_per_sm);
+  const int64_t fits = both <= static_cast<int64_t>(h.smem_per_cta_max) ? 1 : 0;
+  const float r_proxy = F(TM * TN) / F(T_block);
+  const int64_t b_smem = static_cast<int64_t>(h.smem_per_sm) / B_smem;
+  const int64_t regs = std::min<int64_t>(255, 32 + cdiv(TM * TN, T_block));
+  const int64_t b_reg = static_cast<int64_t>(h.regs_per_sm) / (regs * T_block);
+  const int64_t b_arch = std::min<int64_t>(h.max_ctas_per_sm, h.max_threads_per_sm / T_block);
+  const int64_t b_res = std::min(b_smem, std::min(b_reg, b_arch));
+  const int64_t b_eff = std::max<int64_t>(1, b_res);
+
+  // ---- Work decomposition and wave quantisation -------------------------------------------
+  const int64_t n_m = cdiv(M, TM), n_n = cdiv(N, TN), n_k = cdiv(K, TK);
+  const int64_t n_tiles = n_m * n_n;
+  x[23] = F(n_m);
+  x[24] = F(n_n);
+  x[25] = F(n_k);
+  x[26] = F(n_tiles);
+  x[27] = F(n_m * TM - M) / F(M);  // w_M
+  x[28] = F(n_n * TN - N) / F(N);  // w_N
+  x[29] = F(n_tiles) / F(h.num_sms);
+  const int64_t resident = static_cast<int64_t>(h.num_sms) * b_eff;
+  const int64_t waves = cdiv(n_tiles, resident);  // q_SM
+  x[30] = F(waves);
+  const float eta = F(n_tiles) / F(waves * resident);  // eta_last
+  x[31] = eta;
+  x[32] = std::max(0.0f, 1.0f - eta);  // streamK_applicability
+  const int64_t n_c = cdiv(M, cM * TM) * cdiv(N, cN * TN);
+  x[33] = F(n_c * cM * cN - n_tiles) / F(n_tiles);
+  x[34] = F(n_m) / F(cM);
+  x[35] = F(n_n) / F(cN);
+  x[36] = F((cM > n_m || cN > n_n) ? 1 : 0);
+
+  // ---- Memory behaviour ---------------------------------------------------------------------
+  const int64_t bytesA = bA * M * K, bytesB = bB * K * N;
+  const int64_t Q_epi = bD * M * N + (has_bias ? bD * M : 0);
+  x[37] = F(2 * M * N * K) / F(bytesA + bytesB + Q_epi);  // I_problem
+  x[38] = F(2 * TM * TN) / F(TM * bA + TN * bB);          // I_mainloop
+  const int64_t restream = n_n * bytesA + n_m * bytesB;
+  x[39] = F(restream) / F(bytesA + bytesB);  // r_stream
+  x[40] = F(bytesA + bytesB) / F(static_cast<int64_t>(h.l2_bytes));
+  x[41] = F(bA * TM * K) / F(static_cast<int64_t>(h.l2_bytes));
+  x[42] = F(bB * TN * K) / F(static_cast<int64_t>(h.l2_bytes));
+  x[43] = F(restream);
+  x[44] = F(cdiv(n_n, cN) * bytesA + cdiv(n_m, cM) * bytesB);
+  x[45] = F(Q_epi);
+
+  // ---- Resource pressure columns ----------------------------------------------------------
+  x[46] = F(B_stage);
+  x[47] = F(smem_main);
+  x[48] = F(B_epi);
+  x[49] = F(B_smem);
+  x[50] = f_smem;
+  x[51] = F(fits);
+  x[52] = r_proxy;
+  x[53] = F(b_smem);
+  x[54] = F(b_reg);
+  x[55] = F(b_res);
+  x[56] = F(b_eff * T_block) / F(h.max_threads_per_sm);
+
+  // ---- Pipeline balance ---------------------------------------------------------------------
+  const float t_prod =
+      F(static_cast<int64_t>(h.num_sms) * B_stage) / F(static_cast<int64_t>(h.tma_bytes_per_us));
+  const float t_cons =
+      F(2 * TM * TN * TK) /
+      F(n_cons * static_cast<int64_t>(h.tc_flops_per_us_per_sm[p.dtype_ab & 3]));
+  x[57] = t_prod;
+  x[58] = t_cons;
+  x[59] = t_cons / t_prod;                // r_pc
+  x[60] = F(std::min(S, n_k)) / F(S);     // f_fill
+  x[61] = F(n_k) / F(S);                  // a_stage
+  x[62] = F(S) * f_smem;
+  x[63] = 0.0f;
+}
+
+// Model A: walk one tree from its root; returns the leaf's node index.
+int walk(const ONode* tree, int node, const float* x) {
+  const ONode& nd = tree[node];
+  if (nd.feat == 0xFFFF) return node;
+  return walk(tree, x[nd.feat] < nd.v ? nd.left : nd.left + 1, x);
+}
+
+float score_gbdt_row(const float* x, int n_trees, const int64_t* off, const ONode* nodes,
+                     float base, uint16_t* leaf_idx) {
+  double s = base;
+  for (int t = 0; t < n_trees; ++t) {
+    const ONode* tree = nodes + off[t];
+    const int leaf = walk(tree, 0, x);
+    if (leaf_idx) leaf_idx[t] = static_cast<uint16_t>(leaf);
+    s += static_cast<double>(tree[leaf].v);
+  }
+  return static_cast<float>(s);
+}
+
+inline float bf16_to_float(uint16_t b) {
+  uint32_t u = static_cast<uint32_t>(b) << 16;
+  float f;
+  std::memcpy(&f, &u, 4);
+  return f;
+}
+// binary32 -> bfloat16 value (as binary32), round to nearest even.
+inline float round_bf16(float f) {
+  uint32_t u;
+  std::memcpy(&u, &f, 4);
+  if ((u & 0x7F800000u) == 0x7F800000u) return f;  // inf / nan unchanged
+  u += 0x7FFFu + ((u >> 16) & 1u);
+  u &= 0xFFFF0000u;
+  std::memcpy(&f, &u, 4);
+  return f;
+}
+
+struct OMlp {
+  int n_layers;
+  const int* widths;  // n_layers + 1 entries
+  const uint16_t* const* w;
+  const float* const* b;
+  const float* mu;
+  const float* sigma;
+};
+
+// Model B with the standardisation folded in.
+float score_mlp_row(const float* x, const OMlp& m) {
+  std::vector<float> cur(ROW), nxt;
+  for (int j = 0; j < ROW; ++j) {
+    float v = 0.0f;
+    if (j < NF) {
+      v = x[j];
+      if (!std::isfinite(v)) v = 0.0f;
+      v = (v - m.mu[j]) / m.sigma[j];
+    }
+    cur[j] = round_bf16(v);
+  }
+  for (int l = 0; l < m.n_layers; ++l) {
+    const int in = m.widths[l], out = m.widths[l + 1];
+    const bool last = (l == m.n_layers - 1);
+    nxt.assign(out, 0.0f);
+    for (int o = 0; o < out; ++o) {
+      double acc = 0.0;
+      for (int i = 0; i < in; ++i)
+        acc += static_cast<double>(bf16_to_float(m.w[l][static_cast<size_t>(o) * in + i])) *
+               static_cast<double>(cur[i]);
+      float v = static_cast<float>(acc + static_cast<double>(m.b[l][o]));
+      if (!last) {
+        v = v > 0.0f ? v : 0.0f;
+        v = round_bf16(v);
+      }
+      nxt[o] = v;
+    }
+    cur.swap(nxt);
+  }
+  return cur[0];
+}
+
+// Per-problem ranking: full sort by (score descending, pool index ascending).
+void topk_segment(const float* scores, const int32_t* pool_idx, int64_t n, int k, int32_t* out_idx,
+                  float* out_score) {
+  std::vector<int64_t> order(n);
+  for (int64_t i = 0; i < n; ++i) order[i] = i;
+  std::stable_sort(order.begin(), order.end(), [&](int64_t a, int64_t b) {
+    if (scores[a] != scores[b]) return scores[a] > scores[b];
+    return pool_idx[a] < pool_idx[b];
+  });
+  for (int j = 0; j < k; ++j) {
+    if (j < n) {
+      out_idx[j] = pool_idx[order[j]];
+      out_score[j] = scores[order[j]];
+    } else {
+      out_idx[j] = -1;
+      out_score[j] = -std::numeric_limits<float>::infinity();
+    }
+  }
+}
+
+}  // namespace
+
+extern "C" {
+
+int orc_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+void orc_set_threads(int n) {
+#ifdef _OPENMP
+  if (n > 0) omp_set_num_threads(n);
+#else
+  (void)n;
+#endif
+}
+
+// Feature rows for every pair. seg_off == NULL: dense P x C, row i*C + j.
+void orc_featurize(const OProblem* p, int P, const OCandidate* c, int C, const int64_t* seg_off,
+                   const int32_t* seg_idx, const OGpuDesc* h, float* out) {
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int i = 0; i < P; ++i) {
+    const int64_t lo = seg_off ? seg_off[i] : static_cast<int64_t>(i) * C;
+    const int64_t hi = seg_off ? seg_off[i + 1] : lo + C;
+    for (int64_t r = lo; r < hi; ++r) {
+      const int64_t j = seg_off ? seg_idx[r] : r - lo;
+      featurize_pair(p[i], c[j], *h, out + r * ROW);
+    }
+  }
+}
+
+void orc_score_gbdt(const float* feat, int64_t rows, int n_trees, const int64_t* off,
+                    const ONode* nodes, float base, float* scores, uint16_t* leaf_idx) {
+#pragma omp parallel for schedule(static)
+  for (int64_t r = 0; r < rows; ++r)
+    scores[r] = score_gbdt_row(feat + r * ROW, n_trees, off, nodes, base,
+                               leaf_idx ? leaf_idx + r * n_trees : nullptr);
+}
+
+void orc_score_mlp(const float* feat, int64_t rows, int n_layers, const int* widths,
+                   const uint16_t* const* w, const float* const* b, const float* mu,
+                   const float* sigma, float* scores) {
+  const OMlp m{n_layers, widths, w, b, mu, sigma};
+#pragma omp parallel for schedule(static)
+  for (int64_t r = 0; r < rows; ++r) scores[r] = score_mlp_row(feat + r * ROW, m);
+}
+
+// Ranking of given scores. seg_off == NULL: dense, `rows_per_problem` scores per problem and
+// the pool index of row j is j; else segment rows carry pool indices seg_idx.
+void orc_topk(const float* scores, int P, int64_t rows_per_problem, const int64_t* seg_off,
+              const int32_t* seg_idx, int k, int32_t* out_idx, float* out_score) {
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int i = 0; i < P; ++i) {
+    const int64_t lo = seg_off ? seg_off[i] : static_cast<int64_t>(i) * rows_per_problem;
+    const int64_t hi = seg_off ? seg_off[i + 1] : lo + rows_per_problem;
+    std::vector<int32_t> idx(hi - lo);
+    for (int64_t r = lo; r < hi; ++r) idx[r - lo] = seg_off ? seg_idx[r] : static_cast<int32_t>(r - lo);
+    topk_segment(scores + lo, idx.data(), hi - lo, k, out_idx + static_cast<int64_t>(i) * k,
+                 out_score + static_cast<int64_t>(i) * k);
+  }
+}
+
+// The whole path, one problem at a time: featurize every pair of the problem, score it,
+// sort the segment. model_kind 0 = tree ensemble, 1 = MLP. all_scores (nullable) receives
+// the score of every pair, in row order.
+void orc_select(const OProblem* p, int P, const OCandidate* c, int C, const int64_t* seg_off,
+                const int32_t* seg_idx, const OGpuDesc* h, int model_kind, int n_trees,
+                const int64_t* off, const ONode* nodes, float base, int n_layers,
+                const int* widths, const uint16_t* const* w, const float* const* b,
+                const float* mu, const float* sigma, int k, int32_t* out_idx, float* out_score,
+                float* all_scores) {
+  const OMlp m{n_layers, widths, w, b, mu, sigma};
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int i = 0; i < P; ++i) {
+    const int64_t lo = seg_off ? seg_off[i] : static_cast<int64_t>(i) * C;
+    const int64_t hi = seg_off ? seg_off[i + 1] : lo + C;
+    const int64_t n = hi - lo;
+    std::vector<float> sc(n);
+    std::vector<int32_t> idx(n);
+    float x[ROW];
+    for (int64_t r = 0; r < n; ++r) {
+      const int32_t j = seg_off ? seg_idx[lo + r] : static_cast<int32_t>(r);
+      idx[r] = j;
+      featurize_pair(p[i], c[j], *h, x);
+      sc[r] = model_kind == 0 ? score_gbdt_row(x, n_trees, off, nodes, base, nullptr)
+                              : score_mlp_row(x, m);
+      if (all_scores) all_scores[lo + r] = sc[r];
+    }
+    topk_segment(sc.data(), idx.data(), n, k, out_idx + static_cast<int64_t>(i) * k,
+                 out_score + static_cast<int64_t>(i) * k);
+  }
+}
+
+}  // extern "C"
