@@ -1,0 +1,254 @@
+"""ctypes binding of libks (the C ABI declared in include/ks.h).
+
+Argument marshalling only: every step of the selection path runs inside the library's CUDA
+kernels. torch supplies device memory (`tensor.data_ptr()`) and the current stream. There is
+no CPU fallback: importing this module without the built library raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libks.so")
+
+KS_F, KS_F_PAD, KS_MAX_K, KS_MAX_DEPTH = 63, 64, 32, 15
+KS_OK, KS_ERR_INVALID_ARG, KS_ERR_UNSUPPORTED, KS_ERR_CUDA, KS_ERR_TIMEOUT, KS_ERR_OOM = range(6)
+
+EXPORTS = ("ks_create", "ks_destroy", "ks_last_cuda_error", "ks_model_create_gbdt",
+           "ks_model_create_mlp", "ks_model_destroy", "ks_featurize", "ks_score", "ks_select",
+           "ks_select_one", "ks_select_host", "ks_status_string", "ks_feature_count",
+           "ks_feature_name", "ks_launch_count")
+
+
+class KsError(RuntimeError):
+    def __init__(self, status: int, where: str, detail: str = ""):
+        self.status = status
+        msg = f"{where}: {_status_string(status)}"
+        super().__init__(msg + (f" ({detail})" if detail else ""))
+
+
+class _Problem(ctypes.Structure):
+    _fields_ = [("m", ctypes.c_uint32), ("n", ctypes.c_uint32), ("k", ctypes.c_uint32),
+                ("layout", ctypes.c_uint8), ("dtype_ab", ctypes.c_uint8),
+                ("dtype_d", ctypes.c_uint8), ("epi_flags", ctypes.c_uint8)]
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is not built; run `python -c 'import __graft_entry__ as g; "
+                          "g.build()'` (nvcc, sm_100a). There is no fallback path.")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64
+    lib.ks_create.argtypes = [ctypes.POINTER(vp), i32, vp]
+    lib.ks_destroy.argtypes = [vp]
+    lib.ks_last_cuda_error.argtypes = [vp]
+    lib.ks_last_cuda_error.restype = ctypes.c_char_p
+    lib.ks_model_create_gbdt.argtypes = [vp, i32, vp, vp, ctypes.c_float, ctypes.POINTER(vp)]
+    lib.ks_model_create_mlp.argtypes = [vp, i32, vp, vp, vp, vp, vp, ctypes.POINTER(vp)]
+    lib.ks_model_destroy.argtypes = [vp]
+    lib.ks_featurize.argtypes = [vp, vp, i32, vp, i32, vp, vp, i64, vp, vp]
+    lib.ks_score.argtypes = [vp, vp, i64, vp, vp, vp, vp]
+    lib.ks_select.argtypes = [vp, vp, i32, vp, i32, vp, vp, i64, vp, i32, vp, vp, vp]
+    lib.ks_select_one.argtypes = [vp, _Problem, vp, i32, vp, i32, vp, vp, vp]
+    lib.ks_select_host.argtypes = [vp, vp, i32, vp, i32, vp, vp, i64, vp, i32, vp, vp, vp]
+    lib.ks_status_string.argtypes = [i32]
+    lib.ks_status_string.restype = ctypes.c_char_p
+    lib.ks_feature_count.restype = i32
+    lib.ks_feature_name.argtypes = [i32]
+    lib.ks_feature_name.restype = ctypes.c_char_p
+    lib.ks_launch_count.argtypes = [vp]
+    lib.ks_launch_count.restype = i64
+    for name in EXPORTS:
+        fn = getattr(lib, name)
+        if fn.restype is ctypes.c_int and name not in ("ks_feature_count",):
+            fn.restype = ctypes.c_int
+    return lib
+
+
+_lib = _load()
+
+
+def _status_string(s: int) -> str:
+    return _lib.ks_status_string(int(s)).decode()
+
+
+def ks_feature_count() -> int:
+    return int(_lib.ks_feature_count())
+
+
+def ks_feature_name(i: int):
+    s = _lib.ks_feature_name(int(i))
+    return None if s is None else s.decode()
+
+
+def _dptr(t):
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous CUDA tensor")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _hptr(a):
+    if a is None:
+        return None
+    if isinstance(a, torch.Tensor):
+        if a.is_cuda or not a.is_contiguous():
+            raise ValueError("expected a contiguous host tensor")
+        return ctypes.c_void_p(a.data_ptr())
+    if not a.flags["C_CONTIGUOUS"]:
+        raise ValueError("expected a C-contiguous array")
+    return ctypes.c_void_p(a.ctypes.data)
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def to_device(records: np.ndarray, device) -> torch.Tensor:
+    """A numpy record / plain array as a device tensor of raw bytes (records) or values."""
+    a = np.ascontiguousarray(records)
+    if a.dtype.fields is not None:
+        a = a.view(np.uint8).reshape(len(records), -1)
+    return torch.from_numpy(a.copy()).to(device)
+
+
+class Model:
+    def __init__(self, ctx: "Context", handle: ctypes.c_void_p, kind: str, n_trees: int = 0):
+        self.ctx, self._h, self.kind, self.n_trees = ctx, handle, kind, n_trees
+
+    def close(self):
+        if self._h:
+            _lib.ks_model_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class Context:
+    """ks_ctx plus thin methods named after the C entry points."""
+
+    def __init__(self, desc: np.ndarray, device: int = 0):
+        d = np.ascontiguousarray(desc)
+        if d.nbytes != 80:
+            raise ValueError("gpu descriptor must be 80 bytes")
+        self.device = torch.device("cuda", device)
+        h = ctypes.c_void_p()
+        st = _lib.ks_create(ctypes.byref(h), device, _hptr(d.reshape(1)))
+        if st != KS_OK:
+            raise KsError(st, "ks_create")
+        self._h = h
+
+    def close(self):
+        if self._h:
+            _lib.ks_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, st: int, where: str):
+        if st != KS_OK:
+            raise KsError(st, where, _lib.ks_last_cuda_error(self._h).decode())
+
+    def launch_count(self) -> int:
+        return int(_lib.ks_launch_count(self._h))
+
+    # ---- models ---------------------------------------------------------------------------
+    def model_create_gbdt(self, tree_offsets, nodes, base_score: float = 0.0) -> Model:
+        off = np.ascontiguousarray(tree_offsets, dtype=np.int64)
+        nd = np.ascontiguousarray(nodes)
+        if nd.dtype.itemsize != 12:
+            raise ValueError("nodes must be 12-byte records")
+        h = ctypes.c_void_p()
+        st = _lib.ks_model_create_gbdt(self._h, len(off) - 1, _hptr(off), _hptr(nd),
+                                       ctypes.c_float(base_score), ctypes.byref(h))
+        self._check(st, "ks_model_create_gbdt")
+        return Model(self, h, "gbdt", len(off) - 1)
+
+    def model_create_mlp(self, mlp: dict) -> Model:
+        widths = np.ascontiguousarray(mlp["widths"], dtype=np.int32)
+        L = len(widths) - 1
+        ws = [np.ascontiguousarray(w, dtype=np.uint16) for w in mlp["weights"]]
+        bs = [np.ascontiguousarray(b, dtype=np.float32) for b in mlp["biases"]]
+        mu = np.ascontiguousarray(mlp["mu"], dtype=np.float32)
+        sigma = np.ascontiguousarray(mlp["sigma"], dtype=np.float32)
+        wp = (ctypes.c_void_p * L)(*[w.ctypes.data for w in ws])
+        bp = (ctypes.c_void_p * L)(*[b.ctypes.data for b in bs])
+        h = ctypes.c_void_p()
+        st = _lib.ks_model_create_mlp(self._h, L, _hptr(widths), ctypes.cast(wp, ctypes.c_void_p),
+                                      ctypes.cast(bp, ctypes.c_void_p), _hptr(mu), _hptr(sigma),
+                                      ctypes.byref(h))
+        self._check(st, "ks_model_create_mlp")
+        return Model(self, h, "mlp")
+
+    # ---- the path -------------------------------------------------------------------------
+    @staticmethod
+    def _pairs(P, C, seg_off_pairs):
+        return P * C if seg_off_pairs is None else int(seg_off_pairs)
+
+    def featurize(self, d_p, P, d_c, C, d_seg_off=None, d_seg_idx=None, pairs=None, out=None):
+        pairs = P * C if pairs is None else pairs
+        if out is None:
+            out = torch.empty((pairs, KS_F_PAD), dtype=torch.float32, device=self.device)
+        st = _lib.ks_featurize(self._h, _dptr(d_p), P, _dptr(d_c), C, _dptr(d_seg_off),
+                               _dptr(d_seg_idx), pairs, _dptr(out), _stream())
+        self._check(st, "ks_featurize")
+        return out
+
+    def score(self, d_features, model: Model, want_leaf_idx: bool = False):
+        rows = d_features.shape[0]
+        scores = torch.empty(rows, dtype=torch.float32, device=self.device)
+        leaf = (torch.empty((rows, model.n_trees), dtype=torch.uint16, device=self.device)
+                if want_leaf_idx else None)
+        st = _lib.ks_score(self._h, _dptr(d_features), rows, model._h, _dptr(scores), _dptr(leaf),
+                           _stream())
+        self._check(st, "ks_score")
+        return (scores, leaf) if want_leaf_idx else scores
+
+    def select(self, d_p, P, d_c, C, model: Model, k, d_seg_off=None, d_seg_idx=None, pairs=None,
+               out_idx=None, out_score=None):
+        pairs = P * C if pairs is None else pairs
+        if out_idx is None:
+            kk = max(int(k), 1)  # an invalid k is reported by the library, not by torch
+            out_idx = torch.empty((P, kk), dtype=torch.int32, device=self.device)
+            out_score = torch.empty((P, kk), dtype=torch.float32, device=self.device)
+        st = _lib.ks_select(self._h, _dptr(d_p), P, _dptr(d_c), C, _dptr(d_seg_off), _dptr(d_seg_idx),
+                            pairs, model._h, k, _dptr(out_idx), _dptr(out_score), _stream())
+        self._check(st, "ks_select")
+        return out_idx, out_score
+
+    def select_one(self, problem: np.ndarray, d_c, C, model: Model, k, h_idx=None, h_score=None):
+        r = np.ascontiguousarray(problem).reshape(-1)[0]
+        p = _Problem(int(r["m"]), int(r["n"]), int(r["k"]), int(r["layout"]), int(r["dtype_ab"]),
+                     int(r["dtype_d"]), int(r["epi_flags"]))
+        if h_idx is None:
+            h_idx = torch.empty(k, dtype=torch.int32).pin_memory()
+            h_score = torch.empty(k, dtype=torch.float32).pin_memory()
+        st = _lib.ks_select_one(self._h, p, _dptr(d_c), C, model._h, k, _hptr(h_idx), _hptr(h_score),
+                                _stream())
+        self._check(st, "ks_select_one")
+        return h_idx, h_score
+
+    def select_host(self, h_p, P, h_c, C, model: Model, k, h_seg_off=None, h_seg_idx=None, pairs=None,
+                    h_idx=None, h_score=None):
+        pairs = P * C if pairs is None else pairs
+        if h_idx is None:
+            h_idx = torch.empty((P, k), dtype=torch.int32).pin_memory()
+            h_score = torch.empty((P, k), dtype=torch.float32).pin_memory()
+        st = _lib.ks_select_host(self._h, _hptr(h_p), P, _hptr(h_c), C, _hptr(h_seg_off),
+                                 _hptr(h_seg_idx), pairs, model._h, k, _hptr(h_idx), _hptr(h_score),
+                                 _stream())
+        self._check(st, "ks_select_host")
+        return h_idx, h_score

@@ -1,0 +1,413 @@
+// Host side of the C ABI: argument checks, model validation and repacking, workspace
+// management, launches. No exception or abort crosses the boundary.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "ks_internal.h"
+
+namespace {
+
+const char* const kFeatureNames[KS_F] = {
+    "log2_m", "log2_n", "log2_k", "a_col_major", "b_row_major", "dtype_code", "bytes_in",
+    "bytes_out", "has_bias", "act_code", "tile_m", "tile_n", "tile_k", "instr_m", "instr_n",
+    "instr_k", "stages", "kernel_sched", "epi_sched", "uses_streamk", "cluster_m", "cluster_n",
+    "cluster_size", "n_m", "n_n", "n_k", "n_tiles", "w_m", "w_n", "sm_subscription", "waves",
+    "eta_last", "streamk_applicability", "cluster_pad_waste", "tiles_per_cluster_m",
+    "tiles_per_cluster_n", "cluster_overshoot", "i_problem", "i_mainloop", "r_stream",
+    "ws_frac_l2", "panel_a_frac_l2", "panel_b_frac_l2", "traffic_in", "traffic_in_cluster",
+    "traffic_epi", "bytes_per_stage", "smem_mainloop", "smem_epi", "smem_total", "f_smem",
+    "fits_smem", "r_proxy", "b_smem", "b_reg", "b_res", "occupancy", "t_producer_us",
+    "t_consumer_us", "r_pc", "f_fill", "a_stage", "stages_x_fsmem"};
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) prev = -1;
+    if (prev != dev) ok = cudaSetDevice(dev) == cudaSuccess;
+  }
+  ~DeviceGuard() {
+    int cur = -1;
+    if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+  }
+};
+
+ks_status cuda_fail(ks_ctx* ctx, cudaError_t e, const char* what) {
+  if (ctx) std::snprintf(ctx->err, sizeof(ctx->err), "%s: %s", what, cudaGetErrorString(e));
+  cudaGetLastError();  // clear the sticky-free error state
+  return e == cudaErrorMemoryAllocation ? KS_ERR_OOM : KS_ERR_CUDA;
+}
+
+ks_status ensure_workspace(ks_ctx* ctx, size_t bytes) {
+  if (bytes <= ctx->ws_bytes) return KS_OK;
+  if (ctx->ws) {
+    cudaError_t e = cudaFree(ctx->ws);  // synchronises: nothing in flight still uses it
+    ctx->ws = nullptr;
+    ctx->ws_bytes = 0;
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaFree(workspace)");
+  }
+  const size_t want = bytes + bytes / 2 + (1u << 20);
+  cudaError_t e = cudaMalloc(&ctx->ws, want);
+  if (e != cudaSuccess) {
+    ctx->ws = nullptr;
+    return cuda_fail(ctx, e, "cudaMalloc(workspace)");
+  }
+  ctx->ws_bytes = want;
+  return KS_OK;
+}
+
+inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
+
+template <typename T>
+cudaError_t upload(T** dst, const T* src, size_t n) {
+  *dst = nullptr;
+  if (n == 0) return cudaSuccess;
+  cudaError_t e = cudaMalloc(reinterpret_cast<void**>(dst), n * sizeof(T));
+  if (e != cudaSuccess) return e;
+  return cudaMemcpy(*dst, src, n * sizeof(T), cudaMemcpyHostToDevice);
+}
+
+bool valid_desc(const ks_gpu_desc& d) {
+  if (!d.num_sms || !d.smem_per_sm || !d.smem_per_cta_max || !d.regs_per_sm || !d.max_threads_per_sm ||
+      !d.max_ctas_per_sm || !d.l2_bytes || !d.tma_bytes_per_us || d.reserved0)
+    return false;
+  if (d.max_threads_per_sm < 384) return false;
+  for (int i = 0; i < 4; ++i)
+    if (!d.tc_flops_per_us_per_sm[i]) return false;
+  return true;
+}
+
+// Checks one tree; returns its depth or -1.
+int validate_tree(const ks_node_host* t, int64_t n) {
+  if (n < 1 || n > 65535) return -1;
+  std::vector<int> depth(n, -1);
+  depth[0] = 0;
+  int max_depth = 0;
+  int64_t reached = 1;
+  for (int64_t i = 0; i < n; ++i) {
+    const ks_node_host& nd = t[i];
+    if (depth[i] < 0) return -1;  // parents precede children, so an unreached node is an orphan
+    if (!std::isfinite(nd.thr_or_leaf)) return -1;
+    if (nd.feat == 0xFFFF) continue;
+    if (nd.feat >= KS_F) return -1;
+    const int64_t l = nd.left;
+    if (l <= i || l + 1 >= n) return -1;
+    if (depth[l] >= 0 || depth[l + 1] >= 0) return -1;  // a node has exactly one parent
+    depth[l] = depth[l + 1] = depth[i] + 1;
+    reached += 2;
+    if (depth[i] + 1 > max_depth) max_depth = depth[i] + 1;
+  }
+  if (reached != n || max_depth > KS_MAX_DEPTH) return -1;
+  return max_depth;
+}
+
+void free_model(ks_model* m) {
+  if (!m) return;
+  DeviceGuard g(m->ctx->device);
+  cudaFree(m->gbdt.d_nodes);
+  cudaFree(m->gbdt.d_roots);
+  cudaFree(m->gbdt.d_qnodes);
+  cudaFree(m->gbdt.d_qleaves);
+  cudaFree(m->gbdt.d_qleaf_node);
+  cudaFree(m->gbdt.d_qthr);
+  cudaFree(m->gbdt.d_qrow_feat);
+  cudaFree(m->gbdt.d_qrow_count);
+  for (int l = 0; l < KS_MLP_MAX_LAYERS; ++l) {
+    cudaFree(m->mlp.d_w[l]);
+    cudaFree(m->mlp.d_b[l]);
+  }
+  cudaFree(m->mlp.d_mu);
+  cudaFree(m->mlp.d_sigma);
+  delete m;
+}
+
+ks_status check_pairs(int P, int C, const void* seg_off, const void* seg_idx, int64_t pairs) {
+  if (P < 0 || C < 0 || pairs < 0) return KS_ERR_INVALID_ARG;
+  if ((seg_off == nullptr) != (seg_idx == nullptr) && pairs > 0) return KS_ERR_INVALID_ARG;
+  if (!seg_off && pairs != static_cast<int64_t>(P) * C) return KS_ERR_INVALID_ARG;
+  return KS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* ks_status_string(ks_status s) {
+  switch (s) {
+    case KS_OK: return "ok";
+    case KS_ERR_INVALID_ARG: return "invalid argument";
+    case KS_ERR_UNSUPPORTED: return "unsupported";
+    case KS_ERR_CUDA: return "CUDA error";
+    case KS_ERR_TIMEOUT: return "device-side wait timed out";
+    case KS_ERR_OOM: return "out of memory";
+    default: return "unknown status";
+  }
+}
+
+int ks_feature_count(void) { return KS_F; }
+
+const char* ks_feature_name(int index) {
+  return (index >= 0 && index < KS_F) ? kFeatureNames[index] : nullptr;
+}
+
+ks_status ks_create(ks_ctx** out_ctx, int cuda_device, const ks_gpu_desc* desc) {
+  if (!out_ctx) return KS_ERR_INVALID_ARG;
+  *out_ctx = nullptr;
+  if (!desc || !valid_desc(*desc)) return KS_ERR_INVALID_ARG;
+  int n_dev = 0;
+  if (cudaGetDeviceCount(&n_dev) != cudaSuccess) {
+    cudaGetLastError();
+    return KS_ERR_CUDA;
+  }
+  if (cuda_device < 0 || cuda_device >= n_dev) return KS_ERR_INVALID_ARG;
+  DeviceGuard g(cuda_device);
+  if (!g.ok) return KS_ERR_CUDA;
+  ks_ctx* ctx = new (std::nothrow) ks_ctx();
+  if (!ctx) return KS_ERR_OOM;
+  ctx->device = cuda_device;
+  ctx->desc = *desc;
+  ctx->pinned_bytes = KS_MAX_K * (sizeof(int32_t) + sizeof(float));
+  if (cudaMallocHost(&ctx->pinned, ctx->pinned_bytes) != cudaSuccess) {
+    cudaGetLastError();
+    delete ctx;
+    return KS_ERR_OOM;
+  }
+  ks_status s = ensure_workspace(ctx, 1u << 20);
+  if (s != KS_OK) {
+    cudaFreeHost(ctx->pinned);
+    delete ctx;
+    return s;
+  }
+  *out_ctx = ctx;
+  return KS_OK;
+}
+
+ks_status ks_destroy(ks_ctx* ctx) {
+  if (!ctx) return KS_OK;
+  DeviceGuard g(ctx->device);
+  cudaFree(ctx->ws);
+  cudaFreeHost(ctx->pinned);
+  delete ctx;
+  return KS_OK;
+}
+
+const char* ks_last_cuda_error(const ks_ctx* ctx) { return ctx ? ctx->err : ""; }
+
+int64_t ks_launch_count(const ks_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+ks_status ks_model_create_gbdt(ks_ctx* ctx, int n_trees, const int64_t* h_tree_offsets,
+                               const ks_node_host* h_nodes, float base_score, ks_model** out_model) {
+  if (!out_model) return KS_ERR_INVALID_ARG;
+  *out_model = nullptr;
+  if (!ctx || n_trees < 0 || !h_tree_offsets || (n_trees > 0 && !h_nodes) || !std::isfinite(base_score))
+    return KS_ERR_INVALID_ARG;
+  if (h_tree_offsets[0] != 0) return KS_ERR_INVALID_ARG;
+  const int64_t total = h_tree_offsets[n_trees];
+  if (total < 0 || total > (1ll << 31) - 1) return KS_ERR_INVALID_ARG;
+  int max_depth = 0;
+  for (int t = 0; t < n_trees; ++t) {
+    const int64_t lo = h_tree_offsets[t], hi = h_tree_offsets[t + 1];
+    if (hi <= lo) return KS_ERR_INVALID_ARG;
+    const int d = validate_tree(h_nodes + lo, hi - lo);
+    if (d < 0) return KS_ERR_INVALID_ARG;
+    if (d > max_depth) max_depth = d;
+  }
+  std::vector<ks::DevNode> dev(static_cast<size_t>(total));
+  for (int64_t i = 0; i < total; ++i) {
+    dev[i].v = h_nodes[i].thr_or_leaf;
+    dev[i].feat = h_nodes[i].feat;
+    dev[i].left = h_nodes[i].feat == 0xFFFF ? 0 : static_cast<uint16_t>(h_nodes[i].left);
+  }
+  std::vector<int> roots(n_trees + 1);
+  for (int t = 0; t <= n_trees; ++t) roots[t] = static_cast<int>(h_tree_offsets[t]);
+
+  DeviceGuard g(ctx->device);
+  ks_model* m = new (std::nothrow) ks_model();
+  if (!m) return KS_ERR_OOM;
+  m->ctx = ctx;
+  m->kind = 0;
+  m->gbdt.n_trees = n_trees;
+  m->gbdt.max_depth = max_depth;
+  m->gbdt.n_nodes = total;
+  m->gbdt.base = base_score;
+  cudaError_t e = upload(&m->gbdt.d_nodes, dev.data(), dev.size());
+  if (e == cudaSuccess) e = upload(&m->gbdt.d_roots, roots.data(), roots.size());
+  if (e == cudaSuccess) e = ks::build_fast_gbdt(m->gbdt, n_trees, h_tree_offsets, h_nodes);
+  if (e != cudaSuccess) {
+    ks_status s = cuda_fail(ctx, e, "ks_model_create_gbdt");
+    free_model(m);
+    return s;
+  }
+  *out_model = m;
+  return KS_OK;
+}
+
+ks_status ks_model_create_mlp(ks_ctx* ctx, int n_layers, const int* h_widths,
+                              const uint16_t* const* h_w_bf16, const float* const* h_bias,
+                              const float* h_mu, const float* h_sigma, ks_model** out_model) {
+  if (!out_model) return KS_ERR_INVALID_ARG;
+  *out_model = nullptr;
+  if (!ctx || !h_widths || !h_w_bf16 || !h_bias || !h_mu || !h_sigma) return KS_ERR_INVALID_ARG;
+  if (n_layers < 2 || n_layers > KS_MLP_MAX_LAYERS) return KS_ERR_INVALID_ARG;
+  if (h_widths[0] != KS_F_PAD || h_widths[n_layers] != 1) return KS_ERR_INVALID_ARG;
+  int max_width = KS_F_PAD;
+  for (int l = 1; l < n_layers; ++l) {
+    if (h_widths[l] < 64 || h_widths[l] > KS_MLP_MAX_WIDTH || h_widths[l] % 64) return KS_ERR_INVALID_ARG;
+    if (h_widths[l] > max_width) max_width = h_widths[l];
+  }
+  for (int l = 0; l < n_layers; ++l)
+    if (!h_w_bf16[l] || !h_bias[l]) return KS_ERR_INVALID_ARG;
+  for (int j = 0; j < KS_F_PAD; ++j)
+    if (!std::isfinite(h_mu[j]) || !std::isfinite(h_sigma[j]) || h_sigma[j] == 0.0f) return KS_ERR_INVALID_ARG;
+
+  DeviceGuard g(ctx->device);
+  ks_model* m = new (std::nothrow) ks_model();
+  if (!m) return KS_ERR_OOM;
+  m->ctx = ctx;
+  m->kind = 1;
+  m->mlp.n_layers = n_layers;
+  m->mlp.max_width = max_width;
+  for (int l = 0; l <= n_layers; ++l) m->mlp.widths[l] = h_widths[l];
+  cudaError_t e = cudaSuccess;
+  for (int l = 0; l < n_layers && e == cudaSuccess; ++l) {
+    const size_t n = static_cast<size_t>(h_widths[l]) * h_widths[l + 1];
+    e = upload(&m->mlp.d_w[l], h_w_bf16[l], n);
+    if (e == cudaSuccess) e = upload(&m->mlp.d_b[l], h_bias[l], static_cast<size_t>(h_widths[l + 1]));
+  }
+  if (e == cudaSuccess) e = upload(&m->mlp.d_mu, h_mu, static_cast<size_t>(KS_F_PAD));
+  if (e == cudaSuccess) e = upload(&m->mlp.d_sigma, h_sigma, static_cast<size_t>(KS_F_PAD));
+  if (e != cudaSuccess) {
+    ks_status s = cuda_fail(ctx, e, "ks_model_create_mlp");
+    free_model(m);
+    return s;
+  }
+  *out_model = m;
+  return KS_OK;
+}
+
+ks_status ks_model_destroy(ks_model* model) {
+  free_model(model);
+  return KS_OK;
+}
+
+ks_status ks_featurize(ks_ctx* ctx, const ks_problem* d_p, int P, const ks_candidate* d_c, int C,
+                       const int64_t* d_seg_offsets, const int32_t* d_seg_index, int64_t pairs,
+                       float* d_features, void* stream) {
+  if (!ctx) return KS_ERR_INVALID_ARG;
+  ks_status s = check_pairs(P, C, d_seg_offsets, d_seg_index, pairs);
+  if (s != KS_OK) return s;
+  if (pairs == 0) return KS_OK;
+  if (!d_p || !d_c || !d_features) return KS_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  cudaError_t e = ks::launch_featurize(ctx->desc, d_p, P, d_c, C, d_seg_offsets, d_seg_index, pairs,
+                                       d_features, static_cast<cudaStream_t>(stream), &ctx->launches);
+  return e == cudaSuccess ? KS_OK : cuda_fail(ctx, e, "ks_featurize");
+}
+
+ks_status ks_score(ks_ctx* ctx, const float* d_features, int64_t rows, const ks_model* model,
+                   float* d_scores, uint16_t* d_leaf_idx, void* stream) {
+  if (!ctx || !model || model->ctx != ctx || rows < 0) return KS_ERR_INVALID_ARG;
+  if (rows == 0) return KS_OK;
+  if (!d_features || !d_scores) return KS_ERR_INVALID_ARG;
+  if (model->kind == 1 && d_leaf_idx) return KS_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  cudaError_t e =
+      model->kind == 0
+          ? ks::launch_score_gbdt(model->gbdt, d_features, rows, d_scores, d_leaf_idx,
+                                  static_cast<cudaStream_t>(stream), &ctx->launches)
+          : ks::launch_score_mlp(model->mlp, d_features, rows, d_scores,
+                                 static_cast<cudaStream_t>(stream), &ctx->launches);
+  return e == cudaSuccess ? KS_OK : cuda_fail(ctx, e, "ks_score");
+}
+
+ks_status ks_select(ks_ctx* ctx, const ks_problem* d_p, int P, const ks_candidate* d_c, int C,
+                    const int64_t* d_seg_offsets, const int32_t* d_seg_index, int64_t pairs,
+                    const ks_model* model, int k, int32_t* d_topk_idx, float* d_topk_score,
+                    void* stream) {
+  if (!ctx || !model || model->ctx != ctx || k < 1 || k > KS_MAX_K) return KS_ERR_INVALID_ARG;
+  ks_status s = check_pairs(P, C, d_seg_offsets, d_seg_index, pairs);
+  if (s != KS_OK) return s;
+  if (P == 0) return KS_OK;
+  if (!d_p || !d_topk_idx || !d_topk_score || (pairs > 0 && !d_c)) return KS_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  s = ensure_workspace(ctx, ks::select_partial_bytes(*model, P, C, pairs, d_seg_offsets != nullptr, k));
+  if (s != KS_OK) return s;
+  cudaError_t e = ks::launch_select(ctx->desc, *model, d_p, nullptr, P, d_c, C, d_seg_offsets,
+                                    d_seg_index, pairs, k, ctx->ws, d_topk_idx, d_topk_score,
+                                    static_cast<cudaStream_t>(stream), &ctx->launches);
+  return e == cudaSuccess ? KS_OK : cuda_fail(ctx, e, "ks_select");
+}
+
+ks_status ks_select_one(ks_ctx* ctx, ks_problem p, const ks_candidate* d_c, int C, const ks_model* model,
+                        int k, int32_t* h_topk_idx, float* h_topk_score, void* stream) {
+  if (!ctx || !model || model->ctx != ctx || k < 1 || k > KS_MAX_K || C < 0) return KS_ERR_INVALID_ARG;
+  if (!h_topk_idx || !h_topk_score || (C > 0 && !d_c)) return KS_ERR_INVALID_ARG;
+  if (p.m < 1 || p.n < 1 || p.k < 1 || p.m > KS_MAX_DIM || p.n > KS_MAX_DIM || p.k > KS_MAX_DIM ||
+      p.layout > 3 || p.dtype_ab > 3 || p.dtype_d > 3 || p.epi_flags > 5)
+    return KS_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t out_bytes = align_up(k * sizeof(int32_t)) + align_up(k * sizeof(float));
+  const size_t part = align_up(ks::select_partial_bytes(*model, 1, C, C, false, k));
+  ks_status s = ensure_workspace(ctx, part + out_bytes);
+  if (s != KS_OK) return s;
+  char* base = static_cast<char*>(ctx->ws);
+  int32_t* d_idx = reinterpret_cast<int32_t*>(base + part);
+  float* d_sc = reinterpret_cast<float*>(base + part + align_up(k * sizeof(int32_t)));
+  cudaError_t e = ks::launch_select(ctx->desc, *model, nullptr, &p, 1, d_c, C, nullptr, nullptr, C, k,
+                                    ctx->ws, d_idx, d_sc, st, &ctx->launches);
+  int32_t* pin_idx = static_cast<int32_t*>(ctx->pinned);
+  float* pin_sc = reinterpret_cast<float*>(pin_idx + KS_MAX_K);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(pin_idx, d_idx, k * sizeof(int32_t), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(pin_sc, d_sc, k * sizeof(float), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "ks_select_one");
+  std::memcpy(h_topk_idx, pin_idx, k * sizeof(int32_t));
+  std::memcpy(h_topk_score, pin_sc, k * sizeof(float));
+  return KS_OK;
+}
+
+ks_status ks_select_host(ks_ctx* ctx, const ks_problem* h_p, int P, const ks_candidate* h_c, int C,
+                         const int64_t* h_seg_offsets, const int32_t* h_seg_index, int64_t pairs,
+                         const ks_model* model, int k, int32_t* h_topk_idx, float* h_topk_score,
+                         void* stream) {
+  if (!ctx || !model || model->ctx != ctx || k < 1 || k > KS_MAX_K) return KS_ERR_INVALID_ARG;
+  ks_status s = check_pairs(P, C, h_seg_offsets, h_seg_index, pairs);
+  if (s != KS_OK) return s;
+  if (P == 0) return KS_OK;
+  if (!h_p || !h_topk_idx || !h_topk_score || (pairs > 0 && !h_c)) return KS_ERR_INVALID_ARG;
+  const bool seg = h_seg_offsets != nullptr;
+  if (seg && (h_seg_offsets[0] != 0 || h_seg_offsets[P] != pairs)) return KS_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t b_part = align_up(ks::select_partial_bytes(*model, P, C, pairs, seg, k));
+  const size_t b_p = align_up(sizeof(ks_problem) * P), b_c = align_up(sizeof(ks_candidate) * C);
+  const size_t b_so = seg ? align_up(sizeof(int64_t) * (P + 1)) : 0;
+  const size_t b_si = seg ? align_up(sizeof(int32_t) * pairs) : 0;
+  const size_t b_oi = align_up(sizeof(int32_t) * P * k), b_os = align_up(sizeof(float) * P * k);
+  s = ensure_workspace(ctx, b_part + b_p + b_c + b_so + b_si + b_oi + b_os);
+  if (s != KS_OK) return s;
+  char* q = static_cast<char*>(ctx->ws) + b_part;
+  ks_problem* d_p = reinterpret_cast<ks_problem*>(q); q += b_p;
+  ks_candidate* d_c = reinterpret_cast<ks_candidate*>(q); q += b_c;
+  int64_t* d_so = seg ? reinterpret_cast<int64_t*>(q) : nullptr; q += b_so;
+  int32_t* d_si = seg ? reinterpret_cast<int32_t*>(q) : nullptr; q += b_si;
+  int32_t* d_oi = reinterpret_cast<int32_t*>(q); q += b_oi;
+  float* d_os = reinterpret_cast<float*>(q);
+  cudaError_t e = cudaMemcpyAsync(d_p, h_p, sizeof(ks_problem) * P, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess && C > 0) e = cudaMemcpyAsync(d_c, h_c, sizeof(ks_candidate) * C, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess && seg) e = cudaMemcpyAsync(d_so, h_seg_offsets, sizeof(int64_t) * (P + 1), cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess && seg && pairs > 0) e = cudaMemcpyAsync(d_si, h_seg_index, sizeof(int32_t) * pairs, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess)
+    e = ks::launch_select(ctx->desc, *model, d_p, nullptr, P, d_c, C, d_so, d_si, pairs, k, ctx->ws, d_oi,
+                          d_os, st, &ctx->launches);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(h_topk_idx, d_oi, sizeof(int32_t) * P * k, cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(h_topk_score, d_os, sizeof(float) * P * k, cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  return e == cudaSuccess ? KS_OK : cuda_fail(ctx, e, "ks_select_host");
+}
+
+}  // extern "C"

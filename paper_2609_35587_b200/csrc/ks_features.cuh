@@ -1,0 +1,181 @@
+// Device-side feature map x = phi(p, c, h) (Table "Feature groups").
+//
+// Integer quantities are exact in 64-bit arithmetic; every float column is a fixed short
+// sequence of individually rounded binary32 operations issued through the round-to-nearest
+// intrinsics (__ll2float_rn, __fdiv_rn, __fmul_rn, __fsub_rn), which the compiler neither
+// contracts into FMAs nor replaces by approximations, so the bits do not depend on
+// optimisation flags. The split into problem-only, candidate-only and per-pair terms lets a
+// kernel hoist the first two out of its pair loop.
+#pragma once
+
+#include <cstdint>
+
+#include "ks.h"
+
+namespace ks {
+
+constexpr int kRow = KS_F_PAD;
+
+__device__ __forceinline__ float F64i(long long v) { return __ll2float_rn(v); }
+__device__ __forceinline__ float F32i(int v) { return __int2float_rn(v); }
+__device__ __forceinline__ unsigned cdiv_u32(unsigned a, unsigned b) { return (a + b - 1u) / b; }
+__device__ __forceinline__ long long cdiv_i64(long long a, long long b) { return (a + b - 1) / b; }
+
+__device__ __forceinline__ int bytes_ab(int dt) { return dt == 2 ? 1 : (dt == 3 ? 4 : 2); }
+__device__ __forceinline__ int bytes_d(int dt) { return dt == 2 ? 1 : (dt == 3 ? 4 : 2); }
+
+// Problem-only terms (section "Structural Core", "Memory Behavior"): computed once per problem.
+struct ProblemTerms {
+  unsigned M, N, K;
+  int bA, bD, dtype_ab, layout, has_bias, act;
+  long long bytesA, bytesB, Q_epi;  // b_A M K, b_B K N, Q_epilogue
+  float log2m, log2n, log2k;
+  float i_problem, ws_frac_l2, f_bytes_in, f_traffic_epi;
+  unsigned long long tc_rate;  // tensor rate of this problem's input type
+};
+
+__device__ __forceinline__ float log2_dim(unsigned v) {
+  return __double2float_rn(log2(static_cast<double>(v)));
+}
+
+__device__ inline void problem_terms(const ks_problem& p, const ks_gpu_desc& h, ProblemTerms& t) {
+  t.M = p.m; t.N = p.n; t.K = p.k;
+  t.dtype_ab = p.dtype_ab & 3;
+  t.layout = p.layout;
+  t.bA = bytes_ab(t.dtype_ab);
+  t.bD = bytes_d(p.dtype_d & 3);
+  t.has_bias = p.epi_flags & 1;
+  t.act = (p.epi_flags >> 1) & 3;
+  const long long M = t.M, N = t.N, K = t.K;
+  t.bytesA = t.bA * M * K;
+  t.bytesB = t.bA * K * N;
+  t.Q_epi = t.bD * M * N + (t.has_bias ? t.bD * M : 0);
+  t.log2m = log2_dim(t.M);
+  t.log2n = log2_dim(t.N);
+  t.log2k = log2_dim(t.K);
+  t.i_problem = __fdiv_rn(F64i(2 * M * N * K), F64i(t.bytesA + t.bytesB + t.Q_epi));
+  t.ws_frac_l2 = __fdiv_rn(F64i(t.bytesA + t.bytesB), F64i(static_cast<long long>(h.l2_bytes)));
+  t.f_traffic_epi = F64i(t.Q_epi);
+  t.tc_rate = h.tc_flops_per_us_per_sm[t.dtype_ab];
+}
+
+// Writes the 64 columns of one pair through `put(column, value)`.
+template <typename Put>
+__device__ __forceinline__ void featurize_pair(const ProblemTerms& t, const ks_candidate& c,
+                                               const ks_gpu_desc& h, Put put) {
+  const int TM = c.tile_m, TN = c.tile_n, TK = c.tile_k, S = c.stages;
+  const int cM = c.cluster_m, cN = c.cluster_n;
+  const int ks = c.kernel_sched & 3;
+  // (consumer warpgroups in the mainloop, threads per block): WS, Pingpong, Cooperative, basic
+  const int n_cons = (ks == 2) ? 2 : 1;
+  const int T_block = (ks == 0) ? 256 : (ks == 3 ? 128 : 384);
+  const int bA = t.bA, bD = t.bD;
+
+  // ---- structural core ------------------------------------------------------------------
+  put(0, t.log2m);
+  put(1, t.log2n);
+  put(2, t.log2k);
+  put(3, F32i(t.layout == 2 || t.layout == 3));
+  put(4, F32i(t.layout == 1 || t.layout == 3));
+  put(5, F32i(t.dtype_ab));
+  put(6, F32i(bA));
+  put(7, F32i(bD));
+  put(8, F32i(t.has_bias));
+  put(9, F32i(t.act));
+  put(10, F32i(TM));
+  put(11, F32i(TN));
+  put(12, F32i(TK));
+  put(13, F32i(c.instr_m));
+  put(14, F32i(c.instr_n));
+  put(15, F32i(c.instr_k));
+  put(16, F32i(S));
+  put(17, F32i(c.kernel_sched));
+  put(18, F32i(c.epi_sched));
+  put(19, F32i(c.tile_sched));
+  put(20, F32i(cM));
+  put(21, F32i(cN));
+  put(22, F32i(cM * cN));
+
+  // ---- resource pressure and occupancy ----------------------------------------------------
+  const long long B_stage = static_cast<long long>(TK) * (TM * bA + TN * bA);
+  const long long smem_main = S * B_stage;
+  const int E = (ks == 2) ? 128 : 64;
+  const long long B_epi =
+      (c.epi_sched == 0) ? 0 : 2ll * min(TM, E) * min(TN, 32) * bD;
+  const long long both = smem_main + B_epi + h.smem_reserved;
+  const long long B_smem =
+      (ks == 0 || ks == 3) ? max(smem_main, B_epi) + h.smem_reserved : both;
+  const float f_smem = __fdiv_rn(F64i(B_smem), F64i(h.smem_per_sm));
+  const int fits = both <= static_cast<long long>(h.smem_per_cta_max);
+  const long long area = static_cast<long long>(TM) * TN;
+  const long long b_smem = static_cast<long long>(h.smem_per_sm) / B_smem;
+  const long long regs = min(255ll, 32 + cdiv_i64(area, T_block));
+  const long long b_reg = static_cast<long long>(h.regs_per_sm) / (regs * T_block);
+  const long long b_arch =
+      min(static_cast<long long>(h.max_ctas_per_sm), static_cast<long long>(h.max_threads_per_sm / T_block));
+  const long long b_res = min(b_smem, min(b_reg, b_arch));
+  const long long b_eff = max(1ll, b_res);
+
+  // ---- work decomposition and wave quantisation ---------------------------------------------
+  const long long n_m = cdiv_u32(t.M, TM), n_n = cdiv_u32(t.N, TN), n_k = cdiv_u32(t.K, TK);
+  const long long n_tiles = n_m * n_n;
+  put(23, F64i(n_m));
+  put(24, F64i(n_n));
+  put(25, F64i(n_k));
+  put(26, F64i(n_tiles));
+  put(27, __fdiv_rn(F64i(n_m * TM - t.M), F64i(t.M)));
+  put(28, __fdiv_rn(F64i(n_n * TN - t.N), F64i(t.N)));
+  put(29, __fdiv_rn(F64i(n_tiles), F64i(h.num_sms)));
+  const long long resident = static_cast<long long>(h.num_sms) * b_eff;
+  const long long waves = cdiv_i64(n_tiles, resident);
+  put(30, F64i(waves));
+  const float eta = __fdiv_rn(F64i(n_tiles), F64i(waves * resident));
+  put(31, eta);
+  put(32, fmaxf(0.0f, __fsub_rn(1.0f, eta)));
+  const long long n_c = static_cast<long long>(cdiv_i64(t.M, static_cast<long long>(cM) * TM)) *
+                        cdiv_i64(t.N, static_cast<long long>(cN) * TN);
+  put(33, __fdiv_rn(F64i(n_c * cM * cN - n_tiles), F64i(n_tiles)));
+  put(34, __fdiv_rn(F64i(n_m), F64i(cM)));
+  put(35, __fdiv_rn(F64i(n_n), F64i(cN)));
+  put(36, F32i(cM > n_m || cN > n_n));
+
+  // ---- memory behaviour -----------------------------------------------------------------------
+  put(37, t.i_problem);
+  put(38, __fdiv_rn(F64i(2 * area), F64i(static_cast<long long>(TM) * bA + static_cast<long long>(TN) * bA)));
+  const long long restream = n_n * t.bytesA + n_m * t.bytesB;
+  put(39, __fdiv_rn(F64i(restream), F64i(t.bytesA + t.bytesB)));
+  put(40, t.ws_frac_l2);
+  const float fl2 = F64i(static_cast<long long>(h.l2_bytes));
+  put(41, __fdiv_rn(F64i(static_cast<long long>(bA) * TM * t.K), fl2));
+  put(42, __fdiv_rn(F64i(static_cast<long long>(bA) * TN * t.K), fl2));
+  put(43, F64i(restream));
+  put(44, F64i(cdiv_i64(n_n, cN) * t.bytesA + cdiv_i64(n_m, cM) * t.bytesB));
+  put(45, t.f_traffic_epi);
+
+  // ---- resource pressure columns ------------------------------------------------------------
+  put(46, F64i(B_stage));
+  put(47, F64i(smem_main));
+  put(48, F64i(B_epi));
+  put(49, F64i(B_smem));
+  put(50, f_smem);
+  put(51, F32i(fits));
+  put(52, __fdiv_rn(F64i(area), F32i(T_block)));
+  put(53, F64i(b_smem));
+  put(54, F64i(b_reg));
+  put(55, F64i(b_res));
+  put(56, __fdiv_rn(F64i(b_eff * T_block), F64i(h.max_threads_per_sm)));
+
+  // ---- pipeline balance -----------------------------------------------------------------------
+  const float t_prod = __fdiv_rn(F64i(static_cast<long long>(h.num_sms) * B_stage),
+                                 F64i(static_cast<long long>(h.tma_bytes_per_us)));
+  const float t_cons = __fdiv_rn(F64i(2 * area * TK), F64i(n_cons * static_cast<long long>(t.tc_rate)));
+  put(57, t_prod);
+  put(58, t_cons);
+  put(59, __fdiv_rn(t_cons, t_prod));
+  put(60, __fdiv_rn(F64i(min(static_cast<long long>(S), n_k)), F32i(S)));
+  put(61, __fdiv_rn(F64i(n_k), F32i(S)));
+  put(62, __fmul_rn(F32i(S), f_smem));
+  put(63, 0.0f);
+}
+
+}  // namespace ks

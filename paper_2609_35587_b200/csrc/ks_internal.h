@@ -1,0 +1,109 @@
+// Internal declarations shared by the translation units of libks (not part of the ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+
+#include <cstddef>
+#include <cstdint>
+
+#include "ks.h"
+
+namespace ks {
+
+// Generic device form of a tree node: 8 bytes, children tree-relative.
+struct DevNode {
+  float v;        // threshold, or the leaf value
+  uint16_t feat;  // 0xFFFF = leaf
+  uint16_t left;  // left child (right = left + 1)
+};
+
+struct GbdtModel {
+  int n_trees = 0;
+  int max_depth = 0;
+  int64_t n_nodes = 0;
+  float base = 0.0f;
+  DevNode* d_nodes = nullptr;  // all trees back to back
+  int* d_roots = nullptr;      // [n_trees + 1] offsets into d_nodes
+  // quantised fast form (complete trees in level order), see ks_gbdt_fast.cu
+  bool fast = false;
+  int fast_depth = 0;          // every tree padded to this depth
+  int n_qrows = 0;             // quantised feature rows (pseudo-features)
+  uint32_t* d_qnodes = nullptr;    // [n_trees][2^D - 1] packed (row offset, bin)
+  float* d_qleaves = nullptr;      // [n_trees][2^D]
+  uint16_t* d_qleaf_node = nullptr;  // [n_trees][2^D] original node index of each padded leaf
+  float* d_qthr = nullptr;         // [n_qrows][256] sorted thresholds (padded with +inf)
+  int* d_qrow_feat = nullptr;      // [n_qrows] source feature column of each row
+  int* d_qrow_count = nullptr;     // [n_qrows] number of thresholds in the row
+};
+
+struct MlpModel {
+  int n_layers = 0;
+  int widths[KS_MLP_MAX_LAYERS + 1] = {0};
+  int max_width = 0;
+  uint16_t* d_w[KS_MLP_MAX_LAYERS] = {nullptr};  // bf16 [out, in] row-major
+  float* d_b[KS_MLP_MAX_LAYERS] = {nullptr};
+  float* d_mu = nullptr;
+  float* d_sigma = nullptr;
+};
+
+// kernel-side view of an MLP (passed by value)
+struct MlpView {
+  int n_layers;
+  int widths[KS_MLP_MAX_LAYERS + 1];
+  const uint16_t* w[KS_MLP_MAX_LAYERS];
+  const float* b[KS_MLP_MAX_LAYERS];
+  const float* mu;
+  const float* sigma;
+};
+
+}  // namespace ks
+
+struct ks_ctx {
+  int device = 0;
+  ks_gpu_desc desc{};
+  void* ws = nullptr;  // device workspace (partial top-k lists, staging)
+  size_t ws_bytes = 0;
+  void* pinned = nullptr;  // host staging for ks_select_one results
+  size_t pinned_bytes = 0;
+  int64_t launches = 0;
+  char err[256] = {0};
+};
+
+struct ks_model {
+  ks_ctx* ctx = nullptr;
+  int kind = 0;  // 0 tree ensemble, 1 MLP
+  ks::GbdtModel gbdt;
+  ks::MlpModel mlp;
+};
+
+namespace ks {
+
+constexpr int kBlock = 256;            // threads per block of the pair kernels
+constexpr int kSubTilesMax = 8;        // sub-tiles of kBlock rows one block ranks
+
+// Builds the quantised fast form of a validated ensemble when it qualifies (m.fast).
+cudaError_t build_fast_gbdt(GbdtModel& m, int n_trees, const int64_t* h_tree_offsets,
+                            const ks_node_host* h_nodes);
+
+// ---- launchers (each enqueues on `stream`, returns the cudaError of the launch) -----------
+cudaError_t launch_featurize(const ks_gpu_desc& desc, const ks_problem* d_p, int P,
+                             const ks_candidate* d_c, int C, const int64_t* d_seg_off,
+                             const int32_t* d_seg_idx, int64_t pairs, float* d_out,
+                             cudaStream_t stream, int64_t* launches);
+
+cudaError_t launch_score_gbdt(const GbdtModel& m, const float* d_feat, int64_t rows, float* d_scores,
+                              uint16_t* d_leaf_idx, cudaStream_t stream, int64_t* launches);
+
+cudaError_t launch_score_mlp(const MlpModel& m, const float* d_feat, int64_t rows, float* d_scores,
+                             cudaStream_t stream, int64_t* launches);
+
+// Fused featurize + score + top-k. `p_by_value` non-null selects the single-problem form.
+// d_partial: workspace for the per-block partial lists, at least select_partial_bytes().
+size_t select_partial_bytes(const ks_model& model, int P, int C, int64_t pairs, bool segmented, int k);
+cudaError_t launch_select(const ks_gpu_desc& desc, const ks_model& model, const ks_problem* d_p,
+                          const ks_problem* p_by_value, int P, const ks_candidate* d_c, int C,
+                          const int64_t* d_seg_off, const int32_t* d_seg_idx, int64_t pairs, int k,
+                          void* d_partial, int32_t* d_topk_idx, float* d_topk_score,
+                          cudaStream_t stream, int64_t* launches);
+
+}  // namespace ks

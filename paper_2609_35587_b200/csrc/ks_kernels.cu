@@ -1,0 +1,437 @@
+// Generic kernels of libks: the standalone feature map, the standalone scorers, the generic
+// fused featurize + score + top-k kernel (any tree shape, any MLP the ABI accepts) and the
+// per-problem merge of partial top-k lists. The quantised fast path for complete trees lives
+// in ks_gbdt_fast.cu.
+#include <cuda_bf16.h>
+
+#include "ks_features.cuh"
+#include "ks_internal.h"
+#include "ks_topk.cuh"
+
+namespace ks {
+
+// ------------------------------------------------------------------------------------------
+// block -> (problem, chunk) mapping shared by the pair kernels
+// ------------------------------------------------------------------------------------------
+
+struct PairMap {
+  int P, C, nblk;           // nblk blocks per problem
+  int rows_per_block;       // rows one block covers per pass
+  const int64_t* seg_off;   // null = dense
+  const int32_t* seg_idx;
+};
+
+__device__ __forceinline__ void segment_of(const PairMap& m, int prob, int64_t& lo, int64_t& len) {
+  if (m.seg_off) {
+    lo = m.seg_off[prob];
+    len = m.seg_off[prob + 1] - lo;
+  } else {
+    lo = static_cast<int64_t>(prob) * m.C;
+    len = m.C;
+  }
+}
+
+__device__ __forceinline__ int pool_index(const PairMap& m, int64_t lo, int64_t r) {
+  return m.seg_off ? m.seg_idx[lo + r] : static_cast<int>(r);
+}
+
+// ------------------------------------------------------------------------------------------
+// ks_featurize: one thread per pair, rows staged through shared memory for coalesced stores
+// ------------------------------------------------------------------------------------------
+
+__global__ void __launch_bounds__(kBlock)
+featurize_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, const ks_candidate* __restrict__ c,
+                 PairMap map, float* __restrict__ out) {
+  extern __shared__ float s_tile[];  // [kBlock][65]
+  __shared__ ProblemTerms s_pt;
+  const int prob = blockIdx.x / map.nblk, chunk = blockIdx.x % map.nblk;
+  int64_t lo, len;
+  segment_of(map, prob, lo, len);
+  if (threadIdx.x == 0) problem_terms(p[prob], desc, s_pt);
+  __syncthreads();
+  for (int64_t start = static_cast<int64_t>(chunk) * kBlock; start < len;
+       start += static_cast<int64_t>(map.nblk) * kBlock) {
+    const int64_t r = start + threadIdx.x;
+    if (r < len) {
+      const ks_candidate cand = c[pool_index(map, lo, r)];
+      float* row = s_tile + threadIdx.x * 65;
+      featurize_pair(s_pt, cand, desc, [&](int col, float v) { row[col] = v; });
+    }
+    __syncthreads();
+    const int64_t n_rows = (len - start < kBlock) ? (len - start) : static_cast<int64_t>(kBlock);
+    float* dst = out + (lo + start) * kRow;
+    for (int i = threadIdx.x; i < n_rows * kRow; i += kBlock) dst[i] = s_tile[(i >> 6) * 65 + (i & 63)];
+    __syncthreads();
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// generic tree walk: nodes from global memory (read-only path), features from a shared tile
+// laid out [column][thread] so that a warp's reads of one column are conflict-free
+// ------------------------------------------------------------------------------------------
+
+__device__ __forceinline__ DevNode load_node(const DevNode* p) {
+  const uint2 u = __ldg(reinterpret_cast<const uint2*>(p));
+  DevNode n;
+  n.v = __uint_as_float(u.x);
+  n.feat = static_cast<uint16_t>(u.y & 0xFFFFu);
+  n.left = static_cast<uint16_t>(u.y >> 16);
+  return n;
+}
+
+// returns base + sum of leaves; optionally records the leaf node index of every tree
+__device__ __forceinline__ float walk_ensemble(const DevNode* __restrict__ nodes,
+                                               const int* __restrict__ roots, int n_trees, float base,
+                                               const float* s_cols /* [64][kBlock], this thread's lane */,
+                                               uint16_t* leaf_out) {
+  float s = base;
+  for (int t = 0; t < n_trees; ++t) {
+    const DevNode* tree = nodes + roots[t];
+    int i = 0;
+    DevNode nd = load_node(tree);
+#pragma unroll 1
+    for (int d = 0; d <= KS_MAX_DEPTH && nd.feat != 0xFFFFu; ++d) {
+      const float x = s_cols[nd.feat * kBlock];
+      i = nd.left + (x < nd.v ? 0 : 1);
+      nd = load_node(tree + i);
+    }
+    if (leaf_out) leaf_out[t] = static_cast<uint16_t>(i);
+    s += nd.v;
+  }
+  return s;
+}
+
+__global__ void __launch_bounds__(kBlock)
+score_gbdt_kernel(const DevNode* __restrict__ nodes, const int* __restrict__ roots, int n_trees,
+                  float base, const float* __restrict__ feat, int64_t rows, float* __restrict__ scores,
+                  uint16_t* __restrict__ leaf_idx) {
+  extern __shared__ float s_cols[];  // [64][kBlock]
+  const int64_t r = static_cast<int64_t>(blockIdx.x) * kBlock + threadIdx.x;
+  if (r < rows) {
+    const float4* src = reinterpret_cast<const float4*>(feat + r * kRow);
+#pragma unroll 4
+    for (int q = 0; q < kRow / 4; ++q) {
+      const float4 v = __ldg(src + q);
+      s_cols[(4 * q + 0) * kBlock + threadIdx.x] = v.x;
+      s_cols[(4 * q + 1) * kBlock + threadIdx.x] = v.y;
+      s_cols[(4 * q + 2) * kBlock + threadIdx.x] = v.z;
+      s_cols[(4 * q + 3) * kBlock + threadIdx.x] = v.w;
+    }
+    const float s = walk_ensemble(nodes, roots, n_trees, base, s_cols + threadIdx.x,
+                                  leaf_idx ? leaf_idx + r * n_trees : nullptr);
+    scores[r] = s + 0.0f;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// generic MLP on a tile of kBlock rows held as [column][thread] fp32 in shared memory.
+// Rows are processed 32 at a time; thread (r = tid % 32, g = tid / 32) computes the outputs
+// o = g, g + 8, ... of row r. Activations are bf16 in shared memory, [unit][32].
+// ------------------------------------------------------------------------------------------
+
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t b) { return __uint_as_float(b << 16); }
+
+__device__ void mlp_tile(const MlpView& m, int max_width, const float* s_cols /* [64][kBlock] */,
+                         __nv_bfloat16* s_act /* [2][max_width][32] */, float* s_scores /* [kBlock] */) {
+  const int r = threadIdx.x & 31, g = threadIdx.x >> 5;
+  constexpr int kGroups = kBlock / 32;
+  for (int grp = 0; grp < kGroups; ++grp) {
+    __nv_bfloat16* cur = s_act;
+    __nv_bfloat16* nxt = s_act + max_width * 32;
+    for (int col = g; col < kRow; col += kGroups) {
+      float v = 0.0f;
+      if (col < KS_F) {
+        v = s_cols[col * kBlock + grp * 32 + r];
+        if (!isfinite(v)) v = 0.0f;
+        v = __fdiv_rn(__fsub_rn(v, m.mu[col]), m.sigma[col]);
+      }
+      cur[col * 32 + r] = __float2bfloat16_rn(v);
+    }
+    __syncthreads();
+    for (int l = 0; l < m.n_layers; ++l) {
+      const int wi = m.widths[l], wo = m.widths[l + 1];
+      const bool last = (l == m.n_layers - 1);
+      for (int o = g; o < wo; o += kGroups) {
+        const uint4* wrow = reinterpret_cast<const uint4*>(m.w[l] + static_cast<size_t>(o) * wi);
+        float acc = 0.0f;
+        for (int i8 = 0; i8 < wi / 8; ++i8) {
+          const uint4 wv = __ldg(wrow + i8);
+          const uint32_t ww[4] = {wv.x, wv.y, wv.z, wv.w};
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const int i = i8 * 8 + 2 * q;
+            acc = fmaf(bf16_bits_to_float(ww[q] & 0xFFFFu), __bfloat162float(cur[i * 32 + r]), acc);
+            acc = fmaf(bf16_bits_to_float(ww[q] >> 16), __bfloat162float(cur[(i + 1) * 32 + r]), acc);
+          }
+        }
+        float v = acc + m.b[l][o];
+        if (last) {
+          if (o == 0) s_scores[grp * 32 + r] = v;
+        } else {
+          nxt[o * 32 + r] = __float2bfloat16_rn(fmaxf(v, 0.0f));
+        }
+      }
+      __syncthreads();
+      __nv_bfloat16* tmp = cur;
+      cur = nxt;
+      nxt = tmp;
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kBlock)
+score_mlp_kernel(MlpView m, int max_width, const float* __restrict__ feat, int64_t rows,
+                 float* __restrict__ scores) {
+  extern __shared__ __align__(16) unsigned char s_raw[];
+  float* s_cols = reinterpret_cast<float*>(s_raw);                       // [64][kBlock]
+  float* s_scores = s_cols + kRow * kBlock;                              // [kBlock]
+  __nv_bfloat16* s_act = reinterpret_cast<__nv_bfloat16*>(s_scores + kBlock);
+  const int64_t r = static_cast<int64_t>(blockIdx.x) * kBlock + threadIdx.x;
+  const float4* src = reinterpret_cast<const float4*>(feat + min(r, rows - 1) * kRow);
+#pragma unroll 4
+  for (int q = 0; q < kRow / 4; ++q) {
+    const float4 v = __ldg(src + q);
+    s_cols[(4 * q + 0) * kBlock + threadIdx.x] = v.x;
+    s_cols[(4 * q + 1) * kBlock + threadIdx.x] = v.y;
+    s_cols[(4 * q + 2) * kBlock + threadIdx.x] = v.z;
+    s_cols[(4 * q + 3) * kBlock + threadIdx.x] = v.w;
+  }
+  __syncthreads();
+  mlp_tile(m, max_width, s_cols, s_act, s_scores);
+  if (r < rows) scores[r] = s_scores[threadIdx.x] + 0.0f;
+}
+
+// ------------------------------------------------------------------------------------------
+// generic fused select: featurize a sub-tile of kBlock pairs into shared memory, score it,
+// keep one key per thread per sub-tile, rank the block's keys, write a partial top-k list.
+// ------------------------------------------------------------------------------------------
+
+template <int kModel>  // 0 = tree ensemble, 1 = MLP
+__global__ void __launch_bounds__(kBlock)
+select_generic_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_problem p_value,
+                      int use_value, const ks_candidate* __restrict__ c, PairMap map, int sub_tiles,
+                      const DevNode* __restrict__ nodes, const int* __restrict__ roots, int n_trees,
+                      float base, MlpView mlp, int max_width, int k,
+                      unsigned long long* __restrict__ partial /* [P][nblk][k] */) {
+  extern __shared__ __align__(16) unsigned char s_raw[];
+  float* s_cols = reinterpret_cast<float*>(s_raw);  // [64][kBlock]
+  float* s_scores = s_cols + kRow * kBlock;         // [kBlock] (MLP only)
+  __nv_bfloat16* s_act = reinterpret_cast<__nv_bfloat16*>(s_scores + kBlock);
+  __shared__ ProblemTerms s_pt;
+  __shared__ unsigned long long s_warp[kBlock / 32];
+  __shared__ unsigned long long s_list[KS_MAX_K];
+
+  const int prob = blockIdx.x / map.nblk, chunk = blockIdx.x % map.nblk;
+  int64_t lo, len;
+  segment_of(map, prob, lo, len);
+  if (threadIdx.x == 0) problem_terms(use_value ? p_value : p[prob], desc, s_pt);
+  if (threadIdx.x < KS_MAX_K) s_list[threadIdx.x] = 0ull;
+  __syncthreads();
+
+  const int64_t pass_rows = static_cast<int64_t>(sub_tiles) * kBlock;
+  for (int64_t start = static_cast<int64_t>(chunk) * pass_rows; start < len;
+       start += static_cast<int64_t>(map.nblk) * pass_rows) {
+    unsigned long long keys[kSubTilesMax + 1];
+#pragma unroll
+    for (int s = 0; s <= kSubTilesMax; ++s) keys[s] = 0ull;
+    // carry the list of the previous pass in as extra keys
+    if (threadIdx.x < k) keys[kSubTilesMax] = s_list[threadIdx.x];
+#pragma unroll 1
+    for (int s = 0; s < sub_tiles; ++s) {
+      const int64_t r = start + static_cast<int64_t>(s) * kBlock + threadIdx.x;
+      const bool live = r < len;
+      int idx = 0;
+      __syncthreads();  // previous sub-tile's readers are done with s_cols
+      if (live) {
+        idx = pool_index(map, lo, r);
+        const ks_candidate cand = c[idx];
+        float* col0 = s_cols + threadIdx.x;
+        featurize_pair(s_pt, cand, desc, [&](int col, float v) { col0[col * kBlock] = v; });
+      } else if (kModel == 1) {
+        for (int col = 0; col < kRow; ++col) s_cols[col * kBlock + threadIdx.x] = 0.0f;
+      }
+      float score;
+      if (kModel == 0) {
+        score = live ? walk_ensemble(nodes, roots, n_trees, base, s_cols + threadIdx.x, nullptr) : 0.0f;
+      } else {
+        __syncthreads();
+        mlp_tile(mlp, max_width, s_cols, s_act, s_scores);
+        score = s_scores[threadIdx.x];
+      }
+      const unsigned long long key = live ? make_key(score + 0.0f, idx) : 0ull;
+#pragma unroll
+      for (int q = 0; q < kSubTilesMax; ++q)
+        if (q == s) keys[q] = key;
+    }
+    block_topk<kSubTilesMax + 1>(keys, k, s_warp, s_list);
+  }
+  if (threadIdx.x < k)
+    partial[(static_cast<size_t>(prob) * map.nblk + chunk) * k + threadIdx.x] = s_list[threadIdx.x];
+}
+
+// ------------------------------------------------------------------------------------------
+// merge: one warp per problem ranks the nblk * k partial keys
+// ------------------------------------------------------------------------------------------
+
+__global__ void __launch_bounds__(kBlock)
+topk_merge_kernel(const unsigned long long* __restrict__ partial, int P, int n_keys, int k,
+                  int32_t* __restrict__ out_idx, float* __restrict__ out_score) {
+  const int warp = (blockIdx.x * kBlock + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (warp >= P) return;
+  const unsigned long long* keys = partial + static_cast<size_t>(warp) * n_keys;
+  unsigned long long prev = ~0ull;
+  for (int j = 0; j < k; ++j) {
+    unsigned long long best = 0ull;
+    for (int i = lane; i < n_keys; i += 32) {
+      const unsigned long long v = keys[i];
+      if (v < prev && v > best) best = v;
+    }
+    best = warp_max_u64(best);
+    if (lane == 0) {
+      out_idx[static_cast<size_t>(warp) * k + j] = key_index(best);
+      out_score[static_cast<size_t>(warp) * k + j] = key_score(best);
+    }
+    prev = best == 0ull ? 0ull : best;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// launchers
+// ------------------------------------------------------------------------------------------
+
+static PairMap make_map(int P, int C, int64_t pairs, const int64_t* seg_off, const int32_t* seg_idx,
+                        int rows_per_block) {
+  PairMap m;
+  m.P = P;
+  m.C = C;
+  m.seg_off = seg_off;
+  m.seg_idx = seg_idx;
+  m.rows_per_block = rows_per_block;
+  const int64_t per_problem = seg_off ? (P > 0 ? (pairs + P - 1) / P : 0) : C;
+  m.nblk = static_cast<int>(per_problem > 0 ? (per_problem + rows_per_block - 1) / rows_per_block : 1);
+  if (m.nblk < 1) m.nblk = 1;
+  return m;
+}
+
+cudaError_t launch_featurize(const ks_gpu_desc& desc, const ks_problem* d_p, int P,
+                             const ks_candidate* d_c, int C, const int64_t* d_seg_off,
+                             const int32_t* d_seg_idx, int64_t pairs, float* d_out,
+                             cudaStream_t stream, int64_t* launches) {
+  if (P == 0 || pairs == 0) return cudaSuccess;
+  const PairMap map = make_map(P, C, pairs, d_seg_off, d_seg_idx, kBlock);
+  const size_t smem = sizeof(float) * kBlock * 65;
+  cudaError_t e = cudaFuncSetAttribute(featurize_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       static_cast<int>(smem));
+  if (e != cudaSuccess) return e;
+  featurize_kernel<<<static_cast<unsigned>(static_cast<int64_t>(P) * map.nblk), kBlock, smem, stream>>>(
+      desc, d_p, d_c, map, d_out);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_score_gbdt(const GbdtModel& m, const float* d_feat, int64_t rows, float* d_scores,
+                              uint16_t* d_leaf_idx, cudaStream_t stream, int64_t* launches) {
+  if (rows == 0) return cudaSuccess;
+  const size_t smem = sizeof(float) * kRow * kBlock;
+  cudaError_t e = cudaFuncSetAttribute(score_gbdt_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       static_cast<int>(smem));
+  if (e != cudaSuccess) return e;
+  score_gbdt_kernel<<<static_cast<unsigned>((rows + kBlock - 1) / kBlock), kBlock, smem, stream>>>(
+      m.d_nodes, m.d_roots, m.n_trees, m.base, d_feat, rows, d_scores, d_leaf_idx);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+static MlpView make_view(const MlpModel& m) {
+  MlpView v{};
+  v.n_layers = m.n_layers;
+  for (int l = 0; l <= m.n_layers; ++l) v.widths[l] = m.widths[l];
+  for (int l = 0; l < m.n_layers; ++l) {
+    v.w[l] = m.d_w[l];
+    v.b[l] = m.d_b[l];
+  }
+  v.mu = m.d_mu;
+  v.sigma = m.d_sigma;
+  return v;
+}
+
+static size_t mlp_smem_bytes(int max_width) {
+  return sizeof(float) * (kRow * kBlock + kBlock) + sizeof(__nv_bfloat16) * 2 * max_width * 32;
+}
+
+cudaError_t launch_score_mlp(const MlpModel& m, const float* d_feat, int64_t rows, float* d_scores,
+                             cudaStream_t stream, int64_t* launches) {
+  if (rows == 0) return cudaSuccess;
+  const size_t smem = mlp_smem_bytes(m.max_width);
+  cudaError_t e = cudaFuncSetAttribute(score_mlp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       static_cast<int>(smem));
+  if (e != cudaSuccess) return e;
+  score_mlp_kernel<<<static_cast<unsigned>((rows + kBlock - 1) / kBlock), kBlock, smem, stream>>>(
+      make_view(m), m.max_width, d_feat, rows, d_scores);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+static int pick_sub_tiles(int P, int64_t per_problem) {
+  for (int s = kSubTilesMax; s > 1; s >>= 1) {
+    const int64_t nblk = (per_problem + static_cast<int64_t>(s) * kBlock - 1) / (static_cast<int64_t>(s) * kBlock);
+    if (static_cast<int64_t>(P) * nblk >= 4 * 148) return s;
+  }
+  return 1;
+}
+
+static int64_t per_problem_rows(int P, int C, int64_t pairs, bool segmented) {
+  return segmented ? (P > 0 ? (pairs + P - 1) / P : 0) : C;
+}
+
+size_t select_partial_bytes(const ks_model& model, int P, int C, int64_t pairs, bool segmented, int k) {
+  (void)model;
+  const int64_t per = per_problem_rows(P, C, pairs, segmented);
+  const int st = pick_sub_tiles(P, per);
+  int64_t nblk = (per + static_cast<int64_t>(st) * kBlock - 1) / (static_cast<int64_t>(st) * kBlock);
+  if (nblk < 1) nblk = 1;
+  return static_cast<size_t>(P) * nblk * k * sizeof(unsigned long long);
+}
+
+cudaError_t launch_select(const ks_gpu_desc& desc, const ks_model& model, const ks_problem* d_p,
+                          const ks_problem* p_by_value, int P, const ks_candidate* d_c, int C,
+                          const int64_t* d_seg_off, const int32_t* d_seg_idx, int64_t pairs, int k,
+                          void* d_partial, int32_t* d_topk_idx, float* d_topk_score,
+                          cudaStream_t stream, int64_t* launches) {
+  if (P == 0) return cudaSuccess;
+  const int64_t per = per_problem_rows(P, C, pairs, d_seg_off != nullptr);
+  const int st = pick_sub_tiles(P, per);
+  const PairMap map = make_map(P, C, pairs, d_seg_off, d_seg_idx, st * kBlock);
+  unsigned long long* partial = static_cast<unsigned long long*>(d_partial);
+  const unsigned grid = static_cast<unsigned>(static_cast<int64_t>(P) * map.nblk);
+  ks_problem pv{};
+  if (p_by_value) pv = *p_by_value;
+  cudaError_t e;
+  if (model.kind == 0) {
+    const GbdtModel& g = model.gbdt;
+    const size_t smem = sizeof(float) * kRow * kBlock;
+    e = cudaFuncSetAttribute(select_generic_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    select_generic_kernel<0><<<grid, kBlock, smem, stream>>>(
+        desc, d_p, pv, p_by_value != nullptr, d_c, map, st, g.d_nodes, g.d_roots, g.n_trees, g.base,
+        MlpView{}, 0, k, partial);
+  } else {
+    const size_t smem = mlp_smem_bytes(model.mlp.max_width);
+    e = cudaFuncSetAttribute(select_generic_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(smem));
+    if (e != cudaSuccess) return e;
+    select_generic_kernel<1><<<grid, kBlock, smem, stream>>>(
+        desc, d_p, pv, p_by_value != nullptr, d_c, map, st, nullptr, nullptr, 0, 0.0f,
+        make_view(model.mlp), model.mlp.max_width, k, partial);
+  }
+  ++*launches;
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  topk_merge_kernel<<<(P * 32 + kBlock - 1) / kBlock, kBlock, 0, stream>>>(partial, P, map.nblk * k, k,
+                                                                          d_topk_idx, d_topk_score);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+}  // namespace ks

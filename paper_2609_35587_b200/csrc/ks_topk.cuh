@@ -1,0 +1,62 @@
+// Ranking keys and the block / warp selection primitives of the segmented top-k.
+//
+// A (score, pool index) pair becomes one 64-bit key whose unsigned order is the ranking
+// order of the selection rule: higher score first, lower index first among equal scores.
+// Key 0 means "no candidate". Because keys are distinct, the j-th best key is the largest key
+// below the (j-1)-th, so selection needs no removal step.
+#pragma once
+
+#include <cstdint>
+
+namespace ks {
+
+__device__ __forceinline__ unsigned long long make_key(float score, int idx) {
+  unsigned u = __float_as_uint(score);
+  u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+  return (static_cast<unsigned long long>(u) << 32) | static_cast<unsigned>(~idx);
+}
+
+__device__ __forceinline__ int key_index(unsigned long long key) {
+  return key == 0ull ? -1 : static_cast<int>(~static_cast<unsigned>(key));
+}
+
+__device__ __forceinline__ float key_score(unsigned long long key) {
+  if (key == 0ull) return __uint_as_float(0xFF800000u);  // -inf
+  unsigned u = static_cast<unsigned>(key >> 32);
+  u = (u & 0x80000000u) ? (u & 0x7FFFFFFFu) : ~u;
+  return __uint_as_float(u);
+}
+
+__device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
+  const unsigned hi = __reduce_max_sync(0xFFFFFFFFu, static_cast<unsigned>(v >> 32));
+  const unsigned lo =
+      __reduce_max_sync(0xFFFFFFFFu, static_cast<unsigned>(v >> 32) == hi ? static_cast<unsigned>(v) : 0u);
+  return (static_cast<unsigned long long>(hi) << 32) | lo;
+}
+
+// The k largest of the block's keys (N per thread), descending, into s_list[0..k).
+// All threads of the block must call; s_warp holds one slot per warp.
+template <int N>
+__device__ __forceinline__ void block_topk(const unsigned long long (&keys)[N], int k,
+                                           unsigned long long* s_warp, unsigned long long* s_list) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, n_warps = blockDim.x >> 5;
+  unsigned long long prev = ~0ull;
+  for (int j = 0; j < k; ++j) {
+    unsigned long long best = 0ull;
+#pragma unroll
+    for (int q = 0; q < N; ++q) {
+      const unsigned long long v = keys[q];
+      if (v < prev && v > best) best = v;
+    }
+    best = warp_max_u64(best);
+    if (lane == 0) s_warp[warp] = best;
+    __syncthreads();
+    unsigned long long w = 0ull;
+    for (int i = 0; i < n_warps; ++i) w = max(w, s_warp[i]);
+    if (threadIdx.x == 0) s_list[j] = w;
+    prev = w;
+    __syncthreads();
+  }
+}
+
+}  // namespace ks

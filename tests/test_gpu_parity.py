@@ -1,0 +1,315 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle, element by element, on
+seeded inputs that span several tiles and a ragged tail, plus the edge cases of the method.
+
+Bars: integer-valued features, leaf indices and top-k indices bit-exact (top-k up to
+tolerance ties); float features bit-exact expected, gate 1e-5 relative; tree-ensemble scores
+1e-5 * max(1, |s|); MLP scores 2e-2 * max(1, |s|)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2609_35587_b200 import workloads as wl
+from tests.helpers import candidate, problem, topk_accept
+
+pytestmark = pytest.mark.gpu
+
+DESC = wl.gpu_desc()
+TOL_GBDT, TOL_MLP = 1e-5, 2e-2
+
+
+@pytest.fixture(scope="module")
+def ks():
+    from paper_2609_35587_b200 import binding
+    return binding
+
+
+@pytest.fixture(scope="module")
+def ctx(ks):
+    c = ks.Context(DESC, 0)
+    yield c
+    c.close()
+
+
+def dev(ks, a):
+    return ks.to_device(a, torch.device("cuda", 0))
+
+
+def gpu_features(ks, ctx, prob, cand, so=None, si=None):
+    pairs = len(prob) * len(cand) if so is None else int(so[-1])
+    out = ctx.featurize(dev(ks, prob), len(prob), dev(ks, cand), len(cand),
+                        None if so is None else dev(ks, so), None if si is None else dev(ks, si), pairs)
+    torch.cuda.synchronize()
+    return out.cpu().numpy()
+
+
+def assert_features_equal(got, ref):
+    assert got.shape == ref.shape
+    same = got.view(np.uint32) == ref.view(np.uint32)
+    if not same.all():
+        r, c = np.argwhere(~same)[0]
+        raise AssertionError(f"feature [{r}, {c}]: gpu {got[r, c]!r} oracle {ref[r, c]!r} "
+                             f"({(~same).sum()} of {same.size} differ)")
+
+
+# ---------------------------------------------------------------------------------------------
+# ks_featurize
+# ---------------------------------------------------------------------------------------------
+
+def test_featurize_config0_bit_exact(ks, ctx):
+    prob, cand, _, _ = wl.make_inputs(0)
+    assert_features_equal(gpu_features(ks, ctx, prob, cand), oracle.featurize(prob, cand, DESC))
+
+
+def test_featurize_cross_precision_segments_bit_exact(ks, ctx):
+    prob, cand, so, si = wl.make_inputs(2, P=37, seg=333)
+    got = gpu_features(ks, ctx, prob, cand, so, si)
+    assert_features_equal(got, oracle.featurize(prob, cand, DESC, so, si))
+
+
+def test_featurize_stream_problems_and_ragged_sizes(ks, ctx):
+    prob, cand, _, _ = wl.make_inputs(3, P=301, C=70)
+    assert_features_equal(gpu_features(ks, ctx, prob, cand), oracle.featurize(prob, cand, DESC))
+    for C in (1, 255, 256, 257):
+        prob, cand, _, _ = wl.make_inputs(1, P=3, C=C)
+        assert_features_equal(gpu_features(ks, ctx, prob, cand), oracle.featurize(prob, cand, DESC))
+
+
+def test_featurize_extreme_dimensions_and_wide_knobs(ks, ctx):
+    prob = np.concatenate([problem(1, 1, 1), problem(1 << 19, 1 << 19, 1 << 19, 3, 3, 3, 5),
+                           problem(524287, 3, 99991, 1, 2, 1, 4), problem(7, 524288, 13, 2, 1, 1, 1)])
+    cand = np.concatenate([candidate(64, 16, 32, 2), candidate(256, 256, 512, 12, 16, 1, 2, 2, 1),
+                           candidate(192, 80, 256, 9, 1, 16, 1, 1, 0), candidate(128, 48, 64, 5, 4, 4, 3, 0, 0)])
+    assert_features_equal(gpu_features(ks, ctx, prob, cand), oracle.featurize(prob, cand, DESC))
+
+
+def test_featurize_empty_and_uneven_segments(ks, ctx):
+    prob, cand, _, _ = wl.make_inputs(2, P=5, seg=1)
+    so = np.array([0, 0, 600, 601, 601, 1300], np.int64)
+    si = (np.arange(1300) * 7 % len(cand)).astype(np.int32)
+    assert_features_equal(gpu_features(ks, ctx, prob, cand, so, si), oracle.featurize(prob, cand, DESC, so, si))
+
+
+# ---------------------------------------------------------------------------------------------
+# ks_score
+# ---------------------------------------------------------------------------------------------
+
+def test_score_gbdt_leaf_indices_and_scores(ks, ctx):
+    w = wl.make_workload(0, P=16, C=700)
+    x = oracle.featurize(w.problems, w.candidates, DESC)
+    rs, rleaf = oracle.score_gbdt(x, *w.gbdt, want_leaf_idx=True)
+    model = ctx.model_create_gbdt(*w.gbdt)
+    s, leaf = ctx.score(dev(ks, x), model, want_leaf_idx=True)
+    torch.cuda.synchronize()
+    assert np.array_equal(leaf.cpu().numpy().view(np.uint16), rleaf)
+    s = s.cpu().numpy()
+    assert np.all(np.abs(s - rs) <= TOL_GBDT * np.maximum(1, np.abs(rs)))
+    assert len(np.unique(rleaf)) > 32
+
+
+def test_score_gbdt_unbalanced_and_stump_trees(ks, ctx):
+    nodes = np.zeros(9, wl.NODE_DT)
+    # tree 0: root -> (leaf | node -> (leaf | leaf)); tree 1: a single leaf; tree 2: depth 1
+    recs = [(1, 0.0, 1), (None, -1.0, 0), (2, 10.0, 3), (None, 5.0, 0), (None, 7.0, 0),
+            (None, 0.25, 0), (0, 3.0, 1), (None, 100.0, 0), (None, 200.0, 0)]
+    for i, (f, v, left) in enumerate(recs):
+        nodes[i] = (v, 0xFFFF if f is None else f, 0, left)
+    off = np.array([0, 5, 6, 9])
+    x = np.zeros((300, 64), np.float32)
+    rng = np.random.default_rng(0)
+    x[:, :3] = rng.normal(0, 8, size=(300, 3)).astype(np.float32)
+    x[0, 0] = 3.0  # exactly on the threshold: not strictly less, goes right
+    rs, rleaf = oracle.score_gbdt(x, off, nodes, 0.5, want_leaf_idx=True)
+    model = ctx.model_create_gbdt(off, nodes, 0.5)
+    s, leaf = ctx.score(dev(ks, x), model, want_leaf_idx=True)
+    torch.cuda.synchronize()
+    assert np.array_equal(leaf.cpu().numpy().view(np.uint16), rleaf)
+    assert np.array_equal(s.cpu().numpy(), rs)
+
+
+def test_score_mlp(ks, ctx):
+    w = wl.make_workload(4, P=3, C=411)
+    x = oracle.featurize(w.problems, w.candidates, DESC)
+    x[5, 7] = np.nan
+    x[6, 40] = np.inf
+    rs = oracle.score_mlp(x, w.mlp)
+    model = ctx.model_create_mlp(w.mlp)
+    s = ctx.score(dev(ks, x), model).cpu().numpy()
+    assert np.all(np.isfinite(s))
+    assert np.all(np.abs(s - rs) <= TOL_MLP * np.maximum(1, np.abs(rs)))
+    assert np.std(rs) > 1e-2
+
+
+# ---------------------------------------------------------------------------------------------
+# ks_select
+# ---------------------------------------------------------------------------------------------
+
+def check_select(w, idx, sc, tol, sample=None):
+    """Compare [P, k] GPU results with the oracle (all problems, or the sampled ones)."""
+    P = len(w.problems)
+    probs = range(P) if sample is None else sample
+    sel = np.array(list(probs))
+    if w.seg_offsets is None:
+        so = si = None
+        sub_so = None
+    else:
+        so, si = w.seg_offsets, w.seg_index
+    for i in sel:
+        p1 = w.problems[i:i + 1]
+        if so is None:
+            _, _, allsc = oracle.select(p1, w.candidates, w.desc, w.k, gbdt=w.gbdt, mlp=w.mlp, want_scores=True)
+            pool = np.arange(len(w.candidates), dtype=np.int32)
+        else:
+            pool = si[so[i]:so[i + 1]]
+            _, _, allsc = oracle.select(p1, w.candidates, w.desc, w.k, gbdt=w.gbdt, mlp=w.mlp,
+                                        seg_off=np.array([0, len(pool)], np.int64), seg_idx=pool,
+                                        want_scores=True)
+        ok, msg = topk_accept(idx[i], sc[i], allsc, pool, idx.shape[1], tol)
+        assert ok, f"problem {i}: {msg}"
+
+
+def run_select(ks, ctx, w, model, k=None):
+    k = w.k if k is None else k
+    P, C = len(w.problems), len(w.candidates)
+    idx, sc = ctx.select(dev(ks, w.problems), P, dev(ks, w.candidates), C, model, k,
+                         None if w.seg_offsets is None else dev(ks, w.seg_offsets),
+                         None if w.seg_index is None else dev(ks, w.seg_index), w.pairs)
+    torch.cuda.synchronize()
+    return idx.cpu().numpy(), sc.cpu().numpy()
+
+
+def test_select_config0_matches_oracle_exactly(ks, ctx):
+    w = wl.make_workload(0)
+    model = ctx.model_create_gbdt(*w.gbdt)
+    idx, sc = run_select(ks, ctx, w, model)
+    ridx, rsc = oracle.select(w.problems, w.candidates, DESC, w.k, gbdt=w.gbdt)
+    check_select(w, idx, sc, TOL_GBDT)
+    # no tolerance tie occurs in this workload, so the index lists are simply equal
+    assert np.array_equal(idx, ridx)
+    assert np.all(np.abs(sc - rsc) <= TOL_GBDT * np.maximum(1, np.abs(rsc)))
+    idx2, sc2 = run_select(ks, ctx, w, model)
+    assert np.array_equal(idx, idx2) and np.array_equal(sc.view(np.uint32), sc2.view(np.uint32))
+
+
+def test_select_segments_cross_precision(ks, ctx):
+    w = wl.make_workload(2, P=24, seg=3000, trees=60, depth=8)
+    model = ctx.model_create_gbdt(*w.gbdt)
+    idx, sc = run_select(ks, ctx, w, model)
+    check_select(w, idx, sc, TOL_GBDT)
+
+
+def test_select_full_space_shape_small(ks, ctx):
+    w = wl.make_workload(1, P=6, C=5000, trees=50)
+    model = ctx.model_create_gbdt(*w.gbdt)
+    idx, sc = run_select(ks, ctx, w, model)
+    check_select(w, idx, sc, TOL_GBDT)
+    ridx, _ = oracle.select(w.problems, w.candidates, DESC, w.k, gbdt=w.gbdt)
+    assert np.array_equal(idx, ridx)
+
+
+@pytest.mark.parametrize("C,k", [(1, 5), (3, 32), (33, 1), (257, 10), (2049, 32)])
+def test_select_ragged_sizes_and_padding(ks, ctx, C, k):
+    w = wl.make_workload(0, P=3, C=C, trees=9, depth=3)
+    model = ctx.model_create_gbdt(*w.gbdt)
+    idx, sc = run_select(ks, ctx, w, model, k)
+    x = oracle.featurize(w.problems, w.candidates, DESC)
+    s = oracle.score_gbdt(x, *w.gbdt)
+    ridx, rsc = oracle.topk(s, 3, k, rows_per_problem=C)
+    for i in range(3):
+        ok, msg = topk_accept(idx[i], sc[i], s[i * C:(i + 1) * C], np.arange(C, dtype=np.int32), k, TOL_GBDT)
+        assert ok, msg
+    if k > C:
+        assert np.all(idx[:, C:] == -1) and np.all(np.isneginf(sc[:, C:]))
+
+
+def test_select_all_equal_scores_returns_lowest_indices(ks, ctx):
+    nodes = np.zeros(2, wl.NODE_DT)
+    nodes[0] = (0.125, 0xFFFF, 0, 0)
+    nodes[1] = (-0.5, 0xFFFF, 0, 0)
+    prob, cand, _, _ = wl.make_inputs(0, P=4, C=1000)
+    w = wl.Workload("ties", DESC, prob, cand, 7, gbdt=(np.array([0, 1, 2]), nodes, 0.0))
+    model = ctx.model_create_gbdt(*w.gbdt)
+    idx, sc = run_select(ks, ctx, w, model)
+    assert np.array_equal(idx, np.tile(np.arange(7, dtype=np.int32), (4, 1)))
+    assert np.all(sc == np.float32(-0.375))
+
+
+def test_select_empty_and_uneven_segments(ks, ctx):
+    w = wl.make_workload(2, P=5, seg=1, trees=12, depth=4)
+    w.seg_offsets = np.array([0, 0, 600, 601, 601, 5300], np.int64)
+    w.seg_index = np.concatenate([np.sort(np.random.default_rng(i).choice(len(w.candidates), n, replace=False))
+                                  for i, n in enumerate([0, 600, 1, 0, 4699])]).astype(np.int32)
+    model = ctx.model_create_gbdt(*w.gbdt)
+    idx, sc = run_select(ks, ctx, w, model)
+    assert np.all(idx[0] == -1) and np.all(idx[3] == -1) and np.all(np.isneginf(sc[0]))
+    assert idx[2, 0] == w.seg_index[600] and np.all(idx[2, 1:] == -1)
+    check_select(w, idx, sc, TOL_GBDT)
+
+
+def test_select_mlp(ks, ctx):
+    w = wl.make_workload(4, P=3, C=1500)
+    model = ctx.model_create_mlp(w.mlp)
+    idx, sc = run_select(ks, ctx, w, model)
+    check_select(w, idx, sc, TOL_MLP)
+
+
+def test_select_one_and_select_host_agree_with_select(ks, ctx):
+    w = wl.make_workload(3, P=4, C=3000, trees=30)
+    model = ctx.model_create_gbdt(*w.gbdt)
+    idx, sc = run_select(ks, ctx, w, model)
+    d_c = dev(ks, w.candidates)
+    for i in range(4):
+        hi, hs = ctx.select_one(w.problems[i:i + 1], d_c, len(w.candidates), model, w.k)
+        assert np.array_equal(hi.numpy(), idx[i]) and np.array_equal(hs.numpy(), sc[i])
+    hi, hs = ctx.select_host(w.problems, 4, w.candidates, len(w.candidates), model, w.k)
+    assert np.array_equal(hi.numpy(), idx) and np.array_equal(hs.numpy(), sc)
+    check_select(w, idx, sc, TOL_GBDT)
+    w2 = wl.make_workload(2, P=6, seg=500, trees=10, depth=5)
+    model2 = ctx.model_create_gbdt(*w2.gbdt)
+    idx2, sc2 = run_select(ks, ctx, w2, model2)
+    hi, hs = ctx.select_host(w2.problems, 6, w2.candidates, len(w2.candidates), model2, w2.k,
+                             w2.seg_offsets, w2.seg_index, w2.pairs)
+    assert np.array_equal(hi.numpy(), idx2) and np.array_equal(hs.numpy(), sc2)
+
+
+# ---------------------------------------------------------------------------------------------
+# host-side error behaviour (status codes, never a fault)
+# ---------------------------------------------------------------------------------------------
+
+def test_invalid_arguments_return_status_codes(ks, ctx):
+    w = wl.make_workload(0, P=2, C=64, trees=3, depth=2)
+    model = ctx.model_create_gbdt(*w.gbdt)
+    d_p, d_c = dev(ks, w.problems), dev(ks, w.candidates)
+    for k in (0, -1, 33):
+        with pytest.raises(ks.KsError) as e:
+            ctx.select(d_p, 2, d_c, 64, model, k)
+        assert e.value.status == ks.KS_ERR_INVALID_ARG
+    with pytest.raises(ks.KsError):
+        ctx.select(d_p, 2, d_c, 64, model, 5, pairs=127)  # pairs must equal P*C
+    with pytest.raises(ks.KsError):
+        ctx.select(None, 2, d_c, 64, model, 5)
+    idx, sc = ctx.select(d_p, 0, d_c, 64, model, 5, out_idx=torch.zeros((1, 5), dtype=torch.int32, device="cuda"),
+                         out_score=torch.zeros((1, 5), device="cuda"))  # P = 0 is a no-op
+    bad = w.gbdt[1].copy()
+    bad["feat"][0] = 63
+    with pytest.raises(ks.KsError):
+        ctx.model_create_gbdt(w.gbdt[0], bad)
+    bad = w.gbdt[1].copy()
+    bad["left"][0] = 0  # child index not after its parent
+    with pytest.raises(ks.KsError):
+        ctx.model_create_gbdt(w.gbdt[0], bad)
+    bad = w.gbdt[1].copy()
+    bad["v"][1] = np.nan
+    with pytest.raises(ks.KsError):
+        ctx.model_create_gbdt(w.gbdt[0], bad)
+    bad = w.gbdt[1].copy()
+    bad["left"][1] = 5  # two parents for node 5
+    with pytest.raises(ks.KsError):
+        ctx.model_create_gbdt(w.gbdt[0], bad)
+    m4 = wl.make_workload(4, P=1, C=8).mlp
+    m4["sigma"] = m4["sigma"].copy()
+    m4["sigma"][3] = 0
+    with pytest.raises(ks.KsError):
+        ctx.model_create_mlp(m4)
+    with pytest.raises(ks.KsError):
+        ctx.select_one(problem(0, 5, 5), d_c, 64, model, 5)
