@@ -1,0 +1,323 @@
+"""Benchmark of the selection hot path: (problem, candidate) pairs ranked per second through
+the fused featurize + score + top-k call, on seeded synthetic inputs shaped like the paper's
+full configuration space (1,024 problems x 60,000 candidates, 500 trees of depth 8, top-10).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload 1]
+
+One step = one pass of the whole path over the batch. With N > 1 (torchrun) every rank ranks
+its own batch of problems (no data-path collective; weak scaling) and rank 0 prints the line.
+`--impl reference` times the CPU oracle on a bounded sample of the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "problem x candidate pairs ranked/sec (fused featurize+score+top-k)"
+UNIT = "pairs/s"
+# Issue-rate roofline of the tree walk: 148 SMs x 4 schedulers x 32 lanes x 1.965 GHz
+# thread-instructions per second, 4 thread-instructions per node visit.
+ISSUE_PEAK = 148 * 4 * 32 * 1.965e9
+INSTR_PER_VISIT = 4
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            d = json.load(fh)
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained"), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples during the timed region (read-only query)."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.QUERY}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            f = [x.strip() for x in r.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": float(max(smax)) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def workload_config(cfg: int):
+    from paper_2609_35587_b200 import workloads as wl
+    spec = wl.CONFIGS[cfg]
+    return spec
+
+
+def run_reference(args, rank, world):
+    """CPU-oracle arm: each step ranks a bounded sample of the workload on the host cores."""
+    if rank != 0:
+        return
+    import oracle
+    from paper_2609_35587_b200 import workloads as wl
+    cfg = args.workload
+    spec = wl.CONFIGS[cfg]
+    cores = oracle.threads()
+    w = wl.make_workload(cfg, P=max(2, min(spec["P"], args.ref_problems)))
+    kw = dict(gbdt=w.gbdt, mlp=w.mlp, seg_off=w.seg_offsets, seg_idx=w.seg_index)
+    for _ in range(args.warmup):
+        oracle.select(w.problems[:1], w.candidates, w.desc, w.k, gbdt=w.gbdt, mlp=w.mlp,
+                      seg_off=None if w.seg_offsets is None else w.seg_offsets[:2],
+                      seg_idx=w.seg_index)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.select(w.problems, w.candidates, w.desc, w.k, **kw)
+    dt = (time.perf_counter() - t0) / args.steps
+    value = w.pairs / dt
+    sample = f"{len(w.problems)} problems x {w.pairs // len(w.problems)} candidates per step"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic", "config": config_dict(cfg, spec, args),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def config_dict(cfg, spec, args):
+    d = {"workload": f"config {cfg} ({spec['name']})", "problems": spec["P"],
+         "candidates_per_problem": spec["seg"] or spec["C"], "k": spec["k"],
+         "l2": "flushed between steps (256 MiB write)"}
+    if spec["trees"]:
+        d.update(scorer="gbdt", trees=spec["trees"], depth=spec["depth"])
+    else:
+        d.update(scorer="mlp 64-256-256-1 bf16")
+    return d
+
+
+def cpu_baseline(cfg, budget_s=15.0):
+    """The oracle as it stands on this machine's host cores, on a bounded sample of the workload."""
+    import oracle
+    from paper_2609_35587_b200 import workloads as wl
+    spec = wl.CONFIGS[cfg]
+    cores = oracle.threads()
+    probe_p = max(1, min(cores, spec["P"]))
+    w = wl.make_workload(cfg, P=max(probe_p, 2))
+    kw = dict(gbdt=w.gbdt, mlp=w.mlp)
+
+    def run(n):
+        so = None if w.seg_offsets is None else w.seg_offsets[:n + 1]
+        t0 = time.perf_counter()
+        oracle.select(w.problems[:n], w.candidates, w.desc, w.k, seg_off=so, seg_idx=w.seg_index, **kw)
+        return time.perf_counter() - t0
+
+    per = w.pairs // len(w.problems)
+    t_probe = run(probe_p)
+    n = int(max(probe_p, min(spec["P"], probe_p * budget_s / max(t_probe, 1e-3))))
+    n = max(cores, n // cores * cores)
+    if n > len(w.problems):
+        w = wl.make_workload(cfg, P=n)
+    dt = run(n)
+    return {"value": n * per / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"first {n} problems x {per} candidates of the workload, {dt:.1f} s"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=1, choices=[0, 1, 2, 4])
+    ap.add_argument("--ref-problems", type=int, default=16)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2609_35587_b200 import binding as ks
+    from paper_2609_35587_b200 import workloads as wl
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    cfg = args.workload
+    spec = wl.CONFIGS[cfg]
+    # weak scaling: every rank ranks its own batch of problems against the shared catalogue
+    w = wl.make_workload(cfg, seed=wl.BASE_SEED) if rank == 0 else None
+    if rank != 0:
+        w = wl.make_workload(cfg, seed=wl.BASE_SEED)
+        w.problems = wl.make_inputs(cfg, seed=wl.BASE_SEED + 7919 * rank)[0]
+    P, C, k = len(w.problems), len(w.candidates), w.k
+    ctx = ks.Context(w.desc, local_rank)
+    model = ctx.model_create_gbdt(*w.gbdt) if w.gbdt is not None else ctx.model_create_mlp(w.mlp)
+    d_p, d_c = ks.to_device(w.problems, dev), ks.to_device(w.candidates, dev)
+    d_so = None if w.seg_offsets is None else ks.to_device(w.seg_offsets, dev)
+    d_si = None if w.seg_index is None else ks.to_device(w.seg_index, dev)
+    out_idx = torch.empty((P, k), dtype=torch.int32, device=dev)
+    out_sc = torch.empty((P, k), dtype=torch.float32, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    pairs = w.pairs
+
+    def step():
+        ctx.select(d_p, P, d_c, C, model, k, d_so, d_si, pairs, out_idx, out_sc)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+
+    # ---- device-resident timing: K steps, each bracketed by events, L2 flushed in between ----
+    ctx.profile_enable(True)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    launches0 = ctx.launch_count()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+          for _ in range(args.steps)]
+    kern_ms = []
+    barrier()
+    for i in range(args.steps):
+        flush.fill_(i & 0xFF)
+        ev[i][0].record()
+        step()
+        ev[i][1].record()
+        kern_ms.append(ctx.profile_last_ms())
+    barrier()
+    launches = ctx.launch_count() - launches0
+    clocks = sampler.stop()
+    step_ms = [a.elapsed_time(b) for a, b in ev]
+    total_ms = float(sum(step_ms))
+    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * pairs / (ms_per_step * 1e-3)
+
+    # ---- end to end: host buffers in, host results out, through the C ABI ------------------------
+    h_p = torch.from_numpy(w.problems.view(np.uint8).reshape(P, 16).copy()).pin_memory()
+    h_c = torch.from_numpy(w.candidates.view(np.uint8).reshape(C, 16).copy()).pin_memory()
+    h_so = None if w.seg_offsets is None else torch.from_numpy(w.seg_offsets.copy()).pin_memory()
+    h_si = None if w.seg_index is None else torch.from_numpy(w.seg_index.copy()).pin_memory()
+    h_idx = torch.empty((P, k), dtype=torch.int32).pin_memory()
+    h_sc = torch.empty((P, k), dtype=torch.float32).pin_memory()
+    ctx.profile_enable(False)
+    for _ in range(2):
+        ctx.select_host(h_p, P, h_c, C, model, k, h_so, h_si, pairs, h_idx, h_sc)
+    barrier()
+    e2e_steps = max(3, min(args.steps, 10))
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        ctx.select_host(h_p, P, h_c, C, model, k, h_so, h_si, pairs, h_idx, h_sc)
+    barrier()
+    e2e_s = (time.perf_counter() - t0) / e2e_steps
+    t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_value = world * pairs / float(t.item())
+    h2d = P * 16 + C * 16 + (0 if h_so is None else h_so.numel() * 8 + h_si.numel() * 4)
+    d2h = P * k * 8
+
+    if rank == 0:
+        peaks = load_peaks()
+        kms = float(np.mean(kern_ms))
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "data": "synthetic",
+                "config": config_dict(cfg, spec, args), "clocks": clocks, "gpu_launches": int(launches),
+                "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+                        "d2h_bytes_per_step": int(d2h)}}
+        if w.gbdt is not None:
+            visits = pairs * spec["trees"] * spec["depth"]
+            achieved = visits * INSTR_PER_VISIT / (kms * 1e-3)
+            line["dtype"] = "f32"
+            line["roofline"] = {"bound": "alu", "kernel": "fused featurize+gbdt+top-k",
+                                "achieved": achieved / 1e12, "peak": ISSUE_PEAK / 1e12,
+                                "unit": "T thread-instr/s (4 per node visit)",
+                                "frac": achieved / ISSUE_PEAK, "kernel_ms": kms,
+                                "peak_source": "derived: 148 SMs x 4 schedulers x 32 lanes x 1.965 GHz",
+                                "traffic": TRAFFIC_BYTES.get(cfg)}
+        else:
+            flops = pairs * 2.0 * (64 * 256 + 256 * 256)
+            achieved = flops / (kms * 1e-3)
+            line["dtype"] = "bf16"
+            line["roofline"] = {"bound": "tensor", "kernel": "fused featurize+mlp+top-k",
+                                "achieved": achieved / 1e12, "peak": peaks["bf16_tflops_sustained"],
+                                "unit": "TFLOP/s", "frac": achieved / 1e12 / peaks["bf16_tflops_sustained"],
+                                "kernel_ms": kms, "peak_source": peaks["source"] + " (sustained bf16)",
+                                "traffic": TRAFFIC_BYTES.get(cfg)}
+        if not args.no_cpu_baseline and world == 1:
+            line["cpu_baseline"] = cpu_baseline(cfg)
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, per launch, from the
+# ncu summaries under profiles/ (None until a capture exists for that workload).
+TRAFFIC_BYTES = {}
+
+if __name__ == "__main__":
+    main()

@@ -187,6 +187,12 @@ int ks_feature_count(void);             /* KS_F                                 
 const char* ks_feature_name(int index); /* NULL if index is outside 0..KS_F-1              */
 /* Number of kernels libks launched on behalf of this context since creation. */
 int64_t ks_launch_count(const ks_ctx* ctx);
+/* Measurement aid (the paper has no counterpart): with profiling on, every ks_select records a
+ * CUDA event on the caller's stream before and after its dominant kernel (the fused
+ * featurize + score + partial top-k kernel, excluding the small merge that follows).
+ * ks_profile_last_ms waits for the last such kernel and returns its duration. */
+ks_status ks_profile_enable(ks_ctx* ctx, int on);
+ks_status ks_profile_last_ms(ks_ctx* ctx, float* out_ms);
 
 #ifdef __cplusplus
 }

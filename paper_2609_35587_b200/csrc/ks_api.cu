@@ -188,6 +188,8 @@ ks_status ks_create(ks_ctx** out_ctx, int cuda_device, const ks_gpu_desc* desc) 
 ks_status ks_destroy(ks_ctx* ctx) {
   if (!ctx) return KS_OK;
   DeviceGuard g(ctx->device);
+  if (ctx->ev_begin) cudaEventDestroy(ctx->ev_begin);
+  if (ctx->ev_end) cudaEventDestroy(ctx->ev_end);
   cudaFree(ctx->ws);
   cudaFreeHost(ctx->pinned);
   delete ctx;
@@ -197,6 +199,27 @@ ks_status ks_destroy(ks_ctx* ctx) {
 const char* ks_last_cuda_error(const ks_ctx* ctx) { return ctx ? ctx->err : ""; }
 
 int64_t ks_launch_count(const ks_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+ks_status ks_profile_enable(ks_ctx* ctx, int on) {
+  if (!ctx) return KS_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  if (on && !ctx->ev_begin) {
+    cudaError_t e = cudaEventCreate(&ctx->ev_begin);
+    if (e == cudaSuccess) e = cudaEventCreate(&ctx->ev_end);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "ks_profile_enable");
+  }
+  ctx->profile = on != 0;
+  ctx->profile_valid = false;
+  return KS_OK;
+}
+
+ks_status ks_profile_last_ms(ks_ctx* ctx, float* out_ms) {
+  if (!ctx || !out_ms || !ctx->profile_valid) return KS_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  cudaError_t e = cudaEventSynchronize(ctx->ev_end);
+  if (e == cudaSuccess) e = cudaEventElapsedTime(out_ms, ctx->ev_begin, ctx->ev_end);
+  return e == cudaSuccess ? KS_OK : cuda_fail(ctx, e, "ks_profile_last_ms");
+}
 
 ks_status ks_model_create_gbdt(ks_ctx* ctx, int n_trees, const int64_t* h_tree_offsets,
                                const ks_node_host* h_nodes, float base_score, ks_model** out_model) {
@@ -337,7 +360,10 @@ ks_status ks_select(ks_ctx* ctx, const ks_problem* d_p, int P, const ks_candidat
   if (s != KS_OK) return s;
   cudaError_t e = ks::launch_select(ctx->desc, *model, d_p, nullptr, P, d_c, C, d_seg_offsets,
                                     d_seg_index, pairs, k, ctx->ws, d_topk_idx, d_topk_score,
-                                    static_cast<cudaStream_t>(stream), &ctx->launches);
+                                    static_cast<cudaStream_t>(stream), &ctx->launches,
+                                    ctx->profile ? ctx->ev_begin : nullptr,
+                                    ctx->profile ? ctx->ev_end : nullptr);
+  ctx->profile_valid = ctx->profile && e == cudaSuccess;
   return e == cudaSuccess ? KS_OK : cuda_fail(ctx, e, "ks_select");
 }
 

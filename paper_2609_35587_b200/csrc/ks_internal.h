@@ -67,6 +67,10 @@ struct ks_ctx {
   size_t pinned_bytes = 0;
   int64_t launches = 0;
   char err[256] = {0};
+  // optional timing of the dominant kernel of the last ks_select* call (ks_profile_enable)
+  bool profile = false;
+  bool profile_valid = false;
+  cudaEvent_t ev_begin = nullptr, ev_end = nullptr;
 };
 
 struct ks_model {
@@ -104,6 +108,7 @@ cudaError_t launch_select(const ks_gpu_desc& desc, const ks_model& model, const 
                           const ks_problem* p_by_value, int P, const ks_candidate* d_c, int C,
                           const int64_t* d_seg_off, const int32_t* d_seg_idx, int64_t pairs, int k,
                           void* d_partial, int32_t* d_topk_idx, float* d_topk_score,
-                          cudaStream_t stream, int64_t* launches);
+                          cudaStream_t stream, int64_t* launches, cudaEvent_t ev_begin = nullptr,
+                          cudaEvent_t ev_end = nullptr);
 
 }  // namespace ks

@@ -397,7 +397,8 @@ cudaError_t launch_select(const ks_gpu_desc& desc, const ks_model& model, const 
                           const ks_problem* p_by_value, int P, const ks_candidate* d_c, int C,
                           const int64_t* d_seg_off, const int32_t* d_seg_idx, int64_t pairs, int k,
                           void* d_partial, int32_t* d_topk_idx, float* d_topk_score,
-                          cudaStream_t stream, int64_t* launches) {
+                          cudaStream_t stream, int64_t* launches, cudaEvent_t ev_begin,
+                          cudaEvent_t ev_end) {
   if (P == 0) return cudaSuccess;
   const int64_t per = per_problem_rows(P, C, pairs, d_seg_off != nullptr);
   const int st = pick_sub_tiles(P, per);
@@ -407,6 +408,7 @@ cudaError_t launch_select(const ks_gpu_desc& desc, const ks_model& model, const 
   ks_problem pv{};
   if (p_by_value) pv = *p_by_value;
   cudaError_t e;
+  if (ev_begin) cudaEventRecord(ev_begin, stream);
   if (model.kind == 0) {
     const GbdtModel& g = model.gbdt;
     const size_t smem = sizeof(float) * kRow * kBlock;
@@ -428,6 +430,7 @@ cudaError_t launch_select(const ks_gpu_desc& desc, const ks_model& model, const 
   ++*launches;
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
+  if (ev_end) cudaEventRecord(ev_end, stream);
   topk_merge_kernel<<<(P * 32 + kBlock - 1) / kBlock, kBlock, 0, stream>>>(partial, P, map.nblk * k, k,
                                                                           d_topk_idx, d_topk_score);
   ++*launches;
