@@ -187,6 +187,10 @@ int ks_feature_count(void);             /* KS_F                                 
 const char* ks_feature_name(int index); /* NULL if index is outside 0..KS_F-1              */
 /* Number of kernels libks launched on behalf of this context since creation. */
 int64_t ks_launch_count(const ks_ctx* ctx);
+/* Waits for all work of the context's device and reports (then clears) the status word that
+ * kernels set when one of their bounded device-side waits gave up: KS_OK or KS_ERR_TIMEOUT.
+ * ks_select_one and ks_select_host perform this check themselves. */
+ks_status ks_device_status(ks_ctx* ctx);
 /* Measurement aid (the paper has no counterpart): with profiling on, every ks_select records a
  * CUDA event on the caller's stream before and after its dominant kernel (the fused
  * featurize + score + partial top-k kernel, excluding the small merge that follows).

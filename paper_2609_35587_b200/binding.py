@@ -21,7 +21,7 @@ KS_OK, KS_ERR_INVALID_ARG, KS_ERR_UNSUPPORTED, KS_ERR_CUDA, KS_ERR_TIMEOUT, KS_E
 EXPORTS = ("ks_create", "ks_destroy", "ks_last_cuda_error", "ks_model_create_gbdt",
            "ks_model_create_mlp", "ks_model_destroy", "ks_featurize", "ks_score", "ks_select",
            "ks_select_one", "ks_select_host", "ks_status_string", "ks_feature_count",
-           "ks_feature_name", "ks_launch_count", "ks_profile_enable", "ks_profile_last_ms")
+           "ks_feature_name", "ks_launch_count", "ks_profile_enable", "ks_profile_last_ms", "ks_device_status")
 
 
 class KsError(RuntimeError):
@@ -63,6 +63,7 @@ def _load() -> ctypes.CDLL:
     lib.ks_launch_count.argtypes = [vp]
     lib.ks_launch_count.restype = i64
     lib.ks_profile_enable.argtypes = [vp, i32]
+    lib.ks_device_status.argtypes = [vp]
     lib.ks_profile_last_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     for name in EXPORTS:
         fn = getattr(lib, name)
@@ -166,6 +167,9 @@ class Context:
 
     def launch_count(self) -> int:
         return int(_lib.ks_launch_count(self._h))
+
+    def device_status(self) -> int:
+        return int(_lib.ks_device_status(self._h))
 
     def profile_enable(self, on: bool = True):
         self._check(_lib.ks_profile_enable(self._h, int(on)), "ks_profile_enable")

@@ -59,6 +59,16 @@ ks_status ensure_workspace(ks_ctx* ctx, size_t bytes) {
   return KS_OK;
 }
 
+// Reads (and clears) the device status word; the stream must have been synchronised.
+ks_status read_status(ks_ctx* ctx) {
+  const int v = *static_cast<volatile int*>(ctx->h_status);
+  if (v != 0) {
+    *ctx->h_status = 0;
+    return static_cast<ks_status>(v);
+  }
+  return KS_OK;
+}
+
 inline size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
 
 template <typename T>
@@ -110,11 +120,9 @@ void free_model(ks_model* m) {
   cudaFree(m->gbdt.d_nodes);
   cudaFree(m->gbdt.d_roots);
   cudaFree(m->gbdt.d_qnodes);
-  cudaFree(m->gbdt.d_qleaves);
-  cudaFree(m->gbdt.d_qleaf_node);
   cudaFree(m->gbdt.d_qthr);
-  cudaFree(m->gbdt.d_qrow_feat);
-  cudaFree(m->gbdt.d_qrow_count);
+  cudaFree(m->gbdt.d_qrow0);
+  cudaFree(m->gbdt.d_qrowcnt);
   for (int l = 0; l < KS_MLP_MAX_LAYERS; ++l) {
     cudaFree(m->mlp.d_w[l]);
     cudaFree(m->mlp.d_b[l]);
@@ -176,7 +184,17 @@ ks_status ks_create(ks_ctx** out_ctx, int cuda_device, const ks_gpu_desc* desc) 
     return KS_ERR_OOM;
   }
   ks_status s = ensure_workspace(ctx, 1u << 20);
+  // status word in mapped pinned host memory: kernels write it through d_status, the host
+  // reads h_status after a synchronisation without issuing a copy
+  if (s == KS_OK && (cudaHostAlloc(reinterpret_cast<void**>(&ctx->h_status), sizeof(int), cudaHostAllocMapped) != cudaSuccess ||
+                     cudaHostGetDevicePointer(reinterpret_cast<void**>(&ctx->d_status), ctx->h_status, 0) != cudaSuccess)) {
+    cudaGetLastError();
+    s = KS_ERR_OOM;
+  }
+  if (s == KS_OK) *ctx->h_status = 0;
   if (s != KS_OK) {
+    cudaFree(ctx->ws);
+    if (ctx->h_status) cudaFreeHost(ctx->h_status);
     cudaFreeHost(ctx->pinned);
     delete ctx;
     return s;
@@ -191,6 +209,7 @@ ks_status ks_destroy(ks_ctx* ctx) {
   if (ctx->ev_begin) cudaEventDestroy(ctx->ev_begin);
   if (ctx->ev_end) cudaEventDestroy(ctx->ev_end);
   cudaFree(ctx->ws);
+  cudaFreeHost(ctx->h_status);
   cudaFreeHost(ctx->pinned);
   delete ctx;
   return KS_OK;
@@ -199,6 +218,14 @@ ks_status ks_destroy(ks_ctx* ctx) {
 const char* ks_last_cuda_error(const ks_ctx* ctx) { return ctx ? ctx->err : ""; }
 
 int64_t ks_launch_count(const ks_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+ks_status ks_device_status(ks_ctx* ctx) {
+  if (!ctx) return KS_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "ks_device_status");
+  return read_status(ctx);
+}
 
 ks_status ks_profile_enable(ks_ctx* ctx, int on) {
   if (!ctx) return KS_ERR_INVALID_ARG;
@@ -360,7 +387,7 @@ ks_status ks_select(ks_ctx* ctx, const ks_problem* d_p, int P, const ks_candidat
   if (s != KS_OK) return s;
   cudaError_t e = ks::launch_select(ctx->desc, *model, d_p, nullptr, P, d_c, C, d_seg_offsets,
                                     d_seg_index, pairs, k, ctx->ws, d_topk_idx, d_topk_score,
-                                    static_cast<cudaStream_t>(stream), &ctx->launches,
+                                    static_cast<cudaStream_t>(stream), &ctx->launches, ctx->d_status,
                                     ctx->profile ? ctx->ev_begin : nullptr,
                                     ctx->profile ? ctx->ev_end : nullptr);
   ctx->profile_valid = ctx->profile && e == cudaSuccess;
@@ -384,7 +411,7 @@ ks_status ks_select_one(ks_ctx* ctx, ks_problem p, const ks_candidate* d_c, int 
   int32_t* d_idx = reinterpret_cast<int32_t*>(base + part);
   float* d_sc = reinterpret_cast<float*>(base + part + align_up(k * sizeof(int32_t)));
   cudaError_t e = ks::launch_select(ctx->desc, *model, nullptr, &p, 1, d_c, C, nullptr, nullptr, C, k,
-                                    ctx->ws, d_idx, d_sc, st, &ctx->launches);
+                                    ctx->ws, d_idx, d_sc, st, &ctx->launches, ctx->d_status);
   int32_t* pin_idx = static_cast<int32_t*>(ctx->pinned);
   float* pin_sc = reinterpret_cast<float*>(pin_idx + KS_MAX_K);
   if (e == cudaSuccess) e = cudaMemcpyAsync(pin_idx, d_idx, k * sizeof(int32_t), cudaMemcpyDeviceToHost, st);
@@ -393,7 +420,7 @@ ks_status ks_select_one(ks_ctx* ctx, ks_problem p, const ks_candidate* d_c, int 
   if (e != cudaSuccess) return cuda_fail(ctx, e, "ks_select_one");
   std::memcpy(h_topk_idx, pin_idx, k * sizeof(int32_t));
   std::memcpy(h_topk_score, pin_sc, k * sizeof(float));
-  return KS_OK;
+  return read_status(ctx);
 }
 
 ks_status ks_select_host(ks_ctx* ctx, const ks_problem* h_p, int P, const ks_candidate* h_c, int C,
@@ -429,11 +456,11 @@ ks_status ks_select_host(ks_ctx* ctx, const ks_problem* h_p, int P, const ks_can
   if (e == cudaSuccess && seg && pairs > 0) e = cudaMemcpyAsync(d_si, h_seg_index, sizeof(int32_t) * pairs, cudaMemcpyHostToDevice, st);
   if (e == cudaSuccess)
     e = ks::launch_select(ctx->desc, *model, d_p, nullptr, P, d_c, C, d_so, d_si, pairs, k, ctx->ws, d_oi,
-                          d_os, st, &ctx->launches);
+                          d_os, st, &ctx->launches, ctx->d_status);
   if (e == cudaSuccess) e = cudaMemcpyAsync(h_topk_idx, d_oi, sizeof(int32_t) * P * k, cudaMemcpyDeviceToHost, st);
   if (e == cudaSuccess) e = cudaMemcpyAsync(h_topk_score, d_os, sizeof(float) * P * k, cudaMemcpyDeviceToHost, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
-  return e == cudaSuccess ? KS_OK : cuda_fail(ctx, e, "ks_select_host");
+  return e == cudaSuccess ? read_status(ctx) : cuda_fail(ctx, e, "ks_select_host");
 }
 
 }  // extern "C"

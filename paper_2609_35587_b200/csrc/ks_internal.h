@@ -24,16 +24,17 @@ struct GbdtModel {
   float base = 0.0f;
   DevNode* d_nodes = nullptr;  // all trees back to back
   int* d_roots = nullptr;      // [n_trees + 1] offsets into d_nodes
-  // quantised fast form (complete trees in level order), see ks_gbdt_fast.cu
+  // quantised fast form (complete trees, chunked level-order layout), see ks_gbdt_fast.cu
   bool fast = false;
   int fast_depth = 0;          // every tree padded to this depth
-  int n_qrows = 0;             // quantised feature rows (pseudo-features)
-  uint32_t* d_qnodes = nullptr;    // [n_trees][2^D - 1] packed (row offset, bin)
-  float* d_qleaves = nullptr;      // [n_trees][2^D]
-  uint16_t* d_qleaf_node = nullptr;  // [n_trees][2^D] original node index of each padded leaf
-  float* d_qthr = nullptr;         // [n_qrows][256] sorted thresholds (padded with +inf)
-  int* d_qrow_feat = nullptr;      // [n_qrows] source feature column of each row
-  int* d_qrow_count = nullptr;     // [n_qrows] number of thresholds in the row
+  int n_qrows = 0;             // quantised feature rows (a feature, or a 255-threshold slice)
+  int tpc = 0;                 // trees per chunk
+  int n_chunks = 0;
+  int chunk_bytes = 0;
+  uint32_t* d_qnodes = nullptr;  // [n_chunks][chunk_bytes / 4]
+  float* d_qthr = nullptr;       // [n_qrows][256] sorted thresholds padded with +inf
+  uint8_t* d_qrow0 = nullptr;    // [64] first row of each feature column
+  uint8_t* d_qrowcnt = nullptr;  // [64] rows of each feature column
 };
 
 struct MlpModel {
@@ -65,6 +66,8 @@ struct ks_ctx {
   size_t ws_bytes = 0;
   void* pinned = nullptr;  // host staging for ks_select_one results
   size_t pinned_bytes = 0;
+  int* h_status = nullptr;  // status word (mapped pinned host memory) set by kernels whose
+  int* d_status = nullptr;  // bounded waits give up; d_status is its device alias
   int64_t launches = 0;
   char err[256] = {0};
   // optional timing of the dominant kernel of the last ks_select* call (ks_profile_enable)
@@ -84,10 +87,21 @@ namespace ks {
 
 constexpr int kBlock = 256;            // threads per block of the pair kernels
 constexpr int kSubTilesMax = 8;        // sub-tiles of kBlock rows one block ranks
+constexpr int kFastThreads = 512;      // threads per block of the quantised tree kernel
+constexpr int kFastR = 4;              // candidates per thread there
+constexpr int kFastRows = kFastThreads * kFastR;
+constexpr int kFastMaxDepth = 10;
 
 // Builds the quantised fast form of a validated ensemble when it qualifies (m.fast).
 cudaError_t build_fast_gbdt(GbdtModel& m, int n_trees, const int64_t* h_tree_offsets,
                             const ks_node_host* h_nodes);
+
+// Quantised tree path: blocks per problem for `per_problem` rows, and the launch itself.
+void fast_tiling(int P, int64_t per_problem, int* nblk, int* rows_per_cta);
+cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, const ks_problem* d_p,
+                               const ks_problem* p_by_value, int P, const ks_candidate* d_c, int C,
+                               int nblk, int rows_per_cta, const int64_t* seg_off, const int32_t* seg_idx,
+                               int k, unsigned long long* partial, int* status, cudaStream_t stream);
 
 // ---- launchers (each enqueues on `stream`, returns the cudaError of the launch) -----------
 cudaError_t launch_featurize(const ks_gpu_desc& desc, const ks_problem* d_p, int P,
@@ -108,7 +122,7 @@ cudaError_t launch_select(const ks_gpu_desc& desc, const ks_model& model, const 
                           const ks_problem* p_by_value, int P, const ks_candidate* d_c, int C,
                           const int64_t* d_seg_off, const int32_t* d_seg_idx, int64_t pairs, int k,
                           void* d_partial, int32_t* d_topk_idx, float* d_topk_score,
-                          cudaStream_t stream, int64_t* launches, cudaEvent_t ev_begin = nullptr,
-                          cudaEvent_t ev_end = nullptr);
+                          cudaStream_t stream, int64_t* launches, int* d_status,
+                          cudaEvent_t ev_begin = nullptr, cudaEvent_t ev_end = nullptr);
 
 }  // namespace ks

@@ -385,8 +385,12 @@ static int64_t per_problem_rows(int P, int C, int64_t pairs, bool segmented) {
 }
 
 size_t select_partial_bytes(const ks_model& model, int P, int C, int64_t pairs, bool segmented, int k) {
-  (void)model;
   const int64_t per = per_problem_rows(P, C, pairs, segmented);
+  if (model.kind == 0 && model.gbdt.fast) {
+    int nblk, rows;
+    fast_tiling(P, per, &nblk, &rows);
+    return static_cast<size_t>(P) * nblk * k * sizeof(unsigned long long);
+  }
   const int st = pick_sub_tiles(P, per);
   int64_t nblk = (per + static_cast<int64_t>(st) * kBlock - 1) / (static_cast<int64_t>(st) * kBlock);
   if (nblk < 1) nblk = 1;
@@ -397,10 +401,25 @@ cudaError_t launch_select(const ks_gpu_desc& desc, const ks_model& model, const 
                           const ks_problem* p_by_value, int P, const ks_candidate* d_c, int C,
                           const int64_t* d_seg_off, const int32_t* d_seg_idx, int64_t pairs, int k,
                           void* d_partial, int32_t* d_topk_idx, float* d_topk_score,
-                          cudaStream_t stream, int64_t* launches, cudaEvent_t ev_begin,
+                          cudaStream_t stream, int64_t* launches, int* d_status, cudaEvent_t ev_begin,
                           cudaEvent_t ev_end) {
   if (P == 0) return cudaSuccess;
   const int64_t per = per_problem_rows(P, C, pairs, d_seg_off != nullptr);
+  if (model.kind == 0 && model.gbdt.fast) {
+    int nblk, rows;
+    fast_tiling(P, per, &nblk, &rows);
+    unsigned long long* part = static_cast<unsigned long long*>(d_partial);
+    if (ev_begin) cudaEventRecord(ev_begin, stream);
+    cudaError_t e = launch_select_fast(desc, model.gbdt, d_p, p_by_value, P, d_c, C, nblk, rows, d_seg_off,
+                                       d_seg_idx, k, part, d_status, stream);
+    ++*launches;
+    if (e != cudaSuccess) return e;
+    if (ev_end) cudaEventRecord(ev_end, stream);
+    topk_merge_kernel<<<(P * 32 + kBlock - 1) / kBlock, kBlock, 0, stream>>>(part, P, nblk * k, k, d_topk_idx,
+                                                                            d_topk_score);
+    ++*launches;
+    return cudaGetLastError();
+  }
   const int st = pick_sub_tiles(P, per);
   const PairMap map = make_map(P, C, pairs, d_seg_off, d_seg_idx, st * kBlock);
   unsigned long long* partial = static_cast<unsigned long long*>(d_partial);
