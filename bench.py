@@ -134,7 +134,7 @@ def run_reference(args, rank, world):
 
 
 def config_dict(cfg, spec, args):
-    d = {"workload": f"config {cfg} ({spec['name']})", "problems": spec["P"],
+    d = {"workload": f"config {cfg} ({spec['name']})", "problems": args.problems or spec["P"],
          "candidates_per_problem": spec["seg"] or spec["C"], "k": spec["k"],
          "l2": "flushed between steps (256 MiB write)"}
     if spec["trees"]:
@@ -180,6 +180,9 @@ def main():
     ap.add_argument("--workload", type=int, default=1, choices=[0, 1, 2, 4])
     ap.add_argument("--ref-problems", type=int, default=16)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--problems", type=int, default=None,
+                    help="profiling aid: rank only the first N problems of the workload (not a bench line)")
+    ap.add_argument("--skip-e2e", action="store_true", help="profiling aid: skip the host-buffer leg")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -202,10 +205,9 @@ def main():
     cfg = args.workload
     spec = wl.CONFIGS[cfg]
     # weak scaling: every rank ranks its own batch of problems against the shared catalogue
-    w = wl.make_workload(cfg, seed=wl.BASE_SEED) if rank == 0 else None
+    w = wl.make_workload(cfg, P=args.problems, seed=wl.BASE_SEED)
     if rank != 0:
-        w = wl.make_workload(cfg, seed=wl.BASE_SEED)
-        w.problems = wl.make_inputs(cfg, seed=wl.BASE_SEED + 7919 * rank)[0]
+        w.problems = wl.make_inputs(cfg, P=args.problems, seed=wl.BASE_SEED + 7919 * rank)[0]
     P, C, k = len(w.problems), len(w.candidates), w.k
     ctx = ks.Context(w.desc, local_rank)
     model = ctx.model_create_gbdt(*w.gbdt) if w.gbdt is not None else ctx.model_create_mlp(w.mlp)
@@ -225,7 +227,8 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
+    n_warm = args.warmup if args.problems else max(args.warmup, 3)
+    for _ in range(n_warm):
         step()
     barrier()
 
@@ -264,15 +267,15 @@ def main():
     h_idx = torch.empty((P, k), dtype=torch.int32).pin_memory()
     h_sc = torch.empty((P, k), dtype=torch.float32).pin_memory()
     ctx.profile_enable(False)
-    for _ in range(2):
+    e2e_steps = 0 if args.skip_e2e else max(3, min(args.steps, 10))
+    for _ in range(0 if args.skip_e2e else 2):
         ctx.select_host(h_p, P, h_c, C, model, k, h_so, h_si, pairs, h_idx, h_sc)
     barrier()
-    e2e_steps = max(3, min(args.steps, 10))
     t0 = time.perf_counter()
     for _ in range(e2e_steps):
         ctx.select_host(h_p, P, h_c, C, model, k, h_so, h_si, pairs, h_idx, h_sc)
     barrier()
-    e2e_s = (time.perf_counter() - t0) / e2e_steps
+    e2e_s = (time.perf_counter() - t0) / max(e2e_steps, 1)
     t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
     if world > 1:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -284,7 +287,7 @@ def main():
         peaks = load_peaks()
         kms = float(np.mean(kern_ms))
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-                "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+                "warmup": n_warm, "ms_per_step": ms_per_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "data": "synthetic",
                 "config": config_dict(cfg, spec, args), "clocks": clocks, "gpu_launches": int(launches),
                 "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d),

@@ -35,8 +35,9 @@ namespace {
 constexpr int kBufBytes = 32 * 1024;  // one tree-chunk buffer
 constexpr int kMaxRows = 64;          // quantised rows the kernel supports
 constexpr int kThrPerRow = 256;       // 255 thresholds + padding
-constexpr int kRowStride = kFastThreads * 4;  // bytes between rows of the tile
+constexpr int kRowStride = kFastRows;  // bytes between rows of the tile (one byte per candidate)
 constexpr int kSpinLimit = 1 << 22;
+constexpr int kTreesInFlight = 2;     // trees walked concurrently per candidate (tpc is a multiple of 4)
 
 // ---- shared memory map (byte offsets from the dynamic shared base) ----------------------
 constexpr int kOffBuf0 = 0;
@@ -89,6 +90,16 @@ __device__ __forceinline__ float lds_f32(uint32_t addr) {
   float v;
   asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
   return v;
+}
+
+// Byte offset, inside one row of the tile, of a thread's first candidate. A 32-bit word
+// holds four candidates and consecutive lanes of a warp own consecutive words, so a warp's
+// byte loads of any mix of rows touch 32 distinct banks.
+__device__ __forceinline__ int slot_offset(int tid) {
+  constexpr int kWords = kFastRows / 4;            // words per row
+  constexpr int kPerWord = 4 / kFastR;             // threads sharing a word
+  static_assert(kFastThreads == kWords * kPerWord, "tile geometry");
+  return (tid % kWords) * 4 + (tid / kWords) * kFastR;
 }
 
 struct FastView {
@@ -159,7 +170,7 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
       if (row < stop) {
         const int ci = seg_off ? seg_idx[lo + row] : static_cast<int>(row);
         const ks_candidate cand = c[ci];
-        unsigned char* my = tile + tid * 4 + r;
+        unsigned char* my = tile + slot_offset(tid) + r;
         featurize_pair(s_pt, cand, desc, [&](int col, float v) {
           const int r0 = s_row0[col], rc = s_rowcnt[col];
           for (int q = 0; q < rc; ++q) {
@@ -186,12 +197,9 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
       }
     }
     float score[kFastR];
-    uint32_t cbase[kFastR];
 #pragma unroll
-    for (int r = 0; r < kFastR; ++r) {
-      score[r] = fv.base;
-      cbase[r] = sbase + kOffTile + tid * 4 + r;
-    }
+    for (int r = 0; r < kFastR; ++r) score[r] = fv.base;
+    const uint32_t cb = sbase + kOffTile + slot_offset(tid);
     const int tpc = fv.tpc;
 #pragma unroll 1
     for (int ch = 0; ch < fv.n_chunks; ++ch) {
@@ -204,25 +212,40 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
       }
       if (b) phase1 ^= 1; else phase0 ^= 1;
       const uint32_t buf = sbase + (b ? kOffBuf1 : kOffBuf0);
-      const uint32_t leaves = buf + tpc * ((1 << D) - 1) * 4;
+      // With A_l the shared address of a walk's node at level l (levels stored back to back,
+      // [level][tree][node]), A_{l+1} = 2 A_l + (4 tpc - buf) + 4 bit for every level, and
+      // after D steps the address points at the walk's leaf.
+      // The address lives in a float register as a denormal (bit pattern == integer value):
+      // denormal arithmetic is exact fixed-point, so the update is one FFMA plus a predicated
+      // FADD on the FMA pipe instead of integer ALU work.
+      const int k0 = static_cast<int>(4u * tpc) - static_cast<int>(buf);
+      const float K0f = k0 >= 0 ? __uint_as_float(static_cast<uint32_t>(k0))
+                                : -__uint_as_float(static_cast<uint32_t>(-k0));
+      const float four = __uint_as_float(4u);
 #pragma unroll 1
-      for (int t = 0; t < tpc; ++t) {
-        uint32_t jb[kFastR];
+      for (int t = 0; t < tpc; t += kTreesInFlight) {
+        float a[kTreesInFlight][kFastR];
 #pragma unroll
-        for (int r = 0; r < kFastR; ++r) jb[r] = 4u * t;
-        uint32_t lvl = buf;
+        for (int u = 0; u < kTreesInFlight; ++u)
+#pragma unroll
+          for (int r = 0; r < kFastR; ++r) a[u][r] = __uint_as_float(buf + 4u * (t + u));
 #pragma unroll
         for (int l = 0; l < D; ++l) {
 #pragma unroll
-          for (int r = 0; r < kFastR; ++r) {
-            const uint32_t n = lds_u32(lvl + jb[r]);
-            const uint32_t x = lds_u8(cbase[r] + (n >> 8));
-            jb[r] = 2u * jb[r] + ((x > (n & 0xFFu)) ? 4u : 0u);
-          }
-          lvl += (tpc * 4u) << l;
+          for (int u = 0; u < kTreesInFlight; ++u)
+#pragma unroll
+            for (int r = 0; r < kFastR; ++r) {
+              const uint32_t n = lds_u32(__float_as_uint(a[u][r]));
+              const uint32_t x = lds_u8(cb + (n >> 8) + r);
+              float nx = __fmaf_rn(a[u][r], 2.0f, K0f);
+              if (x > (n & 0xFFu)) nx = __fadd_rn(nx, four);
+              a[u][r] = nx;
+            }
         }
 #pragma unroll
-        for (int r = 0; r < kFastR; ++r) score[r] += lds_f32(leaves + jb[r]);
+        for (int u = 0; u < kTreesInFlight; ++u)
+#pragma unroll
+          for (int r = 0; r < kFastR; ++r) score[r] += lds_f32(__float_as_uint(a[u][r]));
       }
       __syncthreads();  // every thread is done with this buffer
       if (tid == 0 && ch + 2 < fv.n_chunks && !s_fail) {
