@@ -123,6 +123,7 @@ void free_model(ks_model* m) {
   cudaFree(m->gbdt.d_qthr);
   cudaFree(m->gbdt.d_qrow0);
   cudaFree(m->gbdt.d_qrowcnt);
+  ks::free_fast_gbdt(m->gbdt);
   for (int l = 0; l < KS_MLP_MAX_LAYERS; ++l) {
     cudaFree(m->mlp.d_w[l]);
     cudaFree(m->mlp.d_b[l]);

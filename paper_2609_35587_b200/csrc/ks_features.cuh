@@ -27,7 +27,7 @@ __device__ __forceinline__ int bytes_d(int dt) { return dt == 2 ? 1 : (dt == 3 ?
 // Problem-only terms (section "Structural Core", "Memory Behavior"): computed once per problem.
 struct ProblemTerms {
   unsigned M, N, K;
-  int bA, bD, dtype_ab, layout, has_bias, act;
+  int bA, bD, dtype_ab, dtype_d, layout, has_bias, act;
   long long bytesA, bytesB, Q_epi;  // b_A M K, b_B K N, Q_epilogue
   float log2m, log2n, log2k;
   float i_problem, ws_frac_l2, f_bytes_in, f_traffic_epi;
@@ -41,9 +41,10 @@ __device__ __forceinline__ float log2_dim(unsigned v) {
 __device__ inline void problem_terms(const ks_problem& p, const ks_gpu_desc& h, ProblemTerms& t) {
   t.M = p.m; t.N = p.n; t.K = p.k;
   t.dtype_ab = p.dtype_ab & 3;
+  t.dtype_d = p.dtype_d & 3;
   t.layout = p.layout;
   t.bA = bytes_ab(t.dtype_ab);
-  t.bD = bytes_d(p.dtype_d & 3);
+  t.bD = bytes_d(t.dtype_d);
   t.has_bias = p.epi_flags & 1;
   t.act = (p.epi_flags >> 1) & 3;
   const long long M = t.M, N = t.N, K = t.K;

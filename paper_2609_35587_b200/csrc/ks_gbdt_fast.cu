@@ -1,27 +1,39 @@
 // Quantised fast path of the fused select kernel for tree ensembles (Model A).
 //
 // Repack (host, at model-create time)
-//   Every split "x[f] < thr" only needs to know how many of feature f's distinct thresholds
-//   are <= x. With the thresholds of f sorted, bin(x) = #{j : thr_j <= x}, and
+//   A split "x[f] < thr" only needs to know how many of feature f's distinct thresholds are
+//   <= x. With the thresholds of f sorted, bin(x) = #{j : thr_j <= x}, and
 //   x < thr_j  <=>  bin(x) <= j  exactly, so a pair's feature row shrinks from 64 floats to
-//   one byte per "row" (a feature, or a 255-threshold slice of one) and a node to one 32-bit
-//   word (row << 19 | j). Trees are padded to complete trees of the ensemble's depth D and
-//   stored in chunks of kTreesPerChunk trees, each chunk laid out level by level
-//   ([level][tree][node]) followed by its leaves, so that a chunk is one contiguous block a
-//   CTA copies into shared memory with a single bulk async copy.
+//   one byte per "row" (a feature, or a 127-threshold slice of one) and a node to one 32-bit
+//   word. Trees are padded to complete trees of the ensemble's depth D and stored in chunks,
+//   each chunk laid out level by level ([level][tree][node]) followed by its leaves, so that a
+//   chunk is one contiguous block a CTA copies into shared memory with one bulk async copy.
+//   The nodes of the top levels are also kept as (row offset, replicated threshold) pairs that
+//   travel as a kernel parameter, i.e. through the constant bank.
 //
-// Kernel (one CTA = one problem x up to kFastRows candidates)
-//   phase A  featurize every pair in registers, quantise each column by an 8-step branch-free
-//            search in the threshold table (held in shared memory), store the bytes in a
-//            [row][thread] tile whose 32-bit word holds the four candidates of one thread:
-//            a warp's byte loads of any mix of rows hit 32 distinct banks;
-//   phase B  stream the ensemble chunk by chunk through two shared-memory buffers
-//            (cp.async.bulk + mbarrier, bounded waits); each thread walks every tree for its
-//            four candidates, the four walks interleaved for latency hiding;
-//   phase C  rank the block's keys and write a partial top-k list.
+// Hoisting
+//   Rows are grouped by what their feature depends on. Candidate-only rows (given the
+//   problem's element types) are quantised once per call by cand_rows_kernel into a table
+//   indexed by (type combination, candidate); problem-only rows once per CTA; only the
+//   per-pair rows are computed and searched for every pair.
+//
+// Kernel (one CTA = one problem x up to kFastRows candidates, 1024 threads)
+//   phase A  fill the [row][candidate] byte tile. A 32-bit word of a row holds the four
+//            candidates that share a lane slot, so a warp's byte loads of any mix of rows
+//            touch 32 distinct banks and one word load serves four candidates;
+//   phase B  stream the ensemble through two shared-memory buffers (cp.async.bulk + mbarrier,
+//            bounded waits). Thread (w, h) owns the four candidates of word w and walks the
+//            trees of half h of every chunk. The top levels are evaluated for all four
+//            candidates at once, node by node, with byte-parallel arithmetic on whole words;
+//            below that each candidate follows its own path, its node address kept in a float
+//            register as a denormal (bit pattern == integer), where a*2+c is exact, so the
+//            address update runs on the FMA pipe;
+//   phase C  add the two halves' partial scores, rank the block's keys, write a partial
+//            top-k list.
 #include <algorithm>
 #include <cmath>
 #include <limits>
+#include <new>
 #include <vector>
 
 #include "ks_features.cuh"
@@ -32,17 +44,29 @@ namespace ks {
 
 namespace {
 
-constexpr int kBufBytes = 32 * 1024;  // one tree-chunk buffer
-constexpr int kMaxRows = 64;          // quantised rows the kernel supports
-constexpr int kThrPerRow = 256;       // 255 thresholds + padding
+constexpr int kBufBytes = 32 * 1024;   // one tree-chunk buffer
+constexpr int kMaxRows = 80;           // quantised rows the kernel supports (tile <= 160 KB)
+constexpr int kThrPerRow = 128;        // 127 thresholds + padding
 constexpr int kRowStride = kFastRows;  // bytes between rows of the tile (one byte per candidate)
+constexpr int kWords = kFastRows / 4;  // words per row = lane slots
 constexpr int kSpinLimit = 1 << 22;
-constexpr int kTreesInFlight = 2;     // trees walked concurrently per candidate (tpc is a multiple of 4)
+constexpr int kCandRec = 64;           // bytes per (combination, candidate) record of quantised rows
+constexpr int kCombos = 16;            // dtype_ab x dtype_d
 
-// ---- shared memory map (byte offsets from the dynamic shared base) ----------------------
+static_assert(kFastThreads == 2 * kWords && kFastR == 2, "tile geometry");
+
+// shared memory map (byte offsets from the dynamic shared base)
 constexpr int kOffBuf0 = 0;
 constexpr int kOffBuf1 = kBufBytes;
 constexpr int kOffTile = 2 * kBufBytes;
+
+// What a feature column depends on (Table "Feature groups"): 0 problem only, 1 candidate only
+// (given the element types), 2 both.
+__host__ __device__ constexpr int feat_class(int col) {
+  return (col <= 9 || col == 37 || col == 40 || col == 45) ? 0
+         : ((col >= 10 && col <= 22) || col == 38 || (col >= 46 && col <= 59) || col == 62) ? 1
+                                                                                            : 2;
+}
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -92,37 +116,148 @@ __device__ __forceinline__ float lds_f32(uint32_t addr) {
   return v;
 }
 
-// Byte offset, inside one row of the tile, of a thread's first candidate. A 32-bit word
-// holds four candidates and consecutive lanes of a warp own consecutive words, so a warp's
-// byte loads of any mix of rows touch 32 distinct banks.
-__device__ __forceinline__ int slot_offset(int tid) {
-  constexpr int kWords = kFastRows / 4;            // words per row
-  constexpr int kPerWord = 4 / kFastR;             // threads sharing a word
-  static_assert(kFastThreads == kWords * kPerWord, "tile geometry");
-  return (tid % kWords) * 4 + (tid / kWords) * kFastR;
+// #{j : T[j] <= v} over 127 sorted thresholds padded with +inf: 7 branch-free steps.
+__device__ __forceinline__ int bin_search(const float* T, float v) {
+  int pos = 0;
+#pragma unroll
+  for (int s = 64; s >= 1; s >>= 1) pos += (T[pos + s - 1] <= v) ? s : 0;
+  return pos;
 }
 
 struct FastView {
-  int n_rows, depth, n_chunks, chunk_bytes, tpc;
+  int n_rows, n_pair_rows, n_cand_rows, n_prob_rows;  // rows are ordered pair, candidate, problem
+  int depth, n_chunks, chunk_bytes, tpc;
   float base;
-  const uint32_t* chunks;       // [n_chunks][chunk_bytes / 4]
-  const float* thr;             // [n_rows][kThrPerRow]
-  const uint8_t* feat_row0;     // [64] first row of each feature column
-  const uint8_t* feat_rowcnt;   // [64] number of rows of each feature column
+  const uint32_t* chunks;      // [n_chunks][chunk_bytes / 4]
+  const float* thr;            // [n_rows][kThrPerRow]
+  const uint8_t* feat_row0;    // [64] first row of each feature column
+  const uint8_t* feat_rowcnt;  // [64] number of rows of each feature column
+  const uint8_t* cand_rows;    // [kCombos][C][kCandRec] quantised candidate-only rows
 };
 
-template <int D>
+// ------------------------------------------------------------------------------------------
+// candidate-only rows, once per call
+// ------------------------------------------------------------------------------------------
+
+__global__ void combo_mask_kernel(const ks_problem* __restrict__ p, int P, unsigned* __restrict__ mask) {
+  unsigned m = 0;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < P; i += gridDim.x * blockDim.x)
+    m |= 1u << ((p[i].dtype_ab & 3) * 4 + (p[i].dtype_d & 3));
+  m = __reduce_or_sync(0xFFFFFFFFu, m);
+  if ((threadIdx.x & 31) == 0 && m) atomicOr(mask, m);
+}
+
+__global__ void __launch_bounds__(256)
+cand_rows_kernel(ks_gpu_desc desc, const ks_candidate* __restrict__ c, int C, const unsigned* mask_ptr,
+                 unsigned mask_value, FastView fv, uint8_t* __restrict__ out) {
+  const int combo = blockIdx.y;
+  const unsigned mask = mask_ptr ? *mask_ptr : mask_value;
+  if (!((mask >> combo) & 1u)) return;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= C) return;
+  ks_problem fake{};
+  fake.m = fake.n = fake.k = 1;
+  fake.dtype_ab = static_cast<uint8_t>(combo >> 2);
+  fake.dtype_d = static_cast<uint8_t>(combo & 3);
+  ProblemTerms t;
+  problem_terms(fake, desc, t);
+  const ks_candidate cand = c[i];
+  uint8_t* rec = out + (static_cast<size_t>(combo) * C + i) * kCandRec;
+  const int first = fv.n_pair_rows;
+  featurize_pair(t, cand, desc, [&](int col, float v) {
+    if (feat_class(col) != 1) return;
+    const int r0 = fv.feat_row0[col], rc = fv.feat_rowcnt[col];
+    for (int q = 0; q < rc; ++q)
+      rec[r0 + q - first] = static_cast<uint8_t>(0x80 | bin_search(fv.thr + (r0 + q) * kThrPerRow, v));
+  });
+}
+
+// ------------------------------------------------------------------------------------------
+// phase A
+// ------------------------------------------------------------------------------------------
+
+// Fills the tile bytes of the two candidates this thread owns in phase A: candidate-only rows
+// from the per-call table, problem-only rows from s_pbin, per-pair rows computed here. Slots
+// past the end of the segment get a neutral byte so that word-wise arithmetic on the tile
+// never borrows across bytes.
+__device__ __noinline__ void fill_tile(const ks_gpu_desc& desc, const ProblemTerms& pt,
+                                       const ks_candidate* __restrict__ c, const FastView& fv,
+                                       const int64_t* __restrict__ seg_off, const int32_t* __restrict__ seg_idx,
+                                       int C, int64_t lo, int64_t start, int64_t stop, const float* s_thr,
+                                       const uint8_t* s_row0, const uint8_t* s_rowcnt, const uint8_t* s_pbin,
+                                       unsigned char* tile) {
+  const int tid = threadIdx.x;
+  const int combo = pt.dtype_ab * 4 + pt.dtype_d;
+#pragma unroll 1
+  for (int r = 0; r < kFastR; ++r) {
+    const int64_t row = start + static_cast<int64_t>(r) * kFastThreads + tid;
+    unsigned char* my = tile + (tid % kWords) * 4 + (tid / kWords) * kFastR + r;
+    if (row >= stop) {
+      for (int q = 0; q < fv.n_rows; ++q) my[q * kRowStride] = 0x80;
+      continue;
+    }
+    const int ci = seg_off ? seg_idx[lo + row] : static_cast<int>(row);
+    const ks_candidate cand = c[ci];
+    // candidate-only rows
+    const uint4* rec = reinterpret_cast<const uint4*>(fv.cand_rows + (static_cast<size_t>(combo) * C + ci) * kCandRec);
+    unsigned char* dst = my + fv.n_pair_rows * kRowStride;
+#pragma unroll
+    for (int v = 0; v < kCandRec / 16; ++v) {
+      if (v * 16 < fv.n_cand_rows) {
+        const uint4 q = __ldg(rec + v);
+        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int b = 0; b < 16; ++b)
+          if (v * 16 + b < fv.n_cand_rows)
+            dst[(v * 16 + b) * kRowStride] = static_cast<unsigned char>(w[b >> 2] >> (8 * (b & 3)));
+      }
+    }
+    // problem-only rows
+    dst = my + (fv.n_pair_rows + fv.n_cand_rows) * kRowStride;
+    for (int q = 0; q < fv.n_prob_rows; ++q) dst[q * kRowStride] = s_pbin[q];
+    // per-pair rows
+    featurize_pair(pt, cand, desc, [&](int col, float v) {
+      if (feat_class(col) != 2) return;
+      const int r0 = s_row0[col], rc = s_rowcnt[col];
+      for (int q = 0; q < rc; ++q)
+        my[(r0 + q) * kRowStride] = static_cast<unsigned char>(0x80 | bin_search(s_thr + (r0 + q) * kThrPerRow, v));
+    });
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// the kernel
+// ------------------------------------------------------------------------------------------
+
+// bytes of `a` where the top bit of the matching byte of `m` is set, else bytes of `b`
+__device__ __forceinline__ uint32_t byte_select(uint32_t m, uint32_t a, uint32_t b) {
+  const uint32_t f = __byte_perm(m, 0u, 0xBA98u);  // top bit of every byte replicated over the byte
+  return (a & f) | (b & ~f);
+}
+
+// one path step of one walk: fetch the node, fetch the candidate's byte, move to the child
+__device__ __forceinline__ float path_step(float a, uint32_t cb_r, float K0f, float four) {
+  const uint32_t n = lds_u32(__float_as_uint(a));
+  const uint32_t xb = lds_u8(cb_r + (n >> 8));
+  float nx = __fmaf_rn(a, 2.0f, K0f);
+  if (xb > (n & 0xFFu)) nx = __fadd_rn(nx, four);
+  return nx;
+}
+
+template <int L, int NP>  // L levels evaluated word-wise; NP path levels unrolled (-1: runtime count)
 __global__ void __launch_bounds__(kFastThreads, 1)
 select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_problem p_value, int use_value,
                    const ks_candidate* __restrict__ c, int P, int C, int nblk, int rows_per_cta,
                    const int64_t* __restrict__ seg_off, const int32_t* __restrict__ seg_idx, FastView fv,
-                   int k, unsigned long long* __restrict__ partial, int* __restrict__ status) {
+                   int k, unsigned long long* __restrict__ partial, int* __restrict__ status,
+                   const __grid_constant__ FastTopParams top) {
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ ProblemTerms s_pt;
   __shared__ unsigned long long s_warp[kFastThreads / 32];
   __shared__ unsigned long long s_list[KS_MAX_K];
   __shared__ __align__(8) unsigned long long s_bar[2];
-  __shared__ uint8_t s_row0[64], s_rowcnt[64];
+  __shared__ uint8_t s_row0[64], s_rowcnt[64], s_pbin[64];
+  __shared__ float s_pfeat[64];
   __shared__ int s_fail;
 
   const int tid = threadIdx.x;
@@ -139,6 +274,13 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
   const uint32_t bar0 = smem_u32(&s_bar[0]), bar1 = smem_u32(&s_bar[1]);
   if (tid == 0) {
     problem_terms(use_value ? p_value : p[prob], desc, s_pt);
+    // problem-only columns do not look at the candidate: evaluate them on a dummy one
+    ks_candidate dummy{};
+    dummy.tile_m = dummy.tile_n = dummy.tile_k = 64;
+    dummy.stages = dummy.cluster_m = dummy.cluster_n = 1;
+    featurize_pair(s_pt, dummy, desc, [&](int col, float v) {
+      if (feat_class(col) == 0) s_pfeat[col] = v;
+    });
     mbar_init(bar0, 1);
     mbar_init(bar1, 1);
     s_fail = 0;
@@ -149,43 +291,32 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
     s_rowcnt[tid] = fv.feat_rowcnt[tid];
   }
   if (tid < KS_MAX_K) s_list[tid] = 0ull;
+  __syncthreads();
+  if (tid < KS_F && feat_class(tid) == 0) {
+    const int first = fv.n_pair_rows + fv.n_cand_rows;
+    for (int q = 0; q < s_rowcnt[tid]; ++q)
+      s_pbin[s_row0[tid] + q - first] =
+          static_cast<uint8_t>(0x80 | bin_search(fv.thr + (s_row0[tid] + q) * kThrPerRow, s_pfeat[tid]));
+  }
   uint32_t phase0 = 0, phase1 = 0;
+  const int word = tid % kWords, half = tid / kWords;
 
   for (int64_t start = static_cast<int64_t>(chunk) * rows_per_cta; start < len;
        start += static_cast<int64_t>(nblk) * rows_per_cta) {
     const int64_t stop = (start + rows_per_cta < len) ? start + rows_per_cta : len;
-    // ---- phase A: threshold table into the (idle) tree buffers, then featurize + quantise ----
+    // ---- phase A ---------------------------------------------------------------------------------
     __syncthreads();
     {
       float4* dst = reinterpret_cast<float4*>(smem + kOffBuf0);
       const float4* src = reinterpret_cast<const float4*>(fv.thr);
-      for (int i = tid; i < fv.n_rows * kThrPerRow / 4; i += kFastThreads) dst[i] = __ldg(src + i);
+      for (int i = tid; i < fv.n_pair_rows * kThrPerRow / 4; i += kFastThreads) dst[i] = __ldg(src + i);
     }
     __syncthreads();
-    const float* s_thr = reinterpret_cast<const float*>(smem + kOffBuf0);
-    unsigned char* tile = smem + kOffTile;
-#pragma unroll 1
-    for (int r = 0; r < kFastR; ++r) {
-      const int64_t row = start + static_cast<int64_t>(r) * kFastThreads + tid;
-      if (row < stop) {
-        const int ci = seg_off ? seg_idx[lo + row] : static_cast<int>(row);
-        const ks_candidate cand = c[ci];
-        unsigned char* my = tile + slot_offset(tid) + r;
-        featurize_pair(s_pt, cand, desc, [&](int col, float v) {
-          const int r0 = s_row0[col], rc = s_rowcnt[col];
-          for (int q = 0; q < rc; ++q) {
-            const float* T = s_thr + (r0 + q) * kThrPerRow;
-            int pos = 0;
-#pragma unroll
-            for (int s = 128; s >= 1; s >>= 1) pos += (T[pos + s - 1] <= v) ? s : 0;
-            my[(r0 + q) * kRowStride] = static_cast<unsigned char>(pos);
-          }
-        });
-      }
-    }
+    fill_tile(desc, s_pt, c, fv, seg_off, seg_idx, C, lo, start, stop,
+              reinterpret_cast<const float*>(smem + kOffBuf0), s_row0, s_rowcnt, s_pbin, smem + kOffTile);
     __syncthreads();  // tile complete; the threshold table is no longer needed
 
-    // ---- phase B: stream the ensemble through the two buffers ---------------------------------
+    // ---- phase B ---------------------------------------------------------------------------------
     if (tid == 0) {
       fence_async_proxy();
       mbar_expect_tx(bar0, fv.chunk_bytes);
@@ -196,11 +327,11 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
                       fv.chunk_bytes, bar1);
       }
     }
-    float score[kFastR];
-#pragma unroll
-    for (int r = 0; r < kFastR; ++r) score[r] = fv.base;
-    const uint32_t cb = sbase + kOffTile + slot_offset(tid);
-    const int tpc = fv.tpc;
+    float score[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    const uint32_t cb = sbase + kOffTile + word * 4;
+    const int tpc = fv.tpc, half_trees = tpc / 2;
+    const int np = NP >= 0 ? NP : fv.depth - L;
+    constexpr int kTop = (1 << L) - 1;
 #pragma unroll 1
     for (int ch = 0; ch < fv.n_chunks; ++ch) {
       const int b = ch & 1;
@@ -212,40 +343,58 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
       }
       if (b) phase1 ^= 1; else phase0 ^= 1;
       const uint32_t buf = sbase + (b ? kOffBuf1 : kOffBuf0);
-      // With A_l the shared address of a walk's node at level l (levels stored back to back,
-      // [level][tree][node]), A_{l+1} = 2 A_l + (4 tpc - buf) + 4 bit for every level, and
-      // after D steps the address points at the walk's leaf.
-      // The address lives in a float register as a denormal (bit pattern == integer value):
-      // denormal arithmetic is exact fixed-point, so the update is one FFMA plus a predicated
-      // FADD on the FMA pipe instead of integer ALU work.
+      // With A_l the shared address of a walk's node at level l, A_{l+1} = 2 A_l + (4 tpc - buf)
+      // + 4 bit for every level, and after the last level A points at the walk's leaf.
       const int k0 = static_cast<int>(4u * tpc) - static_cast<int>(buf);
       const float K0f = k0 >= 0 ? __uint_as_float(static_cast<uint32_t>(k0))
                                 : -__uint_as_float(static_cast<uint32_t>(-k0));
       const float four = __uint_as_float(4u);
+      const uint32_t lvlL = buf + 4u * tpc * kTop;  // first node of level L
 #pragma unroll 1
-      for (int t = 0; t < tpc; t += kTreesInFlight) {
-        float a[kTreesInFlight][kFastR];
+      for (int t = half * half_trees; t < (half + 1) * half_trees; ++t) {
+        float a[4];
+        if (L == 0) {
 #pragma unroll
-        for (int u = 0; u < kTreesInFlight; ++u)
+          for (int r = 0; r < 4; ++r) a[r] = __uint_as_float(buf + 4u * t);
+        } else {
+          // Word-wise evaluation of the top L levels for the four candidates of this word.
+          // A tile byte is 0x80 | bin and a node constant (j + 1) in every byte, so byte r of
+          // d[n] keeps its top bit iff candidate r goes right at node n; no byte borrows.
+          const uint2* tw = top.w + static_cast<size_t>(ch * tpc + t) * kTop;
+          uint32_t d[kTop > 0 ? kTop : 1];
 #pragma unroll
-          for (int r = 0; r < kFastR; ++r) a[u][r] = __uint_as_float(buf + 4u * (t + u));
-#pragma unroll
-        for (int l = 0; l < D; ++l) {
-#pragma unroll
-          for (int u = 0; u < kTreesInFlight; ++u)
-#pragma unroll
-            for (int r = 0; r < kFastR; ++r) {
-              const uint32_t n = lds_u32(__float_as_uint(a[u][r]));
-              const uint32_t x = lds_u8(cb + (n >> 8) + r);
-              float nx = __fmaf_rn(a[u][r], 2.0f, K0f);
-              if (x > (n & 0xFFu)) nx = __fadd_rn(nx, four);
-              a[u][r] = nx;
+          for (int n = 0; n < kTop; ++n) d[n] = lds_u32(cb + tw[n].x) - tw[n].y;
+          uint32_t x = d[0] & 0x80808080u;  // path bits: level 0 in bit 7 of each byte, ...
+          if (L >= 2) {
+            const uint32_t s1 = byte_select(d[0], d[2], d[1]);
+            x |= (s1 >> 1) & 0x40404040u;
+            if (L >= 3) {
+              const uint32_t sa = byte_select(s1, d[4], d[3]);
+              const uint32_t sb = byte_select(s1, d[6], d[5]);
+              const uint32_t s2 = byte_select(d[0], sb, sa);
+              x |= (s2 >> 2) & 0x20202020u;
             }
+          }
+          // byte r of x holds candidate r's node index at level L in its top L bits (the rest
+          // is zero), so x >> (6 - L) holds 4 * index in every byte
+          const uint32_t y = x >> (6 - L);
+          const uint32_t tbase = lvlL + (static_cast<uint32_t>(t) << (L + 2));
+#pragma unroll
+          for (int r = 0; r < 4; ++r) a[r] = __uint_as_float(tbase + __byte_perm(y, 0u, 0x4440u + r));
+        }
+        if (NP >= 0) {
+#pragma unroll
+          for (int l = 0; l < (NP >= 0 ? NP : 0); ++l)
+#pragma unroll
+            for (int r = 0; r < 4; ++r) a[r] = path_step(a[r], cb + r, K0f, four);
+        } else {
+#pragma unroll 1
+          for (int l = 0; l < np; ++l)
+#pragma unroll
+            for (int r = 0; r < 4; ++r) a[r] = path_step(a[r], cb + r, K0f, four);
         }
 #pragma unroll
-        for (int u = 0; u < kTreesInFlight; ++u)
-#pragma unroll
-          for (int r = 0; r < kFastR; ++r) score[r] += lds_f32(__float_as_uint(a[u][r]));
+        for (int r = 0; r < 4; ++r) score[r] += lds_f32(__float_as_uint(a[r]));
       }
       __syncthreads();  // every thread is done with this buffer
       if (tid == 0 && ch + 2 < fv.n_chunks && !s_fail) {
@@ -255,17 +404,27 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
       }
     }
 
-    // ---- phase C: rank -------------------------------------------------------------------------
-    unsigned long long keys[kFastR + 1];
+    // ---- phase C ---------------------------------------------------------------------------------
+    float* s_part = reinterpret_cast<float*>(smem + kOffBuf0);  // [4][kWords], buffers are idle now
+    if (half == 1) {
 #pragma unroll
-    for (int r = 0; r < kFastR; ++r) {
-      const int64_t row = start + static_cast<int64_t>(r) * kFastThreads + tid;
-      keys[r] = 0ull;
-      if (row < stop) keys[r] = make_key(score[r] + 0.0f, seg_off ? seg_idx[lo + row] : static_cast<int>(row));
+      for (int r = 0; r < 4; ++r) s_part[r * kWords + word] = score[r];
     }
-    keys[kFastR] = tid < k ? s_list[tid] : 0ull;
     __syncthreads();
-    block_topk<kFastR + 1>(keys, k, s_warp, s_list);
+    unsigned long long keys[5];
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      keys[r] = 0ull;
+      // byte r of word `word` belongs to phase-A thread word + kWords * (r / 2), candidate r % 2
+      const int64_t row = start + static_cast<int64_t>(r & 1) * kFastThreads + word + kWords * (r >> 1);
+      if (half == 0 && row < stop) {
+        const float s = (fv.base + score[r]) + s_part[r * kWords + word];
+        keys[r] = make_key(s + 0.0f, seg_off ? seg_idx[lo + row] : static_cast<int>(row));
+      }
+    }
+    keys[4] = tid < k ? s_list[tid] : 0ull;
+    __syncthreads();
+    block_topk<5>(keys, k, s_warp, s_list);
   }
   if (tid < k) partial[(static_cast<size_t>(prob) * nblk + chunk) * k + tid] = s_list[tid];
 }
@@ -280,46 +439,53 @@ cudaError_t build_fast_gbdt(GbdtModel& m, int n_trees, const int64_t* off, const
   m.fast = false;
   if (n_trees < 1 || m.max_depth < 1 || m.max_depth > kFastMaxDepth) return cudaSuccess;
   const int D = m.max_depth;
-  // distinct thresholds per feature
+  // distinct thresholds per feature, sliced into rows of at most 127
   std::vector<std::vector<float>> thr(KS_F);
   for (int64_t i = 0; i < off[n_trees]; ++i)
     if (nodes[i].feat != 0xFFFF) thr[nodes[i].feat].push_back(nodes[i].thr_or_leaf);
   std::vector<uint8_t> row0(64, 0), rowcnt(64, 0);
-  std::vector<float> table;
-  int n_rows = 0;
+  int n_rows = 0, n_class[3] = {0, 0, 0};
   for (int f = 0; f < KS_F; ++f) {
     auto& v = thr[f];
     std::sort(v.begin(), v.end());
     v.erase(std::unique(v.begin(), v.end()), v.end());
-    const int cnt = static_cast<int>((v.size() + 254) / 255);
-    if (n_rows + cnt > kMaxRows) return cudaSuccess;  // not eligible: stays on the generic path
-    row0[f] = static_cast<uint8_t>(n_rows);
-    rowcnt[f] = static_cast<uint8_t>(cnt);
-    for (int q = 0; q < cnt; ++q) {
-      for (int j = 0; j < kThrPerRow; ++j) {
-        const size_t s = static_cast<size_t>(q) * 255 + j;
-        table.push_back(j < 255 && s < v.size() ? v[s] : std::numeric_limits<float>::infinity());
-      }
-    }
-    n_rows += cnt;
+    rowcnt[f] = static_cast<uint8_t>((v.size() + 126) / 127);
+    n_class[feat_class(f)] += rowcnt[f];
+    n_rows += rowcnt[f];
   }
-  if (n_rows == 0) return cudaSuccess;
+  if (n_rows == 0 || n_rows > kMaxRows || n_class[1] > kCandRec) return cudaSuccess;  // generic path
+  // rows ordered: per-pair, candidate-only, problem-only
+  std::vector<float> table(static_cast<size_t>(n_rows) * kThrPerRow, std::numeric_limits<float>::infinity());
+  int next = 0;
+  for (int cls : {2, 1, 0}) {
+    for (int f = 0; f < KS_F; ++f) {
+      if (feat_class(f) != cls) continue;
+      row0[f] = static_cast<uint8_t>(next);
+      for (int q = 0; q < rowcnt[f]; ++q, ++next)
+        for (int j = 0; j < 127; ++j) {
+          const size_t s = static_cast<size_t>(q) * 127 + j;
+          if (s < thr[f].size()) table[static_cast<size_t>(next) * kThrPerRow + j] = thr[f][s];
+        }
+    }
+  }
   const int per_tree_words = (2 << D) - 1;
   int tpc = kBufBytes / (per_tree_words * 4) / 4 * 4;  // a multiple of 4 keeps chunks 16-byte sized
   if (tpc < 4) return cudaSuccess;
   if (tpc > (n_trees + 3) / 4 * 4) tpc = (n_trees + 3) / 4 * 4;  // a small ensemble is one short chunk
   const int n_chunks = (n_trees + tpc - 1) / tpc;
-  const int chunk_words = tpc * per_tree_words;  // tpc is a multiple of 4 for D <= 10, so 16-byte sized
-  if ((chunk_words * 4) % 16 != 0) return cudaSuccess;
+  const int chunk_words = tpc * per_tree_words;
+  int L = D < 3 ? D : 3;  // levels whose nodes travel as kernel-parameter constants
+  while (L > 0 && static_cast<int64_t>(n_chunks) * tpc * ((1 << L) - 1) > kFastTopPairs) --L;
+  const int n_top = (1 << L) - 1;
   std::vector<uint32_t> chunks(static_cast<size_t>(n_chunks) * chunk_words);
-  const uint32_t always_left = 255u;  // row 0, bin 255: every byte is <= 255
+  FastTopParams* top = new (std::nothrow) FastTopParams();
+  if (!top) return cudaErrorMemoryAllocation;
+  const uint32_t always_left = 0xFFu;  // row 0, threshold 127: no byte (0x80 | bin) exceeds 0xFF
   for (int ch = 0; ch < n_chunks; ++ch) {
     uint32_t* base = chunks.data() + static_cast<size_t>(ch) * chunk_words;
     float* leaves = reinterpret_cast<float*>(base + tpc * ((1 << D) - 1));
     for (int tt = 0; tt < tpc; ++tt) {
       const int t = ch * tpc + tt;
-      // walk the (padded) complete tree: slot (level l, index i) holds original node `src` or,
-      // below an original leaf, a pass-through node that always goes left
       std::vector<int> src(1, t < n_trees ? 0 : -1);
       std::vector<float> carry(1, 0.0f);  // leaf value carried below an original leaf
       for (int l = 0; l < D; ++l) {
@@ -329,6 +495,7 @@ cudaError_t build_fast_gbdt(GbdtModel& m, int n_trees, const int64_t* off, const
         std::vector<float> ncarry(2 << l);
         for (int i = 0; i < (1 << l); ++i) {
           uint32_t word = always_left;
+          uint2 tw = make_uint2(0u, 128u * 0x01010101u);
           int ls = -1, rs = -1;
           float lc = carry[i], rc = carry[i];
           if (src[i] >= 0) {
@@ -338,13 +505,15 @@ cudaError_t build_fast_gbdt(GbdtModel& m, int n_trees, const int64_t* off, const
             } else {
               const auto& v = thr[nd.feat];
               const int j = static_cast<int>(std::lower_bound(v.begin(), v.end(), nd.thr_or_leaf) - v.begin());
-              const int row = row0[nd.feat] + j / 255;
-              word = (static_cast<uint32_t>(row) * kRowStride) << 8 | static_cast<uint32_t>(j % 255);
+              const uint32_t row = row0[nd.feat] + j / 127, jl = j % 127;
+              word = (row * kRowStride) << 8 | (0x80u | jl);
+              tw = make_uint2(row * kRowStride, (jl + 1) * 0x01010101u);
               ls = nd.left;
               rs = nd.left + 1;
             }
           }
           lvl[tt * (1 << l) + i] = word;
+          if (l < L) top->w[static_cast<size_t>(t) * n_top + ((1 << l) - 1) + i] = tw;
           nsrc[2 * i] = ls;
           nsrc[2 * i + 1] = rs;
           ncarry[2 * i] = lc;
@@ -355,7 +524,7 @@ cudaError_t build_fast_gbdt(GbdtModel& m, int n_trees, const int64_t* off, const
       }
       for (int i = 0; i < (1 << D); ++i) {
         float v = carry[i];
-        if (src[i] >= 0) v = nodes[off[t] + src[i]].thr_or_leaf;  // depth-D original leaf
+        if (src[i] >= 0) v = nodes[off[t] + src[i]].thr_or_leaf;
         leaves[tt * (1 << D) + i] = v;
       }
     }
@@ -368,14 +537,27 @@ cudaError_t build_fast_gbdt(GbdtModel& m, int n_trees, const int64_t* off, const
   if (e == cudaSuccess) e = cudaMemcpy(m.d_qrow0, row0.data(), 64, cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&m.d_qrowcnt), 64);
   if (e == cudaSuccess) e = cudaMemcpy(m.d_qrowcnt, rowcnt.data(), 64, cudaMemcpyHostToDevice);
-  if (e != cudaSuccess) return e;
+  if (e != cudaSuccess) {
+    delete top;
+    return e;
+  }
+  m.h_top = top;
+  m.top_levels = L;
   m.fast = true;
   m.fast_depth = D;
   m.n_qrows = n_rows;
+  m.n_pair_rows = n_class[2];
+  m.n_cand_rows = n_class[1];
+  m.n_prob_rows = n_class[0];
   m.tpc = tpc;
   m.n_chunks = n_chunks;
   m.chunk_bytes = chunk_words * 4;
   return cudaSuccess;
+}
+
+void free_fast_gbdt(GbdtModel& m) {
+  delete m.h_top;
+  m.h_top = nullptr;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -400,14 +582,36 @@ void fast_tiling(int P, int64_t per_problem, int* nblk, int* rows_per_cta) {
   *rows_per_cta = static_cast<int>(rows);
 }
 
-template <int D>
-static cudaError_t launch_d(const ks_gpu_desc& desc, const GbdtModel& g, const ks_problem* d_p,
-                            const ks_problem& pv, int use_value, int P, const ks_candidate* d_c, int C,
-                            int nblk, int rows_per_cta, const int64_t* seg_off, const int32_t* seg_idx,
-                            int k, unsigned long long* partial, int* status, cudaStream_t stream) {
+size_t fast_scratch_bytes(int C) { return 256 + static_cast<size_t>(kCombos) * C * kCandRec; }
+
+template <int L, int NP>
+static cudaError_t launch_ln(const ks_gpu_desc& desc, const ks_problem* d_p, const ks_problem& pv, int uv, int P,
+                             const ks_candidate* d_c, int C, int nblk, int rows_per_cta, const int64_t* seg_off,
+                             const int32_t* seg_idx, const FastView& fv, int k, unsigned long long* partial,
+                             int* status, const FastTopParams& top, cudaStream_t stream) {
+  const size_t smem = kOffTile + static_cast<size_t>(fv.n_rows) * kRowStride;
+  cudaError_t e = cudaFuncSetAttribute(select_fast_kernel<L, NP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       static_cast<int>(smem));
+  if (e != cudaSuccess) return e;
+  select_fast_kernel<L, NP><<<static_cast<unsigned>(static_cast<int64_t>(P) * nblk), kFastThreads, smem, stream>>>(
+      desc, d_p, pv, uv, d_c, P, C, nblk, rows_per_cta, seg_off, seg_idx, fv, k, partial, status, top);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, const ks_problem* d_p,
+                               const ks_problem* p_by_value, int P, const ks_candidate* d_c, int C,
+                               int nblk, int rows_per_cta, const int64_t* seg_off, const int32_t* seg_idx,
+                               int k, unsigned long long* partial, void* scratch, int* status,
+                               cudaStream_t stream, int64_t* launches, cudaEvent_t ev_begin) {
+  ks_problem pv{};
+  if (p_by_value) pv = *p_by_value;
+  const int uv = p_by_value != nullptr;
   FastView fv;
   fv.n_rows = g.n_qrows;
-  fv.depth = D;
+  fv.n_pair_rows = g.n_pair_rows;
+  fv.n_cand_rows = g.n_cand_rows;
+  fv.n_prob_rows = g.n_prob_rows;
+  fv.depth = g.fast_depth;
   fv.n_chunks = g.n_chunks;
   fv.chunk_bytes = g.chunk_bytes;
   fv.tpc = g.tpc;
@@ -416,29 +620,43 @@ static cudaError_t launch_d(const ks_gpu_desc& desc, const GbdtModel& g, const k
   fv.thr = g.d_qthr;
   fv.feat_row0 = g.d_qrow0;
   fv.feat_rowcnt = g.d_qrowcnt;
-  const size_t smem = kOffTile + static_cast<size_t>(g.n_qrows) * kRowStride;
-  cudaError_t e = cudaFuncSetAttribute(select_fast_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       static_cast<int>(smem));
-  if (e != cudaSuccess) return e;
-  select_fast_kernel<D><<<static_cast<unsigned>(static_cast<int64_t>(P) * nblk), kFastThreads, smem, stream>>>(
-      desc, d_p, pv, use_value, d_c, P, C, nblk, rows_per_cta, seg_off, seg_idx, fv, k, partial, status);
-  return cudaGetLastError();
-}
+  unsigned* d_mask = static_cast<unsigned*>(scratch);
+  uint8_t* d_rows = static_cast<uint8_t*>(scratch) + 256;
+  fv.cand_rows = d_rows;
 
-cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, const ks_problem* d_p,
-                               const ks_problem* p_by_value, int P, const ks_candidate* d_c, int C,
-                               int nblk, int rows_per_cta, const int64_t* seg_off, const int32_t* seg_idx,
-                               int k, unsigned long long* partial, int* status, cudaStream_t stream) {
-  ks_problem pv{};
-  if (p_by_value) pv = *p_by_value;
-  const int uv = p_by_value != nullptr;
-#define KS_CASE(D) \
-  case D: return launch_d<D>(desc, g, d_p, pv, uv, P, d_c, C, nblk, rows_per_cta, seg_off, seg_idx, k, partial, status, stream);
-  switch (g.fast_depth) {
-    KS_CASE(1) KS_CASE(2) KS_CASE(3) KS_CASE(4) KS_CASE(5) KS_CASE(6) KS_CASE(7) KS_CASE(8) KS_CASE(9) KS_CASE(10)
-    default: return cudaErrorInvalidValue;
+  // candidate-only rows for the type combinations in use
+  cudaError_t e = cudaSuccess;
+  unsigned mask_value = 0;
+  if (uv) {
+    mask_value = 1u << ((pv.dtype_ab & 3) * 4 + (pv.dtype_d & 3));
+  } else {
+    e = cudaMemsetAsync(d_mask, 0, sizeof(unsigned), stream);
+    if (e != cudaSuccess) return e;
+    combo_mask_kernel<<<P >= 4096 ? 16 : 1, 256, 0, stream>>>(d_p, P, d_mask);
+    ++*launches;
   }
-#undef KS_CASE
+  if (C > 0) {
+    cand_rows_kernel<<<dim3((C + 255) / 256, kCombos), 256, 0, stream>>>(desc, d_c, C, uv ? nullptr : d_mask,
+                                                                         mask_value, fv, d_rows);
+    ++*launches;
+  }
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  if (ev_begin) cudaEventRecord(ev_begin, stream);
+
+  const FastTopParams& top = *g.h_top;
+  const int L = g.top_levels, np = g.fast_depth - L;
+  ++*launches;
+#define KS_GO(LL, NN) \
+  return launch_ln<LL, NN>(desc, d_p, pv, uv, P, d_c, C, nblk, rows_per_cta, seg_off, seg_idx, fv, k, partial, status, top, stream)
+  if (L == 3 && np == 5) KS_GO(3, 5);
+  if (L == 3 && np == 3) KS_GO(3, 3);
+  if (L == 2 && np == 6) KS_GO(2, 6);
+  if (L == 3) KS_GO(3, -1);
+  if (L == 2) KS_GO(2, -1);
+  if (L == 1) KS_GO(1, -1);
+  KS_GO(0, -1);
+#undef KS_GO
 }
 
 }  // namespace ks

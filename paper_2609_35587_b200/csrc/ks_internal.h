@@ -10,6 +10,13 @@
 
 namespace ks {
 
+// Top-level nodes of the quantised trees as kernel-parameter constants (constant bank):
+// x = row offset in the byte tile, y = (threshold index + 1) replicated into the four bytes.
+constexpr int kFastTopPairs = 3584;
+struct FastTopParams {
+  uint2 w[kFastTopPairs];
+};
+
 // Generic device form of a tree node: 8 bytes, children tree-relative.
 struct DevNode {
   float v;        // threshold, or the leaf value
@@ -27,7 +34,10 @@ struct GbdtModel {
   // quantised fast form (complete trees, chunked level-order layout), see ks_gbdt_fast.cu
   bool fast = false;
   int fast_depth = 0;          // every tree padded to this depth
-  int n_qrows = 0;             // quantised feature rows (a feature, or a 255-threshold slice)
+  int n_qrows = 0;             // quantised feature rows (a feature, or a 127-threshold slice)
+  int n_pair_rows = 0, n_cand_rows = 0, n_prob_rows = 0;  // rows by what their feature depends on
+  int top_levels = 0;          // levels whose nodes also live in h_top
+  FastTopParams* h_top = nullptr;  // host copy, passed by value at every launch
   int tpc = 0;                 // trees per chunk
   int n_chunks = 0;
   int chunk_bytes = 0;
@@ -98,10 +108,13 @@ cudaError_t build_fast_gbdt(GbdtModel& m, int n_trees, const int64_t* h_tree_off
 
 // Quantised tree path: blocks per problem for `per_problem` rows, and the launch itself.
 void fast_tiling(int P, int64_t per_problem, int* nblk, int* rows_per_cta);
+size_t fast_scratch_bytes(int C);  // per-call table of candidate-only rows
+void free_fast_gbdt(GbdtModel& m);
 cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, const ks_problem* d_p,
                                const ks_problem* p_by_value, int P, const ks_candidate* d_c, int C,
                                int nblk, int rows_per_cta, const int64_t* seg_off, const int32_t* seg_idx,
-                               int k, unsigned long long* partial, int* status, cudaStream_t stream);
+                               int k, unsigned long long* partial, void* scratch, int* status,
+                               cudaStream_t stream, int64_t* launches, cudaEvent_t ev_begin);
 
 // ---- launchers (each enqueues on `stream`, returns the cudaError of the launch) -----------
 cudaError_t launch_featurize(const ks_gpu_desc& desc, const ks_problem* d_p, int P,
@@ -116,7 +129,8 @@ cudaError_t launch_score_mlp(const MlpModel& m, const float* d_feat, int64_t row
                              cudaStream_t stream, int64_t* launches);
 
 // Fused featurize + score + top-k. `p_by_value` non-null selects the single-problem form.
-// d_partial: workspace for the per-block partial lists, at least select_partial_bytes().
+// d_partial: workspace for the per-block partial lists and per-call tables, at least
+// select_partial_bytes().
 size_t select_partial_bytes(const ks_model& model, int P, int C, int64_t pairs, bool segmented, int k);
 cudaError_t launch_select(const ks_gpu_desc& desc, const ks_model& model, const ks_problem* d_p,
                           const ks_problem* p_by_value, int P, const ks_candidate* d_c, int C,
