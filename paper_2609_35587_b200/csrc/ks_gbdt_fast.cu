@@ -237,10 +237,22 @@ __device__ __forceinline__ uint32_t byte_select(uint32_t m, uint32_t a, uint32_t
 
 // one path step of one walk: fetch the node, fetch the candidate's byte, move to the child
 __device__ __forceinline__ float path_step(float a, uint32_t cb_r, float K0f, float four) {
-  const uint32_t n = lds_u32(__float_as_uint(a));
-  const uint32_t xb = lds_u8(cb_r + (n >> 8));
-  float nx = __fmaf_rn(a, 2.0f, K0f);
-  if (xb > (n & 0xFFu)) nx = __fadd_rn(nx, four);
+  float nx;
+  asm volatile(
+      "{\n"
+      " .reg .u32 n, x, m;\n"
+      " .reg .pred p;\n"
+      " ld.shared.u32 n, [%1];\n"
+      " shr.u32 m, n, 8;\n"
+      " add.u32 m, m, %2;\n"
+      " ld.shared.u8 x, [m];\n"
+      " and.b32 n, n, 255;\n"
+      " setp.gt.u32 p, x, n;\n"
+      " fma.rn.f32 %0, %3, 0f40000000, %4;\n"
+      " @p add.rn.f32 %0, %0, %5;\n"
+      "}\n"
+      : "=f"(nx)
+      : "r"(__float_as_uint(a)), "r"(cb_r), "f"(a), "f"(K0f), "f"(four));
   return nx;
 }
 
