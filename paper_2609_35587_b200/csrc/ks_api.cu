@@ -179,8 +179,23 @@ ks_status ks_create(ks_ctx** out_ctx, int cuda_device, const ks_gpu_desc* desc) 
   ctx->device = cuda_device;
   ctx->desc = *desc;
   ctx->pinned_bytes = KS_MAX_K * (sizeof(int32_t) + sizeof(float));
-  if (cudaMallocHost(&ctx->pinned, ctx->pinned_bytes) != cudaSuccess) {
+  // result staging of ks_select_one: mapped pinned memory, so the kernel's last block can
+  // write the k results where the host reads them, with no copy in between
+  void* d_pin = nullptr;
+  if (cudaHostAlloc(&ctx->pinned, ctx->pinned_bytes, cudaHostAllocMapped) != cudaSuccess ||
+      cudaHostGetDevicePointer(&d_pin, ctx->pinned, 0) != cudaSuccess) {
     cudaGetLastError();
+    if (ctx->pinned) cudaFreeHost(ctx->pinned);
+    delete ctx;
+    return KS_ERR_OOM;
+  }
+  ctx->d_pinned_idx = static_cast<int32_t*>(d_pin);
+  ctx->d_pinned_score = reinterpret_cast<float*>(ctx->d_pinned_idx + KS_MAX_K);
+  if (cudaMalloc(reinterpret_cast<void**>(&ctx->d_counters), sizeof(int) * (ks::kMaxSliceBlocks + 1)) != cudaSuccess ||
+      cudaMemset(ctx->d_counters, 0, sizeof(int) * (ks::kMaxSliceBlocks + 1)) != cudaSuccess) {
+    cudaGetLastError();
+    cudaFree(ctx->d_counters);
+    cudaFreeHost(ctx->pinned);
     delete ctx;
     return KS_ERR_OOM;
   }
@@ -195,6 +210,7 @@ ks_status ks_create(ks_ctx** out_ctx, int cuda_device, const ks_gpu_desc* desc) 
   if (s == KS_OK) *ctx->h_status = 0;
   if (s != KS_OK) {
     cudaFree(ctx->ws);
+    cudaFree(ctx->d_counters);
     if (ctx->h_status) cudaFreeHost(ctx->h_status);
     cudaFreeHost(ctx->pinned);
     delete ctx;
@@ -210,6 +226,7 @@ ks_status ks_destroy(ks_ctx* ctx) {
   if (ctx->ev_begin) cudaEventDestroy(ctx->ev_begin);
   if (ctx->ev_end) cudaEventDestroy(ctx->ev_end);
   cudaFree(ctx->ws);
+  cudaFree(ctx->d_counters);
   cudaFreeHost(ctx->h_status);
   cudaFreeHost(ctx->pinned);
   delete ctx;
@@ -404,6 +421,43 @@ ks_status ks_select_one(ks_ctx* ctx, ks_problem p, const ks_candidate* d_c, int 
     return KS_ERR_INVALID_ARG;
   DeviceGuard g(ctx->device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int32_t* pin_idx = static_cast<int32_t*>(ctx->pinned);
+  float* pin_sc = reinterpret_cast<float*>(pin_idx + KS_MAX_K);
+
+  // Latency path for a qualifying tree model: the trees are split over several CTAs per
+  // candidate block, the last block writes the k results straight into mapped host memory.
+  if (model->kind == 0 && model->gbdt.fast && C > 0) {
+    const int nblk = (C + ks::kFastRows - 1) / ks::kFastRows;
+    const int S = ks::fast_slices(model->gbdt, nblk);
+    if (S > 1 && nblk <= ks::kMaxSliceBlocks) {
+      const size_t b_part = align_up(sizeof(unsigned long long) * nblk * k);
+      const size_t b_scratch = align_up(ks::fast_scratch_bytes(C));
+      const size_t b_scores = align_up(sizeof(float) * static_cast<size_t>(S) * C);
+      ks_status s = ensure_workspace(ctx, b_part + b_scratch + b_scores);
+      if (s != KS_OK) return s;
+      char* base = static_cast<char*>(ctx->ws);
+      ks::FastSlice sl;
+      sl.n_slices = S;
+      sl.scores = reinterpret_cast<float*>(base + b_part + b_scratch);
+      sl.counters = ctx->d_counters;
+      sl.out_idx = ctx->d_pinned_idx;
+      sl.out_score = ctx->d_pinned_score;
+      cudaError_t e = ks::launch_select_fast(ctx->desc, model->gbdt, nullptr, &p, 1, d_c, C, nblk, ks::kFastRows,
+                                             nullptr, nullptr, k, reinterpret_cast<unsigned long long*>(base),
+                                             base + b_part, ctx->d_status, st, &ctx->launches, nullptr, &sl);
+      if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+      if (e != cudaSuccess) return cuda_fail(ctx, e, "ks_select_one");
+      s = read_status(ctx);
+      if (s != KS_OK) {
+        cudaMemset(ctx->d_counters, 0, sizeof(int) * (ks::kMaxSliceBlocks + 1));
+        return s;
+      }
+      std::memcpy(h_topk_idx, pin_idx, k * sizeof(int32_t));
+      std::memcpy(h_topk_score, pin_sc, k * sizeof(float));
+      return KS_OK;
+    }
+  }
+
   const size_t out_bytes = align_up(k * sizeof(int32_t)) + align_up(k * sizeof(float));
   const size_t part = align_up(ks::select_partial_bytes(*model, 1, C, C, false, k));
   ks_status s = ensure_workspace(ctx, part + out_bytes);
@@ -413,8 +467,6 @@ ks_status ks_select_one(ks_ctx* ctx, ks_problem p, const ks_candidate* d_c, int 
   float* d_sc = reinterpret_cast<float*>(base + part + align_up(k * sizeof(int32_t)));
   cudaError_t e = ks::launch_select(ctx->desc, *model, nullptr, &p, 1, d_c, C, nullptr, nullptr, C, k,
                                     ctx->ws, d_idx, d_sc, st, &ctx->launches, ctx->d_status);
-  int32_t* pin_idx = static_cast<int32_t*>(ctx->pinned);
-  float* pin_sc = reinterpret_cast<float*>(pin_idx + KS_MAX_K);
   if (e == cudaSuccess) e = cudaMemcpyAsync(pin_idx, d_idx, k * sizeof(int32_t), cudaMemcpyDeviceToHost, st);
   if (e == cudaSuccess) e = cudaMemcpyAsync(pin_sc, d_sc, k * sizeof(float), cudaMemcpyDeviceToHost, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);

@@ -124,6 +124,18 @@ __device__ __forceinline__ int bin_search(const float* T, float v) {
   return pos;
 }
 
+// Slice mode (single-problem latency call): the trees are split over n_slices CTAs per
+// candidate block. Every CTA stores its partial scores; the last CTA to arrive for a block
+// (atomic counter, nobody waits) adds the slices in a fixed order and ranks the block; the
+// last block overall merges the lists and writes the final result.
+struct SliceArgs {
+  int n_slices;            // 1 = batch mode
+  float* scores;           // [n_slices][C] partial scores
+  int* counters;           // [nblk + 1], zero on entry, reset to zero by the last block
+  int32_t* out_idx;        // [k] final result (device-visible, may be mapped host memory)
+  float* out_score;        // [k]
+};
+
 struct FastView {
   int n_rows, n_pair_rows, n_cand_rows, n_prob_rows;  // rows are ordered pair, candidate, problem
   int depth, n_chunks, chunk_bytes, tpc;
@@ -262,7 +274,7 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
                    const ks_candidate* __restrict__ c, int P, int C, int nblk, int rows_per_cta,
                    const int64_t* __restrict__ seg_off, const int32_t* __restrict__ seg_idx, FastView fv,
                    int k, unsigned long long* __restrict__ partial, int* __restrict__ status,
-                   const __grid_constant__ FastTopParams top) {
+                   SliceArgs sl, const __grid_constant__ FastTopParams top) {
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ ProblemTerms s_pt;
   __shared__ unsigned long long s_warp[kFastThreads / 32];
@@ -270,10 +282,11 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
   __shared__ __align__(8) unsigned long long s_bar[2];
   __shared__ uint8_t s_row0[64], s_rowcnt[64], s_pbin[64];
   __shared__ float s_pfeat[64];
-  __shared__ int s_fail;
+  __shared__ int s_fail, s_last;
 
   const int tid = threadIdx.x;
-  const int prob = blockIdx.x / nblk, chunk = blockIdx.x % nblk;
+  const int S = sl.n_slices;
+  const int prob = blockIdx.x / (nblk * S), chunk = (blockIdx.x / S) % nblk, slice = blockIdx.x % S;
   int64_t lo, len;
   if (seg_off) {
     lo = seg_off[prob];
@@ -282,6 +295,9 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
     lo = static_cast<int64_t>(prob) * C;
     len = C;
   }
+  // chunks of the ensemble this CTA walks
+  const int ch_begin = static_cast<int>(static_cast<int64_t>(fv.n_chunks) * slice / S);
+  const int ch_end = static_cast<int>(static_cast<int64_t>(fv.n_chunks) * (slice + 1) / S);
   const uint32_t sbase = smem_u32(smem);
   const uint32_t bar0 = smem_u32(&s_bar[0]), bar1 = smem_u32(&s_bar[1]);
   if (tid == 0) {
@@ -331,12 +347,14 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
     // ---- phase B ---------------------------------------------------------------------------------
     if (tid == 0) {
       fence_async_proxy();
-      mbar_expect_tx(bar0, fv.chunk_bytes);
-      bulk_copy_g2s(sbase + kOffBuf0, fv.chunks, fv.chunk_bytes, bar0);
-      if (fv.n_chunks > 1) {
+      const char* src = reinterpret_cast<const char*>(fv.chunks) + static_cast<size_t>(ch_begin) * fv.chunk_bytes;
+      if (ch_end > ch_begin) {
+        mbar_expect_tx(bar0, fv.chunk_bytes);
+        bulk_copy_g2s(sbase + kOffBuf0, src, fv.chunk_bytes, bar0);
+      }
+      if (ch_end > ch_begin + 1) {
         mbar_expect_tx(bar1, fv.chunk_bytes);
-        bulk_copy_g2s(sbase + kOffBuf1, reinterpret_cast<const char*>(fv.chunks) + fv.chunk_bytes,
-                      fv.chunk_bytes, bar1);
+        bulk_copy_g2s(sbase + kOffBuf1, src + fv.chunk_bytes, fv.chunk_bytes, bar1);
       }
     }
     float score[4] = {0.0f, 0.0f, 0.0f, 0.0f};
@@ -345,8 +363,8 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
     const int np = NP >= 0 ? NP : fv.depth - L;
     constexpr int kTop = (1 << L) - 1;
 #pragma unroll 1
-    for (int ch = 0; ch < fv.n_chunks; ++ch) {
-      const int b = ch & 1;
+    for (int ch = ch_begin; ch < ch_end; ++ch) {
+      const int b = (ch - ch_begin) & 1;
       const uint32_t bar = b ? bar1 : bar0;
       const uint32_t par = b ? phase1 : phase0;
       if (!mbar_wait_bounded(bar, par)) {
@@ -409,7 +427,7 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
         for (int r = 0; r < 4; ++r) score[r] += lds_f32(__float_as_uint(a[r]));
       }
       __syncthreads();  // every thread is done with this buffer
-      if (tid == 0 && ch + 2 < fv.n_chunks && !s_fail) {
+      if (tid == 0 && ch + 2 < ch_end && !s_fail) {
         mbar_expect_tx(bar, fv.chunk_bytes);
         bulk_copy_g2s(buf, reinterpret_cast<const char*>(fv.chunks) + static_cast<size_t>(ch + 2) * fv.chunk_bytes,
                       fv.chunk_bytes, bar);
@@ -423,6 +441,21 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
       for (int r = 0; r < 4; ++r) s_part[r * kWords + word] = score[r];
     }
     __syncthreads();
+    if (S > 1) {
+      // slice mode: publish this CTA's partial scores, let the last arrival finish the block
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        const int64_t row = start + static_cast<int64_t>(r & 1) * kFastThreads + word + kWords * (r >> 1);
+        if (half == 0 && row < stop)
+          __stcg(sl.scores + static_cast<size_t>(slice) * C + row, score[r] + s_part[r * kWords + word]);
+      }
+      __threadfence();
+      __syncthreads();
+      if (tid == 0) s_last = atomicAdd(sl.counters + chunk, 1) == S - 1;
+      __syncthreads();
+      if (!s_last) return;
+      __threadfence();
+    }
     unsigned long long keys[5];
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
@@ -430,7 +463,13 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
       // byte r of word `word` belongs to phase-A thread word + kWords * (r / 2), candidate r % 2
       const int64_t row = start + static_cast<int64_t>(r & 1) * kFastThreads + word + kWords * (r >> 1);
       if (half == 0 && row < stop) {
-        const float s = (fv.base + score[r]) + s_part[r * kWords + word];
+        float s;
+        if (S > 1) {
+          s = fv.base;
+          for (int q = 0; q < S; ++q) s += __ldcg(sl.scores + static_cast<size_t>(q) * C + row);
+        } else {
+          s = (fv.base + score[r]) + s_part[r * kWords + word];
+        }
         keys[r] = make_key(s + 0.0f, seg_off ? seg_idx[lo + row] : static_cast<int>(row));
       }
     }
@@ -439,6 +478,33 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
     block_topk<5>(keys, k, s_warp, s_list);
   }
   if (tid < k) partial[(static_cast<size_t>(prob) * nblk + chunk) * k + tid] = s_list[tid];
+  if (S > 1) {
+    // the last block to finish merges the per-block lists (one warp) and resets the counters
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) s_last = atomicAdd(sl.counters + nblk, 1) == nblk - 1;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    if (tid < 32) {
+      const int n_keys = nblk * k;
+      unsigned long long prev = ~0ull;
+      for (int j = 0; j < k; ++j) {
+        unsigned long long best = 0ull;
+        for (int i = tid; i < n_keys; i += 32) {
+          const unsigned long long v = __ldcg(partial + i);
+          if (v < prev && v > best) best = v;
+        }
+        best = warp_max_u64(best);
+        if (tid == 0) {
+          sl.out_idx[j] = key_index(best);
+          sl.out_score[j] = key_score(best);
+        }
+        prev = best;
+      }
+    }
+    for (int i = tid; i <= nblk; i += kFastThreads) sl.counters[i] = 0;
+  }
 }
 
 }  // namespace
@@ -596,17 +662,26 @@ void fast_tiling(int P, int64_t per_problem, int* nblk, int* rows_per_cta) {
 
 size_t fast_scratch_bytes(int C) { return 256 + static_cast<size_t>(kCombos) * C * kCandRec; }
 
+// Slice count of the single-problem call: as many tree slices as keep every CTA in the first
+// wave (one CTA per SM).
+int fast_slices(const GbdtModel& g, int nblk) {
+  int s = 148 / (nblk < 1 ? 1 : nblk);
+  if (s > g.n_chunks) s = g.n_chunks;
+  return s < 1 ? 1 : s;
+}
+
 template <int L, int NP>
 static cudaError_t launch_ln(const ks_gpu_desc& desc, const ks_problem* d_p, const ks_problem& pv, int uv, int P,
                              const ks_candidate* d_c, int C, int nblk, int rows_per_cta, const int64_t* seg_off,
                              const int32_t* seg_idx, const FastView& fv, int k, unsigned long long* partial,
-                             int* status, const FastTopParams& top, cudaStream_t stream) {
+                             int* status, const SliceArgs& sl, const FastTopParams& top, cudaStream_t stream) {
   const size_t smem = kOffTile + static_cast<size_t>(fv.n_rows) * kRowStride;
   cudaError_t e = cudaFuncSetAttribute(select_fast_kernel<L, NP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        static_cast<int>(smem));
   if (e != cudaSuccess) return e;
-  select_fast_kernel<L, NP><<<static_cast<unsigned>(static_cast<int64_t>(P) * nblk), kFastThreads, smem, stream>>>(
-      desc, d_p, pv, uv, d_c, P, C, nblk, rows_per_cta, seg_off, seg_idx, fv, k, partial, status, top);
+  select_fast_kernel<L, NP><<<static_cast<unsigned>(static_cast<int64_t>(P) * nblk * sl.n_slices), kFastThreads, smem,
+                              stream>>>(desc, d_p, pv, uv, d_c, P, C, nblk, rows_per_cta, seg_off, seg_idx, fv, k,
+                                        partial, status, sl, top);
   return cudaGetLastError();
 }
 
@@ -614,7 +689,8 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
                                const ks_problem* p_by_value, int P, const ks_candidate* d_c, int C,
                                int nblk, int rows_per_cta, const int64_t* seg_off, const int32_t* seg_idx,
                                int k, unsigned long long* partial, void* scratch, int* status,
-                               cudaStream_t stream, int64_t* launches, cudaEvent_t ev_begin) {
+                               cudaStream_t stream, int64_t* launches, cudaEvent_t ev_begin,
+                               const FastSlice* slice) {
   ks_problem pv{};
   if (p_by_value) pv = *p_by_value;
   const int uv = p_by_value != nullptr;
@@ -656,11 +732,20 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
   if (e != cudaSuccess) return e;
   if (ev_begin) cudaEventRecord(ev_begin, stream);
 
+  SliceArgs sl{};
+  sl.n_slices = 1;
+  if (slice && slice->n_slices > 1) {
+    sl.n_slices = slice->n_slices;
+    sl.scores = slice->scores;
+    sl.counters = slice->counters;
+    sl.out_idx = slice->out_idx;
+    sl.out_score = slice->out_score;
+  }
   const FastTopParams& top = *g.h_top;
   const int L = g.top_levels, np = g.fast_depth - L;
   ++*launches;
 #define KS_GO(LL, NN) \
-  return launch_ln<LL, NN>(desc, d_p, pv, uv, P, d_c, C, nblk, rows_per_cta, seg_off, seg_idx, fv, k, partial, status, top, stream)
+  return launch_ln<LL, NN>(desc, d_p, pv, uv, P, d_c, C, nblk, rows_per_cta, seg_off, seg_idx, fv, k, partial, status, sl, top, stream)
   if (L == 3 && np == 5) KS_GO(3, 5);
   if (L == 3 && np == 3) KS_GO(3, 3);
   if (L == 2 && np == 6) KS_GO(2, 6);

@@ -76,6 +76,9 @@ struct ks_ctx {
   size_t ws_bytes = 0;
   void* pinned = nullptr;  // host staging for ks_select_one results
   size_t pinned_bytes = 0;
+  int* d_counters = nullptr;  // [kMaxSliceBlocks + 1] arrival counters of the slice mode, zero between calls
+  int32_t* d_pinned_idx = nullptr;  // device aliases of `pinned` (mapped host memory)
+  float* d_pinned_score = nullptr;
   int* h_status = nullptr;  // status word (mapped pinned host memory) set by kernels whose
   int* d_status = nullptr;  // bounded waits give up; d_status is its device alias
   int64_t launches = 0;
@@ -101,10 +104,20 @@ constexpr int kFastThreads = 1024;      // threads per block of the quantised tr
 constexpr int kFastR = 2;              // candidates per thread there
 constexpr int kFastRows = kFastThreads * kFastR;
 constexpr int kFastMaxDepth = 10;
+constexpr int kMaxSliceBlocks = 1024;  // candidate blocks the slice mode supports
 
 // Builds the quantised fast form of a validated ensemble when it qualifies (m.fast).
 cudaError_t build_fast_gbdt(GbdtModel& m, int n_trees, const int64_t* h_tree_offsets,
                             const ks_node_host* h_nodes);
+
+// Slice mode of the quantised tree kernel (single-problem latency call).
+struct FastSlice {
+  int n_slices;
+  float* scores;     // [n_slices][C]
+  int* counters;     // [nblk + 1], zero between calls
+  int32_t* out_idx;  // [k], device-visible
+  float* out_score;  // [k]
+};
 
 // Quantised tree path: blocks per problem for `per_problem` rows, and the launch itself.
 void fast_tiling(int P, int64_t per_problem, int* nblk, int* rows_per_cta);
@@ -114,7 +127,9 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
                                const ks_problem* p_by_value, int P, const ks_candidate* d_c, int C,
                                int nblk, int rows_per_cta, const int64_t* seg_off, const int32_t* seg_idx,
                                int k, unsigned long long* partial, void* scratch, int* status,
-                               cudaStream_t stream, int64_t* launches, cudaEvent_t ev_begin);
+                               cudaStream_t stream, int64_t* launches, cudaEvent_t ev_begin,
+                               const FastSlice* slice = nullptr);
+int fast_slices(const GbdtModel& g, int nblk);
 
 // ---- launchers (each enqueues on `stream`, returns the cudaError of the launch) -----------
 cudaError_t launch_featurize(const ks_gpu_desc& desc, const ks_problem* d_p, int P,

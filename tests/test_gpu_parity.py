@@ -259,8 +259,13 @@ def test_select_one_and_select_host_agree_with_select(ks, ctx):
     idx, sc = run_select(ks, ctx, w, model)
     d_c = dev(ks, w.candidates)
     for i in range(4):
+        # the latency form adds the trees' leaves in a different (fixed) order: same ranking,
+        # scores equal up to rounding
         hi, hs = ctx.select_one(w.problems[i:i + 1], d_c, len(w.candidates), model, w.k)
-        assert np.array_equal(hi.numpy(), idx[i]) and np.array_equal(hs.numpy(), sc[i])
+        assert np.array_equal(hi.numpy(), idx[i])
+        assert np.all(np.abs(hs.numpy() - sc[i]) <= TOL_GBDT * np.maximum(1, np.abs(sc[i])))
+        hi2, hs2 = ctx.select_one(w.problems[i:i + 1], d_c, len(w.candidates), model, w.k)
+        assert np.array_equal(hi.numpy(), hi2.numpy()) and np.array_equal(hs.numpy(), hs2.numpy())
     hi, hs = ctx.select_host(w.problems, 4, w.candidates, len(w.candidates), model, w.k)
     assert np.array_equal(hi.numpy(), idx) and np.array_equal(hs.numpy(), sc)
     check_select(w, idx, sc, TOL_GBDT)
@@ -270,6 +275,25 @@ def test_select_one_and_select_host_agree_with_select(ks, ctx):
     hi, hs = ctx.select_host(w2.problems, 6, w2.candidates, len(w2.candidates), model2, w2.k,
                              w2.seg_offsets, w2.seg_index, w2.pairs)
     assert np.array_equal(hi.numpy(), idx2) and np.array_equal(hs.numpy(), sc2)
+
+
+def test_select_one_latency_stream_against_oracle(ks, ctx):
+    """Single problems of the latency stream (arbitrary integer dimensions, decode-like M)
+    against the full catalogue and the 500-tree ensemble, each checked against the oracle."""
+    w = wl.make_workload(3, P=6)
+    model = ctx.model_create_gbdt(*w.gbdt)
+    d_c = dev(ks, w.candidates)
+    C = len(w.candidates)
+    for i in range(len(w.problems)):
+        hi, hs = ctx.select_one(w.problems[i:i + 1], d_c, C, model, w.k)
+        _, _, allsc = oracle.select(w.problems[i:i + 1], w.candidates, DESC, w.k, gbdt=w.gbdt, want_scores=True)
+        ok, msg = topk_accept(hi.numpy(), hs.numpy(), allsc, np.arange(C, dtype=np.int32), w.k, TOL_GBDT)
+        assert ok, f"call {i}: {msg}"
+    for C2 in (1, 2047, 2049, 5000):
+        hi, hs = ctx.select_one(w.problems[:1], d_c, C2, model, w.k)
+        _, _, allsc = oracle.select(w.problems[:1], w.candidates[:C2], DESC, w.k, gbdt=w.gbdt, want_scores=True)
+        ok, msg = topk_accept(hi.numpy(), hs.numpy(), allsc, np.arange(C2, dtype=np.int32), w.k, TOL_GBDT)
+        assert ok, f"C={C2}: {msg}"
 
 
 # ---------------------------------------------------------------------------------------------
