@@ -162,9 +162,19 @@ __global__ void combo_mask_kernel(const ks_problem* __restrict__ p, int P, unsig
 __global__ void __launch_bounds__(256)
 cand_rows_kernel(ks_gpu_desc desc, const ks_candidate* __restrict__ c, int C, const unsigned* mask_ptr,
                  unsigned mask_value, FastView fv, uint8_t* __restrict__ out) {
+  extern __shared__ float s_cthr[];  // thresholds of the candidate-only rows
+  __shared__ uint8_t s_r0[64], s_rc[64];
   const int combo = blockIdx.y;
   const unsigned mask = mask_ptr ? *mask_ptr : mask_value;
   if (!((mask >> combo) & 1u)) return;
+  const int first = fv.n_pair_rows;
+  for (int i = threadIdx.x; i < fv.n_cand_rows * kThrPerRow; i += blockDim.x)
+    s_cthr[i] = __ldg(fv.thr + first * kThrPerRow + i);
+  if (threadIdx.x < 64) {
+    s_r0[threadIdx.x] = fv.feat_row0[threadIdx.x];
+    s_rc[threadIdx.x] = fv.feat_rowcnt[threadIdx.x];
+  }
+  __syncthreads();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= C) return;
   ks_problem fake{};
@@ -174,14 +184,24 @@ cand_rows_kernel(ks_gpu_desc desc, const ks_candidate* __restrict__ c, int C, co
   ProblemTerms t;
   problem_terms(fake, desc, t);
   const ks_candidate cand = c[i];
-  uint8_t* rec = out + (static_cast<size_t>(combo) * C + i) * kCandRec;
-  const int first = fv.n_pair_rows;
+  uint32_t rec[kCandRec / 4];
+#pragma unroll
+  for (int q = 0; q < kCandRec / 4; ++q) rec[q] = 0x80808080u;
   featurize_pair(t, cand, desc, [&](int col, float v) {
     if (feat_class(col) != 1) return;
-    const int r0 = fv.feat_row0[col], rc = fv.feat_rowcnt[col];
-    for (int q = 0; q < rc; ++q)
-      rec[r0 + q - first] = static_cast<uint8_t>(0x80 | bin_search(fv.thr + (r0 + q) * kThrPerRow, v));
+    const int r0 = s_r0[col] - first, rc = s_rc[col];
+    for (int q = 0; q < rc; ++q) {
+      const uint32_t b = 0x80u | bin_search(s_cthr + (r0 + q) * kThrPerRow, v);
+      const int at = r0 + q;
+#pragma unroll
+      for (int w = 0; w < kCandRec / 4; ++w)
+        if (w == (at >> 2)) rec[w] = (rec[w] & ~(0xFFu << (8 * (at & 3)))) | (b << (8 * (at & 3)));
+    }
   });
+  uint4* dst = reinterpret_cast<uint4*>(out + (static_cast<size_t>(combo) * C + i) * kCandRec);
+#pragma unroll
+  for (int q = 0; q < kCandRec / 16; ++q)
+    if (q * 16 < fv.n_cand_rows) dst[q] = make_uint4(rec[4 * q], rec[4 * q + 1], rec[4 * q + 2], rec[4 * q + 3]);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -277,7 +297,7 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
                    SliceArgs sl, const __grid_constant__ FastTopParams top) {
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ ProblemTerms s_pt;
-  __shared__ unsigned long long s_warp[kFastThreads / 32];
+  __shared__ unsigned long long s_warp[kFastThreads / 32 * KS_MAX_K];
   __shared__ unsigned long long s_list[KS_MAX_K];
   __shared__ __align__(8) unsigned long long s_bar[2];
   __shared__ uint8_t s_row0[64], s_rowcnt[64], s_pbin[64];
@@ -724,8 +744,9 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
     ++*launches;
   }
   if (C > 0) {
-    cand_rows_kernel<<<dim3((C + 255) / 256, kCombos), 256, 0, stream>>>(desc, d_c, C, uv ? nullptr : d_mask,
-                                                                         mask_value, fv, d_rows);
+    const size_t cthr = sizeof(float) * kThrPerRow * (g.n_cand_rows > 0 ? g.n_cand_rows : 1);
+    cand_rows_kernel<<<dim3((C + 255) / 256, kCombos), 256, cthr, stream>>>(desc, d_c, C, uv ? nullptr : d_mask,
+                                                                            mask_value, fv, d_rows);
     ++*launches;
   }
   e = cudaGetLastError();

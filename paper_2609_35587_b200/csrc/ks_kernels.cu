@@ -218,7 +218,7 @@ select_generic_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_pro
   float* s_scores = s_cols + kRow * kBlock;         // [kBlock] (MLP only)
   __nv_bfloat16* s_act = reinterpret_cast<__nv_bfloat16*>(s_scores + kBlock);
   __shared__ ProblemTerms s_pt;
-  __shared__ unsigned long long s_warp[kBlock / 32];
+  __shared__ unsigned long long s_warp[kBlock / 32 * KS_MAX_K];
   __shared__ unsigned long long s_list[KS_MAX_K];
 
   const int prob = blockIdx.x / map.nblk, chunk = blockIdx.x % map.nblk;

@@ -35,7 +35,9 @@ __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v)
 }
 
 // The k largest of the block's keys (N per thread), descending, into s_list[0..k).
-// All threads of the block must call; s_warp holds one slot per warp.
+// Two levels: every warp first ranks its own keys (k rounds of warp-wide max, no block
+// barrier), then warp 0 ranks the n_warps * k survivors. All threads of the block must call;
+// s_warp needs n_warps * KS_MAX_K slots.
 template <int N>
 __device__ __forceinline__ void block_topk(const unsigned long long (&keys)[N], int k,
                                            unsigned long long* s_warp, unsigned long long* s_list) {
@@ -49,14 +51,25 @@ __device__ __forceinline__ void block_topk(const unsigned long long (&keys)[N], 
       if (v < prev && v > best) best = v;
     }
     best = warp_max_u64(best);
-    if (lane == 0) s_warp[warp] = best;
-    __syncthreads();
-    unsigned long long w = 0ull;
-    for (int i = 0; i < n_warps; ++i) w = max(w, s_warp[i]);
-    if (threadIdx.x == 0) s_list[j] = w;
-    prev = w;
-    __syncthreads();
+    if (lane == 0) s_warp[warp * k + j] = best;
+    prev = best;
   }
+  __syncthreads();
+  if (warp == 0) {
+    const int n = n_warps * k;
+    prev = ~0ull;
+    for (int j = 0; j < k; ++j) {
+      unsigned long long best = 0ull;
+      for (int i = lane; i < n; i += 32) {
+        const unsigned long long v = s_warp[i];
+        if (v < prev && v > best) best = v;
+      }
+      best = warp_max_u64(best);
+      if (lane == 0) s_list[j] = best;
+      prev = best;
+    }
+  }
+  __syncthreads();
 }
 
 }  // namespace ks
