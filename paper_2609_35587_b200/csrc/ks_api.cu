@@ -130,6 +130,8 @@ void free_model(ks_model* m) {
   }
   cudaFree(m->mlp.d_mu);
   cudaFree(m->mlp.d_sigma);
+  cudaFree(m->mlp.d_tc_image);
+  ks::free_fast_mlp(m->mlp);
   delete m;
 }
 
@@ -347,6 +349,7 @@ ks_status ks_model_create_mlp(ks_ctx* ctx, int n_layers, const int* h_widths,
   }
   if (e == cudaSuccess) e = upload(&m->mlp.d_mu, h_mu, static_cast<size_t>(KS_F_PAD));
   if (e == cudaSuccess) e = upload(&m->mlp.d_sigma, h_sigma, static_cast<size_t>(KS_F_PAD));
+  if (e == cudaSuccess) e = ks::build_fast_mlp(m->mlp, h_w_bf16, h_bias, h_mu, h_sigma);
   if (e != cudaSuccess) {
     ks_status s = cuda_fail(ctx, e, "ks_model_create_mlp");
     free_model(m);

@@ -16,6 +16,14 @@ namespace ks {
 
 constexpr int kRow = KS_F_PAD;
 
+// What a feature column depends on (Table "Feature groups"): 0 problem only, 1 candidate only
+// (given the element types), 2 both.
+__host__ __device__ constexpr int feat_class(int col) {
+  return (col <= 9 || col == 37 || col == 40 || col == 45) ? 0
+         : ((col >= 10 && col <= 22) || col == 38 || (col >= 46 && col <= 59) || col == 62) ? 1
+                                                                                            : 2;
+}
+
 __device__ __forceinline__ float F64i(long long v) { return __ll2float_rn(v); }
 __device__ __forceinline__ float F32i(int v) { return __int2float_rn(v); }
 __device__ __forceinline__ unsigned cdiv_u32(unsigned a, unsigned b) { return (a + b - 1u) / b; }

@@ -60,14 +60,6 @@ constexpr int kOffBuf0 = 0;
 constexpr int kOffBuf1 = kBufBytes;
 constexpr int kOffTile = 2 * kBufBytes;
 
-// What a feature column depends on (Table "Feature groups"): 0 problem only, 1 candidate only
-// (given the element types), 2 both.
-__host__ __device__ constexpr int feat_class(int col) {
-  return (col <= 9 || col == 37 || col == 40 || col == 45) ? 0
-         : ((col >= 10 && col <= 22) || col == 38 || (col >= 46 && col <= 59) || col == 62) ? 1
-                                                                                            : 2;
-}
-
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }

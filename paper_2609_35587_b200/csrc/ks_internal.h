@@ -17,6 +17,14 @@ struct FastTopParams {
   uint2 w[kFastTopPairs];
 };
 
+// Constants of the tensor-core MLP path that travel as a kernel parameter (constant bank):
+// folded standardisation per K position, biases, the last layer's weights widened to fp32.
+struct MlpTcParams {
+  float scale[64], shift[64];
+  float b1[256], b2[256], w3[256];
+  float b3;
+};
+
 // Generic device form of a tree node: 8 bytes, children tree-relative.
 struct DevNode {
   float v;        // threshold, or the leaf value
@@ -55,6 +63,10 @@ struct MlpModel {
   float* d_b[KS_MLP_MAX_LAYERS] = {nullptr};
   float* d_mu = nullptr;
   float* d_sigma = nullptr;
+  // tensor-core path (shape 64-256-256-1 only), see ks_mlp_tc.cu
+  bool tc = false;
+  uint16_t* d_tc_image = nullptr;      // W1 and W2 in the shared-memory operand layout
+  MlpTcParams* h_tc_params = nullptr;  // host copy, passed by value at every launch
 };
 
 // kernel-side view of an MLP (passed by value)
@@ -104,6 +116,8 @@ constexpr int kFastThreads = 1024;      // threads per block of the quantised tr
 constexpr int kFastR = 2;              // candidates per thread there
 constexpr int kFastRows = kFastThreads * kFastR;
 constexpr int kFastMaxDepth = 10;
+constexpr int kMlpThreads = 256;        // threads per block of the tensor-core MLP kernel
+constexpr int kMlpRows = 2048;          // candidates one block ranks per pass
 constexpr int kMaxSliceBlocks = 1024;  // candidate blocks the slice mode supports
 
 // Builds the quantised fast form of a validated ensemble when it qualifies (m.fast).
@@ -130,6 +144,18 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
                                cudaStream_t stream, int64_t* launches, cudaEvent_t ev_begin,
                                const FastSlice* slice = nullptr);
 int fast_slices(const GbdtModel& g, int nblk);
+
+// Tensor-core MLP path.
+cudaError_t build_fast_mlp(MlpModel& m, const uint16_t* const* h_w, const float* const* h_b, const float* h_mu,
+                           const float* h_sigma);
+void free_fast_mlp(MlpModel& m);
+int mlp_tc_blocks_per_problem(int64_t per_problem);
+size_t mlp_tc_scratch_bytes(int C);
+cudaError_t launch_select_mlp_tc(const ks_gpu_desc& desc, const MlpModel& m, const ks_problem* d_p,
+                                 const ks_problem* p_by_value, int P, const ks_candidate* d_c, int C, int nblk,
+                                 const int64_t* seg_off, const int32_t* seg_idx, int k,
+                                 unsigned long long* partial, void* scratch, int* status, cudaStream_t stream,
+                                 int64_t* launches, cudaEvent_t ev_begin);
 
 // ---- launchers (each enqueues on `stream`, returns the cudaError of the launch) -----------
 cudaError_t launch_featurize(const ks_gpu_desc& desc, const ks_problem* d_p, int P,

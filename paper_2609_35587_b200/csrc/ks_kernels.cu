@@ -392,6 +392,11 @@ size_t select_partial_bytes(const ks_model& model, int P, int C, int64_t pairs, 
     const size_t part = (static_cast<size_t>(P) * nblk * k * sizeof(unsigned long long) + 255) / 256 * 256;
     return part + fast_scratch_bytes(C);
   }
+  if (model.kind == 1 && model.mlp.tc) {
+    const int nblk = mlp_tc_blocks_per_problem(per);
+    const size_t part = (static_cast<size_t>(P) * nblk * k * sizeof(unsigned long long) + 255) / 256 * 256;
+    return part + mlp_tc_scratch_bytes(C);
+  }
   const int st = pick_sub_tiles(P, per);
   int64_t nblk = (per + static_cast<int64_t>(st) * kBlock - 1) / (static_cast<int64_t>(st) * kBlock);
   if (nblk < 1) nblk = 1;
@@ -414,6 +419,20 @@ cudaError_t launch_select(const ks_gpu_desc& desc, const ks_model& model, const 
     cudaError_t e = launch_select_fast(desc, model.gbdt, d_p, p_by_value, P, d_c, C, nblk, rows, d_seg_off,
                                        d_seg_idx, k, part, static_cast<char*>(d_partial) + part_bytes, d_status,
                                        stream, launches, ev_begin);
+    if (e != cudaSuccess) return e;
+    if (ev_end) cudaEventRecord(ev_end, stream);
+    topk_merge_kernel<<<(P * 32 + kBlock - 1) / kBlock, kBlock, 0, stream>>>(part, P, nblk * k, k, d_topk_idx,
+                                                                            d_topk_score);
+    ++*launches;
+    return cudaGetLastError();
+  }
+  if (model.kind == 1 && model.mlp.tc) {
+    const int nblk = mlp_tc_blocks_per_problem(per);
+    unsigned long long* part = static_cast<unsigned long long*>(d_partial);
+    const size_t part_bytes = (static_cast<size_t>(P) * nblk * k * sizeof(unsigned long long) + 255) / 256 * 256;
+    cudaError_t e = launch_select_mlp_tc(desc, model.mlp, d_p, p_by_value, P, d_c, C, nblk, d_seg_off, d_seg_idx, k,
+                                         part, static_cast<char*>(d_partial) + part_bytes, d_status, stream,
+                                         launches, ev_begin);
     if (e != cudaSuccess) return e;
     if (ev_end) cudaEventRecord(ev_end, stream);
     topk_merge_kernel<<<(P * 32 + kBlock - 1) / kBlock, kBlock, 0, stream>>>(part, P, nblk * k, k, d_topk_idx,

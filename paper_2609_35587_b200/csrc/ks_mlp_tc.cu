@@ -1,0 +1,528 @@
+// Tensor-core path of the fused select kernel for the feed-forward ranker (Model B) of shape
+// 64 -> 256 -> 256 -> 1: bf16 operands, fp32 accumulation in tensor memory.
+//
+// One CTA (256 threads) ranks one problem against up to kMlpRows candidates, 128 at a time:
+//   F    the 128 feature rows are written straight into shared memory as the bf16 A operand
+//        (candidate-only columns come standardised from a per-call table, problem-only columns
+//        are constant per CTA, the per-pair columns are computed in registers);
+//   L1   4 x tcgen05.mma (M 128, N 256, K 16) against W1, accumulator in TMEM;
+//   E1   TMEM -> registers, + bias, ReLU, round to bf16, written back to shared memory as the A
+//        operand of the next layer (it overwrites the feature tile);
+//   L2   16 x tcgen05.mma against W2 into the same TMEM columns;
+//   E2   TMEM -> registers, + bias, ReLU, round to bf16, dot with w3 on the CUDA cores, + b3:
+//        the score; one ranking key per row.
+// Both weight matrices stay resident in shared memory for the CTA's lifetime; they arrive by
+// bulk async copies (cp.async.bulk, no multicast) of an image the host prepared in the
+// operand layout. All waits are bounded and report through the status word.
+//
+// Operand layout (no swizzle, K-major): element (row, k) of a [rows x K] operand lives at
+// (k / 8) * rows * 16 + row * 16 + (k % 8) * 2 bytes: planes of eight K-columns, 16 bytes per
+// row. In descriptor terms the two 8-column halves of one K = 16 step are `rows * 16` bytes
+// apart (leading offset) and groups of eight rows 128 bytes apart (stride offset).
+#include <cuda_bf16.h>
+
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "ks_features.cuh"
+#include "ks_internal.h"
+#include "ks_topk.cuh"
+
+namespace ks {
+
+namespace {
+
+constexpr int kT = kMlpThreads;
+constexpr int kTileRows = 128;
+constexpr int kTiles = kMlpRows / kTileRows;
+constexpr int kH = 256;                               // hidden width
+constexpr int kW1Bytes = kH * 64 * 2;                 // 32 KB
+constexpr int kW2Bytes = kH * kH * 2;                 // 128 KB
+constexpr int kABytes = kTileRows * kH * 2;           // 64 KB: H1 tile (the feature tile aliases its start)
+constexpr int kOffW1 = 0;
+constexpr int kOffW2 = kW1Bytes;
+constexpr int kOffA = kW1Bytes + kW2Bytes;
+constexpr int kSmemBytes = kOffA + kABytes;           // 224 KB
+constexpr int kPlaneA = kTileRows * 16;               // bytes per 8-column plane of an A operand
+constexpr int kPlaneB = kH * 16;                      // ... of a B operand
+constexpr int kSpinLimit = 1 << 22;
+constexpr int kCandRec = 64;                          // bytes per (combination, candidate) record
+constexpr int kCombos = 16;
+constexpr int kNC = 29, kNPair = 21, kNP = 13;        // columns per class
+
+// position of feature column `col` along K: candidate-only columns first, then per-pair, then
+// problem-only, each class in ascending column order; position 63 is the zero pad
+__host__ __device__ constexpr int kpos(int col) {
+  int pos = 0;
+  const int cls = feat_class(col);
+  const int base = cls == 1 ? 0 : (cls == 2 ? kNC : kNC + kNPair);
+  for (int c = 0; c < col; ++c)
+    if (feat_class(c) == cls) ++pos;
+  return base + pos;
+}
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+  for (int i = 0; i < kSpinLimit; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+      "l"(src), "r"(bytes), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// shared-memory matrix descriptor: no swizzle, K-major, version 1
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lead_bytes, uint32_t stride_bytes) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((saddr >> 4) & 0x3FFFu);
+  d |= static_cast<uint64_t>((lead_bytes >> 4) & 0x3FFFu) << 16;
+  d |= static_cast<uint64_t>((stride_bytes >> 4) & 0x3FFFu) << 32;
+  d |= 1ull << 46;
+  return d;
+}
+
+// instruction descriptor: D fp32, A and B bf16, both K-major, N = 256, M = 128
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | ((128u >> 4) << 24);
+
+__device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+      " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n" ::"r"(tmem_d),
+      "l"(a_desc), "l"(b_desc), "r"(kIdesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// 32 consecutive fp32 columns of this thread's TMEM lane
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  const __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&t);
+}
+__device__ __forceinline__ float round_bf16(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
+
+// ------------------------------------------------------------------------------------------
+// candidate-only columns, standardised and rounded to bf16, once per call
+// ------------------------------------------------------------------------------------------
+
+__global__ void mlp_combo_mask_kernel(const ks_problem* __restrict__ p, int P, unsigned* __restrict__ mask) {
+  unsigned m = 0;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < P; i += gridDim.x * blockDim.x)
+    m |= 1u << ((p[i].dtype_ab & 3) * 4 + (p[i].dtype_d & 3));
+  m = __reduce_or_sync(0xFFFFFFFFu, m);
+  if ((threadIdx.x & 31) == 0 && m) atomicOr(mask, m);
+}
+
+__global__ void __launch_bounds__(256)
+mlp_cand_cols_kernel(ks_gpu_desc desc, const ks_candidate* __restrict__ c, int C, const unsigned* mask_ptr,
+                     unsigned mask_value, const __grid_constant__ MlpTcParams prm, uint8_t* __restrict__ out) {
+  const int combo = blockIdx.y;
+  const unsigned mask = mask_ptr ? *mask_ptr : mask_value;
+  if (!((mask >> combo) & 1u)) return;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= C) return;
+  ks_problem fake{};
+  fake.m = fake.n = fake.k = 1;
+  fake.dtype_ab = static_cast<uint8_t>(combo >> 2);
+  fake.dtype_d = static_cast<uint8_t>(combo & 3);
+  ProblemTerms t;
+  problem_terms(fake, desc, t);
+  float x[32];
+#pragma unroll
+  for (int q = 0; q < 32; ++q) x[q] = 0.0f;
+  featurize_pair(t, c[i], desc, [&](int col, float v) {
+    if (feat_class(col) != 1) return;
+    const int k = kpos(col);
+    x[k] = fmaf(v, prm.scale[k], prm.shift[k]);
+  });
+  uint32_t w[16];
+#pragma unroll
+  for (int q = 0; q < 16; ++q) w[q] = pack_bf16(x[2 * q], x[2 * q + 1]);
+  uint4* dst = reinterpret_cast<uint4*>(out + (static_cast<size_t>(combo) * C + i) * kCandRec);
+#pragma unroll
+  for (int q = 0; q < 4; ++q) dst[q] = make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
+}
+
+// ------------------------------------------------------------------------------------------
+// epilogues (H = which half of the 256 columns this warp owns)
+// ------------------------------------------------------------------------------------------
+
+// E1: h1 = bf16(relu(acc + b1)) for 128 columns of this thread's row, written as A-operand planes
+template <int H>
+__device__ __forceinline__ void epilogue1(uint32_t tmem_row, uint32_t sA_row, const MlpTcParams& prm) {
+#pragma unroll
+  for (int blk = 0; blk < 4; ++blk) {
+    float v[32];
+    tmem_ld32(tmem_row + H * 128 + blk * 32, v);
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {  // eight columns = one plane
+      uint32_t w[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int j = H * 128 + blk * 32 + g * 8 + 2 * q;
+        w[q] = pack_bf16(fmaxf(v[g * 8 + 2 * q] + prm.b1[j], 0.0f), fmaxf(v[g * 8 + 2 * q + 1] + prm.b1[j + 1], 0.0f));
+      }
+      const int plane = (H * 128 + blk * 32 + g * 8) / 8;
+      asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(sA_row + plane * kPlaneA), "r"(w[0]), "r"(w[1]),
+                   "r"(w[2]), "r"(w[3])
+                   : "memory");
+    }
+  }
+}
+
+// E2: partial dot of bf16(relu(acc + b2)) with w3 over 128 columns of this thread's row
+template <int H>
+__device__ __forceinline__ float epilogue2(uint32_t tmem_row, const MlpTcParams& prm) {
+  float s = 0.0f;
+#pragma unroll
+  for (int blk = 0; blk < 4; ++blk) {
+    float v[32];
+    tmem_ld32(tmem_row + H * 128 + blk * 32, v);
+#pragma unroll
+    for (int q = 0; q < 32; ++q) {
+      const int j = H * 128 + blk * 32 + q;
+      s = fmaf(round_bf16(fmaxf(v[q] + prm.b2[j], 0.0f)), prm.w3[j], s);
+    }
+  }
+  return s;
+}
+
+// ------------------------------------------------------------------------------------------
+// the kernel
+// ------------------------------------------------------------------------------------------
+
+__global__ void __launch_bounds__(kT, 1)
+select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_problem p_value, int use_value,
+                     const ks_candidate* __restrict__ c, int P, int C, int nblk,
+                     const int64_t* __restrict__ seg_off, const int32_t* __restrict__ seg_idx,
+                     const uint8_t* __restrict__ w_image, const uint8_t* __restrict__ cand_cols, int k,
+                     unsigned long long* __restrict__ partial, int* __restrict__ status,
+                     const __grid_constant__ MlpTcParams prm) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  __shared__ ProblemTerms s_pt;
+  __shared__ __align__(8) unsigned long long s_bar[2];  // 0: weights, 1: MMA completion
+  __shared__ uint32_t s_tmem;
+  __shared__ uint32_t s_pwords[7];   // problem-only columns (positions 50..63) as packed bf16
+  __shared__ float s_halfsum[kTileRows];
+  __shared__ unsigned long long s_list[KS_MAX_K];
+  __shared__ int s_fail;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int prob = blockIdx.x / nblk, chunk = blockIdx.x % nblk;
+  int64_t lo, len;
+  if (seg_off) {
+    lo = seg_off[prob];
+    len = seg_off[prob + 1] - lo;
+  } else {
+    lo = static_cast<int64_t>(prob) * C;
+    len = C;
+  }
+  const uint32_t sbase = smem_u32(smem);
+  const uint32_t bar_w = smem_u32(&s_bar[0]), bar_mma = smem_u32(&s_bar[1]);
+
+  if (tid == 0) {
+    problem_terms(use_value ? p_value : p[prob], desc, s_pt);
+    ks_candidate dummy{};
+    dummy.tile_m = dummy.tile_n = dummy.tile_k = 64;
+    dummy.stages = dummy.cluster_m = dummy.cluster_n = 1;
+    float pv[16];
+#pragma unroll
+    for (int q = 0; q < 16; ++q) pv[q] = 0.0f;
+    featurize_pair(s_pt, dummy, desc, [&](int col, float v) {
+      if (feat_class(col) != 0) return;
+      const int kk = kpos(col);
+      pv[kk - (kNC + kNPair)] = fmaf(v, prm.scale[kk], prm.shift[kk]);
+    });
+#pragma unroll
+    for (int q = 0; q < 7; ++q) s_pwords[q] = pack_bf16(pv[2 * q], q == 6 ? 0.0f : pv[2 * q + 1]);
+    mbar_init(bar_w, 1);
+    mbar_init(bar_mma, 1);
+    s_fail = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    // both weight matrices, resident for the CTA's lifetime
+    fence_async_proxy();
+    mbar_expect_tx(bar_w, kW1Bytes + kW2Bytes);
+    for (int off = 0; off < kW1Bytes + kW2Bytes; off += 32768)
+      bulk_copy_g2s(sbase + kOffW1 + off, w_image + off, 32768, bar_w);
+  }
+  if (tid < KS_MAX_K) s_list[tid] = 0ull;
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(256)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = s_tmem;
+  const int quarter = warp & 3, half = warp >> 2;
+  const int trow = quarter * 32 + lane;                       // row of the tile this thread reads from TMEM
+  const uint32_t tmem_row = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
+  const uint32_t sA = sbase + kOffA;
+  const int combo = s_pt.dtype_ab * 4 + s_pt.dtype_d;
+  uint32_t mma_phase = 0;
+  bool failed = false;
+
+  if (!mbar_wait_bounded(bar_w, 0)) failed = true;
+
+  for (int64_t start = static_cast<int64_t>(chunk) * kMlpRows; start < len && !failed;
+       start += static_cast<int64_t>(nblk) * kMlpRows) {
+    unsigned long long keys[kTiles + 1];
+#pragma unroll
+    for (int q = 0; q <= kTiles; ++q) keys[q] = 0ull;
+    if (tid < k) keys[kTiles] = s_list[tid];
+#pragma unroll 1
+    for (int tile = 0; tile < kTiles; ++tile) {
+      const int64_t tile0 = start + static_cast<int64_t>(tile) * kTileRows;
+      if (tile0 >= len) break;  // uniform
+      // ---- F: feature rows -> A operand ---------------------------------------------------------
+      int my_idx = 0;
+      const bool live = tid < kTileRows && tile0 + tid < len;
+      if (tid < kTileRows) {
+        uint32_t w[32];
+#pragma unroll
+        for (int q = 0; q < 32; ++q) w[q] = 0u;
+        if (live) {
+          my_idx = seg_off ? seg_idx[lo + tile0 + tid] : static_cast<int>(tile0 + tid);
+          const ks_candidate cand = c[my_idx];
+          const uint4* rec = reinterpret_cast<const uint4*>(cand_cols + (static_cast<size_t>(combo) * C + my_idx) * kCandRec);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const uint4 r = __ldg(rec + q);
+            w[4 * q] = r.x; w[4 * q + 1] = r.y; w[4 * q + 2] = r.z; w[4 * q + 3] = r.w;
+          }
+          float x[64];
+          featurize_pair(s_pt, cand, desc, [&](int col, float v) {
+            if (feat_class(col) != 2) return;
+            const int kk = kpos(col);
+            x[kk] = fmaf(v, prm.scale[kk], prm.shift[kk]);
+          });
+          // positions 0..28 came from the table; 29..49 are the per-pair columns
+          w[14] = (w[14] & 0xFFFFu) | (pack_bf16(0.0f, x[29]) & 0xFFFF0000u);
+#pragma unroll
+          for (int q = 15; q < 25; ++q) w[q] = pack_bf16(x[2 * q], x[2 * q + 1]);
+#pragma unroll
+          for (int q = 0; q < 7; ++q) w[25 + q] = s_pwords[q];
+        }
+        const uint32_t dst = sA + tid * 16;
+#pragma unroll
+        for (int pl = 0; pl < 8; ++pl)
+          asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + pl * kPlaneA), "r"(w[4 * pl]),
+                       "r"(w[4 * pl + 1]), "r"(w[4 * pl + 2]), "r"(w[4 * pl + 3])
+                       : "memory");
+      }
+      fence_async_proxy();
+      tc_fence_before();
+      __syncthreads();
+      // ---- L1 -----------------------------------------------------------------------------------
+      if (tid == 0) {
+        tc_fence_after();
+#pragma unroll
+        for (int ks16 = 0; ks16 < 4; ++ks16)
+          umma(tmem, make_desc(sA + ks16 * 2 * kPlaneA, kPlaneA, 128),
+               make_desc(sbase + kOffW1 + ks16 * 2 * kPlaneB, kPlaneB, 128), ks16 > 0);
+        umma_commit(bar_mma);
+      }
+      if (!mbar_wait_bounded(bar_mma, mma_phase)) failed = true;
+      mma_phase ^= 1;
+      tc_fence_after();
+      // ---- E1 -----------------------------------------------------------------------------------
+      if (half == 0) epilogue1<0>(tmem_row, sA + trow * 16, prm);
+      else epilogue1<1>(tmem_row, sA + trow * 16, prm);
+      fence_async_proxy();
+      tc_fence_before();
+      __syncthreads();
+      // ---- L2 -----------------------------------------------------------------------------------
+      if (tid == 0) {
+        tc_fence_after();
+#pragma unroll
+        for (int ks16 = 0; ks16 < 16; ++ks16)
+          umma(tmem, make_desc(sA + ks16 * 2 * kPlaneA, kPlaneA, 128),
+               make_desc(sbase + kOffW2 + ks16 * 2 * kPlaneB, kPlaneB, 128), ks16 > 0);
+        umma_commit(bar_mma);
+      }
+      if (!mbar_wait_bounded(bar_mma, mma_phase)) failed = true;
+      mma_phase ^= 1;
+      tc_fence_after();
+      // ---- E2 -----------------------------------------------------------------------------------
+      const float part = half == 0 ? epilogue2<0>(tmem_row, prm) : epilogue2<1>(tmem_row, prm);
+      if (half == 1) s_halfsum[trow] = part;
+      tc_fence_before();
+      __syncthreads();
+      if (tid < kTileRows) {
+        // thread tid featurized row tid and (as warp tid / 32, half 0) read the same row from TMEM
+        const float score = (part + s_halfsum[tid]) + prm.b3;
+        const unsigned long long key = live ? make_key(score + 0.0f, my_idx) : 0ull;
+#pragma unroll
+        for (int q = 0; q < kTiles; ++q)
+          if (q == tile) keys[q] = key;
+      }
+      if (__syncthreads_or(failed)) {
+        failed = true;
+        break;
+      }
+    }
+    // rank this pass's keys (the A buffer is idle: use it as scratch)
+    __syncthreads();
+    block_topk<kTiles + 1>(keys, k, reinterpret_cast<unsigned long long*>(smem + kOffA), s_list);
+  }
+  if (failed && tid == 0 && status) atomicExch(status, KS_ERR_TIMEOUT);
+  if (tid < k) partial[(static_cast<size_t>(prob) * nblk + chunk) * k + tid] = failed ? 0ull : s_list[tid];
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256) : "memory");
+  }
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------
+// host
+// ------------------------------------------------------------------------------------------
+
+static float bf16_bits_to_float_host(uint16_t b) {
+  const uint32_t u = static_cast<uint32_t>(b) << 16;
+  float f;
+  std::memcpy(&f, &u, 4);
+  return f;
+}
+
+cudaError_t build_fast_mlp(MlpModel& m, const uint16_t* const* h_w, const float* const* h_b, const float* h_mu,
+                           const float* h_sigma) {
+  m.tc = false;
+  if (m.n_layers != 3 || m.widths[0] != 64 || m.widths[1] != kH || m.widths[2] != kH || m.widths[3] != 1)
+    return cudaSuccess;  // other shapes stay on the generic kernel
+  // column order along K and the folded standardisation x' = x * scale + shift
+  int col_at[64];
+  for (int q = 0; q < 64; ++q) col_at[q] = -1;
+  for (int col = 0; col < KS_F; ++col) col_at[kpos(col)] = col;
+  MlpTcParams* prm = new (std::nothrow) MlpTcParams();
+  if (!prm) return cudaErrorMemoryAllocation;
+  for (int kk = 0; kk < 64; ++kk) {
+    prm->scale[kk] = 0.0f;
+    prm->shift[kk] = 0.0f;
+    if (col_at[kk] >= 0) {
+      const double s = 1.0 / static_cast<double>(h_sigma[col_at[kk]]);
+      prm->scale[kk] = static_cast<float>(s);
+      prm->shift[kk] = static_cast<float>(-static_cast<double>(h_mu[col_at[kk]]) * s);
+    }
+  }
+  for (int j = 0; j < kH; ++j) {
+    prm->b1[j] = h_b[0][j];
+    prm->b2[j] = h_b[1][j];
+    prm->w3[j] = bf16_bits_to_float_host(h_w[2][j]);
+  }
+  prm->b3 = h_b[2][0];
+  // operand images: plane (k / 8), 16 bytes per output unit
+  std::vector<uint16_t> img((kW1Bytes + kW2Bytes) / 2, 0);
+  for (int n = 0; n < kH; ++n)
+    for (int kk = 0; kk < 64; ++kk)
+      if (col_at[kk] >= 0)
+        img[(kk / 8) * (kPlaneB / 2) + n * 8 + (kk % 8)] = h_w[0][static_cast<size_t>(n) * 64 + col_at[kk]];
+  uint16_t* w2 = img.data() + kW1Bytes / 2;
+  for (int n = 0; n < kH; ++n)
+    for (int kk = 0; kk < kH; ++kk) w2[(kk / 8) * (kPlaneB / 2) + n * 8 + (kk % 8)] = h_w[1][static_cast<size_t>(n) * kH + kk];
+  cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&m.d_tc_image), img.size() * 2);
+  if (e == cudaSuccess) e = cudaMemcpy(m.d_tc_image, img.data(), img.size() * 2, cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) {
+    delete prm;
+    return e;
+  }
+  m.h_tc_params = prm;
+  m.tc = true;
+  return cudaSuccess;
+}
+
+void free_fast_mlp(MlpModel& m) {
+  delete m.h_tc_params;
+  m.h_tc_params = nullptr;
+}
+
+int mlp_tc_blocks_per_problem(int64_t per_problem) {
+  const int64_t n = (per_problem + kMlpRows - 1) / kMlpRows;
+  return static_cast<int>(n < 1 ? 1 : n);
+}
+
+size_t mlp_tc_scratch_bytes(int C) { return 256 + static_cast<size_t>(kCombos) * C * kCandRec; }
+
+cudaError_t launch_select_mlp_tc(const ks_gpu_desc& desc, const MlpModel& m, const ks_problem* d_p,
+                                 const ks_problem* p_by_value, int P, const ks_candidate* d_c, int C, int nblk,
+                                 const int64_t* seg_off, const int32_t* seg_idx, int k,
+                                 unsigned long long* partial, void* scratch, int* status, cudaStream_t stream,
+                                 int64_t* launches, cudaEvent_t ev_begin) {
+  ks_problem pv{};
+  if (p_by_value) pv = *p_by_value;
+  const int uv = p_by_value != nullptr;
+  unsigned* d_mask = static_cast<unsigned*>(scratch);
+  uint8_t* d_cols = static_cast<uint8_t*>(scratch) + 256;
+  unsigned mask_value = 0;
+  cudaError_t e;
+  if (uv) {
+    mask_value = 1u << ((pv.dtype_ab & 3) * 4 + (pv.dtype_d & 3));
+  } else {
+    e = cudaMemsetAsync(d_mask, 0, sizeof(unsigned), stream);
+    if (e != cudaSuccess) return e;
+    mlp_combo_mask_kernel<<<P >= 4096 ? 16 : 1, 256, 0, stream>>>(d_p, P, d_mask);
+    ++*launches;
+  }
+  if (C > 0) {
+    mlp_cand_cols_kernel<<<dim3((C + 255) / 256, kCombos), 256, 0, stream>>>(desc, d_c, C, uv ? nullptr : d_mask,
+                                                                             mask_value, *m.h_tc_params, d_cols);
+    ++*launches;
+  }
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  if (ev_begin) cudaEventRecord(ev_begin, stream);
+  e = cudaFuncSetAttribute(select_mlp_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  if (e != cudaSuccess) return e;
+  select_mlp_tc_kernel<<<static_cast<unsigned>(static_cast<int64_t>(P) * nblk), kT, kSmemBytes, stream>>>(
+      desc, d_p, pv, uv, d_c, P, C, nblk, seg_off, seg_idx, reinterpret_cast<const uint8_t*>(m.d_tc_image), d_cols, k,
+      partial, status, *m.h_tc_params);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+}  // namespace ks

@@ -253,6 +253,38 @@ def test_select_mlp(ks, ctx):
     check_select(w, idx, sc, TOL_MLP)
 
 
+def test_select_mlp_every_score(ks, ctx):
+    """k >= |segment| returns every pair's score: each one against the oracle, on sizes that
+    cross the 128-row tile and the 2,048-row block of the tensor-core kernel."""
+    for C in (1, 32, 127, 129):
+        w = wl.make_workload(4, P=5, C=C)
+        model = ctx.model_create_mlp(w.mlp)
+        idx, sc = run_select(ks, ctx, w, model, 32)
+        _, _, allsc = oracle.select(w.problems, w.candidates, DESC, 32, mlp=w.mlp, want_scores=True)
+        for i in range(5):
+            ref = allsc[i * C:(i + 1) * C]
+            n = min(C, 32)
+            got_idx = idx[i, :n]
+            assert len(set(got_idx.tolist())) == n and got_idx.min() >= 0 and got_idx.max() < C
+            err = np.abs(sc[i, :n] - ref[got_idx]) / np.maximum(1, np.abs(ref[got_idx]))
+            assert err.max() < 5e-3, (C, i, err.max())
+            assert np.all(idx[i, n:] == -1)
+    w = wl.make_workload(4, P=2, C=4500)
+    model = ctx.model_create_mlp(w.mlp)
+    idx, sc = run_select(ks, ctx, w, model, 32)
+    check_select(w, idx, sc, TOL_MLP)
+    _, _, allsc = oracle.select(w.problems, w.candidates, DESC, 32, mlp=w.mlp, want_scores=True)
+    for i in range(2):
+        ref = allsc[i * 4500:(i + 1) * 4500]
+        err = np.abs(sc[i] - ref[idx[i]]) / np.maximum(1, np.abs(ref[idx[i]]))
+        assert err.max() < 5e-3
+    # a second MLP shape stays on the generic kernel
+    m2 = wl.mlp_xavier(11, [64, 128, 64, 1], w.mlp["mu"], w.mlp["sigma"])
+    w2 = wl.Workload("mlp2", DESC, w.problems, w.candidates[:300], 10, mlp=m2)
+    idx, sc = run_select(ks, ctx, w2, ctx.model_create_mlp(m2))
+    check_select(w2, idx, sc, TOL_MLP)
+
+
 def test_select_one_and_select_host_agree_with_select(ks, ctx):
     w = wl.make_workload(3, P=4, C=3000, trees=30)
     model = ctx.model_create_gbdt(*w.gbdt)
