@@ -96,6 +96,16 @@ typedef struct {
   int32_t left;    /* index of the left child (right child = left + 1); 0 for a leaf       */
 } ks_node_host;    /* 12 bytes                                                             */
 
+/* Device form of a tree node, for ks_select_trees_static only (models created through
+ * ks_model_create_gbdt are repacked by the library). 8 bytes. */
+typedef struct {
+  float thr_or_leaf; /* threshold of an internal node, value of a leaf                    */
+  uint16_t feat;     /* 0 .. KS_F-1, or 0xFFFF for a leaf                                  */
+  uint16_t left;     /* tree-relative index of the left child (right child = left + 1)     */
+} ks_node_dev;
+
+#define KS_STATIC_MAX_KEYS 524288 /* partial top-k entries ks_select_trees_static can hold  */
+
 typedef struct ks_ctx ks_ctx;
 typedef struct ks_model ks_model;
 
@@ -179,6 +189,43 @@ ks_status ks_select_host(ks_ctx* ctx, const ks_problem* h_p, int P, const ks_can
                          int C, const int64_t* h_seg_offsets, const int32_t* h_seg_index,
                          int64_t pairs, const ks_model* model, int k, int32_t* h_topk_idx,
                          float* h_topk_score, void* stream);
+
+/* ---- selection without any allocation ------------------------------------------------------- */
+
+/* (The paper has no counterpart: this entry point exists for deployment reasons only.)
+ * The dense form of ks_select for a tree ensemble, for callers that cannot allocate device
+ * memory at all: processes whose own pool already owns the whole GPU, code running between
+ * cudaStreamBeginCapture and EndCapture or inside a stream-ordered pipeline that a
+ * synchronising cudaMalloc / cudaFree would stall, hosts that forbid driver allocations after
+ * start-up. Such callers cannot create a ks_ctx or ks_model (both own device buffers), so
+ * everything arrives as plain device pointers on device `cuda_device`:
+ *   d_nodes / d_tree_offsets  the ensemble as ks_node_dev records, tree t occupying
+ *                             [d_tree_offsets[t], d_tree_offsets[t+1]) (n_trees + 1 int32 offsets),
+ *                             node 0 of a tree its root. The arrays are NOT validated (they are
+ *                             device memory): child indices must stay inside their tree, feature
+ *                             ids below KS_F, depth at most KS_MAX_DEPTH.
+ *   d_p[P], d_c[C]            problems and the candidate pool; every problem is ranked against
+ *                             the whole pool.
+ *   d_topk_idx / d_topk_score [P, k] results as for ks_select.
+ * The call launches the same fused kernels as ks_select's generic tree path, asynchronously on
+ * `stream`, and calls no cudaMalloc, cudaFree or other allocating routine. The only scratch the
+ * kernels need, the per-block partial top-k lists, lives in a fixed 4 MiB array inside the
+ * library image (every GPU that loads libks holds it until the process exits). Limits and rules:
+ *   - P * B * k must not exceed KS_STATIC_MAX_KEYS, where B <= ceil(C / 256) is the number of
+ *     candidate blocks per problem the launcher picks; P * ceil(C / 256) * k <=
+ *     KS_STATIC_MAX_KEYS is always sufficient. Larger requests return KS_ERR_UNSUPPORTED and
+ *     launch nothing.
+ *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress);
+ *     make that first call outside any stream capture.
+ *   - All calls share the one array, which keeps the previous call's contents. The kernels
+ *     write every entry they later read, so nothing has to be cleared, but two calls whose
+ *     kernels overlap on the GPU (different streams, or different host threads) race on it:
+ *     serialise them.
+ * Returns KS_OK, KS_ERR_INVALID_ARG, KS_ERR_UNSUPPORTED or KS_ERR_CUDA. */
+ks_status ks_select_trees_static(int cuda_device, const ks_gpu_desc* desc, const ks_problem* d_p, int P,
+                                 const ks_candidate* d_c, int C, const ks_node_dev* d_nodes,
+                                 const int32_t* d_tree_offsets, int n_trees, float base_score, int k,
+                                 int32_t* d_topk_idx, float* d_topk_score, void* stream);
 
 /* ---- introspection -------------------------------------------------------------------- */
 

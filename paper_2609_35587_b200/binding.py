@@ -21,7 +21,7 @@ KS_OK, KS_ERR_INVALID_ARG, KS_ERR_UNSUPPORTED, KS_ERR_CUDA, KS_ERR_TIMEOUT, KS_E
 EXPORTS = ("ks_create", "ks_destroy", "ks_last_cuda_error", "ks_model_create_gbdt",
            "ks_model_create_mlp", "ks_model_destroy", "ks_featurize", "ks_score", "ks_select",
            "ks_select_one", "ks_select_host", "ks_status_string", "ks_feature_count",
-           "ks_feature_name", "ks_launch_count", "ks_profile_enable", "ks_profile_last_ms", "ks_device_status")
+           "ks_feature_name", "ks_launch_count", "ks_profile_enable", "ks_profile_last_ms", "ks_device_status", "ks_select_trees_static")
 
 
 class KsError(RuntimeError):
@@ -64,6 +64,7 @@ def _load() -> ctypes.CDLL:
     lib.ks_launch_count.restype = i64
     lib.ks_profile_enable.argtypes = [vp, i32]
     lib.ks_device_status.argtypes = [vp]
+    lib.ks_select_trees_static.argtypes = [i32, vp, vp, i32, vp, i32, vp, vp, i32, ctypes.c_float, i32, vp, vp, vp]
     lib.ks_profile_last_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     for name in EXPORTS:
         fn = getattr(lib, name)
@@ -118,6 +119,19 @@ def to_device(records: np.ndarray, device) -> torch.Tensor:
     if a.dtype.fields is not None:
         a = a.view(np.uint8).reshape(len(records), -1)
     return torch.from_numpy(a.copy()).to(device)
+
+
+NODE_DEV_DT = np.dtype([("v", "<f4"), ("feat", "<u2"), ("left", "<u2")])
+
+
+def ks_select_trees_static(desc: np.ndarray, d_p, P, d_c, C, d_nodes, d_tree_offsets, n_trees, base_score, k,
+                           d_topk_idx, d_topk_score, device: int = 0) -> int:
+    """Raw call of the allocation-free entry point: every buffer is the caller's (torch device
+    tensors here), nothing is allocated on the way; returns the ks_status."""
+    d = np.ascontiguousarray(desc).reshape(1)
+    return int(_lib.ks_select_trees_static(device, _hptr(d), _dptr(d_p), P, _dptr(d_c), C, _dptr(d_nodes),
+                                           _dptr(d_tree_offsets), n_trees, ctypes.c_float(base_score), k,
+                                           _dptr(d_topk_idx), _dptr(d_topk_score), _stream()))
 
 
 class Model:

@@ -476,4 +476,31 @@ cudaError_t launch_select(const ks_gpu_desc& desc, const ks_model& model, const 
   return cudaGetLastError();
 }
 
+
+// Generic tree select with caller-provided node arrays and partial-list storage (dense form).
+int64_t select_generic_partial_keys(int P, int C, int k) {
+  const int st = pick_sub_tiles(P, C);
+  const PairMap map = make_map(P, C, static_cast<int64_t>(P) * C, nullptr, nullptr, st * kBlock);
+  return static_cast<int64_t>(P) * map.nblk * k;
+}
+
+cudaError_t launch_select_generic_trees(const ks_gpu_desc& desc, const DevNode* d_nodes, const int* d_roots,
+                                        int n_trees, float base, const ks_problem* d_p, int P,
+                                        const ks_candidate* d_c, int C, int k, unsigned long long* partial,
+                                        int32_t* d_topk_idx, float* d_topk_score, cudaStream_t stream) {
+  const int st = pick_sub_tiles(P, C);
+  const PairMap map = make_map(P, C, static_cast<int64_t>(P) * C, nullptr, nullptr, st * kBlock);
+  const size_t smem = sizeof(float) * kRow * kBlock;
+  cudaError_t e = cudaFuncSetAttribute(select_generic_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       static_cast<int>(smem));
+  if (e != cudaSuccess) return e;
+  select_generic_kernel<0><<<static_cast<unsigned>(static_cast<int64_t>(P) * map.nblk), kBlock, smem, stream>>>(
+      desc, d_p, ks_problem{}, 0, d_c, map, st, d_nodes, d_roots, n_trees, base, MlpView{}, 0, k, partial);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  topk_merge_kernel<<<(P * 32 + kBlock - 1) / kBlock, kBlock, 0, stream>>>(partial, P, map.nblk * k, k,
+                                                                          d_topk_idx, d_topk_score);
+  return cudaGetLastError();
+}
+
 }  // namespace ks
