@@ -245,6 +245,7 @@ def main():
     import torch
     import torch.distributed as dist
     from paper_2609_35587_b200 import binding as ks
+    from paper_2609_35587_b200 import sharding
     from paper_2609_35587_b200 import workloads as wl
 
     torch.cuda.set_device(local_rank)
@@ -304,10 +305,8 @@ def main():
     clocks = sampler.stop()
     step_ms = [a.elapsed_time(b) for a, b in ev]
     total_ms = float(sum(step_ms))
-    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
     if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms = float(t.item())
+        total_ms = sharding.max_over_ranks(total_ms, dev)
     ms_per_step = total_ms / args.steps
     value = world * pairs / (ms_per_step * 1e-3)
 
@@ -328,10 +327,9 @@ def main():
         ctx.select_host(h_p, P, h_c, C, model, k, h_so, h_si, pairs, h_idx, h_sc)
     barrier()
     e2e_s = (time.perf_counter() - t0) / max(e2e_steps, 1)
-    t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
     if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_value = world * pairs / float(t.item())
+        e2e_s = sharding.max_over_ranks(e2e_s, dev)
+    e2e_value = world * pairs / e2e_s
     h2d = P * 16 + C * 16 + (0 if h_so is None else h_so.numel() * 8 + h_si.numel() * 4)
     d2h = P * k * 8
 
