@@ -370,7 +370,7 @@ def main():
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, per launch, from the
 # ncu summaries under profiles/ (None until a capture exists for that workload).
-TRAFFIC_BYTES = {}
+TRAFFIC_BYTES = {1: 13.1e6, 4: 10.0e6}
 
 if __name__ == "__main__":
     main()

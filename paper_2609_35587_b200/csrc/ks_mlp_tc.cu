@@ -242,7 +242,7 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
                      const __grid_constant__ MlpTcParams prm) {
   extern __shared__ __align__(1024) unsigned char smem[];
   __shared__ ProblemTerms s_pt;
-  __shared__ __align__(8) unsigned long long s_bar[2];  // 0: weights, 1: MMA completion
+  __shared__ __align__(8) unsigned long long s_bar[4];  // weights; L2 first group; L2 second group; L1
   __shared__ uint32_t s_tmem;
   __shared__ uint32_t s_pwords[7];   // problem-only columns (positions 50..63) as packed bf16
   __shared__ float s_halfsum[kTileRows];
@@ -260,7 +260,8 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
     len = C;
   }
   const uint32_t sbase = smem_u32(smem);
-  const uint32_t bar_w = smem_u32(&s_bar[0]), bar_mma = smem_u32(&s_bar[1]);
+  const uint32_t bar_w = smem_u32(&s_bar[0]), bar_a = smem_u32(&s_bar[1]), bar_b = smem_u32(&s_bar[2]),
+                 bar_c = smem_u32(&s_bar[3]);
 
   if (tid == 0) {
     problem_terms(use_value ? p_value : p[prob], desc, s_pt);
@@ -278,7 +279,9 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
 #pragma unroll
     for (int q = 0; q < 7; ++q) s_pwords[q] = pack_bf16(pv[2 * q], q == 6 ? 0.0f : pv[2 * q + 1]);
     mbar_init(bar_w, 1);
-    mbar_init(bar_mma, 1);
+    mbar_init(bar_a, 1);
+    mbar_init(bar_b, 1);
+    mbar_init(bar_c, 1);
     s_fail = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     // both weight matrices, resident for the CTA's lifetime
@@ -289,7 +292,7 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
   }
   if (tid < KS_MAX_K) s_list[tid] = 0ull;
   if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(256)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(512)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -302,10 +305,62 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
   const uint32_t tmem_row = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
   const uint32_t sA = sbase + kOffA;
   const int combo = s_pt.dtype_ab * 4 + s_pt.dtype_d;
-  uint32_t mma_phase = 0;
   bool failed = false;
 
   if (!mbar_wait_bounded(bar_w, 0)) failed = true;
+
+  // Software pipeline over the tiles of a pass (two TMEM accumulators, one A buffer):
+  //   L2(t) is issued in two groups: K-steps 0-3 (they read the planes the feature tile
+  //   occupied) and K-steps 4-15. Once the first group is done, the feature rows of tile t+1
+  //   are written into those planes while the second group still runs. When L2(t) is complete,
+  //   L1(t+1) goes to the other accumulator and runs under the second epilogue of tile t; the
+  //   first epilogue of tile t+1 then rewrites the whole A buffer with its hidden layer.
+  auto feature_rows = [&](int64_t tile0, int& idx_out, bool& live_out) {
+    live_out = tid < kTileRows && tile0 + tid < len;
+    idx_out = 0;
+    if (tid < kTileRows) {
+      uint32_t w[32];
+#pragma unroll
+      for (int q = 0; q < 32; ++q) w[q] = 0u;
+      if (live_out) {
+        idx_out = seg_off ? seg_idx[lo + tile0 + tid] : static_cast<int>(tile0 + tid);
+        const ks_candidate cand = c[idx_out];
+        const uint4* rec = reinterpret_cast<const uint4*>(cand_cols + (static_cast<size_t>(combo) * C + idx_out) * kCandRec);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const uint4 r = __ldg(rec + q);
+          w[4 * q] = r.x; w[4 * q + 1] = r.y; w[4 * q + 2] = r.z; w[4 * q + 3] = r.w;
+        }
+        float x[64];
+        featurize_pair(s_pt, cand, desc, [&](int col, float v) {
+          if (feat_class(col) != 2) return;
+          const int kk = kpos(col);
+          x[kk] = fmaf(v, prm.scale[kk], prm.shift[kk]);
+        });
+        // positions 0..28 came from the table; 29..49 are the per-pair columns
+        w[14] = (w[14] & 0xFFFFu) | (pack_bf16(0.0f, x[29]) & 0xFFFF0000u);
+#pragma unroll
+        for (int q = 15; q < 25; ++q) w[q] = pack_bf16(x[2 * q], x[2 * q + 1]);
+#pragma unroll
+        for (int q = 0; q < 7; ++q) w[25 + q] = s_pwords[q];
+      }
+      const uint32_t dst = sA + tid * 16;
+#pragma unroll
+      for (int pl = 0; pl < 8; ++pl)
+        asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + pl * kPlaneA), "r"(w[4 * pl]),
+                     "r"(w[4 * pl + 1]), "r"(w[4 * pl + 2]), "r"(w[4 * pl + 3])
+                     : "memory");
+    }
+    fence_async_proxy();
+  };
+  auto issue_l1 = [&](uint32_t acc) {
+#pragma unroll
+    for (int ks16 = 0; ks16 < 4; ++ks16)
+      umma(acc, make_desc(sA + ks16 * 2 * kPlaneA, kPlaneA, 128),
+           make_desc(sbase + kOffW1 + ks16 * 2 * kPlaneB, kPlaneB, 128), ks16 > 0);
+    umma_commit(bar_c);
+  };
+  uint32_t ph_a = 0, ph_b = 0, ph_c = 0;
 
   for (int64_t start = static_cast<int64_t>(chunk) * kMlpRows; start < len && !failed;
        start += static_cast<int64_t>(nblk) * kMlpRows) {
@@ -313,92 +368,83 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
 #pragma unroll
     for (int q = 0; q <= kTiles; ++q) keys[q] = 0ull;
     if (tid < k) keys[kTiles] = s_list[tid];
+    const int64_t rows_left = len - start;
+    const int n_tiles = static_cast<int>(rows_left >= kMlpRows ? kTiles : (rows_left + kTileRows - 1) / kTileRows);
+
+    // ---- prologue: tile 0 up to its hidden layer -------------------------------------------------
+    int cur_idx, nxt_idx = 0;
+    bool cur_live, nxt_live = false;
+    __syncthreads();  // the previous pass's ranking scratch (A buffer) is no longer read
+    feature_rows(start, cur_idx, cur_live);
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0) {
+      tc_fence_after();
+      issue_l1(tmem);
+    }
+    if (!mbar_wait_bounded(bar_c, ph_c)) failed = true;
+    ph_c ^= 1;
+    tc_fence_after();
+    if (half == 0) epilogue1<0>(tmem_row, sA + trow * 16, prm);
+    else epilogue1<1>(tmem_row, sA + trow * 16, prm);
+    fence_async_proxy();
+    tc_fence_before();
+    __syncthreads();
+
 #pragma unroll 1
-    for (int tile = 0; tile < kTiles; ++tile) {
-      const int64_t tile0 = start + static_cast<int64_t>(tile) * kTileRows;
-      if (tile0 >= len) break;  // uniform
-      // ---- F: feature rows -> A operand ---------------------------------------------------------
-      int my_idx = 0;
-      const bool live = tid < kTileRows && tile0 + tid < len;
-      if (tid < kTileRows) {
-        uint32_t w[32];
-#pragma unroll
-        for (int q = 0; q < 32; ++q) w[q] = 0u;
-        if (live) {
-          my_idx = seg_off ? seg_idx[lo + tile0 + tid] : static_cast<int>(tile0 + tid);
-          const ks_candidate cand = c[my_idx];
-          const uint4* rec = reinterpret_cast<const uint4*>(cand_cols + (static_cast<size_t>(combo) * C + my_idx) * kCandRec);
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const uint4 r = __ldg(rec + q);
-            w[4 * q] = r.x; w[4 * q + 1] = r.y; w[4 * q + 2] = r.z; w[4 * q + 3] = r.w;
-          }
-          float x[64];
-          featurize_pair(s_pt, cand, desc, [&](int col, float v) {
-            if (feat_class(col) != 2) return;
-            const int kk = kpos(col);
-            x[kk] = fmaf(v, prm.scale[kk], prm.shift[kk]);
-          });
-          // positions 0..28 came from the table; 29..49 are the per-pair columns
-          w[14] = (w[14] & 0xFFFFu) | (pack_bf16(0.0f, x[29]) & 0xFFFF0000u);
-#pragma unroll
-          for (int q = 15; q < 25; ++q) w[q] = pack_bf16(x[2 * q], x[2 * q + 1]);
-#pragma unroll
-          for (int q = 0; q < 7; ++q) w[25 + q] = s_pwords[q];
-        }
-        const uint32_t dst = sA + tid * 16;
-#pragma unroll
-        for (int pl = 0; pl < 8; ++pl)
-          asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + pl * kPlaneA), "r"(w[4 * pl]),
-                       "r"(w[4 * pl + 1]), "r"(w[4 * pl + 2]), "r"(w[4 * pl + 3])
-                       : "memory");
-      }
-      fence_async_proxy();
-      tc_fence_before();
-      __syncthreads();
-      // ---- L1 -----------------------------------------------------------------------------------
+    for (int tile = 0; tile < n_tiles; ++tile) {
+      const uint32_t acc = tmem + (tile & 1) * 256, acc_next = tmem + ((tile + 1) & 1) * 256;
+      const uint32_t acc_row = tmem_row + (tile & 1) * 256, acc_next_row = tmem_row + ((tile + 1) & 1) * 256;
+      const bool has_next = tile + 1 < n_tiles;
+      // ---- L2(tile), in two groups -----------------------------------------------------------------
       if (tid == 0) {
         tc_fence_after();
 #pragma unroll
         for (int ks16 = 0; ks16 < 4; ++ks16)
-          umma(tmem, make_desc(sA + ks16 * 2 * kPlaneA, kPlaneA, 128),
-               make_desc(sbase + kOffW1 + ks16 * 2 * kPlaneB, kPlaneB, 128), ks16 > 0);
-        umma_commit(bar_mma);
-      }
-      if (!mbar_wait_bounded(bar_mma, mma_phase)) failed = true;
-      mma_phase ^= 1;
-      tc_fence_after();
-      // ---- E1 -----------------------------------------------------------------------------------
-      if (half == 0) epilogue1<0>(tmem_row, sA + trow * 16, prm);
-      else epilogue1<1>(tmem_row, sA + trow * 16, prm);
-      fence_async_proxy();
-      tc_fence_before();
-      __syncthreads();
-      // ---- L2 -----------------------------------------------------------------------------------
-      if (tid == 0) {
-        tc_fence_after();
-#pragma unroll
-        for (int ks16 = 0; ks16 < 16; ++ks16)
-          umma(tmem, make_desc(sA + ks16 * 2 * kPlaneA, kPlaneA, 128),
+          umma(acc, make_desc(sA + ks16 * 2 * kPlaneA, kPlaneA, 128),
                make_desc(sbase + kOffW2 + ks16 * 2 * kPlaneB, kPlaneB, 128), ks16 > 0);
-        umma_commit(bar_mma);
+        umma_commit(bar_a);
+#pragma unroll
+        for (int ks16 = 4; ks16 < 16; ++ks16)
+          umma(acc, make_desc(sA + ks16 * 2 * kPlaneA, kPlaneA, 128),
+               make_desc(sbase + kOffW2 + ks16 * 2 * kPlaneB, kPlaneB, 128), 1u);
+        umma_commit(bar_b);
       }
-      if (!mbar_wait_bounded(bar_mma, mma_phase)) failed = true;
-      mma_phase ^= 1;
+      // ---- feature rows of the next tile under the second group --------------------------------------
+      if (!mbar_wait_bounded(bar_a, ph_a)) failed = true;
+      ph_a ^= 1;
+      if (has_next) {
+        feature_rows(start + static_cast<int64_t>(tile + 1) * kTileRows, nxt_idx, nxt_live);
+        tc_fence_before();
+        __syncthreads();
+      }
+      if (!mbar_wait_bounded(bar_b, ph_b)) failed = true;
+      ph_b ^= 1;
       tc_fence_after();
-      // ---- E2 -----------------------------------------------------------------------------------
-      const float part = half == 0 ? epilogue2<0>(tmem_row, prm) : epilogue2<1>(tmem_row, prm);
+      // ---- L1(tile + 1) into the other accumulator, under E2(tile) -----------------------------------
+      if (has_next && tid == 0) issue_l1(acc_next);
+      const float part = half == 0 ? epilogue2<0>(acc_row, prm) : epilogue2<1>(acc_row, prm);
       if (half == 1) s_halfsum[trow] = part;
-      tc_fence_before();
       __syncthreads();
       if (tid < kTileRows) {
-        // thread tid featurized row tid and (as warp tid / 32, half 0) read the same row from TMEM
         const float score = (part + s_halfsum[tid]) + prm.b3;
-        const unsigned long long key = live ? make_key(score + 0.0f, my_idx) : 0ull;
+        const unsigned long long key = cur_live ? make_key(score + 0.0f, cur_idx) : 0ull;
 #pragma unroll
         for (int q = 0; q < kTiles; ++q)
           if (q == tile) keys[q] = key;
       }
+      // ---- E1(tile + 1): the hidden layer replaces the A buffer -----------------------------------
+      if (has_next) {
+        if (!mbar_wait_bounded(bar_c, ph_c)) failed = true;
+        ph_c ^= 1;
+        tc_fence_after();
+        if (half == 0) epilogue1<0>(acc_next_row, sA + trow * 16, prm);
+        else epilogue1<1>(acc_next_row, sA + trow * 16, prm);
+        fence_async_proxy();
+        cur_idx = nxt_idx;
+        cur_live = nxt_live;
+      }
+      tc_fence_before();
       if (__syncthreads_or(failed)) {
         failed = true;
         break;
@@ -413,7 +459,7 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
   tc_fence_before();
   __syncthreads();
   if (warp == 0) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
   }
 }
 
