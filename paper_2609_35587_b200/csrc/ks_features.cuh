@@ -68,16 +68,106 @@ __device__ inline void problem_terms(const ks_problem& p, const ks_gpu_desc& h, 
   t.tc_rate = h.tc_flops_per_us_per_sm[t.dtype_ab];
 }
 
+// a / b rounded up for non-negative operands; takes the 32-bit path when both fit (same value)
+__device__ __forceinline__ long long cdiv_fit(long long a, long long b) {
+  if (((a | b) >> 32) == 0)
+    return static_cast<long long>(cdiv_u32(static_cast<unsigned>(a), static_cast<unsigned>(b)));
+  return cdiv_i64(a, b);
+}
+__device__ __forceinline__ long long div_fit(long long a, long long b) {
+  if (((a | b) >> 32) == 0) return static_cast<long long>(static_cast<unsigned>(a) / static_cast<unsigned>(b));
+  return a / b;
+}
+
+// kExact: IEEE round-to-nearest division (bit-identical to the CPU definition). !kExact: the
+// fast approximate division, for consumers that round the result to bf16 anyway.
+template <bool kExact>
+__device__ __forceinline__ float fdiv(float a, float b) {
+  return kExact ? __fdiv_rn(a, b) : __fdividef(a, b);
+}
+
+// Candidate-side resource terms (section "Resource Pressure and Occupancy"); they depend on the
+// problem only through its element sizes.
+struct Resources {
+  long long B_stage, smem_main, B_epi, B_smem, area, b_smem, b_reg, b_res, b_eff;
+  int T_block, n_cons, fits;
+  float f_smem;
+};
+
+__device__ __forceinline__ Resources resources(const ProblemTerms& t, const ks_candidate& c,
+                                               const ks_gpu_desc& h) {
+  Resources r;
+  const int TM = c.tile_m, TN = c.tile_n, TK = c.tile_k, S = c.stages;
+  const int ks = c.kernel_sched & 3;
+  // (consumer warpgroups in the mainloop, threads per block): WS, Pingpong, Cooperative, basic
+  r.n_cons = (ks == 2) ? 2 : 1;
+  r.T_block = (ks == 0) ? 256 : (ks == 3 ? 128 : 384);
+  const int bA = t.bA, bD = t.bD;
+  r.B_stage = static_cast<long long>(TK) * (TM * bA + TN * bA);
+  r.smem_main = S * r.B_stage;
+  const int E = (ks == 2) ? 128 : 64;
+  r.B_epi = (c.epi_sched == 0) ? 0 : 2ll * min(TM, E) * min(TN, 32) * bD;
+  const long long both = r.smem_main + r.B_epi + h.smem_reserved;
+  r.B_smem = (ks == 0 || ks == 3) ? max(r.smem_main, r.B_epi) + h.smem_reserved : both;
+  r.f_smem = __fdiv_rn(F64i(r.B_smem), F64i(h.smem_per_sm));
+  r.fits = both <= static_cast<long long>(h.smem_per_cta_max);
+  r.area = static_cast<long long>(TM) * TN;
+  r.b_smem = div_fit(static_cast<long long>(h.smem_per_sm), r.B_smem);
+  const long long regs = min(255ll, 32 + cdiv_fit(r.area, r.T_block));
+  r.b_reg = div_fit(static_cast<long long>(h.regs_per_sm), regs * r.T_block);
+  const long long b_arch =
+      min(static_cast<long long>(h.max_ctas_per_sm), static_cast<long long>(h.max_threads_per_sm / r.T_block));
+  r.b_res = min(r.b_smem, min(r.b_reg, b_arch));
+  r.b_eff = max(1ll, r.b_res);
+  return r;
+}
+
+// The columns that depend on both the problem and the candidate (sections "Work Decomposition
+// and Wave Quantization", "Memory Behavior", "Pipeline Balance"), given the candidate's
+// effective resident-block count b_eff.
+template <bool kExact, typename Put>
+__device__ __forceinline__ void pair_columns(const ProblemTerms& t, const ks_candidate& c, const ks_gpu_desc& h,
+                                             long long b_eff, Put put) {
+  const int TM = c.tile_m, TN = c.tile_n, TK = c.tile_k, S = c.stages;
+  const int cM = c.cluster_m, cN = c.cluster_n;
+  const int bA = t.bA;
+  const long long n_m = cdiv_u32(t.M, TM), n_n = cdiv_u32(t.N, TN), n_k = cdiv_u32(t.K, TK);
+  const long long n_tiles = n_m * n_n;
+  put(23, F64i(n_m));
+  put(24, F64i(n_n));
+  put(25, F64i(n_k));
+  put(26, F64i(n_tiles));
+  put(27, fdiv<kExact>(F64i(n_m * TM - t.M), F64i(t.M)));
+  put(28, fdiv<kExact>(F64i(n_n * TN - t.N), F64i(t.N)));
+  put(29, fdiv<kExact>(F64i(n_tiles), F64i(h.num_sms)));
+  const long long resident = static_cast<long long>(h.num_sms) * b_eff;
+  const long long waves = cdiv_fit(n_tiles, resident);
+  put(30, F64i(waves));
+  const float eta = fdiv<kExact>(F64i(n_tiles), F64i(waves * resident));
+  put(31, eta);
+  put(32, fmaxf(0.0f, __fsub_rn(1.0f, eta)));
+  const long long n_c = cdiv_fit(t.M, static_cast<long long>(cM) * TM) * cdiv_fit(t.N, static_cast<long long>(cN) * TN);
+  put(33, fdiv<kExact>(F64i(n_c * cM * cN - n_tiles), F64i(n_tiles)));
+  put(34, fdiv<kExact>(F64i(n_m), F64i(cM)));
+  put(35, fdiv<kExact>(F64i(n_n), F64i(cN)));
+  put(36, F32i(cM > n_m || cN > n_n));
+  const long long restream = n_n * t.bytesA + n_m * t.bytesB;
+  put(39, fdiv<kExact>(F64i(restream), F64i(t.bytesA + t.bytesB)));
+  const float fl2 = F64i(static_cast<long long>(h.l2_bytes));
+  put(41, fdiv<kExact>(F64i(static_cast<long long>(bA) * TM * t.K), fl2));
+  put(42, fdiv<kExact>(F64i(static_cast<long long>(bA) * TN * t.K), fl2));
+  put(43, F64i(restream));
+  put(44, F64i(cdiv_fit(n_n, cN) * t.bytesA + cdiv_fit(n_m, cM) * t.bytesB));
+  put(60, fdiv<kExact>(F64i(min(static_cast<long long>(S), n_k)), F32i(S)));
+  put(61, fdiv<kExact>(F64i(n_k), F32i(S)));
+}
+
 // Writes the 64 columns of one pair through `put(column, value)`.
 template <typename Put>
 __device__ __forceinline__ void featurize_pair(const ProblemTerms& t, const ks_candidate& c,
                                                const ks_gpu_desc& h, Put put) {
   const int TM = c.tile_m, TN = c.tile_n, TK = c.tile_k, S = c.stages;
   const int cM = c.cluster_m, cN = c.cluster_n;
-  const int ks = c.kernel_sched & 3;
-  // (consumer warpgroups in the mainloop, threads per block): WS, Pingpong, Cooperative, basic
-  const int n_cons = (ks == 2) ? 2 : 1;
-  const int T_block = (ks == 0) ? 256 : (ks == 3 ? 128 : 384);
   const int bA = t.bA, bD = t.bD;
 
   // ---- structural core ------------------------------------------------------------------
@@ -105,85 +195,36 @@ __device__ __forceinline__ void featurize_pair(const ProblemTerms& t, const ks_c
   put(21, F32i(cN));
   put(22, F32i(cM * cN));
 
-  // ---- resource pressure and occupancy ----------------------------------------------------
-  const long long B_stage = static_cast<long long>(TK) * (TM * bA + TN * bA);
-  const long long smem_main = S * B_stage;
-  const int E = (ks == 2) ? 128 : 64;
-  const long long B_epi =
-      (c.epi_sched == 0) ? 0 : 2ll * min(TM, E) * min(TN, 32) * bD;
-  const long long both = smem_main + B_epi + h.smem_reserved;
-  const long long B_smem =
-      (ks == 0 || ks == 3) ? max(smem_main, B_epi) + h.smem_reserved : both;
-  const float f_smem = __fdiv_rn(F64i(B_smem), F64i(h.smem_per_sm));
-  const int fits = both <= static_cast<long long>(h.smem_per_cta_max);
-  const long long area = static_cast<long long>(TM) * TN;
-  const long long b_smem = static_cast<long long>(h.smem_per_sm) / B_smem;
-  const long long regs = min(255ll, 32 + cdiv_i64(area, T_block));
-  const long long b_reg = static_cast<long long>(h.regs_per_sm) / (regs * T_block);
-  const long long b_arch =
-      min(static_cast<long long>(h.max_ctas_per_sm), static_cast<long long>(h.max_threads_per_sm / T_block));
-  const long long b_res = min(b_smem, min(b_reg, b_arch));
-  const long long b_eff = max(1ll, b_res);
+  const Resources r = resources(t, c, h);
+  pair_columns<true>(t, c, h, r.b_eff, put);
 
-  // ---- work decomposition and wave quantisation ---------------------------------------------
-  const long long n_m = cdiv_u32(t.M, TM), n_n = cdiv_u32(t.N, TN), n_k = cdiv_u32(t.K, TK);
-  const long long n_tiles = n_m * n_n;
-  put(23, F64i(n_m));
-  put(24, F64i(n_n));
-  put(25, F64i(n_k));
-  put(26, F64i(n_tiles));
-  put(27, __fdiv_rn(F64i(n_m * TM - t.M), F64i(t.M)));
-  put(28, __fdiv_rn(F64i(n_n * TN - t.N), F64i(t.N)));
-  put(29, __fdiv_rn(F64i(n_tiles), F64i(h.num_sms)));
-  const long long resident = static_cast<long long>(h.num_sms) * b_eff;
-  const long long waves = cdiv_i64(n_tiles, resident);
-  put(30, F64i(waves));
-  const float eta = __fdiv_rn(F64i(n_tiles), F64i(waves * resident));
-  put(31, eta);
-  put(32, fmaxf(0.0f, __fsub_rn(1.0f, eta)));
-  const long long n_c = static_cast<long long>(cdiv_i64(t.M, static_cast<long long>(cM) * TM)) *
-                        cdiv_i64(t.N, static_cast<long long>(cN) * TN);
-  put(33, __fdiv_rn(F64i(n_c * cM * cN - n_tiles), F64i(n_tiles)));
-  put(34, __fdiv_rn(F64i(n_m), F64i(cM)));
-  put(35, __fdiv_rn(F64i(n_n), F64i(cN)));
-  put(36, F32i(cM > n_m || cN > n_n));
-
-  // ---- memory behaviour -----------------------------------------------------------------------
+  // ---- memory behaviour (problem-only and candidate-only columns) ---------------------------
   put(37, t.i_problem);
-  put(38, __fdiv_rn(F64i(2 * area), F64i(static_cast<long long>(TM) * bA + static_cast<long long>(TN) * bA)));
-  const long long restream = n_n * t.bytesA + n_m * t.bytesB;
-  put(39, __fdiv_rn(F64i(restream), F64i(t.bytesA + t.bytesB)));
+  put(38, __fdiv_rn(F64i(2 * r.area), F64i(static_cast<long long>(TM) * bA + static_cast<long long>(TN) * bA)));
   put(40, t.ws_frac_l2);
-  const float fl2 = F64i(static_cast<long long>(h.l2_bytes));
-  put(41, __fdiv_rn(F64i(static_cast<long long>(bA) * TM * t.K), fl2));
-  put(42, __fdiv_rn(F64i(static_cast<long long>(bA) * TN * t.K), fl2));
-  put(43, F64i(restream));
-  put(44, F64i(cdiv_i64(n_n, cN) * t.bytesA + cdiv_i64(n_m, cM) * t.bytesB));
   put(45, t.f_traffic_epi);
 
   // ---- resource pressure columns ------------------------------------------------------------
-  put(46, F64i(B_stage));
-  put(47, F64i(smem_main));
-  put(48, F64i(B_epi));
-  put(49, F64i(B_smem));
-  put(50, f_smem);
-  put(51, F32i(fits));
-  put(52, __fdiv_rn(F64i(area), F32i(T_block)));
-  put(53, F64i(b_smem));
-  put(54, F64i(b_reg));
-  put(55, F64i(b_res));
-  put(56, __fdiv_rn(F64i(b_eff * T_block), F64i(h.max_threads_per_sm)));
+  put(46, F64i(r.B_stage));
+  put(47, F64i(r.smem_main));
+  put(48, F64i(r.B_epi));
+  put(49, F64i(r.B_smem));
+  put(50, r.f_smem);
+  put(51, F32i(r.fits));
+  put(52, __fdiv_rn(F64i(r.area), F32i(r.T_block)));
+  put(53, F64i(r.b_smem));
+  put(54, F64i(r.b_reg));
+  put(55, F64i(r.b_res));
+  put(56, __fdiv_rn(F64i(r.b_eff * r.T_block), F64i(h.max_threads_per_sm)));
 
-  // ---- pipeline balance -----------------------------------------------------------------------
-  const float t_prod = __fdiv_rn(F64i(static_cast<long long>(h.num_sms) * B_stage),
+  // ---- pipeline balance (candidate-only columns) ----------------------------------------------
+  const float t_prod = __fdiv_rn(F64i(static_cast<long long>(h.num_sms) * r.B_stage),
                                  F64i(static_cast<long long>(h.tma_bytes_per_us)));
-  const float t_cons = __fdiv_rn(F64i(2 * area * TK), F64i(n_cons * static_cast<long long>(t.tc_rate)));
+  const float t_cons = __fdiv_rn(F64i(2 * r.area * TK), F64i(r.n_cons * static_cast<long long>(t.tc_rate)));
   put(57, t_prod);
   put(58, t_cons);
   put(59, __fdiv_rn(t_cons, t_prod));
-  put(60, __fdiv_rn(F64i(min(static_cast<long long>(S), n_k)), F32i(S)));
-  put(61, __fdiv_rn(F64i(n_k), F32i(S)));
-  put(62, __fmul_rn(F32i(S), f_smem));
+  put(62, __fmul_rn(F32i(S), r.f_smem));
   put(63, 0.0f);
 }
 

@@ -1,7 +1,7 @@
 // Tensor-core path of the fused select kernel for the feed-forward ranker (Model B) of shape
 // 64 -> 256 -> 256 -> 1: bf16 operands, fp32 accumulation in tensor memory.
 //
-// One CTA (256 threads) ranks one problem against up to kMlpRows candidates, 128 at a time:
+// One CTA (512 threads) ranks one problem against up to kMlpRows candidates, 128 at a time:
 //   F    the 128 feature rows are written straight into shared memory as the bf16 A operand
 //        (candidate-only columns come standardised from a per-call table, problem-only columns
 //        are constant per CTA, the per-pair columns are computed in registers);
@@ -141,7 +141,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   const __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&t);
 }
-__device__ __forceinline__ float round_bf16(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
+// (max(lo, 0), max(hi, 0)) rounded to bf16 and packed, one instruction
+__device__ __forceinline__ uint32_t pack_bf16_relu(float lo, float hi) {
+  uint32_t d;
+  asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
 
 // ------------------------------------------------------------------------------------------
 // candidate-only columns, standardised and rounded to bf16, once per call
@@ -172,7 +177,8 @@ mlp_cand_cols_kernel(ks_gpu_desc desc, const ks_candidate* __restrict__ c, int C
   float x[32];
 #pragma unroll
   for (int q = 0; q < 32; ++q) x[q] = 0.0f;
-  featurize_pair(t, c[i], desc, [&](int col, float v) {
+  const ks_candidate cand = c[i];
+  featurize_pair(t, cand, desc, [&](int col, float v) {
     if (feat_class(col) != 1) return;
     const int k = kpos(col);
     x[k] = fmaf(v, prm.scale[k], prm.shift[k]);
@@ -180,6 +186,9 @@ mlp_cand_cols_kernel(ks_gpu_desc desc, const ks_candidate* __restrict__ c, int C
   uint32_t w[16];
 #pragma unroll
   for (int q = 0; q < 16; ++q) w[q] = pack_bf16(x[2 * q], x[2 * q + 1]);
+  // the last word (positions 30, 31 belong to per-pair columns) carries the candidate's
+  // effective resident-block count for the per-pair wave columns
+  w[15] = static_cast<uint32_t>(resources(t, cand, desc).b_eff) & 0xFFFFu;
   uint4* dst = reinterpret_cast<uint4*>(out + (static_cast<size_t>(combo) * C + i) * kCandRec);
 #pragma unroll
   for (int q = 0; q < 4; ++q) dst[q] = make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
@@ -189,22 +198,23 @@ mlp_cand_cols_kernel(ks_gpu_desc desc, const ks_candidate* __restrict__ c, int C
 // epilogues (H = which half of the 256 columns this warp owns)
 // ------------------------------------------------------------------------------------------
 
-// E1: h1 = bf16(relu(acc + b1)) for 128 columns of this thread's row, written as A-operand planes
-template <int H>
+// E1: h1 = bf16(relu(acc + b1)) for the 64 columns of group G of this thread's row, written as
+// A-operand planes
+template <int G>
 __device__ __forceinline__ void epilogue1(uint32_t tmem_row, uint32_t sA_row, const MlpTcParams& prm) {
 #pragma unroll
-  for (int blk = 0; blk < 4; ++blk) {
+  for (int blk = 0; blk < 2; ++blk) {
     float v[32];
-    tmem_ld32(tmem_row + H * 128 + blk * 32, v);
+    tmem_ld32(tmem_row + G * 64 + blk * 32, v);
 #pragma unroll
     for (int g = 0; g < 4; ++g) {  // eight columns = one plane
       uint32_t w[4];
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        const int j = H * 128 + blk * 32 + g * 8 + 2 * q;
-        w[q] = pack_bf16(fmaxf(v[g * 8 + 2 * q] + prm.b1[j], 0.0f), fmaxf(v[g * 8 + 2 * q + 1] + prm.b1[j + 1], 0.0f));
+        const int j = G * 64 + blk * 32 + g * 8 + 2 * q;
+        w[q] = pack_bf16_relu(v[g * 8 + 2 * q] + prm.b1[j], v[g * 8 + 2 * q + 1] + prm.b1[j + 1]);
       }
-      const int plane = (H * 128 + blk * 32 + g * 8) / 8;
+      const int plane = (G * 64 + blk * 32 + g * 8) / 8;
       asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(sA_row + plane * kPlaneA), "r"(w[0]), "r"(w[1]),
                    "r"(w[2]), "r"(w[3])
                    : "memory");
@@ -212,18 +222,20 @@ __device__ __forceinline__ void epilogue1(uint32_t tmem_row, uint32_t sA_row, co
   }
 }
 
-// E2: partial dot of bf16(relu(acc + b2)) with w3 over 128 columns of this thread's row
-template <int H>
+// E2: partial dot of bf16(relu(acc + b2)) with w3 over the 64 columns of group G
+template <int G>
 __device__ __forceinline__ float epilogue2(uint32_t tmem_row, const MlpTcParams& prm) {
   float s = 0.0f;
 #pragma unroll
-  for (int blk = 0; blk < 4; ++blk) {
+  for (int blk = 0; blk < 2; ++blk) {
     float v[32];
-    tmem_ld32(tmem_row + H * 128 + blk * 32, v);
+    tmem_ld32(tmem_row + G * 64 + blk * 32, v);
 #pragma unroll
-    for (int q = 0; q < 32; ++q) {
-      const int j = H * 128 + blk * 32 + q;
-      s = fmaf(round_bf16(fmaxf(v[q] + prm.b2[j], 0.0f)), prm.w3[j], s);
+    for (int q = 0; q < 16; ++q) {
+      const int j = G * 64 + blk * 32 + 2 * q;
+      const uint32_t pk = pack_bf16_relu(v[2 * q] + prm.b2[j], v[2 * q + 1] + prm.b2[j + 1]);
+      s = fmaf(__uint_as_float(pk << 16), prm.w3[j], s);
+      s = fmaf(__uint_as_float(pk & 0xFFFF0000u), prm.w3[j + 1], s);
     }
   }
   return s;
@@ -245,7 +257,7 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
   __shared__ __align__(8) unsigned long long s_bar[4];  // weights; L2 first group; L2 second group; L1
   __shared__ uint32_t s_tmem;
   __shared__ uint32_t s_pwords[7];   // problem-only columns (positions 50..63) as packed bf16
-  __shared__ float s_halfsum[kTileRows];
+  __shared__ float s_partsum[3][kTileRows];
   __shared__ unsigned long long s_list[KS_MAX_K];
   __shared__ int s_fail;
 
@@ -300,7 +312,7 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = s_tmem;
-  const int quarter = warp & 3, half = warp >> 2;
+  const int quarter = warp & 3, grp = warp >> 2;  // TMEM lane quarter, column group (64 columns)
   const int trow = quarter * 32 + lane;                       // row of the tile this thread reads from TMEM
   const uint32_t tmem_row = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
   const uint32_t sA = sbase + kOffA;
@@ -332,8 +344,7 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
           w[4 * q] = r.x; w[4 * q + 1] = r.y; w[4 * q + 2] = r.z; w[4 * q + 3] = r.w;
         }
         float x[64];
-        featurize_pair(s_pt, cand, desc, [&](int col, float v) {
-          if (feat_class(col) != 2) return;
+        pair_columns<false>(s_pt, cand, desc, static_cast<long long>(w[15] & 0xFFFFu), [&](int col, float v) {
           const int kk = kpos(col);
           x[kk] = fmaf(v, prm.scale[kk], prm.shift[kk]);
         });
@@ -385,8 +396,12 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
     if (!mbar_wait_bounded(bar_c, ph_c)) failed = true;
     ph_c ^= 1;
     tc_fence_after();
-    if (half == 0) epilogue1<0>(tmem_row, sA + trow * 16, prm);
-    else epilogue1<1>(tmem_row, sA + trow * 16, prm);
+    switch (grp) {
+      case 0: epilogue1<0>(tmem_row, sA + trow * 16, prm); break;
+      case 1: epilogue1<1>(tmem_row, sA + trow * 16, prm); break;
+      case 2: epilogue1<2>(tmem_row, sA + trow * 16, prm); break;
+      default: epilogue1<3>(tmem_row, sA + trow * 16, prm); break;
+    }
     fence_async_proxy();
     tc_fence_before();
     __syncthreads();
@@ -423,11 +438,17 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
       tc_fence_after();
       // ---- L1(tile + 1) into the other accumulator, under E2(tile) -----------------------------------
       if (has_next && tid == 0) issue_l1(acc_next);
-      const float part = half == 0 ? epilogue2<0>(acc_row, prm) : epilogue2<1>(acc_row, prm);
-      if (half == 1) s_halfsum[trow] = part;
+      float part;
+      switch (grp) {
+        case 0: part = epilogue2<0>(acc_row, prm); break;
+        case 1: part = epilogue2<1>(acc_row, prm); break;
+        case 2: part = epilogue2<2>(acc_row, prm); break;
+        default: part = epilogue2<3>(acc_row, prm); break;
+      }
+      if (grp > 0) s_partsum[grp - 1][trow] = part;
       __syncthreads();
       if (tid < kTileRows) {
-        const float score = (part + s_halfsum[tid]) + prm.b3;
+        const float score = (((part + s_partsum[0][tid]) + s_partsum[1][tid]) + s_partsum[2][tid]) + prm.b3;
         const unsigned long long key = cur_live ? make_key(score + 0.0f, cur_idx) : 0ull;
 #pragma unroll
         for (int q = 0; q < kTiles; ++q)
@@ -438,8 +459,12 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
         if (!mbar_wait_bounded(bar_c, ph_c)) failed = true;
         ph_c ^= 1;
         tc_fence_after();
-        if (half == 0) epilogue1<0>(acc_next_row, sA + trow * 16, prm);
-        else epilogue1<1>(acc_next_row, sA + trow * 16, prm);
+        switch (grp) {
+          case 0: epilogue1<0>(acc_next_row, sA + trow * 16, prm); break;
+          case 1: epilogue1<1>(acc_next_row, sA + trow * 16, prm); break;
+          case 2: epilogue1<2>(acc_next_row, sA + trow * 16, prm); break;
+          default: epilogue1<3>(acc_next_row, sA + trow * 16, prm); break;
+        }
         fence_async_proxy();
         cur_idx = nxt_idx;
         cur_live = nxt_live;
