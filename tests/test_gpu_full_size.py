@@ -88,3 +88,28 @@ def test_config2_cross_precision(ks, ctx):
     check_properties(w, idx, sc)
     sample = wl.randint(7, 2, np.arange(10), len(w.problems))
     check_sampled(w, idx, sc, [0, len(w.problems) - 1] + sample.tolist(), TOL_GBDT)
+
+
+def test_config4_neural_ranker(ks, ctx):
+    w = wl.make_workload(4)
+    assert w.pairs == 61_440_000
+    model = ctx.model_create_mlp(w.mlp)
+    idx, sc = run_full(ks, ctx, w, model)
+    check_properties(w, idx, sc)
+    check_sampled(w, idx, sc, [0, 517, len(w.problems) - 1], TOL_MLP)
+    idx2, sc2 = run_full(ks, ctx, w, model)
+    assert np.array_equal(idx, idx2) and np.array_equal(sc.view(np.uint32), sc2.view(np.uint32))
+
+
+def test_config3_latency_stream_sample(ks, ctx):
+    """Calls drawn from the 100,000-call stream (first, last and a few in between)."""
+    w = wl.make_workload(3, P=100_000)
+    model = ctx.model_create_gbdt(*w.gbdt)
+    dev = torch.device("cuda", 0)
+    d_c = ks.to_device(w.candidates, dev)
+    C = len(w.candidates)
+    for i in [0, 1, 49_999, 77_777, 99_999]:
+        hi, hs = ctx.select_one(w.problems[i:i + 1], d_c, C, model, w.k)
+        _, _, allsc = oracle.select(w.problems[i:i + 1], w.candidates, w.desc, w.k, gbdt=w.gbdt, want_scores=True)
+        ok, msg = topk_accept(hi.numpy(), hs.numpy(), allsc, np.arange(C, dtype=np.int32), w.k, TOL_GBDT)
+        assert ok, f"call {i}: {msg}"
