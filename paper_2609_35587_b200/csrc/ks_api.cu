@@ -410,7 +410,7 @@ ks_status ks_select(ks_ctx* ctx, const ks_problem* d_p, int P, const ks_candidat
                                     d_seg_index, pairs, k, ctx->ws, d_topk_idx, d_topk_score,
                                     static_cast<cudaStream_t>(stream), &ctx->launches, ctx->d_status,
                                     ctx->profile ? ctx->ev_begin : nullptr,
-                                    ctx->profile ? ctx->ev_end : nullptr);
+                                    ctx->profile ? ctx->ev_end : nullptr, ctx->d_counters);
   ctx->profile_valid = ctx->profile && e == cudaSuccess;
   return e == cudaSuccess ? KS_OK : cuda_fail(ctx, e, "ks_select");
 }
@@ -432,7 +432,7 @@ ks_status ks_select_one(ks_ctx* ctx, ks_problem p, const ks_candidate* d_c, int 
   if (model->kind == 0 && model->gbdt.fast && C > 0) {
     const int nblk = (C + ks::kFastRows - 1) / ks::kFastRows;
     const int S = ks::fast_slices(model->gbdt, nblk);
-    if (S > 1 && nblk <= ks::kMaxSliceBlocks) {
+    if (S > 1) {
       const size_t b_part = align_up(sizeof(unsigned long long) * nblk * k);
       const size_t b_scratch = align_up(ks::fast_scratch_bytes(C));
       const size_t b_scores = align_up(sizeof(float) * static_cast<size_t>(S) * C);
@@ -441,6 +441,7 @@ ks_status ks_select_one(ks_ctx* ctx, ks_problem p, const ks_candidate* d_c, int 
       char* base = static_cast<char*>(ctx->ws);
       ks::FastSlice sl;
       sl.n_slices = S;
+      sl.pairs = C;
       sl.scores = reinterpret_cast<float*>(base + b_part + b_scratch);
       sl.counters = ctx->d_counters;
       sl.out_idx = ctx->d_pinned_idx;
@@ -512,7 +513,7 @@ ks_status ks_select_host(ks_ctx* ctx, const ks_problem* h_p, int P, const ks_can
   if (e == cudaSuccess && seg && pairs > 0) e = cudaMemcpyAsync(d_si, h_seg_index, sizeof(int32_t) * pairs, cudaMemcpyHostToDevice, st);
   if (e == cudaSuccess)
     e = ks::launch_select(ctx->desc, *model, d_p, nullptr, P, d_c, C, d_so, d_si, pairs, k, ctx->ws, d_oi,
-                          d_os, st, &ctx->launches, ctx->d_status);
+                          d_os, st, &ctx->launches, ctx->d_status, nullptr, nullptr, ctx->d_counters);
   if (e == cudaSuccess) e = cudaMemcpyAsync(h_topk_idx, d_oi, sizeof(int32_t) * P * k, cudaMemcpyDeviceToHost, st);
   if (e == cudaSuccess) e = cudaMemcpyAsync(h_topk_score, d_os, sizeof(float) * P * k, cudaMemcpyDeviceToHost, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);

@@ -121,11 +121,12 @@ __device__ __forceinline__ int bin_search(const float* T, float v) {
 // (atomic counter, nobody waits) adds the slices in a fixed order and ranks the block; the
 // last block overall merges the lists and writes the final result.
 struct SliceArgs {
-  int n_slices;            // 1 = batch mode
-  float* scores;           // [n_slices][C] partial scores
-  int* counters;           // [nblk + 1], zero on entry, reset to zero by the last block
-  int32_t* out_idx;        // [k] final result (device-visible, may be mapped host memory)
-  float* out_score;        // [k]
+  int n_slices;            // 1 = every CTA walks the whole ensemble
+  long long pairs;         // rows of the partial-score planes
+  float* scores;           // [n_slices][pairs] partial scores
+  int* counters;           // [P * nblk + 1], zero on entry; every counter is reset by its last user
+  int32_t* out_idx;        // single-problem form only: [k] final result (device-visible, may be
+  float* out_score;        // mapped host memory); null when a merge kernel follows
 };
 
 struct FastView {
@@ -459,11 +460,15 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
       for (int r = 0; r < 4; ++r) {
         const int64_t row = start + static_cast<int64_t>(r & 1) * kFastThreads + word + kWords * (r >> 1);
         if (half == 0 && row < stop)
-          __stcg(sl.scores + static_cast<size_t>(slice) * C + row, score[r] + s_part[r * kWords + word]);
+          __stcg(sl.scores + static_cast<size_t>(slice) * sl.pairs + lo + row, score[r] + s_part[r * kWords + word]);
       }
       __threadfence();
       __syncthreads();
-      if (tid == 0) s_last = atomicAdd(sl.counters + chunk, 1) == S - 1;
+      if (tid == 0) {
+        int* cnt = sl.counters + static_cast<size_t>(prob) * nblk + chunk;
+        s_last = atomicAdd(cnt, 1) == S - 1;
+        if (s_last) *cnt = 0;  // nobody else touches this counter again in this launch
+      }
       __syncthreads();
       if (!s_last) return;
       __threadfence();
@@ -478,7 +483,7 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
         float s;
         if (S > 1) {
           s = fv.base;
-          for (int q = 0; q < S; ++q) s += __ldcg(sl.scores + static_cast<size_t>(q) * C + row);
+          for (int q = 0; q < S; ++q) s += __ldcg(sl.scores + static_cast<size_t>(q) * sl.pairs + lo + row);
         } else {
           s = (fv.base + score[r]) + s_part[r * kWords + word];
         }
@@ -490,8 +495,8 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
     block_topk<5>(keys, k, s_warp, s_list);
   }
   if (tid < k) partial[(static_cast<size_t>(prob) * nblk + chunk) * k + tid] = s_list[tid];
-  if (S > 1) {
-    // the last block to finish merges the per-block lists (one warp) and resets the counters
+  if (S > 1 && sl.out_idx) {
+    // single-problem form: the last block to finish merges the per-block lists (one warp)
     __threadfence();
     __syncthreads();
     if (tid == 0) s_last = atomicAdd(sl.counters + nblk, 1) == nblk - 1;
@@ -515,7 +520,7 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
         prev = best;
       }
     }
-    for (int i = tid; i <= nblk; i += kFastThreads) sl.counters[i] = 0;
+    if (tid == 0) sl.counters[nblk] = 0;
   }
 }
 
@@ -654,32 +659,27 @@ void free_fast_gbdt(GbdtModel& m) {
 // launcher
 // ------------------------------------------------------------------------------------------
 
-// Blocks per problem: full tiles of kFastRows rows, unless that would leave most SMs idle,
-// in which case the rows of a problem are spread over more, shorter blocks.
+// Blocks per problem: full tiles of kFastRows rows. A block's cost does not depend on how many
+// of its slots are live, so an under-filled machine is filled by splitting the trees over
+// several CTAs per block (slices) rather than by shorter blocks.
 void fast_tiling(int P, int64_t per_problem, int* nblk, int* rows_per_cta) {
   int64_t n = (per_problem + kFastRows - 1) / kFastRows;
   if (n < 1) n = 1;
-  const int64_t want = 2 * 148;
-  if (P * n < want && per_problem > 0) {
-    int64_t m = (want + P - 1) / P;
-    const int64_t cap = (per_problem + 127) / 128;  // at least 128 rows per block
-    if (m > cap) m = cap;
-    if (m > n) n = m;
-  }
-  int64_t rows = per_problem > 0 ? (per_problem + n - 1) / n : kFastRows;
-  if (rows > kFastRows) rows = kFastRows;
+  (void)P;
   *nblk = static_cast<int>(n);
-  *rows_per_cta = static_cast<int>(rows);
+  *rows_per_cta = kFastRows;
 }
 
 size_t fast_scratch_bytes(int C) { return 256 + static_cast<size_t>(kCombos) * C * kCandRec; }
 
 // Slice count of the single-problem call: as many tree slices as keep every CTA in the first
 // wave (one CTA per SM).
-int fast_slices(const GbdtModel& g, int nblk) {
-  int s = 148 / (nblk < 1 ? 1 : nblk);
+int fast_slices(const GbdtModel& g, int64_t blocks) {
+  if (blocks < 1) blocks = 1;
+  if (blocks > kMaxSliceBlocks) return 1;
+  int64_t s = 148 / blocks;
   if (s > g.n_chunks) s = g.n_chunks;
-  return s < 1 ? 1 : s;
+  return static_cast<int>(s < 1 ? 1 : s);
 }
 
 template <int L, int NP>
@@ -749,6 +749,7 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
   sl.n_slices = 1;
   if (slice && slice->n_slices > 1) {
     sl.n_slices = slice->n_slices;
+    sl.pairs = slice->pairs;
     sl.scores = slice->scores;
     sl.counters = slice->counters;
     sl.out_idx = slice->out_idx;

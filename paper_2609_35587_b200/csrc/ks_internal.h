@@ -127,10 +127,11 @@ cudaError_t build_fast_gbdt(GbdtModel& m, int n_trees, const int64_t* h_tree_off
 // Slice mode of the quantised tree kernel (single-problem latency call).
 struct FastSlice {
   int n_slices;
-  float* scores;     // [n_slices][C]
-  int* counters;     // [nblk + 1], zero between calls
-  int32_t* out_idx;  // [k], device-visible
-  float* out_score;  // [k]
+  long long pairs;   // rows of one partial-score plane
+  float* scores;     // [n_slices][pairs]
+  int* counters;     // [blocks + 1], zero between calls
+  int32_t* out_idx;  // single-problem form: [k], device-visible; else null (a merge kernel follows)
+  float* out_score;
 };
 
 // Quantised tree path: blocks per problem for `per_problem` rows, and the launch itself.
@@ -143,7 +144,7 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
                                int k, unsigned long long* partial, void* scratch, int* status,
                                cudaStream_t stream, int64_t* launches, cudaEvent_t ev_begin,
                                const FastSlice* slice = nullptr);
-int fast_slices(const GbdtModel& g, int nblk);
+int fast_slices(const GbdtModel& g, int64_t blocks);
 
 // Tensor-core MLP path.
 cudaError_t build_fast_mlp(MlpModel& m, const uint16_t* const* h_w, const float* const* h_b, const float* h_mu,
@@ -178,6 +179,6 @@ cudaError_t launch_select(const ks_gpu_desc& desc, const ks_model& model, const 
                           const int64_t* d_seg_off, const int32_t* d_seg_idx, int64_t pairs, int k,
                           void* d_partial, int32_t* d_topk_idx, float* d_topk_score,
                           cudaStream_t stream, int64_t* launches, int* d_status,
-                          cudaEvent_t ev_begin = nullptr, cudaEvent_t ev_end = nullptr);
+                          cudaEvent_t ev_begin = nullptr, cudaEvent_t ev_end = nullptr, int* d_counters = nullptr);
 
 }  // namespace ks
