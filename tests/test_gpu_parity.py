@@ -369,3 +369,67 @@ def test_invalid_arguments_return_status_codes(ks, ctx):
         ctx.model_create_mlp(m4)
     with pytest.raises(ks.KsError):
         ctx.select_one(problem(0, 5, 5), d_c, 64, model, 5)
+
+
+# ---------------------------------------------------------------------------------------------
+# model shapes that take the other code paths of the fused tree kernel
+# ---------------------------------------------------------------------------------------------
+
+def random_trees(seed, n_trees, max_depth, p_split, thresholds):
+    """Random (unbalanced) trees in breadth-first order; thresholds(feat, rng) draws a split."""
+    rng = np.random.default_rng(seed)
+    nodes, offsets = [], [0]
+    for _ in range(n_trees):
+        tree = [None]            # records (feat or None, value, left)
+        frontier = [(0, 0)]      # (node index, depth)
+        while frontier:
+            i, d = frontier.pop(0)
+            if d < max_depth and (d == 0 or rng.random() < p_split):
+                f = int(rng.integers(0, 63))
+                left = len(tree)
+                tree += [None, None]
+                tree[i] = (f, float(thresholds(f, rng)), left)
+                frontier += [(left, d + 1), (left + 1, d + 1)]
+            else:
+                tree[i] = (None, float(rng.normal(0, 0.1)), 0)
+        nodes += tree
+        offsets.append(len(nodes))
+    nd = np.zeros(len(nodes), wl.NODE_DT)
+    for i, (f, v, left) in enumerate(nodes):
+        nd[i] = (np.float32(v), 0xFFFF if f is None else f, 0, left)
+    return np.array(offsets, np.int64), nd
+
+
+def slot_thresholds(stats_key):
+    thr = wl.feature_stats(stats_key)["thr"]
+    return lambda f, rng: thr[f, rng.integers(0, thr.shape[1])]
+
+
+@pytest.mark.parametrize("case", ["unbalanced_depth8", "deep_generic", "many_shallow_trees", "split_rows",
+                                  "too_many_rows"])
+def test_select_other_model_shapes(ks, ctx, case):
+    prob, cand, _, _ = wl.make_inputs(1, P=5, C=3000)
+    x = oracle.featurize(prob, cand, DESC)
+    if case == "unbalanced_depth8":      # padded to complete trees on the quantised path
+        off, nodes = random_trees(1, 40, 8, 0.7, slot_thresholds("cfg1"))
+    elif case == "deep_generic":         # depth 12 > 10: generic kernel
+        off, nodes = random_trees(2, 12, 12, 0.8, slot_thresholds("cfg1"))
+    elif case == "many_shallow_trees":   # 2,500 trees: fewer top levels fit the constant bank
+        off, nodes = random_trees(3, 2500, 3, 0.9, slot_thresholds("cfg1"))
+    elif case == "split_rows":           # > 127 distinct thresholds on some columns: two rows each
+        lo, hi = x.min(axis=0), x.max(axis=0)
+        def thr(f, rng):
+            if f in (27, 31, 39):
+                return np.float32(lo[f] + (hi[f] - lo[f]) * (rng.integers(1, 300) / 300.0))
+            return slot_thresholds("cfg1")(f, rng)
+        off, nodes = random_trees(4, 120, 7, 0.85, thr)
+    else:                                # continuous thresholds everywhere: too many rows, generic kernel
+        lo, hi = x.min(axis=0), x.max(axis=0)
+        off, nodes = random_trees(5, 150, 7, 0.9, lambda f, rng: np.float32(lo[f] + (hi[f] - lo[f]) * rng.random()))
+    w = wl.Workload(case, DESC, prob, cand, 10, gbdt=(off, nodes, 0.25))
+    model = ctx.model_create_gbdt(off, nodes, 0.25)
+    idx, sc = run_select(ks, ctx, w, model)
+    check_select(w, idx, sc, TOL_GBDT)
+    d_c = dev(ks, cand)
+    hi_, hs_ = ctx.select_one(prob[2:3], d_c, len(cand), model, 10)
+    assert np.array_equal(hi_.numpy(), idx[2])
