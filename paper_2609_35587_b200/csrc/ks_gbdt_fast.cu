@@ -295,7 +295,7 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
   __shared__ __align__(8) unsigned long long s_bar[2];
   __shared__ uint8_t s_row0[64], s_rowcnt[64], s_pbin[64];
   __shared__ float s_pfeat[64];
-  __shared__ int s_fail, s_last;
+  __shared__ int s_fail, s_last, s_done[2];
 
   const int tid = threadIdx.x;
   const int S = sl.n_slices;
@@ -325,6 +325,7 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
     mbar_init(bar0, 1);
     mbar_init(bar1, 1);
     s_fail = 0;
+    s_done[0] = s_done[1] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (tid < 64) {
@@ -439,13 +440,22 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
 #pragma unroll
         for (int r = 0; r < 4; ++r) score[r] += lds_f32(__float_as_uint(a[r]));
       }
-      __syncthreads();  // every thread is done with this buffer
-      if (tid == 0 && ch + 2 < ch_end && !s_fail) {
-        mbar_expect_tx(bar, fv.chunk_bytes);
-        bulk_copy_g2s(buf, reinterpret_cast<const char*>(fv.chunks) + static_cast<size_t>(ch + 2) * fv.chunk_bytes,
-                      fv.chunk_bytes, bar);
+      // Release the buffer without a block-wide barrier: every warp counts itself out, and the
+      // last one to leave refills the buffer (nobody waits; warps may run a chunk ahead).
+      __syncwarp();
+      if ((tid & 31) == 0) {
+        if (atomicAdd(&s_done[b], 1) == kFastThreads / 32 - 1) {
+          s_done[b] = 0;
+          if (ch + 2 < ch_end && !s_fail) {
+            fence_async_proxy();
+            mbar_expect_tx(bar, fv.chunk_bytes);
+            bulk_copy_g2s(buf, reinterpret_cast<const char*>(fv.chunks) + static_cast<size_t>(ch + 2) * fv.chunk_bytes,
+                          fv.chunk_bytes, bar);
+          }
+        }
       }
     }
+    __syncthreads();  // all walks are done: the buffers are free
 
     // ---- phase C ---------------------------------------------------------------------------------
     float* s_part = reinterpret_cast<float*>(smem + kOffBuf0);  // [4][kWords], buffers are idle now
