@@ -49,7 +49,7 @@ constexpr int kMaxRows = 80;           // quantised rows the kernel supports (ti
 constexpr int kThrPerRow = 128;        // 127 thresholds + padding
 constexpr int kRowStride = kFastRows;  // bytes between rows of the tile (one byte per candidate)
 constexpr int kWords = kFastRows / 4;  // words per row = lane slots
-constexpr int kSpinLimit = 1 << 22;
+constexpr int kSpinLimit = 1 << 20;  // probes of up to ~2 us each: a wait gives up after about two seconds
 constexpr int kCandRec = 64;           // bytes per (combination, candidate) record of quantised rows
 constexpr int kCombos = 16;            // dtype_ab x dtype_d
 
@@ -72,9 +72,9 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
-      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}\n"
       : "=r"(ok)
-      : "r"(bar), "r"(parity)
+      : "r"(bar), "r"(parity), "r"(2000u)  // let the hardware park the thread for up to ~2 us per probe
       : "memory");
   return ok != 0;
 }
