@@ -1,7 +1,7 @@
 // Tensor-core path of the fused select kernel for the feed-forward ranker (Model B) of shape
 // 64 -> 256 -> 256 -> 1: bf16 operands, fp32 accumulation in tensor memory.
 //
-// One CTA (512 threads) ranks one problem against up to kMlpRows candidates, 128 at a time:
+// One CTA (384 threads: eight epilogue warps, four feature-row warps) ranks one problem against up to kMlpRows candidates, 128 at a time:
 //   F    the 128 feature rows are written straight into shared memory as the bf16 A operand
 //        (candidate-only columns come standardised from a per-call table, problem-only columns
 //        are constant per CTA, the per-pair columns are computed in registers);
@@ -198,23 +198,23 @@ mlp_cand_cols_kernel(ks_gpu_desc desc, const ks_candidate* __restrict__ c, int C
 // epilogues (H = which half of the 256 columns this warp owns)
 // ------------------------------------------------------------------------------------------
 
-// E1: h1 = bf16(relu(acc + b1)) for the 64 columns of group G of this thread's row, written as
+// E1: h1 = bf16(relu(acc + b1)) for the 128 columns of half H of this thread's row, written as
 // A-operand planes
-template <int G>
+template <int H>
 __device__ __forceinline__ void epilogue1(uint32_t tmem_row, uint32_t sA_row, const MlpTcParams& prm) {
 #pragma unroll
-  for (int blk = 0; blk < 2; ++blk) {
+  for (int blk = 0; blk < 4; ++blk) {
     float v[32];
-    tmem_ld32(tmem_row + G * 64 + blk * 32, v);
+    tmem_ld32(tmem_row + H * 128 + blk * 32, v);
 #pragma unroll
     for (int g = 0; g < 4; ++g) {  // eight columns = one plane
       uint32_t w[4];
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
-        const int j = G * 64 + blk * 32 + g * 8 + 2 * q;
+        const int j = H * 128 + blk * 32 + g * 8 + 2 * q;
         w[q] = pack_bf16_relu(v[g * 8 + 2 * q] + prm.b1[j], v[g * 8 + 2 * q + 1] + prm.b1[j + 1]);
       }
-      const int plane = (G * 64 + blk * 32 + g * 8) / 8;
+      const int plane = (H * 128 + blk * 32 + g * 8) / 8;
       asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(sA_row + plane * kPlaneA), "r"(w[0]), "r"(w[1]),
                    "r"(w[2]), "r"(w[3])
                    : "memory");
@@ -222,17 +222,17 @@ __device__ __forceinline__ void epilogue1(uint32_t tmem_row, uint32_t sA_row, co
   }
 }
 
-// E2: partial dot of bf16(relu(acc + b2)) with w3 over the 64 columns of group G
-template <int G>
+// E2: partial dot of bf16(relu(acc + b2)) with w3 over the 128 columns of half H
+template <int H>
 __device__ __forceinline__ float epilogue2(uint32_t tmem_row, const MlpTcParams& prm) {
   float s = 0.0f;
 #pragma unroll
-  for (int blk = 0; blk < 2; ++blk) {
+  for (int blk = 0; blk < 4; ++blk) {
     float v[32];
-    tmem_ld32(tmem_row + G * 64 + blk * 32, v);
+    tmem_ld32(tmem_row + H * 128 + blk * 32, v);
 #pragma unroll
     for (int q = 0; q < 16; ++q) {
-      const int j = G * 64 + blk * 32 + 2 * q;
+      const int j = H * 128 + blk * 32 + 2 * q;
       const uint32_t pk = pack_bf16_relu(v[2 * q] + prm.b2[j], v[2 * q + 1] + prm.b2[j + 1]);
       s = fmaf(__uint_as_float(pk << 16), prm.w3[j], s);
       s = fmaf(__uint_as_float(pk & 0xFFFF0000u), prm.w3[j + 1], s);
@@ -240,6 +240,12 @@ __device__ __forceinline__ float epilogue2(uint32_t tmem_row, const MlpTcParams&
   }
   return s;
 }
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// barrier among the epilogue warps only
+__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 // ------------------------------------------------------------------------------------------
 // the kernel
@@ -254,14 +260,17 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
                      const __grid_constant__ MlpTcParams prm) {
   extern __shared__ __align__(1024) unsigned char smem[];
   __shared__ ProblemTerms s_pt;
-  __shared__ __align__(8) unsigned long long s_bar[4];  // weights; L2 first group; L2 second group; L1
+  // weights; L2 first group; L2 done; L1 done; feature rows stored; accumulator 0 / 1 read out
+  __shared__ __align__(8) unsigned long long s_bar[7];
   __shared__ uint32_t s_tmem;
   __shared__ uint32_t s_pwords[7];   // problem-only columns (positions 50..63) as packed bf16
-  __shared__ float s_partsum[3][kTileRows];
+  __shared__ float s_partsum[kTileRows];
+  __shared__ int s_idx[2][kTileRows];  // pool index of every row of the tile (-1: no candidate)
   __shared__ unsigned long long s_list[KS_MAX_K];
   __shared__ int s_fail;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const bool is_epi = tid < 256;  // warps 0..7 read the accumulators; warps 8..11 produce feature rows
   const int prob = blockIdx.x / nblk, chunk = blockIdx.x % nblk;
   int64_t lo, len;
   if (seg_off) {
@@ -273,7 +282,8 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
   }
   const uint32_t sbase = smem_u32(smem);
   const uint32_t bar_w = smem_u32(&s_bar[0]), bar_a = smem_u32(&s_bar[1]), bar_b = smem_u32(&s_bar[2]),
-                 bar_c = smem_u32(&s_bar[3]);
+                 bar_c = smem_u32(&s_bar[3]), bar_x = smem_u32(&s_bar[4]), bar_f0 = smem_u32(&s_bar[5]),
+                 bar_f1 = smem_u32(&s_bar[6]);
 
   if (tid == 0) {
     problem_terms(use_value ? p_value : p[prob], desc, s_pt);
@@ -294,6 +304,9 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
     mbar_init(bar_a, 1);
     mbar_init(bar_b, 1);
     mbar_init(bar_c, 1);
+    mbar_init(bar_x, kTileRows);
+    mbar_init(bar_f0, 256);
+    mbar_init(bar_f1, 256);
     s_fail = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     // both weight matrices, resident for the CTA's lifetime
@@ -312,174 +325,154 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = s_tmem;
-  const int quarter = warp & 3, grp = warp >> 2;  // TMEM lane quarter, column group (64 columns)
-  const int trow = quarter * 32 + lane;                       // row of the tile this thread reads from TMEM
-  const uint32_t tmem_row = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
   const uint32_t sA = sbase + kOffA;
   const int combo = s_pt.dtype_ab * 4 + s_pt.dtype_d;
   bool failed = false;
-
   if (!mbar_wait_bounded(bar_w, 0)) failed = true;
+  // Each role tracks the phase of the barriers it waits on. A parity wait can only tell adjacent
+  // phases apart, so every barrier here is consumed before it can complete again; that is why
+  // the two accumulators have a barrier each.
+  uint32_t ph_a = 0, ph_b = 0, ph_c = 0, ph_x = 0, ph_f[2] = {0, 0};
 
-  // Software pipeline over the tiles of a pass (two TMEM accumulators, one A buffer):
-  //   L2(t) is issued in two groups: K-steps 0-3 (they read the planes the feature tile
-  //   occupied) and K-steps 4-15. Once the first group is done, the feature rows of tile t+1
-  //   are written into those planes while the second group still runs. When L2(t) is complete,
-  //   L1(t+1) goes to the other accumulator and runs under the second epilogue of tile t; the
-  //   first epilogue of tile t+1 then rewrites the whole A buffer with its hidden layer.
-  auto feature_rows = [&](int64_t tile0, int& idx_out, bool& live_out) {
-    live_out = tid < kTileRows && tile0 + tid < len;
-    idx_out = 0;
-    if (tid < kTileRows) {
-      uint32_t w[32];
-#pragma unroll
-      for (int q = 0; q < 32; ++q) w[q] = 0u;
-      if (live_out) {
-        idx_out = seg_off ? seg_idx[lo + tile0 + tid] : static_cast<int>(tile0 + tid);
-        const ks_candidate cand = c[idx_out];
-        const uint4* rec = reinterpret_cast<const uint4*>(cand_cols + (static_cast<size_t>(combo) * C + idx_out) * kCandRec);
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const uint4 r = __ldg(rec + q);
-          w[4 * q] = r.x; w[4 * q + 1] = r.y; w[4 * q + 2] = r.z; w[4 * q + 3] = r.w;
-        }
-        float x[64];
-        pair_columns<false>(s_pt, cand, desc, static_cast<long long>(w[15] & 0xFFFFu), [&](int col, float v) {
-          const int kk = kpos(col);
-          x[kk] = fmaf(v, prm.scale[kk], prm.shift[kk]);
-        });
-        // positions 0..28 came from the table; 29..49 are the per-pair columns
-        w[14] = (w[14] & 0xFFFFu) | (pack_bf16(0.0f, x[29]) & 0xFFFF0000u);
-#pragma unroll
-        for (int q = 15; q < 25; ++q) w[q] = pack_bf16(x[2 * q], x[2 * q + 1]);
-#pragma unroll
-        for (int q = 0; q < 7; ++q) w[25 + q] = s_pwords[q];
-      }
-      const uint32_t dst = sA + tid * 16;
-#pragma unroll
-      for (int pl = 0; pl < 8; ++pl)
-        asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + pl * kPlaneA), "r"(w[4 * pl]),
-                     "r"(w[4 * pl + 1]), "r"(w[4 * pl + 2]), "r"(w[4 * pl + 3])
-                     : "memory");
-    }
-    fence_async_proxy();
-  };
-  auto issue_l1 = [&](uint32_t acc) {
-#pragma unroll
-    for (int ks16 = 0; ks16 < 4; ++ks16)
-      umma(acc, make_desc(sA + ks16 * 2 * kPlaneA, kPlaneA, 128),
-           make_desc(sbase + kOffW1 + ks16 * 2 * kPlaneB, kPlaneB, 128), ks16 > 0);
-    umma_commit(bar_c);
-  };
-  uint32_t ph_a = 0, ph_b = 0, ph_c = 0;
-
-  for (int64_t start = static_cast<int64_t>(chunk) * kMlpRows; start < len && !failed;
-       start += static_cast<int64_t>(nblk) * kMlpRows) {
+  // Roles inside a pass (tile t uses accumulator t & 1):
+  //   producers   compute row(t) in registers at any time; once L2(t-1)'s first group has
+  //               released planes 0..7 they store it there; thread 256 then issues L1(t) as soon
+  //               as all rows are stored and accumulator t & 1 has been read out (E2(t-2));
+  //   epilogue    wait L1(t) -> E1(t) -> issue L2(t) in two groups -> wait L2(t) -> E2(t) -> key.
+  for (int64_t start = static_cast<int64_t>(chunk) * kMlpRows; start < len; start += static_cast<int64_t>(nblk) * kMlpRows) {
+    const int64_t rows_left = len - start;
+    const int n_tiles = static_cast<int>(rows_left >= kMlpRows ? kTiles : (rows_left + kTileRows - 1) / kTileRows);
     unsigned long long keys[kTiles + 1];
 #pragma unroll
     for (int q = 0; q <= kTiles; ++q) keys[q] = 0ull;
     if (tid < k) keys[kTiles] = s_list[tid];
-    const int64_t rows_left = len - start;
-    const int n_tiles = static_cast<int>(rows_left >= kMlpRows ? kTiles : (rows_left + kTileRows - 1) / kTileRows);
-
-    // ---- prologue: tile 0 up to its hidden layer -------------------------------------------------
-    int cur_idx, nxt_idx = 0;
-    bool cur_live, nxt_live = false;
     __syncthreads();  // the previous pass's ranking scratch (A buffer) is no longer read
-    feature_rows(start, cur_idx, cur_live);
-    tc_fence_before();
-    __syncthreads();
-    if (tid == 0) {
-      tc_fence_after();
-      issue_l1(tmem);
-    }
-    if (!mbar_wait_bounded(bar_c, ph_c)) failed = true;
-    ph_c ^= 1;
-    tc_fence_after();
-    switch (grp) {
-      case 0: epilogue1<0>(tmem_row, sA + trow * 16, prm); break;
-      case 1: epilogue1<1>(tmem_row, sA + trow * 16, prm); break;
-      case 2: epilogue1<2>(tmem_row, sA + trow * 16, prm); break;
-      default: epilogue1<3>(tmem_row, sA + trow * 16, prm); break;
-    }
-    fence_async_proxy();
-    tc_fence_before();
-    __syncthreads();
 
+    if (!is_epi) {
+      // ---------------------------------- producers -------------------------------------------------
+      const int prow = tid - 256;
+      const uint32_t dst = sA + prow * 16;
 #pragma unroll 1
-    for (int tile = 0; tile < n_tiles; ++tile) {
-      const uint32_t acc = tmem + (tile & 1) * 256, acc_next = tmem + ((tile + 1) & 1) * 256;
-      const uint32_t acc_row = tmem_row + (tile & 1) * 256, acc_next_row = tmem_row + ((tile + 1) & 1) * 256;
-      const bool has_next = tile + 1 < n_tiles;
-      // ---- L2(tile), in two groups -----------------------------------------------------------------
-      if (tid == 0) {
-        tc_fence_after();
+      for (int tile = 0; tile < n_tiles; ++tile) {
+        const int64_t row = start + static_cast<int64_t>(tile) * kTileRows + prow;
+        const bool live = row < len;
+        int idx = -1;
+        uint32_t w[32];
 #pragma unroll
-        for (int ks16 = 0; ks16 < 4; ++ks16)
-          umma(acc, make_desc(sA + ks16 * 2 * kPlaneA, kPlaneA, 128),
-               make_desc(sbase + kOffW2 + ks16 * 2 * kPlaneB, kPlaneB, 128), ks16 > 0);
-        umma_commit(bar_a);
+        for (int q = 0; q < 32; ++q) w[q] = 0u;
+        if (live) {
+          idx = seg_off ? seg_idx[lo + row] : static_cast<int>(row);
+          const ks_candidate cand = c[idx];
+          const uint4* rec = reinterpret_cast<const uint4*>(cand_cols + (static_cast<size_t>(combo) * C + idx) * kCandRec);
 #pragma unroll
-        for (int ks16 = 4; ks16 < 16; ++ks16)
-          umma(acc, make_desc(sA + ks16 * 2 * kPlaneA, kPlaneA, 128),
-               make_desc(sbase + kOffW2 + ks16 * 2 * kPlaneB, kPlaneB, 128), 1u);
-        umma_commit(bar_b);
+          for (int q = 0; q < 4; ++q) {
+            const uint4 r = __ldg(rec + q);
+            w[4 * q] = r.x; w[4 * q + 1] = r.y; w[4 * q + 2] = r.z; w[4 * q + 3] = r.w;
+          }
+          float x[64];
+          pair_columns<false>(s_pt, cand, desc, static_cast<long long>(w[15] & 0xFFFFu), [&](int col, float v) {
+            const int kk = kpos(col);
+            x[kk] = fmaf(v, prm.scale[kk], prm.shift[kk]);
+          });
+          // positions 0..28 came from the table; 29..49 are the per-pair columns
+          w[14] = (w[14] & 0xFFFFu) | (pack_bf16(0.0f, x[29]) & 0xFFFF0000u);
+#pragma unroll
+          for (int q = 15; q < 25; ++q) w[q] = pack_bf16(x[2 * q], x[2 * q + 1]);
+#pragma unroll
+          for (int q = 0; q < 7; ++q) w[25 + q] = s_pwords[q];
+        }
+        if (tile > 0) {  // planes 0..7 are free once the first group of L2(tile - 1) is done
+          if (!mbar_wait_bounded(bar_a, ph_a)) failed = true;
+          ph_a ^= 1;
+        }
+#pragma unroll
+        for (int pl = 0; pl < 8; ++pl)
+          asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + pl * kPlaneA), "r"(w[4 * pl]),
+                       "r"(w[4 * pl + 1]), "r"(w[4 * pl + 2]), "r"(w[4 * pl + 3])
+                       : "memory");
+        s_idx[tile & 1][prow] = idx;
+        fence_async_proxy();
+        mbar_arrive(bar_x);
+        if (prow == 0) {
+          if (!mbar_wait_bounded(bar_x, ph_x)) failed = true;  // every row of the tile is stored
+          ph_x ^= 1;
+          if (tile >= 2) {                                     // accumulator tile & 1 was read out by E2(tile - 2)
+            if (!mbar_wait_bounded((tile & 1) ? bar_f1 : bar_f0, ph_f[tile & 1])) failed = true;
+            ph_f[tile & 1] ^= 1;
+          }
+          tc_fence_after();
+#pragma unroll
+          for (int ks16 = 0; ks16 < 4; ++ks16)
+            umma(tmem + (tile & 1) * 256, make_desc(sA + ks16 * 2 * kPlaneA, kPlaneA, 128),
+                 make_desc(sbase + kOffW1 + ks16 * 2 * kPlaneB, kPlaneB, 128), ks16 > 0);
+          umma_commit(bar_c);
+        }
       }
-      // ---- feature rows of the next tile under the second group --------------------------------------
+      // consume what the loop left pending, so that the phase bits stay in step for the next pass
       if (!mbar_wait_bounded(bar_a, ph_a)) failed = true;
       ph_a ^= 1;
-      if (has_next) {
-        feature_rows(start + static_cast<int64_t>(tile + 1) * kTileRows, nxt_idx, nxt_live);
-        tc_fence_before();
-        __syncthreads();
+      if (prow == 0) {
+        for (int a = 0; a < 2 && a < n_tiles; ++a) {  // the last read-out of each accumulator in use
+          if (!mbar_wait_bounded(a ? bar_f1 : bar_f0, ph_f[a])) failed = true;
+          ph_f[a] ^= 1;
+        }
       }
-      if (!mbar_wait_bounded(bar_b, ph_b)) failed = true;
-      ph_b ^= 1;
-      tc_fence_after();
-      // ---- L1(tile + 1) into the other accumulator, under E2(tile) -----------------------------------
-      if (has_next && tid == 0) issue_l1(acc_next);
-      float part;
-      switch (grp) {
-        case 0: part = epilogue2<0>(acc_row, prm); break;
-        case 1: part = epilogue2<1>(acc_row, prm); break;
-        case 2: part = epilogue2<2>(acc_row, prm); break;
-        default: part = epilogue2<3>(acc_row, prm); break;
-      }
-      if (grp > 0) s_partsum[grp - 1][trow] = part;
-      __syncthreads();
-      if (tid < kTileRows) {
-        const float score = (((part + s_partsum[0][tid]) + s_partsum[1][tid]) + s_partsum[2][tid]) + prm.b3;
-        const unsigned long long key = cur_live ? make_key(score + 0.0f, cur_idx) : 0ull;
-#pragma unroll
-        for (int q = 0; q < kTiles; ++q)
-          if (q == tile) keys[q] = key;
-      }
-      // ---- E1(tile + 1): the hidden layer replaces the A buffer -----------------------------------
-      if (has_next) {
-        if (!mbar_wait_bounded(bar_c, ph_c)) failed = true;
+    } else {
+      // ---------------------------------- epilogue warps --------------------------------------------
+      const int quarter = warp & 3, half = warp >> 2;
+      const int trow = quarter * 32 + lane;
+      const uint32_t tmem_row = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
+#pragma unroll 1
+      for (int tile = 0; tile < n_tiles; ++tile) {
+        const uint32_t acc = tmem + (tile & 1) * 256, acc_row = tmem_row + (tile & 1) * 256;
+        if (!mbar_wait_bounded(bar_c, ph_c)) failed = true;  // L1(tile) is complete
         ph_c ^= 1;
         tc_fence_after();
-        switch (grp) {
-          case 0: epilogue1<0>(acc_next_row, sA + trow * 16, prm); break;
-          case 1: epilogue1<1>(acc_next_row, sA + trow * 16, prm); break;
-          case 2: epilogue1<2>(acc_next_row, sA + trow * 16, prm); break;
-          default: epilogue1<3>(acc_next_row, sA + trow * 16, prm); break;
-        }
+        if (half == 0) epilogue1<0>(acc_row, sA + trow * 16, prm);
+        else epilogue1<1>(acc_row, sA + trow * 16, prm);
         fence_async_proxy();
-        cur_idx = nxt_idx;
-        cur_live = nxt_live;
-      }
-      tc_fence_before();
-      if (__syncthreads_or(failed)) {
-        failed = true;
-        break;
+        tc_fence_before();
+        epi_sync();
+        if (tid == 0) {
+          tc_fence_after();
+#pragma unroll
+          for (int ks16 = 0; ks16 < 4; ++ks16)
+            umma(acc, make_desc(sA + ks16 * 2 * kPlaneA, kPlaneA, 128),
+                 make_desc(sbase + kOffW2 + ks16 * 2 * kPlaneB, kPlaneB, 128), ks16 > 0);
+          umma_commit(bar_a);
+#pragma unroll
+          for (int ks16 = 4; ks16 < 16; ++ks16)
+            umma(acc, make_desc(sA + ks16 * 2 * kPlaneA, kPlaneA, 128),
+                 make_desc(sbase + kOffW2 + ks16 * 2 * kPlaneB, kPlaneB, 128), 1u);
+          umma_commit(bar_b);
+        }
+        if (!mbar_wait_bounded(bar_b, ph_b)) failed = true;  // L2(tile) is complete
+        ph_b ^= 1;
+        tc_fence_after();
+        const float part = half == 0 ? epilogue2<0>(acc_row, prm) : epilogue2<1>(acc_row, prm);
+        tc_fence_before();
+        mbar_arrive((tile & 1) ? bar_f1 : bar_f0);
+        if (half == 1) s_partsum[trow] = part;
+        epi_sync();
+        if (half == 0) {
+          const int idx = s_idx[tile & 1][trow];
+          const float score = (part + s_partsum[trow]) + prm.b3;
+          const unsigned long long key = idx >= 0 ? make_key(score + 0.0f, idx) : 0ull;
+#pragma unroll
+          for (int q = 0; q < kTiles; ++q)
+            if (q == tile) keys[q] = key;
+        }
+        epi_sync();  // s_partsum is free for the next tile
       }
     }
     // rank this pass's keys (the A buffer is idle: use it as scratch)
     __syncthreads();
     block_topk<kTiles + 1>(keys, k, reinterpret_cast<unsigned long long*>(smem + kOffA), s_list);
   }
-  if (failed && tid == 0 && status) atomicExch(status, KS_ERR_TIMEOUT);
+  if (__syncthreads_or(failed)) {
+    if (tid == 0 && status) atomicExch(status, KS_ERR_TIMEOUT);
+    failed = true;
+  }
   if (tid < k) partial[(static_cast<size_t>(prob) * nblk + chunk) * k + tid] = failed ? 0ull : s_list[tid];
   tc_fence_before();
   __syncthreads();
