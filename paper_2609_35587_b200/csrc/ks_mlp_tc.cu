@@ -198,12 +198,12 @@ mlp_cand_cols_kernel(ks_gpu_desc desc, const ks_candidate* __restrict__ c, int C
 // epilogues (H = which half of the 256 columns this warp owns)
 // ------------------------------------------------------------------------------------------
 
-// E1: h1 = bf16(relu(acc + b1)) for the 128 columns of half H of this thread's row, written as
+// E1: h1 = bf16(relu(acc + b1)) for the 256 columns of this thread's row (H = 0), written as
 // A-operand planes
 template <int H>
 __device__ __forceinline__ void epilogue1(uint32_t tmem_row, uint32_t sA_row, const MlpTcParams& prm) {
 #pragma unroll
-  for (int blk = 0; blk < 4; ++blk) {
+  for (int blk = 0; blk < 8; ++blk) {
     float v[32];
     tmem_ld32(tmem_row + H * 128 + blk * 32, v);
 #pragma unroll
@@ -222,12 +222,12 @@ __device__ __forceinline__ void epilogue1(uint32_t tmem_row, uint32_t sA_row, co
   }
 }
 
-// E2: partial dot of bf16(relu(acc + b2)) with w3 over the 128 columns of half H
+// E2: dot of bf16(relu(acc + b2)) with w3 over the 256 columns of this thread's row (H = 0)
 template <int H>
 __device__ __forceinline__ float epilogue2(uint32_t tmem_row, const MlpTcParams& prm) {
   float s = 0.0f;
 #pragma unroll
-  for (int blk = 0; blk < 4; ++blk) {
+  for (int blk = 0; blk < 8; ++blk) {
     float v[32];
     tmem_ld32(tmem_row + H * 128 + blk * 32, v);
 #pragma unroll
@@ -244,8 +244,8 @@ __device__ __forceinline__ float epilogue2(uint32_t tmem_row, const MlpTcParams&
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
-// barrier among the epilogue warps only
-__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+// barrier among the four warps of the first-epilogue group
+__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 // ------------------------------------------------------------------------------------------
 // the kernel
@@ -264,8 +264,7 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
   __shared__ __align__(8) unsigned long long s_bar[7];
   __shared__ uint32_t s_tmem;
   __shared__ uint32_t s_pwords[7];   // problem-only columns (positions 50..63) as packed bf16
-  __shared__ float s_partsum[kTileRows];
-  __shared__ int s_idx[2][kTileRows];  // pool index of every row of the tile (-1: no candidate)
+  __shared__ int s_idx[3][kTileRows];  // pool index of every row of the tile (-1: no candidate)
   __shared__ unsigned long long s_list[KS_MAX_K];
   __shared__ int s_fail;
 
@@ -305,8 +304,8 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
     mbar_init(bar_b, 1);
     mbar_init(bar_c, 1);
     mbar_init(bar_x, kTileRows);
-    mbar_init(bar_f0, 256);
-    mbar_init(bar_f1, 256);
+    mbar_init(bar_f0, kTileRows);
+    mbar_init(bar_f1, kTileRows);
     s_fail = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     // both weight matrices, resident for the CTA's lifetime
@@ -338,7 +337,8 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
   //   producers   compute row(t) in registers at any time; once L2(t-1)'s first group has
   //               released planes 0..7 they store it there; thread 256 then issues L1(t) as soon
   //               as all rows are stored and accumulator t & 1 has been read out (E2(t-2));
-  //   epilogue    wait L1(t) -> E1(t) -> issue L2(t) in two groups -> wait L2(t) -> E2(t) -> key.
+  //   warps 0..3  wait L2(t-1) and L1(t) -> E1(t) -> issue L2(t) in two groups;
+  //   warps 4..7  wait L2(t) -> E2(t) -> key, so E2(t) runs beside E1(t+1) and L2(t+1).
   for (int64_t start = static_cast<int64_t>(chunk) * kMlpRows; start < len; start += static_cast<int64_t>(nblk) * kMlpRows) {
     const int64_t rows_left = len - start;
     const int n_tiles = static_cast<int>(rows_left >= kMlpRows ? kTiles : (rows_left + kTileRows - 1) / kTileRows);
@@ -390,7 +390,7 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
           asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + pl * kPlaneA), "r"(w[4 * pl]),
                        "r"(w[4 * pl + 1]), "r"(w[4 * pl + 2]), "r"(w[4 * pl + 3])
                        : "memory");
-        s_idx[tile & 1][prow] = idx;
+        s_idx[tile % 3][prow] = idx;
         fence_async_proxy();
         mbar_arrive(bar_x);
         if (prow == 0) {
@@ -419,50 +419,58 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
       }
     } else {
       // ---------------------------------- epilogue warps --------------------------------------------
-      const int quarter = warp & 3, half = warp >> 2;
+      // warps 0..3: first epilogue + L2 issue; warps 4..7: second epilogue + ranking keys. Thread
+      // (quarter, lane) of either group owns row quarter * 32 + lane and all 256 columns.
+      const int quarter = warp & 3, group = warp >> 2;
       const int trow = quarter * 32 + lane;
       const uint32_t tmem_row = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
+      if (group == 0) {
 #pragma unroll 1
-      for (int tile = 0; tile < n_tiles; ++tile) {
-        const uint32_t acc = tmem + (tile & 1) * 256, acc_row = tmem_row + (tile & 1) * 256;
-        if (!mbar_wait_bounded(bar_c, ph_c)) failed = true;  // L1(tile) is complete
-        ph_c ^= 1;
-        tc_fence_after();
-        if (half == 0) epilogue1<0>(acc_row, sA + trow * 16, prm);
-        else epilogue1<1>(acc_row, sA + trow * 16, prm);
-        fence_async_proxy();
-        tc_fence_before();
-        epi_sync();
-        if (tid == 0) {
+        for (int tile = 0; tile < n_tiles; ++tile) {
+          const uint32_t acc = tmem + (tile & 1) * 256, acc_row = tmem_row + (tile & 1) * 256;
+          if (tile > 0) {  // the A buffer is free once L2(tile - 1) is complete
+            if (!mbar_wait_bounded(bar_b, ph_b)) failed = true;
+            ph_b ^= 1;
+          }
+          if (!mbar_wait_bounded(bar_c, ph_c)) failed = true;  // L1(tile) is complete
+          ph_c ^= 1;
           tc_fence_after();
+          epilogue1<0>(acc_row, sA + trow * 16, prm);
+          fence_async_proxy();
+          tc_fence_before();
+          epi_sync();
+          if (tid == 0) {
+            tc_fence_after();
 #pragma unroll
-          for (int ks16 = 0; ks16 < 4; ++ks16)
-            umma(acc, make_desc(sA + ks16 * 2 * kPlaneA, kPlaneA, 128),
-                 make_desc(sbase + kOffW2 + ks16 * 2 * kPlaneB, kPlaneB, 128), ks16 > 0);
-          umma_commit(bar_a);
+            for (int ks16 = 0; ks16 < 4; ++ks16)
+              umma(acc, make_desc(sA + ks16 * 2 * kPlaneA, kPlaneA, 128),
+                   make_desc(sbase + kOffW2 + ks16 * 2 * kPlaneB, kPlaneB, 128), ks16 > 0);
+            umma_commit(bar_a);
 #pragma unroll
-          for (int ks16 = 4; ks16 < 16; ++ks16)
-            umma(acc, make_desc(sA + ks16 * 2 * kPlaneA, kPlaneA, 128),
-                 make_desc(sbase + kOffW2 + ks16 * 2 * kPlaneB, kPlaneB, 128), 1u);
-          umma_commit(bar_b);
+            for (int ks16 = 4; ks16 < 16; ++ks16)
+              umma(acc, make_desc(sA + ks16 * 2 * kPlaneA, kPlaneA, 128),
+                   make_desc(sbase + kOffW2 + ks16 * 2 * kPlaneB, kPlaneB, 128), 1u);
+            umma_commit(bar_b);
+          }
         }
-        if (!mbar_wait_bounded(bar_b, ph_b)) failed = true;  // L2(tile) is complete
+        if (!mbar_wait_bounded(bar_b, ph_b)) failed = true;  // the last L2: keeps the phase bit in step
         ph_b ^= 1;
-        tc_fence_after();
-        const float part = half == 0 ? epilogue2<0>(acc_row, prm) : epilogue2<1>(acc_row, prm);
-        tc_fence_before();
-        mbar_arrive((tile & 1) ? bar_f1 : bar_f0);
-        if (half == 1) s_partsum[trow] = part;
-        epi_sync();
-        if (half == 0) {
-          const int idx = s_idx[tile & 1][trow];
-          const float score = (part + s_partsum[trow]) + prm.b3;
+      } else {
+#pragma unroll 1
+        for (int tile = 0; tile < n_tiles; ++tile) {
+          const uint32_t acc_row = tmem_row + (tile & 1) * 256;
+          if (!mbar_wait_bounded(bar_b, ph_b)) failed = true;  // L2(tile) is complete
+          ph_b ^= 1;
+          tc_fence_after();
+          const int idx = s_idx[tile % 3][trow];
+          const float score = epilogue2<0>(acc_row, prm) + prm.b3;
+          tc_fence_before();
+          mbar_arrive((tile & 1) ? bar_f1 : bar_f0);
           const unsigned long long key = idx >= 0 ? make_key(score + 0.0f, idx) : 0ull;
 #pragma unroll
           for (int q = 0; q < kTiles; ++q)
             if (q == tile) keys[q] = key;
         }
-        epi_sync();  // s_partsum is free for the next tile
       }
     }
     // rank this pass's keys (the A buffer is idle: use it as scratch)
