@@ -150,7 +150,7 @@ int fast_slices(const GbdtModel& g, int64_t blocks);
 cudaError_t build_fast_mlp(MlpModel& m, const uint16_t* const* h_w, const float* const* h_b, const float* h_mu,
                            const float* h_sigma);
 void free_fast_mlp(MlpModel& m);
-int mlp_tc_blocks_per_problem(int64_t per_problem);
+int mlp_tc_blocks_per_problem(int P, int64_t per_problem);
 size_t mlp_tc_scratch_bytes(int C);
 cudaError_t launch_select_mlp_tc(const ks_gpu_desc& desc, const MlpModel& m, const ks_problem* d_p,
                                  const ks_problem* p_by_value, int P, const ks_candidate* d_c, int C, int nblk,

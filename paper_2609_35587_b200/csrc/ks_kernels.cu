@@ -395,7 +395,7 @@ size_t select_partial_bytes(const ks_model& model, int P, int C, int64_t pairs, 
     return part + (fast_scratch_bytes(C) + 255) / 256 * 256 + planes;
   }
   if (model.kind == 1 && model.mlp.tc) {
-    const int nblk = mlp_tc_blocks_per_problem(per);
+    const int nblk = mlp_tc_blocks_per_problem(P, per);
     const size_t part = (static_cast<size_t>(P) * nblk * k * sizeof(unsigned long long) + 255) / 256 * 256;
     return part + mlp_tc_scratch_bytes(C);
   }
@@ -439,7 +439,7 @@ cudaError_t launch_select(const ks_gpu_desc& desc, const ks_model& model, const 
     return cudaGetLastError();
   }
   if (model.kind == 1 && model.mlp.tc) {
-    const int nblk = mlp_tc_blocks_per_problem(per);
+    const int nblk = mlp_tc_blocks_per_problem(P, per);
     unsigned long long* part = static_cast<unsigned long long*>(d_partial);
     const size_t part_bytes = (static_cast<size_t>(P) * nblk * k * sizeof(unsigned long long) + 255) / 256 * 256;
     cudaError_t e = launch_select_mlp_tc(desc, model.mlp, d_p, p_by_value, P, d_c, C, nblk, d_seg_off, d_seg_idx, k,

@@ -553,9 +553,16 @@ void free_fast_mlp(MlpModel& m) {
   m.h_tc_params = nullptr;
 }
 
-int mlp_tc_blocks_per_problem(int64_t per_problem) {
-  const int64_t n = (per_problem + kMlpRows - 1) / kMlpRows;
-  return static_cast<int>(n < 1 ? 1 : n);
+// CTAs per problem. A CTA's set-up (160 KB of weights, TMEM, problem terms) is worth several
+// passes of kMlpRows candidates, so with enough problems to fill the GPU each CTA takes up to
+// four passes (the kernel strides over its problem's blocks).
+int mlp_tc_blocks_per_problem(int P, int64_t per_problem) {
+  int64_t blocks = (per_problem + kMlpRows - 1) / kMlpRows;
+  if (blocks < 1) blocks = 1;
+  int64_t passes = static_cast<int64_t>(P) * blocks / (4 * 148);
+  if (passes > 4) passes = 4;
+  if (passes < 1) passes = 1;
+  return static_cast<int>((blocks + passes - 1) / passes);
 }
 
 size_t mlp_tc_scratch_bytes(int C) { return 256 + static_cast<size_t>(kCombos) * C * kCandRec; }
