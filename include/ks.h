@@ -135,8 +135,9 @@ ks_status ks_model_create_gbdt(ks_ctx* ctx, int n_trees, const int64_t* h_tree_o
  * x'_j = (x_j - mu_j) / sigma_j for j < 63 with a non-finite x_j replaced by 0 first,
  * x'_63 = 0, rounded to bf16; every hidden layer is h = ReLU(W h_prev + b) with fp32
  * accumulation, rounded to bf16; the last layer (width 1) is s = w . h + b in fp32.
- * h_widths = {64, w_1, ..., w_{L-1}, 1} (n_layers = L weight matrices, 2 <= L <=
- * KS_MLP_MAX_LAYERS; hidden widths multiples of 64, <= KS_MLP_MAX_WIDTH). h_w_bf16[l] is
+ * h_widths = {64, w_1, ..., w_{L-1}, 1} (n_layers = L weight matrices, 1 <= L <=
+ * KS_MLP_MAX_LAYERS; hidden widths multiples of 64, <= KS_MLP_MAX_WIDTH). L = 1 is the linear
+ * scorer w . x' + b of section "Linear Ridge Baseline". h_w_bf16[l] is
  * row-major [out, in] bf16 bit patterns, h_bias[l] is [out] fp32; h_mu / h_sigma are [64]
  * fp32 with sigma != 0. Synchronous. */
 ks_status ks_model_create_mlp(ks_ctx* ctx, int n_layers, const int* h_widths,

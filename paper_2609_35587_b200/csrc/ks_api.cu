@@ -321,7 +321,7 @@ ks_status ks_model_create_mlp(ks_ctx* ctx, int n_layers, const int* h_widths,
   if (!out_model) return KS_ERR_INVALID_ARG;
   *out_model = nullptr;
   if (!ctx || !h_widths || !h_w_bf16 || !h_bias || !h_mu || !h_sigma) return KS_ERR_INVALID_ARG;
-  if (n_layers < 2 || n_layers > KS_MLP_MAX_LAYERS) return KS_ERR_INVALID_ARG;
+  if (n_layers < 1 || n_layers > KS_MLP_MAX_LAYERS) return KS_ERR_INVALID_ARG;
   if (h_widths[0] != KS_F_PAD || h_widths[n_layers] != 1) return KS_ERR_INVALID_ARG;
   int max_width = KS_F_PAD;
   for (int l = 1; l < n_layers; ++l) {

@@ -433,3 +433,22 @@ def test_select_other_model_shapes(ks, ctx, case):
     d_c = dev(ks, cand)
     hi_, hs_ = ctx.select_one(prob[2:3], d_c, len(cand), model, 10)
     assert np.array_equal(hi_.numpy(), idx[2])
+
+
+def test_select_ridge_and_paper_sized_models(ks, ctx):
+    """The linear (ridge) scorer as a one-layer model, and models of the sizes the paper ships:
+    916 trees of depth 7, and the largest MLP preset 64-1024-1024-512-256-1."""
+    st = wl.feature_stats("cfg1")
+    prob, cand, _, _ = wl.make_inputs(1, P=3, C=900)
+    ridge = wl.mlp_xavier(21, [64, 1], st["mu"], st["sigma"])
+    w = wl.Workload("ridge", DESC, prob, cand, 10, mlp=ridge)
+    idx, sc = run_select(ks, ctx, w, ctx.model_create_mlp(ridge))
+    check_select(w, idx, sc, TOL_MLP)
+    big = wl.mlp_xavier(22, [64, 1024, 1024, 512, 256, 1], st["mu"], st["sigma"])
+    w = wl.Workload("mlp_big", DESC, prob[:1], cand[:200], 10, mlp=big)
+    idx, sc = run_select(ks, ctx, w, ctx.model_create_mlp(big))
+    check_select(w, idx, sc, TOL_MLP)
+    off, nodes = wl.gbdt_complete(wl.BASE_SEED + 9, 916, 7, st["thr"], 0.1)
+    w = wl.Workload("gbdt_916x7", DESC, prob, cand, 10, gbdt=(off, nodes, 0.0))
+    idx, sc = run_select(ks, ctx, w, ctx.model_create_gbdt(off, nodes, 0.0))
+    check_select(w, idx, sc, TOL_GBDT)

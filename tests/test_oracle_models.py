@@ -213,3 +213,18 @@ def test_select_is_the_composition_of_its_steps():
     ridx, _ = oracle.topk(s, 2, 10, rows_per_problem=100)
     idx, _ = oracle.select(w4.problems, w4.candidates, DESC, 10, mlp=w4.mlp)
     assert np.array_equal(idx, ridx)
+
+
+def test_one_layer_model_is_the_linear_scorer():
+    """n_layers = 1: s = w . bf16((x - mu) / sigma) + b, against a numpy dot product in fp64."""
+    st = wl.feature_stats("cfg1")
+    prob, cand, _, _ = wl.make_inputs(1, P=2, C=40)
+    x = oracle.featurize(prob, cand, DESC)
+    m = wl.mlp_xavier(21, [64, 1], st["mu"], st["sigma"])
+    s = oracle.score_mlp(x, m)
+    xs = ((x - m["mu"]) / m["sigma"]).astype(np.float32)
+    xs[:, 63] = 0
+    xs = torch.from_numpy(xs).to(torch.bfloat16).to(torch.float64).numpy()
+    wv = bf16_bits_to_f32(m["weights"][0]).astype(np.float64)[0]
+    ref = xs @ wv + float(m["biases"][0][0])
+    np.testing.assert_allclose(s, ref, rtol=1e-6, atol=1e-6)
