@@ -144,6 +144,14 @@ ks_status ks_model_create_mlp(ks_ctx* ctx, int n_layers, const int* h_widths,
                               const uint16_t* const* h_w_bf16, const float* const* h_bias,
                               const float* h_mu, const float* h_sigma, ks_model** out_model);
 
+/* The static sampling score of the paper's data-collection policy as a scorer with no learned
+ * parameters: with n_c = ceil(M / (c_M T_M)) * ceil(N / (c_N T_N)) clusters and
+ * W = ceil(n_c / S_SM) cluster waves, s = n_c / (W S_SM c_M c_N) * S * sqrt(T_M T_N T_K)
+ * (S_SM read as the SM count). Usable with ks_select / ks_select_one / ks_select_host (ranking
+ * by it is the paper's "static top-B" policy); ks_score returns KS_ERR_UNSUPPORTED because the
+ * score is a function of (p, c), not of the feature row. */
+ks_status ks_model_create_static(ks_ctx* ctx, ks_model** out_model);
+
 ks_status ks_model_destroy(ks_model* model);
 
 /* ---- the three calls of the selection path -------------------------------------------- */

@@ -127,10 +127,11 @@ def topk(scores, P, k, rows_per_problem=0, seg_off=None, seg_idx=None):
 
 
 def select(problems, candidates, desc, k, gbdt=None, mlp=None, seg_off=None, seg_idx=None,
-           want_scores=False):
-    """Featurize + score + full sort per problem. gbdt = (tree_offsets, nodes, base_score)."""
-    if (gbdt is None) == (mlp is None):
-        raise ValueError("pass exactly one of gbdt / mlp")
+           want_scores=False, static=False):
+    """Featurize + score + full sort per problem. gbdt = (tree_offsets, nodes, base_score);
+    static=True ranks by the static sampling score instead of a learned model."""
+    if (gbdt is not None) + (mlp is not None) + bool(static) != 1:
+        raise ValueError("pass exactly one of gbdt / mlp / static")
     p = _check(problems, 16, "problems")
     c = _check(candidates, 16, "candidates")
     so = None if seg_off is None else np.ascontiguousarray(seg_off, dtype=np.int64)
@@ -139,7 +140,12 @@ def select(problems, candidates, desc, k, gbdt=None, mlp=None, seg_off=None, seg
     idx = np.empty((P, k), dtype=np.int32)
     sc = np.empty((P, k), dtype=np.float32)
     allsc = np.empty(_pairs(P, len(c), so), dtype=np.float32) if want_scores else None
-    if gbdt is not None:
+    if static:
+        lib().orc_select(_p(p), ctypes.c_int(P), _p(c), ctypes.c_int(len(c)), _p(so), _p(si),
+                         _p(_desc(desc)), ctypes.c_int(2), ctypes.c_int(0), None, None,
+                         ctypes.c_float(0.0), ctypes.c_int(0), None, None, None, None, None,
+                         ctypes.c_int(k), _p(idx), _p(sc), _p(allsc))
+    elif gbdt is not None:
         off = np.ascontiguousarray(gbdt[0], dtype=np.int64)
         nd = _check(gbdt[1], 12, "nodes")
         base = float(gbdt[2]) if len(gbdt) > 2 else 0.0

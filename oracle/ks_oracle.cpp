@@ -195,6 +195,19 @@ void featurize_pair(const OProblem& p, const OCandidate& c, const OGpuDesc& h, f
   x[63] = 0.0f;
 }
 
+// Static sampling score (section on the sampling policy): n_c clusters, W cluster waves over
+// S_SM, s = n_c / (W S_SM c_M c_N) * S * sqrt(T_M T_N T_K); S_SM read as the SM count.
+float static_score(const OProblem& p, const OCandidate& c, const OGpuDesc& h) {
+  const int64_t M = p.m, N = p.n, TM = c.tile_m, TN = c.tile_n, TK = c.tile_k, S = c.stages;
+  const int64_t cM = c.cluster_m, cN = c.cluster_n, SM = h.num_sms;
+  const int64_t n_c = cdiv(M, cM * TM) * cdiv(N, cN * TN);
+  const int64_t W = cdiv(n_c, SM);
+  float s = F(n_c) / F(W * SM * cM * cN);
+  s = s * F(S);
+  s = s * std::sqrt(F(TM * TN * TK));
+  return s;
+}
+
 // Model A: walk one tree from its root; returns the leaf's node index.
 int walk(const ONode* tree, int node, const float* x) {
   const ONode& nd = tree[node];
@@ -359,7 +372,7 @@ void orc_topk(const float* scores, int P, int64_t rows_per_problem, const int64_
 }
 
 // The whole path, one problem at a time: featurize every pair of the problem, score it,
-// sort the segment. model_kind 0 = tree ensemble, 1 = MLP. all_scores (nullable) receives
+// sort the segment. model_kind 0 = tree ensemble, 1 = MLP, 2 = static sampling score. all_scores (nullable) receives
 // the score of every pair, in row order.
 void orc_select(const OProblem* p, int P, const OCandidate* c, int C, const int64_t* seg_off,
                 const int32_t* seg_idx, const OGpuDesc* h, int model_kind, int n_trees,
@@ -380,8 +393,9 @@ void orc_select(const OProblem* p, int P, const OCandidate* c, int C, const int6
       const int32_t j = seg_off ? seg_idx[lo + r] : static_cast<int32_t>(r);
       idx[r] = j;
       featurize_pair(p[i], c[j], *h, x);
-      sc[r] = model_kind == 0 ? score_gbdt_row(x, n_trees, off, nodes, base, nullptr)
-                              : score_mlp_row(x, m);
+      if (model_kind == 2) sc[r] = static_score(p[i], c[j], *h);
+      else sc[r] = model_kind == 0 ? score_gbdt_row(x, n_trees, off, nodes, base, nullptr)
+                                   : score_mlp_row(x, m);
       if (all_scores) all_scores[lo + r] = sc[r];
     }
     topk_segment(sc.data(), idx.data(), n, k, out_idx + static_cast<int64_t>(i) * k,

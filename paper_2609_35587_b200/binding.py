@@ -19,7 +19,7 @@ KS_F, KS_F_PAD, KS_MAX_K, KS_MAX_DEPTH = 63, 64, 32, 15
 KS_OK, KS_ERR_INVALID_ARG, KS_ERR_UNSUPPORTED, KS_ERR_CUDA, KS_ERR_TIMEOUT, KS_ERR_OOM = range(6)
 
 EXPORTS = ("ks_create", "ks_destroy", "ks_last_cuda_error", "ks_model_create_gbdt",
-           "ks_model_create_mlp", "ks_model_destroy", "ks_featurize", "ks_score", "ks_select",
+           "ks_model_create_mlp", "ks_model_create_static", "ks_model_destroy", "ks_featurize", "ks_score", "ks_select",
            "ks_select_one", "ks_select_host", "ks_status_string", "ks_feature_count",
            "ks_feature_name", "ks_launch_count", "ks_profile_enable", "ks_profile_last_ms", "ks_device_status", "ks_select_trees_static")
 
@@ -49,6 +49,7 @@ def _load() -> ctypes.CDLL:
     lib.ks_last_cuda_error.restype = ctypes.c_char_p
     lib.ks_model_create_gbdt.argtypes = [vp, i32, vp, vp, ctypes.c_float, ctypes.POINTER(vp)]
     lib.ks_model_create_mlp.argtypes = [vp, i32, vp, vp, vp, vp, vp, ctypes.POINTER(vp)]
+    lib.ks_model_create_static.argtypes = [vp, ctypes.POINTER(vp)]
     lib.ks_model_destroy.argtypes = [vp]
     lib.ks_featurize.argtypes = [vp, vp, i32, vp, i32, vp, vp, i64, vp, vp]
     lib.ks_score.argtypes = [vp, vp, i64, vp, vp, vp, vp]
@@ -220,6 +221,11 @@ class Context:
                                       ctypes.byref(h))
         self._check(st, "ks_model_create_mlp")
         return Model(self, h, "mlp")
+
+    def model_create_static(self) -> Model:
+        h = ctypes.c_void_p()
+        self._check(_lib.ks_model_create_static(self._h, ctypes.byref(h)), "ks_model_create_static")
+        return Model(self, h, "static")
 
     # ---- the path -------------------------------------------------------------------------
     @staticmethod

@@ -359,6 +359,18 @@ ks_status ks_model_create_mlp(ks_ctx* ctx, int n_layers, const int* h_widths,
   return KS_OK;
 }
 
+ks_status ks_model_create_static(ks_ctx* ctx, ks_model** out_model) {
+  if (!out_model) return KS_ERR_INVALID_ARG;
+  *out_model = nullptr;
+  if (!ctx) return KS_ERR_INVALID_ARG;
+  ks_model* m = new (std::nothrow) ks_model();
+  if (!m) return KS_ERR_OOM;
+  m->ctx = ctx;
+  m->kind = 2;
+  *out_model = m;
+  return KS_OK;
+}
+
 ks_status ks_model_destroy(ks_model* model) {
   free_model(model);
   return KS_OK;
@@ -383,6 +395,7 @@ ks_status ks_score(ks_ctx* ctx, const float* d_features, int64_t rows, const ks_
   if (!ctx || !model || model->ctx != ctx || rows < 0) return KS_ERR_INVALID_ARG;
   if (rows == 0) return KS_OK;
   if (!d_features || !d_scores) return KS_ERR_INVALID_ARG;
+  if (model->kind == 2) return KS_ERR_UNSUPPORTED;  // the static score is a function of (p, c), not of x
   if (model->kind == 1 && d_leaf_idx) return KS_ERR_INVALID_ARG;
   DeviceGuard g(ctx->device);
   cudaError_t e =

@@ -162,6 +162,17 @@ __device__ __forceinline__ void pair_columns(const ProblemTerms& t, const ks_can
   put(61, fdiv<kExact>(F64i(n_k), F32i(S)));
 }
 
+// Static sampling score (the paper's sampling policy): n_c clusters, W = ceil(n_c / S_SM)
+// cluster waves, s = n_c / (W S_SM c_M c_N) * S * sqrt(T_M T_N T_K), each step rounded to fp32.
+__device__ __forceinline__ float static_score(const ProblemTerms& t, const ks_candidate& c, const ks_gpu_desc& h) {
+  const long long TM = c.tile_m, TN = c.tile_n, TK = c.tile_k, cM = c.cluster_m, cN = c.cluster_n;
+  const long long n_c = cdiv_fit(t.M, cM * TM) * cdiv_fit(t.N, cN * TN);
+  const long long W = cdiv_fit(n_c, h.num_sms);
+  float s = __fdiv_rn(F64i(n_c), F64i(W * h.num_sms * cM * cN));
+  s = __fmul_rn(s, F32i(c.stages));
+  return __fmul_rn(s, __fsqrt_rn(F64i(TM * TN * TK)));
+}
+
 // Writes the 64 columns of one pair through `put(column, value)`.
 template <typename Put>
 __device__ __forceinline__ void featurize_pair(const ProblemTerms& t, const ks_candidate& c,

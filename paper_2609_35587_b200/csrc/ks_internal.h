@@ -103,7 +103,7 @@ struct ks_ctx {
 
 struct ks_model {
   ks_ctx* ctx = nullptr;
-  int kind = 0;  // 0 tree ensemble, 1 MLP
+  int kind = 0;  // 0 tree ensemble, 1 MLP, 2 static sampling score
   ks::GbdtModel gbdt;
   ks::MlpModel mlp;
 };

@@ -206,7 +206,7 @@ score_mlp_kernel(MlpView m, int max_width, const float* __restrict__ feat, int64
 // keep one key per thread per sub-tile, rank the block's keys, write a partial top-k list.
 // ------------------------------------------------------------------------------------------
 
-template <int kModel>  // 0 = tree ensemble, 1 = MLP
+template <int kModel>  // 0 = tree ensemble, 1 = MLP, 2 = static sampling score (no feature tile)
 __global__ void __launch_bounds__(kBlock)
 select_generic_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_problem p_value,
                       int use_value, const ks_candidate* __restrict__ c, PairMap map, int sub_tiles,
@@ -242,16 +242,23 @@ select_generic_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_pro
       const bool live = r < len;
       int idx = 0;
       __syncthreads();  // previous sub-tile's readers are done with s_cols
+      float direct = 0.0f;
       if (live) {
         idx = pool_index(map, lo, r);
         const ks_candidate cand = c[idx];
-        float* col0 = s_cols + threadIdx.x;
-        featurize_pair(s_pt, cand, desc, [&](int col, float v) { col0[col * kBlock] = v; });
+        if (kModel == 2) {
+          direct = static_score(s_pt, cand, desc);
+        } else {
+          float* col0 = s_cols + threadIdx.x;
+          featurize_pair(s_pt, cand, desc, [&](int col, float v) { col0[col * kBlock] = v; });
+        }
       } else if (kModel == 1) {
         for (int col = 0; col < kRow; ++col) s_cols[col * kBlock + threadIdx.x] = 0.0f;
       }
       float score;
-      if (kModel == 0) {
+      if (kModel == 2) {
+        score = direct;
+      } else if (kModel == 0) {
         score = live ? walk_ensemble(nodes, roots, n_trees, base, s_cols + threadIdx.x, nullptr) : 0.0f;
       } else {
         __syncthreads();
@@ -460,7 +467,10 @@ cudaError_t launch_select(const ks_gpu_desc& desc, const ks_model& model, const 
   if (p_by_value) pv = *p_by_value;
   cudaError_t e;
   if (ev_begin) cudaEventRecord(ev_begin, stream);
-  if (model.kind == 0) {
+  if (model.kind == 2) {
+    select_generic_kernel<2><<<grid, kBlock, 0, stream>>>(desc, d_p, pv, p_by_value != nullptr, d_c, map, st, nullptr,
+                                                          nullptr, 0, 0.0f, MlpView{}, 0, k, partial);
+  } else if (model.kind == 0) {
     const GbdtModel& g = model.gbdt;
     const size_t smem = sizeof(float) * kRow * kBlock;
     e = cudaFuncSetAttribute(select_generic_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,

@@ -452,3 +452,63 @@ def test_select_ridge_and_paper_sized_models(ks, ctx):
     w = wl.Workload("gbdt_916x7", DESC, prob, cand, 10, gbdt=(off, nodes, 0.0))
     idx, sc = run_select(ks, ctx, w, ctx.model_create_gbdt(off, nodes, 0.0))
     check_select(w, idx, sc, TOL_GBDT)
+
+
+# ---------------------------------------------------------------------------------------------
+# the static sampling score as a scorer (no learned model)
+# ---------------------------------------------------------------------------------------------
+
+def test_select_static_score_bit_exact(ks, ctx):
+    model = ctx.model_create_static()
+    # every score: k >= C returns all of them
+    for C in (1, 31, 32):
+        prob, cand, _, _ = wl.make_inputs(3, P=7, C=C)
+        idx, sc = ctx.select(dev(ks, prob), 7, dev(ks, cand), C, model, 32)
+        torch.cuda.synchronize()
+        idx, sc = idx.cpu().numpy(), sc.cpu().numpy()
+        ridx, rsc = oracle.select(prob, cand, DESC, 32, static=True)
+        assert np.array_equal(idx, ridx)
+        assert np.array_equal(sc[:, :C].view(np.uint32), rsc[:, :C].view(np.uint32))
+        assert np.all(idx[:, C:] == -1) and np.all(np.isneginf(sc[:, C:]))
+    # dense batch over several blocks with a ragged tail; equal scores rank by index
+    prob, cand, _, _ = wl.make_inputs(1, P=5, C=9001)
+    idx, sc = ctx.select(dev(ks, prob), 5, dev(ks, cand), 9001, model, 20)
+    torch.cuda.synchronize()
+    ridx, rsc = oracle.select(prob, cand, DESC, 20, static=True)
+    assert np.array_equal(idx.cpu().numpy(), ridx)
+    assert np.array_equal(sc.cpu().numpy().view(np.uint32), rsc.view(np.uint32))
+    # segments (cross-precision shape), empty segment included
+    prob, cand, so, si = wl.make_inputs(2, P=6, seg=1500)
+    so = so.copy()
+    so[1:] -= so[1]
+    so[0] = 0
+    pairs = int(so[-1])
+    si = si[len(si) - pairs:] if pairs < len(si) else si
+    idx, sc = ctx.select(dev(ks, prob), 6, dev(ks, cand), len(cand), model, 10, dev(ks, so), dev(ks, si), pairs)
+    torch.cuda.synchronize()
+    ridx, rsc = oracle.select(prob, cand, DESC, 10, static=True, seg_off=so, seg_idx=si)
+    assert np.array_equal(idx.cpu().numpy(), ridx)
+    assert np.array_equal(sc.cpu().numpy().view(np.uint32), rsc.view(np.uint32))
+    assert np.all(ridx[0] == -1)
+    # the single-problem and host-buffer forms
+    prob, cand, _, _ = wl.make_inputs(3, P=3, C=5000)
+    d_c = dev(ks, cand)
+    ridx, rsc = oracle.select(prob, cand, DESC, 10, static=True)
+    for i in range(3):
+        hi, hs = ctx.select_one(prob[i:i + 1], d_c, 5000, model, 10)
+        assert np.array_equal(hi.numpy(), ridx[i]) and np.array_equal(hs.numpy(), rsc[i])
+    hi, hs = ctx.select_host(prob, 3, cand, 5000, model, 10)
+    assert np.array_equal(hi.numpy(), ridx) and np.array_equal(hs.numpy(), rsc)
+    # extreme dimensions
+    prob = np.concatenate([problem(1, 1, 1), problem(1 << 19, 1 << 19, 1 << 19), problem(524287, 3, 5)])
+    cand = np.concatenate([candidate(64, 8, 16, 1), candidate(256, 256, 256, 12, 4, 4), candidate(128, 64, 32, 3, 2, 1)])
+    idx, sc = ctx.select(dev(ks, prob), 3, dev(ks, cand), 3, model, 3)
+    torch.cuda.synchronize()
+    ridx, rsc = oracle.select(prob, cand, DESC, 3, static=True)
+    assert np.array_equal(idx.cpu().numpy(), ridx)
+    assert np.array_equal(sc.cpu().numpy().view(np.uint32), rsc.view(np.uint32))
+    # the score is a function of (p, c), not of a feature row
+    x = torch.zeros((4, 64), dtype=torch.float32, device="cuda")
+    with pytest.raises(ks.KsError) as ei:
+        ctx.score(x, model)
+    assert ei.value.status == ks.KS_ERR_UNSUPPORTED
