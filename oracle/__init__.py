@@ -160,3 +160,34 @@ def select(problems, candidates, desc, k, gbdt=None, mlp=None, seg_off=None, seg
                          ctypes.c_float(0.0), ctypes.c_int(L), _p(widths), wp, bp, _p(mu), _p(sigma),
                          ctypes.c_int(k), _p(idx), _p(sc), _p(allsc))
     return (idx, sc, allsc) if want_scores else (idx, sc)
+
+
+CANDIDATE_BYTES = 16
+
+
+def catalogue_size() -> int:
+    lib().orc_catalogue_size.restype = ctypes.c_int64
+    return int(lib().orc_catalogue_size())
+
+
+def enumerate_candidates(first: int, count: int, dtype) -> np.ndarray:
+    """Search-space records with ids first .. first+count-1 (dtype: a 16-byte record dtype)."""
+    out = np.zeros(count, dtype=dtype)
+    assert out.dtype.itemsize == CANDIDATE_BYTES
+    lib().orc_enumerate(ctypes.c_int64(first), ctypes.c_int64(count), _p(out))
+    return out
+
+
+def valid_catalogue(problem, desc, flags: int, candidates=None, count=None, dtype=None):
+    """Stable filter of `candidates` (None: the search space's first `count` ids) by the static
+    validity rules. Returns (kept records, their positions int32)."""
+    p = _check(problem, 16, "problem")
+    c = None if candidates is None else _check(candidates, 16, "candidates")
+    C = len(c) if c is not None else (catalogue_size() if count is None else int(count))
+    dt = c.dtype if c is not None else dtype
+    out_c = np.zeros(C, dtype=dt)
+    out_i = np.empty(C, dtype=np.int32)
+    f = lib().orc_valid_catalogue
+    f.restype = ctypes.c_int64
+    n = int(f(_p(p), _p(c), ctypes.c_int64(C), _p(_desc(desc)), ctypes.c_uint(flags), _p(out_c), _p(out_i)))
+    return out_c[:n].copy(), out_i[:n].copy()

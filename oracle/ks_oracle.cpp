@@ -16,6 +16,11 @@
 // intensity, f_fill*S == min(S, n_K), footprint linear in S ...), closed forms (square GEMM
 // intensity 2s/(3b)), brute-force nested-if evaluation of tiny ensembles, torch CPU linear
 // layers for the MLP, and numpy sorting for the top-k.
+// The search-space enumerator is pinned by the paper's 534,600 and by the knob table's value
+// lists; the validity filter by the paper's between-layout count differences (55 / 55 / 99,
+// exact), its per-layout totals (within 1 %), and a hand-listed T_K = 512 family. The
+// "wasteful candidate" rule (flag bit 1) is parity unpinned: the paper's table of per-shape
+// counts contradicts the rule as printed.
 // Parity unpinned (the paper names the quantity but prints no formula; the readings are this
 // build's own and are listed in the design notes): B_epi, T_block / n_consumer per schedule,
 // the register estimate behind b_reg, Q_epilogue, the cache-fraction, cluster-fit and
@@ -206,6 +211,83 @@ float static_score(const OProblem& p, const OCandidate& c, const OGpuDesc& h) {
   s = s * F(S);
   s = s * std::sqrt(F(TM * TN * TK));
   return s;
+}
+
+// Search space (Table "Configuration knobs"): the Cartesian product of the searched axes for one
+// layout, 4 * 9 * 5 * 11 * 15 * 3 * 3 * 2 = 534,600 combinations. A linear id is read as a
+// mixed-radix number whose digits follow the table's rows, first row slowest; the 15 cluster
+// shapes are the pairs of {1,2,4,8,16} with c_M c_N <= 16, c_M slowest. The instruction shape
+// is the bf16 one: 64 x T_N x 16.
+constexpr int64_t kCatalogue = 4LL * 9 * 5 * 11 * 15 * 3 * 3 * 2;
+
+void enumerate_one(int64_t id, OCandidate* c) {
+  static const int kTM[4] = {64, 128, 192, 256};
+  static const int kTN[9] = {16, 32, 48, 64, 80, 96, 128, 192, 256};
+  static const int kTK[5] = {32, 64, 128, 256, 512};
+  int cl_m[15], cl_n[15], n_cl = 0;
+  for (int a = 1; a <= 16; a *= 2)
+    for (int b = 1; b <= 16; b *= 2)
+      if (a * b <= 16) { cl_m[n_cl] = a; cl_n[n_cl] = b; ++n_cl; }
+  const int tile_sched = static_cast<int>(id % 2); id /= 2;
+  const int epi_sched = static_cast<int>(id % 3); id /= 3;
+  const int kernel_sched = static_cast<int>(id % 3); id /= 3;
+  const int cl = static_cast<int>(id % 15); id /= 15;
+  const int stages = 2 + static_cast<int>(id % 11); id /= 11;
+  const int tk = static_cast<int>(id % 5); id /= 5;
+  const int tn = static_cast<int>(id % 9); id /= 9;
+  const int tm = static_cast<int>(id);
+  std::memset(c, 0, sizeof(*c));
+  c->tile_m = static_cast<uint16_t>(kTM[tm]);
+  c->tile_n = static_cast<uint16_t>(kTN[tn]);
+  c->tile_k = static_cast<uint16_t>(kTK[tk]);
+  c->instr_n = c->tile_n;
+  c->stages = static_cast<uint8_t>(stages);
+  c->cluster_m = static_cast<uint8_t>(cl_m[cl]);
+  c->cluster_n = static_cast<uint8_t>(cl_n[cl]);
+  c->kernel_sched = static_cast<uint8_t>(kernel_sched);  // 0 WS, 1 Pingpong, 2 Cooperative
+  c->epi_sched = static_cast<uint8_t>(epi_sched);        // 0 NoSmem, 1 TMA, 2 TMA-Cooperative
+  c->tile_sched = static_cast<uint8_t>(tile_sched);      // 0 Persistent, 1 Stream-K
+  c->instr_m = 64;
+  c->instr_k = 16;
+}
+
+// Shared-memory footprint of one CTA as the feature map counts it (section "Resource Pressure
+// and Occupancy", same reading as columns 47-49): warp-specialised mainloops may reuse the
+// mainloop buffers for the epilogue, ping-pong and cooperative ones hold both.
+int64_t smem_total(const OProblem& p, const OCandidate& c, const OGpuDesc& h) {
+  static const int64_t kBytes[4] = {2, 2, 1, 4};
+  const int64_t bA = kBytes[p.dtype_ab & 3], bD = kBytes[p.dtype_d & 3];
+  const int64_t TM = c.tile_m, TN = c.tile_n, TK = c.tile_k, S = c.stages;
+  const int ks = c.kernel_sched & 3;
+  const int64_t smem_main = S * TK * (TM * bA + TN * bA);
+  const int64_t E = (ks == 2) ? 128 : 64;
+  const int64_t B_epi =
+      (c.epi_sched == 0) ? 0 : 2 * std::min<int64_t>(TM, E) * std::min<int64_t>(TN, 32) * bD;
+  return ((ks == 0 || ks == 3) ? std::max(smem_main, B_epi) : smem_main + B_epi) + h.smem_reserved;
+}
+
+// Table "Static validity constraints", rule by rule. flags bit 0 adds the two couplings between
+// epilogue and mainloop schedule that CUTLASS's naming implies (TMA-Cooperative epilogue <=>
+// cooperative mainloop; TMA epilogue => non-cooperative mainloop); bit 1 adds the section's
+// "wasteful candidate" rule T_N > 2M or T_N > 2N.
+bool is_valid(const OProblem& p, const OCandidate& c, const OGpuDesc& h, unsigned flags) {
+  const bool coop = c.kernel_sched == 2;
+  const bool a_col_major = p.layout == 2 || p.layout == 3;  // NN, NT
+  const bool b_row_major = p.layout == 1 || p.layout == 3;  // TT, NT
+  if (c.tile_sched == 1 && !coop) return false;             // Stream-K => cooperative mainloop
+  if (coop && c.tile_m % 128 != 0) return false;            // cooperative => T_M = 0 mod 128
+  if (smem_total(p, c, h) > static_cast<int64_t>(h.smem_per_cta_max)) return false;  // capacity
+  if (a_col_major && c.tile_k > 256 * c.cluster_n) return false;  // A column-major: T_K <= 256 C_N
+  if (b_row_major && c.tile_k > 256 * c.cluster_m) return false;  // B row-major: T_K <= 256 C_M
+  if (flags & 1u) {
+    if (c.epi_sched == 2 && !coop) return false;
+    if (c.epi_sched == 1 && coop) return false;
+  }
+  if (flags & 2u) {
+    if (static_cast<int64_t>(c.tile_n) > 2 * static_cast<int64_t>(p.m)) return false;
+    if (static_cast<int64_t>(c.tile_n) > 2 * static_cast<int64_t>(p.n)) return false;
+  }
+  return true;
 }
 
 // Model A: walk one tree from its root; returns the leaf's node index.
@@ -401,6 +483,32 @@ void orc_select(const OProblem* p, int P, const OCandidate* c, int C, const int6
     topk_segment(sc.data(), idx.data(), n, k, out_idx + static_cast<int64_t>(i) * k,
                  out_score + static_cast<int64_t>(i) * k);
   }
+}
+
+
+int64_t orc_catalogue_size() { return kCatalogue; }
+
+// Candidates with ids first .. first+count-1 of the search space.
+void orc_enumerate(int64_t first, int64_t count, OCandidate* out) {
+  for (int64_t i = 0; i < count; ++i) enumerate_one(first + i, out + i);
+}
+
+// Valid catalogue of one problem (its layout and element sizes; M and N only under flag bit 1):
+// walk the candidates in order (c == NULL: the search space's ids 0 .. C-1), keep the valid
+// ones. out_c / out_index (each nullable) receive the kept records and their positions; returns
+// how many were kept.
+int64_t orc_valid_catalogue(const OProblem* p, const OCandidate* c, int64_t C, const OGpuDesc* h,
+                            unsigned flags, OCandidate* out_c, int32_t* out_index) {
+  int64_t n = 0;
+  for (int64_t j = 0; j < C; ++j) {
+    OCandidate cj;
+    if (c) cj = c[j]; else enumerate_one(j, &cj);
+    if (!is_valid(*p, cj, *h, flags)) continue;
+    if (out_c) out_c[n] = cj;
+    if (out_index) out_index[n] = static_cast<int32_t>(j);
+    ++n;
+  }
+  return n;
 }
 
 }  // extern "C"
