@@ -220,6 +220,71 @@ def run_latency_stream(args, rank, local_rank, dev):
     print(json.dumps(line), flush=True)
 
 
+def run_catalogue(args, rank, local_rank, dev):
+    """The steps in front of the path: the four layouts' valid catalogues built from the
+    534,600-id search space (generate each candidate from its id, test the validity rules,
+    pack the survivors in id order). One step = the four layouts; timed with CUDA events."""
+    if rank != 0:
+        return
+    import torch
+    from paper_2609_35587_b200 import binding as ks
+    from paper_2609_35587_b200 import workloads as wl
+    desc = wl.gpu_desc()
+    ctx = ks.Context(desc, local_rank)
+    probs = np.zeros(4, wl.PROBLEM_DT)
+    probs["m"] = probs["n"] = probs["k"] = 4096
+    probs["layout"] = np.arange(4)
+    probs["dtype_ab"] = probs["dtype_d"] = 1
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    def step():
+        return [ctx.valid_catalogue(probs[i:i + 1], ks.KS_VALID_COUPLED, sync=False) for i in range(4)]
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    launches0 = ctx.launch_count()
+    ms = []
+    for _ in range(args.steps):
+        flush.fill_(1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        res = step()
+        e1.record()
+        torch.cuda.synchronize()
+        ms.append(e0.elapsed_time(e1))
+    clocks = sampler.stop()
+    launches = int(ctx.launch_count() - launches0)
+    t = float(np.mean(ms)) * 1e-3
+    tested = 4 * ks.KS_CATALOGUE_SIZE
+    kept = sum(int(r[2].item()) for r in res)
+    out_bytes = kept * 20
+    cpu = None
+    if not args.no_cpu_baseline:
+        import oracle
+        t0 = time.perf_counter()
+        n_ref = sum(len(oracle.valid_catalogue(probs[i:i + 1], desc, 1, dtype=wl.CANDIDATE_DT)[1])
+                    for i in range(4))
+        t_ref = time.perf_counter() - t0
+        assert n_ref == kept, (n_ref, kept)
+        cpu = {"value": tested / t_ref, "unit": "candidates/s", "cores": 1, "kind": "oracle",
+               "sample": f"the same four layouts, {t_ref:.2f} s"}
+    peaks = load_peaks()
+    line = {"metric": "candidates/sec tested (enumerate + validity rules + ordered compaction, 4 layouts)",
+            "value": tested / t, "unit": "candidates/s", "n_gpus": 1, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+            "config": {"workload": "search space of Table Configuration knobs, 534,600 ids x 4 layouts",
+                       "valid": kept, "l2": "256 MiB flush between steps"},
+            "clocks": clocks, "gpu_launches": launches,
+            "roofline": {"bound": "hbm", "achieved": out_bytes / t / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": out_bytes / t / 1e9 / peaks["hbm_gbs"], "traffic": None,
+                         "note": "20 B written per valid candidate, nothing read: twelve launches of a few "
+                                 "microseconds each, launch-latency bound"},
+            "cpu_baseline": cpu, "e2e": None}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -233,6 +298,8 @@ def main():
     ap.add_argument("--problems", type=int, default=None,
                     help="profiling aid: rank only the first N problems of the workload (not a bench line)")
     ap.add_argument("--skip-e2e", action="store_true", help="profiling aid: skip the host-buffer leg")
+    ap.add_argument("--catalogue", action="store_true",
+                    help="measure the search-space enumeration + validity filter instead of a selection workload")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -252,8 +319,11 @@ def main():
     dev = torch.device("cuda", local_rank)
     cfg = args.workload
     spec = wl.CONFIGS[cfg]
-    if world > 1 and cfg != 3:
+    if world > 1 and cfg != 3 and not args.catalogue:
         dist.init_process_group("nccl", device_id=dev)
+    if args.catalogue:
+        run_catalogue(args, rank, local_rank, dev)
+        return
     if cfg == 3:
         run_latency_stream(args, rank, local_rank, dev)
         return

@@ -154,6 +154,59 @@ ks_status ks_model_create_static(ks_ctx* ctx, ks_model** out_model);
 
 ks_status ks_model_destroy(ks_model* model);
 
+/* ---- search space and validity (the steps in front of the path) --------------------------- */
+
+/* Combinations per layout of the searched knobs (Table "Configuration knobs"):
+ * 4 tile_m * 9 tile_n * 5 tile_k * 11 stages * 15 cluster shapes * 3 kernel schedules *
+ * 3 epilogue schedules * 2 tile schedulers. */
+#define KS_CATALOGUE_SIZE 534600
+
+/* ks_valid_catalogue flags. KS_VALID_COUPLED adds the two couplings between epilogue and
+ * mainloop schedule that the schedule names imply but the paper's table does not list
+ * (TMA-Cooperative epilogue <=> cooperative mainloop; TMA epilogue => non-cooperative mainloop).
+ * KS_VALID_WASTEFUL adds the rule of section "Validity Constraints" that drops candidates with
+ * T_N > 2M or T_N > 2N. */
+#define KS_VALID_COUPLED 1u
+#define KS_VALID_WASTEFUL 2u
+
+/* Writes the candidates with linear ids first .. first+count-1 of the search space to
+ * d_out[0..count) (device, 16-byte aligned, caller-owned). The id is a mixed-radix number whose
+ * digits follow the rows of Table "Configuration knobs", first row slowest: tile_m
+ * {64,128,192,256}, tile_n {16,32,48,64,80,96,128,192,256}, tile_k {32,64,128,256,512}, stages
+ * 2..12, cluster shape (the 15 pairs of {1,2,4,8,16} with c_M c_N <= 16, c_M slowest),
+ * kernel_sched {0 WS, 1 Pingpong, 2 Cooperative}, epi_sched {0 NoSmem, 1 TMA, 2 TMA-Cooperative},
+ * tile_sched {0 Persistent, 1 Stream-K}; instruction shape 64 x tile_n x 16. Asynchronous on
+ * `stream`. KS_ERR_INVALID_ARG unless 0 <= first, 0 <= count, first + count <=
+ * KS_CATALOGUE_SIZE. */
+ks_status ks_enumerate(ks_ctx* ctx, int64_t first, int64_t count, ks_candidate* d_out, void* stream);
+
+/* Static validity filter (Table "Static validity constraints") with order-preserving
+ * compaction. The rules: Stream-K => cooperative mainloop; cooperative mainloop => T_M = 0 mod
+ * 128; shared-memory footprint of one CTA (feature column smem_total, which includes the
+ * descriptor's reserve) <= smem_per_cta_max; A column-major => T_K <= 256 C_N; B row-major =>
+ * T_K <= 256 C_M; plus the rules `flags` selects.
+ *   problem       host pointer, one record: its layout and element types decide; m and n are
+ *                 read only under KS_VALID_WASTEFUL
+ *   d_candidates  device, [C] records, 16-byte aligned; NULL = the search space's ids 0..C-1
+ *                 generated on the fly (then C <= KS_CATALOGUE_SIZE)
+ *   d_out         device, capacity C records, 16-byte aligned, or NULL: the valid candidates in
+ *                 input order
+ *   d_out_index   device, capacity C, or NULL: their positions in the input (= ids)
+ *   d_count       device, one int32: how many are valid
+ *   h_count       host, or NULL; when given the call copies the count there and waits for the
+ *                 stream, otherwise it is asynchronous on `stream`
+ * Entries of d_out / d_out_index past the count are left untouched. Uses the context's
+ * workspace (calls on one context must not overlap). */
+ks_status ks_valid_catalogue(ks_ctx* ctx, const ks_problem* problem, unsigned flags,
+                             const ks_candidate* d_candidates, int C, ks_candidate* d_out,
+                             int32_t* d_out_index, int32_t* d_count, int32_t* h_count, void* stream);
+
+/* d_idx[i] <- d_map[d_idx[i]] for 0 <= d_idx[i] < map_len, else -1: turns top-k positions in a
+ * compacted catalogue (ks_select on ks_valid_catalogue's d_out) back into positions of the
+ * unfiltered one (d_map = its d_out_index). In place, asynchronous on `stream`. */
+ks_status ks_remap_indices(ks_ctx* ctx, int32_t* d_idx, int64_t n, const int32_t* d_map, int map_len,
+                           void* stream);
+
 /* ---- the three calls of the selection path -------------------------------------------- */
 
 /* Candidate sets: with d_seg_offsets == NULL every problem is ranked against the whole pool

@@ -16,12 +16,15 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libks.so")
 
 KS_F, KS_F_PAD, KS_MAX_K, KS_MAX_DEPTH = 63, 64, 32, 15
+KS_CATALOGUE_SIZE = 534600
+KS_VALID_COUPLED, KS_VALID_WASTEFUL = 1, 2
 KS_OK, KS_ERR_INVALID_ARG, KS_ERR_UNSUPPORTED, KS_ERR_CUDA, KS_ERR_TIMEOUT, KS_ERR_OOM = range(6)
 
 EXPORTS = ("ks_create", "ks_destroy", "ks_last_cuda_error", "ks_model_create_gbdt",
            "ks_model_create_mlp", "ks_model_create_static", "ks_model_destroy", "ks_featurize", "ks_score", "ks_select",
            "ks_select_one", "ks_select_host", "ks_status_string", "ks_feature_count",
-           "ks_feature_name", "ks_launch_count", "ks_profile_enable", "ks_profile_last_ms", "ks_device_status", "ks_select_trees_static")
+           "ks_feature_name", "ks_launch_count", "ks_profile_enable", "ks_profile_last_ms", "ks_device_status", "ks_select_trees_static",
+           "ks_enumerate", "ks_valid_catalogue", "ks_remap_indices")
 
 
 class KsError(RuntimeError):
@@ -67,6 +70,10 @@ def _load() -> ctypes.CDLL:
     lib.ks_device_status.argtypes = [vp]
     lib.ks_select_trees_static.argtypes = [i32, vp, vp, i32, vp, i32, vp, vp, i32, ctypes.c_float, i32, vp, vp, vp]
     lib.ks_profile_last_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
+    lib.ks_enumerate.argtypes = [vp, i64, i64, vp, vp]
+    lib.ks_valid_catalogue.argtypes = [vp, ctypes.POINTER(_Problem), ctypes.c_uint, vp, i32, vp, vp, vp,
+                                       ctypes.POINTER(ctypes.c_int32), vp]
+    lib.ks_remap_indices.argtypes = [vp, vp, i64, vp, i32, vp]
     for name in EXPORTS:
         fn = getattr(lib, name)
         if fn.restype is ctypes.c_int and name not in ("ks_feature_count",):
@@ -286,3 +293,37 @@ class Context:
                                  _stream())
         self._check(st, "ks_select_host")
         return h_idx, h_score
+
+    # ---- search space and validity ----------------------------------------------------------
+    def enumerate(self, first: int, count: int, out=None):
+        """Candidates with search-space ids first .. first+count-1 as a [count, 16] uint8 tensor."""
+        if out is None:
+            out = torch.empty((max(int(count), 0), 16), dtype=torch.uint8, device=self.device)
+        self._check(_lib.ks_enumerate(self._h, first, count, _dptr(out), _stream()), "ks_enumerate")
+        return out
+
+    def valid_catalogue(self, problem: np.ndarray, flags: int, d_c=None, C=None, want_records=True,
+                        want_index=True, sync=True):
+        """Validity filter + compaction. Returns (records [C,16] u8 or None, index [C] i32 or
+        None, count); count is an int when sync, else a 1-element device tensor, and only the
+        first `count` entries of the outputs are meaningful."""
+        r = np.ascontiguousarray(problem).reshape(-1)[0]
+        p = _Problem(int(r["m"]), int(r["n"]), int(r["k"]), int(r["layout"]), int(r["dtype_ab"]),
+                     int(r["dtype_d"]), int(r["epi_flags"]))
+        C = (KS_CATALOGUE_SIZE if d_c is None else d_c.shape[0]) if C is None else int(C)
+        cap = max(C, 0)
+        out = torch.empty((cap, 16), dtype=torch.uint8, device=self.device) if want_records else None
+        idx = torch.empty(cap, dtype=torch.int32, device=self.device) if want_index else None
+        d_count = torch.zeros(1, dtype=torch.int32, device=self.device)
+        h_count = ctypes.c_int32(-1)
+        st = _lib.ks_valid_catalogue(self._h, ctypes.byref(p), flags, _dptr(d_c), C, _dptr(out), _dptr(idx),
+                                     _dptr(d_count), ctypes.byref(h_count) if sync else None, _stream())
+        self._check(st, "ks_valid_catalogue")
+        return out, idx, (int(h_count.value) if sync else d_count)
+
+    def remap_indices(self, d_idx, d_map, map_len=None):
+        n = d_idx.numel()
+        map_len = d_map.numel() if map_len is None else int(map_len)
+        self._check(_lib.ks_remap_indices(self._h, _dptr(d_idx), n, _dptr(d_map), map_len, _stream()),
+                    "ks_remap_indices")
+        return d_idx

@@ -376,6 +376,49 @@ ks_status ks_model_destroy(ks_model* model) {
   return KS_OK;
 }
 
+ks_status ks_enumerate(ks_ctx* ctx, int64_t first, int64_t count, ks_candidate* d_out, void* stream) {
+  if (!ctx || first < 0 || count < 0 || first > KS_CATALOGUE_SIZE || count > KS_CATALOGUE_SIZE - first)
+    return KS_ERR_INVALID_ARG;
+  if (count == 0) return KS_OK;
+  if (!d_out || (reinterpret_cast<uintptr_t>(d_out) & 15u)) return KS_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  cudaError_t e = ks::launch_enumerate(first, count, d_out, static_cast<cudaStream_t>(stream), &ctx->launches);
+  return e == cudaSuccess ? KS_OK : cuda_fail(ctx, e, "ks_enumerate");
+}
+
+ks_status ks_valid_catalogue(ks_ctx* ctx, const ks_problem* problem, unsigned flags,
+                             const ks_candidate* d_candidates, int C, ks_candidate* d_out,
+                             int32_t* d_out_index, int32_t* d_count, int32_t* h_count, void* stream) {
+  if (!ctx || !problem || !d_count || C < 0) return KS_ERR_INVALID_ARG;
+  if (flags & ~(KS_VALID_COUPLED | KS_VALID_WASTEFUL)) return KS_ERR_INVALID_ARG;
+  if (problem->layout > 3 || problem->dtype_ab > 3 || problem->dtype_d > 3) return KS_ERR_INVALID_ARG;
+  if (!d_candidates && C > KS_CATALOGUE_SIZE) return KS_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(d_candidates) & 15u) || (reinterpret_cast<uintptr_t>(d_out) & 15u))
+    return KS_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  ks_status s = ensure_workspace(ctx, ks::valid_catalogue_scratch_bytes(C));
+  if (s != KS_OK) return s;
+  cudaError_t e = ks::launch_valid_catalogue(ctx->desc, *problem, flags, d_candidates, C, ctx->ws, d_out,
+                                             d_out_index, d_count, st, &ctx->launches);
+  if (e == cudaSuccess && h_count) {
+    e = cudaMemcpyAsync(h_count, d_count, sizeof(int32_t), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  }
+  return e == cudaSuccess ? KS_OK : cuda_fail(ctx, e, "ks_valid_catalogue");
+}
+
+ks_status ks_remap_indices(ks_ctx* ctx, int32_t* d_idx, int64_t n, const int32_t* d_map, int map_len,
+                           void* stream) {
+  if (!ctx || n < 0 || map_len < 0) return KS_ERR_INVALID_ARG;
+  if (n == 0) return KS_OK;
+  if (!d_idx || (map_len > 0 && !d_map)) return KS_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  cudaError_t e = ks::launch_remap_indices(d_idx, n, d_map, map_len, static_cast<cudaStream_t>(stream),
+                                           &ctx->launches);
+  return e == cudaSuccess ? KS_OK : cuda_fail(ctx, e, "ks_remap_indices");
+}
+
 ks_status ks_featurize(ks_ctx* ctx, const ks_problem* d_p, int P, const ks_candidate* d_c, int C,
                        const int64_t* d_seg_offsets, const int32_t* d_seg_index, int64_t pairs,
                        float* d_features, void* stream) {

@@ -88,6 +88,26 @@ __device__ __forceinline__ float fdiv(float a, float b) {
 
 // Candidate-side resource terms (section "Resource Pressure and Occupancy"); they depend on the
 // problem only through its element sizes.
+// Shared-memory footprint of one CTA: mainloop stages, epilogue staging, and their total.
+// The warp-specialised (and the basic) mainloop may reuse the mainloop buffers for the
+// epilogue; ping-pong and cooperative hold both at once.
+struct SmemTerms {
+  long long B_stage, smem_main, B_epi, both, B_smem;
+};
+
+__device__ __forceinline__ SmemTerms smem_terms(int bA, int bD, const ks_candidate& c, const ks_gpu_desc& h) {
+  SmemTerms s;
+  const int TM = c.tile_m, TN = c.tile_n, TK = c.tile_k, S = c.stages;
+  const int ks = c.kernel_sched & 3;
+  s.B_stage = static_cast<long long>(TK) * (TM * bA + TN * bA);
+  s.smem_main = S * s.B_stage;
+  const int E = (ks == 2) ? 128 : 64;
+  s.B_epi = (c.epi_sched == 0) ? 0 : 2ll * min(TM, E) * min(TN, 32) * bD;
+  s.both = s.smem_main + s.B_epi + h.smem_reserved;
+  s.B_smem = (ks == 0 || ks == 3) ? max(s.smem_main, s.B_epi) + h.smem_reserved : s.both;
+  return s;
+}
+
 struct Resources {
   long long B_stage, smem_main, B_epi, B_smem, area, b_smem, b_reg, b_res, b_eff;
   int T_block, n_cons, fits;
@@ -102,13 +122,12 @@ __device__ __forceinline__ Resources resources(const ProblemTerms& t, const ks_c
   // (consumer warpgroups in the mainloop, threads per block): WS, Pingpong, Cooperative, basic
   r.n_cons = (ks == 2) ? 2 : 1;
   r.T_block = (ks == 0) ? 256 : (ks == 3 ? 128 : 384);
-  const int bA = t.bA, bD = t.bD;
-  r.B_stage = static_cast<long long>(TK) * (TM * bA + TN * bA);
-  r.smem_main = S * r.B_stage;
-  const int E = (ks == 2) ? 128 : 64;
-  r.B_epi = (c.epi_sched == 0) ? 0 : 2ll * min(TM, E) * min(TN, 32) * bD;
-  const long long both = r.smem_main + r.B_epi + h.smem_reserved;
-  r.B_smem = (ks == 0 || ks == 3) ? max(r.smem_main, r.B_epi) + h.smem_reserved : both;
+  const SmemTerms sm = smem_terms(t.bA, t.bD, c, h);
+  r.B_stage = sm.B_stage;
+  r.smem_main = sm.smem_main;
+  r.B_epi = sm.B_epi;
+  const long long both = sm.both;
+  r.B_smem = sm.B_smem;
   r.f_smem = __fdiv_rn(F64i(r.B_smem), F64i(h.smem_per_sm));
   r.fits = both <= static_cast<long long>(h.smem_per_cta_max);
   r.area = static_cast<long long>(TM) * TN;

@@ -134,6 +134,17 @@ struct FastSlice {
   float* out_score;
 };
 
+// Search-space enumeration and validity filtering (ks_catalogue.cu).
+cudaError_t launch_enumerate(long long first, long long count, ks_candidate* d_out, cudaStream_t stream,
+                             int64_t* launches);
+size_t valid_catalogue_scratch_bytes(int C);
+cudaError_t launch_valid_catalogue(const ks_gpu_desc& desc, const ks_problem& p, unsigned flags,
+                                   const ks_candidate* d_c, int C, void* d_scratch, ks_candidate* d_out,
+                                   int32_t* d_out_index, int32_t* d_count, cudaStream_t stream,
+                                   int64_t* launches);
+cudaError_t launch_remap_indices(int32_t* d_idx, long long n, const int32_t* d_map, int map_len,
+                                 cudaStream_t stream, int64_t* launches);
+
 // Quantised tree path: blocks per problem for `per_problem` rows, and the launch itself.
 void fast_tiling(int P, int64_t per_problem, int* nblk, int* rows_per_cta);
 size_t fast_scratch_bytes(int C);  // per-call table of candidate-only rows
