@@ -181,6 +181,87 @@ __device__ __forceinline__ void pair_columns(const ProblemTerms& t, const ks_can
   put(61, fdiv<kExact>(F64i(n_k), F32i(S)));
 }
 
+// ---- per-pair columns for consumers that round them to bf16 ------------------------------------
+// Same quantities as pair_columns, evaluated in 32-bit integer and single-precision arithmetic:
+// the integer counts (tiles, waves, clusters) stay exact, the ratios and byte counts carry
+// float rounding (relative error ~1e-7, far below the bf16 rounding that follows). Valid when
+// the tile counts are small enough for that (ok == true); otherwise the caller falls back to
+// pair_columns.
+struct PairFastTerms {
+  float inv_M, inv_N, inv_sms, f_bytesA, f_bytesB, inv_bytes, k_bytes_over_l2;
+};
+
+__device__ inline void pair_fast_terms(const ProblemTerms& t, const ks_gpu_desc& h, PairFastTerms& f) {
+  f.inv_M = __fdividef(1.0f, F64i(t.M));
+  f.inv_N = __fdividef(1.0f, F64i(t.N));
+  f.inv_sms = __fdividef(1.0f, F64i(h.num_sms));
+  f.f_bytesA = F64i(t.bytesA);
+  f.f_bytesB = F64i(t.bytesB);
+  f.inv_bytes = __fdividef(1.0f, F64i(t.bytesA + t.bytesB));
+  f.k_bytes_over_l2 = __fdividef(F64i(static_cast<long long>(t.bA) * t.K), F64i(static_cast<long long>(h.l2_bytes)));
+}
+
+// floor(a / b) for a < 2^24, 0 < b, given rb ~ 1 / b: the float quotient is within one of the
+// answer and one multiply-back settles it
+__device__ __forceinline__ unsigned udiv_small(unsigned a, unsigned b, float rb) {
+  unsigned q = __float2uint_rz(__fmul_rz(__uint2float_rz(a), rb));
+  const int r = static_cast<int>(a - q * b);
+  q += (r >= static_cast<int>(b)) ? 1u : 0u;
+  q -= (r < 0) ? 1u : 0u;
+  return q;
+}
+__device__ __forceinline__ unsigned cdiv_small(unsigned a, unsigned b, float rb) {
+  return udiv_small(a + b - 1u, b, rb);
+}
+
+template <typename Put>
+__device__ __forceinline__ bool pair_columns_bf16(const ProblemTerms& t, const PairFastTerms& f,
+                                                  const ks_candidate& c, const ks_gpu_desc& h, unsigned b_eff,
+                                                  Put put) {
+  const unsigned TM = c.tile_m, TN = c.tile_n, TK = c.tile_k, S = c.stages;
+  const unsigned cM = c.cluster_m, cN = c.cluster_n;
+  const float fTM = __uint2float_rn(TM), fTN = __uint2float_rn(TN);
+  const float rTM = __fdividef(1.0f, fTM), rTN = __fdividef(1.0f, fTN);
+  const float rTK = __fdividef(1.0f, __uint2float_rn(TK)), rS = __fdividef(1.0f, __uint2float_rn(S));
+  const float rcM = __fdividef(1.0f, __uint2float_rn(cM)), rcN = __fdividef(1.0f, __uint2float_rn(cN));
+  const unsigned n_m = cdiv_small(t.M, TM, rTM), n_n = cdiv_small(t.N, TN, rTN), n_k = cdiv_small(t.K, TK, rTK);
+  if (n_m > 2048u || n_n > 2048u) return false;  // keeps every integer below 2^23
+  const unsigned n_tiles = n_m * n_n;
+  const float fn_m = __uint2float_rn(n_m), fn_n = __uint2float_rn(n_n), fn_k = __uint2float_rn(n_k);
+  const float fn_tiles = __uint2float_rn(n_tiles);
+  put(23, fn_m);
+  put(24, fn_n);
+  put(25, fn_k);
+  put(26, fn_tiles);
+  put(27, __uint2float_rn(n_m * TM - t.M) * f.inv_M);
+  put(28, __uint2float_rn(n_n * TN - t.N) * f.inv_N);
+  put(29, fn_tiles * f.inv_sms);
+  const unsigned resident = h.num_sms * b_eff;
+  const unsigned waves = cdiv_small(n_tiles, resident, __fdividef(1.0f, __uint2float_rn(resident)));
+  put(30, __uint2float_rn(waves));
+  const float eta = __fdividef(fn_tiles, __uint2float_rn(waves * resident));
+  put(31, eta);
+  put(32, fmaxf(0.0f, 1.0f - eta));
+  const unsigned cmtm = cM * TM, cntn = cN * TN;
+  const unsigned n_cm = cmtm >= t.M ? 1u : cdiv_small(t.M, cmtm, rcM * rTM);
+  const unsigned n_cn = cntn >= t.N ? 1u : cdiv_small(t.N, cntn, rcN * rTN);
+  const float r_tiles = __fdividef(1.0f, fn_tiles);
+  put(33, __uint2float_rn(n_cm * cM * n_cn * cN - n_tiles) * r_tiles);
+  put(34, fn_m * rcM);
+  put(35, fn_n * rcN);
+  put(36, (cM > n_m || cN > n_n) ? 1.0f : 0.0f);
+  const float restream = fmaf(fn_n, f.f_bytesA, fn_m * f.f_bytesB);
+  put(39, restream * f.inv_bytes);
+  put(41, fTM * f.k_bytes_over_l2);
+  put(42, fTN * f.k_bytes_over_l2);
+  put(43, restream);
+  put(44, fmaf(__uint2float_rn(cdiv_small(n_n, cN, rcN)), f.f_bytesA,
+               __uint2float_rn(cdiv_small(n_m, cM, rcM)) * f.f_bytesB));
+  put(60, __uint2float_rn(min(S, n_k)) * rS);
+  put(61, fn_k * rS);
+  return true;
+}
+
 // Static sampling score (the paper's sampling policy): n_c clusters, W = ceil(n_c / S_SM)
 // cluster waves, s = n_c / (W S_SM c_M c_N) * S * sqrt(T_M T_N T_K), each step rounded to fp32.
 __device__ __forceinline__ float static_score(const ProblemTerms& t, const ks_candidate& c, const ks_gpu_desc& h) {

@@ -19,7 +19,7 @@ struct FastTopParams {
 
 // Constants of the tensor-core MLP path that travel as a kernel parameter (constant bank):
 // folded standardisation per K position, biases, the last layer's weights widened to fp32.
-struct MlpTcParams {
+struct alignas(16) MlpTcParams {
   float scale[64], shift[64];
   float b1[256], b2[256], w3[256];
   float b3;

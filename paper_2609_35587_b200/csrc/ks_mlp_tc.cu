@@ -198,21 +198,79 @@ mlp_cand_cols_kernel(ks_gpu_desc desc, const ks_candidate* __restrict__ c, int C
 // epilogues (H = which half of the 256 columns this warp owns)
 // ------------------------------------------------------------------------------------------
 
-// E1: h1 = bf16(relu(acc + b1)) for the 256 columns of this thread's row (H = 0), written as
-// A-operand planes
+// 32 consecutive fp32 columns of this thread's TMEM lane, without waiting for them
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+}
+// Waits for this thread's outstanding TMEM loads. The registers of the load being waited for
+// pass through as read-write operands, so that no use of them is scheduled above the wait.
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]),
+                 "+r"(r[15]), "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]),
+                 "+r"(r[22]), "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]),
+                 "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+               :
+               : "memory");
+}
+
+// two fp32 lanes per 64-bit register: (lo, hi) + (lo, hi), and a * b + c, each lane rounded as
+// the scalar instruction would
+__device__ __forceinline__ unsigned long long pack2(uint32_t lo, uint32_t hi) {
+  unsigned long long d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
+  return d;
+}
+__device__ __forceinline__ void unpack2(unsigned long long v, float& lo, float& hi) {
+  uint32_t a, b;
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
+  lo = __uint_as_float(a);
+  hi = __uint_as_float(b);
+}
+__device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigned long long b) {
+  unsigned long long d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+  unsigned long long d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ unsigned long long const2(const float* p) {  // two consecutive floats, 8-byte aligned
+  return *reinterpret_cast<const unsigned long long*>(p);
+}
+
+// E1: h1 = bf16(relu(acc + b1)) for the 256 columns of this thread's row, written as A-operand
+// planes. The TMEM load of the next 32 columns is in flight while the current ones are processed.
 template <int H>
 __device__ __forceinline__ void epilogue1(uint32_t tmem_row, uint32_t sA_row, const MlpTcParams& prm) {
+  uint32_t ra[32], rb[32];
+  tmem_ld32_issue(tmem_row + H * 128, ra);
 #pragma unroll
   for (int blk = 0; blk < 8; ++blk) {
-    float v[32];
-    tmem_ld32(tmem_row + H * 128 + blk * 32, v);
+    uint32_t(&cur)[32] = (blk & 1) ? rb : ra;
+    uint32_t(&nxt)[32] = (blk & 1) ? ra : rb;
+    tmem_ld_wait(cur);
+    if (blk < 7) tmem_ld32_issue(tmem_row + H * 128 + (blk + 1) * 32, nxt);
 #pragma unroll
     for (int g = 0; g < 4; ++g) {  // eight columns = one plane
       uint32_t w[4];
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         const int j = H * 128 + blk * 32 + g * 8 + 2 * q;
-        w[q] = pack_bf16_relu(v[g * 8 + 2 * q] + prm.b1[j], v[g * 8 + 2 * q + 1] + prm.b1[j + 1]);
+        float lo, hi;
+        unpack2(add2(pack2(cur[g * 8 + 2 * q], cur[g * 8 + 2 * q + 1]), const2(&prm.b1[j])), lo, hi);
+        w[q] = pack_bf16_relu(lo, hi);
       }
       const int plane = (H * 128 + blk * 32 + g * 8) / 8;
       asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(sA_row + plane * kPlaneA), "r"(w[0]), "r"(w[1]),
@@ -222,23 +280,34 @@ __device__ __forceinline__ void epilogue1(uint32_t tmem_row, uint32_t sA_row, co
   }
 }
 
-// E2: dot of bf16(relu(acc + b2)) with w3 over the 256 columns of this thread's row (H = 0)
+// E2: dot of bf16(relu(acc + b2)) with w3 over the 256 columns of this thread's row; even and
+// odd columns accumulate in the two lanes of one packed register
 template <int H>
 __device__ __forceinline__ float epilogue2(uint32_t tmem_row, const MlpTcParams& prm) {
-  float s = 0.0f;
+  unsigned long long s0 = 0ull, s1 = 0ull;  // (0.0f, 0.0f)
+  uint32_t ra[32], rb[32];
+  tmem_ld32_issue(tmem_row + H * 128, ra);
 #pragma unroll
   for (int blk = 0; blk < 8; ++blk) {
-    float v[32];
-    tmem_ld32(tmem_row + H * 128 + blk * 32, v);
+    uint32_t(&cur)[32] = (blk & 1) ? rb : ra;
+    uint32_t(&nxt)[32] = (blk & 1) ? ra : rb;
+    tmem_ld_wait(cur);
+    if (blk < 7) tmem_ld32_issue(tmem_row + H * 128 + (blk + 1) * 32, nxt);
 #pragma unroll
     for (int q = 0; q < 16; ++q) {
       const int j = H * 128 + blk * 32 + 2 * q;
-      const uint32_t pk = pack_bf16_relu(v[2 * q] + prm.b2[j], v[2 * q + 1] + prm.b2[j + 1]);
-      s = fmaf(__uint_as_float(pk << 16), prm.w3[j], s);
-      s = fmaf(__uint_as_float(pk & 0xFFFF0000u), prm.w3[j + 1], s);
+      float lo, hi;
+      unpack2(add2(pack2(cur[2 * q], cur[2 * q + 1]), const2(&prm.b2[j])), lo, hi);
+      const uint32_t pk = pack_bf16_relu(lo, hi);
+      const unsigned long long h2 = pack2(pk << 16, pk & 0xFFFF0000u);
+      if (q & 1) s1 = fma2(h2, const2(&prm.w3[j]), s1);
+      else s0 = fma2(h2, const2(&prm.w3[j]), s0);
     }
   }
-  return s;
+  float a, b, c, d;
+  unpack2(s0, a, b);
+  unpack2(s1, c, d);
+  return (a + b) + (c + d);
 }
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
@@ -260,6 +329,7 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
                      const __grid_constant__ MlpTcParams prm) {
   extern __shared__ __align__(1024) unsigned char smem[];
   __shared__ ProblemTerms s_pt;
+  __shared__ PairFastTerms s_pf;
   // weights; L2 first group; L2 done; L1 done; feature rows stored; accumulator 0 / 1 read out
   __shared__ __align__(8) unsigned long long s_bar[7];
   __shared__ uint32_t s_tmem;
@@ -286,6 +356,7 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
 
   if (tid == 0) {
     problem_terms(use_value ? p_value : p[prob], desc, s_pt);
+    pair_fast_terms(s_pt, desc, s_pf);
     ks_candidate dummy{};
     dummy.tile_m = dummy.tile_n = dummy.tile_k = 64;
     dummy.stages = dummy.cluster_m = dummy.cluster_n = 1;
@@ -370,10 +441,14 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
             w[4 * q] = r.x; w[4 * q + 1] = r.y; w[4 * q + 2] = r.z; w[4 * q + 3] = r.w;
           }
           float x[64];
-          pair_columns<false>(s_pt, cand, desc, static_cast<long long>(w[15] & 0xFFFFu), [&](int col, float v) {
+          auto put = [&](int col, float v) {
             const int kk = kpos(col);
             x[kk] = fmaf(v, prm.scale[kk], prm.shift[kk]);
-          });
+          };
+          // single-precision evaluation (the values are rounded to bf16 next); the exact
+          // 64-bit form only for tile counts beyond its range
+          if (!pair_columns_bf16(s_pt, s_pf, cand, desc, w[15] & 0xFFFFu, put))
+            pair_columns<false>(s_pt, cand, desc, static_cast<long long>(w[15] & 0xFFFFu), put);
           // positions 0..28 came from the table; 29..49 are the per-pair columns
           w[14] = (w[14] & 0xFFFFu) | (pack_bf16(0.0f, x[29]) & 0xFFFF0000u);
 #pragma unroll
