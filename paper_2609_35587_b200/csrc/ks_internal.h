@@ -116,8 +116,8 @@ constexpr int kFastThreads = 1024;      // threads per block of the quantised tr
 constexpr int kFastR = 2;              // candidates per thread there
 constexpr int kFastRows = kFastThreads * kFastR;
 constexpr int kFastMaxDepth = 10;
-constexpr int kMlpThreads = 384;        // threads per block of the tensor-core MLP kernel
-constexpr int kMlpRows = 2048;          // candidates one block ranks per pass
+constexpr int kMlpThreads = 512;        // threads per block of the tensor-core MLP kernel
+constexpr int kMlpRows = 4096;          // candidates one block ranks per pass
 constexpr int kMaxSliceBlocks = 1024;  // candidate blocks the slice mode supports
 
 // Builds the quantised fast form of a validated ensemble when it qualifies (m.fast).

@@ -1,7 +1,8 @@
 // Tensor-core path of the fused select kernel for the feed-forward ranker (Model B) of shape
 // 64 -> 256 -> 256 -> 1: bf16 operands, fp32 accumulation in tensor memory.
 //
-// One CTA (384 threads: eight epilogue warps, four feature-row warps) ranks one problem against up to kMlpRows candidates, 128 at a time:
+// One CTA (512 threads: eight epilogue warps, eight feature-row warps in two groups that take
+// alternate tiles) ranks one problem against up to kMlpRows candidates, 128 at a time:
 //   F    the 128 feature rows are written straight into shared memory as the bf16 A operand
 //        (candidate-only columns come standardised from a per-call table, problem-only columns
 //        are constant per CTA, the per-pair columns are computed in registers);
@@ -331,7 +332,7 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
   __shared__ ProblemTerms s_pt;
   __shared__ PairFastTerms s_pf;
   // weights; L2 first group; L2 done; L1 done; feature rows stored; accumulator 0 / 1 read out
-  __shared__ __align__(8) unsigned long long s_bar[7];
+  __shared__ __align__(8) unsigned long long s_bar[9];
   __shared__ uint32_t s_tmem;
   __shared__ uint32_t s_pwords[7];   // problem-only columns (positions 50..63) as packed bf16
   __shared__ int s_idx[3][kTileRows];  // pool index of every row of the tile (-1: no candidate)
@@ -339,7 +340,7 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
   __shared__ int s_fail;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const bool is_epi = tid < 256;  // warps 0..7 read the accumulators; warps 8..11 produce feature rows
+  const bool is_epi = tid < 256;  // warps 0..7 read the accumulators; warps 8..15 produce feature rows
   const int prob = blockIdx.x / nblk, chunk = blockIdx.x % nblk;
   int64_t lo, len;
   if (seg_off) {
@@ -350,9 +351,9 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
     len = C;
   }
   const uint32_t sbase = smem_u32(smem);
-  const uint32_t bar_w = smem_u32(&s_bar[0]), bar_a = smem_u32(&s_bar[1]), bar_b = smem_u32(&s_bar[2]),
-                 bar_c = smem_u32(&s_bar[3]), bar_x = smem_u32(&s_bar[4]), bar_f0 = smem_u32(&s_bar[5]),
-                 bar_f1 = smem_u32(&s_bar[6]);
+  const uint32_t bar_w = smem_u32(&s_bar[0]), bar_a0 = smem_u32(&s_bar[1]), bar_b = smem_u32(&s_bar[2]),
+                 bar_c = smem_u32(&s_bar[3]), bar_x0 = smem_u32(&s_bar[4]), bar_f0 = smem_u32(&s_bar[5]),
+                 bar_f1 = smem_u32(&s_bar[6]), bar_a1 = smem_u32(&s_bar[7]), bar_x1 = smem_u32(&s_bar[8]);
 
   if (tid == 0) {
     problem_terms(use_value ? p_value : p[prob], desc, s_pt);
@@ -371,10 +372,12 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
 #pragma unroll
     for (int q = 0; q < 7; ++q) s_pwords[q] = pack_bf16(pv[2 * q], q == 6 ? 0.0f : pv[2 * q + 1]);
     mbar_init(bar_w, 1);
-    mbar_init(bar_a, 1);
+    mbar_init(bar_a0, 1);
+    mbar_init(bar_a1, 1);
     mbar_init(bar_b, 1);
     mbar_init(bar_c, 1);
-    mbar_init(bar_x, kTileRows);
+    mbar_init(bar_x0, kTileRows);
+    mbar_init(bar_x1, kTileRows);
     mbar_init(bar_f0, kTileRows);
     mbar_init(bar_f1, kTileRows);
     s_fail = 0;
@@ -421,10 +424,13 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
 
     if (!is_epi) {
       // ---------------------------------- producers -------------------------------------------------
-      const int prow = tid - 256;
+      // two groups of four warps take alternate tiles, so each has two tile periods per tile
+      const int pg = (tid - 256) >> 7, prow = (tid - 256) & 127;
       const uint32_t dst = sA + prow * 16;
+      const uint32_t bar_a_prev = pg ? bar_a0 : bar_a1;  // first group of L2 of the other parity's tiles
+      const uint32_t bar_x = pg ? bar_x1 : bar_x0, bar_f = pg ? bar_f1 : bar_f0;
 #pragma unroll 1
-      for (int tile = 0; tile < n_tiles; ++tile) {
+      for (int tile = pg; tile < n_tiles; tile += 2) {
         const int64_t row = start + static_cast<int64_t>(tile) * kTileRows + prow;
         const bool live = row < len;
         int idx = -1;
@@ -457,7 +463,7 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
           for (int q = 0; q < 7; ++q) w[25 + q] = s_pwords[q];
         }
         if (tile > 0) {  // planes 0..7 are free once the first group of L2(tile - 1) is done
-          if (!mbar_wait_bounded(bar_a, ph_a)) failed = true;
+          if (!mbar_wait_bounded(bar_a_prev, ph_a)) failed = true;
           ph_a ^= 1;
         }
 #pragma unroll
@@ -472,8 +478,8 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
           if (!mbar_wait_bounded(bar_x, ph_x)) failed = true;  // every row of the tile is stored
           ph_x ^= 1;
           if (tile >= 2) {                                     // accumulator tile & 1 was read out by E2(tile - 2)
-            if (!mbar_wait_bounded((tile & 1) ? bar_f1 : bar_f0, ph_f[tile & 1])) failed = true;
-            ph_f[tile & 1] ^= 1;
+            if (!mbar_wait_bounded(bar_f, ph_f[0])) failed = true;
+            ph_f[0] ^= 1;
           }
           tc_fence_after();
 #pragma unroll
@@ -483,14 +489,15 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
           umma_commit(bar_c);
         }
       }
-      // consume what the loop left pending, so that the phase bits stay in step for the next pass
-      if (!mbar_wait_bounded(bar_a, ph_a)) failed = true;
-      ph_a ^= 1;
-      if (prow == 0) {
-        for (int a = 0; a < 2 && a < n_tiles; ++a) {  // the last read-out of each accumulator in use
-          if (!mbar_wait_bounded(a ? bar_f1 : bar_f0, ph_f[a])) failed = true;
-          ph_f[a] ^= 1;
-        }
+      // consume what the loop left pending, so that the phase bits stay in step for the next pass:
+      // the last tile's first L2 group belongs to the group that does not own that tile
+      if (((n_tiles - 1) & 1) != pg) {
+        if (!mbar_wait_bounded(bar_a_prev, ph_a)) failed = true;
+        ph_a ^= 1;
+      }
+      if (prow == 0 && n_tiles > pg) {  // the last read-out of this group's accumulator
+        if (!mbar_wait_bounded(bar_f, ph_f[0])) failed = true;
+        ph_f[0] ^= 1;
       }
     } else {
       // ---------------------------------- epilogue warps --------------------------------------------
@@ -520,7 +527,7 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
             for (int ks16 = 0; ks16 < 4; ++ks16)
               umma(acc, make_desc(sA + ks16 * 2 * kPlaneA, kPlaneA, 128),
                    make_desc(sbase + kOffW2 + ks16 * 2 * kPlaneB, kPlaneB, 128), ks16 > 0);
-            umma_commit(bar_a);
+            umma_commit((tile & 1) ? bar_a1 : bar_a0);
 #pragma unroll
             for (int ks16 = 4; ks16 < 16; ++ks16)
               umma(acc, make_desc(sA + ks16 * 2 * kPlaneA, kPlaneA, 128),
@@ -548,9 +555,15 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
         }
       }
     }
-    // rank this pass's keys (the A buffer is idle: use it as scratch)
+    // rank this pass's keys (the A buffer is idle: use it as scratch); only the second-epilogue
+    // warps and the holders of the running list have any
     __syncthreads();
-    block_topk<kTiles + 1>(keys, k, reinterpret_cast<unsigned long long*>(smem + kOffA), s_list);
+    if ((warp >= 4 && warp < 8) || warp == 0) {
+      block_topk<kTiles + 1>(keys, k, reinterpret_cast<unsigned long long*>(smem + kOffA), s_list);
+    } else {
+      const unsigned long long none[1] = {0ull};
+      block_topk<1>(none, k, reinterpret_cast<unsigned long long*>(smem + kOffA), s_list);
+    }
   }
   if (__syncthreads_or(failed)) {
     if (tid == 0 && status) atomicExch(status, KS_ERR_TIMEOUT);
@@ -679,4 +692,6 @@ cudaError_t launch_select_mlp_tc(const ks_gpu_desc& desc, const MlpModel& m, con
   return cudaGetLastError();
 }
 
+
 }  // namespace ks
+
