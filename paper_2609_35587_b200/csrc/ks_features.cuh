@@ -117,7 +117,7 @@ struct Resources {
 __device__ __forceinline__ Resources resources(const ProblemTerms& t, const ks_candidate& c,
                                                const ks_gpu_desc& h) {
   Resources r;
-  const int TM = c.tile_m, TN = c.tile_n, TK = c.tile_k, S = c.stages;
+  const int TM = c.tile_m, TN = c.tile_n;
   const int ks = c.kernel_sched & 3;
   // (consumer warpgroups in the mainloop, threads per block): WS, Pingpong, Cooperative, basic
   r.n_cons = (ks == 2) ? 2 : 1;

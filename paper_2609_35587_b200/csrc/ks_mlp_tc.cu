@@ -1,8 +1,9 @@
 // Tensor-core path of the fused select kernel for the feed-forward ranker (Model B) of shape
 // 64 -> 256 -> 256 -> 1: bf16 operands, fp32 accumulation in tensor memory.
 //
-// One CTA (512 threads: eight epilogue warps, eight feature-row warps in two groups that take
-// alternate tiles) ranks one problem against up to kMlpRows candidates, 128 at a time:
+// One CTA (512 threads: four first-epilogue warps, four second-epilogue warps, eight feature-row
+// warps in two groups that take alternate tiles) ranks one problem against its share of the
+// candidates, 128 at a time, as one continuous pipeline of tiles:
 //   F    the 128 feature rows are written straight into shared memory as the bf16 A operand
 //        (candidate-only columns come standardised from a per-call table, problem-only columns
 //        are constant per CTA, the per-pair columns are computed in registers);
@@ -11,7 +12,9 @@
 //        operand of the next layer (it overwrites the feature tile);
 //   L2   16 x tcgen05.mma against W2 into the same TMEM columns;
 //   E2   TMEM -> registers, + bias, ReLU, round to bf16, dot with w3 on the CUDA cores, + b3:
-//        the score; one ranking key per row.
+//        the score; one ranking key per row, merged into the warp's running top-k list (one
+//        entry per lane), so ranking costs a warp-wide max per tile and nothing per pass.
+// The four lists are merged once, when the CTA has walked all its tiles.
 // Both weight matrices stay resident in shared memory for the CTA's lifetime; they arrive by
 // bulk async copies (cp.async.bulk, no multicast) of an image the host prepared in the
 // operand layout. All waits are bounded and report through the status word.
@@ -82,11 +85,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-  for (int i = 0; i < kSpinLimit; ++i)
-    if (mbar_try_wait(bar, parity)) return true;
-  return false;
-}
 __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile(
       "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
@@ -153,6 +151,11 @@ __device__ __forceinline__ uint32_t pack_bf16_relu(float lo, float hi) {
 // candidate-only columns, standardised and rounded to bf16, once per call
 // ------------------------------------------------------------------------------------------
 
+// Raised by a CTA whose bounded wait ran out, so that the CTAs after it leave at once; cleared by
+// the per-call table kernel that precedes every launch. (The status word itself lives in mapped
+// host memory: reading it from every CTA would cost a PCIe round trip each.)
+__device__ int g_mlp_abort;
+
 __global__ void mlp_combo_mask_kernel(const ks_problem* __restrict__ p, int P, unsigned* __restrict__ mask) {
   unsigned m = 0;
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < P; i += gridDim.x * blockDim.x)
@@ -165,6 +168,7 @@ __global__ void __launch_bounds__(256)
 mlp_cand_cols_kernel(ks_gpu_desc desc, const ks_candidate* __restrict__ c, int C, const unsigned* mask_ptr,
                      unsigned mask_value, const __grid_constant__ MlpTcParams prm, uint8_t* __restrict__ out) {
   const int combo = blockIdx.y;
+  if (blockIdx.x == 0 && combo == 0 && threadIdx.x == 0) g_mlp_abort = 0;
   const unsigned mask = mask_ptr ? *mask_ptr : mask_value;
   if (!((mask >> combo) & 1u)) return;
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
@@ -332,14 +336,19 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
   __shared__ ProblemTerms s_pt;
   __shared__ PairFastTerms s_pf;
   // weights; L2 first group; L2 done; L1 done; feature rows stored; accumulator 0 / 1 read out
-  __shared__ __align__(8) unsigned long long s_bar[9];
+  __shared__ __align__(8) unsigned long long s_bar[10];
   __shared__ uint32_t s_tmem;
   __shared__ uint32_t s_pwords[7];   // problem-only columns (positions 50..63) as packed bf16
-  __shared__ int s_idx[3][kTileRows];  // pool index of every row of the tile (-1: no candidate)
-  __shared__ unsigned long long s_list[KS_MAX_K];
-  __shared__ int s_fail;
+  __shared__ unsigned long long s_merge[4][32];  // the second-epilogue warps' final lists
+  __shared__ int s_fail, s_abort;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (tid == 0) s_abort = *reinterpret_cast<volatile int*>(&g_mlp_abort);
+  __syncthreads();
+  if (s_abort) {  // a wait ran out in an earlier CTA of this launch: the call fails, leave at once
+    if (tid < k) partial[static_cast<size_t>(blockIdx.x) * k + tid] = 0ull;
+    return;
+  }
   const bool is_epi = tid < 256;  // warps 0..7 read the accumulators; warps 8..15 produce feature rows
   const int prob = blockIdx.x / nblk, chunk = blockIdx.x % nblk;
   int64_t lo, len;
@@ -351,9 +360,10 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
     len = C;
   }
   const uint32_t sbase = smem_u32(smem);
-  const uint32_t bar_w = smem_u32(&s_bar[0]), bar_a0 = smem_u32(&s_bar[1]), bar_b = smem_u32(&s_bar[2]),
+  const uint32_t bar_w = smem_u32(&s_bar[0]), bar_a0 = smem_u32(&s_bar[1]), bar_b0 = smem_u32(&s_bar[2]),
                  bar_c = smem_u32(&s_bar[3]), bar_x0 = smem_u32(&s_bar[4]), bar_f0 = smem_u32(&s_bar[5]),
-                 bar_f1 = smem_u32(&s_bar[6]), bar_a1 = smem_u32(&s_bar[7]), bar_x1 = smem_u32(&s_bar[8]);
+                 bar_f1 = smem_u32(&s_bar[6]), bar_a1 = smem_u32(&s_bar[7]), bar_x1 = smem_u32(&s_bar[8]),
+                 bar_b1 = smem_u32(&s_bar[9]);
 
   if (tid == 0) {
     problem_terms(use_value ? p_value : p[prob], desc, s_pt);
@@ -374,7 +384,8 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
     mbar_init(bar_w, 1);
     mbar_init(bar_a0, 1);
     mbar_init(bar_a1, 1);
-    mbar_init(bar_b, 1);
+    mbar_init(bar_b0, 1);
+    mbar_init(bar_b1, 1);
     mbar_init(bar_c, 1);
     mbar_init(bar_x0, kTileRows);
     mbar_init(bar_x1, kTileRows);
@@ -388,7 +399,7 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
     for (int off = 0; off < kW1Bytes + kW2Bytes; off += 32768)
       bulk_copy_g2s(sbase + kOffW1 + off, w_image + off, 32768, bar_w);
   }
-  if (tid < KS_MAX_K) s_list[tid] = 0ull;
+  if (tid < 128) s_merge[tid >> 5][tid & 31] = 0ull;
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(512)
                  : "memory");
@@ -401,86 +412,102 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
   const uint32_t sA = sbase + kOffA;
   const int combo = s_pt.dtype_ab * 4 + s_pt.dtype_d;
   bool failed = false;
-  if (!mbar_wait_bounded(bar_w, 0)) failed = true;
+  // Bounded wait. After the first one that runs out, every later wait of the CTA gives up after a
+  // few probes, and the CTAs that start later leave at once (device flag).
+  auto wait_ok = [&](uint32_t bar, uint32_t parity) {
+    for (int i = 0; i < kSpinLimit; ++i) {
+      if (mbar_try_wait(bar, parity)) return true;
+      if ((i & 255) == 255 && *reinterpret_cast<volatile int*>(&s_fail)) break;
+    }
+    *reinterpret_cast<volatile int*>(&s_fail) = 1;
+    atomicExch(&g_mlp_abort, 1);
+    return false;
+  };
+  if (!wait_ok(bar_w, 0)) failed = true;
   // Each role tracks the phase of the barriers it waits on. A parity wait can only tell adjacent
   // phases apart, so every barrier here is consumed before it can complete again; that is why
-  // the two accumulators have a barrier each.
-  uint32_t ph_a = 0, ph_b = 0, ph_c = 0, ph_x = 0, ph_f[2] = {0, 0};
+  // the barriers of alternating tiles come in pairs.
+  uint32_t ph_a = 0, ph_b[2] = {0, 0}, ph_c = 0, ph_x = 0, ph_f = 0;
 
-  // Roles inside a pass (tile t uses accumulator t & 1):
-  //   producers   compute row(t) in registers at any time; once L2(t-1)'s first group has
-  //               released planes 0..7 they store it there; thread 256 then issues L1(t) as soon
-  //               as all rows are stored and accumulator t & 1 has been read out (E2(t-2));
-  //   warps 0..3  wait L2(t-1) and L1(t) -> E1(t) -> issue L2(t) in two groups;
-  //   warps 4..7  wait L2(t) -> E2(t) -> key, so E2(t) runs beside E1(t+1) and L2(t+1).
+  // This CTA's tiles: blocks of kMlpRows rows at a stride of nblk blocks; every block but the last
+  // one is full. The tile pipeline runs through all of them without draining in between.
+  int total_tiles = 0;
   for (int64_t start = static_cast<int64_t>(chunk) * kMlpRows; start < len; start += static_cast<int64_t>(nblk) * kMlpRows) {
     const int64_t rows_left = len - start;
-    const int n_tiles = static_cast<int>(rows_left >= kMlpRows ? kTiles : (rows_left + kTileRows - 1) / kTileRows);
-    unsigned long long keys[kTiles + 1];
-#pragma unroll
-    for (int q = 0; q <= kTiles; ++q) keys[q] = 0ull;
-    if (tid < k) keys[kTiles] = s_list[tid];
-    __syncthreads();  // the previous pass's ranking scratch (A buffer) is no longer read
+    total_tiles += static_cast<int>(rows_left >= kMlpRows ? kTiles : (rows_left + kTileRows - 1) / kTileRows);
+  }
+  auto tile_row0 = [&](int tile) {
+    return (static_cast<int64_t>(chunk) + static_cast<int64_t>(tile / kTiles) * nblk) * kMlpRows +
+           static_cast<int64_t>(tile % kTiles) * kTileRows;
+  };
+  unsigned long long top = 0ull;  // second-epilogue warps: lane j holds the warp's j-th best key
 
-    if (!is_epi) {
-      // ---------------------------------- producers -------------------------------------------------
-      // two groups of four warps take alternate tiles, so each has two tile periods per tile
-      const int pg = (tid - 256) >> 7, prow = (tid - 256) & 127;
-      const uint32_t dst = sA + prow * 16;
-      const uint32_t bar_a_prev = pg ? bar_a0 : bar_a1;  // first group of L2 of the other parity's tiles
-      const uint32_t bar_x = pg ? bar_x1 : bar_x0, bar_f = pg ? bar_f1 : bar_f0;
+  // Roles (tile t uses accumulator t & 1):
+  //   feature rows  two groups of four warps take alternate tiles: compute row(t) in registers at
+  //                 any time; once L2(t-1)'s first group has released planes 0..7 store it there;
+  //                 the group's first warp then issues L1(t) as soon as all rows are stored and
+  //                 accumulator t & 1 has been read out (E2(t-2));
+  //   warps 0..3    wait L2(t-1) and L1(t) -> E1(t) -> issue L2(t) in two groups;
+  //   warps 4..7    wait L2(t) -> E2(t) -> key -> the warp's running top-k list, so E2(t) runs
+  //                 beside E1(t+1) and L2(t+1).
+  if (!is_epi) {
+    // ---------------------------------- feature rows ------------------------------------------------
+    const int pg = (tid - 256) >> 7, prow = (tid - 256) & 127;
+    const uint32_t dst = sA + prow * 16;
+    const uint32_t bar_a_prev = pg ? bar_a0 : bar_a1;  // first group of L2 of the other parity's tiles
+    const uint32_t bar_x = pg ? bar_x1 : bar_x0, bar_f = pg ? bar_f1 : bar_f0;
 #pragma unroll 1
-      for (int tile = pg; tile < n_tiles; tile += 2) {
-        const int64_t row = start + static_cast<int64_t>(tile) * kTileRows + prow;
-        const bool live = row < len;
-        int idx = -1;
-        uint32_t w[32];
+    for (int tile = pg; tile < total_tiles; tile += 2) {
+      const int64_t row = tile_row0(tile) + prow;
+      const bool live = row < len;
+      uint32_t w[32];
 #pragma unroll
-        for (int q = 0; q < 32; ++q) w[q] = 0u;
-        if (live) {
-          idx = seg_off ? seg_idx[lo + row] : static_cast<int>(row);
-          const ks_candidate cand = c[idx];
-          const uint4* rec = reinterpret_cast<const uint4*>(cand_cols + (static_cast<size_t>(combo) * C + idx) * kCandRec);
+      for (int q = 0; q < 32; ++q) w[q] = 0u;
+      if (live) {
+        const int idx = seg_off ? seg_idx[lo + row] : static_cast<int>(row);
+        const ks_candidate cand = c[idx];
+        const uint4* rec = reinterpret_cast<const uint4*>(cand_cols + (static_cast<size_t>(combo) * C + idx) * kCandRec);
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const uint4 r = __ldg(rec + q);
-            w[4 * q] = r.x; w[4 * q + 1] = r.y; w[4 * q + 2] = r.z; w[4 * q + 3] = r.w;
-          }
-          float x[64];
-          auto put = [&](int col, float v) {
-            const int kk = kpos(col);
-            x[kk] = fmaf(v, prm.scale[kk], prm.shift[kk]);
-          };
-          // single-precision evaluation (the values are rounded to bf16 next); the exact
-          // 64-bit form only for tile counts beyond its range
-          if (!pair_columns_bf16(s_pt, s_pf, cand, desc, w[15] & 0xFFFFu, put))
-            pair_columns<false>(s_pt, cand, desc, static_cast<long long>(w[15] & 0xFFFFu), put);
-          // positions 0..28 came from the table; 29..49 are the per-pair columns
-          w[14] = (w[14] & 0xFFFFu) | (pack_bf16(0.0f, x[29]) & 0xFFFF0000u);
-#pragma unroll
-          for (int q = 15; q < 25; ++q) w[q] = pack_bf16(x[2 * q], x[2 * q + 1]);
-#pragma unroll
-          for (int q = 0; q < 7; ++q) w[25 + q] = s_pwords[q];
+        for (int q = 0; q < 4; ++q) {
+          const uint4 r = __ldg(rec + q);
+          w[4 * q] = r.x; w[4 * q + 1] = r.y; w[4 * q + 2] = r.z; w[4 * q + 3] = r.w;
         }
-        if (tile > 0) {  // planes 0..7 are free once the first group of L2(tile - 1) is done
-          if (!mbar_wait_bounded(bar_a_prev, ph_a)) failed = true;
-          ph_a ^= 1;
-        }
+        float x[64];
+        auto put = [&](int col, float v) {
+          const int kk = kpos(col);
+          x[kk] = fmaf(v, prm.scale[kk], prm.shift[kk]);
+        };
+        // single-precision evaluation (the values are rounded to bf16 next); the exact
+        // 64-bit form only for tile counts beyond its range
+        if (!pair_columns_bf16(s_pt, s_pf, cand, desc, w[15] & 0xFFFFu, put))
+          pair_columns<false>(s_pt, cand, desc, static_cast<long long>(w[15] & 0xFFFFu), put);
+        // positions 0..28 came from the table; 29..49 are the per-pair columns
+        w[14] = (w[14] & 0xFFFFu) | (pack_bf16(0.0f, x[29]) & 0xFFFF0000u);
 #pragma unroll
-        for (int pl = 0; pl < 8; ++pl)
-          asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + pl * kPlaneA), "r"(w[4 * pl]),
-                       "r"(w[4 * pl + 1]), "r"(w[4 * pl + 2]), "r"(w[4 * pl + 3])
-                       : "memory");
-        s_idx[tile % 3][prow] = idx;
-        fence_async_proxy();
-        mbar_arrive(bar_x);
-        if (prow == 0) {
-          if (!mbar_wait_bounded(bar_x, ph_x)) failed = true;  // every row of the tile is stored
-          ph_x ^= 1;
-          if (tile >= 2) {                                     // accumulator tile & 1 was read out by E2(tile - 2)
-            if (!mbar_wait_bounded(bar_f, ph_f[0])) failed = true;
-            ph_f[0] ^= 1;
-          }
+        for (int q = 15; q < 25; ++q) w[q] = pack_bf16(x[2 * q], x[2 * q + 1]);
+#pragma unroll
+        for (int q = 0; q < 7; ++q) w[25 + q] = s_pwords[q];
+      }
+      if (tile > 0) {  // planes 0..7 are free once the first group of L2(tile - 1) is done
+        if (!wait_ok(bar_a_prev, ph_a)) failed = true;
+        ph_a ^= 1;
+      }
+#pragma unroll
+      for (int pl = 0; pl < 8; ++pl)
+        asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst + pl * kPlaneA), "r"(w[4 * pl]),
+                     "r"(w[4 * pl + 1]), "r"(w[4 * pl + 2]), "r"(w[4 * pl + 3])
+                     : "memory");
+      fence_async_proxy();
+      mbar_arrive(bar_x);
+      if ((warp & 3) == 0) {
+        // the group's first warp issues L1; its lanes wait together
+        if (!wait_ok(bar_x, ph_x)) failed = true;  // every row of the tile is stored
+        ph_x ^= 1;
+        if (tile >= 2) {  // accumulator tile & 1 was read out by E2(tile - 2)
+          if (!wait_ok(bar_f, ph_f)) failed = true;
+          ph_f ^= 1;
+        }
+        if (lane == 0) {
           tc_fence_after();
 #pragma unroll
           for (int ks16 = 0; ks16 < 4; ++ks16)
@@ -488,88 +515,83 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
                  make_desc(sbase + kOffW1 + ks16 * 2 * kPlaneB, kPlaneB, 128), ks16 > 0);
           umma_commit(bar_c);
         }
-      }
-      // consume what the loop left pending, so that the phase bits stay in step for the next pass:
-      // the last tile's first L2 group belongs to the group that does not own that tile
-      if (((n_tiles - 1) & 1) != pg) {
-        if (!mbar_wait_bounded(bar_a_prev, ph_a)) failed = true;
-        ph_a ^= 1;
-      }
-      if (prow == 0 && n_tiles > pg) {  // the last read-out of this group's accumulator
-        if (!mbar_wait_bounded(bar_f, ph_f[0])) failed = true;
-        ph_f[0] ^= 1;
-      }
-    } else {
-      // ---------------------------------- epilogue warps --------------------------------------------
-      // warps 0..3: first epilogue + L2 issue; warps 4..7: second epilogue + ranking keys. Thread
-      // (quarter, lane) of either group owns row quarter * 32 + lane and all 256 columns.
-      const int quarter = warp & 3, group = warp >> 2;
-      const int trow = quarter * 32 + lane;
-      const uint32_t tmem_row = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
-      if (group == 0) {
-#pragma unroll 1
-        for (int tile = 0; tile < n_tiles; ++tile) {
-          const uint32_t acc = tmem + (tile & 1) * 256, acc_row = tmem_row + (tile & 1) * 256;
-          if (tile > 0) {  // the A buffer is free once L2(tile - 1) is complete
-            if (!mbar_wait_bounded(bar_b, ph_b)) failed = true;
-            ph_b ^= 1;
-          }
-          if (!mbar_wait_bounded(bar_c, ph_c)) failed = true;  // L1(tile) is complete
-          ph_c ^= 1;
-          tc_fence_after();
-          epilogue1<0>(acc_row, sA + trow * 16, prm);
-          fence_async_proxy();
-          tc_fence_before();
-          epi_sync();
-          if (tid == 0) {
-            tc_fence_after();
-#pragma unroll
-            for (int ks16 = 0; ks16 < 4; ++ks16)
-              umma(acc, make_desc(sA + ks16 * 2 * kPlaneA, kPlaneA, 128),
-                   make_desc(sbase + kOffW2 + ks16 * 2 * kPlaneB, kPlaneB, 128), ks16 > 0);
-            umma_commit((tile & 1) ? bar_a1 : bar_a0);
-#pragma unroll
-            for (int ks16 = 4; ks16 < 16; ++ks16)
-              umma(acc, make_desc(sA + ks16 * 2 * kPlaneA, kPlaneA, 128),
-                   make_desc(sbase + kOffW2 + ks16 * 2 * kPlaneB, kPlaneB, 128), 1u);
-            umma_commit(bar_b);
-          }
-        }
-        if (!mbar_wait_bounded(bar_b, ph_b)) failed = true;  // the last L2: keeps the phase bit in step
-        ph_b ^= 1;
-      } else {
-#pragma unroll 1
-        for (int tile = 0; tile < n_tiles; ++tile) {
-          const uint32_t acc_row = tmem_row + (tile & 1) * 256;
-          if (!mbar_wait_bounded(bar_b, ph_b)) failed = true;  // L2(tile) is complete
-          ph_b ^= 1;
-          tc_fence_after();
-          const int idx = s_idx[tile % 3][trow];
-          const float score = epilogue2<0>(acc_row, prm) + prm.b3;
-          tc_fence_before();
-          mbar_arrive((tile & 1) ? bar_f1 : bar_f0);
-          const unsigned long long key = idx >= 0 ? make_key(score + 0.0f, idx) : 0ull;
-#pragma unroll
-          for (int q = 0; q < kTiles; ++q)
-            if (q == tile) keys[q] = key;
-        }
+        __syncwarp();
       }
     }
-    // rank this pass's keys (the A buffer is idle: use it as scratch); only the second-epilogue
-    // warps and the holders of the running list have any
-    __syncthreads();
-    if ((warp >= 4 && warp < 8) || warp == 0) {
-      block_topk<kTiles + 1>(keys, k, reinterpret_cast<unsigned long long*>(smem + kOffA), s_list);
+  } else {
+    // ---------------------------------- epilogue warps ----------------------------------------------
+    // warps 0..3: first epilogue + L2 issue; warps 4..7: second epilogue + ranking keys. Thread
+    // (quarter, lane) of either group owns row quarter * 32 + lane and all 256 columns.
+    const int quarter = warp & 3, group = warp >> 2;
+    const int trow = quarter * 32 + lane;
+    const uint32_t tmem_row = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
+    if (group == 0) {
+#pragma unroll 1
+      for (int tile = 0; tile < total_tiles; ++tile) {
+        const uint32_t acc = tmem + (tile & 1) * 256, acc_row = tmem_row + (tile & 1) * 256;
+        if (tile > 0) {  // the A buffer is free once L2(tile - 1) is complete
+          if (!wait_ok((tile & 1) ? bar_b0 : bar_b1, ph_b[(tile - 1) & 1])) failed = true;
+          ph_b[(tile - 1) & 1] ^= 1;
+        }
+        if (!wait_ok(bar_c, ph_c)) failed = true;  // L1(tile) is complete
+        ph_c ^= 1;
+        tc_fence_after();
+        epilogue1<0>(acc_row, sA + trow * 16, prm);
+        fence_async_proxy();
+        tc_fence_before();
+        epi_sync();
+        if (tid == 0) {
+          tc_fence_after();
+#pragma unroll
+          for (int ks16 = 0; ks16 < 4; ++ks16)
+            umma(acc, make_desc(sA + ks16 * 2 * kPlaneA, kPlaneA, 128),
+                 make_desc(sbase + kOffW2 + ks16 * 2 * kPlaneB, kPlaneB, 128), ks16 > 0);
+          umma_commit((tile & 1) ? bar_a1 : bar_a0);
+#pragma unroll
+          for (int ks16 = 4; ks16 < 16; ++ks16)
+            umma(acc, make_desc(sA + ks16 * 2 * kPlaneA, kPlaneA, 128),
+                 make_desc(sbase + kOffW2 + ks16 * 2 * kPlaneB, kPlaneB, 128), 1u);
+          umma_commit((tile & 1) ? bar_b1 : bar_b0);
+        }
+      }
     } else {
-      const unsigned long long none[1] = {0ull};
-      block_topk<1>(none, k, reinterpret_cast<unsigned long long*>(smem + kOffA), s_list);
+#pragma unroll 1
+      for (int tile = 0; tile < total_tiles; ++tile) {
+        const uint32_t acc_row = tmem_row + (tile & 1) * 256;
+        const int64_t row = tile_row0(tile) + trow;
+        int idx = -1;  // fetched before the wait, so that its latency hides behind it
+        if (row < len) idx = seg_off ? __ldg(seg_idx + lo + row) : static_cast<int>(row);
+        if (!wait_ok((tile & 1) ? bar_b1 : bar_b0, ph_b[tile & 1])) failed = true;  // L2(tile) is complete
+        ph_b[tile & 1] ^= 1;
+        tc_fence_after();
+        const float score = epilogue2<0>(acc_row, prm) + prm.b3;
+        tc_fence_before();
+        mbar_arrive((tile & 1) ? bar_f1 : bar_f0);
+        warp_topk_insert(top, idx >= 0 ? make_key(score + 0.0f, idx) : 0ull, k);
+      }
+      s_merge[quarter][lane] = top;
     }
   }
+  // merge the four warps' lists: the j-th best is the largest key below the (j-1)-th
   if (__syncthreads_or(failed)) {
     if (tid == 0 && status) atomicExch(status, KS_ERR_TIMEOUT);
     failed = true;
   }
-  if (tid < k) partial[(static_cast<size_t>(prob) * nblk + chunk) * k + tid] = failed ? 0ull : s_list[tid];
+  if (warp == 0) {
+    unsigned long long mine[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) mine[q] = s_merge[q][lane];
+    unsigned long long prev = ~0ull;
+    for (int j = 0; j < k; ++j) {
+      unsigned long long best = 0ull;
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        if (mine[q] < prev && mine[q] > best) best = mine[q];
+      best = warp_max_u64(best);
+      if (lane == 0) partial[(static_cast<size_t>(prob) * nblk + chunk) * k + j] = failed ? 0ull : best;
+      prev = best;
+    }
+  }
   tc_fence_before();
   __syncthreads();
   if (warp == 0) {

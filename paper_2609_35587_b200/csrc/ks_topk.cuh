@@ -34,6 +34,24 @@ __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v)
   return (static_cast<unsigned long long>(hi) << 32) | lo;
 }
 
+// A warp's running top-k list: lane j < k holds the j-th best key seen so far, the other lanes 0.
+// Merges one new key per lane (0 = none) into it. Each round takes the warp's largest new key;
+// the loop ends as soon as that key would not make the list, which after the first few calls is
+// at once for almost every call. Keys are distinct, so the owner of the round's key is unique.
+__device__ __forceinline__ void warp_topk_insert(unsigned long long& mine, unsigned long long v, int k) {
+  const int lane = threadIdx.x & 31;
+  for (;;) {
+    const unsigned long long m = warp_max_u64(v);
+    const unsigned long long kth = __shfl_sync(0xFFFFFFFFu, mine, k - 1);
+    if (m <= kth) break;
+    const int pos = __popc(__ballot_sync(0xFFFFFFFFu, mine > m));  // entries that stay ahead of m
+    const unsigned long long up = __shfl_up_sync(0xFFFFFFFFu, mine, 1);
+    if (lane == pos) mine = m;
+    else if (lane > pos && lane < k) mine = up;
+    if (v == m) v = 0ull;
+  }
+}
+
 // The k largest of the block's keys (N per thread), descending, into s_list[0..k).
 // Two levels: every warp first ranks its own keys (k rounds of warp-wide max, no block
 // barrier), then warp 0 ranks the n_warps * k survivors. All threads of the block must call;
