@@ -64,6 +64,8 @@ ks_status read_status(ks_ctx* ctx) {
   const int v = *static_cast<volatile int*>(ctx->h_status);
   if (v != 0) {
     *ctx->h_status = 0;
+    // a failed launch may have left arrival counters of the slice mode behind
+    if (ctx->d_counters) cudaMemset(ctx->d_counters, 0, sizeof(int) * (ks::kMaxSliceBlocks + 1));
     return static_cast<ks_status>(v);
   }
   return KS_OK;

@@ -108,6 +108,10 @@ __device__ __forceinline__ float lds_f32(uint32_t addr) {
   return v;
 }
 
+// Raised by a CTA whose bounded wait ran out, so that the CTAs after it leave at once; cleared by
+// the per-call table kernel that precedes every launch of the select kernel.
+__device__ int g_fast_abort;
+
 // #{j : T[j] <= v} over 127 sorted thresholds padded with +inf: 7 branch-free steps.
 __device__ __forceinline__ int bin_search(const float* T, float v) {
   int pos = 0;
@@ -158,6 +162,7 @@ cand_rows_kernel(ks_gpu_desc desc, const ks_candidate* __restrict__ c, int C, co
   extern __shared__ float s_cthr[];  // thresholds of the candidate-only rows
   __shared__ uint8_t s_r0[64], s_rc[64];
   const int combo = blockIdx.y;
+  if (blockIdx.x == 0 && combo == 0 && threadIdx.x == 0) g_fast_abort = 0;
   const unsigned mask = mask_ptr ? *mask_ptr : mask_value;
   if (!((mask >> combo) & 1u)) return;
   const int first = fv.n_pair_rows;
@@ -295,11 +300,17 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
   __shared__ __align__(8) unsigned long long s_bar[2];
   __shared__ uint8_t s_row0[64], s_rowcnt[64], s_pbin[64];
   __shared__ float s_pfeat[64];
-  __shared__ int s_fail, s_last, s_done[2];
+  __shared__ int s_fail, s_last, s_done[2], s_abort;
 
   const int tid = threadIdx.x;
   const int S = sl.n_slices;
   const int prob = blockIdx.x / (nblk * S), chunk = (blockIdx.x / S) % nblk, slice = blockIdx.x % S;
+  if (tid == 0) s_abort = *reinterpret_cast<volatile int*>(&g_fast_abort);
+  __syncthreads();
+  if (s_abort) {  // a wait ran out in an earlier CTA of this launch: the call fails, leave at once
+    if (tid < k && slice == 0) partial[(static_cast<size_t>(prob) * nblk + chunk) * k + tid] = 0ull;
+    return;
+  }
   int64_t lo, len;
   if (seg_off) {
     lo = seg_off[prob];
@@ -381,9 +392,14 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
       const int b = (ch - ch_begin) & 1;
       const uint32_t bar = b ? bar1 : bar0;
       const uint32_t par = b ? phase1 : phase0;
-      if (!mbar_wait_bounded(bar, par)) {
-        s_fail = 1;
-        if (status) atomicExch(status, KS_ERR_TIMEOUT);
+      // after one wait has run out the CTA stops waiting (and refilling): the call fails, and
+      // the CTAs that start later leave at once
+      if (*reinterpret_cast<volatile int*>(&s_fail) || !mbar_wait_bounded(bar, par)) {
+        if (!*reinterpret_cast<volatile int*>(&s_fail)) {
+          s_fail = 1;
+          atomicExch(&g_fast_abort, 1);
+          if (status) atomicExch(status, KS_ERR_TIMEOUT);
+        }
       }
       if (b) phase1 ^= 1; else phase0 ^= 1;
       const uint32_t buf = sbase + (b ? kOffBuf1 : kOffBuf0);
