@@ -291,10 +291,22 @@ bool is_valid(const OProblem& p, const OCandidate& c, const OGpuDesc& h, unsigne
 }
 
 // Model A: walk one tree from its root; returns the leaf's node index.
+// A node with pad bit 0 set is a partition split on a categorical field (native categorical
+// handling with a fixed level ordering): the bit pattern of v is a membership mask over the
+// field's level codes, and a row whose code is in the set goes to the right child.
 int walk(const ONode* tree, int node, const float* x) {
   const ONode& nd = tree[node];
   if (nd.feat == 0xFFFF) return node;
-  return walk(tree, x[nd.feat] < nd.v ? nd.left : nd.left + 1, x);
+  bool right;
+  if (nd.pad & 1) {
+    uint32_t mask;
+    std::memcpy(&mask, &nd.v, 4);
+    const int code = static_cast<int>(x[nd.feat]);
+    right = code >= 0 && code < 32 && ((mask >> code) & 1u);
+  } else {
+    right = !(x[nd.feat] < nd.v);
+  }
+  return walk(tree, right ? nd.left + 1 : nd.left, x);
 }
 
 float score_gbdt_row(const float* x, int n_trees, const int64_t* off, const ONode* nodes,

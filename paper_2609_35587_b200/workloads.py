@@ -215,6 +215,26 @@ def segments(seed: int, P: int, pool: int, per_problem: int):
 # models
 # ------------------------------------------------------------------------------------------
 
+# Feature columns that hold a categorical field's level code, with the number of levels: layout
+# flags, operand type, bias flag, activation, kernel / epilogue schedule, tile scheduler.
+CATEGORICAL_LEVELS = {3: 2, 4: 2, 5: 4, 8: 2, 9: 3, 17: 4, 18: 3, 19: 2}
+_S_PARTITION = 0x70617274
+
+
+def with_partition_splits(seed: int, nodes: np.ndarray) -> np.ndarray:
+    """Copy of `nodes` in which every internal node on a categorical column becomes a partition
+    split: pad = 1 and the bit pattern of v = a seeded, non-empty, proper subset of the field's
+    levels (the members go to the right child)."""
+    out = nodes.copy()
+    for i in np.nonzero(np.isin(out["feat"], list(CATEGORICAL_LEVELS)))[0]:
+        levels = CATEGORICAL_LEVELS[int(out["feat"][i])]
+        full = (1 << levels) - 1
+        mask = 1 + int(mix64(seed, _S_PARTITION, np.array([i], dtype=np.uint64))[0] % np.uint64(full - 1))
+        out["v"][i] = np.array([mask], dtype=np.uint32).view(np.float32)[0]
+        out["pad"][i] = 1
+    return out
+
+
 _stats_cache = None
 
 

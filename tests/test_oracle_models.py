@@ -228,3 +228,83 @@ def test_one_layer_model_is_the_linear_scorer():
     wv = bf16_bits_to_f32(m["weights"][0]).astype(np.float64)[0]
     ref = xs @ wv + float(m["biases"][0][0])
     np.testing.assert_allclose(s, ref, rtol=1e-6, atol=1e-6)
+
+
+# ---------------------------------------------------------------------------------------------
+# partition splits on categorical fields (native categorical handling)
+# ---------------------------------------------------------------------------------------------
+
+def cat_node(feat, mask, left):
+    nd = np.zeros(1, wl.NODE_DT)
+    nd["feat"], nd["pad"], nd["left"] = feat, 1, left
+    nd["v"] = np.array([mask], np.uint32).view(np.float32)
+    return nd
+
+
+def test_partition_split_membership_goes_right():
+    """kernel_sched (column 17) has codes 0..3; members of the set go right."""
+    x = np.zeros((4, 64), np.float32)
+    x[:, 17] = [0, 1, 2, 3]
+    leaves = make_tree([(None, -1.0, 0), (None, 2.0, 0)])
+    for mask in range(1, 15):
+        nodes = np.concatenate([cat_node(17, mask, 1), leaves])
+        s, leaf = oracle.score_gbdt(x, np.array([0, 3]), nodes, want_leaf_idx=True)
+        want = [2.0 if (mask >> c) & 1 else -1.0 for c in range(4)]
+        assert s.tolist() == want and leaf[:, 0].tolist() == [2 if v > 0 else 1 for v in want]
+
+
+def test_partition_split_of_an_upper_set_equals_a_numeric_split():
+    """The set {c, c+1, ...} is the numeric split x < c: same leaves on real feature rows."""
+    prob, cand, _, _ = wl.make_inputs(1, P=3, C=400)
+    x = oracle.featurize(prob, cand, DESC)
+    rng = np.random.default_rng(3)
+    for col, levels in wl.CATEGORICAL_LEVELS.items():
+        for c in range(1, levels):
+            upper = sum(1 << v for v in range(c, levels))
+            leaves = make_tree([(None, float(rng.normal()), 0), (None, float(rng.normal()), 0)])
+            numeric = np.concatenate([make_tree([(col, float(c), 1)]), leaves])
+            part = np.concatenate([cat_node(col, upper, 1), leaves])
+            a = oracle.score_gbdt(x, np.array([0, 3]), numeric)
+            b = oracle.score_gbdt(x, np.array([0, 3]), part)
+            assert np.array_equal(a, b), (col, c)
+
+
+def test_partition_ensemble_against_nested_ifs():
+    prob, cand, _, _ = wl.make_inputs(2, P=2, seg=150)
+    x = oracle.featurize(prob, cand[:150], DESC)
+    thr = wl.feature_stats("cfg2")["thr"]
+    off, nodes = wl.gbdt_complete(17, 40, 4, thr, 0.1)
+    pnodes = wl.with_partition_splits(5, nodes)
+    assert pnodes["pad"].sum() > 20 and np.array_equal(pnodes["feat"], nodes["feat"])
+    got = oracle.score_gbdt(x, off, pnodes, base_score=0.25)
+    want = np.empty(len(x))
+    for r in range(len(x)):
+        s = 0.25
+        for t in range(len(off) - 1):
+            tree = pnodes[off[t]:off[t + 1]]
+            i = 0
+            while tree[i]["feat"] != 0xFFFF:
+                f, v = int(tree[i]["feat"]), tree[i]["v"]
+                if tree[i]["pad"] & 1:
+                    right = (int(np.float32(v).view(np.uint32)) >> int(x[r, f])) & 1
+                else:
+                    right = not (x[r, f] < v)
+                i = int(tree[i]["left"]) + (1 if right else 0)
+            s += float(tree[i]["v"])
+        want[r] = s
+    np.testing.assert_allclose(got, want, rtol=1e-6, atol=1e-6)
+    # complementing a set and swapping the children changes nothing
+    flipped = pnodes.copy()
+    for t in range(len(off) - 1):
+        lo = off[t]
+        for i in range(lo, off[t + 1]):
+            if flipped[i]["pad"] & 1:
+                levels = wl.CATEGORICAL_LEVELS[int(flipped[i]["feat"])]
+                m = int(flipped["v"][i:i + 1].view(np.uint32)[0]) ^ ((1 << levels) - 1)
+                flipped["v"][i] = np.array([m], np.uint32).view(np.float32)[0]
+                l = lo + int(flipped[i]["left"])
+                if flipped[l]["feat"] == 0xFFFF and flipped[l + 1]["feat"] == 0xFFFF:
+                    flipped[[l, l + 1]] = flipped[[l + 1, l]]
+                else:  # only leaf pairs can be swapped in place; undo the complement here
+                    flipped["v"][i] = pnodes["v"][i]
+    np.testing.assert_allclose(oracle.score_gbdt(x, off, flipped, base_score=0.25), got, rtol=1e-6, atol=1e-6)
