@@ -88,11 +88,19 @@ typedef struct {
 
 /* Interchange form of one tree node. Node 0 of a tree is its root. An internal node sends
  * a row to `left` when x[feat] < thr (strict, fp32) and to `left + 1` otherwise; a leaf has
- * feat == 0xFFFF and carries its value in thr_or_leaf. Indices are relative to the tree. */
+ * feat == 0xFFFF and carries its value in thr_or_leaf. Indices are relative to the tree.
+ * kind == KS_NODE_PARTITION marks a partition split on a categorical field (section "Model A":
+ * native categorical handling with a fixed level ordering): feat must be one of the columns
+ * that hold a level code (layout flags 3, 4; operand type 5; bias flag 8; activation 9; kernel
+ * schedule 17; epilogue schedule 18; tile scheduler 19), the bit pattern of thr_or_leaf is a
+ * non-zero membership mask over the field's level codes (bit c = level c), and a row whose
+ * level is in the set goes to `left + 1`, any other row to `left`. */
+#define KS_NODE_NUMERIC 0
+#define KS_NODE_PARTITION 1
 typedef struct {
   float thr_or_leaf;
   uint16_t feat;   /* 0 .. KS_F-1, or 0xFFFF for a leaf                                    */
-  uint16_t pad;    /* must be 0                                                            */
+  uint16_t kind;   /* KS_NODE_NUMERIC or KS_NODE_PARTITION; 0 for a leaf                   */
   int32_t left;    /* index of the left child (right child = left + 1); 0 for a leaf       */
 } ks_node_host;    /* 12 bytes                                                             */
 
@@ -100,7 +108,8 @@ typedef struct {
  * ks_model_create_gbdt are repacked by the library). 8 bytes. */
 typedef struct {
   float thr_or_leaf; /* threshold of an internal node, value of a leaf                    */
-  uint16_t feat;     /* 0 .. KS_F-1, or 0xFFFF for a leaf                                  */
+  uint16_t feat;     /* 0 .. KS_F-1 (| 0x8000: partition split, thr_or_leaf = level mask), */
+                     /* or 0xFFFF for a leaf                                               */
   uint16_t left;     /* tree-relative index of the left child (right child = left + 1)     */
 } ks_node_dev;
 
@@ -124,7 +133,8 @@ const char* ks_last_cuda_error(const ks_ctx* ctx);
 /* Model A (section "Model A (gradient-boosted ranker)"): f(x) = base_score + sum_m h_m(x).
  * h_nodes holds the trees back to back, tree t in [h_tree_offsets[t], h_tree_offsets[t+1]).
  * All structural validation happens here, on the host: feature ids < KS_F, children inside
- * the tree and after their parent, finite thresholds and leaves, depth <= KS_MAX_DEPTH,
+ * the tree and after their parent, finite thresholds and leaves, partition splits only on
+ * level-code columns with a non-zero mask inside the field's levels, depth <= KS_MAX_DEPTH,
  * every node reachable exactly once. The trees are repacked into a private device layout;
  * the host arrays may be freed on return. Synchronous. */
 ks_status ks_model_create_gbdt(ks_ctx* ctx, int n_trees, const int64_t* h_tree_offsets,

@@ -55,7 +55,7 @@ struct OGpuDesc {
 struct ONode {
   float v;
   uint16_t feat;
-  uint16_t pad;
+  uint16_t kind;  // 0 numeric split (or leaf), 1 partition split
   int32_t left;
 };
 static_assert(sizeof(OProblem) == 16 && sizeof(OCandidate) == 16 && sizeof(OGpuDesc) == 80 &&
@@ -291,14 +291,14 @@ bool is_valid(const OProblem& p, const OCandidate& c, const OGpuDesc& h, unsigne
 }
 
 // Model A: walk one tree from its root; returns the leaf's node index.
-// A node with pad bit 0 set is a partition split on a categorical field (native categorical
+// A node of kind 1 is a partition split on a categorical field (native categorical
 // handling with a fixed level ordering): the bit pattern of v is a membership mask over the
 // field's level codes, and a row whose code is in the set goes to the right child.
 int walk(const ONode* tree, int node, const float* x) {
   const ONode& nd = tree[node];
   if (nd.feat == 0xFFFF) return node;
   bool right;
-  if (nd.pad & 1) {
+  if (nd.kind == 1) {
     uint32_t mask;
     std::memcpy(&mask, &nd.v, 4);
     const int code = static_cast<int>(x[nd.feat]);

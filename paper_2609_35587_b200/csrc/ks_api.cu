@@ -102,7 +102,16 @@ int validate_tree(const ks_node_host* t, int64_t n) {
   for (int64_t i = 0; i < n; ++i) {
     const ks_node_host& nd = t[i];
     if (depth[i] < 0) return -1;  // parents precede children, so an unreached node is an orphan
-    if (!std::isfinite(nd.thr_or_leaf)) return -1;
+    if (nd.kind > KS_NODE_PARTITION) return -1;
+    if (nd.kind == KS_NODE_PARTITION) {
+      if (nd.feat == 0xFFFF) return -1;
+      const int levels = ks::categorical_levels(nd.feat);
+      uint32_t mask;
+      std::memcpy(&mask, &nd.thr_or_leaf, 4);
+      if (levels == 0 || mask == 0 || (mask >> levels) != 0) return -1;
+    } else if (!std::isfinite(nd.thr_or_leaf)) {
+      return -1;
+    }
     if (nd.feat == 0xFFFF) continue;
     if (nd.feat >= KS_F) return -1;
     const int64_t l = nd.left;
@@ -290,7 +299,8 @@ ks_status ks_model_create_gbdt(ks_ctx* ctx, int n_trees, const int64_t* h_tree_o
   std::vector<ks::DevNode> dev(static_cast<size_t>(total));
   for (int64_t i = 0; i < total; ++i) {
     dev[i].v = h_nodes[i].thr_or_leaf;
-    dev[i].feat = h_nodes[i].feat;
+    dev[i].feat = h_nodes[i].kind == KS_NODE_PARTITION ? static_cast<uint16_t>(h_nodes[i].feat | 0x8000u)
+                                                       : h_nodes[i].feat;
     dev[i].left = h_nodes[i].feat == 0xFFFF ? 0 : static_cast<uint16_t>(h_nodes[i].left);
   }
   std::vector<int> roots(n_trees + 1);

@@ -10,6 +10,10 @@
 //   chunk is one contiguous block a CTA copies into shared memory with one bulk async copy.
 //   The nodes of the top levels are also kept as (row offset, replicated threshold) pairs that
 //   travel as a kernel parameter, i.e. through the constant bank.
+//   A partition split on a categorical field ("level in S goes right") joins the same scheme
+//   through rank rows: a row whose byte is the rank of the pair's level in a fixed ordering of
+//   the field's levels, chosen so that S or its complement is the set of ranks >= c; the node
+//   then is the ordinary "bin <= c - 1 goes left", with its children exchanged for a complement.
 //
 // Hoisting
 //   Rows are grouped by what their feature depends on. Candidate-only rows (given the
@@ -32,6 +36,7 @@
 //            top-k list.
 #include <algorithm>
 #include <cmath>
+#include <cstring>
 #include <limits>
 #include <new>
 #include <vector>
@@ -120,6 +125,17 @@ __device__ __forceinline__ int bin_search(const float* T, float v) {
   return pos;
 }
 
+// Bin of value v in one row of the threshold table. A row whose last slot is negative infinity is
+// a rank row of a categorical field: slot c holds the rank of level c in the row's ordering of
+// the levels (see build_fast_gbdt), and the bin is that rank.
+__device__ __forceinline__ int row_bin(const float* T, float v) {
+  if (T[kThrPerRow - 1] < 0.0f) {
+    const int code = __float2int_rz(v);
+    return (code >= 0 && code < 4) ? __float2int_rz(T[code]) : 0;
+  }
+  return bin_search(T, v);
+}
+
 // Slice mode (single-problem latency call): the trees are split over n_slices CTAs per
 // candidate block. Every CTA stores its partial scores; the last CTA to arrive for a block
 // (atomic counter, nobody waits) adds the slices in a fixed order and ranks the block; the
@@ -189,7 +205,7 @@ cand_rows_kernel(ks_gpu_desc desc, const ks_candidate* __restrict__ c, int C, co
     if (feat_class(col) != 1) return;
     const int r0 = s_r0[col] - first, rc = s_rc[col];
     for (int q = 0; q < rc; ++q) {
-      const uint32_t b = 0x80u | bin_search(s_cthr + (r0 + q) * kThrPerRow, v);
+      const uint32_t b = 0x80u | row_bin(s_cthr + (r0 + q) * kThrPerRow, v);
       const int at = r0 + q;
 #pragma unroll
       for (int w = 0; w < kCandRec / 4; ++w)
@@ -349,7 +365,7 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
     const int first = fv.n_pair_rows + fv.n_cand_rows;
     for (int q = 0; q < s_rowcnt[tid]; ++q)
       s_pbin[s_row0[tid] + q - first] =
-          static_cast<uint8_t>(0x80 | bin_search(fv.thr + (s_row0[tid] + q) * kThrPerRow, s_pfeat[tid]));
+          static_cast<uint8_t>(0x80 | row_bin(fv.thr + (s_row0[tid] + q) * kThrPerRow, s_pfeat[tid]));
   }
   uint32_t phase0 = 0, phase1 = 0;
   const int word = tid % kWords, half = tid / kWords;
@@ -556,23 +572,73 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
 // host: repack
 // ------------------------------------------------------------------------------------------
 
+// The orderings of L levels used by rank rows (lowest rank first).
+static const int* partition_perm(int L, int q) {
+  static const int p2[1][4] = {{0, 1, 0, 0}};
+  static const int p3[2][4] = {{0, 1, 2, 0}, {0, 2, 1, 0}};
+  static const int p4[3][4] = {{0, 1, 2, 3}, {1, 3, 0, 2}, {1, 2, 0, 3}};
+  return L == 2 ? p2[q] : (L == 3 ? p3[q] : p4[q]);
+}
+// How a membership mask is tested: levels of rank >= cut in ordering `perm` go right, or, with
+// `swap`, go left (the mask is the complement of that upper set).
+struct PartitionCode {
+  int perm, cut;
+  bool swap;
+};
+static std::vector<PartitionCode> partition_codes(int L) {
+  const int n_perm = L == 2 ? 1 : (L == 3 ? 2 : 3);
+  const uint32_t full = (1u << L) - 1;
+  std::vector<PartitionCode> code(full + 1, PartitionCode{-1, 0, false});
+  for (int q = 0; q < n_perm; ++q)
+    for (int c = 1; c < L; ++c) {
+      uint32_t up = 0;
+      for (int r = c; r < L; ++r) up |= 1u << partition_perm(L, q)[r];
+      if (code[up].perm < 0) code[up] = PartitionCode{q, c, false};
+      if (code[full ^ up].perm < 0) code[full ^ up] = PartitionCode{q, c, true};
+    }
+  return code;
+}
+
 cudaError_t build_fast_gbdt(GbdtModel& m, int n_trees, const int64_t* off, const ks_node_host* nodes) {
   m.fast = false;
   if (n_trees < 1 || m.max_depth < 1 || m.max_depth > kFastMaxDepth) return cudaSuccess;
   const int D = m.max_depth;
   // distinct thresholds per feature, sliced into rows of at most 127
   std::vector<std::vector<float>> thr(KS_F);
-  for (int64_t i = 0; i < off[n_trees]; ++i)
-    if (nodes[i].feat != 0xFFFF) thr[nodes[i].feat].push_back(nodes[i].thr_or_leaf);
+  // Partition splits: "level in S goes right" becomes a bin comparison on a rank row. A rank row
+  // orders the field's levels by one of a few fixed permutations; S (or its complement, with the
+  // node's children exchanged) is then the set of levels of rank >= c for some c, i.e. the
+  // ordinary test "bin <= c - 1 goes left". The permutations below reach every proper subset of
+  // 2, 3 and 4 levels up to complement.
+  std::vector<std::vector<PartitionCode>> part(KS_F);  // per feature: code of every mask
+  bool perm_used[KS_F][3] = {};
+  for (int64_t i = 0; i < off[n_trees]; ++i) {
+    const ks_node_host& nd = nodes[i];
+    if (nd.feat == 0xFFFF) continue;
+    if (nd.kind == KS_NODE_PARTITION) {
+      const int L = categorical_levels(nd.feat);
+      if (L == 0) return cudaSuccess;
+      if (part[nd.feat].empty()) part[nd.feat] = partition_codes(L);
+      uint32_t mask;
+      std::memcpy(&mask, &nd.thr_or_leaf, 4);
+      if (mask == 0 || mask >= (1u << L)) return cudaSuccess;
+      if (mask != (1u << L) - 1) perm_used[nd.feat][part[nd.feat][mask].perm] = true;
+    } else {
+      thr[nd.feat].push_back(nd.thr_or_leaf);
+    }
+  }
   std::vector<uint8_t> row0(64, 0), rowcnt(64, 0);
+  int rank_row[KS_F][3];  // row offset (within the feature's rows) of each permutation in use
   int n_rows = 0, n_class[3] = {0, 0, 0};
   for (int f = 0; f < KS_F; ++f) {
     auto& v = thr[f];
     std::sort(v.begin(), v.end());
     v.erase(std::unique(v.begin(), v.end()), v.end());
-    rowcnt[f] = static_cast<uint8_t>((v.size() + 126) / 127);
-    n_class[feat_class(f)] += rowcnt[f];
-    n_rows += rowcnt[f];
+    int cnt = static_cast<int>((v.size() + 126) / 127);
+    for (int q = 0; q < 3; ++q) rank_row[f][q] = perm_used[f][q] ? cnt++ : -1;
+    rowcnt[f] = static_cast<uint8_t>(cnt);
+    n_class[feat_class(f)] += cnt;
+    n_rows += cnt;
   }
   if (n_rows == 0 || n_rows > kMaxRows || n_class[1] > kCandRec) return cudaSuccess;  // generic path
   // rows ordered: per-pair, candidate-only, problem-only
@@ -582,11 +648,21 @@ cudaError_t build_fast_gbdt(GbdtModel& m, int n_trees, const int64_t* off, const
     for (int f = 0; f < KS_F; ++f) {
       if (feat_class(f) != cls) continue;
       row0[f] = static_cast<uint8_t>(next);
-      for (int q = 0; q < rowcnt[f]; ++q, ++next)
+      const int n_thr_rows = static_cast<int>((thr[f].size() + 126) / 127);
+      for (int q = 0; q < n_thr_rows; ++q, ++next)
         for (int j = 0; j < 127; ++j) {
           const size_t s = static_cast<size_t>(q) * 127 + j;
           if (s < thr[f].size()) table[static_cast<size_t>(next) * kThrPerRow + j] = thr[f][s];
         }
+      for (int q = 0; q < 3; ++q) {  // rank rows: slot c = rank of level c, last slot = marker
+        if (rank_row[f][q] < 0) continue;
+        const int L = categorical_levels(f);
+        float* row = table.data() + static_cast<size_t>(next) * kThrPerRow;
+        for (int c = 0; c < 4; ++c) row[c] = 0.0f;
+        for (int r = 0; r < L; ++r) row[partition_perm(L, q)[r]] = static_cast<float>(r);
+        row[kThrPerRow - 1] = -std::numeric_limits<float>::infinity();
+        ++next;
+      }
     }
   }
   const int per_tree_words = (2 << D) - 1;
@@ -624,13 +700,36 @@ cudaError_t build_fast_gbdt(GbdtModel& m, int n_trees, const int64_t* off, const
             if (nd.feat == 0xFFFF) {
               lc = rc = nd.thr_or_leaf;
             } else {
-              const auto& v = thr[nd.feat];
-              const int j = static_cast<int>(std::lower_bound(v.begin(), v.end(), nd.thr_or_leaf) - v.begin());
-              const uint32_t row = row0[nd.feat] + j / 127, jl = j % 127;
-              word = (row * kRowStride) << 8 | (0x80u | jl);
-              tw = make_uint2(row * kRowStride, (jl + 1) * 0x01010101u);
+              uint32_t row, jl;
+              bool swap = false, always_right = false;
+              if (nd.kind == KS_NODE_PARTITION) {
+                uint32_t mask;
+                std::memcpy(&mask, &nd.thr_or_leaf, 4);
+                if (mask == (1u << categorical_levels(nd.feat)) - 1) {
+                  always_right = true;  // every level is a member
+                  row = 0;
+                  jl = 127;
+                } else {
+                  const PartitionCode pc = part[nd.feat][mask];
+                  row = row0[nd.feat] + rank_row[nd.feat][pc.perm];
+                  jl = pc.cut - 1;
+                  swap = pc.swap;
+                }
+              } else {
+                const auto& v = thr[nd.feat];
+                const int j = static_cast<int>(std::lower_bound(v.begin(), v.end(), nd.thr_or_leaf) - v.begin());
+                row = row0[nd.feat] + j / 127;
+                jl = j % 127;
+              }
               ls = nd.left;
               rs = nd.left + 1;
+              if (always_right) {
+                ls = rs;  // the walk always goes left here: put the right subtree on both sides
+              } else {
+                word = (row * kRowStride) << 8 | (0x80u | jl);
+                tw = make_uint2(row * kRowStride, (jl + 1) * 0x01010101u);
+                if (swap) std::swap(ls, rs);
+              }
             }
           }
           lvl[tt * (1 << l) + i] = word;

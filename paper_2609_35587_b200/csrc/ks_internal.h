@@ -120,6 +120,17 @@ constexpr int kMlpThreads = 512;        // threads per block of the tensor-core 
 constexpr int kMlpRows = 4096;          // candidates one block ranks per pass
 constexpr int kMaxSliceBlocks = 1024;  // candidate blocks the slice mode supports
 
+// Levels of the categorical field held by feature column `col` (0: not a level-code column):
+// layout flags, operand type, bias flag, activation, kernel / epilogue schedule, tile scheduler.
+inline int categorical_levels(int col) {
+  switch (col) {
+    case 3: case 4: case 8: case 19: return 2;
+    case 9: case 18: return 3;
+    case 5: case 17: return 4;
+    default: return 0;
+  }
+}
+
 // Builds the quantised fast form of a validated ensemble when it qualifies (m.fast).
 cudaError_t build_fast_gbdt(GbdtModel& m, int n_trees, const int64_t* h_tree_offsets,
                             const ks_node_host* h_nodes);

@@ -91,8 +91,15 @@ __device__ __forceinline__ float walk_ensemble(const DevNode* __restrict__ nodes
     DevNode nd = load_node(tree);
 #pragma unroll 1
     for (int d = 0; d <= KS_MAX_DEPTH && nd.feat != 0xFFFFu; ++d) {
-      const float x = s_cols[nd.feat * kBlock];
-      i = nd.left + (x < nd.v ? 0 : 1);
+      const float x = s_cols[(nd.feat & 0x7FFFu) * kBlock];
+      int right;
+      if (nd.feat & 0x8000u) {  // partition split: v's bits are the set of levels that go right
+        const unsigned code = static_cast<unsigned>(__float2int_rz(x));
+        right = code < 32u ? (__float_as_uint(nd.v) >> code) & 1u : 0;
+      } else {
+        right = x < nd.v ? 0 : 1;
+      }
+      i = nd.left + right;
       nd = load_node(tree + i);
     }
     if (leaf_out) leaf_out[t] = static_cast<uint16_t>(i);

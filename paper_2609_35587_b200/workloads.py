@@ -31,7 +31,7 @@ CANDIDATE_DT = np.dtype([("tile_m", "<u2"), ("tile_n", "<u2"), ("tile_k", "<u2")
                          ("instr_n", "<u2"), ("stages", "u1"), ("cluster_m", "u1"),
                          ("cluster_n", "u1"), ("kernel_sched", "u1"), ("epi_sched", "u1"),
                          ("tile_sched", "u1"), ("instr_m", "u1"), ("instr_k", "u1")])
-NODE_DT = np.dtype([("v", "<f4"), ("feat", "<u2"), ("pad", "<u2"), ("left", "<i4")])
+NODE_DT = np.dtype([("v", "<f4"), ("feat", "<u2"), ("kind", "<u2"), ("left", "<i4")])
 GPU_DESC_DT = np.dtype([("num_sms", "<u4"), ("smem_per_sm", "<u4"), ("smem_per_cta_max", "<u4"),
                         ("smem_reserved", "<u4"), ("regs_per_sm", "<u4"),
                         ("max_threads_per_sm", "<u4"), ("max_ctas_per_sm", "<u4"),
@@ -223,7 +223,7 @@ _S_PARTITION = 0x70617274
 
 def with_partition_splits(seed: int, nodes: np.ndarray) -> np.ndarray:
     """Copy of `nodes` in which every internal node on a categorical column becomes a partition
-    split: pad = 1 and the bit pattern of v = a seeded, non-empty, proper subset of the field's
+    split: kind = 1 and the bit pattern of v = a seeded, non-empty, proper subset of the field's
     levels (the members go to the right child)."""
     out = nodes.copy()
     for i in np.nonzero(np.isin(out["feat"], list(CATEGORICAL_LEVELS)))[0]:
@@ -231,7 +231,7 @@ def with_partition_splits(seed: int, nodes: np.ndarray) -> np.ndarray:
         full = (1 << levels) - 1
         mask = 1 + int(mix64(seed, _S_PARTITION, np.array([i], dtype=np.uint64))[0] % np.uint64(full - 1))
         out["v"][i] = np.array([mask], dtype=np.uint32).view(np.float32)[0]
-        out["pad"][i] = 1
+        out["kind"][i] = 1
     return out
 
 

@@ -512,3 +512,68 @@ def test_select_static_score_bit_exact(ks, ctx):
     with pytest.raises(ks.KsError) as ei:
         ctx.score(x, model)
     assert ei.value.status == ks.KS_ERR_UNSUPPORTED
+
+
+# ---------------------------------------------------------------------------------------------
+# partition splits on categorical fields (general tree kernel)
+# ---------------------------------------------------------------------------------------------
+
+def test_partition_split_ensembles(ks, ctx):
+    # leaf indices and scores of the standalone scorer
+    prob, cand, so, si = wl.make_inputs(2, P=5, seg=700)
+    x = oracle.featurize(prob, cand, DESC, so, si)
+    off, nodes = wl.gbdt_complete(23, 64, 6, wl.feature_stats("cfg2")["thr"], 0.1)
+    pnodes = wl.with_partition_splits(9, nodes)
+    assert pnodes["kind"].sum() > 100
+    model = ctx.model_create_gbdt(off, pnodes, 0.5)
+    sc, leaf = ctx.score(dev(ks, x), model, want_leaf_idx=True)
+    torch.cuda.synchronize()
+    rs, rleaf = oracle.score_gbdt(x, off, pnodes, 0.5, want_leaf_idx=True)
+    assert np.array_equal(leaf.cpu().numpy(), rleaf)
+    assert np.all(np.abs(sc.cpu().numpy() - rs) <= TOL_GBDT * np.maximum(1, np.abs(rs)))
+    # the partitions matter: the same trees with numeric splits score differently
+    assert not np.array_equal(oracle.score_gbdt(x, off, nodes, 0.5), rs)
+    # the fused path, dense and segmented, against the oracle
+    w = wl.Workload("partition", DESC, prob, cand, 10, gbdt=(off, pnodes, 0.5), seg_offsets=so, seg_index=si)
+    idx, sc = run_select(ks, ctx, w, model)
+    check_select(w, idx, sc, TOL_GBDT)
+    w2 = wl.make_workload(1, P=3, C=3000, trees=40)
+    pn2 = wl.with_partition_splits(4, w2.gbdt[1])
+    w2.gbdt = (w2.gbdt[0], pn2, w2.gbdt[2])
+    m2 = ctx.model_create_gbdt(*w2.gbdt)
+    idx, sc = run_select(ks, ctx, w2, m2)
+    check_select(w2, idx, sc, TOL_GBDT)
+    hi, hs = ctx.select_one(w2.problems[:1], dev(ks, w2.candidates), len(w2.candidates), m2, w2.k)
+    assert np.array_equal(hi.numpy(), idx[0])
+    # every subset of the levels of a four-level field, the full set included, as the root of a
+    # depth-2 tree (quantised kernel: rank rows, exchanged children, always-right)
+    for mask in range(1, 16):
+        nd = np.zeros(7, wl.NODE_DT)
+        nd[0] = (np.array([mask], np.uint32).view(np.float32)[0], 17, 1, 1)
+        nd[1] = (np.array([1], np.uint32).view(np.float32)[0], 19, 1, 3)
+        nd[2] = (3.5, 10, 0, 5)
+        for j, v in enumerate((0.25, -0.5, 1.0, -2.0)):
+            nd[3 + j] = (v, 0xFFFF, 0, 0)
+        w3 = wl.Workload("subset", DESC, w2.problems, w2.candidates[:2500], 10, gbdt=(np.array([0, 7]), nd, 0.0))
+        idx, sc = run_select(ks, ctx, w3, ctx.model_create_gbdt(*w3.gbdt))
+        check_select(w3, idx, sc, TOL_GBDT)
+        _, rsc = oracle.select(w3.problems, w3.candidates, DESC, 10, gbdt=w3.gbdt)
+        assert np.array_equal(sc, rsc), mask
+    # an ensemble too deep for the quantised kernel keeps its partition splits on the general one
+    off5, n5 = wl.gbdt_complete(31, 6, 11, wl.feature_stats("cfg1")["thr"], 0.1)
+    p5 = wl.with_partition_splits(2, n5)
+    w5 = wl.Workload("deep", DESC, w2.problems, w2.candidates[:1200], 10, gbdt=(off5, p5, 0.0))
+    idx, sc = run_select(ks, ctx, w5, ctx.model_create_gbdt(*w5.gbdt))
+    check_select(w5, idx, sc, TOL_GBDT)
+    # validation: partition splits only on level-code columns, with a mask inside the levels
+    def one(feat, mask, kind=1):
+        nd = np.zeros(3, wl.NODE_DT)
+        nd[0] = (np.array([mask], np.uint32).view(np.float32)[0], feat, kind, 1)
+        nd[1] = (0.5, 0xFFFF, 0, 0)
+        nd[2] = (-0.5, 0xFFFF, 0, 0)
+        return np.array([0, 3]), nd
+    ctx.model_create_gbdt(*one(17, 0b1010), 0.0)
+    for feat, mask, kind in ((17, 0, 1), (17, 0b10000, 1), (19, 0b100, 1), (10, 1, 1), (17, 1, 2)):
+        with pytest.raises(ks.KsError) as ei:
+            ctx.model_create_gbdt(*one(feat, mask, kind), 0.0)
+        assert ei.value.status == ks.KS_ERR_INVALID_ARG

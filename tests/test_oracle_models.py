@@ -236,7 +236,7 @@ def test_one_layer_model_is_the_linear_scorer():
 
 def cat_node(feat, mask, left):
     nd = np.zeros(1, wl.NODE_DT)
-    nd["feat"], nd["pad"], nd["left"] = feat, 1, left
+    nd["feat"], nd["kind"], nd["left"] = feat, 1, left
     nd["v"] = np.array([mask], np.uint32).view(np.float32)
     return nd
 
@@ -275,7 +275,7 @@ def test_partition_ensemble_against_nested_ifs():
     thr = wl.feature_stats("cfg2")["thr"]
     off, nodes = wl.gbdt_complete(17, 40, 4, thr, 0.1)
     pnodes = wl.with_partition_splits(5, nodes)
-    assert pnodes["pad"].sum() > 20 and np.array_equal(pnodes["feat"], nodes["feat"])
+    assert pnodes["kind"].sum() > 20 and np.array_equal(pnodes["feat"], nodes["feat"])
     got = oracle.score_gbdt(x, off, pnodes, base_score=0.25)
     want = np.empty(len(x))
     for r in range(len(x)):
@@ -285,7 +285,7 @@ def test_partition_ensemble_against_nested_ifs():
             i = 0
             while tree[i]["feat"] != 0xFFFF:
                 f, v = int(tree[i]["feat"]), tree[i]["v"]
-                if tree[i]["pad"] & 1:
+                if tree[i]["kind"] & 1:
                     right = (int(np.float32(v).view(np.uint32)) >> int(x[r, f])) & 1
                 else:
                     right = not (x[r, f] < v)
@@ -298,7 +298,7 @@ def test_partition_ensemble_against_nested_ifs():
     for t in range(len(off) - 1):
         lo = off[t]
         for i in range(lo, off[t + 1]):
-            if flipped[i]["pad"] & 1:
+            if flipped[i]["kind"] & 1:
                 levels = wl.CATEGORICAL_LEVELS[int(flipped[i]["feat"])]
                 m = int(flipped["v"][i:i + 1].view(np.uint32)[0]) ^ ((1 << levels) - 1)
                 flipped["v"][i] = np.array([m], np.uint32).view(np.float32)[0]
