@@ -49,7 +49,7 @@ namespace ks {
 
 namespace {
 
-constexpr int kBufBytes = 32 * 1024;   // one tree-chunk buffer
+constexpr int kBufBytes = 16 * 1024;   // one tree-chunk buffer
 constexpr int kMaxRows = 80;           // quantised rows the kernel supports (tile <= 160 KB)
 constexpr int kThrPerRow = 128;        // 127 thresholds + padding
 constexpr int kRowStride = kFastRows;  // bytes between rows of the tile (one byte per candidate)
@@ -303,7 +303,7 @@ __device__ __forceinline__ float path_step(float a, uint32_t cb_r, float K0f, fl
 }
 
 template <int L, int NP>  // L levels evaluated word-wise; NP path levels unrolled (-1: runtime count)
-__global__ void __launch_bounds__(kFastThreads, 1)
+__global__ void __launch_bounds__(kFastThreads, 2)
 select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_problem p_value, int use_value,
                    const ks_candidate* __restrict__ c, int P, int C, int nblk, int rows_per_cta,
                    const int64_t* __restrict__ seg_off, const int32_t* __restrict__ seg_idx, FastView fv,
@@ -802,7 +802,7 @@ size_t fast_scratch_bytes(int C) { return 256 + static_cast<size_t>(kCombos) * C
 int fast_slices(const GbdtModel& g, int64_t blocks) {
   if (blocks < 1) blocks = 1;
   if (blocks > kMaxSliceBlocks) return 1;
-  int64_t s = 148 / blocks;
+  int64_t s = 296 / blocks;
   if (s > g.n_chunks) s = g.n_chunks;
   return static_cast<int>(s < 1 ? 1 : s);
 }

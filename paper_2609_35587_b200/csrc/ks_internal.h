@@ -112,7 +112,7 @@ namespace ks {
 
 constexpr int kBlock = 256;            // threads per block of the pair kernels
 constexpr int kSubTilesMax = 8;        // sub-tiles of kBlock rows one block ranks
-constexpr int kFastThreads = 1024;      // threads per block of the quantised tree kernel
+constexpr int kFastThreads = 512;      // threads per block of the quantised tree kernel
 constexpr int kFastR = 2;              // candidates per thread there
 constexpr int kFastRows = kFastThreads * kFastR;
 constexpr int kFastMaxDepth = 10;
