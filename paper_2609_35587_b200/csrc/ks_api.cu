@@ -502,7 +502,8 @@ ks_status ks_select_one(ks_ctx* ctx, ks_problem p, const ks_candidate* d_c, int 
     const int S = ks::fast_slices(model->gbdt, nblk);
     if (S > 1) {
       const size_t b_part = align_up(sizeof(unsigned long long) * nblk * k);
-      const size_t b_scratch = align_up(ks::fast_scratch_bytes(C));
+      // scratch of this path: the prepared tiles, one per candidate block (no per-call table)
+      const size_t b_scratch = align_up(static_cast<size_t>(nblk) * model->gbdt.n_qrows * ks::kFastRows);
       const size_t b_scores = align_up(sizeof(float) * static_cast<size_t>(S) * C);
       ks_status s = ensure_workspace(ctx, b_part + b_scratch + b_scores);
       if (s != KS_OK) return s;
@@ -514,6 +515,7 @@ ks_status ks_select_one(ks_ctx* ctx, ks_problem p, const ks_candidate* d_c, int 
       sl.counters = ctx->d_counters;
       sl.out_idx = ctx->d_pinned_idx;
       sl.out_score = ctx->d_pinned_score;
+      sl.tiles = reinterpret_cast<uint8_t*>(base + b_part);
       cudaError_t e = ks::launch_select_fast(ctx->desc, model->gbdt, nullptr, &p, 1, d_c, C, nblk, ks::kFastRows,
                                              nullptr, nullptr, k, reinterpret_cast<unsigned long long*>(base),
                                              base + b_part, ctx->d_status, st, &ctx->launches, nullptr, &sl);

@@ -147,6 +147,7 @@ struct SliceArgs {
   int* counters;           // [P * nblk + 1], zero on entry; every counter is reset by its last user
   int32_t* out_idx;        // single-problem form only: [k] final result (device-visible, may be
   float* out_score;        // mapped host memory); null when a merge kernel follows
+  const uint8_t* tiles;    // prepared tiles [blocks][rows][kRowStride] (tile_one_kernel), or null
 };
 
 struct FastView {
@@ -216,6 +217,58 @@ cand_rows_kernel(ks_gpu_desc desc, const ks_candidate* __restrict__ c, int C, co
 #pragma unroll
   for (int q = 0; q < kCandRec / 16; ++q)
     if (q * 16 < fv.n_cand_rows) dst[q] = make_uint4(rec[4 * q], rec[4 * q + 1], rec[4 * q + 2], rec[4 * q + 3]);
+}
+
+// ------------------------------------------------------------------------------------------
+// single-problem call: the whole tile of every candidate block, once per call
+// ------------------------------------------------------------------------------------------
+
+// One thread per tile slot writes all rows of its candidate's tile column, in the layout phase A
+// would produce, for the one problem of the call. The CTAs that share a candidate block in slice
+// mode then copy the block's tile instead of each rebuilding it. Slots past the catalogue get the
+// neutral byte. Also clears the abort flag (this kernel precedes the select kernel).
+template <bool kPairRows>  // true: the per-pair rows; false: the candidate-only and problem-only rows
+__device__ __forceinline__ void tile_one_rows(const ks_gpu_desc& desc, const ks_problem& p_value,
+                                              const ks_candidate* __restrict__ c, int C, const FastView& fv,
+                                              uint8_t* __restrict__ tiles, float* s_thr) {
+  __shared__ ProblemTerms s_pt;
+  __shared__ uint8_t s_r0[64], s_rc[64];
+  const int tid = threadIdx.x;
+  if (blockIdx.x == 0 && tid == 0) g_fast_abort = 0;
+  // rows are ordered per-pair, candidate-only, problem-only
+  const int first = kPairRows ? 0 : fv.n_pair_rows;
+  const int count = kPairRows ? fv.n_pair_rows : fv.n_rows - fv.n_pair_rows;
+  for (int i = tid; i < count * kThrPerRow; i += blockDim.x) s_thr[i] = __ldg(fv.thr + first * kThrPerRow + i);
+  if (tid < 64) {
+    s_r0[tid] = fv.feat_row0[tid];
+    s_rc[tid] = fv.feat_rowcnt[tid];
+  }
+  if (tid == 0) problem_terms(p_value, desc, s_pt);
+  __syncthreads();
+  const int slot = blockIdx.x * blockDim.x + tid;
+  const int blk = slot / kFastRows, in = slot % kFastRows;
+  const int t = in % kFastThreads, r = in / kFastThreads;  // phase-A thread and its candidate
+  uint8_t* my = tiles + static_cast<size_t>(blk) * fv.n_rows * kRowStride + (t % kWords) * 4 + (t / kWords) * kFastR + r;
+  if (slot >= C) {
+    for (int q = first; q < first + count; ++q) my[q * kRowStride] = 0x80;
+    return;
+  }
+  const ks_candidate cand = c[slot];
+  featurize_pair(s_pt, cand, desc, [&](int col, float v) {
+    if ((feat_class(col) == 2) != kPairRows) return;
+    const int r0 = s_r0[col], rc = s_rc[col];
+    for (int q = 0; q < rc; ++q)
+      my[(r0 + q) * kRowStride] = static_cast<uint8_t>(0x80 | row_bin(s_thr + (r0 + q - first) * kThrPerRow, v));
+  });
+}
+
+// blockIdx.y picks the role, so that both halves of the work are in flight together
+__global__ void __launch_bounds__(256)
+tile_one_kernel(ks_gpu_desc desc, ks_problem p_value, const ks_candidate* __restrict__ c, int C, FastView fv,
+                uint8_t* __restrict__ tiles) {
+  extern __shared__ float s_thr[];  // thresholds of this role's rows
+  if (blockIdx.y == 0) tile_one_rows<true>(desc, p_value, c, C, fv, tiles, s_thr);
+  else tile_one_rows<false>(desc, p_value, c, C, fv, tiles, s_thr);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -375,14 +428,21 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
     const int64_t stop = (start + rows_per_cta < len) ? start + rows_per_cta : len;
     // ---- phase A ---------------------------------------------------------------------------------
     __syncthreads();
-    {
-      float4* dst = reinterpret_cast<float4*>(smem + kOffBuf0);
-      const float4* src = reinterpret_cast<const float4*>(fv.thr);
-      for (int i = tid; i < fv.n_pair_rows * kThrPerRow / 4; i += kFastThreads) dst[i] = __ldg(src + i);
+    if (sl.tiles) {
+      // single-problem call: the block's tile was built once for all the CTAs that share it
+      const uint4* src = reinterpret_cast<const uint4*>(sl.tiles + static_cast<size_t>(chunk) * fv.n_rows * kRowStride);
+      uint4* dst = reinterpret_cast<uint4*>(smem + kOffTile);
+      for (int i = tid; i < fv.n_rows * (kRowStride / 16); i += kFastThreads) dst[i] = __ldcg(src + i);
+    } else {
+      {
+        float4* dst = reinterpret_cast<float4*>(smem + kOffBuf0);
+        const float4* src = reinterpret_cast<const float4*>(fv.thr);
+        for (int i = tid; i < fv.n_pair_rows * kThrPerRow / 4; i += kFastThreads) dst[i] = __ldg(src + i);
+      }
+      __syncthreads();
+      fill_tile(desc, s_pt, c, fv, seg_off, seg_idx, C, lo, start, stop,
+                reinterpret_cast<const float*>(smem + kOffBuf0), s_row0, s_rowcnt, s_pbin, smem + kOffTile);
     }
-    __syncthreads();
-    fill_tile(desc, s_pt, c, fv, seg_off, seg_idx, C, lo, start, stop,
-              reinterpret_cast<const float*>(smem + kOffBuf0), s_row0, s_rowcnt, s_pbin, smem + kOffTile);
     __syncthreads();  // tile complete; the threshold table is no longer needed
 
     // ---- phase B ---------------------------------------------------------------------------------
@@ -860,7 +920,15 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
     combo_mask_kernel<<<P >= 4096 ? 16 : 1, 256, 0, stream>>>(d_p, P, d_mask);
     ++*launches;
   }
-  if (C > 0) {
+  const bool tiles_mode = uv && slice && slice->n_slices > 1 && slice->tiles && P == 1 && !seg_off;
+  if (tiles_mode) {
+    // one launch, two roles (blockIdx.y): the per-pair rows, and the candidate- / problem-only rows
+    const size_t tthr = sizeof(float) * kThrPerRow * g.n_qrows;
+    e = cudaFuncSetAttribute(tile_one_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(tthr));
+    if (e != cudaSuccess) return e;
+    tile_one_kernel<<<dim3(nblk * (kFastRows / 256), 2), 256, tthr, stream>>>(desc, pv, d_c, C, fv, slice->tiles);
+    ++*launches;
+  } else if (C > 0) {
     const size_t cthr = sizeof(float) * kThrPerRow * (g.n_cand_rows > 0 ? g.n_cand_rows : 1);
     cand_rows_kernel<<<dim3((C + 255) / 256, kCombos), 256, cthr, stream>>>(desc, d_c, C, uv ? nullptr : d_mask,
                                                                             mask_value, fv, d_rows);
@@ -879,6 +947,7 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
     sl.counters = slice->counters;
     sl.out_idx = slice->out_idx;
     sl.out_score = slice->out_score;
+    sl.tiles = tiles_mode ? slice->tiles : nullptr;
   }
   const FastTopParams& top = *g.h_top;
   const int L = g.top_levels, np = g.fast_depth - L;

@@ -143,6 +143,7 @@ struct FastSlice {
   int* counters;     // [blocks + 1], zero between calls
   int32_t* out_idx;  // single-problem form: [k], device-visible; else null (a merge kernel follows)
   float* out_score;
+  uint8_t* tiles;    // single-problem form: scratch for the prepared tiles [blocks][rows][kFastRows], or null
 };
 
 // Search-space enumeration and validity filtering (ks_catalogue.cu).
