@@ -440,7 +440,7 @@ def main():
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, per launch, from the
 # ncu summaries under profiles/ (None until a capture exists for that workload).
-TRAFFIC_BYTES = {1: 13.1e6, 4: 10.0e6}
+TRAFFIC_BYTES = {1: 16.6e6, 4: 5.7e6}
 
 if __name__ == "__main__":
     main()
