@@ -61,9 +61,9 @@ constexpr int kCombos = 16;            // dtype_ab x dtype_d
 static_assert(kFastThreads == 2 * kWords && kFastR == 2, "tile geometry");
 
 // shared memory map (byte offsets from the dynamic shared base)
+constexpr int kNBuf = 2;                // tree-chunk buffers (a ring; four of half the size measured slower)
 constexpr int kOffBuf0 = 0;
-constexpr int kOffBuf1 = kBufBytes;
-constexpr int kOffTile = 2 * kBufBytes;
+constexpr int kOffTile = kNBuf * kBufBytes;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -366,10 +366,10 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
   __shared__ ProblemTerms s_pt;
   __shared__ unsigned long long s_warp[kFastThreads / 32 * KS_MAX_K];
   __shared__ unsigned long long s_list[KS_MAX_K];
-  __shared__ __align__(8) unsigned long long s_bar[2];
+  __shared__ __align__(8) unsigned long long s_bar[kNBuf];
   __shared__ uint8_t s_row0[64], s_rowcnt[64], s_pbin[64];
   __shared__ float s_pfeat[64];
-  __shared__ int s_fail, s_last, s_done[2], s_abort;
+  __shared__ int s_fail, s_last, s_done[kNBuf], s_abort;
 
   const int tid = threadIdx.x;
   const int S = sl.n_slices;
@@ -392,7 +392,7 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
   const int ch_begin = static_cast<int>(static_cast<int64_t>(fv.n_chunks) * slice / S);
   const int ch_end = static_cast<int>(static_cast<int64_t>(fv.n_chunks) * (slice + 1) / S);
   const uint32_t sbase = smem_u32(smem);
-  const uint32_t bar0 = smem_u32(&s_bar[0]), bar1 = smem_u32(&s_bar[1]);
+  const uint32_t bar0 = smem_u32(&s_bar[0]);  // barrier of buffer b: bar0 + 8 b
   if (tid == 0) {
     problem_terms(use_value ? p_value : p[prob], desc, s_pt);
     // problem-only columns do not look at the candidate: evaluate them on a dummy one
@@ -402,10 +402,9 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
     featurize_pair(s_pt, dummy, desc, [&](int col, float v) {
       if (feat_class(col) == 0) s_pfeat[col] = v;
     });
-    mbar_init(bar0, 1);
-    mbar_init(bar1, 1);
+    for (int b = 0; b < kNBuf; ++b) mbar_init(bar0 + 8u * b, 1);
     s_fail = 0;
-    s_done[0] = s_done[1] = 0;
+    for (int b = 0; b < kNBuf; ++b) s_done[b] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (tid < 64) {
@@ -420,7 +419,7 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
       s_pbin[s_row0[tid] + q - first] =
           static_cast<uint8_t>(0x80 | row_bin(fv.thr + (s_row0[tid] + q) * kThrPerRow, s_pfeat[tid]));
   }
-  uint32_t phase0 = 0, phase1 = 0;
+  uint32_t phases = 0;  // bit b: parity of buffer b's barrier
   const int word = tid % kWords, half = tid / kWords;
 
   for (int64_t start = static_cast<int64_t>(chunk) * rows_per_cta; start < len;
@@ -449,13 +448,10 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
     if (tid == 0) {
       fence_async_proxy();
       const char* src = reinterpret_cast<const char*>(fv.chunks) + static_cast<size_t>(ch_begin) * fv.chunk_bytes;
-      if (ch_end > ch_begin) {
-        mbar_expect_tx(bar0, fv.chunk_bytes);
-        bulk_copy_g2s(sbase + kOffBuf0, src, fv.chunk_bytes, bar0);
-      }
-      if (ch_end > ch_begin + 1) {
-        mbar_expect_tx(bar1, fv.chunk_bytes);
-        bulk_copy_g2s(sbase + kOffBuf1, src + fv.chunk_bytes, fv.chunk_bytes, bar1);
+      for (int b = 0; b < kNBuf && ch_begin + b < ch_end; ++b) {
+        mbar_expect_tx(bar0 + 8u * b, fv.chunk_bytes);
+        bulk_copy_g2s(sbase + kOffBuf0 + b * kBufBytes, src + static_cast<size_t>(b) * fv.chunk_bytes, fv.chunk_bytes,
+                      bar0 + 8u * b);
       }
     }
     float score[4] = {0.0f, 0.0f, 0.0f, 0.0f};
@@ -465,9 +461,9 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
     constexpr int kTop = (1 << L) - 1;
 #pragma unroll 1
     for (int ch = ch_begin; ch < ch_end; ++ch) {
-      const int b = (ch - ch_begin) & 1;
-      const uint32_t bar = b ? bar1 : bar0;
-      const uint32_t par = b ? phase1 : phase0;
+      const int b = (ch - ch_begin) % kNBuf;
+      const uint32_t bar = bar0 + 8u * b;
+      const uint32_t par = (phases >> b) & 1u;
       // after one wait has run out the CTA stops waiting (and refilling): the call fails, and
       // the CTAs that start later leave at once
       if (*reinterpret_cast<volatile int*>(&s_fail) || !mbar_wait_bounded(bar, par)) {
@@ -477,8 +473,8 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
           if (status) atomicExch(status, KS_ERR_TIMEOUT);
         }
       }
-      if (b) phase1 ^= 1; else phase0 ^= 1;
-      const uint32_t buf = sbase + (b ? kOffBuf1 : kOffBuf0);
+      phases ^= 1u << b;
+      const uint32_t buf = sbase + kOffBuf0 + b * kBufBytes;
       // With A_l the shared address of a walk's node at level l, A_{l+1} = 2 A_l + (4 tpc - buf)
       // + 4 bit for every level, and after the last level A points at the walk's leaf.
       const int k0 = static_cast<int>(4u * tpc) - static_cast<int>(buf);
@@ -538,10 +534,10 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
       if ((tid & 31) == 0) {
         if (atomicAdd(&s_done[b], 1) == kFastThreads / 32 - 1) {
           s_done[b] = 0;
-          if (ch + 2 < ch_end && !s_fail) {
+          if (ch + kNBuf < ch_end && !s_fail) {
             fence_async_proxy();
             mbar_expect_tx(bar, fv.chunk_bytes);
-            bulk_copy_g2s(buf, reinterpret_cast<const char*>(fv.chunks) + static_cast<size_t>(ch + 2) * fv.chunk_bytes,
+            bulk_copy_g2s(buf, reinterpret_cast<const char*>(fv.chunks) + static_cast<size_t>(ch + kNBuf) * fv.chunk_bytes,
                           fv.chunk_bytes, bar);
           }
         }
