@@ -347,13 +347,40 @@ struct OMlp {
   const float* sigma;
 };
 
-// Model B with the standardisation folded in.
+// One-hot input of Model B (width 80): the columns of the feature row except the four
+// multi-level categorical fields, in ascending column order (positions 0..58), then one
+// indicator per level of operand type (column 5, 4 levels), activation (9, 3), kernel schedule
+// (17, 4) and epilogue schedule (18, 3) at positions 59..72, then zeros.
+constexpr int ROW_ONEHOT = 80;
+void onehot_row(const float* x, float* y) {
+  static const int kField[4] = {5, 9, 17, 18};
+  static const int kLevels[4] = {4, 3, 4, 3};
+  int p = 0;
+  for (int j = 0; j < NF; ++j)
+    if (j != 5 && j != 9 && j != 17 && j != 18) y[p++] = x[j];
+  for (int f = 0; f < 4; ++f)
+    for (int l = 0; l < kLevels[f]; ++l) y[p++] = (static_cast<int>(x[kField[f]]) == l) ? 1.0f : 0.0f;
+  while (p < ROW_ONEHOT) y[p++] = 0.0f;
+}
+
+// Model B with the standardisation folded in. Input width 64: the feature row as it is (ordinal
+// codes for the categorical fields); input width 80: its one-hot form.
 float score_mlp_row(const float* x, const OMlp& m) {
-  std::vector<float> cur(ROW), nxt;
-  for (int j = 0; j < ROW; ++j) {
+  const int in0 = m.widths[0];
+  float xin[ROW_ONEHOT];
+  int live;  // inputs that carry a value (the rest of the width is zero padding)
+  if (in0 == ROW_ONEHOT) {
+    onehot_row(x, xin);
+    live = 73;
+  } else {
+    for (int j = 0; j < ROW; ++j) xin[j] = x[j];
+    live = NF;
+  }
+  std::vector<float> cur(in0), nxt;
+  for (int j = 0; j < in0; ++j) {
     float v = 0.0f;
-    if (j < NF) {
-      v = x[j];
+    if (j < live) {
+      v = xin[j];
       if (!std::isfinite(v)) v = 0.0f;
       v = (v - m.mu[j]) / m.sigma[j];
     }

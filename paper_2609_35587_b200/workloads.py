@@ -294,6 +294,20 @@ def mlp_xavier(seed: int, widths, mu: np.ndarray, sigma: np.ndarray) -> dict:
             "sigma": np.ascontiguousarray(sigma, dtype=np.float32)}
 
 
+ONEHOT_WIDTH = 80
+ONEHOT_FIELDS = ((5, 4), (9, 3), (17, 4), (18, 3))   # (feature column, levels) expanded to indicators
+
+
+def onehot_stats(mu: np.ndarray, sigma: np.ndarray):
+    """Standardisation constants of the one-hot input layout from those of the 64-wide row: the
+    59 kept columns keep theirs (ascending column order), the 14 indicators and the padding
+    get mu = 0, sigma = 1."""
+    keep = [j for j in range(63) if j not in (5, 9, 17, 18)]
+    mu2, sg2 = np.zeros(ONEHOT_WIDTH, np.float32), np.ones(ONEHOT_WIDTH, np.float32)
+    mu2[:59], sg2[:59] = np.asarray(mu, np.float32)[keep], np.asarray(sigma, np.float32)[keep]
+    return mu2, sg2
+
+
 # ------------------------------------------------------------------------------------------
 # the five workloads
 # ------------------------------------------------------------------------------------------

@@ -308,3 +308,67 @@ def test_partition_ensemble_against_nested_ifs():
                 else:  # only leaf pairs can be swapped in place; undo the complement here
                     flipped["v"][i] = pnodes["v"][i]
     np.testing.assert_allclose(oracle.score_gbdt(x, off, flipped, base_score=0.25), got, rtol=1e-6, atol=1e-6)
+
+
+# ---------------------------------------------------------------------------------------------
+# one-hot input of the ranker (width 80)
+# ---------------------------------------------------------------------------------------------
+
+def onehot_numpy(x):
+    """The 80-wide input built with numpy indexing: kept columns, then np.eye rows per field."""
+    keep = [j for j in range(63) if j not in (5, 9, 17, 18)]
+    parts = [x[:, keep]]
+    for col, levels in wl.ONEHOT_FIELDS:
+        parts.append(np.eye(levels, dtype=np.float32)[x[:, col].astype(np.int64)])
+    y = np.concatenate(parts, axis=1)
+    return np.concatenate([y, np.zeros((len(x), 80 - y.shape[1]), np.float32)], axis=1)
+
+
+def test_onehot_mlp_matches_torch_linear_on_the_expanded_input():
+    prob, cand, _, _ = wl.make_inputs(2, P=3, seg=120)
+    x = oracle.featurize(prob, cand[:120], DESC)
+    st = wl.feature_stats("cfg2")
+    mu, sg = wl.onehot_stats(st["mu"], st["sigma"])
+    mlp = wl.mlp_xavier(21, [80, 128, 64, 1], mu, sg)
+    s = oracle.score_mlp(x, mlp)
+    y = onehot_numpy(x)
+    assert y.shape == (360, 80) and np.all(y[:, 59:73].sum(axis=1) == 4) and np.all(y[:, 73:] == 0)
+    h = (torch.from_numpy(y) - torch.from_numpy(mu)) / torch.from_numpy(sg)
+    h[:, 73:] = 0
+    h = h.to(torch.bfloat16).to(torch.float64)
+    L = len(mlp["weights"])
+    for l in range(L):
+        W = torch.from_numpy(bf16_bits_to_f32(mlp["weights"][l]).astype(np.float64))
+        h = torch.nn.functional.linear(h, W, torch.from_numpy(mlp["biases"][l].astype(np.float64)))
+        h = h.to(torch.float32)
+        if l < L - 1:
+            h = torch.relu(h).to(torch.bfloat16).to(torch.float64)
+    np.testing.assert_allclose(s, h[:, 0].numpy(), rtol=2e-6, atol=2e-6)
+
+
+def test_onehot_ridge_with_level_proportional_weights_equals_the_ordinal_ridge():
+    """A linear scorer whose indicator weights are level x w reproduces the ordinal-code scorer
+    (codes enter unscaled: mu = 0, sigma = 1), when level x w is exact in bf16."""
+    prob, cand, _, _ = wl.make_inputs(1, P=4, C=300)
+    x = oracle.featurize(prob, cand, DESC)
+    st = wl.feature_stats("cfg1")
+    mu, sg = st["mu"].copy(), st["sigma"].copy()
+    for col, _ in wl.ONEHOT_FIELDS:
+        mu[col], sg[col] = 0.0, 1.0
+    rng = np.random.default_rng(8)
+    w64 = (rng.integers(-8, 9, 64) / 16.0).astype(np.float32)      # few mantissa bits
+    w64[63] = 0
+    ordinal = {"widths": np.array([64, 1], np.int32), "weights": [wl.float_to_bf16_bits(w64).reshape(1, 64)],
+               "biases": [np.array([0.375], np.float32)], "mu": mu, "sigma": sg}
+    keep = [j for j in range(63) if j not in (5, 9, 17, 18)]
+    w80 = np.zeros(80, np.float32)
+    w80[:59] = w64[keep]
+    p = 59
+    for col, levels in wl.ONEHOT_FIELDS:
+        for l in range(levels):
+            w80[p] = l * w64[col]
+            p += 1
+    mu80, sg80 = wl.onehot_stats(mu, sg)
+    onehot = {"widths": np.array([80, 1], np.int32), "weights": [wl.float_to_bf16_bits(w80).reshape(1, 80)],
+              "biases": [np.array([0.375], np.float32)], "mu": mu80, "sigma": sg80}
+    np.testing.assert_allclose(oracle.score_mlp(x, onehot), oracle.score_mlp(x, ordinal), rtol=1e-6, atol=1e-6)
