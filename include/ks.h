@@ -31,6 +31,7 @@ extern "C" {
 
 #define KS_F 63          /* number of features (columns 0..62 of a feature row)            */
 #define KS_F_PAD 64      /* a feature row is 64 fp32; column 63 is always 0                */
+#define KS_F_ONEHOT 80   /* input width of the ranker's one-hot form */
 #define KS_MAX_K 32      /* largest k accepted by ks_select / ks_select_one                */
 #define KS_MAX_DEPTH 15  /* deepest tree accepted (a leaf index must fit 16 bits)          */
 #define KS_MAX_DIM (1u << 19) /* largest M, N or K for which all int64 products are exact  */
@@ -148,8 +149,13 @@ ks_status ks_model_create_gbdt(ks_ctx* ctx, int n_trees, const int64_t* h_tree_o
  * h_widths = {64, w_1, ..., w_{L-1}, 1} (n_layers = L weight matrices, 1 <= L <=
  * KS_MLP_MAX_LAYERS; hidden widths multiples of 64, <= KS_MLP_MAX_WIDTH). L = 1 is the linear
  * scorer w . x' + b of section "Linear Ridge Baseline". h_w_bf16[l] is
- * row-major [out, in] bf16 bit patterns, h_bias[l] is [out] fp32; h_mu / h_sigma are [64]
- * fp32 with sigma != 0. Synchronous. */
+ * row-major [out, in] bf16 bit patterns, h_bias[l] is [out] fp32; h_mu / h_sigma are
+ * [h_widths[0]] fp32 with sigma != 0. Synchronous.
+ * h_widths[0] = KS_F_ONEHOT selects the one-hot input form (section "Model B": categorical
+ * fields one-hot encoded): positions 0..58 are the feature columns other than 5, 9, 17, 18 in
+ * ascending order; 59..62, 63..65, 66..69, 70..72 are the level indicators (0 / 1) of operand
+ * type (column 5), activation (9), kernel schedule (17) and epilogue schedule (18); 73..79 are
+ * zero. mu / sigma apply position by position (indicators included). */
 ks_status ks_model_create_mlp(ks_ctx* ctx, int n_layers, const int* h_widths,
                               const uint16_t* const* h_w_bf16, const float* const* h_bias,
                               const float* h_mu, const float* h_sigma, ks_model** out_model);

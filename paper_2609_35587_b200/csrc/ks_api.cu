@@ -334,15 +334,16 @@ ks_status ks_model_create_mlp(ks_ctx* ctx, int n_layers, const int* h_widths,
   *out_model = nullptr;
   if (!ctx || !h_widths || !h_w_bf16 || !h_bias || !h_mu || !h_sigma) return KS_ERR_INVALID_ARG;
   if (n_layers < 1 || n_layers > KS_MLP_MAX_LAYERS) return KS_ERR_INVALID_ARG;
-  if (h_widths[0] != KS_F_PAD || h_widths[n_layers] != 1) return KS_ERR_INVALID_ARG;
-  int max_width = KS_F_PAD;
+  const int in0 = h_widths[0];
+  if ((in0 != KS_F_PAD && in0 != KS_F_ONEHOT) || h_widths[n_layers] != 1) return KS_ERR_INVALID_ARG;
+  int max_width = in0;
   for (int l = 1; l < n_layers; ++l) {
     if (h_widths[l] < 64 || h_widths[l] > KS_MLP_MAX_WIDTH || h_widths[l] % 64) return KS_ERR_INVALID_ARG;
     if (h_widths[l] > max_width) max_width = h_widths[l];
   }
   for (int l = 0; l < n_layers; ++l)
     if (!h_w_bf16[l] || !h_bias[l]) return KS_ERR_INVALID_ARG;
-  for (int j = 0; j < KS_F_PAD; ++j)
+  for (int j = 0; j < in0; ++j)
     if (!std::isfinite(h_mu[j]) || !std::isfinite(h_sigma[j]) || h_sigma[j] == 0.0f) return KS_ERR_INVALID_ARG;
 
   DeviceGuard g(ctx->device);
@@ -359,8 +360,8 @@ ks_status ks_model_create_mlp(ks_ctx* ctx, int n_layers, const int* h_widths,
     e = upload(&m->mlp.d_w[l], h_w_bf16[l], n);
     if (e == cudaSuccess) e = upload(&m->mlp.d_b[l], h_bias[l], static_cast<size_t>(h_widths[l + 1]));
   }
-  if (e == cudaSuccess) e = upload(&m->mlp.d_mu, h_mu, static_cast<size_t>(KS_F_PAD));
-  if (e == cudaSuccess) e = upload(&m->mlp.d_sigma, h_sigma, static_cast<size_t>(KS_F_PAD));
+  if (e == cudaSuccess) e = upload(&m->mlp.d_mu, h_mu, static_cast<size_t>(in0));
+  if (e == cudaSuccess) e = upload(&m->mlp.d_sigma, h_sigma, static_cast<size_t>(in0));
   if (e == cudaSuccess) e = ks::build_fast_mlp(m->mlp, h_w_bf16, h_bias, h_mu, h_sigma);
   if (e != cudaSuccess) {
     ks_status s = cuda_fail(ctx, e, "ks_model_create_mlp");

@@ -145,14 +145,31 @@ __device__ void mlp_tile(const MlpView& m, int max_width, const float* s_cols /*
   for (int grp = 0; grp < kGroups; ++grp) {
     __nv_bfloat16* cur = s_act;
     __nv_bfloat16* nxt = s_act + max_width * 32;
-    for (int col = g; col < kRow; col += kGroups) {
+    const bool onehot = m.widths[0] == KS_F_ONEHOT;
+    for (int pos = g; pos < m.widths[0]; pos += kGroups) {
       float v = 0.0f;
-      if (col < KS_F) {
-        v = s_cols[col * kBlock + grp * 32 + r];
-        if (!isfinite(v)) v = 0.0f;
-        v = __fdiv_rn(__fsub_rn(v, m.mu[col]), m.sigma[col]);
+      bool live;
+      if (!onehot) {
+        live = pos < KS_F;
+        if (live) v = s_cols[pos * kBlock + grp * 32 + r];
+      } else {
+        // one-hot form: the columns other than 5, 9, 17, 18 in order, then the level indicators
+        live = pos < 73;
+        if (pos < 59) {
+          const int col = pos + (pos >= 5) + (pos >= 8) + 2 * (pos >= 15);
+          v = s_cols[col * kBlock + grp * 32 + r];
+        } else if (live) {
+          const int q = pos - 59;  // operand type 0..3, activation 4..6, kernel sched 7..10, epilogue sched 11..13
+          const int col = q < 4 ? 5 : (q < 7 ? 9 : (q < 11 ? 17 : 18));
+          const int level = q < 4 ? q : (q < 7 ? q - 4 : (q < 11 ? q - 7 : q - 11));
+          v = __float2int_rz(s_cols[col * kBlock + grp * 32 + r]) == level ? 1.0f : 0.0f;
+        }
       }
-      cur[col * 32 + r] = __float2bfloat16_rn(v);
+      if (live) {
+        if (!isfinite(v)) v = 0.0f;
+        v = __fdiv_rn(__fsub_rn(v, m.mu[pos]), m.sigma[pos]);
+      }
+      cur[pos * 32 + r] = __float2bfloat16_rn(v);
     }
     __syncthreads();
     for (int l = 0; l < m.n_layers; ++l) {

@@ -577,3 +577,39 @@ def test_partition_split_ensembles(ks, ctx):
         with pytest.raises(ks.KsError) as ei:
             ctx.model_create_gbdt(*one(feat, mask, kind), 0.0)
         assert ei.value.status == ks.KS_ERR_INVALID_ARG
+
+
+# ---------------------------------------------------------------------------------------------
+# one-hot input form of the ranker
+# ---------------------------------------------------------------------------------------------
+
+def test_onehot_mlp(ks, ctx):
+    st = wl.feature_stats("cfg1")
+    mu, sg = wl.onehot_stats(st["mu"], st["sigma"])
+    prob, cand, _, _ = wl.make_inputs(1, P=4, C=900)
+    x = oracle.featurize(prob, cand, DESC)
+    for widths in ([80, 128, 64, 1], [80, 1], [80, 256, 256, 1]):
+        mlp = wl.mlp_xavier(13, widths, mu, sg)
+        model = ctx.model_create_mlp(mlp)
+        sc = ctx.score(dev(ks, x), model)
+        torch.cuda.synchronize()
+        rs = oracle.score_mlp(x, mlp)
+        assert np.all(np.abs(sc.cpu().numpy() - rs) <= 5e-3 * np.maximum(1, np.abs(rs))), widths
+        w = wl.Workload("onehot", DESC, prob, cand, 10, mlp=mlp)
+        idx, s2 = run_select(ks, ctx, w, model)
+        check_select(w, idx, s2, TOL_MLP)
+    # the one-hot form reads its own positions: indicator weights change the score
+    mlp = wl.mlp_xavier(13, [80, 1], mu, sg)
+    base = oracle.score_mlp(x, mlp)
+    w2 = {k: (v.copy() if isinstance(v, np.ndarray) else [a.copy() for a in v]) for k, v in mlp.items()}
+    w2["weights"][0][0, 66:70] = wl.float_to_bf16_bits(np.array([1.0, -1.0, 0.5, -0.5], np.float32))
+    m2 = ctx.model_create_mlp(w2)
+    got = ctx.score(dev(ks, x), m2).cpu().numpy()
+    ref = oracle.score_mlp(x, w2)
+    assert np.all(np.abs(got - ref) <= 5e-3 * np.maximum(1, np.abs(ref))) and not np.allclose(ref, base)
+    # invalid: another input width, or constants shorter than the width
+    bad = dict(mlp)
+    bad["widths"] = np.array([72, 1], np.int32)
+    bad["weights"] = [mlp["weights"][0][:, :72].copy()]
+    with pytest.raises(ks.KsError):
+        ctx.model_create_mlp(bad)
