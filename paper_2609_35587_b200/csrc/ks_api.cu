@@ -143,6 +143,7 @@ void free_model(ks_model* m) {
   cudaFree(m->mlp.d_sigma);
   cudaFree(m->mlp.d_tc_image);
   ks::free_fast_mlp(m->mlp);
+  ks::free_ridge(m->mlp);
   delete m;
 }
 
@@ -363,6 +364,7 @@ ks_status ks_model_create_mlp(ks_ctx* ctx, int n_layers, const int* h_widths,
   if (e == cudaSuccess) e = upload(&m->mlp.d_mu, h_mu, static_cast<size_t>(in0));
   if (e == cudaSuccess) e = upload(&m->mlp.d_sigma, h_sigma, static_cast<size_t>(in0));
   if (e == cudaSuccess) e = ks::build_fast_mlp(m->mlp, h_w_bf16, h_bias, h_mu, h_sigma);
+  if (e == cudaSuccess) e = ks::build_ridge(m->mlp, h_w_bf16[0], h_bias[0], h_mu, h_sigma);
   if (e != cudaSuccess) {
     ks_status s = cuda_fail(ctx, e, "ks_model_create_mlp");
     free_model(m);

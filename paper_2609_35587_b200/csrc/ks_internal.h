@@ -25,6 +25,15 @@ struct alignas(16) MlpTcParams {
   float b3;
 };
 
+// Linear scorer (one weight layer) in a form the fused ridge kernel consumes: per feature column
+// the weight and the standardisation, per expanded categorical field (one-hot input form) the
+// contribution of every level, and the bias. Passed by value at every launch.
+struct RidgeParams {
+  float w[64], mu[64], sigma[64];  // by feature column; w = 0 for a column that is expanded
+  float lut5[4], lut9[4], lut17[4], lut18[4];  // one-hot form: contribution of each level (else 0)
+  float bias;
+};
+
 // Generic device form of a tree node: 8 bytes, children tree-relative.
 struct DevNode {
   float v;        // threshold, or the leaf value
@@ -63,6 +72,8 @@ struct MlpModel {
   float* d_b[KS_MLP_MAX_LAYERS] = {nullptr};
   float* d_mu = nullptr;
   float* d_sigma = nullptr;
+  // one weight layer (the linear ridge scorer): fused kernel without a feature tile
+  RidgeParams* h_ridge = nullptr;
   // tensor-core path (shape 64-256-256-1 only), see ks_mlp_tc.cu
   bool tc = false;
   uint16_t* d_tc_image = nullptr;      // W1 and W2 in the shared-memory operand layout
@@ -173,6 +184,11 @@ int fast_slices(const GbdtModel& g, int64_t blocks);
 cudaError_t build_fast_mlp(MlpModel& m, const uint16_t* const* h_w, const float* const* h_b, const float* h_mu,
                            const float* h_sigma);
 void free_fast_mlp(MlpModel& m);
+// Linear scorer: fills m.h_ridge when the model has one weight layer.
+cudaError_t build_ridge(MlpModel& m, const uint16_t* h_w, const float* h_b, const float* h_mu,
+                        const float* h_sigma);
+void free_ridge(MlpModel& m);
+size_t ridge_scratch_bytes(int C);
 int mlp_tc_blocks_per_problem(int P, int64_t per_problem);
 size_t mlp_tc_scratch_bytes(int C);
 cudaError_t launch_select_mlp_tc(const ks_gpu_desc& desc, const MlpModel& m, const ks_problem* d_p,

@@ -4,6 +4,9 @@
 // in ks_gbdt_fast.cu.
 #include <cuda_bf16.h>
 
+#include <cstring>
+#include <new>
+
 #include "ks_features.cuh"
 #include "ks_internal.h"
 #include "ks_topk.cuh"
@@ -301,6 +304,117 @@ select_generic_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_pro
 }
 
 // ------------------------------------------------------------------------------------------
+// linear scorer (one weight layer): s = b + sum_j w_j * bf16((x_j - mu_j) / sigma_j). The sum
+// splits by what a column depends on: the candidate-only part is formed once per call and
+// candidate (per element-type combination), the problem-only part once per block, and only the
+// 21 per-pair columns are evaluated per pair, without a feature tile.
+// ------------------------------------------------------------------------------------------
+
+__device__ __forceinline__ float ridge_term(const RidgeParams& prm, int col, float v) {
+  if (!isfinite(v)) v = 0.0f;
+  const float x = __bfloat162float(__float2bfloat16_rn(__fdiv_rn(__fsub_rn(v, prm.mu[col]), prm.sigma[col])));
+  return prm.w[col] * x;
+}
+__device__ __forceinline__ float ridge_level(const float (&lut)[4], float v) {
+  const int code = __float2int_rz(v);
+  return (code >= 0 && code < 4) ? lut[code] : 0.0f;
+}
+
+// per (type combination, candidate): (candidate-only part of the sum, resident-block count)
+__global__ void __launch_bounds__(256)
+ridge_cand_kernel(ks_gpu_desc desc, const ks_candidate* __restrict__ c, int C, const unsigned* mask_ptr,
+                  unsigned mask_value, const __grid_constant__ RidgeParams prm, float2* __restrict__ out) {
+  const int combo = blockIdx.y;
+  const unsigned mask = mask_ptr ? *mask_ptr : mask_value;
+  if (!((mask >> combo) & 1u)) return;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= C) return;
+  ks_problem fake{};
+  fake.m = fake.n = fake.k = 1;
+  fake.dtype_ab = static_cast<uint8_t>(combo >> 2);
+  fake.dtype_d = static_cast<uint8_t>(combo & 3);
+  ProblemTerms t;
+  problem_terms(fake, desc, t);
+  const ks_candidate cand = c[i];
+  float s = 0.0f;
+  featurize_pair(t, cand, desc, [&](int col, float v) {
+    if (feat_class(col) != 1) return;
+    s += ridge_term(prm, col, v);
+    if (col == 17) s += ridge_level(prm.lut17, v);
+    if (col == 18) s += ridge_level(prm.lut18, v);
+  });
+  out[static_cast<size_t>(combo) * C + i] = make_float2(s, static_cast<float>(resources(t, cand, desc).b_eff));
+}
+
+__global__ void ridge_combo_mask_kernel(const ks_problem* __restrict__ p, int P, unsigned* __restrict__ mask) {
+  unsigned m = 0;
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < P; i += gridDim.x * blockDim.x)
+    m |= 1u << ((p[i].dtype_ab & 3) * 4 + (p[i].dtype_d & 3));
+  m = __reduce_or_sync(0xFFFFFFFFu, m);
+  if ((threadIdx.x & 31) == 0 && m) atomicOr(mask, m);
+}
+
+__global__ void __launch_bounds__(kBlock)
+select_ridge_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_problem p_value, int use_value,
+                    const ks_candidate* __restrict__ c, PairMap map, int sub_tiles,
+                    const float2* __restrict__ cand_tab, const __grid_constant__ RidgeParams prm, int k,
+                    unsigned long long* __restrict__ partial /* [P][nblk][k] */) {
+  __shared__ ProblemTerms s_pt;
+  __shared__ float s_prob;  // bias + problem-only part of the sum
+  __shared__ unsigned long long s_warp[kBlock / 32 * KS_MAX_K];
+  __shared__ unsigned long long s_list[KS_MAX_K];
+  const int prob = blockIdx.x / map.nblk, chunk = blockIdx.x % map.nblk;
+  int64_t lo, len;
+  segment_of(map, prob, lo, len);
+  if (threadIdx.x == 0) {
+    problem_terms(use_value ? p_value : p[prob], desc, s_pt);
+    ks_candidate dummy{};
+    dummy.tile_m = dummy.tile_n = dummy.tile_k = 64;
+    dummy.stages = dummy.cluster_m = dummy.cluster_n = 1;
+    float s = prm.bias;
+    featurize_pair(s_pt, dummy, desc, [&](int col, float v) {
+      if (feat_class(col) != 0) return;
+      s += ridge_term(prm, col, v);
+      if (col == 5) s += ridge_level(prm.lut5, v);
+      if (col == 9) s += ridge_level(prm.lut9, v);
+    });
+    s_prob = s;
+  }
+  if (threadIdx.x < KS_MAX_K) s_list[threadIdx.x] = 0ull;
+  __syncthreads();
+  const float2* tab = cand_tab + static_cast<size_t>(s_pt.dtype_ab * 4 + s_pt.dtype_d) * map.C;
+
+  const int64_t pass_rows = static_cast<int64_t>(sub_tiles) * kBlock;
+  for (int64_t start = static_cast<int64_t>(chunk) * pass_rows; start < len;
+       start += static_cast<int64_t>(map.nblk) * pass_rows) {
+    unsigned long long keys[kSubTilesMax + 1];
+#pragma unroll
+    for (int s = 0; s <= kSubTilesMax; ++s) keys[s] = 0ull;
+    if (threadIdx.x < k) keys[kSubTilesMax] = s_list[threadIdx.x];
+#pragma unroll 1
+    for (int s = 0; s < sub_tiles; ++s) {
+      const int64_t r = start + static_cast<int64_t>(s) * kBlock + threadIdx.x;
+      unsigned long long key = 0ull;
+      if (r < len) {
+        const int idx = pool_index(map, lo, r);
+        const ks_candidate cand = c[idx];
+        const float2 t = __ldg(tab + idx);
+        float pair = 0.0f;
+        pair_columns<true>(s_pt, cand, desc, static_cast<long long>(t.y),
+                           [&](int col, float v) { pair += ridge_term(prm, col, v); });
+        key = make_key(((s_prob + t.x) + pair) + 0.0f, idx);
+      }
+#pragma unroll
+      for (int q = 0; q < kSubTilesMax; ++q)
+        if (q == s) keys[q] = key;
+    }
+    block_topk<kSubTilesMax + 1>(keys, k, s_warp, s_list);
+  }
+  if (threadIdx.x < k)
+    partial[(static_cast<size_t>(prob) * map.nblk + chunk) * k + threadIdx.x] = s_list[threadIdx.x];
+}
+
+// ------------------------------------------------------------------------------------------
 // merge: one warp per problem ranks the nblk * k partial keys
 // ------------------------------------------------------------------------------------------
 
@@ -403,6 +517,70 @@ cudaError_t launch_score_mlp(const MlpModel& m, const float* d_feat, int64_t row
   return cudaGetLastError();
 }
 
+static float bf16_bits_host(uint16_t b) {
+  const uint32_t u = static_cast<uint32_t>(b) << 16;
+  float f;
+  std::memcpy(&f, &u, 4);
+  return f;
+}
+static float round_bf16_host(float v) {
+  uint32_t u;
+  std::memcpy(&u, &v, 4);
+  if ((u & 0x7F800000u) == 0x7F800000u) return v;
+  u += 0x7FFFu + ((u >> 16) & 1u);
+  u &= 0xFFFF0000u;
+  std::memcpy(&v, &u, 4);
+  return v;
+}
+
+cudaError_t build_ridge(MlpModel& m, const uint16_t* h_w, const float* h_b, const float* h_mu,
+                        const float* h_sigma) {
+  if (m.n_layers != 1) return cudaSuccess;
+  RidgeParams* r = new (std::nothrow) RidgeParams();
+  if (!r) return cudaErrorMemoryAllocation;
+  std::memset(r, 0, sizeof(*r));
+  for (int j = 0; j < 64; ++j) r->sigma[j] = 1.0f;
+  r->bias = h_b[0];
+  if (m.widths[0] == KS_F_PAD) {
+    for (int j = 0; j < KS_F; ++j) {
+      r->w[j] = bf16_bits_host(h_w[j]);
+      r->mu[j] = h_mu[j];
+      r->sigma[j] = h_sigma[j];
+    }
+  } else {  // one-hot form: kept columns in ascending order, then the level indicators
+    int pos = 0;
+    for (int j = 0; j < KS_F; ++j) {
+      if (j == 5 || j == 9 || j == 17 || j == 18) continue;
+      r->w[j] = bf16_bits_host(h_w[pos]);
+      r->mu[j] = h_mu[pos];
+      r->sigma[j] = h_sigma[pos];
+      ++pos;
+    }
+    float* luts[4] = {r->lut5, r->lut9, r->lut17, r->lut18};
+    const int levels[4] = {4, 3, 4, 3};
+    for (int f = 0; f < 4; ++f) {
+      for (int lv = 0; lv < levels[f]; ++lv) {  // the field is at level lv: one indicator is 1
+        float s = 0.0f;
+        for (int q = 0; q < levels[f]; ++q) {
+          const float x = round_bf16_host(((q == lv ? 1.0f : 0.0f) - h_mu[pos + q]) / h_sigma[pos + q]);
+          s += bf16_bits_host(h_w[pos + q]) * x;
+        }
+        luts[f][lv] = s;
+      }
+      pos += levels[f];
+    }
+  }
+  m.h_ridge = r;
+  return cudaSuccess;
+}
+
+void free_ridge(MlpModel& m) {
+  delete m.h_ridge;
+  m.h_ridge = nullptr;
+}
+
+size_t ridge_scratch_bytes(int C) { return 256 + sizeof(float2) * 16 * static_cast<size_t>(C); }
+
 static int pick_sub_tiles(int P, int64_t per_problem) {
   for (int s = kSubTilesMax; s > 1; s >>= 1) {
     const int64_t nblk = (per_problem + static_cast<int64_t>(s) * kBlock - 1) / (static_cast<int64_t>(s) * kBlock);
@@ -433,7 +611,9 @@ size_t select_partial_bytes(const ks_model& model, int P, int C, int64_t pairs, 
   const int st = pick_sub_tiles(P, per);
   int64_t nblk = (per + static_cast<int64_t>(st) * kBlock - 1) / (static_cast<int64_t>(st) * kBlock);
   if (nblk < 1) nblk = 1;
-  return static_cast<size_t>(P) * nblk * k * sizeof(unsigned long long);
+  const size_t part = static_cast<size_t>(P) * nblk * k * sizeof(unsigned long long);
+  if (model.kind == 1 && model.mlp.h_ridge) return (part + 255) / 256 * 256 + ridge_scratch_bytes(C);
+  return part;
 }
 
 cudaError_t launch_select(const ks_gpu_desc& desc, const ks_model& model, const ks_problem* d_p,
@@ -490,6 +670,37 @@ cudaError_t launch_select(const ks_gpu_desc& desc, const ks_model& model, const 
   ks_problem pv{};
   if (p_by_value) pv = *p_by_value;
   cudaError_t e;
+  if (model.kind == 1 && model.mlp.h_ridge) {
+    // linear scorer: per-call table of candidate-only sums, then the fused kernel
+    const size_t part_bytes = (static_cast<size_t>(P) * map.nblk * k * sizeof(unsigned long long) + 255) / 256 * 256;
+    unsigned* d_mask = reinterpret_cast<unsigned*>(static_cast<char*>(d_partial) + part_bytes);
+    float2* d_tab = reinterpret_cast<float2*>(static_cast<char*>(d_partial) + part_bytes + 256);
+    unsigned mask_value = 0;
+    if (p_by_value) {
+      mask_value = 1u << ((pv.dtype_ab & 3) * 4 + (pv.dtype_d & 3));
+    } else {
+      e = cudaMemsetAsync(d_mask, 0, sizeof(unsigned), stream);
+      if (e != cudaSuccess) return e;
+      ridge_combo_mask_kernel<<<P >= 4096 ? 16 : 1, 256, 0, stream>>>(d_p, P, d_mask);
+      ++*launches;
+    }
+    if (C > 0) {
+      ridge_cand_kernel<<<dim3((C + 255) / 256, 16), 256, 0, stream>>>(desc, d_c, C, p_by_value ? nullptr : d_mask,
+                                                                      mask_value, *model.mlp.h_ridge, d_tab);
+      ++*launches;
+    }
+    if (ev_begin) cudaEventRecord(ev_begin, stream);
+    select_ridge_kernel<<<grid, kBlock, 0, stream>>>(desc, d_p, pv, p_by_value != nullptr, d_c, map, st, d_tab,
+                                                     *model.mlp.h_ridge, k, partial);
+    ++*launches;
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    if (ev_end) cudaEventRecord(ev_end, stream);
+    topk_merge_kernel<<<(P * 32 + kBlock - 1) / kBlock, kBlock, 0, stream>>>(partial, P, map.nblk * k, k,
+                                                                            d_topk_idx, d_topk_score);
+    ++*launches;
+    return cudaGetLastError();
+  }
   if (ev_begin) cudaEventRecord(ev_begin, stream);
   if (model.kind == 2) {
     select_generic_kernel<2><<<grid, kBlock, 0, stream>>>(desc, d_p, pv, p_by_value != nullptr, d_c, map, st, nullptr,

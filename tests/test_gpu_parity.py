@@ -442,8 +442,25 @@ def test_select_ridge_and_paper_sized_models(ks, ctx):
     prob, cand, _, _ = wl.make_inputs(1, P=3, C=900)
     ridge = wl.mlp_xavier(21, [64, 1], st["mu"], st["sigma"])
     w = wl.Workload("ridge", DESC, prob, cand, 10, mlp=ridge)
-    idx, sc = run_select(ks, ctx, w, ctx.model_create_mlp(ridge))
+    rmodel = ctx.model_create_mlp(ridge)
+    idx, sc = run_select(ks, ctx, w, rmodel)
     check_select(w, idx, sc, TOL_MLP)
+    # the fused linear kernel evaluates exact features: only the order of the sum differs
+    ridx, rsc = oracle.select(prob, cand, DESC, 10, mlp=ridge)
+    assert np.array_equal(idx, ridx) and np.all(np.abs(sc - rsc) <= 1e-4 * np.maximum(1, np.abs(rsc)))
+    hi, hs = ctx.select_one(prob[1:2], dev(ks, cand), len(cand), rmodel, 10)
+    assert np.array_equal(hi.numpy(), ridx[1])
+    hi, hs = ctx.select_host(prob, 3, cand, len(cand), rmodel, 10)
+    assert np.array_equal(hi.numpy(), ridx)
+    # mixed element types and per-problem segments, ordinal and one-hot form
+    w2 = wl.make_workload(2, P=9, seg=2500, trees=4, depth=2)
+    for form in (64, 80):
+        mu, sg = (st["mu"], st["sigma"]) if form == 64 else wl.onehot_stats(st["mu"], st["sigma"])
+        r2 = wl.mlp_xavier(5, [form, 1], mu, sg)
+        wr = wl.Workload("ridge_seg", DESC, w2.problems, w2.candidates, 10, seg_offsets=w2.seg_offsets,
+                         seg_index=w2.seg_index, mlp=r2)
+        idx2, sc2 = run_select(ks, ctx, wr, ctx.model_create_mlp(r2))
+        check_select(wr, idx2, sc2, 1e-4)
     big = wl.mlp_xavier(22, [64, 1024, 1024, 512, 256, 1], st["mu"], st["sigma"])
     w = wl.Workload("mlp_big", DESC, prob[:1], cand[:200], 10, mlp=big)
     idx, sc = run_select(ks, ctx, w, ctx.model_create_mlp(big))
