@@ -153,7 +153,7 @@ def test_valid_counts_against_the_papers_table():
     # totals: within 1 % of the paper's (its epilogue-footprint estimator is not printed)
     for lay in range(4):
         assert abs(n[lay] - PAPER_COUNTS[lay]) <= 0.01 * PAPER_COUNTS[lay], (lay, n[lay])
-    # "around 11.36 %" of the space survives
+    # the surviving share of the space is close to the paper's 11.36 %
     assert abs(sum(n.values()) / (4 * 534600) - 0.1136) < 0.002
     # the problem's dimensions do not enter without the wasteful-tile flag
     c2, idx2 = oracle.valid_catalogue(bf16(TN_, 64, 64, 64), DESC, COUPLED, dtype=DT)
