@@ -142,6 +142,7 @@ void free_model(ks_model* m) {
   cudaFree(m->mlp.d_mu);
   cudaFree(m->mlp.d_sigma);
   cudaFree(m->mlp.d_tc_image);
+  cudaFree(m->mlp.d_w1_prob);
   ks::free_fast_mlp(m->mlp);
   ks::free_ridge(m->mlp);
   delete m;

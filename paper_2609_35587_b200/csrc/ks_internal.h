@@ -23,6 +23,12 @@ struct alignas(16) MlpTcParams {
   float scale[64], shift[64];
   float b1[256], b2[256], w3[256];
   float b3;
+  // one-hot input form: the problem-only inputs (11 columns + 7 level indicators) are folded
+  // into a per-CTA bias, the 7 candidate-side level indicators are formed from the record
+  int onehot;
+  uint16_t ind0[8], ind1[8];           // bf16 of an indicator's standardised value when 0 / 1 (kernel sched 0..3, epilogue sched 0..2)
+  float p_scale[18], p_shift[18];      // standardisation of the folded inputs
+  const float* w1_prob;                // device, [18][256]: first-layer weights of the folded inputs
 };
 
 // Linear scorer (one weight layer) in a form the fused ridge kernel consumes: per feature column
@@ -77,6 +83,7 @@ struct MlpModel {
   // tensor-core path (shape 64-256-256-1 only), see ks_mlp_tc.cu
   bool tc = false;
   uint16_t* d_tc_image = nullptr;      // W1 and W2 in the shared-memory operand layout
+  float* d_w1_prob = nullptr;          // one-hot form: first-layer weights of the folded inputs
   MlpTcParams* h_tc_params = nullptr;  // host copy, passed by value at every launch
 };
 

@@ -67,6 +67,31 @@ __host__ __device__ constexpr int kpos(int col) {
   return base + pos;
 }
 
+// One-hot input form: the candidate-only columns other than kernel / epilogue schedule at 0..26,
+// the per-pair columns where they always are (29..49), the seven schedule-level indicators at
+// 50..56; everything else is zero. The problem-only inputs do not enter the MMA (-1): they are
+// folded into a per-CTA bias.
+__host__ __device__ constexpr int kpos_oh(int col) {
+  const int cls = feat_class(col);
+  if (cls == 0 || col == 17 || col == 18) return -1;
+  if (cls == 2) return kpos(col);
+  int pos = 0;
+  for (int c = 0; c < col; ++c)
+    if (feat_class(c) == 1 && c != 17 && c != 18) ++pos;
+  return pos;
+}
+constexpr int kIndPos = 50;  // K position of the first level indicator
+// the folded inputs in order: problem-only columns other than operand type (5) and activation (9),
+// then the four operand-type indicators, then the three activation indicators
+__host__ __device__ constexpr int kfold(int col) {
+  if (feat_class(col) != 0 || col == 5 || col == 9) return -1;
+  int pos = 0;
+  for (int c = 0; c < col; ++c)
+    if (feat_class(c) == 0 && c != 5 && c != 9) ++pos;
+  return pos;
+}
+constexpr int kFoldCols = 11, kFold = 18;
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
@@ -183,11 +208,19 @@ mlp_cand_cols_kernel(ks_gpu_desc desc, const ks_candidate* __restrict__ c, int C
 #pragma unroll
   for (int q = 0; q < 32; ++q) x[q] = 0.0f;
   const ks_candidate cand = c[i];
-  featurize_pair(t, cand, desc, [&](int col, float v) {
-    if (feat_class(col) != 1) return;
-    const int k = kpos(col);
-    x[k] = fmaf(v, prm.scale[k], prm.shift[k]);
-  });
+  if (prm.onehot) {
+    featurize_pair(t, cand, desc, [&](int col, float v) {
+      if (feat_class(col) != 1 || col == 17 || col == 18) return;
+      const int k = kpos_oh(col);
+      x[k] = fmaf(v, prm.scale[k], prm.shift[k]);
+    });
+  } else {
+    featurize_pair(t, cand, desc, [&](int col, float v) {
+      if (feat_class(col) != 1) return;
+      const int k = kpos(col);
+      x[k] = fmaf(v, prm.scale[k], prm.shift[k]);
+    });
+  }
   uint32_t w[16];
 #pragma unroll
   for (int q = 0; q < 16; ++q) w[q] = pack_bf16(x[2 * q], x[2 * q + 1]);
@@ -257,8 +290,11 @@ __device__ __forceinline__ unsigned long long const2(const float* p) {  // two c
 
 // E1: h1 = bf16(relu(acc + b1)) for the 256 columns of this thread's row, written as A-operand
 // planes. The TMEM load of the next 32 columns is in flight while the current ones are processed.
-template <int H>
-__device__ __forceinline__ void epilogue1(uint32_t tmem_row, uint32_t sA_row, const MlpTcParams& prm) {
+// kSmemBias: the bias comes from shared memory (per-CTA vector of the one-hot form) instead of the
+// constant bank.
+template <int H, bool kSmemBias>
+__device__ __forceinline__ void epilogue1(uint32_t tmem_row, uint32_t sA_row, const MlpTcParams& prm,
+                                          const float* s_b1) {
   uint32_t ra[32], rb[32];
   tmem_ld32_issue(tmem_row + H * 128, ra);
 #pragma unroll
@@ -274,7 +310,8 @@ __device__ __forceinline__ void epilogue1(uint32_t tmem_row, uint32_t sA_row, co
       for (int q = 0; q < 4; ++q) {
         const int j = H * 128 + blk * 32 + g * 8 + 2 * q;
         float lo, hi;
-        unpack2(add2(pack2(cur[g * 8 + 2 * q], cur[g * 8 + 2 * q + 1]), const2(&prm.b1[j])), lo, hi);
+        unpack2(add2(pack2(cur[g * 8 + 2 * q], cur[g * 8 + 2 * q + 1]), const2(kSmemBias ? &s_b1[j] : &prm.b1[j])),
+                lo, hi);
         w[q] = pack_bf16_relu(lo, hi);
       }
       const int plane = (H * 128 + blk * 32 + g * 8) / 8;
@@ -325,6 +362,7 @@ __device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 128;" :::
 // the kernel
 // ------------------------------------------------------------------------------------------
 
+template <bool kOneHot>  // input form: ordinal codes (K positions as kpos) or one-hot (kpos_oh + folded bias)
 __global__ void __launch_bounds__(kT, 1)
 select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_problem p_value, int use_value,
                      const ks_candidate* __restrict__ c, int P, int C, int nblk,
@@ -339,7 +377,11 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
   __shared__ __align__(8) unsigned long long s_bar[10];
   __shared__ uint32_t s_tmem;
   __shared__ uint32_t s_pwords[7];   // problem-only columns (positions 50..63) as packed bf16
-  __shared__ unsigned long long s_merge[4][32];  // the second-epilogue warps' final lists
+  // the second-epilogue warps' final lists; until they are written (after the last tile) the
+  // same kilobyte holds the per-CTA first-layer bias of the one-hot form
+  __shared__ __align__(16) unsigned long long s_merge[4][32];
+  float* s_b1 = reinterpret_cast<float*>(&s_merge[0][0]);
+  __shared__ float s_xp[kFold];  // one-hot form: the folded inputs, standardised and rounded to bf16
   __shared__ int s_fail, s_abort;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -381,6 +423,19 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
     });
 #pragma unroll
     for (int q = 0; q < 7; ++q) s_pwords[q] = pack_bf16(pv[2 * q], q == 6 ? 0.0f : pv[2 * q + 1]);
+    if (kOneHot) {
+      featurize_pair(s_pt, dummy, desc, [&](int col, float v) {
+        const int q = kfold(col);
+        if (q < 0) return;
+        s_xp[q] = __bfloat162float(__float2bfloat16_rn(fmaf(v, prm.p_scale[q], prm.p_shift[q])));
+      });
+      for (int l = 0; l < 4; ++l)
+        s_xp[kFoldCols + l] = __bfloat162float(__float2bfloat16_rn(
+            fmaf(s_pt.dtype_ab == l ? 1.0f : 0.0f, prm.p_scale[kFoldCols + l], prm.p_shift[kFoldCols + l])));
+      for (int l = 0; l < 3; ++l)
+        s_xp[kFoldCols + 4 + l] = __bfloat162float(__float2bfloat16_rn(
+            fmaf(s_pt.act == l ? 1.0f : 0.0f, prm.p_scale[kFoldCols + 4 + l], prm.p_shift[kFoldCols + 4 + l])));
+    }
     mbar_init(bar_w, 1);
     mbar_init(bar_a0, 1);
     mbar_init(bar_a1, 1);
@@ -399,7 +454,6 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
     for (int off = 0; off < kW1Bytes + kW2Bytes; off += 32768)
       bulk_copy_g2s(sbase + kOffW1 + off, w_image + off, 32768, bar_w);
   }
-  if (tid < 128) s_merge[tid >> 5][tid & 31] = 0ull;
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(512)
                  : "memory");
@@ -410,6 +464,14 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
   tc_fence_after();
   const uint32_t tmem = s_tmem;
   const uint32_t sA = sbase + kOffA;
+  if (kOneHot) {  // per-CTA bias: b1 + the folded problem-only inputs through their weights
+    if (tid < kH) {
+      float acc = prm.b1[tid];
+      for (int q = 0; q < kFold; ++q) acc = fmaf(__ldg(prm.w1_prob + q * kH + tid), s_xp[q], acc);
+      s_b1[tid] = acc;
+    }
+    __syncthreads();
+  }
   const int combo = s_pt.dtype_ab * 4 + s_pt.dtype_d;
   bool failed = false;
   // Bounded wait. After the first one that runs out, every later wait of the CTA gives up after a
@@ -474,7 +536,7 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
         }
         float x[64];
         auto put = [&](int col, float v) {
-          const int kk = kpos(col);
+          const int kk = kpos(col);  // the per-pair columns sit at the same positions in both forms
           x[kk] = fmaf(v, prm.scale[kk], prm.shift[kk]);
         };
         // single-precision evaluation (the values are rounded to bf16 next); the exact
@@ -485,8 +547,18 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
         w[14] = (w[14] & 0xFFFFu) | (pack_bf16(0.0f, x[29]) & 0xFFFF0000u);
 #pragma unroll
         for (int q = 15; q < 25; ++q) w[q] = pack_bf16(x[2 * q], x[2 * q + 1]);
+        if (kOneHot) {
+          // positions 50..56: the level indicators of kernel schedule (4) and epilogue schedule (3)
+          const unsigned ks = cand.kernel_sched, es = cand.epi_sched;
+          auto ind = [&](int q, bool on) { return static_cast<uint32_t>(on ? prm.ind1[q] : prm.ind0[q]); };
+          w[25] = ind(0, ks == 0) | (ind(1, ks == 1) << 16);
+          w[26] = ind(2, ks == 2) | (ind(3, ks == 3) << 16);
+          w[27] = ind(4, es == 0) | (ind(5, es == 1) << 16);
+          w[28] = ind(6, es == 2);
+        } else {
 #pragma unroll
-        for (int q = 0; q < 7; ++q) w[25 + q] = s_pwords[q];
+          for (int q = 0; q < 7; ++q) w[25 + q] = s_pwords[q];
+        }
       }
       if (tile > 0) {  // planes 0..7 are free once the first group of L2(tile - 1) is done
         if (!wait_ok(bar_a_prev, ph_a)) failed = true;
@@ -536,7 +608,8 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
         if (!wait_ok(bar_c, ph_c)) failed = true;  // L1(tile) is complete
         ph_c ^= 1;
         tc_fence_after();
-        epilogue1<0>(acc_row, sA + trow * 16, prm);
+        if (kOneHot) epilogue1<0, true>(acc_row, sA + trow * 16, prm, s_b1);
+        else epilogue1<0, false>(acc_row, sA + trow * 16, prm, s_b1);
         fence_async_proxy();
         tc_fence_before();
         epi_sync();
@@ -615,40 +688,84 @@ static float bf16_bits_to_float_host(uint16_t b) {
 cudaError_t build_fast_mlp(MlpModel& m, const uint16_t* const* h_w, const float* const* h_b, const float* h_mu,
                            const float* h_sigma) {
   m.tc = false;
-  if (m.n_layers != 3 || m.widths[0] != 64 || m.widths[1] != kH || m.widths[2] != kH || m.widths[3] != 1)
+  const int in0 = m.widths[0];
+  if (m.n_layers != 3 || (in0 != KS_F_PAD && in0 != KS_F_ONEHOT) || m.widths[1] != kH || m.widths[2] != kH ||
+      m.widths[3] != 1)
     return cudaSuccess;  // other shapes stay on the generic kernel
-  // column order along K and the folded standardisation x' = x * scale + shift
-  int col_at[64];
-  for (int q = 0; q < 64; ++q) col_at[q] = -1;
-  for (int col = 0; col < KS_F; ++col) col_at[kpos(col)] = col;
+  const bool onehot = in0 == KS_F_ONEHOT;
+  // source of every K position: the model's input position that feeds it (-1: zero), and the
+  // folded standardisation x' = x * scale + shift
+  int src_at[64];
+  for (int q = 0; q < 64; ++q) src_at[q] = -1;
+  int oh_pos[KS_F];  // one-hot form: input position of every kept feature column
+  {
+    int pos = 0;
+    for (int col = 0; col < KS_F; ++col) oh_pos[col] = (col == 5 || col == 9 || col == 17 || col == 18) ? -1 : pos++;
+  }
+  if (!onehot) {
+    for (int col = 0; col < KS_F; ++col) src_at[kpos(col)] = col;
+  } else {
+    for (int col = 0; col < KS_F; ++col)
+      if (kpos_oh(col) >= 0) src_at[kpos_oh(col)] = oh_pos[col];
+    for (int q = 0; q < 7; ++q) src_at[kIndPos + q] = 66 + q;  // kernel schedule 66..69, epilogue schedule 70..72
+  }
   MlpTcParams* prm = new (std::nothrow) MlpTcParams();
   if (!prm) return cudaErrorMemoryAllocation;
-  for (int kk = 0; kk < 64; ++kk) {
-    prm->scale[kk] = 0.0f;
-    prm->shift[kk] = 0.0f;
-    if (col_at[kk] >= 0) {
-      const double s = 1.0 / static_cast<double>(h_sigma[col_at[kk]]);
-      prm->scale[kk] = static_cast<float>(s);
-      prm->shift[kk] = static_cast<float>(-static_cast<double>(h_mu[col_at[kk]]) * s);
-    }
-  }
+  std::memset(prm, 0, sizeof(*prm));
+  auto fold = [&](int src, float& scale, float& shift) {
+    const double s = 1.0 / static_cast<double>(h_sigma[src]);
+    scale = static_cast<float>(s);
+    shift = static_cast<float>(-static_cast<double>(h_mu[src]) * s);
+  };
+  for (int kk = 0; kk < 64; ++kk)
+    if (src_at[kk] >= 0) fold(src_at[kk], prm->scale[kk], prm->shift[kk]);
   for (int j = 0; j < kH; ++j) {
     prm->b1[j] = h_b[0][j];
     prm->b2[j] = h_b[1][j];
     prm->w3[j] = bf16_bits_to_float_host(h_w[2][j]);
   }
   prm->b3 = h_b[2][0];
+  prm->onehot = onehot ? 1 : 0;
+  std::vector<float> w1p;
+  if (onehot) {
+    auto bf16_of = [](float v) {
+      const __nv_bfloat16 b = __float2bfloat16_rn(v);
+      uint16_t u;
+      std::memcpy(&u, &b, 2);
+      return u;
+    };
+    for (int q = 0; q < 7; ++q) {
+      prm->ind0[q] = bf16_of(fmaf(0.0f, prm->scale[kIndPos + q], prm->shift[kIndPos + q]));
+      prm->ind1[q] = bf16_of(fmaf(1.0f, prm->scale[kIndPos + q], prm->shift[kIndPos + q]));
+    }
+    // the folded inputs: their input positions, standardisation and first-layer weights
+    int fold_src[kFold];
+    for (int col = 0; col < KS_F; ++col)
+      if (kfold(col) >= 0) fold_src[kfold(col)] = oh_pos[col];
+    for (int l = 0; l < 7; ++l) fold_src[kFoldCols + l] = 59 + l;  // operand type 59..62, activation 63..65
+    w1p.resize(static_cast<size_t>(kFold) * kH);
+    for (int q = 0; q < kFold; ++q) {
+      fold(fold_src[q], prm->p_scale[q], prm->p_shift[q]);
+      for (int n = 0; n < kH; ++n)
+        w1p[static_cast<size_t>(q) * kH + n] = bf16_bits_to_float_host(h_w[0][static_cast<size_t>(n) * in0 + fold_src[q]]);
+    }
+  }
   // operand images: plane (k / 8), 16 bytes per output unit
   std::vector<uint16_t> img((kW1Bytes + kW2Bytes) / 2, 0);
   for (int n = 0; n < kH; ++n)
     for (int kk = 0; kk < 64; ++kk)
-      if (col_at[kk] >= 0)
-        img[(kk / 8) * (kPlaneB / 2) + n * 8 + (kk % 8)] = h_w[0][static_cast<size_t>(n) * 64 + col_at[kk]];
+      if (src_at[kk] >= 0)
+        img[(kk / 8) * (kPlaneB / 2) + n * 8 + (kk % 8)] = h_w[0][static_cast<size_t>(n) * in0 + src_at[kk]];
   uint16_t* w2 = img.data() + kW1Bytes / 2;
   for (int n = 0; n < kH; ++n)
     for (int kk = 0; kk < kH; ++kk) w2[(kk / 8) * (kPlaneB / 2) + n * 8 + (kk % 8)] = h_w[1][static_cast<size_t>(n) * kH + kk];
   cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&m.d_tc_image), img.size() * 2);
   if (e == cudaSuccess) e = cudaMemcpy(m.d_tc_image, img.data(), img.size() * 2, cudaMemcpyHostToDevice);
+  if (e == cudaSuccess && onehot) {
+    e = cudaMalloc(reinterpret_cast<void**>(&m.d_w1_prob), w1p.size() * sizeof(float));
+    if (e == cudaSuccess) e = cudaMemcpy(m.d_w1_prob, w1p.data(), w1p.size() * sizeof(float), cudaMemcpyHostToDevice);
+    prm->w1_prob = m.d_w1_prob;
+  }
   if (e != cudaSuccess) {
     delete prm;
     return e;
@@ -705,11 +822,19 @@ cudaError_t launch_select_mlp_tc(const ks_gpu_desc& desc, const MlpModel& m, con
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (ev_begin) cudaEventRecord(ev_begin, stream);
-  e = cudaFuncSetAttribute(select_mlp_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-  if (e != cudaSuccess) return e;
-  select_mlp_tc_kernel<<<static_cast<unsigned>(static_cast<int64_t>(P) * nblk), kT, kSmemBytes, stream>>>(
-      desc, d_p, pv, uv, d_c, P, C, nblk, seg_off, seg_idx, reinterpret_cast<const uint8_t*>(m.d_tc_image), d_cols, k,
-      partial, status, *m.h_tc_params);
+  const unsigned grid = static_cast<unsigned>(static_cast<int64_t>(P) * nblk);
+  const uint8_t* image = reinterpret_cast<const uint8_t*>(m.d_tc_image);
+  if (m.h_tc_params->onehot) {
+    e = cudaFuncSetAttribute(select_mlp_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    select_mlp_tc_kernel<true><<<grid, kT, kSmemBytes, stream>>>(desc, d_p, pv, uv, d_c, P, C, nblk, seg_off, seg_idx,
+                                                                 image, d_cols, k, partial, status, *m.h_tc_params);
+  } else {
+    e = cudaFuncSetAttribute(select_mlp_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    select_mlp_tc_kernel<false><<<grid, kT, kSmemBytes, stream>>>(desc, d_p, pv, uv, d_c, P, C, nblk, seg_off, seg_idx,
+                                                                  image, d_cols, k, partial, status, *m.h_tc_params);
+  }
   ++*launches;
   return cudaGetLastError();
 }

@@ -615,6 +615,24 @@ def test_onehot_mlp(ks, ctx):
         w = wl.Workload("onehot", DESC, prob, cand, 10, mlp=mlp)
         idx, s2 = run_select(ks, ctx, w, model)
         check_select(w, idx, s2, TOL_MLP)
+    # the 80-256-256-1 shape runs on the tensor-core kernel (problem-only inputs folded into a
+    # per-CTA bias): every score, on problems of mixed element types and epilogues
+    mlp = wl.mlp_xavier(17, [80, 256, 256, 1], mu, sg)
+    model = ctx.model_create_mlp(mlp)
+    prob2, cand2, _, _ = wl.make_inputs(2, P=12, seg=100)
+    assert len(set(prob2["dtype_ab"].tolist())) > 1 and len(set((prob2["epi_flags"] >> 1).tolist())) > 1
+    for C in (129, 4500):
+        idx, s2 = ctx.select(dev(ks, prob2), 12, dev(ks, cand2[:C]), C, model, 32)
+        torch.cuda.synchronize()
+        idx, s2 = idx.cpu().numpy(), s2.cpu().numpy()
+        _, _, allsc = oracle.select(prob2, cand2[:C], DESC, 32, mlp=mlp, want_scores=True)
+        for i in range(12):
+            ref = allsc[i * C:(i + 1) * C]
+            assert len(set(idx[i].tolist())) == 32 and idx[i].min() >= 0 and idx[i].max() < C
+            err = np.abs(s2[i] - ref[idx[i]]) / np.maximum(1, np.abs(ref[idx[i]]))
+            assert err.max() < 5e-3, (C, i, err.max())
+            ok, msg = topk_accept(idx[i], s2[i], ref, np.arange(C, dtype=np.int32), 32, TOL_MLP)
+            assert ok, msg
     # the one-hot form reads its own positions: indicator weights change the score
     mlp = wl.mlp_xavier(13, [80, 1], mu, sg)
     base = oracle.score_mlp(x, mlp)
