@@ -253,6 +253,26 @@ def test_select_mlp(ks, ctx):
     check_select(w, idx, sc, TOL_MLP)
 
 
+def test_select_mlp_segments_and_uneven_sizes(ks, ctx):
+    """The tensor-core kernel on per-problem segments (uneven, one empty), and on sizes around
+    its 4,096-row blocks, where CTAs of one problem walk different numbers of tiles."""
+    w = wl.make_workload(2, P=6, seg=5000, trees=4, depth=2)
+    w.mlp = wl.make_workload(4, P=1, C=16).mlp
+    w.gbdt = None
+    w.seg_offsets = np.array([0, 4097, 4097, 9000, 9001, 17193, 21500], np.int64)
+    w.seg_index = np.concatenate([np.sort(np.random.default_rng(i).choice(len(w.candidates), n, replace=False))
+                                  for i, n in enumerate(np.diff(w.seg_offsets))]).astype(np.int32)
+    model = ctx.model_create_mlp(w.mlp)
+    idx, sc = run_select(ks, ctx, w, model)
+    assert np.all(idx[1] == -1) and np.all(np.isneginf(sc[1]))
+    assert idx[3, 0] == w.seg_index[9000] and np.all(idx[3, 1:] == -1)
+    check_select(w, idx, sc, TOL_MLP)
+    for C in (4095, 4096, 4097, 8193):
+        wd = wl.make_workload(4, P=2, C=C)
+        idx, sc = run_select(ks, ctx, wd, ctx.model_create_mlp(wd.mlp))
+        check_select(wd, idx, sc, TOL_MLP)
+
+
 def test_select_mlp_every_score(ks, ctx):
     """k >= |segment| returns every pair's score: each one against the oracle, on sizes that
     cross the 128-row tile and the 2,048-row block of the tensor-core kernel."""
