@@ -1,6 +1,7 @@
 // Host side of the C ABI: argument checks, model validation and repacking, workspace
 // management, launches. No exception or abort crosses the boundary.
 #include <cmath>
+#include <mutex>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -58,6 +59,36 @@ ks_status ensure_workspace(ks_ctx* ctx, size_t bytes) {
   ctx->ws_bytes = want;
   return KS_OK;
 }
+
+}  // namespace
+
+namespace ks {
+cudaError_t ensure_dynamic_smem(const void* kernel, size_t bytes) {
+  struct Entry {
+    const void* kernel;
+    int device;
+    size_t bytes;
+  };
+  static Entry table[64];
+  static int used = 0;
+  static std::mutex mu;
+  int device = 0;
+  cudaError_t e = cudaGetDevice(&device);
+  if (e != cudaSuccess) return e;
+  std::lock_guard<std::mutex> lock(mu);
+  Entry* hit = nullptr;
+  for (int i = 0; i < used; ++i)
+    if (table[i].kernel == kernel && table[i].device == device) hit = &table[i];
+  if (hit && hit->bytes >= bytes) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes));
+  if (e != cudaSuccess) return e;
+  if (hit) hit->bytes = bytes;
+  else if (used < 64) table[used++] = Entry{kernel, device, bytes};
+  return cudaSuccess;
+}
+}  // namespace ks
+
+namespace {
 
 // Reads (and clears) the device status word; the stream must have been synchronised.
 ks_status read_status(ks_ctx* ctx) {
@@ -193,7 +224,7 @@ ks_status ks_create(ks_ctx** out_ctx, int cuda_device, const ks_gpu_desc* desc) 
   if (!ctx) return KS_ERR_OOM;
   ctx->device = cuda_device;
   ctx->desc = *desc;
-  ctx->pinned_bytes = KS_MAX_K * (sizeof(int32_t) + sizeof(float));
+  ctx->pinned_bytes = KS_MAX_K * (sizeof(int32_t) + sizeof(float)) + 64;  // results + the sequence word
   // result staging of ks_select_one: mapped pinned memory, so the kernel's last block can
   // write the k results where the host reads them, with no copy in between
   void* d_pin = nullptr;
@@ -204,6 +235,7 @@ ks_status ks_create(ks_ctx** out_ctx, int cuda_device, const ks_gpu_desc* desc) 
     delete ctx;
     return KS_ERR_OOM;
   }
+  std::memset(ctx->pinned, 0, ctx->pinned_bytes);
   ctx->d_pinned_idx = static_cast<int32_t*>(d_pin);
   ctx->d_pinned_score = reinterpret_cast<float*>(ctx->d_pinned_idx + KS_MAX_K);
   if (cudaMalloc(reinterpret_cast<void**>(&ctx->d_counters), sizeof(int) * (ks::kMaxSliceBlocks + 1)) != cudaSuccess ||
@@ -520,10 +552,20 @@ ks_status ks_select_one(ks_ctx* ctx, ks_problem p, const ks_candidate* d_c, int 
       sl.out_idx = ctx->d_pinned_idx;
       sl.out_score = ctx->d_pinned_score;
       sl.tiles = reinterpret_cast<uint8_t*>(base + b_part);
+      // the kernel stores this call's sequence number after the results; polling that word
+      // returns a few microseconds before the stream reports completion
+      int* h_seq = reinterpret_cast<int*>(pin_sc + KS_MAX_K);
+      sl.out_seq = reinterpret_cast<int*>(ctx->d_pinned_score + KS_MAX_K);
+      sl.seq = ++ctx->select_one_seq;
       cudaError_t e = ks::launch_select_fast(ctx->desc, model->gbdt, nullptr, &p, 1, d_c, C, nblk, ks::kFastRows,
                                              nullptr, nullptr, k, reinterpret_cast<unsigned long long*>(base),
                                              base + b_part, ctx->d_status, st, &ctx->launches, nullptr, &sl);
-      if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+      if (e == cudaSuccess) {
+        bool seen = false;
+        for (int spin = 0; spin < (1 << 22) && !seen; ++spin) seen = *static_cast<volatile int*>(h_seq) == sl.seq;
+        // not seen within a few milliseconds (a failed launch never writes it): wait the regular way
+        if (!seen) e = cudaStreamSynchronize(st);
+      }
       if (e != cudaSuccess) return cuda_fail(ctx, e, "ks_select_one");
       s = read_status(ctx);
       if (s != KS_OK) {

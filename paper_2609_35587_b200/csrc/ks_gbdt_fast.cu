@@ -148,6 +148,8 @@ struct SliceArgs {
   int32_t* out_idx;        // single-problem form only: [k] final result (device-visible, may be
   float* out_score;        // mapped host memory); null when a merge kernel follows
   const uint8_t* tiles;    // prepared tiles [blocks][rows][kRowStride] (tile_one_kernel), or null
+  int* out_seq;            // single-problem form: receives `seq` once the k results are written
+  int seq;
 };
 
 struct FastView {
@@ -393,15 +395,18 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
   const int ch_end = static_cast<int>(static_cast<int64_t>(fv.n_chunks) * (slice + 1) / S);
   const uint32_t sbase = smem_u32(smem);
   const uint32_t bar0 = smem_u32(&s_bar[0]);  // barrier of buffer b: bar0 + 8 b
+  const bool tiles_given = sl.tiles != nullptr;  // the tiles were built in front: no feature work here
   if (tid == 0) {
-    problem_terms(use_value ? p_value : p[prob], desc, s_pt);
-    // problem-only columns do not look at the candidate: evaluate them on a dummy one
-    ks_candidate dummy{};
-    dummy.tile_m = dummy.tile_n = dummy.tile_k = 64;
-    dummy.stages = dummy.cluster_m = dummy.cluster_n = 1;
-    featurize_pair(s_pt, dummy, desc, [&](int col, float v) {
-      if (feat_class(col) == 0) s_pfeat[col] = v;
-    });
+    if (!tiles_given) {
+      problem_terms(use_value ? p_value : p[prob], desc, s_pt);
+      // problem-only columns do not look at the candidate: evaluate them on a dummy one
+      ks_candidate dummy{};
+      dummy.tile_m = dummy.tile_n = dummy.tile_k = 64;
+      dummy.stages = dummy.cluster_m = dummy.cluster_n = 1;
+      featurize_pair(s_pt, dummy, desc, [&](int col, float v) {
+        if (feat_class(col) == 0) s_pfeat[col] = v;
+      });
+    }
     for (int b = 0; b < kNBuf; ++b) mbar_init(bar0 + 8u * b, 1);
     s_fail = 0;
     for (int b = 0; b < kNBuf; ++b) s_done[b] = 0;
@@ -413,7 +418,7 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
   }
   if (tid < KS_MAX_K) s_list[tid] = 0ull;
   __syncthreads();
-  if (tid < KS_F && feat_class(tid) == 0) {
+  if (!tiles_given && tid < KS_F && feat_class(tid) == 0) {
     const int first = fv.n_pair_rows + fv.n_cand_rows;
     for (int q = 0; q < s_rowcnt[tid]; ++q)
       s_pbin[s_row0[tid] + q - first] =
@@ -618,7 +623,13 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
         prev = best;
       }
     }
-    if (tid == 0) sl.counters[nblk] = 0;
+    if (tid == 0) {
+      sl.counters[nblk] = 0;
+      if (sl.out_seq) {  // the results are in place: tell the host, which polls this word
+        __threadfence_system();
+        *reinterpret_cast<volatile int*>(sl.out_seq) = sl.seq;
+      }
+    }
   }
 }
 
@@ -869,8 +880,7 @@ static cudaError_t launch_ln(const ks_gpu_desc& desc, const ks_problem* d_p, con
                              const int32_t* seg_idx, const FastView& fv, int k, unsigned long long* partial,
                              int* status, const SliceArgs& sl, const FastTopParams& top, cudaStream_t stream) {
   const size_t smem = kOffTile + static_cast<size_t>(fv.n_rows) * kRowStride;
-  cudaError_t e = cudaFuncSetAttribute(select_fast_kernel<L, NP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       static_cast<int>(smem));
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(&select_fast_kernel<L, NP>), smem);
   if (e != cudaSuccess) return e;
   select_fast_kernel<L, NP><<<static_cast<unsigned>(static_cast<int64_t>(P) * nblk * sl.n_slices), kFastThreads, smem,
                               stream>>>(desc, d_p, pv, uv, d_c, P, C, nblk, rows_per_cta, seg_off, seg_idx, fv, k,
@@ -920,7 +930,7 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
   if (tiles_mode) {
     // one launch, two roles (blockIdx.y): the per-pair rows, and the candidate- / problem-only rows
     const size_t tthr = sizeof(float) * kThrPerRow * g.n_qrows;
-    e = cudaFuncSetAttribute(tile_one_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(tthr));
+    e = ensure_dynamic_smem(reinterpret_cast<const void*>(&tile_one_kernel), tthr);
     if (e != cudaSuccess) return e;
     tile_one_kernel<<<dim3(nblk * (kFastRows / 256), 2), 256, tthr, stream>>>(desc, pv, d_c, C, fv, slice->tiles);
     ++*launches;
@@ -944,6 +954,8 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
     sl.out_idx = slice->out_idx;
     sl.out_score = slice->out_score;
     sl.tiles = tiles_mode ? slice->tiles : nullptr;
+    sl.out_seq = slice->out_seq;
+    sl.seq = slice->seq;
   }
   const FastTopParams& top = *g.h_top;
   const int L = g.top_levels, np = g.fast_depth - L;

@@ -112,6 +112,7 @@ struct ks_ctx {
   int* h_status = nullptr;  // status word (mapped pinned host memory) set by kernels whose
   int* d_status = nullptr;  // bounded waits give up; d_status is its device alias
   int64_t launches = 0;
+  int select_one_seq = 0;  // sequence number of the last single-problem call
   char err[256] = {0};
   // optional timing of the dominant kernel of the last ks_select* call (ks_profile_enable)
   bool profile = false;
@@ -149,6 +150,10 @@ inline int categorical_levels(int col) {
   }
 }
 
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) costs a driver call; remembers, per kernel and
+// device, the largest size already granted (ks_api.cu).
+cudaError_t ensure_dynamic_smem(const void* kernel, size_t bytes);
+
 // Builds the quantised fast form of a validated ensemble when it qualifies (m.fast).
 cudaError_t build_fast_gbdt(GbdtModel& m, int n_trees, const int64_t* h_tree_offsets,
                             const ks_node_host* h_nodes);
@@ -162,6 +167,8 @@ struct FastSlice {
   int32_t* out_idx;  // single-problem form: [k], device-visible; else null (a merge kernel follows)
   float* out_score;
   uint8_t* tiles;    // single-problem form: scratch for the prepared tiles [blocks][rows][kFastRows], or null
+  int* out_seq;      // single-problem form: device-visible word that receives `seq` after the results
+  int seq;
 };
 
 // Search-space enumeration and validity filtering (ks_catalogue.cu).

@@ -465,8 +465,7 @@ cudaError_t launch_featurize(const ks_gpu_desc& desc, const ks_problem* d_p, int
   if (P == 0 || pairs == 0) return cudaSuccess;
   const PairMap map = make_map(P, C, pairs, d_seg_off, d_seg_idx, kBlock);
   const size_t smem = sizeof(float) * kBlock * 65;
-  cudaError_t e = cudaFuncSetAttribute(featurize_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       static_cast<int>(smem));
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(&featurize_kernel), smem);
   if (e != cudaSuccess) return e;
   featurize_kernel<<<static_cast<unsigned>(static_cast<int64_t>(P) * map.nblk), kBlock, smem, stream>>>(
       desc, d_p, d_c, map, d_out);
@@ -478,8 +477,7 @@ cudaError_t launch_score_gbdt(const GbdtModel& m, const float* d_feat, int64_t r
                               uint16_t* d_leaf_idx, cudaStream_t stream, int64_t* launches) {
   if (rows == 0) return cudaSuccess;
   const size_t smem = sizeof(float) * kRow * kBlock;
-  cudaError_t e = cudaFuncSetAttribute(score_gbdt_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       static_cast<int>(smem));
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(&score_gbdt_kernel), smem);
   if (e != cudaSuccess) return e;
   score_gbdt_kernel<<<static_cast<unsigned>((rows + kBlock - 1) / kBlock), kBlock, smem, stream>>>(
       m.d_nodes, m.d_roots, m.n_trees, m.base, d_feat, rows, d_scores, d_leaf_idx);
@@ -508,8 +506,7 @@ cudaError_t launch_score_mlp(const MlpModel& m, const float* d_feat, int64_t row
                              cudaStream_t stream, int64_t* launches) {
   if (rows == 0) return cudaSuccess;
   const size_t smem = mlp_smem_bytes(m.max_width);
-  cudaError_t e = cudaFuncSetAttribute(score_mlp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       static_cast<int>(smem));
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(&score_mlp_kernel), smem);
   if (e != cudaSuccess) return e;
   score_mlp_kernel<<<static_cast<unsigned>((rows + kBlock - 1) / kBlock), kBlock, smem, stream>>>(
       make_view(m), m.max_width, d_feat, rows, d_scores);
@@ -708,16 +705,14 @@ cudaError_t launch_select(const ks_gpu_desc& desc, const ks_model& model, const 
   } else if (model.kind == 0) {
     const GbdtModel& g = model.gbdt;
     const size_t smem = sizeof(float) * kRow * kBlock;
-    e = cudaFuncSetAttribute(select_generic_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             static_cast<int>(smem));
+    e = ensure_dynamic_smem(reinterpret_cast<const void*>(&select_generic_kernel<0>), smem);
     if (e != cudaSuccess) return e;
     select_generic_kernel<0><<<grid, kBlock, smem, stream>>>(
         desc, d_p, pv, p_by_value != nullptr, d_c, map, st, g.d_nodes, g.d_roots, g.n_trees, g.base,
         MlpView{}, 0, k, partial);
   } else {
     const size_t smem = mlp_smem_bytes(model.mlp.max_width);
-    e = cudaFuncSetAttribute(select_generic_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             static_cast<int>(smem));
+    e = ensure_dynamic_smem(reinterpret_cast<const void*>(&select_generic_kernel<1>), smem);
     if (e != cudaSuccess) return e;
     select_generic_kernel<1><<<grid, kBlock, smem, stream>>>(
         desc, d_p, pv, p_by_value != nullptr, d_c, map, st, nullptr, nullptr, 0, 0.0f,
@@ -748,8 +743,7 @@ cudaError_t launch_select_generic_trees(const ks_gpu_desc& desc, const DevNode* 
   const int st = pick_sub_tiles(P, C);
   const PairMap map = make_map(P, C, static_cast<int64_t>(P) * C, nullptr, nullptr, st * kBlock);
   const size_t smem = sizeof(float) * kRow * kBlock;
-  cudaError_t e = cudaFuncSetAttribute(select_generic_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       static_cast<int>(smem));
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(&select_generic_kernel<0>), smem);
   if (e != cudaSuccess) return e;
   select_generic_kernel<0><<<static_cast<unsigned>(static_cast<int64_t>(P) * map.nblk), kBlock, smem, stream>>>(
       desc, d_p, ks_problem{}, 0, d_c, map, st, d_nodes, d_roots, n_trees, base, MlpView{}, 0, k, partial);

@@ -825,12 +825,12 @@ cudaError_t launch_select_mlp_tc(const ks_gpu_desc& desc, const MlpModel& m, con
   const unsigned grid = static_cast<unsigned>(static_cast<int64_t>(P) * nblk);
   const uint8_t* image = reinterpret_cast<const uint8_t*>(m.d_tc_image);
   if (m.h_tc_params->onehot) {
-    e = cudaFuncSetAttribute(select_mlp_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    e = ensure_dynamic_smem(reinterpret_cast<const void*>(&select_mlp_tc_kernel<true>), kSmemBytes);
     if (e != cudaSuccess) return e;
     select_mlp_tc_kernel<true><<<grid, kT, kSmemBytes, stream>>>(desc, d_p, pv, uv, d_c, P, C, nblk, seg_off, seg_idx,
                                                                  image, d_cols, k, partial, status, *m.h_tc_params);
   } else {
-    e = cudaFuncSetAttribute(select_mlp_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    e = ensure_dynamic_smem(reinterpret_cast<const void*>(&select_mlp_tc_kernel<false>), kSmemBytes);
     if (e != cudaSuccess) return e;
     select_mlp_tc_kernel<false><<<grid, kT, kSmemBytes, stream>>>(desc, d_p, pv, uv, d_c, P, C, nblk, seg_off, seg_idx,
                                                                   image, d_cols, k, partial, status, *m.h_tc_params);
