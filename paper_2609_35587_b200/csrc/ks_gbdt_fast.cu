@@ -29,9 +29,8 @@
 //            bounded waits). Thread (w, h) owns the four candidates of word w and walks the
 //            trees of half h of every chunk. The top levels are evaluated for all four
 //            candidates at once, node by node, with byte-parallel arithmetic on whole words;
-//            below that each candidate follows its own path, its node address kept in a float
-//            register as a denormal (bit pattern == integer), where a*2+c is exact, so the
-//            address update runs on the FMA pipe;
+//            below that each candidate follows its own path: a' = 2 a + k0 (+ 4 to go right), a
+//            multiply-add plus a predicated add;
 //   phase C  add the two halves' partial scores, rank the block's keys, write a partial
 //            top-k list.
 #include <algorithm>
@@ -336,9 +335,10 @@ __device__ __forceinline__ uint32_t byte_select(uint32_t m, uint32_t a, uint32_t
   return (a & f) | (b & ~f);
 }
 
-// one path step of one walk: fetch the node, fetch the candidate's byte, move to the child
-__device__ __forceinline__ float path_step(float a, uint32_t cb_r, float K0f, float four) {
-  float nx;
+// one path step of one walk: fetch the node, fetch the candidate's byte, move to the child:
+// next = 2 a + k0 (+ 4 when the candidate goes right)
+__device__ __forceinline__ uint32_t path_step(uint32_t a, uint32_t cb_r, uint32_t k0) {
+  uint32_t nx;
   asm volatile(
       "{\n"
       " .reg .u32 n, x, m;\n"
@@ -349,11 +349,11 @@ __device__ __forceinline__ float path_step(float a, uint32_t cb_r, float K0f, fl
       " ld.shared.u8 x, [m];\n"
       " and.b32 n, n, 255;\n"
       " setp.gt.u32 p, x, n;\n"
-      " fma.rn.f32 %0, %3, 0f40000000, %4;\n"
-      " @p add.rn.f32 %0, %0, %5;\n"
+      " mad.lo.u32 %0, %1, 2, %3;\n"
+      " @p add.u32 %0, %0, 4;\n"
       "}\n"
-      : "=f"(nx)
-      : "r"(__float_as_uint(a)), "r"(cb_r), "f"(a), "f"(K0f), "f"(four));
+      : "=r"(nx)
+      : "r"(a), "r"(cb_r), "r"(k0));
   return nx;
 }
 
@@ -482,17 +482,14 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
       const uint32_t buf = sbase + kOffBuf0 + b * kBufBytes;
       // With A_l the shared address of a walk's node at level l, A_{l+1} = 2 A_l + (4 tpc - buf)
       // + 4 bit for every level, and after the last level A points at the walk's leaf.
-      const int k0 = static_cast<int>(4u * tpc) - static_cast<int>(buf);
-      const float K0f = k0 >= 0 ? __uint_as_float(static_cast<uint32_t>(k0))
-                                : -__uint_as_float(static_cast<uint32_t>(-k0));
-      const float four = __uint_as_float(4u);
+      const uint32_t k0 = 4u * tpc - buf;  // modulo 2^32, like the additions it enters
       const uint32_t lvlL = buf + 4u * tpc * kTop;  // first node of level L
 #pragma unroll 1
       for (int t = half * half_trees; t < (half + 1) * half_trees; ++t) {
-        float a[4];
+        uint32_t a[4];
         if (L == 0) {
 #pragma unroll
-          for (int r = 0; r < 4; ++r) a[r] = __uint_as_float(buf + 4u * t);
+          for (int r = 0; r < 4; ++r) a[r] = buf + 4u * t;
         } else {
           // Word-wise evaluation of the top L levels for the four candidates of this word.
           // A tile byte is 0x80 | bin and a node constant (j + 1) in every byte, so byte r of
@@ -517,21 +514,21 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
           const uint32_t y = x >> (6 - L);
           const uint32_t tbase = lvlL + (static_cast<uint32_t>(t) << (L + 2));
 #pragma unroll
-          for (int r = 0; r < 4; ++r) a[r] = __uint_as_float(tbase + __byte_perm(y, 0u, 0x4440u + r));
+          for (int r = 0; r < 4; ++r) a[r] = tbase + __byte_perm(y, 0u, 0x4440u + r);
         }
         if (NP >= 0) {
 #pragma unroll
           for (int l = 0; l < (NP >= 0 ? NP : 0); ++l)
 #pragma unroll
-            for (int r = 0; r < 4; ++r) a[r] = path_step(a[r], cb + r, K0f, four);
+            for (int r = 0; r < 4; ++r) a[r] = path_step(a[r], cb + r, k0);
         } else {
 #pragma unroll 1
           for (int l = 0; l < np; ++l)
 #pragma unroll
-            for (int r = 0; r < 4; ++r) a[r] = path_step(a[r], cb + r, K0f, four);
+            for (int r = 0; r < 4; ++r) a[r] = path_step(a[r], cb + r, k0);
         }
 #pragma unroll
-        for (int r = 0; r < 4; ++r) score[r] += lds_f32(__float_as_uint(a[r]));
+        for (int r = 0; r < 4; ++r) score[r] += lds_f32(a[r]);
       }
       // Release the buffer without a block-wide barrier: every warp counts itself out, and the
       // last one to leave refills the buffer (nobody waits; warps may run a chunk ahead).
