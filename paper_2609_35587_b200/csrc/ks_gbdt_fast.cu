@@ -962,6 +962,8 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
   if (L == 3 && np == 5) KS_GO(3, 5);
   if (L == 3 && np == 3) KS_GO(3, 3);
   if (L == 2 && np == 6) KS_GO(2, 6);
+  if (L == 2 && np == 5) KS_GO(2, 5);  // the paper-sized ensemble: 916 trees of depth 7
+  if (L == 3 && np == 4) KS_GO(3, 4);
   if (L == 3) KS_GO(3, -1);
   if (L == 2) KS_GO(2, -1);
   if (L == 1) KS_GO(1, -1);
