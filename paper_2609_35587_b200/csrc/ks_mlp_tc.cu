@@ -685,14 +685,37 @@ static float bf16_bits_to_float_host(uint16_t b) {
   return f;
 }
 
-cudaError_t build_fast_mlp(MlpModel& m, const uint16_t* const* h_w, const float* const* h_b, const float* h_mu,
-                           const float* h_sigma) {
+cudaError_t build_fast_mlp(MlpModel& m, const uint16_t* const* h_w_in, const float* const* h_b_in,
+                           const float* h_mu, const float* h_sigma) {
   m.tc = false;
   const int in0 = m.widths[0];
-  if (m.n_layers != 3 || (in0 != KS_F_PAD && in0 != KS_F_ONEHOT) || m.widths[1] != kH || m.widths[2] != kH ||
-      m.widths[3] != 1)
-    return cudaSuccess;  // other shapes stay on the generic kernel
+  // One or two hidden layers of at most kH units each: narrower layers are padded with units
+  // whose weights and bias are zero (they stay zero through ReLU and contribute nothing), and a
+  // single hidden layer gets an identity second layer (its activations are non-negative bf16
+  // values, which ReLU and the rounding leave unchanged). Other shapes stay on the generic kernel.
+  if ((m.n_layers != 2 && m.n_layers != 3) || (in0 != KS_F_PAD && in0 != KS_F_ONEHOT)) return cudaSuccess;
+  for (int l = 1; l < m.n_layers; ++l)
+    if (m.widths[l] > kH) return cudaSuccess;
   const bool onehot = in0 == KS_F_ONEHOT;
+  const int h1 = m.widths[1], h2 = m.n_layers == 3 ? m.widths[2] : m.widths[1];
+  std::vector<uint16_t> pw1(static_cast<size_t>(kH) * in0, 0), pw2(static_cast<size_t>(kH) * kH, 0), pw3(kH, 0);
+  std::vector<float> pb1(kH, 0.0f), pb2(kH, 0.0f);
+  for (int n = 0; n < h1; ++n) {
+    std::memcpy(&pw1[static_cast<size_t>(n) * in0], &h_w_in[0][static_cast<size_t>(n) * in0], sizeof(uint16_t) * in0);
+    pb1[n] = h_b_in[0][n];
+  }
+  if (m.n_layers == 3) {
+    for (int n = 0; n < h2; ++n) {
+      for (int kk = 0; kk < h1; ++kk) pw2[static_cast<size_t>(n) * kH + kk] = h_w_in[1][static_cast<size_t>(n) * h1 + kk];
+      pb2[n] = h_b_in[1][n];
+    }
+  } else {
+    for (int n = 0; n < h1; ++n) pw2[static_cast<size_t>(n) * kH + n] = 0x3F80;  // bf16 1.0
+  }
+  for (int n = 0; n < h2; ++n) pw3[n] = h_w_in[m.n_layers - 1][n];
+  const uint16_t* h_w[3] = {pw1.data(), pw2.data(), pw3.data()};
+  const float b3v = h_b_in[m.n_layers - 1][0];
+  const float* h_b[3] = {pb1.data(), pb2.data(), &b3v};
   // source of every K position: the model's input position that feeds it (-1: zero), and the
   // folded standardisation x' = x * scale + shift
   int src_at[64];

@@ -298,11 +298,21 @@ def test_select_mlp_every_score(ks, ctx):
         ref = allsc[i * 4500:(i + 1) * 4500]
         err = np.abs(sc[i] - ref[idx[i]]) / np.maximum(1, np.abs(ref[idx[i]]))
         assert err.max() < 5e-3
-    # a second MLP shape stays on the generic kernel
-    m2 = wl.mlp_xavier(11, [64, 128, 64, 1], w.mlp["mu"], w.mlp["sigma"])
-    w2 = wl.Workload("mlp2", DESC, w.problems, w.candidates[:300], 10, mlp=m2)
-    idx, sc = run_select(ks, ctx, w2, ctx.model_create_mlp(m2))
-    check_select(w2, idx, sc, TOL_MLP)
+    # narrower layers and a single hidden layer run on the same kernel, padded with zero units
+    # (and an identity second layer); three hidden layers stay on the general kernel
+    st = wl.feature_stats("cfg1")
+    ohm, ohs = wl.onehot_stats(st["mu"], st["sigma"])
+    for widths in ([64, 128, 64, 1], [64, 64, 1], [64, 256, 128, 1], [80, 192, 1], [80, 64, 256, 1], [64, 128, 128, 64, 1]):
+        mu, sg = (w.mlp["mu"], w.mlp["sigma"]) if widths[0] == 64 else (ohm, ohs)
+        m2 = wl.mlp_xavier(11, widths, mu, sg)
+        w2 = wl.Workload("mlp2", DESC, w.problems, w.candidates[:300], 32, mlp=m2)
+        idx, sc = run_select(ks, ctx, w2, ctx.model_create_mlp(m2))
+        check_select(w2, idx, sc, TOL_MLP)
+        _, _, allsc = oracle.select(w2.problems, w2.candidates, DESC, 32, mlp=m2, want_scores=True)
+        for i in range(2):
+            ref = allsc[i * 300:(i + 1) * 300]
+            err = np.abs(sc[i] - ref[idx[i]]) / np.maximum(1, np.abs(ref[idx[i]]))
+            assert err.max() < 5e-3, (widths, err.max())
 
 
 def test_select_one_and_select_host_agree_with_select(ks, ctx):
