@@ -136,7 +136,6 @@ constexpr int kFastR = 2;              // candidates per thread there
 constexpr int kFastRows = kFastThreads * kFastR;
 constexpr int kFastMaxDepth = 10;
 constexpr int kMlpThreads = 512;        // threads per block of the tensor-core MLP kernel
-constexpr int kMlpRows = 4096;          // candidates one block ranks per pass
 constexpr int kMaxSliceBlocks = 1024;  // candidate blocks the slice mode supports
 
 // Levels of the categorical field held by feature column `col` (0: not a level-code column):

@@ -40,7 +40,6 @@ namespace {
 
 constexpr int kT = kMlpThreads;
 constexpr int kTileRows = 128;
-constexpr int kTiles = kMlpRows / kTileRows;
 constexpr int kH = 256;                               // hidden width
 constexpr int kW1Bytes = kH * 64 * 2;                 // 32 KB
 constexpr int kW2Bytes = kH * kH * 2;                 // 128 KB
@@ -491,17 +490,12 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
   // the barriers of alternating tiles come in pairs.
   uint32_t ph_a = 0, ph_b[2] = {0, 0}, ph_c = 0, ph_x = 0, ph_f = 0;
 
-  // This CTA's tiles: blocks of kMlpRows rows at a stride of nblk blocks; every block but the last
-  // one is full. The tile pipeline runs through all of them without draining in between.
-  int total_tiles = 0;
-  for (int64_t start = static_cast<int64_t>(chunk) * kMlpRows; start < len; start += static_cast<int64_t>(nblk) * kMlpRows) {
-    const int64_t rows_left = len - start;
-    total_tiles += static_cast<int>(rows_left >= kMlpRows ? kTiles : (rows_left + kTileRows - 1) / kTileRows);
-  }
-  auto tile_row0 = [&](int tile) {
-    return (static_cast<int64_t>(chunk) + static_cast<int64_t>(tile / kTiles) * nblk) * kMlpRows +
-           static_cast<int64_t>(tile % kTiles) * kTileRows;
-  };
+  // This CTA's tiles: an equal share (to within one) of the problem's 128-row tiles, contiguous.
+  // The tile pipeline runs through all of them without draining in between.
+  const int64_t problem_tiles = (len + kTileRows - 1) / kTileRows;
+  const int64_t tile_first = problem_tiles * chunk / nblk;
+  const int total_tiles = static_cast<int>(problem_tiles * (chunk + 1) / nblk - tile_first);
+  auto tile_row0 = [&](int tile) { return (tile_first + tile) * kTileRows; };
   unsigned long long top = 0ull;  // second-epilogue warps: lane j holds the warp's j-th best key
 
   // Roles (tile t uses accumulator t & 1):
@@ -803,16 +797,15 @@ void free_fast_mlp(MlpModel& m) {
   m.h_tc_params = nullptr;
 }
 
-// CTAs per problem. A CTA's set-up (160 KB of weights, TMEM, problem terms) is worth several
-// passes of kMlpRows candidates, so with enough problems to fill the GPU each CTA takes up to
-// four passes (the kernel strides over its problem's blocks).
+// CTAs per problem. A CTA's set-up (160 KB of weights, TMEM, problem terms) is worth about 128
+// tiles; with few problems the tiles are spread over one CTA per SM instead.
 int mlp_tc_blocks_per_problem(int P, int64_t per_problem) {
-  int64_t blocks = (per_problem + kMlpRows - 1) / kMlpRows;
-  if (blocks < 1) blocks = 1;
-  int64_t passes = static_cast<int64_t>(P) * blocks / (4 * 148);
-  if (passes > 4) passes = 4;
-  if (passes < 1) passes = 1;
-  return static_cast<int>((blocks + passes - 1) / passes);
+  int64_t tiles = (per_problem + kTileRows - 1) / kTileRows;
+  if (tiles < 1) tiles = 1;
+  int64_t nblk = (tiles + 127) / 128;
+  const int64_t fill = (148 + P - 1) / (P > 0 ? P : 1);  // CTAs per problem that fill the machine once
+  if (nblk < fill) nblk = fill < tiles ? fill : tiles;
+  return static_cast<int>(nblk);
 }
 
 size_t mlp_tc_scratch_bytes(int C) { return 256 + static_cast<size_t>(kCombos) * C * kCandRec; }
