@@ -578,17 +578,14 @@ ks_status ks_select_one(ks_ctx* ctx, ks_problem p, const ks_candidate* d_c, int 
     }
   }
 
-  const size_t out_bytes = align_up(k * sizeof(int32_t)) + align_up(k * sizeof(float));
+  // every other model: the general path with one problem; its merge kernel writes the k results
+  // straight into the mapped host block, so there is no copy between the kernel and the caller
   const size_t part = align_up(ks::select_partial_bytes(*model, 1, C, C, false, k));
-  ks_status s = ensure_workspace(ctx, part + out_bytes);
+  ks_status s = ensure_workspace(ctx, part);
   if (s != KS_OK) return s;
-  char* base = static_cast<char*>(ctx->ws);
-  int32_t* d_idx = reinterpret_cast<int32_t*>(base + part);
-  float* d_sc = reinterpret_cast<float*>(base + part + align_up(k * sizeof(int32_t)));
   cudaError_t e = ks::launch_select(ctx->desc, *model, nullptr, &p, 1, d_c, C, nullptr, nullptr, C, k,
-                                    ctx->ws, d_idx, d_sc, st, &ctx->launches, ctx->d_status);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(pin_idx, d_idx, k * sizeof(int32_t), cudaMemcpyDeviceToHost, st);
-  if (e == cudaSuccess) e = cudaMemcpyAsync(pin_sc, d_sc, k * sizeof(float), cudaMemcpyDeviceToHost, st);
+                                    ctx->ws, ctx->d_pinned_idx, ctx->d_pinned_score, st, &ctx->launches,
+                                    ctx->d_status);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "ks_select_one");
   std::memcpy(h_topk_idx, pin_idx, k * sizeof(int32_t));
