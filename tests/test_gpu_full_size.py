@@ -113,3 +113,24 @@ def test_config3_latency_stream_sample(ks, ctx):
         _, _, allsc = oracle.select(w.problems[i:i + 1], w.candidates, w.desc, w.k, gbdt=w.gbdt, want_scores=True)
         ok, msg = topk_accept(hi.numpy(), hs.numpy(), allsc, np.arange(C, dtype=np.int32), w.k, TOL_GBDT)
         assert ok, f"call {i}: {msg}"
+
+
+def test_full_size_paper_forms(ks, ctx):
+    """The paper's own model forms at config-1 / config-4 size: partition splits on the
+    categorical fields, the one-hot ranker input, and the linear ridge scorer."""
+    w = wl.make_workload(1)
+    w.gbdt = (w.gbdt[0], wl.with_partition_splits(3, w.gbdt[1]), w.gbdt[2])
+    idx, sc = run_full(ks, ctx, w, ctx.model_create_gbdt(*w.gbdt))
+    check_properties(w, idx, sc)
+    check_sampled(w, idx, sc, [0, 333, len(w.problems) - 1], TOL_GBDT)
+    st = wl.feature_stats("cfg1")
+    mu, sg = wl.onehot_stats(st["mu"], st["sigma"])
+    w4 = wl.make_workload(4)
+    w4.mlp = wl.mlp_xavier(31, [80, 256, 256, 1], mu, sg)
+    idx, sc = run_full(ks, ctx, w4, ctx.model_create_mlp(w4.mlp))
+    check_properties(w4, idx, sc)
+    check_sampled(w4, idx, sc, [0, 700], TOL_MLP)
+    w4.mlp = wl.mlp_xavier(32, [64, 1], st["mu"], st["sigma"])
+    idx, sc = run_full(ks, ctx, w4, ctx.model_create_mlp(w4.mlp))
+    check_properties(w4, idx, sc)
+    check_sampled(w4, idx, sc, [0, 511, len(w4.problems) - 1], 1e-4)
