@@ -53,7 +53,11 @@ constexpr int kMaxRows = 80;           // quantised rows the kernel supports (ti
 constexpr int kThrPerRow = 128;        // 127 thresholds + padding
 constexpr int kRowStride = kFastRows;  // bytes between rows of the tile (one byte per candidate)
 constexpr int kWords = kFastRows / 4;  // words per row = lane slots
-constexpr int kSpinLimit = 1 << 20;  // probes of up to ~2 us each: a wait gives up after about two seconds
+constexpr int kSpinLimit = 1 << 22;  // probes about kSleepNs apart: a wait gives up after about two seconds
+#ifndef KS_SLEEP_NS
+#define KS_SLEEP_NS 400
+#endif
+constexpr unsigned kSleepNs = KS_SLEEP_NS;
 constexpr int kCandRec = 64;           // bytes per (combination, candidate) record of quantised rows
 constexpr int kCombos = 16;            // dtype_ab x dtype_d
 
@@ -73,19 +77,23 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, int count) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
-      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}\n"
+      "{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
       : "=r"(ok)
-      : "r"(bar), "r"(parity), "r"(2000u)  // let the hardware park the thread for up to ~2 us per probe
+      : "r"(bar), "r"(parity)
       : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up after kSpinLimit probes and reports false.
+// Bounded wait: one probe, then sleep-and-probe (a sleeping warp takes no issue slots from the
+// warps that still walk); gives up after kSpinLimit probes and reports false.
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-  for (int i = 0; i < kSpinLimit; ++i)
-    if (mbar_try_wait(bar, parity)) return true;
+  if (mbar_test_wait(bar, parity)) return true;
+  for (int i = 0; i < kSpinLimit; ++i) {
+    __nanosleep(kSleepNs);
+    if (mbar_test_wait(bar, parity)) return true;
+  }
   return false;
 }
 __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
