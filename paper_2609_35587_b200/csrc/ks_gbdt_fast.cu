@@ -55,7 +55,7 @@ constexpr int kRowStride = kFastRows;  // bytes between rows of the tile (one by
 constexpr int kWords = kFastRows / 4;  // words per row = lane slots
 constexpr int kSpinLimit = 1 << 22;  // probes about kSleepNs apart: a wait gives up after about two seconds
 #ifndef KS_SLEEP_NS
-#define KS_SLEEP_NS 400
+#define KS_SLEEP_NS 1200
 #endif
 constexpr unsigned kSleepNs = KS_SLEEP_NS;
 constexpr int kCandRec = 64;           // bytes per (combination, candidate) record of quantised rows
@@ -64,7 +64,7 @@ constexpr int kCombos = 16;            // dtype_ab x dtype_d
 static_assert(kFastThreads == 2 * kWords && kFastR == 2, "tile geometry");
 
 // shared memory map (byte offsets from the dynamic shared base)
-constexpr int kNBuf = 2;                // tree-chunk buffers (a ring; four of half the size measured slower)
+constexpr int kNBuf = 2;                // tree-chunk buffers (a ring; four of 8 KB and three of 12 KB measured slower)
 constexpr int kOffBuf0 = 0;
 constexpr int kOffTile = kNBuf * kBufBytes;
 
@@ -733,11 +733,11 @@ cudaError_t build_fast_gbdt(GbdtModel& m, int n_trees, const int64_t* off, const
     }
   }
   const int per_tree_words = (2 << D) - 1;
-  int tpc = kBufBytes / (per_tree_words * 4) / 4 * 4;  // a multiple of 4 keeps chunks 16-byte sized
-  if (tpc < 4) return cudaSuccess;
-  if (tpc > (n_trees + 3) / 4 * 4) tpc = (n_trees + 3) / 4 * 4;  // a small ensemble is one short chunk
+  int tpc = kBufBytes / (per_tree_words * 4) / 2 * 2;  // even: the two halves of a CTA share a chunk's trees
+  if (tpc < 2) return cudaSuccess;
+  if (tpc > (n_trees + 1) / 2 * 2) tpc = (n_trees + 1) / 2 * 2;  // a small ensemble is one short chunk
   const int n_chunks = (n_trees + tpc - 1) / tpc;
-  const int chunk_words = tpc * per_tree_words;
+  const int chunk_words = (tpc * per_tree_words + 3) / 4 * 4;  // bulk copies move multiples of 16 bytes
   int L = D < 3 ? D : 3;  // levels whose nodes travel as kernel-parameter constants
   while (L > 0 && static_cast<int64_t>(n_chunks) * tpc * ((1 << L) - 1) > kFastTopPairs) --L;
   const int n_top = (1 << L) - 1;

@@ -435,13 +435,19 @@ def slot_thresholds(stats_key):
     return lambda f, rng: thr[f, rng.integers(0, thr.shape[1])]
 
 
-@pytest.mark.parametrize("case", ["unbalanced_depth8", "deep_generic", "many_shallow_trees", "split_rows",
-                                  "too_many_rows"])
+@pytest.mark.parametrize("case", ["unbalanced_depth8", "depth9", "depth10", "odd_tree_count", "deep_generic",
+                                  "many_shallow_trees", "split_rows", "too_many_rows"])
 def test_select_other_model_shapes(ks, ctx, case):
     prob, cand, _, _ = wl.make_inputs(1, P=5, C=3000)
     x = oracle.featurize(prob, cand, DESC)
     if case == "unbalanced_depth8":      # padded to complete trees on the quantised path
         off, nodes = random_trees(1, 40, 8, 0.7, slot_thresholds("cfg1"))
+    elif case == "depth9":               # four trees per 16 KB chunk
+        off, nodes = random_trees(6, 30, 9, 0.8, slot_thresholds("cfg1"))
+    elif case == "depth10":              # two trees per chunk: each half of a CTA walks one
+        off, nodes = random_trees(7, 21, 10, 0.8, slot_thresholds("cfg1"))
+    elif case == "odd_tree_count":       # the last chunk is padded with empty trees
+        off, nodes = random_trees(8, 13, 8, 0.8, slot_thresholds("cfg1"))
     elif case == "deep_generic":         # depth 12 > 10: generic kernel
         off, nodes = random_trees(2, 12, 12, 0.8, slot_thresholds("cfg1"))
     elif case == "many_shallow_trees":   # 2,500 trees: fewer top levels fit the constant bank
