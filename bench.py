@@ -285,6 +285,69 @@ def run_catalogue(args, rank, local_rank, dev):
     print(json.dumps(line), flush=True)
 
 
+def run_stages(args, rank, local_rank, dev):
+    """The unfused calls of the boundary, one at a time: `ks_featurize` writes the padded feature
+    rows of every pair to HBM (256 B each), `ks_score` reads them back and scores them with the
+    tree ensemble of config 1 and with the MLP of config 4. The fused `ks_select` never does this
+    round trip; these lines say what it would cost. Each call is timed alone with CUDA events,
+    with a 256 MiB L2 flush in front (the feature matrix is far larger than L2 anyway)."""
+    if rank != 0:
+        return
+    import torch
+    from paper_2609_35587_b200 import binding as ks
+    from paper_2609_35587_b200 import workloads as wl
+    P = args.problems or 64
+    w = wl.make_workload(1, P=P)
+    w4 = wl.make_workload(4, P=1)
+    C = len(w.candidates)
+    pairs = P * C
+    ctx = ks.Context(w.desc, local_rank)
+    gbdt = ctx.model_create_gbdt(*w.gbdt)
+    mlp = ctx.model_create_mlp(w4.mlp)
+    d_p, d_c = ks.to_device(w.problems, dev), ks.to_device(w.candidates, dev)
+    feat = torch.empty((pairs, ks.KS_F_PAD), dtype=torch.float32, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    peaks = load_peaks()
+    row_bytes = 4 * ks.KS_F_PAD
+    calls = [
+        ("ks_featurize", lambda: ctx.featurize(d_p, P, d_c, C, out=feat), pairs * row_bytes + C * 16 + P * 16),
+        ("ks_score (500 trees, depth 8)", lambda: ctx.score(feat, gbdt), pairs * (row_bytes + 4)),
+        ("ks_score (MLP 64-256-256-1)", lambda: ctx.score(feat, mlp), pairs * (row_bytes + 4)),
+    ]
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    launches0 = ctx.launch_count()
+    stages = []
+    for name, fn, nbytes in calls:
+        for _ in range(max(args.warmup, 3)):
+            fn()
+        torch.cuda.synchronize()
+        ms = []
+        for _ in range(args.steps):
+            flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            ms.append(e0.elapsed_time(e1))
+        t = float(np.mean(ms)) * 1e-3
+        stages.append({"call": name, "ms": t * 1e3, "pairs_per_s": pairs / t,
+                       "roofline": {"bound": "hbm", "achieved": nbytes / t / 1e9, "peak": peaks["hbm_gbs"],
+                                    "unit": "GB/s", "frac": nbytes / t / 1e9 / peaks["hbm_gbs"],
+                                    "peak_source": peaks["source"]}})
+    clocks = sampler.stop()
+    line = {"metric": "unfused boundary calls, each timed alone (feature rows through HBM)",
+            "value": stages[0]["pairs_per_s"], "unit": "pairs/s (ks_featurize)", "n_gpus": 1, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": stages[0]["ms"], "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "config 1 (full_space) catalogue and ensemble, config 4 MLP", "problems": P,
+                       "candidates_per_problem": C, "l2": "256 MiB flush before every call"},
+            "clocks": clocks, "gpu_launches": int(ctx.launch_count() - launches0), "stages": stages,
+            "cpu_baseline": None, "e2e": None}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -300,6 +363,8 @@ def main():
     ap.add_argument("--skip-e2e", action="store_true", help="profiling aid: skip the host-buffer leg")
     ap.add_argument("--catalogue", action="store_true",
                     help="measure the search-space enumeration + validity filter instead of a selection workload")
+    ap.add_argument("--stages", action="store_true",
+                    help="time the unfused calls (ks_featurize, ks_score) one at a time instead of ks_select")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -319,10 +384,13 @@ def main():
     dev = torch.device("cuda", local_rank)
     cfg = args.workload
     spec = wl.CONFIGS[cfg]
-    if world > 1 and cfg != 3 and not args.catalogue:
+    if world > 1 and cfg != 3 and not args.catalogue and not args.stages:
         dist.init_process_group("nccl", device_id=dev)
     if args.catalogue:
         run_catalogue(args, rank, local_rank, dev)
+        return
+    if args.stages:
+        run_stages(args, rank, local_rank, dev)
         return
     if cfg == 3:
         run_latency_stream(args, rank, local_rank, dev)

@@ -95,7 +95,10 @@ typedef struct {
  * that hold a level code (layout flags 3, 4; operand type 5; bias flag 8; activation 9; kernel
  * schedule 17; epilogue schedule 18; tile scheduler 19), the bit pattern of thr_or_leaf is a
  * non-zero membership mask over the field's level codes (bit c = level c), and a row whose
- * level is in the set goes to `left + 1`, any other row to `left`. */
+ * level is in the set goes to `left + 1`, any other row to `left`. Feature rows given to
+ * ks_score must hold one of the field's level codes in such a column; which way any other
+ * value (not a level, NaN, infinite) goes at a partition split is unspecified. At a numeric
+ * split a NaN goes to `left + 1`, as x < thr is false. */
 #define KS_NODE_NUMERIC 0
 #define KS_NODE_PARTITION 1
 typedef struct {
@@ -239,7 +242,10 @@ ks_status ks_featurize(ks_ctx* ctx, const ks_problem* d_p, int P, const ks_candi
 
 /* s = f_theta(x) for `rows` feature rows (row-major [rows, 64] fp32). For a tree model,
  * d_leaf_idx (nullable, [rows, n_trees] uint16) receives the tree-relative node index of
- * the leaf each tree ends in. Must be NULL for an MLP. */
+ * the leaf each tree ends in. Must be NULL for an MLP. Without leaf indices, an ensemble that
+ * qualifies for the quantised walk of ks_select is scored by that walk on the given rows (the
+ * leaf values are then added in that kernel's order, not tree by tree; same tolerance); the
+ * call may grow the context's workspace, so it orders after earlier work like ks_select does. */
 ks_status ks_score(ks_ctx* ctx, const float* d_features, int64_t rows, const ks_model* model,
                    float* d_scores, uint16_t* d_leaf_idx, void* stream);
 

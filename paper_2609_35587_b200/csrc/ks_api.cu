@@ -489,6 +489,14 @@ ks_status ks_score(ks_ctx* ctx, const float* d_features, int64_t rows, const ks_
   if (model->kind == 2) return KS_ERR_UNSUPPORTED;  // the static score is a function of (p, c), not of x
   if (model->kind == 1 && d_leaf_idx) return KS_ERR_INVALID_ARG;
   DeviceGuard g(ctx->device);
+  if (model->kind == 0 && model->gbdt.fast && !d_leaf_idx) {
+    // quantised path: the same walk as ks_select, on tiles built from the given rows
+    ks_status s = ensure_workspace(ctx, ks::score_fast_scratch_bytes(model->gbdt, rows));
+    if (s != KS_OK) return s;
+    cudaError_t e = ks::launch_score_fast(ctx->desc, model->gbdt, d_features, rows, d_scores, ctx->ws,
+                                          ctx->d_status, static_cast<cudaStream_t>(stream), &ctx->launches);
+    return e == cudaSuccess ? KS_OK : cuda_fail(ctx, e, "ks_score");
+  }
   cudaError_t e =
       model->kind == 0
           ? ks::launch_score_gbdt(model->gbdt, d_features, rows, d_scores, d_leaf_idx,

@@ -149,6 +149,7 @@ struct SliceArgs {
   const uint8_t* tiles;    // prepared tiles [blocks][rows][kRowStride] (tile_one_kernel), or null
   int* out_seq;            // single-problem form: receives `seq` once the k results are written
   int seq;
+  float* score_out;        // scoring call (ks_score): the scores of the block's rows go here, no ranking
 };
 
 struct FastView {
@@ -270,6 +271,58 @@ tile_one_kernel(ks_gpu_desc desc, ks_problem p_value, const ks_candidate* __rest
   extern __shared__ float s_thr[];  // thresholds of this role's rows
   if (blockIdx.y == 0) tile_one_rows<true>(desc, p_value, c, C, fv, tiles, s_thr);
   else tile_one_rows<false>(desc, p_value, c, C, fv, tiles, s_thr);
+}
+
+// ------------------------------------------------------------------------------------------
+// scoring call: tiles from feature rows
+// ------------------------------------------------------------------------------------------
+
+// ks_score with a qualifying ensemble: one thread per feature row quantises all of the row's
+// columns into the tile layout of phase A; the walk kernel then copies the tiles as in the
+// single-problem call and writes scores instead of ranking. A NaN goes right at every numeric
+// split (x < t is false), like +inf: the last bin. Also clears the abort flag.
+__global__ void __launch_bounds__(256)
+tile_rows_kernel(const float* __restrict__ feat, int64_t rows, FastView fv, uint8_t* __restrict__ tiles) {
+  extern __shared__ float s_thr[];  // thresholds of every row
+  __shared__ uint8_t s_r0[64], s_rc[64];
+  const int tid = threadIdx.x;
+  if (blockIdx.x == 0 && tid == 0) g_fast_abort = 0;
+  {
+    const float4* src = reinterpret_cast<const float4*>(fv.thr);
+    float4* dst = reinterpret_cast<float4*>(s_thr);
+    for (int i = tid; i < fv.n_rows * (kThrPerRow / 4); i += blockDim.x) dst[i] = __ldg(src + i);
+  }
+  if (tid < 64) {
+    s_r0[tid] = fv.feat_row0[tid];
+    s_rc[tid] = fv.feat_rowcnt[tid];
+  }
+  __syncthreads();
+  const int64_t slot = static_cast<int64_t>(blockIdx.x) * blockDim.x + tid;
+  const int64_t blk = slot / kFastRows;
+  const int in = static_cast<int>(slot % kFastRows);
+  const int t = in % kFastThreads, r = in / kFastThreads;  // phase-A thread and its candidate
+  uint8_t* my = tiles + static_cast<size_t>(blk) * fv.n_rows * kRowStride + (t % kWords) * 4 + (t / kWords) * kFastR + r;
+  if (slot >= rows) {
+    for (int q = 0; q < fv.n_rows; ++q) my[q * kRowStride] = 0x80;
+    return;
+  }
+  const float4* src = reinterpret_cast<const float4*>(feat + slot * KS_F_PAD);
+#pragma unroll 4
+  for (int q4 = 0; q4 < KS_F_PAD / 4; ++q4) {
+    const float4 v4 = __ldg(src + q4);
+    const float v[4] = {v4.x, v4.y, v4.z, v4.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int col = 4 * q4 + j;
+      if (col >= KS_F) continue;
+      const int r0 = s_r0[col], rc = s_rc[col];
+      for (int q = 0; q < rc; ++q) {
+        const float* T = s_thr + (r0 + q) * kThrPerRow;
+        const int bin = (v[j] != v[j] && !(T[kThrPerRow - 1] < 0.0f)) ? kThrPerRow - 1 : row_bin(T, v[j]);
+        my[(r0 + q) * kRowStride] = static_cast<uint8_t>(0x80 | bin);
+      }
+    }
+  }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -554,6 +607,16 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
       for (int r = 0; r < 4; ++r) s_part[r * kWords + word] = score[r];
     }
     __syncthreads();
+    if (sl.score_out) {
+      // scoring call: the scores are the result (same order of additions as the ranking path)
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        const int64_t row = start + static_cast<int64_t>(r & 1) * kFastThreads + word + kWords * (r >> 1);
+        if (half == 0 && row < stop)
+          sl.score_out[lo + row] = ((fv.base + score[r]) + s_part[r * kWords + word]) + 0.0f;
+      }
+      continue;
+    }
     if (S > 1) {
       // slice mode: publish this CTA's partial scores, let the last arrival finish the block
 #pragma unroll
@@ -969,6 +1032,69 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
   if (L == 1) KS_GO(1, -1);
   KS_GO(0, -1);
 #undef KS_GO
+}
+
+// ks_score on the quantised path. Rows are taken in batches so that the tiles (n_rows bytes per
+// row) stay a bounded workspace; every batch is one tile launch and one walk launch.
+constexpr int64_t kScoreBatchBlocks = 4096;
+
+size_t score_fast_scratch_bytes(const GbdtModel& g, int64_t rows) {
+  int64_t blocks = (rows + kFastRows - 1) / kFastRows;
+  if (blocks > kScoreBatchBlocks) blocks = kScoreBatchBlocks;
+  return static_cast<size_t>(blocks) * g.n_qrows * kRowStride;
+}
+
+cudaError_t launch_score_fast(const ks_gpu_desc& desc, const GbdtModel& g, const float* d_feat, int64_t rows,
+                              float* d_scores, void* scratch, int* status, cudaStream_t stream,
+                              int64_t* launches) {
+  FastView fv{};
+  fv.n_rows = g.n_qrows;
+  fv.n_pair_rows = g.n_pair_rows;
+  fv.n_cand_rows = g.n_cand_rows;
+  fv.n_prob_rows = g.n_prob_rows;
+  fv.depth = g.fast_depth;
+  fv.n_chunks = g.n_chunks;
+  fv.chunk_bytes = g.chunk_bytes;
+  fv.tpc = g.tpc;
+  fv.base = g.base;
+  fv.chunks = g.d_qnodes;
+  fv.thr = g.d_qthr;
+  fv.feat_row0 = g.d_qrow0;
+  fv.feat_rowcnt = g.d_qrowcnt;
+  uint8_t* tiles = static_cast<uint8_t*>(scratch);
+  const size_t tthr = sizeof(float) * kThrPerRow * g.n_qrows;
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(&tile_rows_kernel), tthr);
+  if (e != cudaSuccess) return e;
+  const FastTopParams& top = *g.h_top;
+  const int L = g.top_levels, np = g.fast_depth - L;
+  const ks_problem pv{};
+  for (int64_t first = 0; first < rows; first += kScoreBatchBlocks * kFastRows) {
+    const int64_t n = rows - first < kScoreBatchBlocks * kFastRows ? rows - first : kScoreBatchBlocks * kFastRows;
+    const int nblk = static_cast<int>((n + kFastRows - 1) / kFastRows);
+    tile_rows_kernel<<<nblk * (kFastRows / 256), 256, tthr, stream>>>(d_feat + first * KS_F_PAD, n, fv, tiles);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    SliceArgs sl{};
+    sl.n_slices = 1;
+    sl.tiles = tiles;
+    sl.score_out = d_scores + first;
+    *launches += 2;
+#define KS_GO(LL, NN)                                                                                          \
+  e = launch_ln<LL, NN>(desc, nullptr, pv, 1, 1, nullptr, static_cast<int>(n), nblk, kFastRows, nullptr, nullptr, \
+                        fv, 0, nullptr, status, sl, top, stream)
+    if (L == 3 && np == 5) KS_GO(3, 5);
+    else if (L == 3 && np == 3) KS_GO(3, 3);
+    else if (L == 2 && np == 6) KS_GO(2, 6);
+    else if (L == 2 && np == 5) KS_GO(2, 5);
+    else if (L == 3 && np == 4) KS_GO(3, 4);
+    else if (L == 3) KS_GO(3, -1);
+    else if (L == 2) KS_GO(2, -1);
+    else if (L == 1) KS_GO(1, -1);
+    else KS_GO(0, -1);
+#undef KS_GO
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
 }
 
 }  // namespace ks

@@ -192,6 +192,11 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
                                cudaStream_t stream, int64_t* launches, cudaEvent_t ev_begin,
                                const FastSlice* slice = nullptr);
 int fast_slices(const GbdtModel& g, int64_t blocks);
+// ks_score with a qualifying ensemble: tiles quantised from the feature rows, then the same walk.
+size_t score_fast_scratch_bytes(const GbdtModel& g, int64_t rows);
+cudaError_t launch_score_fast(const ks_gpu_desc& desc, const GbdtModel& g, const float* d_feat, int64_t rows,
+                              float* d_scores, void* scratch, int* status, cudaStream_t stream,
+                              int64_t* launches);
 
 // Tensor-core MLP path.
 cudaError_t build_fast_mlp(MlpModel& m, const uint16_t* const* h_w, const float* const* h_b, const float* h_mu,

@@ -134,3 +134,19 @@ def test_full_size_paper_forms(ks, ctx):
     idx, sc = run_full(ks, ctx, w4, ctx.model_create_mlp(w4.mlp))
     check_properties(w4, idx, sc)
     check_sampled(w4, idx, sc, [0, 511, len(w4.problems) - 1], 1e-4)
+
+
+def test_score_rows_in_batches(ks, ctx):
+    """ks_score on the quantised path takes 4,096 blocks of 1,024 rows per batch: more rows than
+    one batch, with a ragged last block."""
+    w = wl.make_workload(1, P=4, C=4000, trees=6, depth=5)
+    x = oracle.featurize(w.problems, w.candidates, w.desc)
+    rows = 4096 * 1024 + 777
+    x = np.ascontiguousarray(np.resize(x, (rows, x.shape[1])))
+    x[-1, 3] = np.nan
+    rs = oracle.score_gbdt(x, *w.gbdt)
+    model = ctx.model_create_gbdt(*w.gbdt)
+    n0 = ctx.launch_count()
+    s = ctx.score(ks.to_device(x, torch.device("cuda", 0)), model).cpu().numpy()
+    assert ctx.launch_count() - n0 == 4
+    assert np.all(np.abs(s - rs) <= TOL_GBDT * np.maximum(1, np.abs(rs)))

@@ -127,6 +127,33 @@ def test_score_gbdt_unbalanced_and_stump_trees(ks, ctx):
     assert np.array_equal(s.cpu().numpy(), rs)
 
 
+def test_score_gbdt_quantised_path(ks, ctx):
+    """Scores without leaf indices from a qualifying ensemble take the quantised walk on tiles
+    built from the given rows: ragged row count, non-finite inputs (a NaN goes right at a numeric
+    split, as x < t is false), partition splits."""
+    w = wl.make_workload(1, P=5, C=3000, trees=60, depth=8)
+    x = oracle.featurize(w.problems, w.candidates, DESC)
+    rng = np.random.default_rng(3)
+    numeric = np.array([c for c in range(63) if c not in wl.CATEGORICAL_LEVELS])
+    for v in (np.nan, np.inf, -np.inf):
+        x[rng.integers(0, len(x), 200), numeric[rng.integers(0, len(numeric), 200)]] = v
+    for gbdt in (w.gbdt, (w.gbdt[0], wl.with_partition_splits(5, w.gbdt[1]), w.gbdt[2])):
+        rs = oracle.score_gbdt(x, *gbdt)
+        model = ctx.model_create_gbdt(*gbdt)
+        d_x = dev(ks, x)
+        n0 = ctx.launch_count()
+        s = ctx.score(d_x, model).cpu().numpy()
+        assert ctx.launch_count() - n0 == 2          # tile launch + walk launch
+        assert np.all(np.abs(s - rs) <= TOL_GBDT * np.maximum(1, np.abs(rs)))
+        s2, leaf = ctx.score(d_x, model, want_leaf_idx=True)   # the general kernel
+        _, rleaf = oracle.score_gbdt(x, *gbdt, want_leaf_idx=True)
+        assert np.array_equal(leaf.cpu().numpy().view(np.uint16), rleaf)
+        assert np.all(np.abs(s - s2.cpu().numpy()) <= TOL_GBDT * np.maximum(1, np.abs(rs)))
+    for n in (1, 1023, 1024, 1025):
+        s = ctx.score(dev(ks, x[:n]), model).cpu().numpy()
+        assert np.all(np.abs(s - rs[:n]) <= TOL_GBDT * np.maximum(1, np.abs(rs[:n])))
+
+
 def test_score_mlp(ks, ctx):
     w = wl.make_workload(4, P=3, C=411)
     x = oracle.featurize(w.problems, w.candidates, DESC)
