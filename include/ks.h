@@ -245,7 +245,10 @@ ks_status ks_featurize(ks_ctx* ctx, const ks_problem* d_p, int P, const ks_candi
  * the leaf each tree ends in. Must be NULL for an MLP. Without leaf indices, an ensemble that
  * qualifies for the quantised walk of ks_select is scored by that walk on the given rows (the
  * leaf values are then added in that kernel's order, not tree by tree; same tolerance); the
- * call may grow the context's workspace, so it orders after earlier work like ks_select does. */
+ * call may grow the context's workspace, so it orders after earlier work like ks_select does.
+ * An MLP that the tensor-core kernel of ks_select serves (input width 64, one or two hidden
+ * layers of at most 256 units) is scored by that kernel on the given rows. Non-finite inputs
+ * of an MLP count as 0 before standardisation. */
 ks_status ks_score(ks_ctx* ctx, const float* d_features, int64_t rows, const ks_model* model,
                    float* d_scores, uint16_t* d_leaf_idx, void* stream);
 

@@ -497,6 +497,11 @@ ks_status ks_score(ks_ctx* ctx, const float* d_features, int64_t rows, const ks_
                                           ctx->d_status, static_cast<cudaStream_t>(stream), &ctx->launches);
     return e == cudaSuccess ? KS_OK : cuda_fail(ctx, e, "ks_score");
   }
+  if (model->kind == 1 && ks::score_mlp_tc_ok(model->mlp)) {
+    cudaError_t e = ks::launch_score_mlp_tc(ctx->desc, model->mlp, d_features, rows, d_scores, ctx->d_status,
+                                            static_cast<cudaStream_t>(stream), &ctx->launches);
+    return e == cudaSuccess ? KS_OK : cuda_fail(ctx, e, "ks_score");
+  }
   cudaError_t e =
       model->kind == 0
           ? ks::launch_score_gbdt(model->gbdt, d_features, rows, d_scores, d_leaf_idx,

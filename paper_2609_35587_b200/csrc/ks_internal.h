@@ -209,6 +209,10 @@ void free_ridge(MlpModel& m);
 size_t ridge_scratch_bytes(int C);
 int mlp_tc_blocks_per_problem(int P, int64_t per_problem);
 size_t mlp_tc_scratch_bytes(int C);
+// ks_score on the tensor-core kernel (ordinal input form only): the given rows are the input.
+bool score_mlp_tc_ok(const MlpModel& m);
+cudaError_t launch_score_mlp_tc(const ks_gpu_desc& desc, const MlpModel& m, const float* d_feat, int64_t rows,
+                                float* d_scores, int* status, cudaStream_t stream, int64_t* launches);
 cudaError_t launch_select_mlp_tc(const ks_gpu_desc& desc, const MlpModel& m, const ks_problem* d_p,
                                  const ks_problem* p_by_value, int P, const ks_candidate* d_c, int C, int nblk,
                                  const int64_t* seg_off, const int32_t* seg_idx, int k,

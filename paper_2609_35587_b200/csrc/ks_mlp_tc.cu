@@ -163,6 +163,9 @@ __device__ __forceinline__ uint32_t pack_bf16_relu(float lo, float hi) {
 // host memory: reading it from every CTA would cost a PCIe round trip each.)
 __device__ int g_mlp_abort;
 
+// the scoring call has no per-call table kernel in front: this clears the abort flag instead
+__global__ void mlp_reset_abort_kernel() { g_mlp_abort = 0; }
+
 __global__ void mlp_combo_mask_kernel(const ks_problem* __restrict__ p, int P, unsigned* __restrict__ mask) {
   unsigned m = 0;
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < P; i += gridDim.x * blockDim.x)
@@ -344,14 +347,19 @@ __device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 128;" :::
 // the kernel
 // ------------------------------------------------------------------------------------------
 
-template <bool kOneHot>  // input form: ordinal codes (K positions as kpos) or one-hot (kpos_oh + folded bias)
+// kForm 0: ordinal input form (K positions as kpos); 1: one-hot form (kpos_oh + folded bias);
+// 2: scoring call - the rows of `feat_rows` (ordinal form) are the input, every score is written to
+// `score_out`, nothing is ranked (one "problem" whose candidates are the rows).
+template <int kForm>
 __global__ void __launch_bounds__(kT, 1)
 select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_problem p_value, int use_value,
                      const ks_candidate* __restrict__ c, int P, int C, int nblk,
                      const int64_t* __restrict__ seg_off, const int32_t* __restrict__ seg_idx,
                      const uint8_t* __restrict__ w_image, const uint8_t* __restrict__ cand_cols, int k,
                      unsigned long long* __restrict__ partial, int* __restrict__ status,
+                     const float* __restrict__ feat_rows, float* __restrict__ score_out,
                      const __grid_constant__ MlpTcParams prm) {
+  constexpr bool kOneHot = kForm == 1, kRows = kForm == 2;
   extern __shared__ __align__(1024) unsigned char smem[];
   __shared__ ProblemTerms s_pt;
   __shared__ PairFastTerms s_pf;
@@ -370,7 +378,7 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
   if (tid == 0) s_abort = *reinterpret_cast<volatile int*>(&g_mlp_abort);
   __syncthreads();
   if (s_abort) {  // a wait ran out in an earlier CTA of this launch: the call fails, leave at once
-    if (tid < k) partial[static_cast<size_t>(blockIdx.x) * k + tid] = 0ull;
+    if (!kRows && tid < k) partial[static_cast<size_t>(blockIdx.x) * k + tid] = 0ull;
     return;
   }
   const bool is_epi = tid < 256;  // warps 0..7 read the accumulators; warps 8..15 produce feature rows
@@ -389,7 +397,7 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
                  bar_f1 = smem_u32(&s_bar[6]), bar_a1 = smem_u32(&s_bar[7]), bar_x1 = smem_u32(&s_bar[8]),
                  bar_b1 = smem_u32(&s_bar[9]);
 
-  if (tid == 0) {
+  if (tid == 0 && !kRows) {
     problem_terms(use_value ? p_value : p[prob], desc, s_pt);
     pair_fast_terms(s_pt, desc, s_pf);
     ks_candidate dummy{};
@@ -418,6 +426,8 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
         s_xp[kFoldCols + 4 + l] = __bfloat162float(__float2bfloat16_rn(
             fmaf(s_pt.act == l ? 1.0f : 0.0f, prm.p_scale[kFoldCols + 4 + l], prm.p_shift[kFoldCols + 4 + l])));
     }
+  }
+  if (tid == 0) {
     mbar_init(bar_w, 1);
     mbar_init(bar_a0, 1);
     mbar_init(bar_a1, 1);
@@ -454,7 +464,7 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
     }
     __syncthreads();
   }
-  const int combo = s_pt.dtype_ab * 4 + s_pt.dtype_d;
+  const int combo = kRows ? 0 : s_pt.dtype_ab * 4 + s_pt.dtype_d;
   bool failed = false;
   // Bounded wait. After the first one that runs out, every later wait of the CTA gives up after a
   // few probes, and the CTAs that start later leave at once (device flag).
@@ -502,7 +512,28 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
       uint32_t w[32];
 #pragma unroll
       for (int q = 0; q < 32; ++q) w[q] = 0u;
-      if (live) {
+      if (kRows) {
+        if (live) {
+          // the given row: non-finite entries count as 0, every column standardised and rounded
+          const float4* src = reinterpret_cast<const float4*>(feat_rows + row * KS_F_PAD);
+          float x[64];
+          x[63] = 0.0f;
+#pragma unroll
+          for (int q4 = 0; q4 < KS_F_PAD / 4; ++q4) {
+            const float4 v4 = __ldg(src + q4);
+            const float v[4] = {v4.x, v4.y, v4.z, v4.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              if (4 * q4 + j >= KS_F) continue;
+              const int kk = kpos(4 * q4 + j);
+              const float f = (fabsf(v[j]) <= 3.402823466e38f) ? v[j] : 0.0f;
+              x[kk] = fmaf(f, prm.scale[kk], prm.shift[kk]);
+            }
+          }
+#pragma unroll
+          for (int q = 0; q < 32; ++q) w[q] = pack_bf16(x[2 * q], x[2 * q + 1]);
+        }
+      } else if (live) {
         const int idx = seg_off ? seg_idx[lo + row] : static_cast<int>(row);
         const ks_candidate cand = c[idx];
         const uint4* rec = reinterpret_cast<const uint4*>(cand_cols + (static_cast<size_t>(combo) * C + idx) * kCandRec);
@@ -610,14 +641,18 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
         const uint32_t acc_row = tmem_row + (tile & 1) * 256;
         const int64_t row = tile_row0(tile) + trow;
         int idx = -1;  // fetched before the wait, so that its latency hides behind it
-        if (row < len) idx = seg_off ? __ldg(seg_idx + lo + row) : static_cast<int>(row);
+        if (row < len) idx = (!kRows && seg_off) ? __ldg(seg_idx + lo + row) : static_cast<int>(row);
         if (!wait_ok((tile & 1) ? bar_b1 : bar_b0, ph_b[tile & 1])) failed = true;  // L2(tile) is complete
         ph_b[tile & 1] ^= 1;
         tc_fence_after();
         const float score = epilogue2<0>(acc_row, prm) + prm.b3;
         tc_fence_before();
         mbar_arrive((tile & 1) ? bar_f1 : bar_f0);
-        warp_topk_insert(top, idx >= 0 ? make_key(score + 0.0f, idx) : 0ull, k);
+        if (kRows) {
+          if (idx >= 0) score_out[row] = score + 0.0f;
+        } else {
+          warp_topk_insert(top, idx >= 0 ? make_key(score + 0.0f, idx) : 0ull, k);
+        }
       }
       s_merge[quarter][lane] = top;
     }
@@ -627,7 +662,7 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
     if (tid == 0 && status) atomicExch(status, KS_ERR_TIMEOUT);
     failed = true;
   }
-  if (warp == 0) {
+  if (warp == 0 && !kRows) {
     unsigned long long mine[4];
 #pragma unroll
     for (int q = 0; q < 4; ++q) mine[q] = s_merge[q][lane];
@@ -824,20 +859,49 @@ cudaError_t launch_select_mlp_tc(const ks_gpu_desc& desc, const MlpModel& m, con
   const unsigned grid = static_cast<unsigned>(static_cast<int64_t>(P) * nblk);
   const uint8_t* image = reinterpret_cast<const uint8_t*>(m.d_tc_image);
   if (m.h_tc_params->onehot) {
-    e = ensure_dynamic_smem(reinterpret_cast<const void*>(&select_mlp_tc_kernel<true>), kSmemBytes);
+    e = ensure_dynamic_smem(reinterpret_cast<const void*>(&select_mlp_tc_kernel<1>), kSmemBytes);
     if (e != cudaSuccess) return e;
-    select_mlp_tc_kernel<true><<<grid, kT, kSmemBytes, stream>>>(desc, d_p, pv, uv, d_c, P, C, nblk, seg_off, seg_idx,
-                                                                 image, d_cols, k, partial, status, *m.h_tc_params);
+    select_mlp_tc_kernel<1><<<grid, kT, kSmemBytes, stream>>>(desc, d_p, pv, uv, d_c, P, C, nblk, seg_off, seg_idx, image,
+                                                              d_cols, k, partial, status, nullptr, nullptr,
+                                                              *m.h_tc_params);
   } else {
-    e = ensure_dynamic_smem(reinterpret_cast<const void*>(&select_mlp_tc_kernel<false>), kSmemBytes);
+    e = ensure_dynamic_smem(reinterpret_cast<const void*>(&select_mlp_tc_kernel<0>), kSmemBytes);
     if (e != cudaSuccess) return e;
-    select_mlp_tc_kernel<false><<<grid, kT, kSmemBytes, stream>>>(desc, d_p, pv, uv, d_c, P, C, nblk, seg_off, seg_idx,
-                                                                  image, d_cols, k, partial, status, *m.h_tc_params);
+    select_mlp_tc_kernel<0><<<grid, kT, kSmemBytes, stream>>>(desc, d_p, pv, uv, d_c, P, C, nblk, seg_off, seg_idx, image,
+                                                              d_cols, k, partial, status, nullptr, nullptr,
+                                                              *m.h_tc_params);
   }
   ++*launches;
   return cudaGetLastError();
 }
 
+// ks_score on the tensor-core kernel (ordinal input form): one CTA per SM, each with an equal
+// share of the 128-row tiles; rows in batches that fit the kernel's 32-bit row count.
+bool score_mlp_tc_ok(const MlpModel& m) { return m.tc && m.h_tc_params && !m.h_tc_params->onehot; }
+
+cudaError_t launch_score_mlp_tc(const ks_gpu_desc& desc, const MlpModel& m, const float* d_feat, int64_t rows,
+                                float* d_scores, int* status, cudaStream_t stream, int64_t* launches) {
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(&select_mlp_tc_kernel<2>), kSmemBytes);
+  if (e != cudaSuccess) return e;
+  const uint8_t* image = reinterpret_cast<const uint8_t*>(m.d_tc_image);
+  const ks_problem pv{};
+  constexpr int64_t kBatch = int64_t{1} << 30;
+  mlp_reset_abort_kernel<<<1, 1, 0, stream>>>();
+  ++*launches;
+  for (int64_t first = 0; first < rows; first += kBatch) {
+    const int64_t n = rows - first < kBatch ? rows - first : kBatch;
+    const int64_t tiles = (n + kTileRows - 1) / kTileRows;
+    const int nblk = static_cast<int>(tiles < 148 ? tiles : 148);
+    select_mlp_tc_kernel<2><<<nblk, kT, kSmemBytes, stream>>>(desc, nullptr, pv, 1, nullptr, 1, static_cast<int>(n), nblk,
+                                                              nullptr, nullptr, image, nullptr, 0, nullptr, status,
+                                                              d_feat + first * KS_F_PAD, d_scores + first,
+                                                              *m.h_tc_params);
+    ++*launches;
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
 
 }  // namespace ks
 

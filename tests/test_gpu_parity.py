@@ -167,6 +167,30 @@ def test_score_mlp(ks, ctx):
     assert np.std(rs) > 1e-2
 
 
+def test_score_mlp_tensor_core_path(ks, ctx):
+    """ks_score with a model the tensor-core kernel serves (ordinal input, one or two hidden layers
+    of at most 256 units) runs there on the given rows: more tiles than CTAs with an uneven share,
+    a ragged last tile, tiny inputs, padded shapes; the one-hot form and wider models take the
+    general kernel."""
+    w = wl.make_workload(4, P=8, C=5003)
+    x = oracle.featurize(w.problems, w.candidates, DESC)
+    x[17, 3] = np.nan
+    x[40001, 62] = -np.inf
+    st = wl.feature_stats("cfg1")
+    for shape in ([64, 256, 256, 1], [64, 128, 1], [64, 256, 64, 1]):
+        mlp = w.mlp if shape == [64, 256, 256, 1] else wl.mlp_xavier(77, shape, st["mu"], st["sigma"])
+        rs = oracle.score_mlp(x, mlp)
+        model = ctx.model_create_mlp(mlp)
+        d_x = dev(ks, x)
+        n0 = ctx.launch_count()
+        s = ctx.score(d_x, model).cpu().numpy()
+        assert ctx.launch_count() - n0 == 2            # flag reset + the tensor-core kernel
+        assert np.all(np.abs(s - rs) <= TOL_MLP * np.maximum(1, np.abs(rs)))
+        for n in (1, 127, 128, 129, 148 * 128 + 5):
+            s = ctx.score(dev(ks, x[:n]), model).cpu().numpy()
+            assert np.all(np.abs(s - rs[:n]) <= TOL_MLP * np.maximum(1, np.abs(rs[:n])))
+
+
 # ---------------------------------------------------------------------------------------------
 # ks_select
 # ---------------------------------------------------------------------------------------------
