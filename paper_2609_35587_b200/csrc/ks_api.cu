@@ -476,8 +476,10 @@ ks_status ks_featurize(ks_ctx* ctx, const ks_problem* d_p, int P, const ks_candi
   if (pairs == 0) return KS_OK;
   if (!d_p || !d_c || !d_features) return KS_ERR_INVALID_ARG;
   DeviceGuard g(ctx->device);
+  s = ensure_workspace(ctx, ks::featurize_scratch_bytes(P));
+  if (s != KS_OK) return s;
   cudaError_t e = ks::launch_featurize(ctx->desc, d_p, P, d_c, C, d_seg_offsets, d_seg_index, pairs,
-                                       d_features, static_cast<cudaStream_t>(stream), &ctx->launches);
+                                       d_features, ctx->ws, static_cast<cudaStream_t>(stream), &ctx->launches);
   return e == cudaSuccess ? KS_OK : cuda_fail(ctx, e, "ks_featurize");
 }
 

@@ -222,8 +222,9 @@ cudaError_t launch_select_mlp_tc(const ks_gpu_desc& desc, const MlpModel& m, con
 // ---- launchers (each enqueues on `stream`, returns the cudaError of the launch) -----------
 cudaError_t launch_featurize(const ks_gpu_desc& desc, const ks_problem* d_p, int P,
                              const ks_candidate* d_c, int C, const int64_t* d_seg_off,
-                             const int32_t* d_seg_idx, int64_t pairs, float* d_out,
+                             const int32_t* d_seg_idx, int64_t pairs, float* d_out, void* scratch,
                              cudaStream_t stream, int64_t* launches);
+size_t featurize_scratch_bytes(int P);  // table of problem terms for the dense form
 
 cudaError_t launch_score_gbdt(const GbdtModel& m, const float* d_feat, int64_t rows, float* d_scores,
                               uint16_t* d_leaf_idx, cudaStream_t stream, int64_t* launches);

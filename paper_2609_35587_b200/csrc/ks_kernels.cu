@@ -52,19 +52,112 @@ featurize_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, const ks_ca
   segment_of(map, prob, lo, len);
   if (threadIdx.x == 0) problem_terms(p[prob], desc, s_pt);
   __syncthreads();
+  // every warp stages and stores its own 32 rows, so that one warp's stores overlap another's
+  // arithmetic without block-wide barriers
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  float* w_tile = s_tile + warp * 32 * 65;
   for (int64_t start = static_cast<int64_t>(chunk) * kBlock; start < len;
        start += static_cast<int64_t>(map.nblk) * kBlock) {
-    const int64_t r = start + threadIdx.x;
-    if (r < len) {
-      const ks_candidate cand = c[pool_index(map, lo, r)];
-      float* row = s_tile + threadIdx.x * 65;
+    const int64_t w0 = start + warp * 32;  // first row of this warp
+    if (w0 >= len) break;
+    if (w0 + lane < len) {
+      const ks_candidate cand = c[pool_index(map, lo, w0 + lane)];
+      float* row = w_tile + lane * 65;
       featurize_pair(s_pt, cand, desc, [&](int col, float v) { row[col] = v; });
     }
-    __syncthreads();
-    const int64_t n_rows = (len - start < kBlock) ? (len - start) : static_cast<int64_t>(kBlock);
-    float* dst = out + (lo + start) * kRow;
-    for (int i = threadIdx.x; i < n_rows * kRow; i += kBlock) dst[i] = s_tile[(i >> 6) * 65 + (i & 63)];
-    __syncthreads();
+    __syncwarp();
+    const int n_rows = (len - w0 < 32) ? static_cast<int>(len - w0) : 32;
+    float* dst = out + (lo + w0) * kRow;
+    for (int i = lane; i < n_rows * kRow; i += 32) __stcs(dst + i, w_tile[(i >> 6) * 65 + (i & 63)]);
+    __syncwarp();
+  }
+}
+
+// Dense form (every problem against the whole pool). The work is cut into items of 32
+// candidates x 1 problem, ordered candidate slab first, and every warp of the grid takes a
+// contiguous run of items of equal length (to within one), so that no SM idles in a last
+// partial wave. A lane keeps its candidate, the candidate-only columns and the candidate's
+// resident-block count in registers while the problems of the run change (re-evaluated only
+// when the element-type combination does); the problem-only terms and columns come from a
+// table written once per call. Only the per-pair columns are arithmetic per pair. Same
+// functions, same operands: the rows are bit-identical to featurize_pair's.
+struct ProblemEntry {
+  ProblemTerms t;
+  float pc[16];  // the problem-only columns, in column order
+};
+
+__host__ __device__ constexpr int class_slot(int col) {
+  int n = 0;
+  for (int q = 0; q < col; ++q)
+    if (feat_class(q) == feat_class(col)) ++n;
+  return n;
+}
+
+__global__ void __launch_bounds__(128)
+problem_table_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, int P, ProblemEntry* __restrict__ tab) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= P) return;
+  ProblemEntry e;
+  problem_terms(p[i], desc, e.t);
+  ks_candidate dummy{};
+  dummy.tile_m = dummy.tile_n = dummy.tile_k = 64;
+  dummy.stages = dummy.cluster_m = dummy.cluster_n = 1;
+#pragma unroll
+  for (int q = 0; q < 16; ++q) e.pc[q] = 0.0f;
+  featurize_pair(e.t, dummy, desc, [&](int col, float v) {
+    if (feat_class(col) == 0) e.pc[class_slot(col)] = v;
+  });
+  tab[i] = e;
+}
+
+__global__ void __launch_bounds__(kBlock, 3)
+featurize_dense_kernel(ks_gpu_desc desc, const ProblemEntry* __restrict__ tab, const ks_candidate* __restrict__ c,
+                       int P, int C, float* __restrict__ out) {
+  extern __shared__ float s_tile[];  // [kBlock][65], one 32-row slab per warp
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  float* row = s_tile + (warp * 32 + lane) * 65;
+  const float* w_tile = s_tile + warp * 32 * 65;
+  const int64_t n_warps = static_cast<int64_t>(gridDim.x) * (kBlock / 32);
+  const int64_t me = static_cast<int64_t>(blockIdx.x) * (kBlock / 32) + warp;
+  const int64_t total = static_cast<int64_t>((C + 31) / 32) * P;
+  const int64_t i_end = total * (me + 1) / n_warps;
+  ks_candidate cand{};
+  float cc[29];
+  long long b_eff = 1;
+  int slab_prev = -1, combo_prev = -1, w0 = 0, n_rows = 0;
+  bool live = false;
+#pragma unroll 1
+  for (int64_t i = total * me / n_warps; i < i_end; ++i) {
+    const int slab = static_cast<int>(i / P), prob = static_cast<int>(i - static_cast<int64_t>(slab) * P);
+    if (slab != slab_prev) {
+      slab_prev = slab;
+      combo_prev = -1;
+      w0 = slab * 32;
+      n_rows = C - w0 < 32 ? C - w0 : 32;
+      live = lane < n_rows;
+      cand = c[live ? w0 + lane : C - 1];
+    }
+    const ProblemEntry& e = tab[prob];
+    const ProblemTerms t = e.t;
+    const int combo = t.dtype_ab * 4 + t.dtype_d;
+    if (combo != combo_prev) {  // the same for every lane
+      combo_prev = combo;
+      b_eff = resources(t, cand, desc).b_eff;
+      featurize_pair(t, cand, desc, [&](int col, float v) {
+        if (feat_class(col) == 1) cc[class_slot(col)] = v;
+      });
+    }
+#pragma unroll
+    for (int col = 0; col < KS_F; ++col) {
+      if (feat_class(col) == 1) row[col] = cc[class_slot(col)];
+      if (feat_class(col) == 0) row[col] = __ldg(&e.pc[class_slot(col)]);
+    }
+    row[KS_F] = 0.0f;
+    pair_columns<true>(t, cand, desc, b_eff, [&](int col, float v) { row[col] = v; });
+    __syncwarp();
+    float* dst = out + (static_cast<int64_t>(prob) * C + w0) * kRow;
+    for (int q = lane; q < n_rows * kRow; q += 32) __stcs(dst + q, w_tile[(q >> 6) * 65 + (q & 63)]);
+    __syncwarp();
   }
 }
 
@@ -460,11 +553,23 @@ static PairMap make_map(int P, int C, int64_t pairs, const int64_t* seg_off, con
 
 cudaError_t launch_featurize(const ks_gpu_desc& desc, const ks_problem* d_p, int P,
                              const ks_candidate* d_c, int C, const int64_t* d_seg_off,
-                             const int32_t* d_seg_idx, int64_t pairs, float* d_out,
+                             const int32_t* d_seg_idx, int64_t pairs, float* d_out, void* scratch,
                              cudaStream_t stream, int64_t* launches) {
   if (P == 0 || pairs == 0) return cudaSuccess;
   const PairMap map = make_map(P, C, pairs, d_seg_off, d_seg_idx, kBlock);
   const size_t smem = sizeof(float) * kBlock * 65;
+  if (!d_seg_off && C > 0 && scratch) {
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(&featurize_dense_kernel), smem);
+    if (e != cudaSuccess) return e;
+    ProblemEntry* tab = static_cast<ProblemEntry*>(scratch);
+    problem_table_kernel<<<(P + 127) / 128, 128, 0, stream>>>(desc, d_p, P, tab);
+    const int64_t total = static_cast<int64_t>((C + 31) / 32) * P;
+    int64_t grid = (total + kBlock / 32 - 1) / (kBlock / 32);
+    if (grid > 3 * 148) grid = 3 * 148;  // three resident blocks per SM
+    featurize_dense_kernel<<<static_cast<unsigned>(grid), kBlock, smem, stream>>>(desc, tab, d_c, P, C, d_out);
+    *launches += 2;
+    return cudaGetLastError();
+  }
   cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(&featurize_kernel), smem);
   if (e != cudaSuccess) return e;
   featurize_kernel<<<static_cast<unsigned>(static_cast<int64_t>(P) * map.nblk), kBlock, smem, stream>>>(
@@ -753,5 +858,7 @@ cudaError_t launch_select_generic_trees(const ks_gpu_desc& desc, const DevNode* 
                                                                           d_topk_idx, d_topk_score);
   return cudaGetLastError();
 }
+
+size_t featurize_scratch_bytes(int P) { return sizeof(ProblemEntry) * static_cast<size_t>(P > 0 ? P : 1); }
 
 }  // namespace ks

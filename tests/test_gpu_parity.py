@@ -67,6 +67,15 @@ def test_featurize_cross_precision_segments_bit_exact(ks, ctx):
     assert_features_equal(got, oracle.featurize(prob, cand, DESC, so, si))
 
 
+def test_featurize_dense_mixed_element_types_bit_exact(ks, ctx):
+    """Dense form with the element types changing from problem to problem: the candidate-only
+    columns a lane keeps across problems are re-evaluated whenever the combination changes."""
+    prob, cand, _, _ = wl.make_inputs(2, P=41, seg=64)
+    cand = cand[:1500]
+    assert len(np.unique(prob["dtype_ab"].astype(int) * 4 + prob["dtype_d"])) > 3
+    assert_features_equal(gpu_features(ks, ctx, prob, cand), oracle.featurize(prob, cand, DESC))
+
+
 def test_featurize_stream_problems_and_ragged_sizes(ks, ctx):
     prob, cand, _, _ = wl.make_inputs(3, P=301, C=70)
     assert_features_equal(gpu_features(ks, ctx, prob, cand), oracle.featurize(prob, cand, DESC))
