@@ -277,40 +277,47 @@ tile_one_kernel(ks_gpu_desc desc, ks_problem p_value, const ks_candidate* __rest
 // scoring call: tiles from feature rows
 // ------------------------------------------------------------------------------------------
 
-// ks_score with a qualifying ensemble: one thread per feature row quantises all of the row's
-// columns into the tile layout of phase A; the walk kernel then copies the tiles as in the
-// single-problem call and writes scores instead of ranking. A NaN goes right at every numeric
-// split (x < t is false), like +inf: the last bin. Also clears the abort flag.
-__global__ void __launch_bounds__(256)
+// ks_score with a qualifying ensemble: one thread per tile word quantises all columns of the
+// word's four feature rows into the tile layout of phase A and stores whole words, so that a
+// warp's stores are full lines; the walk kernel then copies the tiles as in the single-problem
+// call and writes scores instead of ranking. A NaN goes right at every numeric split (x < t is
+// false), like +inf: the last bin. Slots past the last row get the neutral byte. Also clears
+// the abort flag.
+__global__ void __launch_bounds__(kWords)
 tile_rows_kernel(const float* __restrict__ feat, int64_t rows, FastView fv, uint8_t* __restrict__ tiles) {
   extern __shared__ float s_thr[];  // thresholds of every row
   __shared__ uint8_t s_r0[64], s_rc[64];
-  const int tid = threadIdx.x;
-  if (blockIdx.x == 0 && tid == 0) g_fast_abort = 0;
+  const int word = threadIdx.x;
+  if (blockIdx.x == 0 && word == 0) g_fast_abort = 0;
   {
     const float4* src = reinterpret_cast<const float4*>(fv.thr);
     float4* dst = reinterpret_cast<float4*>(s_thr);
-    for (int i = tid; i < fv.n_rows * (kThrPerRow / 4); i += blockDim.x) dst[i] = __ldg(src + i);
+    for (int i = word; i < fv.n_rows * (kThrPerRow / 4); i += kWords) dst[i] = __ldg(src + i);
   }
-  if (tid < 64) {
-    s_r0[tid] = fv.feat_row0[tid];
-    s_rc[tid] = fv.feat_rowcnt[tid];
+  if (word < 64) {
+    s_r0[word] = fv.feat_row0[word];
+    s_rc[word] = fv.feat_rowcnt[word];
   }
   __syncthreads();
-  const int64_t slot = static_cast<int64_t>(blockIdx.x) * blockDim.x + tid;
-  const int64_t blk = slot / kFastRows;
-  const int in = static_cast<int>(slot % kFastRows);
-  const int t = in % kFastThreads, r = in / kFastThreads;  // phase-A thread and its candidate
-  uint8_t* my = tiles + static_cast<size_t>(blk) * fv.n_rows * kRowStride + (t % kWords) * 4 + (t / kWords) * kFastR + r;
-  if (slot >= rows) {
-    for (int q = 0; q < fv.n_rows; ++q) my[q * kRowStride] = 0x80;
-    return;
+  // byte b of the word belongs to phase-A thread word + kWords * (b / 2), candidate b % 2
+  const int64_t base = static_cast<int64_t>(blockIdx.x) * kFastRows;
+  const float4* src[4];
+  bool live[4];
+#pragma unroll
+  for (int b = 0; b < 4; ++b) {
+    const int64_t slot = base + (b & 1) * kFastThreads + word + kWords * (b >> 1);
+    live[b] = slot < rows;
+    src[b] = reinterpret_cast<const float4*>(feat + (live[b] ? slot : 0) * KS_F_PAD);
   }
-  const float4* src = reinterpret_cast<const float4*>(feat + slot * KS_F_PAD);
-#pragma unroll 4
+  uint32_t* out = reinterpret_cast<uint32_t*>(tiles + static_cast<size_t>(blockIdx.x) * fv.n_rows * kRowStride) + word;
+#pragma unroll 2
   for (int q4 = 0; q4 < KS_F_PAD / 4; ++q4) {
-    const float4 v4 = __ldg(src + q4);
-    const float v[4] = {v4.x, v4.y, v4.z, v4.w};
+    float v[4][4];
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      const float4 t = __ldg(src[b] + q4);
+      v[b][0] = t.x; v[b][1] = t.y; v[b][2] = t.z; v[b][3] = t.w;
+    }
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const int col = 4 * q4 + j;
@@ -318,8 +325,16 @@ tile_rows_kernel(const float* __restrict__ feat, int64_t rows, FastView fv, uint
       const int r0 = s_r0[col], rc = s_rc[col];
       for (int q = 0; q < rc; ++q) {
         const float* T = s_thr + (r0 + q) * kThrPerRow;
-        const int bin = (v[j] != v[j] && !(T[kThrPerRow - 1] < 0.0f)) ? kThrPerRow - 1 : row_bin(T, v[j]);
-        my[(r0 + q) * kRowStride] = static_cast<uint8_t>(0x80 | bin);
+        const bool rank_row = T[kThrPerRow - 1] < 0.0f;
+        uint32_t w = 0;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+          const float x = v[b][j];
+          int bin = (x != x && !rank_row) ? kThrPerRow - 1 : row_bin(T, x);
+          if (!live[b]) bin = 0;
+          w |= static_cast<uint32_t>(0x80 | bin) << (8 * b);
+        }
+        out[static_cast<size_t>(r0 + q) * (kRowStride / 4)] = w;
       }
     }
   }
@@ -1071,7 +1086,7 @@ cudaError_t launch_score_fast(const ks_gpu_desc& desc, const GbdtModel& g, const
   for (int64_t first = 0; first < rows; first += kScoreBatchBlocks * kFastRows) {
     const int64_t n = rows - first < kScoreBatchBlocks * kFastRows ? rows - first : kScoreBatchBlocks * kFastRows;
     const int nblk = static_cast<int>((n + kFastRows - 1) / kFastRows);
-    tile_rows_kernel<<<nblk * (kFastRows / 256), 256, tthr, stream>>>(d_feat + first * KS_F_PAD, n, fv, tiles);
+    tile_rows_kernel<<<nblk, kWords, tthr, stream>>>(d_feat + first * KS_F_PAD, n, fv, tiles);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     SliceArgs sl{};
