@@ -355,7 +355,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=1, choices=[0, 1, 2, 3, 4])
-    ap.add_argument("--calls", type=int, default=20000, help="latency stream (workload 3): timed calls")
+    ap.add_argument("--calls", type=int, default=100000, help="latency stream (workload 3): timed calls")
     ap.add_argument("--ref-problems", type=int, default=16)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--problems", type=int, default=None,
