@@ -161,6 +161,29 @@ struct FastView {
   const uint8_t* feat_row0;    // [64] first row of each feature column
   const uint8_t* feat_rowcnt;  // [64] number of rows of each feature column
   const uint8_t* cand_rows;    // [kCombos][C][kCandRec] quantised candidate-only rows
+  const unsigned* pair_class;  // [kCombos][C] class of every candidate, or null (no memo)
+  const uint8_t* pair_tab;     // [P][kMemoCap][kMemoRec] per-pair tile bytes of every (problem, class)
+};
+
+// Memo of the per-pair rows. The per-pair columns see a candidate only through (T_M, T_N, T_K,
+// S, c_M, c_N) and its resident-block count, and a catalogue holds far fewer such classes than
+// candidates (the schedules and the instruction shape do not enter). Per call: every candidate
+// is given its class (a slot of a per-type-combination hash table, filled with atomicCAS; the
+// slot also remembers one member); per problem: the tile bytes of the per-pair rows are
+// evaluated once per occupied slot from that member; phase A then copies a 64-byte record
+// instead of evaluating 21 columns and searching their rows. A candidate whose fields do not
+// fit the key, or whose probe sequence runs out, has no class and is evaluated directly.
+constexpr int kMemoCap = 8192;  // slots per type combination (a power of two)
+constexpr int kMemoRec = 64;    // bytes per record = most per-pair rows a memoised model may have
+constexpr int kMemoMinProblems = 32;
+constexpr unsigned kNoClass = 0xFFFFFFFFu;
+struct MemoView {
+  unsigned long long* keys;  // [kCombos][kMemoCap], 0 = empty
+  int* count;                // [kCombos] occupied slots (the word after the keys)
+  int* dense;                // [kCombos][kMemoCap] the occupied slots, packed
+  int* reps;                 // [kCombos][kMemoCap] one member of the class
+  unsigned* cls;             // [kCombos][C]
+  uint8_t* tab;              // [P][kMemoCap][kMemoRec]
 };
 
 // ------------------------------------------------------------------------------------------
@@ -177,7 +200,7 @@ __global__ void combo_mask_kernel(const ks_problem* __restrict__ p, int P, unsig
 
 __global__ void __launch_bounds__(256)
 cand_rows_kernel(ks_gpu_desc desc, const ks_candidate* __restrict__ c, int C, const unsigned* mask_ptr,
-                 unsigned mask_value, FastView fv, uint8_t* __restrict__ out) {
+                 unsigned mask_value, FastView fv, uint8_t* __restrict__ out, MemoView memo) {
   extern __shared__ float s_cthr[];  // thresholds of the candidate-only rows
   __shared__ uint8_t s_r0[64], s_rc[64];
   const int combo = blockIdx.y;
@@ -219,6 +242,78 @@ cand_rows_kernel(ks_gpu_desc desc, const ks_candidate* __restrict__ c, int C, co
 #pragma unroll
   for (int q = 0; q < kCandRec / 16; ++q)
     if (q * 16 < fv.n_cand_rows) dst[q] = make_uint4(rec[4 * q], rec[4 * q + 1], rec[4 * q + 2], rec[4 * q + 3]);
+  if (memo.keys) {
+    unsigned cid = kNoClass;
+    const long long b_eff = resources(t, cand, desc).b_eff;
+    if (cand.tile_m < 4096 && cand.tile_n < 4096 && cand.tile_k < 4096 && cand.cluster_m < 32 &&
+        cand.cluster_n < 32 && b_eff < 64) {
+      const unsigned long long key =
+          (1ull << 63) | cand.tile_m | (static_cast<unsigned long long>(cand.tile_n) << 12) |
+          (static_cast<unsigned long long>(cand.tile_k) << 24) | (static_cast<unsigned long long>(cand.stages) << 36) |
+          (static_cast<unsigned long long>(cand.cluster_m) << 44) | (static_cast<unsigned long long>(cand.cluster_n) << 49) |
+          (static_cast<unsigned long long>(b_eff) << 54);
+      unsigned long long* K = memo.keys + static_cast<size_t>(combo) * kMemoCap;
+      unsigned h = static_cast<unsigned>((key * 0x9E3779B97F4A7C15ull) >> 40) & (kMemoCap - 1);
+      for (int probe = 0; probe < 64; ++probe) {
+        const unsigned long long prev = atomicCAS(K + h, 0ull, key);
+        if (prev == 0ull) memo.reps[static_cast<size_t>(combo) * kMemoCap + h] = i;  // this thread made the slot
+        if (prev == 0ull || prev == key) {
+          cid = h;
+          break;
+        }
+        h = (h + 1) & (kMemoCap - 1);
+      }
+    }
+    memo.cls[static_cast<size_t>(combo) * C + i] = cid;
+  }
+}
+
+// Packs the occupied slots of every type combination's table (one block per combination), so
+// that the per-problem kernel runs full warps over classes only.
+__global__ void __launch_bounds__(1024)
+memo_compact_kernel(MemoView memo) {
+  __shared__ int s_n;
+  const int combo = blockIdx.x;
+  if (threadIdx.x == 0) s_n = 0;
+  __syncthreads();
+  for (int slot = threadIdx.x; slot < kMemoCap; slot += 1024)
+    if (memo.keys[static_cast<size_t>(combo) * kMemoCap + slot] != 0ull)
+      memo.dense[static_cast<size_t>(combo) * kMemoCap + atomicAdd(&s_n, 1)] = slot;
+  __syncthreads();
+  if (threadIdx.x == 0) memo.count[combo] = s_n;
+}
+
+// Per problem: the tile bytes of the per-pair rows of every class, from the class's member.
+// grid (kMemoCap / 256, P); blocks past the number of classes leave at once.
+__global__ void __launch_bounds__(256)
+pair_table_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, const ks_candidate* __restrict__ c,
+                  FastView fv, MemoView memo) {
+  extern __shared__ float s_pthr[];  // thresholds of the per-pair rows
+  __shared__ ProblemTerms s_pt;
+  __shared__ uint8_t s_r0[64], s_rc[64];
+  const int prob = blockIdx.y, j = blockIdx.x * 256 + threadIdx.x;
+  const ks_problem pr = p[prob];
+  const int combo = (pr.dtype_ab & 3) * 4 + (pr.dtype_d & 3);
+  const int n_classes = memo.count[combo];
+  if (blockIdx.x * 256 >= n_classes) return;
+  const int slot = j < n_classes ? memo.dense[static_cast<size_t>(combo) * kMemoCap + j] : 0;
+  const unsigned long long key = j < n_classes ? 1ull : 0ull;
+  for (int i = threadIdx.x; i < fv.n_pair_rows * kThrPerRow; i += 256) s_pthr[i] = __ldg(fv.thr + i);
+  if (threadIdx.x < 64) {
+    s_r0[threadIdx.x] = fv.feat_row0[threadIdx.x];
+    s_rc[threadIdx.x] = fv.feat_rowcnt[threadIdx.x];
+  }
+  if (threadIdx.x == 0) problem_terms(pr, desc, s_pt);
+  __syncthreads();
+  if (key == 0ull) return;
+  const ks_candidate cand = c[memo.reps[static_cast<size_t>(combo) * kMemoCap + slot]];
+  const long long b_eff = resources(s_pt, cand, desc).b_eff;
+  uint8_t* rec = memo.tab + (static_cast<size_t>(prob) * kMemoCap + slot) * kMemoRec;
+  pair_columns<true>(s_pt, cand, desc, b_eff, [&](int col, float v) {
+    const int r0 = s_r0[col], rc = s_rc[col];
+    for (int q = 0; q < rc; ++q)
+      rec[r0 + q] = static_cast<uint8_t>(0x80 | bin_search(s_pthr + (r0 + q) * kThrPerRow, v));
+  });
 }
 
 // ------------------------------------------------------------------------------------------
@@ -353,7 +448,7 @@ __device__ __noinline__ void fill_tile(const ks_gpu_desc& desc, const ProblemTer
                                        const int64_t* __restrict__ seg_off, const int32_t* __restrict__ seg_idx,
                                        int C, int64_t lo, int64_t start, int64_t stop, const float* s_thr,
                                        const uint8_t* s_row0, const uint8_t* s_rowcnt, const uint8_t* s_pbin,
-                                       unsigned char* tile) {
+                                       unsigned char* tile, int prob) {
   const int tid = threadIdx.x;
   const int combo = pt.dtype_ab * 4 + pt.dtype_d;
 #pragma unroll 1
@@ -383,7 +478,26 @@ __device__ __noinline__ void fill_tile(const ks_gpu_desc& desc, const ProblemTer
     // problem-only rows
     dst = my + (fv.n_pair_rows + fv.n_cand_rows) * kRowStride;
     for (int q = 0; q < fv.n_prob_rows; ++q) dst[q * kRowStride] = s_pbin[q];
-    // per-pair rows
+    // per-pair rows: the record of the candidate's class, when there is one
+    if (fv.pair_class) {
+      const unsigned cid = __ldg(fv.pair_class + static_cast<size_t>(combo) * C + ci);
+      if (cid != kNoClass) {
+        const uint4* prec =
+            reinterpret_cast<const uint4*>(fv.pair_tab + (static_cast<size_t>(prob) * kMemoCap + cid) * kMemoRec);
+#pragma unroll
+        for (int v = 0; v < kMemoRec / 16; ++v) {
+          if (v * 16 < fv.n_pair_rows) {
+            const uint4 q = __ldg(prec + v);
+            const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+            for (int b = 0; b < 16; ++b)
+              if (v * 16 + b < fv.n_pair_rows)
+                my[(v * 16 + b) * kRowStride] = static_cast<unsigned char>(w[b >> 2] >> (8 * (b & 3)));
+          }
+        }
+        continue;
+      }
+    }
     featurize_pair(pt, cand, desc, [&](int col, float v) {
       if (feat_class(col) != 2) return;
       const int r0 = s_row0[col], rc = s_rowcnt[col];
@@ -513,7 +627,7 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
       }
       __syncthreads();
       fill_tile(desc, s_pt, c, fv, seg_off, seg_idx, C, lo, start, stop,
-                reinterpret_cast<const float*>(smem + kOffBuf0), s_row0, s_rowcnt, s_pbin, smem + kOffTile);
+                reinterpret_cast<const float*>(smem + kOffBuf0), s_row0, s_rowcnt, s_pbin, smem + kOffTile, prob);
     }
     __syncthreads();  // tile complete; the threshold table is no longer needed
 
@@ -939,6 +1053,17 @@ void fast_tiling(int P, int64_t per_problem, int* nblk, int* rows_per_cta) {
 
 size_t fast_scratch_bytes(int C) { return 256 + static_cast<size_t>(kCombos) * C * kCandRec; }
 
+// Memo of the per-pair rows (see MemoView): worth its per-problem table only for a batch of
+// problems, and only when the per-pair rows fit a record. 0 = not used.
+static size_t memo_fixed_bytes(int C) {
+  return static_cast<size_t>(kCombos) * kMemoCap * (sizeof(unsigned long long) + 2 * sizeof(int)) + 256 +
+         (static_cast<size_t>(kCombos) * C * sizeof(unsigned) + 255) / 256 * 256;
+}
+size_t fast_memo_bytes(const GbdtModel& g, int P, int C) {
+  if (P < kMemoMinProblems || C < 1 || g.n_pair_rows < 1 || g.n_pair_rows > kMemoRec) return 0;
+  return memo_fixed_bytes(C) + static_cast<size_t>(P) * kMemoCap * kMemoRec;
+}
+
 // Slice count of the single-problem call: as many tree slices as keep every CTA in the first
 // wave (one CTA per SM).
 int fast_slices(const GbdtModel& g, int64_t blocks) {
@@ -968,7 +1093,7 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
                                int nblk, int rows_per_cta, const int64_t* seg_off, const int32_t* seg_idx,
                                int k, unsigned long long* partial, void* scratch, int* status,
                                cudaStream_t stream, int64_t* launches, cudaEvent_t ev_begin,
-                               const FastSlice* slice) {
+                               const FastSlice* slice, void* memo_mem) {
   ks_problem pv{};
   if (p_by_value) pv = *p_by_value;
   const int uv = p_by_value != nullptr;
@@ -989,6 +1114,19 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
   unsigned* d_mask = static_cast<unsigned*>(scratch);
   uint8_t* d_rows = static_cast<uint8_t*>(scratch) + 256;
   fv.cand_rows = d_rows;
+  fv.pair_class = nullptr;
+  fv.pair_tab = nullptr;
+  MemoView memo{};
+  if (memo_mem && !p_by_value && fast_memo_bytes(g, P, C) != 0) {
+    char* m = static_cast<char*>(memo_mem);
+    const size_t slots = static_cast<size_t>(kCombos) * kMemoCap;
+    memo.keys = reinterpret_cast<unsigned long long*>(m);
+    memo.count = reinterpret_cast<int*>(m + slots * sizeof(unsigned long long));
+    memo.dense = reinterpret_cast<int*>(m + slots * sizeof(unsigned long long) + 256);
+    memo.reps = memo.dense + slots;
+    memo.cls = reinterpret_cast<unsigned*>(memo.reps + slots);
+    memo.tab = reinterpret_cast<uint8_t*>(m + memo_fixed_bytes(C));
+  }
 
   // candidate-only rows for the type combinations in use
   cudaError_t e = cudaSuccess;
@@ -1011,9 +1149,23 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
     ++*launches;
   } else if (C > 0) {
     const size_t cthr = sizeof(float) * kThrPerRow * (g.n_cand_rows > 0 ? g.n_cand_rows : 1);
+    if (memo.keys) {
+      e = cudaMemsetAsync(memo.keys, 0, static_cast<size_t>(kCombos) * kMemoCap * sizeof(unsigned long long), stream);
+      if (e != cudaSuccess) return e;
+    }
     cand_rows_kernel<<<dim3((C + 255) / 256, kCombos), 256, cthr, stream>>>(desc, d_c, C, uv ? nullptr : d_mask,
-                                                                            mask_value, fv, d_rows);
+                                                                            mask_value, fv, d_rows, memo);
     ++*launches;
+    if (memo.keys) {
+      const size_t pthr = sizeof(float) * kThrPerRow * g.n_pair_rows;
+      e = ensure_dynamic_smem(reinterpret_cast<const void*>(&pair_table_kernel), pthr);
+      if (e != cudaSuccess) return e;
+      memo_compact_kernel<<<kCombos, 1024, 0, stream>>>(memo);
+      pair_table_kernel<<<dim3(kMemoCap / 256, P), 256, pthr, stream>>>(desc, d_p, d_c, fv, memo);
+      *launches += 2;
+      fv.pair_class = memo.cls;
+      fv.pair_tab = memo.tab;
+    }
   }
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;

@@ -184,13 +184,14 @@ cudaError_t launch_remap_indices(int32_t* d_idx, long long n, const int32_t* d_m
 // Quantised tree path: blocks per problem for `per_problem` rows, and the launch itself.
 void fast_tiling(int P, int64_t per_problem, int* nblk, int* rows_per_cta);
 size_t fast_scratch_bytes(int C);  // per-call table of candidate-only rows
+size_t fast_memo_bytes(const GbdtModel& g, int P, int C);  // memo of the per-pair rows (0: not used)
 void free_fast_gbdt(GbdtModel& m);
 cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, const ks_problem* d_p,
                                const ks_problem* p_by_value, int P, const ks_candidate* d_c, int C,
                                int nblk, int rows_per_cta, const int64_t* seg_off, const int32_t* seg_idx,
                                int k, unsigned long long* partial, void* scratch, int* status,
                                cudaStream_t stream, int64_t* launches, cudaEvent_t ev_begin,
-                               const FastSlice* slice = nullptr);
+                               const FastSlice* slice = nullptr, void* memo_mem = nullptr);
 int fast_slices(const GbdtModel& g, int64_t blocks);
 // ks_score with a qualifying ensemble: tiles quantised from the feature rows, then the same walk.
 size_t score_fast_scratch_bytes(const GbdtModel& g, int64_t rows);

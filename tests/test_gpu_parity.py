@@ -531,6 +531,41 @@ def test_select_other_model_shapes(ks, ctx, case):
     assert np.array_equal(hi_.numpy(), idx[2])
 
 
+def test_select_pair_row_memo_paths(ks, ctx):
+    """Batches of 32 problems or more copy the per-pair tile rows from a per-(problem, class)
+    table, a class being (T_M, T_N, T_K, S, c_M, c_N, resident blocks). Cases: mixed element
+    types (one class table per combination), candidates whose fields do not fit the class key
+    (evaluated directly), more classes than the table holds (the late ones evaluated directly),
+    and segments."""
+    # mixed element types, dense, a few candidates outside the key's range
+    w = wl.make_workload(2, P=40, seg=64, trees=30, depth=6)
+    cand = w.candidates[:2500].copy()
+    cand["tile_m"][::97] = 4096 + 64
+    cand["tile_k"][5::211] = 8192
+    w = wl.Workload("memo_mixed", DESC, w.problems, cand, 10, gbdt=w.gbdt)
+    model = ctx.model_create_gbdt(*w.gbdt)
+    idx, sc = run_select(ks, ctx, w, model)
+    check_select(w, idx, sc, TOL_GBDT)
+    # more distinct classes than slots: 12,000 different tile shapes
+    i = np.arange(12000)
+    big = np.zeros(12000, wl.CANDIDATE_DT)
+    big["tile_m"], big["tile_n"], big["tile_k"] = 16 * (1 + i % 16), 8 * (1 + (i // 16) % 32), 16 * (1 + (i // 512) % 32)
+    big["instr_n"], big["instr_m"], big["instr_k"] = big["tile_n"], 64, 16
+    big["stages"], big["cluster_m"], big["cluster_n"] = 2 + i % 3, 1 + (i // 7) % 2, 1
+    big["kernel_sched"], big["epi_sched"], big["tile_sched"] = i % 4, i % 3, i % 2
+    assert len(np.unique(big[["tile_m", "tile_n", "tile_k", "stages", "cluster_m"]])) > 8192
+    w1 = wl.make_workload(1, P=33, C=10, trees=12, depth=5)
+    wb = wl.Workload("memo_overflow", DESC, w1.problems, big, 10, gbdt=w1.gbdt)
+    model = ctx.model_create_gbdt(*w1.gbdt)
+    idx, sc = run_select(ks, ctx, wb, model)
+    check_select(wb, idx, sc, TOL_GBDT)
+    # segments over the pool
+    ws = wl.make_workload(2, P=48, seg=700, trees=20, depth=5)
+    model = ctx.model_create_gbdt(*ws.gbdt)
+    idx, sc = run_select(ks, ctx, ws, model)
+    check_select(ws, idx, sc, TOL_GBDT)
+
+
 def test_select_ridge_and_paper_sized_models(ks, ctx):
     """The linear (ridge) scorer as a one-layer model, and models of the sizes the paper ships:
     916 trees of depth 7, and the largest MLP preset 64-1024-1024-512-256-1."""
