@@ -507,8 +507,11 @@ def main():
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, per launch, from the
-# ncu summaries under profiles/ (None until a capture exists for that workload).
-TRAFFIC_BYTES = {1: 16.6e6, 4: 5.7e6}
+# ncu summaries under profiles/ (None until a capture exists for that workload). Config 1: the
+# 48-problem capture (17.6 MB) splits into 7.4 MB that do not depend on the number of problems
+# and 0.21 MB per problem (the problem's table of per-pair tile rows, read back through L2),
+# plus the partial lists of the full-size launch (9.7 MB): 7.4 + 1,024 x 0.21 + 9.7.
+TRAFFIC_BYTES = {1: 234e6, 4: 5.7e6}
 
 if __name__ == "__main__":
     main()
