@@ -19,9 +19,16 @@
 //   Rows are grouped by what their feature depends on. Candidate-only rows (given the
 //   problem's element types) are quantised once per call by cand_rows_kernel into a table
 //   indexed by (type combination, candidate); problem-only rows once per CTA; only the
-//   per-pair rows are computed and searched for every pair.
+//   per-pair rows are computed and searched for every pair - or, in a batch of problems, once
+//   per (problem, class of candidates that look alike to the per-pair columns) and copied
+//   (see MemoView).
 //
-// Kernel (one CTA = one problem x up to kFastRows candidates, 1024 threads)
+// Other entries into the same walk
+//   single-problem call: the trees are split over several CTAs per candidate block (slices),
+//   the tiles are built once by tile_one_kernel; scoring call (ks_score): tiles are quantised
+//   from given feature rows by tile_rows_kernel and the scores are stored instead of ranked.
+//
+// Kernel (one CTA = one problem x up to kFastRows candidates, kFastThreads threads, two CTAs per SM)
 //   phase A  fill the [row][candidate] byte tile. A 32-bit word of a row holds the four
 //            candidates that share a lane slot, so a warp's byte loads of any mix of rows
 //            touch 32 distinct banks and one word load serves four candidates;
