@@ -259,8 +259,8 @@ ks_status ks_score(ks_ctx* ctx, const float* d_features, int64_t rows, const ks_
  * matrix and the scores are never written to memory. `pairs` as in ks_featurize. The call
  * sizes the context's workspace (owned by the context, grown on demand, which synchronises the
  * device when it happens): partial lists, a per-call table of 16 x C x 64 bytes, and, for a
- * tree model on a batch of 32 problems or more, P x 512 KiB for the tables of per-pair tile
- * rows (KS_ERR_OOM if that cannot be had). */
+ * tree model on a batch of 32 to 8,192 problems, P x 512 KiB for the tables of per-pair tile
+ * rows (KS_ERR_OOM if the workspace cannot be had). */
 ks_status ks_select(ks_ctx* ctx, const ks_problem* d_p, int P, const ks_candidate* d_c, int C,
                     const int64_t* d_seg_offsets, const int32_t* d_seg_index, int64_t pairs,
                     const ks_model* model, int k, int32_t* d_topk_idx, float* d_topk_score,

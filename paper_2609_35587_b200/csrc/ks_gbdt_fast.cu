@@ -183,6 +183,7 @@ struct FastView {
 constexpr int kMemoCap = 8192;  // slots per type combination (a power of two)
 constexpr int kMemoRec = 64;    // bytes per record = most per-pair rows a memoised model may have
 constexpr int kMemoMinProblems = 32;
+constexpr int kMemoMaxProblems = 8192;  // 4 GiB of records at most; larger batches evaluate in place
 constexpr unsigned kNoClass = 0xFFFFFFFFu;
 struct MemoView {
   unsigned long long* keys;  // [kCombos][kMemoCap], 0 = empty
@@ -1067,7 +1068,7 @@ static size_t memo_fixed_bytes(int C) {
          (static_cast<size_t>(kCombos) * C * sizeof(unsigned) + 255) / 256 * 256;
 }
 size_t fast_memo_bytes(const GbdtModel& g, int P, int C) {
-  if (P < kMemoMinProblems || C < 1 || g.n_pair_rows < 1 || g.n_pair_rows > kMemoRec) return 0;
+  if (P < kMemoMinProblems || P > kMemoMaxProblems || C < 1 || g.n_pair_rows < 1 || g.n_pair_rows > kMemoRec) return 0;
   return memo_fixed_bytes(C) + static_cast<size_t>(P) * kMemoCap * kMemoRec;
 }
 
