@@ -674,8 +674,10 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
       // + 4 bit for every level, and after the last level A points at the walk's leaf.
       const uint32_t k0 = 4u * tpc - buf;  // modulo 2^32, like the additions it enters
       const uint32_t lvlL = buf + 4u * tpc * kTop;  // first node of level L
-#pragma unroll 1
-      for (int t = half * half_trees; t < (half + 1) * half_trees; ++t) {
+      const int t_first = half * half_trees;
+#pragma unroll 4
+      for (int tt = 0; tt < half_trees; ++tt) {
+        const int t = t_first + tt;
         uint32_t a[4];
         if (L == 0) {
 #pragma unroll
