@@ -57,6 +57,16 @@ def test_strict_less_than_goes_left():
     assert s.tolist() == [1.0, 2.0, 2.0]
 
 
+def test_non_finite_values_at_a_numeric_split():
+    """Model A sends a row left iff x < t: a NaN and +inf are not less than anything (right),
+    -inf is less than every finite threshold (left)."""
+    nodes = make_tree([(5, 2.0, 1), (None, 1.0, 0), (None, 2.0, 0)])
+    x = np.zeros((3, 64), np.float32)
+    x[:, 5] = [np.nan, np.inf, -np.inf]
+    s = oracle.score_gbdt(x, np.array([0, 3]), nodes)
+    assert s.tolist() == [2.0, 2.0, 1.0]
+
+
 def brute_force_score(x, off, nodes, base=0.0):
     """Explicit loop evaluation, pure Python, fp64 sum in tree order."""
     out = []
