@@ -121,6 +121,15 @@ def _stream():
     return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
 
 
+def problem_structs(problems: np.ndarray):
+    """The problem records as an array of by-value arguments for `Context.select_one_caller`
+    (the 16-byte record is the C struct: a byte copy)."""
+    a = np.ascontiguousarray(problems).reshape(-1)
+    if a.dtype.itemsize != ctypes.sizeof(_Problem):
+        raise ValueError("expected ks_problem records")
+    return (_Problem * len(a)).from_buffer_copy(a.tobytes())
+
+
 def to_device(records: np.ndarray, device) -> torch.Tensor:
     """A numpy record / plain array as a device tensor of raw bytes (records) or values."""
     a = np.ascontiguousarray(records)
@@ -269,6 +278,26 @@ class Context:
                             pairs, model._h, k, _dptr(out_idx), _dptr(out_score), _stream())
         self._check(st, "ks_select")
         return out_idx, out_score
+
+    def select_one_caller(self, d_c, C, model: Model, k, h_idx=None, h_score=None):
+        """For a stream of single problems: resolves the pointers, the model handle and the
+        current stream once and returns f(p) -> (h_idx, h_score), where p is one element of
+        `problem_structs(...)`. Per call only ks_select_one itself runs; the result tensors are
+        reused from call to call."""
+        if h_idx is None:
+            h_idx = torch.empty(k, dtype=torch.int32).pin_memory()
+            h_score = torch.empty(k, dtype=torch.float32).pin_memory()
+        fn, check = _lib.ks_select_one, self._check
+        args = (_dptr(d_c), C, model._h, k, _hptr(h_idx), _hptr(h_score), _stream())
+        ctx_h = self._h
+        keep = (d_c, model, h_idx, h_score)  # the closure keeps the buffers alive
+
+        def call(p):
+            st = fn(ctx_h, p, *args)
+            if st != KS_OK:
+                check(st, "ks_select_one")
+            return keep[2], keep[3]
+        return call
 
     def select_one(self, problem: np.ndarray, d_c, C, model: Model, k, h_idx=None, h_score=None):
         r = np.ascontiguousarray(problem).reshape(-1)[0]

@@ -113,6 +113,13 @@ def test_config3_latency_stream_sample(ks, ctx):
         _, _, allsc = oracle.select(w.problems[i:i + 1], w.candidates, w.desc, w.k, gbdt=w.gbdt, want_scores=True)
         ok, msg = topk_accept(hi.numpy(), hs.numpy(), allsc, np.arange(C, dtype=np.int32), w.k, TOL_GBDT)
         assert ok, f"call {i}: {msg}"
+    # the prepared caller (the form bench.py times) is the same call
+    call = ctx.select_one_caller(d_c, C, model, w.k)
+    structs = ks.problem_structs(w.problems[:300])
+    for i in [0, 7, 299]:
+        hi, hs = ctx.select_one(w.problems[i:i + 1], d_c, C, model, w.k)
+        ci, cs = call(structs[i])
+        assert np.array_equal(ci.numpy(), hi.numpy()) and np.array_equal(cs.numpy(), hs.numpy())
 
 
 def test_full_size_paper_forms(ks, ctx):
