@@ -547,7 +547,10 @@ __device__ __forceinline__ uint32_t path_step(uint32_t a, uint32_t cb_r, uint32_
   return nx;
 }
 
-template <int L, int NP>  // L levels evaluated word-wise; NP path levels unrolled (-1: runtime count)
+// L levels evaluated word-wise; NP path levels unrolled (-1: runtime count); kCompact: the top
+// levels' constants travel as one 32-bit word per node (row offset << 8 | j + 1) instead of a
+// (row offset, replicated j + 1) pair, so that twice as many trees keep their word-wise levels.
+template <int L, int NP, bool kCompact = false>
 __global__ void __launch_bounds__(kFastThreads, 2)
 select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_problem p_value, int use_value,
                    const ks_candidate* __restrict__ c, int P, int C, int nblk, int rows_per_cta,
@@ -686,10 +689,19 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
           // Word-wise evaluation of the top L levels for the four candidates of this word.
           // A tile byte is 0x80 | bin and a node constant (j + 1) in every byte, so byte r of
           // d[n] keeps its top bit iff candidate r goes right at node n; no byte borrows.
-          const uint2* tw = top.w + static_cast<size_t>(ch * tpc + t) * kTop;
           uint32_t d[kTop > 0 ? kTop : 1];
+          if (kCompact) {
+            const uint32_t* tw = reinterpret_cast<const uint32_t*>(top.w) + static_cast<size_t>(ch * tpc + t) * kTop;
 #pragma unroll
-          for (int n = 0; n < kTop; ++n) d[n] = lds_u32(cb + tw[n].x) - tw[n].y;
+            for (int n = 0; n < kTop; ++n) {
+              const uint32_t v = tw[n];
+              d[n] = lds_u32(cb + (v >> 8)) - __byte_perm(v, 0u, 0u);
+            }
+          } else {
+            const uint2* tw = top.w + static_cast<size_t>(ch * tpc + t) * kTop;
+#pragma unroll
+            for (int n = 0; n < kTop; ++n) d[n] = lds_u32(cb + tw[n].x) - tw[n].y;
+          }
           uint32_t x = d[0] & 0x80808080u;  // path bits: level 0 in bit 7 of each byte, ...
           if (L >= 2) {
             const uint32_t s1 = byte_select(d[0], d[2], d[1]);
@@ -939,6 +951,12 @@ cudaError_t build_fast_gbdt(GbdtModel& m, int n_trees, const int64_t* off, const
   const int chunk_words = (tpc * per_tree_words + 3) / 4 * 4;  // bulk copies move multiples of 16 bytes
   int L = D < 3 ? D : 3;  // levels whose nodes travel as kernel-parameter constants
   while (L > 0 && static_cast<int64_t>(n_chunks) * tpc * ((1 << L) - 1) > kFastTopPairs) --L;
+  // three levels in the compact form (one word per node) when the pair form would leave fewer
+  bool compact = false;
+  if (L < 3 && D >= 3 && static_cast<int64_t>(n_chunks) * tpc * 7 <= 2 * kFastTopPairs) {
+    L = 3;
+    compact = true;
+  }
   const int n_top = (1 << L) - 1;
   std::vector<uint32_t> chunks(static_cast<size_t>(n_chunks) * chunk_words);
   FastTopParams* top = new (std::nothrow) FastTopParams();
@@ -999,7 +1017,11 @@ cudaError_t build_fast_gbdt(GbdtModel& m, int n_trees, const int64_t* off, const
             }
           }
           lvl[tt * (1 << l) + i] = word;
-          if (l < L) top->w[static_cast<size_t>(t) * n_top + ((1 << l) - 1) + i] = tw;
+          if (l < L) {
+            const size_t at = static_cast<size_t>(t) * n_top + ((1 << l) - 1) + i;
+            if (compact) reinterpret_cast<uint32_t*>(top->w)[at] = (tw.x << 8) | (tw.y & 0xFFu);
+            else top->w[at] = tw;
+          }
           nsrc[2 * i] = ls;
           nsrc[2 * i + 1] = rs;
           ncarry[2 * i] = lc;
@@ -1029,6 +1051,7 @@ cudaError_t build_fast_gbdt(GbdtModel& m, int n_trees, const int64_t* off, const
   }
   m.h_top = top;
   m.top_levels = L;
+  m.top_compact = compact;
   m.fast = true;
   m.fast_depth = D;
   m.n_qrows = n_rows;
@@ -1084,15 +1107,15 @@ int fast_slices(const GbdtModel& g, int64_t blocks) {
   return static_cast<int>(s < 1 ? 1 : s);
 }
 
-template <int L, int NP>
+template <int L, int NP, bool kCompact = false>
 static cudaError_t launch_ln(const ks_gpu_desc& desc, const ks_problem* d_p, const ks_problem& pv, int uv, int P,
                              const ks_candidate* d_c, int C, int nblk, int rows_per_cta, const int64_t* seg_off,
                              const int32_t* seg_idx, const FastView& fv, int k, unsigned long long* partial,
                              int* status, const SliceArgs& sl, const FastTopParams& top, cudaStream_t stream) {
   const size_t smem = kOffTile + static_cast<size_t>(fv.n_rows) * kRowStride;
-  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(&select_fast_kernel<L, NP>), smem);
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(&select_fast_kernel<L, NP, kCompact>), smem);
   if (e != cudaSuccess) return e;
-  select_fast_kernel<L, NP><<<static_cast<unsigned>(static_cast<int64_t>(P) * nblk * sl.n_slices), kFastThreads, smem,
+  select_fast_kernel<L, NP, kCompact><<<static_cast<unsigned>(static_cast<int64_t>(P) * nblk * sl.n_slices), kFastThreads, smem,
                               stream>>>(desc, d_p, pv, uv, d_c, P, C, nblk, rows_per_cta, seg_off, seg_idx, fv, k,
                                         partial, status, sl, top);
   return cudaGetLastError();
@@ -1199,6 +1222,14 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
   ++*launches;
 #define KS_GO(LL, NN) \
   return launch_ln<LL, NN>(desc, d_p, pv, uv, P, d_c, C, nblk, rows_per_cta, seg_off, seg_idx, fv, k, partial, status, sl, top, stream)
+  if (g.top_compact) {
+#define KS_GOC(NN) \
+  return launch_ln<3, NN, true>(desc, d_p, pv, uv, P, d_c, C, nblk, rows_per_cta, seg_off, seg_idx, fv, k, partial, status, sl, top, stream)
+    if (np == 5) KS_GOC(5);
+    if (np == 4) KS_GOC(4);
+    KS_GOC(-1);
+#undef KS_GOC
+  }
   if (L == 3 && np == 5) KS_GO(3, 5);
   if (L == 3 && np == 3) KS_GO(3, 3);
   if (L == 2 && np == 6) KS_GO(2, 6);
@@ -1259,7 +1290,10 @@ cudaError_t launch_score_fast(const ks_gpu_desc& desc, const GbdtModel& g, const
 #define KS_GO(LL, NN)                                                                                          \
   e = launch_ln<LL, NN>(desc, nullptr, pv, 1, 1, nullptr, static_cast<int>(n), nblk, kFastRows, nullptr, nullptr, \
                         fv, 0, nullptr, status, sl, top, stream)
-    if (L == 3 && np == 5) KS_GO(3, 5);
+    if (g.top_compact && np == 5) e = launch_ln<3, 5, true>(desc, nullptr, pv, 1, 1, nullptr, static_cast<int>(n), nblk, kFastRows, nullptr, nullptr, fv, 0, nullptr, status, sl, top, stream);
+    else if (g.top_compact && np == 4) e = launch_ln<3, 4, true>(desc, nullptr, pv, 1, 1, nullptr, static_cast<int>(n), nblk, kFastRows, nullptr, nullptr, fv, 0, nullptr, status, sl, top, stream);
+    else if (g.top_compact) e = launch_ln<3, -1, true>(desc, nullptr, pv, 1, 1, nullptr, static_cast<int>(n), nblk, kFastRows, nullptr, nullptr, fv, 0, nullptr, status, sl, top, stream);
+    else if (L == 3 && np == 5) KS_GO(3, 5);
     else if (L == 3 && np == 3) KS_GO(3, 3);
     else if (L == 2 && np == 6) KS_GO(2, 6);
     else if (L == 2 && np == 5) KS_GO(2, 5);

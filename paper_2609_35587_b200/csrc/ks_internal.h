@@ -60,6 +60,7 @@ struct GbdtModel {
   int n_qrows = 0;             // quantised feature rows (a feature, or a 127-threshold slice)
   int n_pair_rows = 0, n_cand_rows = 0, n_prob_rows = 0;  // rows by what their feature depends on
   int top_levels = 0;          // levels whose nodes also live in h_top
+  bool top_compact = false;    // h_top holds one 32-bit word per node instead of a pair
   FastTopParams* h_top = nullptr;  // host copy, passed by value at every launch
   int tpc = 0;                 // trees per chunk
   int n_chunks = 0;
