@@ -49,6 +49,7 @@
 
 #include "ks_features.cuh"
 #include "ks_internal.h"
+#include "ks_memo.cuh"
 #include "ks_topk.cuh"
 
 namespace ks {
@@ -172,27 +173,10 @@ struct FastView {
   const uint8_t* pair_tab;     // [P][kMemoCap][kMemoRec] per-pair tile bytes of every (problem, class)
 };
 
-// Memo of the per-pair rows. The per-pair columns see a candidate only through (T_M, T_N, T_K,
-// S, c_M, c_N) and its resident-block count, and a catalogue holds far fewer such classes than
-// candidates (the schedules and the instruction shape do not enter). Per call: every candidate
-// is given its class (a slot of a per-type-combination hash table, filled with atomicCAS; the
-// slot also remembers one member); per problem: the tile bytes of the per-pair rows are
-// evaluated once per occupied slot from that member; phase A then copies a 64-byte record
-// instead of evaluating 21 columns and searching their rows. A candidate whose fields do not
-// fit the key, or whose probe sequence runs out, has no class and is evaluated directly.
-constexpr int kMemoCap = 8192;  // slots per type combination (a power of two)
-constexpr int kMemoRec = 64;    // bytes per record = most per-pair rows a memoised model may have
-constexpr int kMemoMinProblems = 32;
-constexpr int kMemoMaxProblems = 8192;  // 4 GiB of records at most; larger batches evaluate in place
-constexpr unsigned kNoClass = 0xFFFFFFFFu;
-struct MemoView {
-  unsigned long long* keys;  // [kCombos][kMemoCap], 0 = empty
-  int* count;                // [kCombos] occupied slots (the word after the keys)
-  int* dense;                // [kCombos][kMemoCap] the occupied slots, packed
-  int* reps;                 // [kCombos][kMemoCap] one member of the class
-  unsigned* cls;             // [kCombos][C]
-  uint8_t* tab;              // [P][kMemoCap][kMemoRec]
-};
+// Memo of the per-pair rows (classes: ks_memo.cuh). Per problem the tile bytes of the per-pair
+// rows are evaluated once per class from the class's member; phase A then copies a 64-byte
+// record instead of evaluating 21 columns and searching their rows.
+constexpr int kMemoRec = 64;  // bytes per record = most per-pair rows a memoised model may have
 
 // ------------------------------------------------------------------------------------------
 // candidate-only rows, once per call
@@ -250,30 +234,8 @@ cand_rows_kernel(ks_gpu_desc desc, const ks_candidate* __restrict__ c, int C, co
 #pragma unroll
   for (int q = 0; q < kCandRec / 16; ++q)
     if (q * 16 < fv.n_cand_rows) dst[q] = make_uint4(rec[4 * q], rec[4 * q + 1], rec[4 * q + 2], rec[4 * q + 3]);
-  if (memo.keys) {
-    unsigned cid = kNoClass;
-    const long long b_eff = resources(t, cand, desc).b_eff;
-    if (cand.tile_m < 4096 && cand.tile_n < 4096 && cand.tile_k < 4096 && cand.cluster_m < 32 &&
-        cand.cluster_n < 32 && b_eff < 64) {
-      const unsigned long long key =
-          (1ull << 63) | cand.tile_m | (static_cast<unsigned long long>(cand.tile_n) << 12) |
-          (static_cast<unsigned long long>(cand.tile_k) << 24) | (static_cast<unsigned long long>(cand.stages) << 36) |
-          (static_cast<unsigned long long>(cand.cluster_m) << 44) | (static_cast<unsigned long long>(cand.cluster_n) << 49) |
-          (static_cast<unsigned long long>(b_eff) << 54);
-      unsigned long long* K = memo.keys + static_cast<size_t>(combo) * kMemoCap;
-      unsigned h = static_cast<unsigned>((key * 0x9E3779B97F4A7C15ull) >> 40) & (kMemoCap - 1);
-      for (int probe = 0; probe < 64; ++probe) {
-        const unsigned long long prev = atomicCAS(K + h, 0ull, key);
-        if (prev == 0ull) memo.reps[static_cast<size_t>(combo) * kMemoCap + h] = i;  // this thread made the slot
-        if (prev == 0ull || prev == key) {
-          cid = h;
-          break;
-        }
-        h = (h + 1) & (kMemoCap - 1);
-      }
-    }
-    memo.cls[static_cast<size_t>(combo) * C + i] = cid;
-  }
+  if (memo.keys)
+    memo.cls[static_cast<size_t>(combo) * C + i] = memo_assign(memo, combo, i, cand, resources(t, cand, desc).b_eff);
 }
 
 // Packs the occupied slots of every type combination's table (one block per combination), so
@@ -316,7 +278,7 @@ pair_table_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, const ks_c
   if (key == 0ull) return;
   const ks_candidate cand = c[memo.reps[static_cast<size_t>(combo) * kMemoCap + slot]];
   const long long b_eff = resources(s_pt, cand, desc).b_eff;
-  uint8_t* rec = memo.tab + (static_cast<size_t>(prob) * kMemoCap + slot) * kMemoRec;
+  uint8_t* rec = static_cast<uint8_t*>(memo.tab) + (static_cast<size_t>(prob) * kMemoCap + slot) * kMemoRec;
   pair_columns<true>(s_pt, cand, desc, b_eff, [&](int col, float v) {
     const int r0 = s_r0[col], rc = s_rc[col];
     for (int q = 0; q < rc; ++q)
@@ -1088,10 +1050,30 @@ size_t fast_scratch_bytes(int C) { return 256 + static_cast<size_t>(kCombos) * C
 
 // Memo of the per-pair rows (see MemoView): worth its per-problem table only for a batch of
 // problems, and only when the per-pair rows fit a record. 0 = not used.
-static size_t memo_fixed_bytes(int C) {
-  return static_cast<size_t>(kCombos) * kMemoCap * (sizeof(unsigned long long) + 2 * sizeof(int)) + 256 +
-         (static_cast<size_t>(kCombos) * C * sizeof(unsigned) + 255) / 256 * 256;
+size_t memo_fixed_bytes(int C) {
+  return static_cast<size_t>(kMemoCombos) * kMemoCap * (sizeof(unsigned long long) + 2 * sizeof(int)) + 256 +
+         (static_cast<size_t>(kMemoCombos) * C * sizeof(unsigned) + 255) / 256 * 256;
 }
+MemoView memo_view(void* mem, int C) {
+  char* m = static_cast<char*>(mem);
+  const size_t slots = static_cast<size_t>(kMemoCombos) * kMemoCap;
+  MemoView v{};
+  v.keys = reinterpret_cast<unsigned long long*>(m);
+  v.count = reinterpret_cast<int*>(m + slots * sizeof(unsigned long long));
+  v.dense = reinterpret_cast<int*>(m + slots * sizeof(unsigned long long) + 256);
+  v.reps = v.dense + slots;
+  v.cls = reinterpret_cast<unsigned*>(v.reps + slots);
+  v.tab = m + memo_fixed_bytes(C);
+  return v;
+}
+cudaError_t memo_clear(const MemoView& memo, cudaStream_t stream) {
+  return cudaMemsetAsync(memo.keys, 0, static_cast<size_t>(kMemoCombos) * kMemoCap * sizeof(unsigned long long), stream);
+}
+cudaError_t memo_compact(const MemoView& memo, cudaStream_t stream) {
+  memo_compact_kernel<<<kMemoCombos, 1024, 0, stream>>>(memo);
+  return cudaGetLastError();
+}
+
 size_t fast_memo_bytes(const GbdtModel& g, int P, int C) {
   if (P < kMemoMinProblems || P > kMemoMaxProblems || C < 1 || g.n_pair_rows < 1 || g.n_pair_rows > kMemoRec) return 0;
   return memo_fixed_bytes(C) + static_cast<size_t>(P) * kMemoCap * kMemoRec;
@@ -1150,16 +1132,7 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
   fv.pair_class = nullptr;
   fv.pair_tab = nullptr;
   MemoView memo{};
-  if (memo_mem && !p_by_value && fast_memo_bytes(g, P, C) != 0) {
-    char* m = static_cast<char*>(memo_mem);
-    const size_t slots = static_cast<size_t>(kCombos) * kMemoCap;
-    memo.keys = reinterpret_cast<unsigned long long*>(m);
-    memo.count = reinterpret_cast<int*>(m + slots * sizeof(unsigned long long));
-    memo.dense = reinterpret_cast<int*>(m + slots * sizeof(unsigned long long) + 256);
-    memo.reps = memo.dense + slots;
-    memo.cls = reinterpret_cast<unsigned*>(memo.reps + slots);
-    memo.tab = reinterpret_cast<uint8_t*>(m + memo_fixed_bytes(C));
-  }
+  if (memo_mem && !p_by_value && fast_memo_bytes(g, P, C) != 0) memo = memo_view(memo_mem, C);
 
   // candidate-only rows for the type combinations in use
   cudaError_t e = cudaSuccess;
@@ -1183,7 +1156,7 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
   } else if (C > 0) {
     const size_t cthr = sizeof(float) * kThrPerRow * (g.n_cand_rows > 0 ? g.n_cand_rows : 1);
     if (memo.keys) {
-      e = cudaMemsetAsync(memo.keys, 0, static_cast<size_t>(kCombos) * kMemoCap * sizeof(unsigned long long), stream);
+      e = memo_clear(memo, stream);
       if (e != cudaSuccess) return e;
     }
     cand_rows_kernel<<<dim3((C + 255) / 256, kCombos), 256, cthr, stream>>>(desc, d_c, C, uv ? nullptr : d_mask,
@@ -1193,11 +1166,12 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
       const size_t pthr = sizeof(float) * kThrPerRow * g.n_pair_rows;
       e = ensure_dynamic_smem(reinterpret_cast<const void*>(&pair_table_kernel), pthr);
       if (e != cudaSuccess) return e;
-      memo_compact_kernel<<<kCombos, 1024, 0, stream>>>(memo);
+      e = memo_compact(memo, stream);
+      if (e != cudaSuccess) return e;
       pair_table_kernel<<<dim3(kMemoCap / 256, P), 256, pthr, stream>>>(desc, d_p, d_c, fv, memo);
       *launches += 2;
       fv.pair_class = memo.cls;
-      fv.pair_tab = memo.tab;
+      fv.pair_tab = static_cast<const uint8_t*>(memo.tab);
     }
   }
   e = cudaGetLastError();

@@ -9,6 +9,7 @@
 
 #include "ks_features.cuh"
 #include "ks_internal.h"
+#include "ks_memo.cuh"
 #include "ks_topk.cuh"
 
 namespace ks {
@@ -416,7 +417,8 @@ __device__ __forceinline__ float ridge_level(const float (&lut)[4], float v) {
 // per (type combination, candidate): (candidate-only part of the sum, resident-block count)
 __global__ void __launch_bounds__(256)
 ridge_cand_kernel(ks_gpu_desc desc, const ks_candidate* __restrict__ c, int C, const unsigned* mask_ptr,
-                  unsigned mask_value, const __grid_constant__ RidgeParams prm, float2* __restrict__ out) {
+                  unsigned mask_value, const __grid_constant__ RidgeParams prm, float2* __restrict__ out,
+                  MemoView memo) {
   const int combo = blockIdx.y;
   const unsigned mask = mask_ptr ? *mask_ptr : mask_value;
   if (!((mask >> combo) & 1u)) return;
@@ -436,7 +438,33 @@ ridge_cand_kernel(ks_gpu_desc desc, const ks_candidate* __restrict__ c, int C, c
     if (col == 17) s += ridge_level(prm.lut17, v);
     if (col == 18) s += ridge_level(prm.lut18, v);
   });
-  out[static_cast<size_t>(combo) * C + i] = make_float2(s, static_cast<float>(resources(t, cand, desc).b_eff));
+  const long long b_eff = resources(t, cand, desc).b_eff;
+  out[static_cast<size_t>(combo) * C + i] = make_float2(s, static_cast<float>(b_eff));
+  if (memo.keys) memo.cls[static_cast<size_t>(combo) * C + i] = memo_assign(memo, combo, i, cand, b_eff);
+}
+
+// Per (problem, class): the per-pair part of the sum, from the class's member (classes:
+// ks_memo.cuh). grid (kMemoCap / 256, P); blocks past the number of classes leave at once.
+__global__ void __launch_bounds__(256)
+ridge_pair_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, const ks_candidate* __restrict__ c,
+                  const float2* __restrict__ cand_tab, int C, const __grid_constant__ RidgeParams prm, MemoView memo) {
+  __shared__ ProblemTerms s_pt;
+  const int prob = blockIdx.y, j = blockIdx.x * 256 + threadIdx.x;
+  const ks_problem pr = p[prob];
+  const int combo = (pr.dtype_ab & 3) * 4 + (pr.dtype_d & 3);
+  const int n_classes = memo.count[combo];
+  if (blockIdx.x * 256 >= n_classes) return;
+  if (threadIdx.x == 0) problem_terms(pr, desc, s_pt);
+  __syncthreads();
+  if (j >= n_classes) return;
+  const int slot = memo.dense[static_cast<size_t>(combo) * kMemoCap + j];
+  const int rep = memo.reps[static_cast<size_t>(combo) * kMemoCap + slot];
+  const ks_candidate cand = c[rep];
+  const float2 t = __ldg(cand_tab + static_cast<size_t>(combo) * C + rep);
+  float pair = 0.0f;
+  pair_columns<true>(s_pt, cand, desc, static_cast<long long>(t.y),
+                     [&](int col, float v) { pair += ridge_term(prm, col, v); });
+  static_cast<float*>(memo.tab)[static_cast<size_t>(prob) * kMemoCap + slot] = pair;
 }
 
 __global__ void ridge_combo_mask_kernel(const ks_problem* __restrict__ p, int P, unsigned* __restrict__ mask) {
@@ -451,7 +479,7 @@ __global__ void __launch_bounds__(kBlock)
 select_ridge_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_problem p_value, int use_value,
                     const ks_candidate* __restrict__ c, PairMap map, int sub_tiles,
                     const float2* __restrict__ cand_tab, const __grid_constant__ RidgeParams prm, int k,
-                    unsigned long long* __restrict__ partial /* [P][nblk][k] */) {
+                    unsigned long long* __restrict__ partial /* [P][nblk][k] */, MemoView memo) {
   __shared__ ProblemTerms s_pt;
   __shared__ float s_prob;  // bias + problem-only part of the sum
   __shared__ unsigned long long s_warp[kBlock / 32 * KS_MAX_K];
@@ -476,6 +504,9 @@ select_ridge_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_probl
   if (threadIdx.x < KS_MAX_K) s_list[threadIdx.x] = 0ull;
   __syncthreads();
   const float2* tab = cand_tab + static_cast<size_t>(s_pt.dtype_ab * 4 + s_pt.dtype_d) * map.C;
+  // with classes: the per-pair part is one float per (problem, class)
+  const unsigned* cls = memo.keys ? memo.cls + static_cast<size_t>(s_pt.dtype_ab * 4 + s_pt.dtype_d) * map.C : nullptr;
+  const float* pair_tab = memo.keys ? static_cast<const float*>(memo.tab) + static_cast<size_t>(prob) * kMemoCap : nullptr;
 
   const int64_t pass_rows = static_cast<int64_t>(sub_tiles) * kBlock;
   for (int64_t start = static_cast<int64_t>(chunk) * pass_rows; start < len;
@@ -490,11 +521,16 @@ select_ridge_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_probl
       unsigned long long key = 0ull;
       if (r < len) {
         const int idx = pool_index(map, lo, r);
-        const ks_candidate cand = c[idx];
         const float2 t = __ldg(tab + idx);
+        const unsigned cid = cls ? __ldg(cls + idx) : kNoClass;
         float pair = 0.0f;
-        pair_columns<true>(s_pt, cand, desc, static_cast<long long>(t.y),
-                           [&](int col, float v) { pair += ridge_term(prm, col, v); });
+        if (cid != kNoClass) {
+          pair = __ldg(pair_tab + cid);
+        } else {
+          const ks_candidate cand = c[idx];
+          pair_columns<true>(s_pt, cand, desc, static_cast<long long>(t.y),
+                             [&](int col, float v) { pair += ridge_term(prm, col, v); });
+        }
         key = make_key(((s_prob + t.x) + pair) + 0.0f, idx);
       }
 #pragma unroll
@@ -681,7 +717,12 @@ void free_ridge(MlpModel& m) {
   m.h_ridge = nullptr;
 }
 
-size_t ridge_scratch_bytes(int C) { return 256 + sizeof(float2) * 16 * static_cast<size_t>(C); }
+size_t ridge_scratch_bytes(int C) { return (256 + sizeof(float2) * 16 * static_cast<size_t>(C) + 255) / 256 * 256; }
+// classes and the per-(problem, class) sums of the linear scorer (0: not used)
+size_t ridge_memo_bytes(int P, int C) {
+  if (P < kMemoMinProblems || P > kMemoMaxProblems || C < 1) return 0;
+  return memo_fixed_bytes(C) + sizeof(float) * static_cast<size_t>(P) * kMemoCap;
+}
 
 static int pick_sub_tiles(int P, int64_t per_problem) {
   for (int s = kSubTilesMax; s > 1; s >>= 1) {
@@ -714,7 +755,8 @@ size_t select_partial_bytes(const ks_model& model, int P, int C, int64_t pairs, 
   int64_t nblk = (per + static_cast<int64_t>(st) * kBlock - 1) / (static_cast<int64_t>(st) * kBlock);
   if (nblk < 1) nblk = 1;
   const size_t part = static_cast<size_t>(P) * nblk * k * sizeof(unsigned long long);
-  if (model.kind == 1 && model.mlp.h_ridge) return (part + 255) / 256 * 256 + ridge_scratch_bytes(C);
+  if (model.kind == 1 && model.mlp.h_ridge)
+    return (part + 255) / 256 * 256 + ridge_scratch_bytes(C) + ridge_memo_bytes(P, C);
   return part;
 }
 
@@ -791,14 +833,29 @@ cudaError_t launch_select(const ks_gpu_desc& desc, const ks_model& model, const 
       ridge_combo_mask_kernel<<<P >= 4096 ? 16 : 1, 256, 0, stream>>>(d_p, P, d_mask);
       ++*launches;
     }
+    MemoView memo{};
+    if (!p_by_value && ridge_memo_bytes(P, C) != 0)
+      memo = memo_view(static_cast<char*>(d_partial) + part_bytes + ridge_scratch_bytes(C), C);
     if (C > 0) {
+      if (memo.keys) {
+        e = memo_clear(memo, stream);
+        if (e != cudaSuccess) return e;
+      }
       ridge_cand_kernel<<<dim3((C + 255) / 256, 16), 256, 0, stream>>>(desc, d_c, C, p_by_value ? nullptr : d_mask,
-                                                                      mask_value, *model.mlp.h_ridge, d_tab);
+                                                                      mask_value, *model.mlp.h_ridge, d_tab, memo);
       ++*launches;
+      if (memo.keys) {
+        e = memo_compact(memo, stream);
+        if (e != cudaSuccess) return e;
+        ridge_pair_kernel<<<dim3(kMemoCap / 256, P), 256, 0, stream>>>(desc, d_p, d_c, d_tab, C, *model.mlp.h_ridge, memo);
+        *launches += 2;
+      }
+    } else {
+      memo = MemoView{};
     }
     if (ev_begin) cudaEventRecord(ev_begin, stream);
     select_ridge_kernel<<<grid, kBlock, 0, stream>>>(desc, d_p, pv, p_by_value != nullptr, d_c, map, st, d_tab,
-                                                     *model.mlp.h_ridge, k, partial);
+                                                     *model.mlp.h_ridge, k, partial, memo);
     ++*launches;
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
