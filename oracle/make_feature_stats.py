@@ -1,7 +1,9 @@
 """Write paper_2609_35587_b200/data/feature_stats.npz: per workload, per feature column, the
 128 split-threshold slots (sample quantiles of the column, each placed midway between two
-adjacent distinct sample values) and the standardisation constants (mu, sigma) used by the
-synthetic tree ensembles and MLPs. The feature values come from the CPU oracle only.
+adjacent distinct sample values), the column's empirical distribution over the sample (its
+distinct values with cumulative counts, from which the generator takes any quantile), and the
+standardisation constants (mu, sigma) used by the synthetic tree ensembles and MLPs. The
+feature values come from the CPU oracle only.
 
 Run from the repository root:  python -m oracle.make_feature_stats
 """
@@ -60,14 +62,22 @@ def stats_for(cfg: int) -> dict:
     # a value the workload can produce
     xp = oracle.featurize(prob, cand[:1], desc)
     thr = np.empty((wl.KS_F, wl.N_QUANTILE_SLOTS), dtype=np.float32)
+    dval, dcum, doff = [], [], [0]
     for f in range(wl.KS_F):
-        thr[f] = slots_from_values(xp[:, f] if f in LOG2_COLS else x[:, f], wl.N_QUANTILE_SLOTS)
+        col = xp[:, f] if f in LOG2_COLS else x[:, f]
+        thr[f] = slots_from_values(col, wl.N_QUANTILE_SLOTS)
+        d, cnt = np.unique(col.astype(np.float32), return_counts=True)
+        dval.append(d)
+        dcum.append(np.cumsum(cnt))
+        doff.append(doff[-1] + len(d))
     mu = x.astype(np.float64).mean(axis=0)
     sigma = x.astype(np.float64).std(axis=0)
     sigma[sigma < 1e-12] = 1.0
     for f in CATEGORICAL + (63,):
         mu[f], sigma[f] = 0.0, 1.0
-    return {"thr": thr, "mu": mu.astype(np.float32), "sigma": sigma.astype(np.float32)}
+    return {"thr": thr, "mu": mu.astype(np.float32), "sigma": sigma.astype(np.float32),
+            "dval": np.concatenate(dval).astype(np.float32), "dcum": np.concatenate(dcum).astype(np.int32),
+            "doff": np.asarray(doff, dtype=np.int32)}
 
 
 def main() -> None:

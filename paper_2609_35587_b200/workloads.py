@@ -7,9 +7,15 @@ dtypes and fusion flags of the transfer study).
 This module is shared by the tests of the CPU oracle and of the CUDA library and therefore
 holds NONE of the method's arithmetic: no feature formula, no model evaluation, no ranking.
 Split thresholds and the MLP's standardisation constants are read from
-``data/feature_stats.npz``, a table of per-column sample quantiles / moments of each
+``data/feature_stats.npz``, a table of per-column sample distributions / moments of each
 workload's own feature distribution (written once by the committed script next to the
 oracle that produced it).
+
+Three threshold laws are offered for the synthetic ensembles (``LAWS``): "pernode", every
+internal node draws its own quantile q ~ U(0.05, 0.95) of its column's sample (an ensemble
+trained by exact greedy splitting: thousands of distinct thresholds per continuous column);
+"hist256", q snapped to one of the 255 edges between 256 equal-mass bins (histogram-based
+training); "slots128", one of 128 fixed quantile slots per column.
 
 Random numbers come from a counter-based generator: a 64-bit mix of (seed, stream, index),
 so every array is reproducible element by element and independent of generation order.
@@ -46,7 +52,7 @@ _STATS_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "data", "
 # stream ids (one per generated array)
 _S_M, _S_N, _S_K, _S_LAYOUT, _S_DTYPE, _S_EPI, _S_DECODE = 1, 2, 3, 4, 5, 6, 7
 _S_CAND_SHUFFLE, _S_SEG = 10, 11
-_S_TREE_FEAT, _S_TREE_SLOT, _S_TREE_LEAF_A, _S_TREE_LEAF_B = 20, 21, 22, 23
+_S_TREE_FEAT, _S_TREE_SLOT, _S_TREE_LEAF_A, _S_TREE_LEAF_B, _S_TREE_Q = 20, 21, 22, 23, 24
 _S_MLP_W, _S_MLP_B = 30, 40
 _S_SAMPLE = 50
 
@@ -247,12 +253,45 @@ def feature_stats(key: str) -> dict:
         with np.load(_STATS_PATH) as z:
             _stats_cache = {k: z[k] for k in z.files}
     return {"thr": _stats_cache[f"{key}_thr"], "mu": _stats_cache[f"{key}_mu"],
-            "sigma": _stats_cache[f"{key}_sigma"]}
+            "sigma": _stats_cache[f"{key}_sigma"], "dval": _stats_cache[f"{key}_dval"],
+            "dcum": _stats_cache[f"{key}_dcum"], "doff": _stats_cache[f"{key}_doff"]}
 
 
-def gbdt_complete(seed: int, n_trees: int, depth: int, thr_slots: np.ndarray, leaf_sigma: float):
+LAWS = ("pernode", "hist256", "slots128")
+DEFAULT_LAW = "pernode"
+
+
+def quantile_thresholds(stats: dict, feat: np.ndarray, q: np.ndarray) -> np.ndarray:
+    """Split threshold of every node: the q-quantile of the node's column over the stored sample,
+    placed midway (in fp32) between the two adjacent distinct sample values around it; value +
+    0.5 for a column that is constant in the sample."""
+    feat = np.asarray(feat)
+    q = np.asarray(q, dtype=np.float64)
+    out = np.empty(feat.shape, dtype=np.float32)
+    dval, dcum, doff = stats["dval"], stats["dcum"], stats["doff"]
+    for f in range(KS_F):
+        sel = feat == f
+        if not sel.any():
+            continue
+        d = dval[doff[f]:doff[f + 1]]
+        cum = dcum[doff[f]:doff[f + 1]]
+        n = int(cum[-1])
+        pos = np.floor(q[sel] * (n - 1)).astype(np.int64)
+        i = np.searchsorted(cum, pos, side="right")  # the distinct value holding order statistic `pos`
+        if len(d) == 1:
+            out[sel] = np.float32(d[0] + np.float32(0.5))
+            continue
+        lo_i = np.where(i + 1 < len(d), i, i - 1)
+        lo, hi = d[lo_i], d[lo_i + 1]
+        t = ((lo.astype(np.float64) + hi.astype(np.float64)) / 2.0).astype(np.float32)
+        out[sel] = np.where(t <= lo, hi, t)
+    return out
+
+
+def gbdt_complete(seed: int, n_trees: int, depth: int, stats: dict, leaf_sigma: float,
+                  law: str = DEFAULT_LAW):
     """`n_trees` complete binary trees of `depth` in level order. Split feature uniform over the
-    63 columns; threshold = one of the column's quantile slots; leaves ~ N(0, leaf_sigma).
+    63 columns; threshold by `law` (see the module text); leaves ~ N(0, leaf_sigma).
     Returns (tree_offsets int64 [n_trees+1], nodes NODE_DT)."""
     n_int = (1 << depth) - 1
     n_leaf = 1 << depth
@@ -260,9 +299,18 @@ def gbdt_complete(seed: int, n_trees: int, depth: int, thr_slots: np.ndarray, le
     nodes = np.zeros(n_trees * per, dtype=NODE_DT).reshape(n_trees, per)
     iidx = (np.arange(n_trees)[:, None] * n_int + np.arange(n_int)[None, :])
     feat = randint(seed, _S_TREE_FEAT, iidx, KS_F)
-    slot = randint(seed, _S_TREE_SLOT, iidx, thr_slots.shape[1])
     nodes["feat"][:, :n_int] = feat
-    nodes["v"][:, :n_int] = thr_slots[feat, slot]
+    if law == "slots128":
+        thr_slots = stats["thr"]
+        slot = randint(seed, _S_TREE_SLOT, iidx, thr_slots.shape[1])
+        nodes["v"][:, :n_int] = thr_slots[feat, slot]
+    elif law in ("pernode", "hist256"):
+        q = 0.05 + 0.9 * uniform(seed, _S_TREE_Q, iidx)
+        if law == "hist256":
+            q = (np.floor(q * 256.0) + 1.0) / 256.0
+        nodes["v"][:, :n_int] = quantile_thresholds(stats, feat, q)
+    else:
+        raise ValueError(f"unknown threshold law {law!r}")
     nodes["left"][:, :n_int] = 2 * np.arange(n_int)[None, :] + 1
     lidx = (np.arange(n_trees)[:, None] * n_leaf + np.arange(n_leaf)[None, :])
     nodes["feat"][:, n_int:] = 0xFFFF
@@ -364,18 +412,18 @@ def make_inputs(cfg: int, P: int | None = None, C: int | None = None, seg: int |
 
 def make_workload(cfg: int, P: int | None = None, C: int | None = None, seg: int | None = None,
                   trees: int | None = None, depth: int | None = None,
-                  seed: int = BASE_SEED) -> Workload:
+                  seed: int = BASE_SEED, law: str = DEFAULT_LAW) -> Workload:
     spec = CONFIGS[cfg]
     prob, cand, so, si = make_inputs(cfg, P, C, seg, seed)
     st = feature_stats(spec["stats"])
     w = Workload(name=spec["name"], desc=gpu_desc(), problems=prob, candidates=cand, k=spec["k"],
-                 seg_offsets=so, seg_index=si, meta=dict(cfg=cfg, seed=seed))
+                 seg_offsets=so, seg_index=si, meta=dict(cfg=cfg, seed=seed, law=law))
     if cfg == 4:
         w.mlp = mlp_xavier(seed + 4000, [64, 256, 256, 1], st["mu"], st["sigma"])
     else:
         ms = seed + 1000 if cfg == 3 else seed + 1000 * cfg  # config 3 uses config 1's ensemble
         T = spec["trees"] if trees is None else trees
         D = spec["depth"] if depth is None else depth
-        off, nodes = gbdt_complete(ms, T, D, st["thr"], spec["leaf_sigma"])
+        off, nodes = gbdt_complete(ms, T, D, st, spec["leaf_sigma"], law)
         w.gbdt = (off, nodes, 0.0)
     return w

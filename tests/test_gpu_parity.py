@@ -596,7 +596,7 @@ def test_select_ridge_and_paper_sized_models(ks, ctx):
     w = wl.Workload("mlp_big", DESC, prob[:1], cand[:200], 10, mlp=big)
     idx, sc = run_select(ks, ctx, w, ctx.model_create_mlp(big))
     check_select(w, idx, sc, TOL_MLP)
-    off, nodes = wl.gbdt_complete(wl.BASE_SEED + 9, 916, 7, st["thr"], 0.1)
+    off, nodes = wl.gbdt_complete(wl.BASE_SEED + 9, 916, 7, st, 0.1)
     w = wl.Workload("gbdt_916x7", DESC, prob, cand, 10, gbdt=(off, nodes, 0.0))
     idx, sc = run_select(ks, ctx, w, ctx.model_create_gbdt(off, nodes, 0.0))
     check_select(w, idx, sc, TOL_GBDT)
@@ -670,7 +670,7 @@ def test_partition_split_ensembles(ks, ctx):
     # leaf indices and scores of the standalone scorer
     prob, cand, so, si = wl.make_inputs(2, P=5, seg=700)
     x = oracle.featurize(prob, cand, DESC, so, si)
-    off, nodes = wl.gbdt_complete(23, 64, 6, wl.feature_stats("cfg2")["thr"], 0.1)
+    off, nodes = wl.gbdt_complete(23, 64, 6, wl.feature_stats("cfg2"), 0.1)
     pnodes = wl.with_partition_splits(9, nodes)
     assert pnodes["kind"].sum() > 100
     model = ctx.model_create_gbdt(off, pnodes, 0.5)
@@ -708,7 +708,7 @@ def test_partition_split_ensembles(ks, ctx):
         _, rsc = oracle.select(w3.problems, w3.candidates, DESC, 10, gbdt=w3.gbdt)
         assert np.array_equal(sc, rsc), mask
     # an ensemble too deep for the quantised kernel keeps its partition splits on the general one
-    off5, n5 = wl.gbdt_complete(31, 6, 11, wl.feature_stats("cfg1")["thr"], 0.1)
+    off5, n5 = wl.gbdt_complete(31, 6, 11, wl.feature_stats("cfg1"), 0.1)
     p5 = wl.with_partition_splits(2, n5)
     w5 = wl.Workload("deep", DESC, w2.problems, w2.candidates[:1200], 10, gbdt=(off5, p5, 0.0))
     idx, sc = run_select(ks, ctx, w5, ctx.model_create_gbdt(*w5.gbdt))

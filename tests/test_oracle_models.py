@@ -282,8 +282,7 @@ def test_partition_split_of_an_upper_set_equals_a_numeric_split():
 def test_partition_ensemble_against_nested_ifs():
     prob, cand, _, _ = wl.make_inputs(2, P=2, seg=150)
     x = oracle.featurize(prob, cand[:150], DESC)
-    thr = wl.feature_stats("cfg2")["thr"]
-    off, nodes = wl.gbdt_complete(17, 40, 4, thr, 0.1)
+    off, nodes = wl.gbdt_complete(17, 40, 4, wl.feature_stats("cfg2"), 0.1)
     pnodes = wl.with_partition_splits(5, nodes)
     assert pnodes["kind"].sum() > 20 and np.array_equal(pnodes["feat"], nodes["feat"])
     got = oracle.score_gbdt(x, off, pnodes, base_score=0.25)

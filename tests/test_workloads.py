@@ -80,14 +80,41 @@ def test_models():
     assert np.all(m["sigma"] != 0) and m["mu"][63] == 0 and m["sigma"][63] == 1
 
 
+def test_threshold_laws():
+    """Distinct thresholds per column under the three laws (config 1's ensemble): a quantile per
+    node gives a continuous column well over a thousand, 256 bins at most 255, the slot table at
+    most 128; every threshold lies strictly between two sample values of its column or beside
+    its only one."""
+    st = wl.feature_stats("cfg1")
+    most = {}
+    for law in wl.LAWS:
+        nodes = wl.make_workload(1, P=1, C=8, law=law).gbdt[1]
+        it = nodes[nodes["feat"] != 0xFFFF]
+        assert len(it) == 500 * 255
+        most[law] = max(len(np.unique(it["v"][it["feat"] == f])) for f in range(63))
+        for f in (0, 16, 39, 44):
+            d = st["dval"][st["doff"][f]:st["doff"][f + 1]]
+            t = np.unique(it["v"][it["feat"] == f])
+            assert not np.isin(t, d).any() and t.min() > d[0] and (t.max() < d[-1] or len(d) == 1)
+    assert most["pernode"] > 1000 and 128 < most["hist256"] <= 255 and most["slots128"] <= 128
+    # the quantile of a node: q = 0.5 of a column with values {1, 2, 3, 4} x 16 is the midpoint 2.5
+    toy = {"dval": np.tile(np.array([1, 2, 3, 4], np.float32), 63), "doff": np.arange(64) * 4,
+           "dcum": np.tile(np.array([16, 32, 48, 64], np.int32), 63)}
+    got = wl.quantile_thresholds(toy, np.array([0, 5, 62, 7]), np.array([0.5, 0.05, 0.94, 0.99]))
+    assert got.tolist() == [2.5, 1.5, 3.5, 3.5]
+
+
 def test_checksums():
     """Drift guard: any change to the generators or the stats table shows up here."""
     prob, cand, _, _ = wl.make_inputs(0)
     w = wl.make_workload(0)
     got = dict(prob0=crc(prob), cand0=crc(cand), nodes0=crc(w.gbdt[1]),
+               nodes0_hist256=crc(wl.make_workload(0, law="hist256").gbdt[1]),
+               nodes0_slots128=crc(wl.make_workload(0, law="slots128").gbdt[1]),
                cand1=crc(wl.make_inputs(1, P=1)[1]), prob1=crc(wl.make_inputs(1)[0]))
     want = CHECKSUMS
     assert got == want, got
 
 
-CHECKSUMS = {'prob0': 783310851, 'cand0': 485305090, 'nodes0': 3560579726, 'cand1': 3090539893, 'prob1': 1331788314}
+CHECKSUMS = {'prob0': 783310851, 'cand0': 485305090, 'nodes0': 3578089389, 'nodes0_hist256': 2769579378,
+             'nodes0_slots128': 3560579726, 'cand1': 3090539893, 'prob1': 1331788314}
