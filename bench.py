@@ -112,7 +112,7 @@ def run_reference(args, rank, world):
     cfg = args.workload
     spec = wl.CONFIGS[cfg]
     cores = oracle.threads()
-    w = wl.make_workload(cfg, P=max(2, min(spec["P"], args.ref_problems)))
+    w = wl.make_workload(cfg, P=max(2, min(spec["P"], args.ref_problems)), law=args.law)
     kw = dict(gbdt=w.gbdt, mlp=w.mlp, seg_off=w.seg_offsets, seg_idx=w.seg_index)
     for _ in range(args.warmup):
         oracle.select(w.problems[:1], w.candidates, w.desc, w.k, gbdt=w.gbdt, mlp=w.mlp,
@@ -138,20 +138,21 @@ def config_dict(cfg, spec, args):
          "candidates_per_problem": spec["seg"] or spec["C"], "k": spec["k"],
          "l2": "flushed between steps (256 MiB write)"}
     if spec["trees"]:
-        d.update(scorer="gbdt", trees=spec["trees"], depth=spec["depth"])
+        d.update(scorer="gbdt", trees=spec["trees"], depth=spec["depth"], threshold_law=args.law)
+        d["workload"] += f", thresholds: {args.law}"
     else:
         d.update(scorer="mlp 64-256-256-1 bf16")
     return d
 
 
-def cpu_baseline(cfg, budget_s=15.0):
+def cpu_baseline(cfg, law, budget_s=15.0):
     """The oracle as it stands on this machine's host cores, on a bounded sample of the workload."""
     import oracle
     from paper_2609_35587_b200 import workloads as wl
     spec = wl.CONFIGS[cfg]
     cores = oracle.threads()
     probe_p = max(1, min(cores, spec["P"]))
-    w = wl.make_workload(cfg, P=max(probe_p, 2))
+    w = wl.make_workload(cfg, P=max(probe_p, 2), law=law)
     kw = dict(gbdt=w.gbdt, mlp=w.mlp)
 
     def run(n):
@@ -165,7 +166,7 @@ def cpu_baseline(cfg, budget_s=15.0):
     n = int(max(probe_p, min(spec["P"], probe_p * budget_s / max(t_probe, 1e-3))))
     n = max(cores, n // cores * cores)
     if n > len(w.problems):
-        w = wl.make_workload(cfg, P=n)
+        w = wl.make_workload(cfg, P=n, law=law)
     dt = run(n)
     return {"value": n * per / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"first {n} problems x {per} candidates of the workload, {dt:.1f} s"}
@@ -182,7 +183,7 @@ def run_latency_stream(args, rank, local_rank, dev):
     from paper_2609_35587_b200 import binding as ks
     from paper_2609_35587_b200 import workloads as wl
     n_warm, n = (1000 if args.calls >= 1000 else 10), args.calls
-    w = wl.make_workload(3, P=n_warm + n)
+    w = wl.make_workload(3, P=n_warm + n, law=args.law)
     ctx = ks.Context(w.desc, local_rank)
     model = ctx.model_create_gbdt(*w.gbdt)
     d_c = ks.to_device(w.candidates, dev)
@@ -358,6 +359,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=1, choices=[0, 1, 2, 3, 4])
+    ap.add_argument("--law", default="pernode", choices=["pernode", "hist256", "slots128"],
+                    help="threshold law of the synthetic tree ensemble (workloads.LAWS)")
     ap.add_argument("--calls", type=int, default=100000, help="latency stream (workload 3): timed calls")
     ap.add_argument("--ref-problems", type=int, default=16)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -399,7 +402,7 @@ def main():
         run_latency_stream(args, rank, local_rank, dev)
         return
     # weak scaling: every rank ranks its own batch of problems against the shared catalogue
-    w = wl.make_workload(cfg, P=args.problems, seed=wl.BASE_SEED)
+    w = wl.make_workload(cfg, P=args.problems, seed=wl.BASE_SEED, law=args.law)
     if rank != 0:
         w.problems = wl.make_inputs(cfg, P=args.problems, seed=wl.BASE_SEED + 7919 * rank)[0]
     P, C, k = len(w.problems), len(w.candidates), w.k
@@ -487,7 +490,7 @@ def main():
             visits = pairs * spec["trees"] * spec["depth"]
             achieved = visits * INSTR_PER_VISIT / (kms * 1e-3)
             line["dtype"] = "f32"
-            line["roofline"] = {"bound": "alu", "kernel": "fused featurize+gbdt+top-k",
+            line["roofline"] = {"bound": "alu", "kernel": model.describe(),
                                 "achieved": achieved / 1e12, "peak": ISSUE_PEAK / 1e12,
                                 "unit": "T thread-instr/s (4 per node visit)",
                                 "frac": achieved / ISSUE_PEAK, "kernel_ms": kms,
@@ -497,13 +500,13 @@ def main():
             flops = pairs * 2.0 * (64 * 256 + 256 * 256)
             achieved = flops / (kms * 1e-3)
             line["dtype"] = "bf16"
-            line["roofline"] = {"bound": "tensor", "kernel": "fused featurize+mlp+top-k",
+            line["roofline"] = {"bound": "tensor", "kernel": model.describe(),
                                 "achieved": achieved / 1e12, "peak": peaks["bf16_tflops_sustained"],
                                 "unit": "TFLOP/s", "frac": achieved / 1e12 / peaks["bf16_tflops_sustained"],
                                 "kernel_ms": kms, "peak_source": peaks["source"] + " (sustained bf16)",
                                 "traffic": TRAFFIC_BYTES.get(cfg)}
         if not args.no_cpu_baseline and world == 1:
-            line["cpu_baseline"] = cpu_baseline(cfg)
+            line["cpu_baseline"] = cpu_baseline(cfg, args.law)
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

@@ -258,9 +258,11 @@ ks_status ks_score(ks_ctx* ctx, const float* d_features, int64_t rows, const ks_
  * members), d_topk_score [P, k] the scores (-inf there). 1 <= k <= KS_MAX_K. The feature
  * matrix and the scores are never written to memory. `pairs` as in ks_featurize. The call
  * sizes the context's workspace (owned by the context, grown on demand, which synchronises the
- * device when it happens): partial lists, a per-call table of 16 x C x 64 bytes, and, for a
- * tree model on a batch of 32 to 8,192 problems, P x 512 KiB for the tables of per-pair tile
- * rows (KS_ERR_OOM if the workspace cannot be had). */
+ * device when it happens): partial lists, a per-call table of 16 x C records of at most 256
+ * bytes, and, for a tree model on a batch of 32 problems or more, at most 256 MiB for the
+ * tables of per-pair tile rows (larger batches are served in several launches that reuse it);
+ * KS_ERR_OOM if the workspace cannot be had. d_p and d_c must be 16-byte aligned (each record
+ * is fetched with one 128-bit load), else KS_ERR_INVALID_ARG. */
 ks_status ks_select(ks_ctx* ctx, const ks_problem* d_p, int P, const ks_candidate* d_c, int C,
                     const int64_t* d_seg_offsets, const int32_t* d_seg_index, int64_t pairs,
                     const ks_model* model, int k, int32_t* d_topk_idx, float* d_topk_score,
@@ -335,6 +337,26 @@ ks_status ks_device_status(ks_ctx* ctx);
  * ks_profile_last_ms waits for the last such kernel and returns its duration. */
 ks_status ks_profile_enable(ks_ctx* ctx, int on);
 ks_status ks_profile_last_ms(ks_ctx* ctx, float* out_ms);
+/* One line naming the fused kernel that ks_select runs for this model and, for a tree
+ * ensemble on the quantised path, its tile geometry (threads per CTA x candidates per CTA),
+ * rows and distinct thresholds. Written to buf (at most len bytes, always terminated). */
+ks_status ks_model_describe(const ks_model* model, char* buf, int len);
+
+/* ---- test hooks (the paper has no counterpart) ------------------------------------------- */
+
+/* Bounded device-side waits of this context's kernels: `probe_limit` > 0 replaces the number
+ * of probes a wait may take before it gives up (0 restores the default, tens of milliseconds);
+ * `starve` != 0 makes the tree kernel arm each chunk barrier for 16 bytes more than its copy
+ * brings, and the tensor-core kernel skip the copy of its weight image, so that the first wait
+ * runs out, the kernel sets the status word and returns, and the call reports KS_ERR_TIMEOUT
+ * without any fault: the failure path can be tested on a healthy GPU. */
+ks_status ks_debug_set_wait(ks_ctx* ctx, int probe_limit, int starve);
+/* Checked build only (libks_debug.so, compiled with KS_DEBUG_BOUNDS): the kernels compare
+ * every index they form from data with its range and, instead of touching memory out of range,
+ * record the source line of the first violation. Returns that line, 0 when there was none,
+ * -1 in a regular build; ks_debug_bounds_clear resets it. Both synchronise the device. */
+int ks_debug_bounds_line(void);
+void ks_debug_bounds_clear(void);
 
 #ifdef __cplusplus
 }

@@ -13,7 +13,8 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libks.so")
+# KS_LIBRARY names another build of the same library (the checked build libks_debug.so)
+LIB_PATH = os.environ.get("KS_LIBRARY") or os.path.join(_HERE, "libks.so")
 
 KS_F, KS_F_PAD, KS_MAX_K, KS_MAX_DEPTH = 63, 64, 32, 15
 KS_CATALOGUE_SIZE = 534600
@@ -24,7 +25,8 @@ EXPORTS = ("ks_create", "ks_destroy", "ks_last_cuda_error", "ks_model_create_gbd
            "ks_model_create_mlp", "ks_model_create_static", "ks_model_destroy", "ks_featurize", "ks_score", "ks_select",
            "ks_select_one", "ks_select_host", "ks_status_string", "ks_feature_count",
            "ks_feature_name", "ks_launch_count", "ks_profile_enable", "ks_profile_last_ms", "ks_device_status", "ks_select_trees_static",
-           "ks_enumerate", "ks_valid_catalogue", "ks_remap_indices")
+           "ks_enumerate", "ks_valid_catalogue", "ks_remap_indices", "ks_model_describe",
+           "ks_debug_set_wait", "ks_debug_bounds_line", "ks_debug_bounds_clear")
 
 
 class KsError(RuntimeError):
@@ -74,6 +76,10 @@ def _load() -> ctypes.CDLL:
     lib.ks_valid_catalogue.argtypes = [vp, ctypes.POINTER(_Problem), ctypes.c_uint, vp, i32, vp, vp, vp,
                                        ctypes.POINTER(ctypes.c_int32), vp]
     lib.ks_remap_indices.argtypes = [vp, vp, i64, vp, i32, vp]
+    lib.ks_model_describe.argtypes = [vp, ctypes.c_char_p, i32]
+    lib.ks_debug_set_wait.argtypes = [vp, i32, i32]
+    lib.ks_debug_bounds_line.restype = i32
+    lib.ks_debug_bounds_clear.restype = None
     for name in EXPORTS:
         fn = getattr(lib, name)
         if fn.restype is ctypes.c_int and name not in ("ks_feature_count",):
@@ -151,9 +157,27 @@ def ks_select_trees_static(desc: np.ndarray, d_p, P, d_c, C, d_nodes, d_tree_off
                                            _dptr(d_topk_idx), _dptr(d_topk_score), _stream()))
 
 
+def debug_bounds_line() -> int:
+    """Checked build: source line of the first out-of-range index the kernels met (0: none);
+    -1 in a regular build."""
+    return int(_lib.ks_debug_bounds_line())
+
+
+def debug_bounds_clear() -> None:
+    _lib.ks_debug_bounds_clear()
+
+
 class Model:
     def __init__(self, ctx: "Context", handle: ctypes.c_void_p, kind: str, n_trees: int = 0):
         self.ctx, self._h, self.kind, self.n_trees = ctx, handle, kind, n_trees
+
+    def describe(self) -> str:
+        """The fused kernel ks_select runs for this model, with its tile geometry."""
+        buf = ctypes.create_string_buffer(256)
+        st = _lib.ks_model_describe(self._h, buf, 256)
+        if st != KS_OK:
+            raise KsError(st, "ks_model_describe")
+        return buf.value.decode()
 
     def close(self):
         if self._h:
@@ -201,6 +225,10 @@ class Context:
 
     def device_status(self) -> int:
         return int(_lib.ks_device_status(self._h))
+
+    def debug_set_wait(self, probe_limit: int = 0, starve: bool = False):
+        """Test hook: probe budget of the kernels' bounded waits, and the starved-wait mode."""
+        self._check(_lib.ks_debug_set_wait(self._h, int(probe_limit), int(starve)), "ks_debug_set_wait")
 
     def profile_enable(self, on: bool = True):
         self._check(_lib.ks_profile_enable(self._h, int(on)), "ks_profile_enable")

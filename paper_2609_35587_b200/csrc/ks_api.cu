@@ -69,7 +69,7 @@ cudaError_t ensure_dynamic_smem(const void* kernel, size_t bytes) {
     int device;
     size_t bytes;
   };
-  static Entry table[64];
+  static Entry table[256];
   static int used = 0;
   static std::mutex mu;
   int device = 0;
@@ -83,7 +83,7 @@ cudaError_t ensure_dynamic_smem(const void* kernel, size_t bytes) {
   e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes));
   if (e != cudaSuccess) return e;
   if (hit) hit->bytes = bytes;
-  else if (used < 64) table[used++] = Entry{kernel, device, bytes};
+  else if (used < 256) table[used++] = Entry{kernel, device, bytes};
   return cudaSuccess;
 }
 }  // namespace ks
@@ -163,8 +163,7 @@ void free_model(ks_model* m) {
   cudaFree(m->gbdt.d_roots);
   cudaFree(m->gbdt.d_qnodes);
   cudaFree(m->gbdt.d_qthr);
-  cudaFree(m->gbdt.d_qrow0);
-  cudaFree(m->gbdt.d_qrowcnt);
+  cudaFree(m->gbdt.d_qfeat);
   ks::free_fast_gbdt(m->gbdt);
   for (int l = 0; l < KS_MLP_MAX_LAYERS; ++l) {
     cudaFree(m->mlp.d_w[l]);
@@ -185,6 +184,9 @@ ks_status check_pairs(int P, int C, const void* seg_off, const void* seg_idx, in
   if (!seg_off && pairs != static_cast<int64_t>(P) * C) return KS_ERR_INVALID_ARG;
   return KS_OK;
 }
+
+// problem and candidate records are fetched with 128-bit loads
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 }  // namespace
 
@@ -311,6 +313,44 @@ ks_status ks_profile_last_ms(ks_ctx* ctx, float* out_ms) {
   cudaError_t e = cudaEventSynchronize(ctx->ev_end);
   if (e == cudaSuccess) e = cudaEventElapsedTime(out_ms, ctx->ev_begin, ctx->ev_end);
   return e == cudaSuccess ? KS_OK : cuda_fail(ctx, e, "ks_profile_last_ms");
+}
+
+ks_status ks_model_describe(const ks_model* model, char* buf, int len) {
+  if (!model || !buf || len < 1) return KS_ERR_INVALID_ARG;
+  if (model->kind == 0 && model->gbdt.fast) {
+    const ks::GbdtModel& g = model->gbdt;
+    std::snprintf(buf, len, "select_fast_kernel threads=%d block=%d rows=%d thresholds=%d top_levels=%d%s trees=%d depth=%d",
+                  g.fast_threads, g.block_cands, g.n_qrows, g.n_qthr, g.top_levels, g.top_compact ? "c" : "",
+                  g.n_trees, g.fast_depth);
+  } else if (model->kind == 0) {
+    std::snprintf(buf, len, "select_generic_kernel trees=%d depth=%d", model->gbdt.n_trees, model->gbdt.max_depth);
+  } else if (model->kind == 1 && model->mlp.tc) {
+    std::snprintf(buf, len, "select_mlp_tc_kernel");
+  } else if (model->kind == 1 && model->mlp.h_ridge) {
+    std::snprintf(buf, len, "select_ridge_kernel");
+  } else if (model->kind == 1) {
+    std::snprintf(buf, len, "select_generic_kernel mlp layers=%d", model->mlp.n_layers);
+  } else {
+    std::snprintf(buf, len, "select_generic_kernel static score");
+  }
+  return KS_OK;
+}
+
+ks_status ks_debug_set_wait(ks_ctx* ctx, int probe_limit, int starve) {
+  if (!ctx || probe_limit < 0) return KS_ERR_INVALID_ARG;
+  ctx->wait.limit = probe_limit;
+  ctx->wait.starve = starve != 0;
+  return KS_OK;
+}
+
+int ks_debug_bounds_line(void) {
+  cudaDeviceSynchronize();
+  return ks::fast_bounds_line();
+}
+
+void ks_debug_bounds_clear(void) {
+  cudaDeviceSynchronize();
+  ks::fast_bounds_clear();
 }
 
 ks_status ks_model_create_gbdt(ks_ctx* ctx, int n_trees, const int64_t* h_tree_offsets,
@@ -474,7 +514,7 @@ ks_status ks_featurize(ks_ctx* ctx, const ks_problem* d_p, int P, const ks_candi
   ks_status s = check_pairs(P, C, d_seg_offsets, d_seg_index, pairs);
   if (s != KS_OK) return s;
   if (pairs == 0) return KS_OK;
-  if (!d_p || !d_c || !d_features) return KS_ERR_INVALID_ARG;
+  if (!d_p || !d_c || !d_features || !aligned16(d_p) || !aligned16(d_c)) return KS_ERR_INVALID_ARG;
   DeviceGuard g(ctx->device);
   s = ensure_workspace(ctx, ks::featurize_scratch_bytes(P));
   if (s != KS_OK) return s;
@@ -496,7 +536,8 @@ ks_status ks_score(ks_ctx* ctx, const float* d_features, int64_t rows, const ks_
     ks_status s = ensure_workspace(ctx, ks::score_fast_scratch_bytes(model->gbdt, rows));
     if (s != KS_OK) return s;
     cudaError_t e = ks::launch_score_fast(ctx->desc, model->gbdt, d_features, rows, d_scores, ctx->ws,
-                                          ctx->d_status, static_cast<cudaStream_t>(stream), &ctx->launches);
+                                          ctx->d_status, static_cast<cudaStream_t>(stream), &ctx->launches,
+                                          &ctx->wait);
     return e == cudaSuccess ? KS_OK : cuda_fail(ctx, e, "ks_score");
   }
   if (model->kind == 1 && ks::score_mlp_tc_ok(model->mlp)) {
@@ -522,6 +563,7 @@ ks_status ks_select(ks_ctx* ctx, const ks_problem* d_p, int P, const ks_candidat
   if (s != KS_OK) return s;
   if (P == 0) return KS_OK;
   if (!d_p || !d_topk_idx || !d_topk_score || (pairs > 0 && !d_c)) return KS_ERR_INVALID_ARG;
+  if (!aligned16(d_p) || !aligned16(d_c)) return KS_ERR_INVALID_ARG;
   DeviceGuard g(ctx->device);
   s = ensure_workspace(ctx, ks::select_partial_bytes(*model, P, C, pairs, d_seg_offsets != nullptr, k));
   if (s != KS_OK) return s;
@@ -529,7 +571,7 @@ ks_status ks_select(ks_ctx* ctx, const ks_problem* d_p, int P, const ks_candidat
                                     d_seg_index, pairs, k, ctx->ws, d_topk_idx, d_topk_score,
                                     static_cast<cudaStream_t>(stream), &ctx->launches, ctx->d_status,
                                     ctx->profile ? ctx->ev_begin : nullptr,
-                                    ctx->profile ? ctx->ev_end : nullptr, ctx->d_counters);
+                                    ctx->profile ? ctx->ev_end : nullptr, ctx->d_counters, &ctx->wait);
   ctx->profile_valid = ctx->profile && e == cudaSuccess;
   return e == cudaSuccess ? KS_OK : cuda_fail(ctx, e, "ks_select");
 }
@@ -537,7 +579,7 @@ ks_status ks_select(ks_ctx* ctx, const ks_problem* d_p, int P, const ks_candidat
 ks_status ks_select_one(ks_ctx* ctx, ks_problem p, const ks_candidate* d_c, int C, const ks_model* model,
                         int k, int32_t* h_topk_idx, float* h_topk_score, void* stream) {
   if (!ctx || !model || model->ctx != ctx || k < 1 || k > KS_MAX_K || C < 0) return KS_ERR_INVALID_ARG;
-  if (!h_topk_idx || !h_topk_score || (C > 0 && !d_c)) return KS_ERR_INVALID_ARG;
+  if (!h_topk_idx || !h_topk_score || (C > 0 && !d_c) || !aligned16(d_c)) return KS_ERR_INVALID_ARG;
   if (p.m < 1 || p.n < 1 || p.k < 1 || p.m > KS_MAX_DIM || p.n > KS_MAX_DIM || p.k > KS_MAX_DIM ||
       p.layout > 3 || p.dtype_ab > 3 || p.dtype_d > 3 || p.epi_flags > 5)
     return KS_ERR_INVALID_ARG;
@@ -549,12 +591,13 @@ ks_status ks_select_one(ks_ctx* ctx, ks_problem p, const ks_candidate* d_c, int 
   // Latency path for a qualifying tree model: the trees are split over several CTAs per
   // candidate block, the last block writes the k results straight into mapped host memory.
   if (model->kind == 0 && model->gbdt.fast && C > 0) {
-    const int nblk = (C + ks::kFastRows - 1) / ks::kFastRows;
+    const int NC = model->gbdt.block_cands;
+    const int nblk = (C + NC - 1) / NC;
     const int S = ks::fast_slices(model->gbdt, nblk);
     if (S > 1) {
       const size_t b_part = align_up(sizeof(unsigned long long) * nblk * k);
       // scratch of this path: the prepared tiles, one per candidate block (no per-call table)
-      const size_t b_scratch = align_up(static_cast<size_t>(nblk) * model->gbdt.n_qrows * ks::kFastRows);
+      const size_t b_scratch = align_up(static_cast<size_t>(nblk) * model->gbdt.n_qrows * NC);
       const size_t b_scores = align_up(sizeof(float) * static_cast<size_t>(S) * C);
       ks_status s = ensure_workspace(ctx, b_part + b_scratch + b_scores);
       if (s != KS_OK) return s;
@@ -572,9 +615,10 @@ ks_status ks_select_one(ks_ctx* ctx, ks_problem p, const ks_candidate* d_c, int 
       int* h_seq = reinterpret_cast<int*>(pin_sc + KS_MAX_K);
       sl.out_seq = reinterpret_cast<int*>(ctx->d_pinned_score + KS_MAX_K);
       sl.seq = ++ctx->select_one_seq;
-      cudaError_t e = ks::launch_select_fast(ctx->desc, model->gbdt, nullptr, &p, 1, d_c, C, nblk, ks::kFastRows,
+      cudaError_t e = ks::launch_select_fast(ctx->desc, model->gbdt, nullptr, &p, 1, d_c, C, nblk, NC,
                                              nullptr, nullptr, k, reinterpret_cast<unsigned long long*>(base),
-                                             base + b_part, ctx->d_status, st, &ctx->launches, nullptr, &sl);
+                                             base + b_part, ctx->d_status, st, &ctx->launches, nullptr, &sl, nullptr,
+                                             &ctx->wait);
       if (e == cudaSuccess) {
         bool seen = false;
         for (int spin = 0; spin < (1 << 22) && !seen; ++spin) seen = *static_cast<volatile int*>(h_seq) == sl.seq;
@@ -600,7 +644,7 @@ ks_status ks_select_one(ks_ctx* ctx, ks_problem p, const ks_candidate* d_c, int 
   if (s != KS_OK) return s;
   cudaError_t e = ks::launch_select(ctx->desc, *model, nullptr, &p, 1, d_c, C, nullptr, nullptr, C, k,
                                     ctx->ws, ctx->d_pinned_idx, ctx->d_pinned_score, st, &ctx->launches,
-                                    ctx->d_status);
+                                    ctx->d_status, nullptr, nullptr, nullptr, &ctx->wait);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "ks_select_one");
   std::memcpy(h_topk_idx, pin_idx, k * sizeof(int32_t));
@@ -641,7 +685,7 @@ ks_status ks_select_host(ks_ctx* ctx, const ks_problem* h_p, int P, const ks_can
   if (e == cudaSuccess && seg && pairs > 0) e = cudaMemcpyAsync(d_si, h_seg_index, sizeof(int32_t) * pairs, cudaMemcpyHostToDevice, st);
   if (e == cudaSuccess)
     e = ks::launch_select(ctx->desc, *model, d_p, nullptr, P, d_c, C, d_so, d_si, pairs, k, ctx->ws, d_oi,
-                          d_os, st, &ctx->launches, ctx->d_status, nullptr, nullptr, ctx->d_counters);
+                          d_os, st, &ctx->launches, ctx->d_status, nullptr, nullptr, ctx->d_counters, &ctx->wait);
   if (e == cudaSuccess) e = cudaMemcpyAsync(h_topk_idx, d_oi, sizeof(int32_t) * P * k, cudaMemcpyDeviceToHost, st);
   if (e == cudaSuccess) e = cudaMemcpyAsync(h_topk_score, d_os, sizeof(float) * P * k, cudaMemcpyDeviceToHost, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);

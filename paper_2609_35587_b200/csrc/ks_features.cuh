@@ -24,6 +24,38 @@ __host__ __device__ constexpr int feat_class(int col) {
                                                                                             : 2;
 }
 
+// Descriptor fetch: a problem or candidate record is 16 bytes and sits on a 16-byte boundary
+// (checked where the arrays enter the library), so it is one 128-bit load.
+__device__ __forceinline__ ks_problem load_problem(const ks_problem* p) {
+  const uint4 v = __ldg(reinterpret_cast<const uint4*>(p));
+  ks_problem r;
+  r.m = v.x;
+  r.n = v.y;
+  r.k = v.z;
+  r.layout = static_cast<uint8_t>(v.w);
+  r.dtype_ab = static_cast<uint8_t>(v.w >> 8);
+  r.dtype_d = static_cast<uint8_t>(v.w >> 16);
+  r.epi_flags = static_cast<uint8_t>(v.w >> 24);
+  return r;
+}
+__device__ __forceinline__ ks_candidate load_candidate(const ks_candidate* p) {
+  const uint4 v = __ldg(reinterpret_cast<const uint4*>(p));
+  ks_candidate r;
+  r.tile_m = static_cast<uint16_t>(v.x);
+  r.tile_n = static_cast<uint16_t>(v.x >> 16);
+  r.tile_k = static_cast<uint16_t>(v.y);
+  r.instr_n = static_cast<uint16_t>(v.y >> 16);
+  r.stages = static_cast<uint8_t>(v.z);
+  r.cluster_m = static_cast<uint8_t>(v.z >> 8);
+  r.cluster_n = static_cast<uint8_t>(v.z >> 16);
+  r.kernel_sched = static_cast<uint8_t>(v.z >> 24);
+  r.epi_sched = static_cast<uint8_t>(v.w);
+  r.tile_sched = static_cast<uint8_t>(v.w >> 8);
+  r.instr_m = static_cast<uint8_t>(v.w >> 16);
+  r.instr_k = static_cast<uint8_t>(v.w >> 24);
+  return r;
+}
+
 __device__ __forceinline__ float F64i(long long v) { return __ll2float_rn(v); }
 __device__ __forceinline__ float F32i(int v) { return __int2float_rn(v); }
 __device__ __forceinline__ unsigned cdiv_u32(unsigned a, unsigned b) { return (a + b - 1u) / b; }

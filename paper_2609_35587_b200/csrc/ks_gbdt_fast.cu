@@ -3,13 +3,16 @@
 // Repack (host, at model-create time)
 //   A split "x[f] < thr" only needs to know how many of feature f's distinct thresholds are
 //   <= x. With the thresholds of f sorted, bin(x) = #{j : thr_j <= x}, and
-//   x < thr_j  <=>  bin(x) <= j  exactly, so a pair's feature row shrinks from 64 floats to
-//   one byte per "row" (a feature, or a 127-threshold slice of one) and a node to one 32-bit
-//   word. Trees are padded to complete trees of the ensemble's depth D and stored in chunks,
-//   each chunk laid out level by level ([level][tree][node]) followed by its leaves, so that a
-//   chunk is one contiguous block a CTA copies into shared memory with one bulk async copy.
-//   The nodes of the top levels are also kept as (row offset, replicated threshold) pairs that
-//   travel as a kernel parameter, i.e. through the constant bank.
+//   x < thr_j  <=>  bin(x) <= j  exactly. A feature's thresholds are cut into slices of 127; a
+//   "row" is one slice, a pair's byte in that row the number of the slice's thresholds that are
+//   <= x (0..127), and a node one 32-bit word (row offset, index within the slice). A feature
+//   with thousands of distinct thresholds (an ensemble trained by exact greedy splitting) simply
+//   owns more rows; the tile geometry follows the row count (see FastGeom). Trees are padded to
+//   complete trees of the ensemble's depth D and stored in chunks, each chunk laid out level by
+//   level ([level][tree][node]) followed by its leaves, so that a chunk is one contiguous block
+//   a CTA copies into shared memory with one bulk async copy. The nodes of the top levels are
+//   also kept as (row offset, replicated threshold) pairs that travel as a kernel parameter,
+//   i.e. through the constant bank.
 //   A partition split on a categorical field ("level in S goes right") joins the same scheme
 //   through rank rows: a row whose byte is the rank of the pair's level in a fixed ordering of
 //   the field's levels, chosen so that S or its complement is the set of ranks >= c; the node
@@ -28,20 +31,21 @@
 //   the tiles are built once by tile_one_kernel; scoring call (ks_score): tiles are quantised
 //   from given feature rows by tile_rows_kernel and the scores are stored instead of ranked.
 //
-// Kernel (one CTA = one problem x up to kFastRows candidates, kFastThreads threads, two CTAs per SM)
+// Kernel (one CTA = one problem x up to NC candidates, THREADS threads)
 //   phase A  fill the [row][candidate] byte tile. A 32-bit word of a row holds the four
 //            candidates that share a lane slot, so a warp's byte loads of any mix of rows
 //            touch 32 distinct banks and one word load serves four candidates;
 //   phase B  stream the ensemble through two shared-memory buffers (cp.async.bulk + mbarrier,
-//            bounded waits). Thread (w, h) owns the four candidates of word w and walks the
-//            trees of half h of every chunk. The top levels are evaluated for all four
+//            bounded waits). Thread (w, g) owns the four candidates of word w and walks the
+//            trees of group g of every chunk. The top levels are evaluated for all four
 //            candidates at once, node by node, with byte-parallel arithmetic on whole words;
 //            below that each candidate follows its own path: a' = 2 a + k0 (+ 4 to go right), a
 //            multiply-add plus a predicated add;
-//   phase C  add the two halves' partial scores, rank the block's keys, write a partial
-//            top-k list.
+//   phase C  add the groups' partial scores, rank the block's keys, write a partial top-k list.
 #include <algorithm>
 #include <cmath>
+#include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <limits>
 #include <new>
@@ -56,22 +60,30 @@ namespace ks {
 
 namespace {
 
-constexpr int kBufBytes = 16 * 1024;   // one tree-chunk buffer
-constexpr int kMaxRows = 80;           // quantised rows the kernel supports (tile <= 160 KB)
-constexpr int kThrPerRow = 128;        // 127 thresholds + padding
-constexpr int kRowStride = kFastRows;  // bytes between rows of the tile (one byte per candidate)
-constexpr int kWords = kFastRows / 4;  // words per row = lane slots
-constexpr unsigned kSleepNs = 1200;  // asked-for sleep between two probes of a chunk barrier (400 to 2500 measured alike)
-constexpr int kSpinLimit = 1 << 23;  // probes (a sleep ends early, ~0.2 us measured): a wait gives up after a few seconds
-constexpr int kCandRec = 64;           // bytes per (combination, candidate) record of quantised rows
+constexpr int kBufBytes = 16 * 1024;   // one tree-chunk buffer (twice that where the shared memory allows)
+constexpr int kSlice = 127;            // thresholds per row: a byte is 0x80 | (0..127)
+constexpr unsigned kSleepNs = 1200;    // asked-for sleep between two probes of a chunk barrier (400 to 2500 measured alike)
 constexpr int kCombos = 16;            // dtype_ab x dtype_d
 
-static_assert(kFastThreads == 2 * kWords && kFastR == 2, "tile geometry");
-
-// shared memory map (byte offsets from the dynamic shared base)
+// shared memory map (byte offsets from the dynamic shared base): the chunk buffers, then the tile
 constexpr int kNBuf = 2;                // tree-chunk buffers (a ring; four of 8 KB and three of 12 KB measured slower)
 constexpr int kOffBuf0 = 0;
-constexpr int kOffTile = kNBuf * kBufBytes;
+
+#ifdef KS_DEBUG_BOUNDS
+// Checked build: every index formed from data (tile byte, node, chunk, record, partial list) is
+// compared with its range; a violation records its source line in this word and uses element 0.
+__device__ int g_bounds_line;
+__device__ __forceinline__ long long checked_index(long long i, long long n, int line) {
+  if (i < 0 || i >= n) {
+    atomicCAS(&g_bounds_line, 0, line);
+    return 0;
+  }
+  return i;
+}
+#define KS_IDX(i, n) checked_index(static_cast<long long>(i), static_cast<long long>(n), __LINE__)
+#else
+#define KS_IDX(i, n) (i)
+#endif
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -92,12 +104,14 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait: one probe, then sleep-and-probe (measured faster than the blocking try_wait with
-// or without a time hint); gives up after kSpinLimit probes and reports false.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+// or without a time hint); gives up after `limit` probes, or as soon as another warp of the CTA
+// has given up (`fail`), and reports false.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, int limit, volatile int* fail) {
   if (mbar_test_wait(bar, parity)) return true;
-  for (int i = 0; i < kSpinLimit; ++i) {
+  for (int i = 0; i < limit; ++i) {
     __nanosleep(kSleepNs);
     if (mbar_test_wait(bar, parity)) return true;
+    if ((i & 63) == 63 && *fail) return false;
   }
   return false;
 }
@@ -124,24 +138,40 @@ __device__ __forceinline__ float lds_f32(uint32_t addr) {
 // the per-call table kernel that precedes every launch of the select kernel.
 __device__ int g_fast_abort;
 
-// #{j : T[j] <= v} over 127 sorted thresholds padded with +inf: 7 branch-free steps.
-__device__ __forceinline__ int bin_search(const float* T, float v) {
+// #{j < n : T[j] <= v} over n sorted thresholds.
+__device__ __forceinline__ int count_le(const float* T, int n, float v) {
   int pos = 0;
-#pragma unroll
-  for (int s = 64; s >= 1; s >>= 1) pos += (T[pos + s - 1] <= v) ? s : 0;
+  for (int s = n > 0 ? 1 << (31 - __clz(n)) : 0; s >= 1; s >>= 1) {
+    const int np = pos + s;
+    if (np <= n && T[np - 1] <= v) pos = np;
+  }
   return pos;
 }
 
-// Bin of value v in one row of the threshold table. A row whose last slot is negative infinity is
-// a rank row of a categorical field: slot c holds the rank of level c in the row's ordering of
-// the levels (see build_fast_gbdt), and the bin is that rank.
-__device__ __forceinline__ int row_bin(const float* T, float v) {
-  if (T[kThrPerRow - 1] < 0.0f) {
-    const int code = __float2int_rz(v);
-    return (code >= 0 && code < 4) ? __float2int_rz(T[code]) : 0;
+// Tile bytes of one feature value: slice s of the feature's thresholds gets the number of its
+// thresholds that are <= v, i.e. the overall count less 127 s clamped to 0..127; a rank row gets
+// the rank of the level code v. `T` is the feature's own sorted threshold array. With
+// `nan_right` a NaN takes the last bin of every slice (x < t is false: it goes right).
+template <typename Put>
+__device__ __forceinline__ void quantise(const FeatQ& q, const float* T, float v, bool nan_right, Put put) {
+  if (q.nslice) {
+    const int pos = (nan_right && v != v) ? q.nthr : count_le(T, q.nthr, v);
+    for (int s = 0; s < q.nslice; ++s) {
+      int b = pos - kSlice * s;
+      b = b < 0 ? 0 : (b > kSlice ? kSlice : b);
+      put(q.row0 + s, static_cast<uint8_t>(0x80 | b));
+    }
   }
-  return bin_search(T, v);
+  if (q.nrank) {
+    const int code = __float2int_rz(v);
+    for (int r = 0; r < q.nrank; ++r)
+      put(q.row0 + q.nslice + r, static_cast<uint8_t>(0x80 | ((code >= 0 && code < 4) ? q.rank[r][code] : 0)));
+  }
 }
+
+// Byte of candidate i (0 .. 4 W - 1) of a block within one tile row of W words: the four
+// candidates of a word are i, i + W, i + 2 W, i + 3 W.
+__device__ __forceinline__ int tile_byte(int i, int W) { return (i % W) * 4 + i / W; }
 
 // Slice mode (single-problem latency call): the trees are split over n_slices CTAs per
 // candidate block. Every CTA stores its partial scores; the last CTA to arrive for a block
@@ -154,7 +184,7 @@ struct SliceArgs {
   int* counters;           // [P * nblk + 1], zero on entry; every counter is reset by its last user
   int32_t* out_idx;        // single-problem form only: [k] final result (device-visible, may be
   float* out_score;        // mapped host memory); null when a merge kernel follows
-  const uint8_t* tiles;    // prepared tiles [blocks][rows][kRowStride] (tile_one_kernel), or null
+  const uint8_t* tiles;    // prepared tiles [blocks][rows][NC] (tile_one_kernel), or null
   int* out_seq;            // single-problem form: receives `seq` once the k results are written
   int seq;
   float* score_out;        // scoring call (ks_score): the scores of the block's rows go here, no ranking
@@ -163,20 +193,18 @@ struct SliceArgs {
 struct FastView {
   int n_rows, n_pair_rows, n_cand_rows, n_prob_rows;  // rows are ordered pair, candidate, problem
   int depth, n_chunks, chunk_bytes, tpc;
+  int n_thr, thr_cand0, thr_prob0;  // thresholds in all, and where the candidate-only / problem-only features' begin
+  int cand_rec, pair_rec;           // bytes per record of the per-call tables (multiples of 16)
+  int wait_limit, starve;           // probes a chunk wait may take; test hook: arm the barrier for bytes that never come
+  int buf_bytes;                    // size of one chunk buffer in shared memory
   float base;
   const uint32_t* chunks;      // [n_chunks][chunk_bytes / 4]
-  const float* thr;            // [n_rows][kThrPerRow]
-  const uint8_t* feat_row0;    // [64] first row of each feature column
-  const uint8_t* feat_rowcnt;  // [64] number of rows of each feature column
-  const uint8_t* cand_rows;    // [kCombos][C][kCandRec] quantised candidate-only rows
+  const float* thr;            // [n_thr] sorted thresholds, feature after feature (per-pair features first)
+  const FeatQ* feat;           // [64] rows and thresholds of each feature column
+  const uint8_t* cand_rows;    // [kCombos][C][cand_rec] quantised candidate-only rows
   const unsigned* pair_class;  // [kCombos][C] class of every candidate, or null (no memo)
-  const uint8_t* pair_tab;     // [P][kMemoCap][kMemoRec] per-pair tile bytes of every (problem, class)
+  const uint8_t* pair_tab;     // [P][kMemoCap][pair_rec] per-pair tile bytes of every (problem, class)
 };
-
-// Memo of the per-pair rows (classes: ks_memo.cuh). Per problem the tile bytes of the per-pair
-// rows are evaluated once per class from the class's member; phase A then copies a 64-byte
-// record instead of evaluating 21 columns and searching their rows.
-constexpr int kMemoRec = 64;  // bytes per record = most per-pair rows a memoised model may have
 
 // ------------------------------------------------------------------------------------------
 // candidate-only rows, once per call
@@ -184,28 +212,34 @@ constexpr int kMemoRec = 64;  // bytes per record = most per-pair rows a memoise
 
 __global__ void combo_mask_kernel(const ks_problem* __restrict__ p, int P, unsigned* __restrict__ mask) {
   unsigned m = 0;
-  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < P; i += gridDim.x * blockDim.x)
-    m |= 1u << ((p[i].dtype_ab & 3) * 4 + (p[i].dtype_d & 3));
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < P; i += gridDim.x * blockDim.x) {
+    const ks_problem pr = load_problem(p + i);
+    m |= 1u << ((pr.dtype_ab & 3) * 4 + (pr.dtype_d & 3));
+  }
   m = __reduce_or_sync(0xFFFFFFFFu, m);
   if ((threadIdx.x & 31) == 0 && m) atomicOr(mask, m);
 }
 
+// Thresholds of a range of features into shared memory when they fit `cap` floats, else the
+// global array is searched in place. Returns the pointer that stands for fv.thr + first.
+__device__ __forceinline__ const float* stage_thresholds(const FastView& fv, int first, int count, float* s_thr,
+                                                         int cap) {
+  if (count > cap) return fv.thr + first;
+  for (int i = threadIdx.x; i < count; i += blockDim.x) s_thr[i] = __ldg(fv.thr + first + i);
+  return s_thr;
+}
+
 __global__ void __launch_bounds__(256)
 cand_rows_kernel(ks_gpu_desc desc, const ks_candidate* __restrict__ c, int C, const unsigned* mask_ptr,
-                 unsigned mask_value, FastView fv, uint8_t* __restrict__ out, MemoView memo) {
-  extern __shared__ float s_cthr[];  // thresholds of the candidate-only rows
-  __shared__ uint8_t s_r0[64], s_rc[64];
+                 unsigned mask_value, FastView fv, uint8_t* __restrict__ out, MemoView memo, int thr_cap) {
+  extern __shared__ float s_cthr[];  // thresholds of the candidate-only features
+  __shared__ FeatQ s_fq[64];
   const int combo = blockIdx.y;
   if (blockIdx.x == 0 && combo == 0 && threadIdx.x == 0) g_fast_abort = 0;
   const unsigned mask = mask_ptr ? *mask_ptr : mask_value;
   if (!((mask >> combo) & 1u)) return;
-  const int first = fv.n_pair_rows;
-  for (int i = threadIdx.x; i < fv.n_cand_rows * kThrPerRow; i += blockDim.x)
-    s_cthr[i] = __ldg(fv.thr + first * kThrPerRow + i);
-  if (threadIdx.x < 64) {
-    s_r0[threadIdx.x] = fv.feat_row0[threadIdx.x];
-    s_rc[threadIdx.x] = fv.feat_rowcnt[threadIdx.x];
-  }
+  const float* T = stage_thresholds(fv, fv.thr_cand0, fv.thr_prob0 - fv.thr_cand0, s_cthr, thr_cap) - fv.thr_cand0;
+  if (threadIdx.x < 64) s_fq[threadIdx.x] = fv.feat[threadIdx.x];
   __syncthreads();
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= C) return;
@@ -215,25 +249,14 @@ cand_rows_kernel(ks_gpu_desc desc, const ks_candidate* __restrict__ c, int C, co
   fake.dtype_d = static_cast<uint8_t>(combo & 3);
   ProblemTerms t;
   problem_terms(fake, desc, t);
-  const ks_candidate cand = c[i];
-  uint32_t rec[kCandRec / 4];
-#pragma unroll
-  for (int q = 0; q < kCandRec / 4; ++q) rec[q] = 0x80808080u;
+  const ks_candidate cand = load_candidate(c + i);
+  uint8_t* rec = out + (static_cast<size_t>(combo) * C + i) * fv.cand_rec;
+  const int first = fv.n_pair_rows;
   featurize_pair(t, cand, desc, [&](int col, float v) {
     if (feat_class(col) != 1) return;
-    const int r0 = s_r0[col] - first, rc = s_rc[col];
-    for (int q = 0; q < rc; ++q) {
-      const uint32_t b = 0x80u | row_bin(s_cthr + (r0 + q) * kThrPerRow, v);
-      const int at = r0 + q;
-#pragma unroll
-      for (int w = 0; w < kCandRec / 4; ++w)
-        if (w == (at >> 2)) rec[w] = (rec[w] & ~(0xFFu << (8 * (at & 3)))) | (b << (8 * (at & 3)));
-    }
+    const FeatQ& q = s_fq[col];
+    quantise(q, T + q.thr0, v, false, [&](int row, uint8_t b) { rec[KS_IDX(row - first, fv.cand_rec)] = b; });
   });
-  uint4* dst = reinterpret_cast<uint4*>(out + (static_cast<size_t>(combo) * C + i) * kCandRec);
-#pragma unroll
-  for (int q = 0; q < kCandRec / 16; ++q)
-    if (q * 16 < fv.n_cand_rows) dst[q] = make_uint4(rec[4 * q], rec[4 * q + 1], rec[4 * q + 2], rec[4 * q + 3]);
   if (memo.keys)
     memo.cls[static_cast<size_t>(combo) * C + i] = memo_assign(memo, combo, i, cand, resources(t, cand, desc).b_eff);
 }
@@ -254,35 +277,31 @@ memo_compact_kernel(MemoView memo) {
 }
 
 // Per problem: the tile bytes of the per-pair rows of every class, from the class's member.
-// grid (kMemoCap / 256, P); blocks past the number of classes leave at once.
+// grid (kMemoCap / 256, batch of problems); blocks past the number of classes leave at once.
+// `p` points at the batch's first problem, and record (problem within the batch, slot) is written.
 __global__ void __launch_bounds__(256)
 pair_table_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, const ks_candidate* __restrict__ c,
-                  FastView fv, MemoView memo) {
-  extern __shared__ float s_pthr[];  // thresholds of the per-pair rows
+                  FastView fv, MemoView memo, int thr_cap) {
+  extern __shared__ float s_pthr[];  // thresholds of the per-pair features
   __shared__ ProblemTerms s_pt;
-  __shared__ uint8_t s_r0[64], s_rc[64];
+  __shared__ FeatQ s_fq[64];
   const int prob = blockIdx.y, j = blockIdx.x * 256 + threadIdx.x;
-  const ks_problem pr = p[prob];
+  const ks_problem pr = load_problem(p + prob);
   const int combo = (pr.dtype_ab & 3) * 4 + (pr.dtype_d & 3);
   const int n_classes = memo.count[combo];
   if (blockIdx.x * 256 >= n_classes) return;
   const int slot = j < n_classes ? memo.dense[static_cast<size_t>(combo) * kMemoCap + j] : 0;
-  const unsigned long long key = j < n_classes ? 1ull : 0ull;
-  for (int i = threadIdx.x; i < fv.n_pair_rows * kThrPerRow; i += 256) s_pthr[i] = __ldg(fv.thr + i);
-  if (threadIdx.x < 64) {
-    s_r0[threadIdx.x] = fv.feat_row0[threadIdx.x];
-    s_rc[threadIdx.x] = fv.feat_rowcnt[threadIdx.x];
-  }
+  const float* T = stage_thresholds(fv, 0, fv.thr_cand0, s_pthr, thr_cap);
+  if (threadIdx.x < 64) s_fq[threadIdx.x] = fv.feat[threadIdx.x];
   if (threadIdx.x == 0) problem_terms(pr, desc, s_pt);
   __syncthreads();
-  if (key == 0ull) return;
-  const ks_candidate cand = c[memo.reps[static_cast<size_t>(combo) * kMemoCap + slot]];
+  if (j >= n_classes) return;
+  const ks_candidate cand = load_candidate(c + memo.reps[static_cast<size_t>(combo) * kMemoCap + slot]);
   const long long b_eff = resources(s_pt, cand, desc).b_eff;
-  uint8_t* rec = static_cast<uint8_t*>(memo.tab) + (static_cast<size_t>(prob) * kMemoCap + slot) * kMemoRec;
+  uint8_t* rec = static_cast<uint8_t*>(memo.tab) + (static_cast<size_t>(prob) * kMemoCap + slot) * fv.pair_rec;
   pair_columns<true>(s_pt, cand, desc, b_eff, [&](int col, float v) {
-    const int r0 = s_r0[col], rc = s_rc[col];
-    for (int q = 0; q < rc; ++q)
-      rec[r0 + q] = static_cast<uint8_t>(0x80 | bin_search(s_pthr + (r0 + q) * kThrPerRow, v));
+    const FeatQ& q = s_fq[col];
+    quantise(q, T + q.thr0, v, false, [&](int row, uint8_t b) { rec[KS_IDX(row, fv.pair_rec)] = b; });
   });
 }
 
@@ -297,45 +316,42 @@ pair_table_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, const ks_c
 template <bool kPairRows>  // true: the per-pair rows; false: the candidate-only and problem-only rows
 __device__ __forceinline__ void tile_one_rows(const ks_gpu_desc& desc, const ks_problem& p_value,
                                               const ks_candidate* __restrict__ c, int C, const FastView& fv,
-                                              uint8_t* __restrict__ tiles, float* s_thr) {
+                                              int NC, uint8_t* __restrict__ tiles, float* s_thr, int thr_cap) {
   __shared__ ProblemTerms s_pt;
-  __shared__ uint8_t s_r0[64], s_rc[64];
+  __shared__ FeatQ s_fq[64];
   const int tid = threadIdx.x;
   if (blockIdx.x == 0 && tid == 0) g_fast_abort = 0;
-  // rows are ordered per-pair, candidate-only, problem-only
+  // rows and thresholds are ordered per-pair, candidate-only, problem-only
   const int first = kPairRows ? 0 : fv.n_pair_rows;
   const int count = kPairRows ? fv.n_pair_rows : fv.n_rows - fv.n_pair_rows;
-  for (int i = tid; i < count * kThrPerRow; i += blockDim.x) s_thr[i] = __ldg(fv.thr + first * kThrPerRow + i);
-  if (tid < 64) {
-    s_r0[tid] = fv.feat_row0[tid];
-    s_rc[tid] = fv.feat_rowcnt[tid];
-  }
+  const int t_first = kPairRows ? 0 : fv.thr_cand0;
+  const int t_count = kPairRows ? fv.thr_cand0 : fv.n_thr - fv.thr_cand0;
+  const float* T = stage_thresholds(fv, t_first, t_count, s_thr, thr_cap) - t_first;
+  if (tid < 64) s_fq[tid] = fv.feat[tid];
   if (tid == 0) problem_terms(p_value, desc, s_pt);
   __syncthreads();
   const int slot = blockIdx.x * blockDim.x + tid;
-  const int blk = slot / kFastRows, in = slot % kFastRows;
-  const int t = in % kFastThreads, r = in / kFastThreads;  // phase-A thread and its candidate
-  uint8_t* my = tiles + static_cast<size_t>(blk) * fv.n_rows * kRowStride + (t % kWords) * 4 + (t / kWords) * kFastR + r;
+  const int blk = slot / NC, in = slot % NC;
+  uint8_t* my = tiles + static_cast<size_t>(blk) * fv.n_rows * NC + tile_byte(in, NC / 4);
   if (slot >= C) {
-    for (int q = first; q < first + count; ++q) my[q * kRowStride] = 0x80;
+    for (int q = first; q < first + count; ++q) my[static_cast<size_t>(q) * NC] = 0x80;
     return;
   }
-  const ks_candidate cand = c[slot];
+  const ks_candidate cand = load_candidate(c + slot);
   featurize_pair(s_pt, cand, desc, [&](int col, float v) {
-    if ((feat_class(col) == 2) != kPairRows) return;
-    const int r0 = s_r0[col], rc = s_rc[col];
-    for (int q = 0; q < rc; ++q)
-      my[(r0 + q) * kRowStride] = static_cast<uint8_t>(0x80 | row_bin(s_thr + (r0 + q - first) * kThrPerRow, v));
+    if (col >= KS_F || (feat_class(col) == 2) != kPairRows) return;
+    const FeatQ& q = s_fq[col];
+    quantise(q, T + q.thr0, v, false, [&](int row, uint8_t b) { my[static_cast<size_t>(KS_IDX(row, fv.n_rows)) * NC] = b; });
   });
 }
 
 // blockIdx.y picks the role, so that both halves of the work are in flight together
 __global__ void __launch_bounds__(256)
 tile_one_kernel(ks_gpu_desc desc, ks_problem p_value, const ks_candidate* __restrict__ c, int C, FastView fv,
-                uint8_t* __restrict__ tiles) {
-  extern __shared__ float s_thr[];  // thresholds of this role's rows
-  if (blockIdx.y == 0) tile_one_rows<true>(desc, p_value, c, C, fv, tiles, s_thr);
-  else tile_one_rows<false>(desc, p_value, c, C, fv, tiles, s_thr);
+                int NC, uint8_t* __restrict__ tiles, int thr_cap) {
+  extern __shared__ float s_thr[];  // thresholds of this role's features
+  if (blockIdx.y == 0) tile_one_rows<true>(desc, p_value, c, C, fv, NC, tiles, s_thr, thr_cap);
+  else tile_one_rows<false>(desc, p_value, c, C, fv, NC, tiles, s_thr, thr_cap);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -345,36 +361,31 @@ tile_one_kernel(ks_gpu_desc desc, ks_problem p_value, const ks_candidate* __rest
 // ks_score with a qualifying ensemble: one thread per tile word quantises all columns of the
 // word's four feature rows into the tile layout of phase A and stores whole words, so that a
 // warp's stores are full lines; the walk kernel then copies the tiles as in the single-problem
-// call and writes scores instead of ranking. A NaN goes right at every numeric split (x < t is
+// call and writes the scores instead of ranking. A NaN goes right at every numeric split (x < t is
 // false), like +inf: the last bin. Slots past the last row get the neutral byte. Also clears
-// the abort flag.
-__global__ void __launch_bounds__(kWords)
-tile_rows_kernel(const float* __restrict__ feat, int64_t rows, FastView fv, uint8_t* __restrict__ tiles) {
-  extern __shared__ float s_thr[];  // thresholds of every row
-  __shared__ uint8_t s_r0[64], s_rc[64];
+// the abort flag. Launched with one thread per word of a row (NC / 4).
+__global__ void __launch_bounds__(256)
+tile_rows_kernel(const float* __restrict__ feat, int64_t rows, FastView fv, uint8_t* __restrict__ tiles,
+                 int thr_cap) {
+  extern __shared__ float s_thr[];  // thresholds of every feature
+  __shared__ FeatQ s_fq[64];
+  const int W = blockDim.x, NC = 4 * W;
   const int word = threadIdx.x;
   if (blockIdx.x == 0 && word == 0) g_fast_abort = 0;
-  {
-    const float4* src = reinterpret_cast<const float4*>(fv.thr);
-    float4* dst = reinterpret_cast<float4*>(s_thr);
-    for (int i = word; i < fv.n_rows * (kThrPerRow / 4); i += kWords) dst[i] = __ldg(src + i);
-  }
-  if (word < 64) {
-    s_r0[word] = fv.feat_row0[word];
-    s_rc[word] = fv.feat_rowcnt[word];
-  }
+  const float* T = stage_thresholds(fv, 0, fv.n_thr, s_thr, thr_cap);
+  if (word < 64) s_fq[word] = fv.feat[word];
   __syncthreads();
-  // byte b of the word belongs to phase-A thread word + kWords * (b / 2), candidate b % 2
-  const int64_t base = static_cast<int64_t>(blockIdx.x) * kFastRows;
+  // byte b of the word is row b W + word of the block
+  const int64_t base = static_cast<int64_t>(blockIdx.x) * NC;
   const float4* src[4];
   bool live[4];
 #pragma unroll
   for (int b = 0; b < 4; ++b) {
-    const int64_t slot = base + (b & 1) * kFastThreads + word + kWords * (b >> 1);
+    const int64_t slot = base + b * W + word;
     live[b] = slot < rows;
     src[b] = reinterpret_cast<const float4*>(feat + (live[b] ? slot : 0) * KS_F_PAD);
   }
-  uint32_t* out = reinterpret_cast<uint32_t*>(tiles + static_cast<size_t>(blockIdx.x) * fv.n_rows * kRowStride) + word;
+  uint32_t* out = reinterpret_cast<uint32_t*>(tiles + static_cast<size_t>(blockIdx.x) * fv.n_rows * NC) + word;
 #pragma unroll 2
   for (int q4 = 0; q4 < KS_F_PAD / 4; ++q4) {
     float v[4][4];
@@ -387,19 +398,30 @@ tile_rows_kernel(const float* __restrict__ feat, int64_t rows, FastView fv, uint
     for (int j = 0; j < 4; ++j) {
       const int col = 4 * q4 + j;
       if (col >= KS_F) continue;
-      const int r0 = s_r0[col], rc = s_rc[col];
-      for (int q = 0; q < rc; ++q) {
-        const float* T = s_thr + (r0 + q) * kThrPerRow;
-        const bool rank_row = T[kThrPerRow - 1] < 0.0f;
+      const FeatQ& q = s_fq[col];
+      int pos[4], code[4];
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        const float x = v[b][j];
+        pos[b] = !live[b] ? 0 : ((x != x) ? q.nthr : count_le(T + q.thr0, q.nthr, x));
+        code[b] = live[b] ? __float2int_rz(x) : -1;
+      }
+      for (int s = 0; s < q.nslice; ++s) {
         uint32_t w = 0;
 #pragma unroll
         for (int b = 0; b < 4; ++b) {
-          const float x = v[b][j];
-          int bin = (x != x && !rank_row) ? kThrPerRow - 1 : row_bin(T, x);
-          if (!live[b]) bin = 0;
+          int bin = pos[b] - kSlice * s;
+          bin = bin < 0 ? 0 : (bin > kSlice ? kSlice : bin);
           w |= static_cast<uint32_t>(0x80 | bin) << (8 * b);
         }
-        out[static_cast<size_t>(r0 + q) * (kRowStride / 4)] = w;
+        out[static_cast<size_t>(KS_IDX(q.row0 + s, fv.n_rows)) * W] = w;
+      }
+      for (int r = 0; r < q.nrank; ++r) {
+        uint32_t w = 0;
+#pragma unroll
+        for (int b = 0; b < 4; ++b)
+          w |= static_cast<uint32_t>(0x80 | ((code[b] >= 0 && code[b] < 4) ? q.rank[r][code[b]] : 0)) << (8 * b);
+        out[static_cast<size_t>(KS_IDX(q.row0 + q.nslice + r, fv.n_rows)) * W] = w;
       }
     }
   }
@@ -409,70 +431,58 @@ tile_rows_kernel(const float* __restrict__ feat, int64_t rows, FastView fv, uint
 // phase A
 // ------------------------------------------------------------------------------------------
 
-// Fills the tile bytes of the two candidates this thread owns in phase A: candidate-only rows
-// from the per-call table, problem-only rows from s_pbin, per-pair rows computed here. Slots
-// past the end of the segment get a neutral byte so that word-wise arithmetic on the tile
-// never borrows across bytes.
+// Scatters a 16-byte-aligned record of `n` row bytes into a tile column.
+__device__ __forceinline__ void scatter_record(const uint8_t* __restrict__ rec, int n, unsigned char* dst, int NC) {
+  const uint4* src = reinterpret_cast<const uint4*>(rec);
+  for (int v = 0; v * 16 < n; ++v) {
+    const uint4 q = __ldg(src + v);
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int b = 0; b < 16; ++b)
+      if (v * 16 + b < n) dst[(v * 16 + b) * NC] = static_cast<unsigned char>(w[b >> 2] >> (8 * (b & 3)));
+  }
+}
+
+// Fills the tile bytes of the candidates this thread owns in phase A: candidate-only rows
+// from the per-call table, problem-only rows from s_pbin, per-pair rows from the memo record of
+// the candidate's class or computed here. Slots past the end of the segment get a neutral byte
+// so that word-wise arithmetic on the tile never borrows across bytes.
+template <int THREADS, int NC>
 __device__ __noinline__ void fill_tile(const ks_gpu_desc& desc, const ProblemTerms& pt,
                                        const ks_candidate* __restrict__ c, const FastView& fv,
                                        const int64_t* __restrict__ seg_off, const int32_t* __restrict__ seg_idx,
-                                       int C, int64_t lo, int64_t start, int64_t stop, const float* s_thr,
-                                       const uint8_t* s_row0, const uint8_t* s_rowcnt, const uint8_t* s_pbin,
-                                       unsigned char* tile, int prob) {
+                                       int C, int64_t lo, int64_t start, int64_t stop, const float* T,
+                                       const FeatQ* s_fq, const uint8_t* s_pbin, unsigned char* tile, int prob) {
   const int tid = threadIdx.x;
   const int combo = pt.dtype_ab * 4 + pt.dtype_d;
 #pragma unroll 1
-  for (int r = 0; r < kFastR; ++r) {
-    const int64_t row = start + static_cast<int64_t>(r) * kFastThreads + tid;
-    unsigned char* my = tile + (tid % kWords) * 4 + (tid / kWords) * kFastR + r;
+  for (int i = tid; i < NC; i += THREADS) {
+    const int64_t row = start + i;
+    unsigned char* my = tile + tile_byte(i, NC / 4);
     if (row >= stop) {
-      for (int q = 0; q < fv.n_rows; ++q) my[q * kRowStride] = 0x80;
+      for (int q = 0; q < fv.n_rows; ++q) my[q * NC] = 0x80;
       continue;
     }
     const int ci = seg_off ? seg_idx[lo + row] : static_cast<int>(row);
-    const ks_candidate cand = c[ci];
     // candidate-only rows
-    const uint4* rec = reinterpret_cast<const uint4*>(fv.cand_rows + (static_cast<size_t>(combo) * C + ci) * kCandRec);
-    unsigned char* dst = my + fv.n_pair_rows * kRowStride;
-#pragma unroll
-    for (int v = 0; v < kCandRec / 16; ++v) {
-      if (v * 16 < fv.n_cand_rows) {
-        const uint4 q = __ldg(rec + v);
-        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-        for (int b = 0; b < 16; ++b)
-          if (v * 16 + b < fv.n_cand_rows)
-            dst[(v * 16 + b) * kRowStride] = static_cast<unsigned char>(w[b >> 2] >> (8 * (b & 3)));
-      }
-    }
+    scatter_record(fv.cand_rows + (static_cast<size_t>(combo) * C + KS_IDX(ci, C)) * fv.cand_rec, fv.n_cand_rows,
+                   my + fv.n_pair_rows * NC, NC);
     // problem-only rows
-    dst = my + (fv.n_pair_rows + fv.n_cand_rows) * kRowStride;
-    for (int q = 0; q < fv.n_prob_rows; ++q) dst[q * kRowStride] = s_pbin[q];
+    unsigned char* dst = my + (fv.n_pair_rows + fv.n_cand_rows) * NC;
+    for (int q = 0; q < fv.n_prob_rows; ++q) dst[q * NC] = s_pbin[q];
     // per-pair rows: the record of the candidate's class, when there is one
     if (fv.pair_class) {
       const unsigned cid = __ldg(fv.pair_class + static_cast<size_t>(combo) * C + ci);
       if (cid != kNoClass) {
-        const uint4* prec =
-            reinterpret_cast<const uint4*>(fv.pair_tab + (static_cast<size_t>(prob) * kMemoCap + cid) * kMemoRec);
-#pragma unroll
-        for (int v = 0; v < kMemoRec / 16; ++v) {
-          if (v * 16 < fv.n_pair_rows) {
-            const uint4 q = __ldg(prec + v);
-            const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-            for (int b = 0; b < 16; ++b)
-              if (v * 16 + b < fv.n_pair_rows)
-                my[(v * 16 + b) * kRowStride] = static_cast<unsigned char>(w[b >> 2] >> (8 * (b & 3)));
-          }
-        }
+        scatter_record(fv.pair_tab + (static_cast<size_t>(prob) * kMemoCap + KS_IDX(cid, kMemoCap)) * fv.pair_rec,
+                       fv.n_pair_rows, my, NC);
         continue;
       }
     }
-    featurize_pair(pt, cand, desc, [&](int col, float v) {
-      if (feat_class(col) != 2) return;
-      const int r0 = s_row0[col], rc = s_rowcnt[col];
-      for (int q = 0; q < rc; ++q)
-        my[(r0 + q) * kRowStride] = static_cast<unsigned char>(0x80 | bin_search(s_thr + (r0 + q) * kThrPerRow, v));
+    const ks_candidate cand = load_candidate(c + ci);
+    pair_columns<true>(pt, cand, desc, resources(pt, cand, desc).b_eff, [&](int col, float v) {
+      const FeatQ& q = s_fq[col];
+      quantise(q, T + q.thr0, v, false, [&](int r, uint8_t b) { my[KS_IDX(r, fv.n_pair_rows) * NC] = b; });
     });
   }
 }
@@ -489,7 +499,8 @@ __device__ __forceinline__ uint32_t byte_select(uint32_t m, uint32_t a, uint32_t
 
 // one path step of one walk: fetch the node, fetch the candidate's byte, move to the child:
 // next = 2 a + k0 (+ 4 when the candidate goes right)
-__device__ __forceinline__ uint32_t path_step(uint32_t a, uint32_t cb_r, uint32_t k0) {
+#ifndef KS_DEBUG_BOUNDS
+__device__ __forceinline__ uint32_t path_step(uint32_t a, uint32_t cb_r, uint32_t k0, uint32_t, uint32_t, uint32_t) {
   uint32_t nx;
   asm volatile(
       "{\n"
@@ -508,33 +519,52 @@ __device__ __forceinline__ uint32_t path_step(uint32_t a, uint32_t cb_r, uint32_
       : "r"(a), "r"(cb_r), "r"(k0));
   return nx;
 }
+#else
+// checked build: the node address must lie in the chunk buffer, the byte address in the tile
+__device__ __forceinline__ uint32_t path_step(uint32_t a, uint32_t cb_r, uint32_t k0, uint32_t buf,
+                                              uint32_t tile0, uint32_t tile_bytes) {
+  a = buf + static_cast<uint32_t>(KS_IDX((a - buf) >> 2, 2 * kBufBytes / 4)) * 4u;
+  const uint32_t n = lds_u32(a);
+  uint32_t m = (n >> 8) + cb_r;
+  m = tile0 + static_cast<uint32_t>(KS_IDX(m - tile0, tile_bytes));
+  uint32_t x;
+  asm volatile("ld.shared.u8 %0, [%1];" : "=r"(x) : "r"(m));
+  return 2u * a + k0 + (x > (n & 255u) ? 4u : 0u);
+}
+#endif
 
 // L levels evaluated word-wise; NP path levels unrolled (-1: runtime count); kCompact: the top
 // levels' constants travel as one 32-bit word per node (row offset << 8 | j + 1) instead of a
 // (row offset, replicated j + 1) pair, so that twice as many trees keep their word-wise levels.
-template <int L, int NP, bool kCompact = false>
-__global__ void __launch_bounds__(kFastThreads, 2)
+// THREADS threads rank NC candidates: NC / 4 words times THREADS / (NC / 4) tree groups.
+template <int L, int NP, bool kCompact, int THREADS, int NC>
+__global__ void __launch_bounds__(THREADS, THREADS == 512 ? 2 : 1)
 select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_problem p_value, int use_value,
                    const ks_candidate* __restrict__ c, int P, int C, int nblk, int rows_per_cta,
                    const int64_t* __restrict__ seg_off, const int32_t* __restrict__ seg_idx, FastView fv,
                    int k, unsigned long long* __restrict__ partial, int* __restrict__ status,
                    SliceArgs sl, const __grid_constant__ FastTopParams top) {
+  constexpr int W = NC / 4;        // words per tile row = lane slots
+  constexpr int G = THREADS / W;   // tree groups
+  static_assert(THREADS % W == 0 && W % 32 == 0 && G >= 1, "tile geometry");
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ ProblemTerms s_pt;
-  __shared__ unsigned long long s_warp[kFastThreads / 32 * KS_MAX_K];
+  __shared__ unsigned long long s_warp[THREADS / 32 * KS_MAX_K];
   __shared__ unsigned long long s_list[KS_MAX_K];
   __shared__ __align__(8) unsigned long long s_bar[kNBuf];
-  __shared__ uint8_t s_row0[64], s_rowcnt[64], s_pbin[64];
+  __shared__ FeatQ s_fq[64];
+  __shared__ uint8_t s_pbin[kFastMaxProbRows];
   __shared__ float s_pfeat[64];
-  __shared__ int s_fail, s_last, s_done[kNBuf], s_abort;
+  __shared__ int s_fail, s_last, s_done[kNBuf], s_abort, s_pending[kNBuf];
 
   const int tid = threadIdx.x;
+  const int kOffTile = kNBuf * fv.buf_bytes;
   const int S = sl.n_slices;
   const int prob = blockIdx.x / (nblk * S), chunk = (blockIdx.x / S) % nblk, slice = blockIdx.x % S;
   if (tid == 0) s_abort = *reinterpret_cast<volatile int*>(&g_fast_abort);
   __syncthreads();
   if (s_abort) {  // a wait ran out in an earlier CTA of this launch: the call fails, leave at once
-    if (tid < k && slice == 0) partial[(static_cast<size_t>(prob) * nblk + chunk) * k + tid] = 0ull;
+    if (tid < k && slice == 0 && partial) partial[(static_cast<size_t>(prob) * nblk + chunk) * k + tid] = 0ull;
     return;
   }
   int64_t lo, len;
@@ -553,7 +583,7 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
   const bool tiles_given = sl.tiles != nullptr;  // the tiles were built in front: no feature work here
   if (tid == 0) {
     if (!tiles_given) {
-      problem_terms(use_value ? p_value : p[prob], desc, s_pt);
+      problem_terms(use_value ? p_value : load_problem(p + prob), desc, s_pt);
       // problem-only columns do not look at the candidate: evaluate them on a dummy one
       ks_candidate dummy{};
       dummy.tile_m = dummy.tile_n = dummy.tile_k = 64;
@@ -564,23 +594,21 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
     }
     for (int b = 0; b < kNBuf; ++b) mbar_init(bar0 + 8u * b, 1);
     s_fail = 0;
-    for (int b = 0; b < kNBuf; ++b) s_done[b] = 0;
+    for (int b = 0; b < kNBuf; ++b) s_done[b] = s_pending[b] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (tid < 64) {
-    s_row0[tid] = fv.feat_row0[tid];
-    s_rowcnt[tid] = fv.feat_rowcnt[tid];
-  }
+  if (tid < 64) s_fq[tid] = fv.feat[tid];
   if (tid < KS_MAX_K) s_list[tid] = 0ull;
   __syncthreads();
   if (!tiles_given && tid < KS_F && feat_class(tid) == 0) {
     const int first = fv.n_pair_rows + fv.n_cand_rows;
-    for (int q = 0; q < s_rowcnt[tid]; ++q)
-      s_pbin[s_row0[tid] + q - first] =
-          static_cast<uint8_t>(0x80 | row_bin(fv.thr + (s_row0[tid] + q) * kThrPerRow, s_pfeat[tid]));
+    const FeatQ& q = s_fq[tid];
+    quantise(q, fv.thr + q.thr0, s_pfeat[tid], false,
+             [&](int row, uint8_t b) { s_pbin[KS_IDX(row - first, kFastMaxProbRows)] = b; });
   }
   uint32_t phases = 0;  // bit b: parity of buffer b's barrier
-  const int word = tid % kWords, half = tid / kWords;
+  const int word = tid % W, grp = tid / W;
+  volatile int* v_fail = &s_fail;
 
   for (int64_t start = static_cast<int64_t>(chunk) * rows_per_cta; start < len;
        start += static_cast<int64_t>(nblk) * rows_per_cta) {
@@ -589,18 +617,16 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
     __syncthreads();
     if (sl.tiles) {
       // single-problem call: the block's tile was built once for all the CTAs that share it
-      const uint4* src = reinterpret_cast<const uint4*>(sl.tiles + static_cast<size_t>(chunk) * fv.n_rows * kRowStride);
+      const uint4* src = reinterpret_cast<const uint4*>(sl.tiles + static_cast<size_t>(chunk) * fv.n_rows * NC);
       uint4* dst = reinterpret_cast<uint4*>(smem + kOffTile);
-      for (int i = tid; i < fv.n_rows * (kRowStride / 16); i += kFastThreads) dst[i] = __ldcg(src + i);
+      for (int i = tid; i < fv.n_rows * (NC / 16); i += THREADS) dst[i] = __ldcg(src + i);
     } else {
-      {
-        float4* dst = reinterpret_cast<float4*>(smem + kOffBuf0);
-        const float4* src = reinterpret_cast<const float4*>(fv.thr);
-        for (int i = tid; i < fv.n_pair_rows * kThrPerRow / 4; i += kFastThreads) dst[i] = __ldg(src + i);
-      }
+      // thresholds of the per-pair features: into the idle chunk buffers when they fit
+      const float* T = stage_thresholds(fv, 0, fv.thr_cand0, reinterpret_cast<float*>(smem + kOffBuf0),
+                                        fv.pair_class ? 0 : kNBuf * fv.buf_bytes / 4);
       __syncthreads();
-      fill_tile(desc, s_pt, c, fv, seg_off, seg_idx, C, lo, start, stop,
-                reinterpret_cast<const float*>(smem + kOffBuf0), s_row0, s_rowcnt, s_pbin, smem + kOffTile, prob);
+      fill_tile<THREADS, NC>(desc, s_pt, c, fv, seg_off, seg_idx, C, lo, start, stop, T, s_fq, s_pbin,
+                             smem + kOffTile, prob);
     }
     __syncthreads();  // tile complete; the threshold table is no longer needed
 
@@ -609,39 +635,48 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
       fence_async_proxy();
       const char* src = reinterpret_cast<const char*>(fv.chunks) + static_cast<size_t>(ch_begin) * fv.chunk_bytes;
       for (int b = 0; b < kNBuf && ch_begin + b < ch_end; ++b) {
-        mbar_expect_tx(bar0 + 8u * b, fv.chunk_bytes);
-        bulk_copy_g2s(sbase + kOffBuf0 + b * kBufBytes, src + static_cast<size_t>(b) * fv.chunk_bytes, fv.chunk_bytes,
-                      bar0 + 8u * b);
+        // test hook: a barrier armed for more bytes than its copy brings never completes
+        mbar_expect_tx(bar0 + 8u * b, fv.chunk_bytes + (fv.starve ? 16 : 0));
+        bulk_copy_g2s(sbase + kOffBuf0 + b * fv.buf_bytes, src + static_cast<size_t>(b) * fv.chunk_bytes,
+                      fv.chunk_bytes, bar0 + 8u * b);
+        s_pending[b] = 1;
       }
     }
     float score[4] = {0.0f, 0.0f, 0.0f, 0.0f};
     const uint32_t cb = sbase + kOffTile + word * 4;
-    const int tpc = fv.tpc, half_trees = tpc / 2;
+    const int tpc = fv.tpc, grp_trees = (tpc + G - 1) / G;
     const int np = NP >= 0 ? NP : fv.depth - L;
     constexpr int kTop = (1 << L) - 1;
+    const int t_first = grp * grp_trees;
+    const int t_count = t_first + grp_trees <= tpc ? grp_trees : (tpc > t_first ? tpc - t_first : 0);
+#ifdef KS_DEBUG_BOUNDS
+    const uint32_t tile0 = sbase + kOffTile, tile_bytes = static_cast<uint32_t>(fv.n_rows) * NC;
+#else
+    constexpr uint32_t tile0 = 0, tile_bytes = 0;
+#endif
 #pragma unroll 1
     for (int ch = ch_begin; ch < ch_end; ++ch) {
       const int b = (ch - ch_begin) % kNBuf;
       const uint32_t bar = bar0 + 8u * b;
       const uint32_t par = (phases >> b) & 1u;
-      // after one wait has run out the CTA stops waiting (and refilling): the call fails, and
-      // the CTAs that start later leave at once
-      if (*reinterpret_cast<volatile int*>(&s_fail) || !mbar_wait_bounded(bar, par)) {
-        if (!*reinterpret_cast<volatile int*>(&s_fail)) {
+      // A wait that runs out ends the walk of this CTA: the buffer was never filled, so it is not
+      // read; the call fails, and the CTAs that start later leave at once.
+      if (*v_fail || !mbar_wait_bounded(bar, par, fv.wait_limit, v_fail)) {
+        if (!*v_fail) {
           s_fail = 1;
           atomicExch(&g_fast_abort, 1);
           if (status) atomicExch(status, KS_ERR_TIMEOUT);
         }
+        break;
       }
       phases ^= 1u << b;
-      const uint32_t buf = sbase + kOffBuf0 + b * kBufBytes;
+      const uint32_t buf = sbase + kOffBuf0 + b * fv.buf_bytes;
       // With A_l the shared address of a walk's node at level l, A_{l+1} = 2 A_l + (4 tpc - buf)
       // + 4 bit for every level, and after the last level A points at the walk's leaf.
       const uint32_t k0 = 4u * tpc - buf;  // modulo 2^32, like the additions it enters
       const uint32_t lvlL = buf + 4u * tpc * kTop;  // first node of level L
-      const int t_first = half * half_trees;
 #pragma unroll 4
-      for (int tt = 0; tt < half_trees; ++tt) {
+      for (int tt = 0; tt < t_count; ++tt) {
         const int t = t_first + tt;
         uint32_t a[4];
         if (L == 0) {
@@ -653,16 +688,18 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
           // d[n] keeps its top bit iff candidate r goes right at node n; no byte borrows.
           uint32_t d[kTop > 0 ? kTop : 1];
           if (kCompact) {
-            const uint32_t* tw = reinterpret_cast<const uint32_t*>(top.w) + static_cast<size_t>(ch * tpc + t) * kTop;
+            const uint32_t* tw = reinterpret_cast<const uint32_t*>(top.w) +
+                                 static_cast<size_t>(KS_IDX(ch * tpc + t, 2 * kFastTopPairs / kTop)) * kTop;
 #pragma unroll
             for (int n = 0; n < kTop; ++n) {
               const uint32_t v = tw[n];
-              d[n] = lds_u32(cb + (v >> 8)) - __byte_perm(v, 0u, 0u);
+              d[n] = lds_u32(cb + static_cast<uint32_t>(KS_IDX(v >> 8, fv.n_rows * NC))) - __byte_perm(v, 0u, 0u);
             }
           } else {
-            const uint2* tw = top.w + static_cast<size_t>(ch * tpc + t) * kTop;
+            const uint2* tw = top.w + static_cast<size_t>(KS_IDX(ch * tpc + t, kFastTopPairs / kTop)) * kTop;
 #pragma unroll
-            for (int n = 0; n < kTop; ++n) d[n] = lds_u32(cb + tw[n].x) - tw[n].y;
+            for (int n = 0; n < kTop; ++n)
+              d[n] = lds_u32(cb + static_cast<uint32_t>(KS_IDX(tw[n].x, fv.n_rows * NC))) - tw[n].y;
           }
           uint32_t x = d[0] & 0x80808080u;  // path bits: level 0 in bit 7 of each byte, ...
           if (L >= 2) {
@@ -686,47 +723,80 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
 #pragma unroll
           for (int l = 0; l < (NP >= 0 ? NP : 0); ++l)
 #pragma unroll
-            for (int r = 0; r < 4; ++r) a[r] = path_step(a[r], cb + r, k0);
+            for (int r = 0; r < 4; ++r) a[r] = path_step(a[r], cb + r, k0, buf, tile0, tile_bytes);
         } else {
 #pragma unroll 1
           for (int l = 0; l < np; ++l)
 #pragma unroll
-            for (int r = 0; r < 4; ++r) a[r] = path_step(a[r], cb + r, k0);
+            for (int r = 0; r < 4; ++r) a[r] = path_step(a[r], cb + r, k0, buf, tile0, tile_bytes);
         }
 #pragma unroll
-        for (int r = 0; r < 4; ++r) score[r] += lds_f32(a[r]);
+        for (int r = 0; r < 4; ++r) {
+#ifdef KS_DEBUG_BOUNDS
+          a[r] = buf + 4u * static_cast<uint32_t>(KS_IDX((a[r] - buf) >> 2, fv.buf_bytes / 4));
+#endif
+          score[r] += lds_f32(a[r]);
+        }
       }
       // Release the buffer without a block-wide barrier: every warp counts itself out, and the
       // last one to leave refills the buffer (nobody waits; warps may run a chunk ahead).
       __syncwarp();
       if ((tid & 31) == 0) {
-        if (atomicAdd(&s_done[b], 1) == kFastThreads / 32 - 1) {
+        if (atomicAdd(&s_done[b], 1) == THREADS / 32 - 1) {
           s_done[b] = 0;
-          if (ch + kNBuf < ch_end && !s_fail) {
+          s_pending[b] = 0;
+          if (ch + kNBuf < ch_end && !*v_fail) {
             fence_async_proxy();
-            mbar_expect_tx(bar, fv.chunk_bytes);
-            bulk_copy_g2s(buf, reinterpret_cast<const char*>(fv.chunks) + static_cast<size_t>(ch + kNBuf) * fv.chunk_bytes,
+            mbar_expect_tx(bar, fv.chunk_bytes + (fv.starve ? 16 : 0));
+            bulk_copy_g2s(buf, reinterpret_cast<const char*>(fv.chunks) +
+                                   static_cast<size_t>(KS_IDX(ch + kNBuf, fv.n_chunks)) * fv.chunk_bytes,
                           fv.chunk_bytes, bar);
+            s_pending[b] = 1;
           }
         }
       }
     }
     __syncthreads();  // all walks are done: the buffers are free
+    if (*v_fail) {
+      // The call has failed. Before this CTA gives its shared memory back, give the copies that
+      // may still be in flight the time to land (bounded again); the test hook's copies land in
+      // full although their barriers never complete, so there a short pause stands in for it.
+      if (tid == 0) {
+        for (int b = 0; b < kNBuf; ++b) {
+          if (!s_pending[b]) continue;
+          if (fv.starve) {
+            for (int i = 0; i < 64; ++i) __nanosleep(kSleepNs);
+          } else {
+            mbar_wait_bounded(bar0 + 8u * b, (phases >> b) & 1u, fv.wait_limit, &s_abort /* stays 0 */);
+          }
+        }
+      }
+      __syncthreads();
+      if (tid < k && slice == 0 && partial) partial[(static_cast<size_t>(prob) * nblk + chunk) * k + tid] = 0ull;
+      return;
+    }
 
     // ---- phase C ---------------------------------------------------------------------------------
-    float* s_part = reinterpret_cast<float*>(smem + kOffBuf0);  // [4][kWords], buffers are idle now
-    if (half == 1) {
+    float* s_part = reinterpret_cast<float*>(smem + kOffBuf0);  // [G - 1][4][W], buffers are idle now
+    if (grp > 0) {
 #pragma unroll
-      for (int r = 0; r < 4; ++r) s_part[r * kWords + word] = score[r];
+      for (int r = 0; r < 4; ++r) s_part[((grp - 1) * 4 + r) * W + word] = score[r];
     }
     __syncthreads();
+    // this thread's sum over the groups, in a fixed order
+    float total[4];
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      total[r] = score[r];
+      if (grp == 0)
+        for (int g = 1; g < G; ++g) total[r] += s_part[((g - 1) * 4 + r) * W + word];
+    }
     if (sl.score_out) {
       // scoring call: the scores are the result (same order of additions as the ranking path)
 #pragma unroll
       for (int r = 0; r < 4; ++r) {
-        const int64_t row = start + static_cast<int64_t>(r & 1) * kFastThreads + word + kWords * (r >> 1);
-        if (half == 0 && row < stop)
-          sl.score_out[lo + row] = ((fv.base + score[r]) + s_part[r * kWords + word]) + 0.0f;
+        const int64_t row = start + r * W + word;
+        if (grp == 0 && row < stop) sl.score_out[lo + row] = (fv.base + total[r]) + 0.0f;
       }
       continue;
     }
@@ -734,9 +804,8 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
       // slice mode: publish this CTA's partial scores, let the last arrival finish the block
 #pragma unroll
       for (int r = 0; r < 4; ++r) {
-        const int64_t row = start + static_cast<int64_t>(r & 1) * kFastThreads + word + kWords * (r >> 1);
-        if (half == 0 && row < stop)
-          __stcg(sl.scores + static_cast<size_t>(slice) * sl.pairs + lo + row, score[r] + s_part[r * kWords + word]);
+        const int64_t row = start + r * W + word;
+        if (grp == 0 && row < stop) __stcg(sl.scores + static_cast<size_t>(slice) * sl.pairs + lo + row, total[r]);
       }
       __threadfence();
       __syncthreads();
@@ -753,15 +822,15 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
       keys[r] = 0ull;
-      // byte r of word `word` belongs to phase-A thread word + kWords * (r / 2), candidate r % 2
-      const int64_t row = start + static_cast<int64_t>(r & 1) * kFastThreads + word + kWords * (r >> 1);
-      if (half == 0 && row < stop) {
+      // byte r of word `word` is row r W + word of the block
+      const int64_t row = start + r * W + word;
+      if (grp == 0 && row < stop) {
         float s;
         if (S > 1) {
           s = fv.base;
           for (int q = 0; q < S; ++q) s += __ldcg(sl.scores + static_cast<size_t>(q) * sl.pairs + lo + row);
         } else {
-          s = (fv.base + score[r]) + s_part[r * kWords + word];
+          s = fv.base + total[r];
         }
         keys[r] = make_key(s + 0.0f, seg_off ? seg_idx[lo + row] : static_cast<int>(row));
       }
@@ -770,6 +839,7 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
     __syncthreads();
     block_topk<5>(keys, k, s_warp, s_list);
   }
+  if (sl.score_out) return;
   if (tid < k) partial[(static_cast<size_t>(prob) * nblk + chunk) * k + tid] = s_list[tid];
   if (S > 1 && sl.out_idx) {
     // single-problem form: the last block to finish merges the per-block lists (one warp)
@@ -839,6 +909,50 @@ static std::vector<PartitionCode> partition_codes(int L) {
   return code;
 }
 
+// Tile geometry by the number of rows: the [row][candidate] tile and the two chunk buffers have to
+// fit the shared memory of one SM (228 KiB, 1 KiB of it reserved per CTA; a CTA's own limit is
+// 227 KiB including its static part). Two CTAs of 512 threads per SM are preferred, since one
+// CTA's tile fill and ranking then overlap the other's walk: with 1,024 candidates each up to 72
+// rows, with 512 candidates up to 149. Beyond that one CTA of 1,024 threads: 1,024 candidates up
+// to 183 rows, 512 candidates up to 367. Every CTA streams the whole ensemble, so a halved block
+// doubles that traffic. More rows than that: the general kernel. A single CTA per SM takes
+// 32 KB chunk buffers when they fit. KS_FAST_GEOMETRY="threads,candidates,buffer KiB" overrides
+// the choice (a tuning aid; a geometry that does not fit is refused).
+struct Geometry {
+  int threads, cands, buf_bytes, ctas_per_sm;
+};
+static size_t geometry_smem(const Geometry& g, int n_rows) {
+  const size_t stat = g.threads == 512 ? 6656 + 256 : 10752 + 256;  // static shared memory of the kernel, with slack
+  return static_cast<size_t>(kNBuf) * g.buf_bytes + static_cast<size_t>(n_rows) * g.cands + stat;
+}
+static bool geometry_fits(const Geometry& g, int n_rows) {
+  const size_t per_cta = geometry_smem(g, n_rows);
+  if (per_cta > 227 * 1024) return false;
+  return g.ctas_per_sm * (per_cta + 1024) <= 228 * 1024;
+}
+static bool pick_geometry(int n_rows, Geometry* out) {
+  if (const char* env = std::getenv("KS_FAST_GEOMETRY")) {
+    int t = 0, c = 0, kb = 0;
+    if (std::sscanf(env, "%d,%d,%d", &t, &c, &kb) == 3 && (t == 512 || t == 1024) && (c == 512 || c == 1024) &&
+        (kb == 16 || kb == 32)) {
+      Geometry g{t, c, kb * 1024, t == 512 ? 2 : 1};
+      if (!geometry_fits(g, n_rows)) g.ctas_per_sm = 1;
+      if (geometry_fits(g, n_rows)) {
+        *out = g;
+        return true;
+      }
+    }
+  }
+  const Geometry order[] = {{512, 1024, kBufBytes, 2},      {512, 512, kBufBytes, 2},  {1024, 1024, 2 * kBufBytes, 1},
+                            {1024, 1024, kBufBytes, 1},     {1024, 512, 2 * kBufBytes, 1}, {1024, 512, kBufBytes, 1}};
+  for (const Geometry& g : order)
+    if (geometry_fits(g, n_rows)) {
+      *out = g;
+      return true;
+    }
+  return false;
+}
+
 cudaError_t build_fast_gbdt(GbdtModel& m, int n_trees, const int64_t* off, const ks_node_host* nodes) {
   m.fast = false;
   if (n_trees < 1 || m.max_depth < 1 || m.max_depth > kFastMaxDepth) return cudaSuccess;
@@ -867,50 +981,58 @@ cudaError_t build_fast_gbdt(GbdtModel& m, int n_trees, const int64_t* off, const
       thr[nd.feat].push_back(nd.thr_or_leaf);
     }
   }
-  std::vector<uint8_t> row0(64, 0), rowcnt(64, 0);
+  FeatQ fq[64];
+  std::memset(fq, 0, sizeof(fq));
   int rank_row[KS_F][3];  // row offset (within the feature's rows) of each permutation in use
-  int n_rows = 0, n_class[3] = {0, 0, 0};
+  int n_rows = 0, n_class[3] = {0, 0, 0}, thr_class[3] = {0, 0, 0};
   for (int f = 0; f < KS_F; ++f) {
     auto& v = thr[f];
     std::sort(v.begin(), v.end());
     v.erase(std::unique(v.begin(), v.end()), v.end());
-    int cnt = static_cast<int>((v.size() + 126) / 127);
-    for (int q = 0; q < 3; ++q) rank_row[f][q] = perm_used[f][q] ? cnt++ : -1;
-    rowcnt[f] = static_cast<uint8_t>(cnt);
+    if (v.size() > 65000) return cudaSuccess;
+    const int n_slices = static_cast<int>((v.size() + kSlice - 1) / kSlice);
+    int cnt = n_slices, n_rank = 0;
+    for (int q = 0; q < 3; ++q) {
+      rank_row[f][q] = perm_used[f][q] ? cnt++ : -1;
+      if (perm_used[f][q]) {
+        const int L = categorical_levels(f);
+        for (int r = 0; r < L; ++r) fq[f].rank[n_rank][partition_perm(L, q)[r]] = static_cast<uint8_t>(r);
+        ++n_rank;
+      }
+    }
+    fq[f].nthr = static_cast<uint16_t>(v.size());
+    fq[f].nslice = static_cast<uint16_t>(n_slices);
+    fq[f].nrank = static_cast<uint16_t>(n_rank);
     n_class[feat_class(f)] += cnt;
+    thr_class[feat_class(f)] += static_cast<int>(v.size());
     n_rows += cnt;
   }
-  if (n_rows == 0 || n_rows > kMaxRows || n_class[1] > kCandRec) return cudaSuccess;  // generic path
-  // rows ordered: per-pair, candidate-only, problem-only
-  std::vector<float> table(static_cast<size_t>(n_rows) * kThrPerRow, std::numeric_limits<float>::infinity());
+  Geometry geom{};
+  if (n_rows == 0 || !pick_geometry(n_rows, &geom)) return cudaSuccess;  // generic path
+  if (n_class[0] > kFastMaxProbRows || n_class[1] > kFastMaxCandRec) return cudaSuccess;
+  const int NC = geom.cands, threads = geom.threads;
+  // rows and thresholds ordered: per-pair, candidate-only, problem-only features
+  std::vector<float> table;
   int next = 0;
   for (int cls : {2, 1, 0}) {
     for (int f = 0; f < KS_F; ++f) {
       if (feat_class(f) != cls) continue;
-      row0[f] = static_cast<uint8_t>(next);
-      const int n_thr_rows = static_cast<int>((thr[f].size() + 126) / 127);
-      for (int q = 0; q < n_thr_rows; ++q, ++next)
-        for (int j = 0; j < 127; ++j) {
-          const size_t s = static_cast<size_t>(q) * 127 + j;
-          if (s < thr[f].size()) table[static_cast<size_t>(next) * kThrPerRow + j] = thr[f][s];
-        }
-      for (int q = 0; q < 3; ++q) {  // rank rows: slot c = rank of level c, last slot = marker
-        if (rank_row[f][q] < 0) continue;
-        const int L = categorical_levels(f);
-        float* row = table.data() + static_cast<size_t>(next) * kThrPerRow;
-        for (int c = 0; c < 4; ++c) row[c] = 0.0f;
-        for (int r = 0; r < L; ++r) row[partition_perm(L, q)[r]] = static_cast<float>(r);
-        row[kThrPerRow - 1] = -std::numeric_limits<float>::infinity();
-        ++next;
-      }
+      fq[f].row0 = static_cast<uint16_t>(next);
+      fq[f].thr0 = static_cast<uint32_t>(table.size());
+      table.insert(table.end(), thr[f].begin(), thr[f].end());
+      next += fq[f].nslice + fq[f].nrank;
     }
   }
+  if (table.empty()) table.push_back(0.0f);
+  const int G = threads / (NC / 4);
   const int per_tree_words = (2 << D) - 1;
-  int tpc = kBufBytes / (per_tree_words * 4) / 2 * 2;  // even: the two halves of a CTA share a chunk's trees
+  int tpc = geom.buf_bytes / (per_tree_words * 4) / 2 * 2;  // even: the two groups of the smallest geometry share a chunk's trees
   if (tpc < 2) return cudaSuccess;
-  if (tpc > (n_trees + 1) / 2 * 2) tpc = (n_trees + 1) / 2 * 2;  // a small ensemble is one short chunk
+  if (tpc >= G) tpc = tpc / G * G;  // whole groups (fewer trees than groups: the spare groups idle)
+  if (tpc > (n_trees + G - 1) / G * G) tpc = (n_trees + G - 1) / G * G;  // a small ensemble is one short chunk
   const int n_chunks = (n_trees + tpc - 1) / tpc;
   const int chunk_words = (tpc * per_tree_words + 3) / 4 * 4;  // bulk copies move multiples of 16 bytes
+  if (chunk_words * 4 > geom.buf_bytes) return cudaSuccess;
   int L = D < 3 ? D : 3;  // levels whose nodes travel as kernel-parameter constants
   while (L > 0 && static_cast<int64_t>(n_chunks) * tpc * ((1 << L) - 1) > kFastTopPairs) --L;
   // three levels in the compact form (one word per node) when the pair form would leave fewer
@@ -957,23 +1079,23 @@ cudaError_t build_fast_gbdt(GbdtModel& m, int n_trees, const int64_t* off, const
                   jl = 127;
                 } else {
                   const PartitionCode pc = part[nd.feat][mask];
-                  row = row0[nd.feat] + rank_row[nd.feat][pc.perm];
+                  row = fq[nd.feat].row0 + rank_row[nd.feat][pc.perm];
                   jl = pc.cut - 1;
                   swap = pc.swap;
                 }
               } else {
                 const auto& v = thr[nd.feat];
                 const int j = static_cast<int>(std::lower_bound(v.begin(), v.end(), nd.thr_or_leaf) - v.begin());
-                row = row0[nd.feat] + j / 127;
-                jl = j % 127;
+                row = fq[nd.feat].row0 + j / kSlice;
+                jl = j % kSlice;
               }
               ls = nd.left;
               rs = nd.left + 1;
               if (always_right) {
                 ls = rs;  // the walk always goes left here: put the right subtree on both sides
               } else {
-                word = (row * kRowStride) << 8 | (0x80u | jl);
-                tw = make_uint2(row * kRowStride, (jl + 1) * 0x01010101u);
+                word = (row * NC) << 8 | (0x80u | jl);
+                tw = make_uint2(row * NC, (jl + 1) * 0x01010101u);
                 if (swap) std::swap(ls, rs);
               }
             }
@@ -1003,10 +1125,8 @@ cudaError_t build_fast_gbdt(GbdtModel& m, int n_trees, const int64_t* off, const
   if (e == cudaSuccess) e = cudaMemcpy(m.d_qnodes, chunks.data(), chunks.size() * 4, cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&m.d_qthr), table.size() * 4);
   if (e == cudaSuccess) e = cudaMemcpy(m.d_qthr, table.data(), table.size() * 4, cudaMemcpyHostToDevice);
-  if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&m.d_qrow0), 64);
-  if (e == cudaSuccess) e = cudaMemcpy(m.d_qrow0, row0.data(), 64, cudaMemcpyHostToDevice);
-  if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&m.d_qrowcnt), 64);
-  if (e == cudaSuccess) e = cudaMemcpy(m.d_qrowcnt, rowcnt.data(), 64, cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaMalloc(reinterpret_cast<void**>(&m.d_qfeat), sizeof(fq));
+  if (e == cudaSuccess) e = cudaMemcpy(m.d_qfeat, fq, sizeof(fq), cudaMemcpyHostToDevice);
   if (e != cudaSuccess) {
     delete top;
     return e;
@@ -1016,10 +1136,17 @@ cudaError_t build_fast_gbdt(GbdtModel& m, int n_trees, const int64_t* off, const
   m.top_compact = compact;
   m.fast = true;
   m.fast_depth = D;
+  m.fast_threads = threads;
+  m.block_cands = NC;
+  m.buf_bytes = geom.buf_bytes;
+  m.ctas_per_sm = geom.ctas_per_sm;
   m.n_qrows = n_rows;
   m.n_pair_rows = n_class[2];
   m.n_cand_rows = n_class[1];
   m.n_prob_rows = n_class[0];
+  m.n_qthr = thr_class[0] + thr_class[1] + thr_class[2];
+  m.thr_cand0 = thr_class[2];
+  m.thr_prob0 = thr_class[2] + thr_class[1];
   m.tpc = tpc;
   m.n_chunks = n_chunks;
   m.chunk_bytes = chunk_words * 4;
@@ -1035,21 +1162,27 @@ void free_fast_gbdt(GbdtModel& m) {
 // launcher
 // ------------------------------------------------------------------------------------------
 
-// Blocks per problem: full tiles of kFastRows rows. A block's cost does not depend on how many
-// of its slots are live, so an under-filled machine is filled by splitting the trees over
+// Blocks per problem: full tiles of the model's block size. A block's cost does not depend on how
+// many of its slots are live, so an under-filled machine is filled by splitting the trees over
 // several CTAs per block (slices) rather than by shorter blocks.
-void fast_tiling(int P, int64_t per_problem, int* nblk, int* rows_per_cta) {
-  int64_t n = (per_problem + kFastRows - 1) / kFastRows;
+void fast_tiling(const GbdtModel& g, int P, int64_t per_problem, int* nblk, int* rows_per_cta) {
+  int64_t n = (per_problem + g.block_cands - 1) / g.block_cands;
   if (n < 1) n = 1;
   (void)P;
   *nblk = static_cast<int>(n);
-  *rows_per_cta = kFastRows;
+  *rows_per_cta = g.block_cands;
 }
 
-size_t fast_scratch_bytes(int C) { return 256 + static_cast<size_t>(kCombos) * C * kCandRec; }
+static int cand_rec_bytes(const GbdtModel& g) { return g.n_cand_rows > 0 ? (g.n_cand_rows + 15) / 16 * 16 : 16; }
+static int pair_rec_bytes(const GbdtModel& g) { return (g.n_pair_rows + 15) / 16 * 16; }
+
+size_t fast_scratch_bytes(const GbdtModel& g, int C) {
+  return 256 + static_cast<size_t>(kCombos) * C * cand_rec_bytes(g);
+}
 
 // Memo of the per-pair rows (see MemoView): worth its per-problem table only for a batch of
-// problems, and only when the per-pair rows fit a record. 0 = not used.
+// problems. The table is held for at most `fast_memo_batch` problems at a time (256 MiB of
+// records); a larger call is served batch by batch. 0 = not used.
 size_t memo_fixed_bytes(int C) {
   return static_cast<size_t>(kMemoCombos) * kMemoCap * (sizeof(unsigned long long) + 2 * sizeof(int)) + 256 +
          (static_cast<size_t>(kMemoCombos) * C * sizeof(unsigned) + 255) / 256 * 256;
@@ -1074,161 +1207,91 @@ cudaError_t memo_compact(const MemoView& memo, cudaStream_t stream) {
   return cudaGetLastError();
 }
 
-size_t fast_memo_bytes(const GbdtModel& g, int P, int C) {
-  if (P < kMemoMinProblems || P > kMemoMaxProblems || C < 1 || g.n_pair_rows < 1 || g.n_pair_rows > kMemoRec) return 0;
-  return memo_fixed_bytes(C) + static_cast<size_t>(P) * kMemoCap * kMemoRec;
+int fast_memo_batch(const GbdtModel& g, int P) {
+  if (P < kMemoMinProblems || g.n_pair_rows < 1 || g.n_pair_rows > kFastMaxPairRec) return 0;
+  const size_t per_problem = static_cast<size_t>(kMemoCap) * pair_rec_bytes(g);
+  int64_t batch = static_cast<int64_t>(kMemoTableBytes / per_problem);
+  if (batch < kMemoMinProblems) batch = kMemoMinProblems;
+  return static_cast<int>(batch < P ? batch : P);
 }
 
-// Slice count of the single-problem call: as many tree slices as keep every CTA in the first
-// wave (one CTA per SM).
+size_t fast_memo_bytes(const GbdtModel& g, int P, int C) {
+  const int batch = fast_memo_batch(g, P);
+  if (batch == 0 || C < 1) return 0;
+  return memo_fixed_bytes(C) + static_cast<size_t>(batch) * kMemoCap * pair_rec_bytes(g);
+}
+
+// Slice count of the single-problem call: as many tree slices as keep every CTA in the first wave.
 int fast_slices(const GbdtModel& g, int64_t blocks) {
   if (blocks < 1) blocks = 1;
   if (blocks > kMaxSliceBlocks) return 1;
-  int64_t s = 296 / blocks;
+  int64_t s = (g.ctas_per_sm * 148) / blocks;
   if (s > g.n_chunks) s = g.n_chunks;
   return static_cast<int>(s < 1 ? 1 : s);
 }
 
-template <int L, int NP, bool kCompact = false>
-static cudaError_t launch_ln(const ks_gpu_desc& desc, const ks_problem* d_p, const ks_problem& pv, int uv, int P,
-                             const ks_candidate* d_c, int C, int nblk, int rows_per_cta, const int64_t* seg_off,
-                             const int32_t* seg_idx, const FastView& fv, int k, unsigned long long* partial,
-                             int* status, const SliceArgs& sl, const FastTopParams& top, cudaStream_t stream) {
-  const size_t smem = kOffTile + static_cast<size_t>(fv.n_rows) * kRowStride;
-  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(&select_fast_kernel<L, NP, kCompact>), smem);
+namespace {
+
+struct WalkArgs {
+  ks_gpu_desc desc;
+  const ks_problem* d_p;
+  ks_problem pv;
+  int uv;
+  const ks_candidate* d_c;
+  int P, C, nblk, rows_per_cta;
+  const int64_t* seg_off;
+  const int32_t* seg_idx;
+  FastView fv;
+  int k;
+  unsigned long long* partial;
+  int* status;
+  SliceArgs sl;
+  const FastTopParams* top;
+  cudaStream_t stream;
+};
+
+template <int L, int NP, bool kCompact, int THREADS, int NC>
+cudaError_t launch_ln(const WalkArgs& a) {
+  const size_t smem = static_cast<size_t>(kNBuf) * a.fv.buf_bytes + static_cast<size_t>(a.fv.n_rows) * NC;
+  auto kernel = &select_fast_kernel<L, NP, kCompact, THREADS, NC>;
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), smem);
   if (e != cudaSuccess) return e;
-  select_fast_kernel<L, NP, kCompact><<<static_cast<unsigned>(static_cast<int64_t>(P) * nblk * sl.n_slices), kFastThreads, smem,
-                              stream>>>(desc, d_p, pv, uv, d_c, P, C, nblk, rows_per_cta, seg_off, seg_idx, fv, k,
-                                        partial, status, sl, top);
+  kernel<<<static_cast<unsigned>(static_cast<int64_t>(a.P) * a.nblk * a.sl.n_slices), THREADS, smem, a.stream>>>(
+      a.desc, a.d_p, a.pv, a.uv, a.d_c, a.P, a.C, a.nblk, a.rows_per_cta, a.seg_off, a.seg_idx, a.fv, a.k, a.partial,
+      a.status, a.sl, *a.top);
   return cudaGetLastError();
 }
 
-cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, const ks_problem* d_p,
-                               const ks_problem* p_by_value, int P, const ks_candidate* d_c, int C,
-                               int nblk, int rows_per_cta, const int64_t* seg_off, const int32_t* seg_idx,
-                               int k, unsigned long long* partial, void* scratch, int* status,
-                               cudaStream_t stream, int64_t* launches, cudaEvent_t ev_begin,
-                               const FastSlice* slice, void* memo_mem) {
-  ks_problem pv{};
-  if (p_by_value) pv = *p_by_value;
-  const int uv = p_by_value != nullptr;
-  FastView fv;
-  fv.n_rows = g.n_qrows;
-  fv.n_pair_rows = g.n_pair_rows;
-  fv.n_cand_rows = g.n_cand_rows;
-  fv.n_prob_rows = g.n_prob_rows;
-  fv.depth = g.fast_depth;
-  fv.n_chunks = g.n_chunks;
-  fv.chunk_bytes = g.chunk_bytes;
-  fv.tpc = g.tpc;
-  fv.base = g.base;
-  fv.chunks = g.d_qnodes;
-  fv.thr = g.d_qthr;
-  fv.feat_row0 = g.d_qrow0;
-  fv.feat_rowcnt = g.d_qrowcnt;
-  unsigned* d_mask = static_cast<unsigned*>(scratch);
-  uint8_t* d_rows = static_cast<uint8_t*>(scratch) + 256;
-  fv.cand_rows = d_rows;
-  fv.pair_class = nullptr;
-  fv.pair_tab = nullptr;
-  MemoView memo{};
-  if (memo_mem && !p_by_value && fast_memo_bytes(g, P, C) != 0) memo = memo_view(memo_mem, C);
-
-  // candidate-only rows for the type combinations in use
-  cudaError_t e = cudaSuccess;
-  unsigned mask_value = 0;
-  if (uv) {
-    mask_value = 1u << ((pv.dtype_ab & 3) * 4 + (pv.dtype_d & 3));
-  } else {
-    e = cudaMemsetAsync(d_mask, 0, sizeof(unsigned), stream);
-    if (e != cudaSuccess) return e;
-    combo_mask_kernel<<<P >= 4096 ? 16 : 1, 256, 0, stream>>>(d_p, P, d_mask);
-    ++*launches;
-  }
-  const bool tiles_mode = uv && slice && slice->n_slices > 1 && slice->tiles && P == 1 && !seg_off;
-  if (tiles_mode) {
-    // one launch, two roles (blockIdx.y): the per-pair rows, and the candidate- / problem-only rows
-    const size_t tthr = sizeof(float) * kThrPerRow * g.n_qrows;
-    e = ensure_dynamic_smem(reinterpret_cast<const void*>(&tile_one_kernel), tthr);
-    if (e != cudaSuccess) return e;
-    tile_one_kernel<<<dim3(nblk * (kFastRows / 256), 2), 256, tthr, stream>>>(desc, pv, d_c, C, fv, slice->tiles);
-    ++*launches;
-  } else if (C > 0) {
-    const size_t cthr = sizeof(float) * kThrPerRow * (g.n_cand_rows > 0 ? g.n_cand_rows : 1);
-    if (memo.keys) {
-      e = memo_clear(memo, stream);
-      if (e != cudaSuccess) return e;
-    }
-    cand_rows_kernel<<<dim3((C + 255) / 256, kCombos), 256, cthr, stream>>>(desc, d_c, C, uv ? nullptr : d_mask,
-                                                                            mask_value, fv, d_rows, memo);
-    ++*launches;
-    if (memo.keys) {
-      const size_t pthr = sizeof(float) * kThrPerRow * g.n_pair_rows;
-      e = ensure_dynamic_smem(reinterpret_cast<const void*>(&pair_table_kernel), pthr);
-      if (e != cudaSuccess) return e;
-      e = memo_compact(memo, stream);
-      if (e != cudaSuccess) return e;
-      pair_table_kernel<<<dim3(kMemoCap / 256, P), 256, pthr, stream>>>(desc, d_p, d_c, fv, memo);
-      *launches += 2;
-      fv.pair_class = memo.cls;
-      fv.pair_tab = static_cast<const uint8_t*>(memo.tab);
-    }
-  }
-  e = cudaGetLastError();
-  if (e != cudaSuccess) return e;
-  if (ev_begin) cudaEventRecord(ev_begin, stream);
-
-  SliceArgs sl{};
-  sl.n_slices = 1;
-  if (slice && slice->n_slices > 1) {
-    sl.n_slices = slice->n_slices;
-    sl.pairs = slice->pairs;
-    sl.scores = slice->scores;
-    sl.counters = slice->counters;
-    sl.out_idx = slice->out_idx;
-    sl.out_score = slice->out_score;
-    sl.tiles = tiles_mode ? slice->tiles : nullptr;
-    sl.out_seq = slice->out_seq;
-    sl.seq = slice->seq;
-  }
-  const FastTopParams& top = *g.h_top;
+// the instantiation for a model's top levels and depth, within one tile geometry
+template <int THREADS, int NC>
+cudaError_t launch_walk_geom(const GbdtModel& g, const WalkArgs& a) {
   const int L = g.top_levels, np = g.fast_depth - L;
-  ++*launches;
-#define KS_GO(LL, NN) \
-  return launch_ln<LL, NN>(desc, d_p, pv, uv, P, d_c, C, nblk, rows_per_cta, seg_off, seg_idx, fv, k, partial, status, sl, top, stream)
   if (g.top_compact) {
-#define KS_GOC(NN) \
-  return launch_ln<3, NN, true>(desc, d_p, pv, uv, P, d_c, C, nblk, rows_per_cta, seg_off, seg_idx, fv, k, partial, status, sl, top, stream)
-    if (np == 5) KS_GOC(5);
-    if (np == 4) KS_GOC(4);
-    KS_GOC(-1);
-#undef KS_GOC
+    if (np == 5) return launch_ln<3, 5, true, THREADS, NC>(a);
+    if (np == 4) return launch_ln<3, 4, true, THREADS, NC>(a);
+    return launch_ln<3, -1, true, THREADS, NC>(a);
   }
-  if (L == 3 && np == 5) KS_GO(3, 5);
-  if (L == 3 && np == 3) KS_GO(3, 3);
-  if (L == 2 && np == 6) KS_GO(2, 6);
-  if (L == 2 && np == 5) KS_GO(2, 5);  // the paper-sized ensemble: 916 trees of depth 7
-  if (L == 3 && np == 4) KS_GO(3, 4);
-  if (L == 3) KS_GO(3, -1);
-  if (L == 2) KS_GO(2, -1);
-  if (L == 1) KS_GO(1, -1);
-  KS_GO(0, -1);
-#undef KS_GO
+  if (L == 3 && np == 5) return launch_ln<3, 5, false, THREADS, NC>(a);
+  if (THREADS == 512 && NC == 1024) {  // the shapes met so far only in small ensembles
+    if (L == 3 && np == 3) return launch_ln<3, 3, false, 512, 1024>(a);
+    if (L == 2 && np == 6) return launch_ln<2, 6, false, 512, 1024>(a);
+    if (L == 2 && np == 5) return launch_ln<2, 5, false, 512, 1024>(a);  // the paper-sized ensemble: 916 trees of depth 7
+  }
+  if (L == 3 && np == 4) return launch_ln<3, 4, false, THREADS, NC>(a);
+  if (L == 3) return launch_ln<3, -1, false, THREADS, NC>(a);
+  if (L == 2) return launch_ln<2, -1, false, THREADS, NC>(a);
+  if (L == 1) return launch_ln<1, -1, false, THREADS, NC>(a);
+  return launch_ln<0, -1, false, THREADS, NC>(a);
 }
 
-// ks_score on the quantised path. Rows are taken in batches so that the tiles (n_rows bytes per
-// row) stay a bounded workspace; every batch is one tile launch and one walk launch.
-constexpr int64_t kScoreBatchBlocks = 4096;
-
-size_t score_fast_scratch_bytes(const GbdtModel& g, int64_t rows) {
-  int64_t blocks = (rows + kFastRows - 1) / kFastRows;
-  if (blocks > kScoreBatchBlocks) blocks = kScoreBatchBlocks;
-  return static_cast<size_t>(blocks) * g.n_qrows * kRowStride;
+cudaError_t launch_walk(const GbdtModel& g, const WalkArgs& a) {
+  if (g.fast_threads == 512 && g.block_cands == 1024) return launch_walk_geom<512, 1024>(g, a);
+  if (g.fast_threads == 512) return launch_walk_geom<512, 512>(g, a);
+  if (g.block_cands == 1024) return launch_walk_geom<1024, 1024>(g, a);
+  return launch_walk_geom<1024, 512>(g, a);
 }
 
-cudaError_t launch_score_fast(const ks_gpu_desc& desc, const GbdtModel& g, const float* d_feat, int64_t rows,
-                              float* d_scores, void* scratch, int* status, cudaStream_t stream,
-                              int64_t* launches) {
+FastView make_view(const GbdtModel& g, const FastWait* wait) {
   FastView fv{};
   fv.n_rows = g.n_qrows;
   fv.n_pair_rows = g.n_pair_rows;
@@ -1238,48 +1301,199 @@ cudaError_t launch_score_fast(const ks_gpu_desc& desc, const GbdtModel& g, const
   fv.n_chunks = g.n_chunks;
   fv.chunk_bytes = g.chunk_bytes;
   fv.tpc = g.tpc;
+  fv.n_thr = g.n_qthr;
+  fv.thr_cand0 = g.thr_cand0;
+  fv.thr_prob0 = g.thr_prob0;
+  fv.cand_rec = cand_rec_bytes(g);
+  fv.pair_rec = pair_rec_bytes(g);
+  fv.wait_limit = wait && wait->limit > 0 ? wait->limit : kFastWaitLimit;
+  fv.starve = wait ? wait->starve : 0;
+  fv.buf_bytes = g.buf_bytes;
   fv.base = g.base;
   fv.chunks = g.d_qnodes;
   fv.thr = g.d_qthr;
-  fv.feat_row0 = g.d_qrow0;
-  fv.feat_rowcnt = g.d_qrowcnt;
-  uint8_t* tiles = static_cast<uint8_t*>(scratch);
-  const size_t tthr = sizeof(float) * kThrPerRow * g.n_qrows;
-  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(&tile_rows_kernel), tthr);
-  if (e != cudaSuccess) return e;
-  const FastTopParams& top = *g.h_top;
-  const int L = g.top_levels, np = g.fast_depth - L;
-  const ks_problem pv{};
-  for (int64_t first = 0; first < rows; first += kScoreBatchBlocks * kFastRows) {
-    const int64_t n = rows - first < kScoreBatchBlocks * kFastRows ? rows - first : kScoreBatchBlocks * kFastRows;
-    const int nblk = static_cast<int>((n + kFastRows - 1) / kFastRows);
-    tile_rows_kernel<<<nblk, kWords, tthr, stream>>>(d_feat + first * KS_F_PAD, n, fv, tiles);
-    e = cudaGetLastError();
+  fv.feat = g.d_qfeat;
+  return fv;
+}
+
+// Dynamic shared memory for `count` staged thresholds: all of them when they fit, else none (the
+// kernel then searches the global array). Returns the capacity in floats to pass to the kernel.
+int staged_floats(int count, size_t* bytes) {
+  constexpr int kCap = 48 * 1024;  // floats: 192 KB
+  const int cap = count <= kCap ? (count > 0 ? count : 1) : 0;
+  *bytes = static_cast<size_t>(cap > 0 ? cap : 1) * sizeof(float);
+  return cap;
+}
+
+}  // namespace
+
+cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, const ks_problem* d_p,
+                               const ks_problem* p_by_value, int P, const ks_candidate* d_c, int C,
+                               int nblk, int rows_per_cta, const int64_t* seg_off, const int32_t* seg_idx,
+                               int k, unsigned long long* partial, void* scratch, int* status,
+                               cudaStream_t stream, int64_t* launches, cudaEvent_t ev_begin,
+                               const FastSlice* slice, void* memo_mem, const FastWait* wait) {
+  WalkArgs a{};
+  a.desc = desc;
+  if (p_by_value) a.pv = *p_by_value;
+  a.uv = p_by_value != nullptr;
+  a.d_c = d_c;
+  a.C = C;
+  a.nblk = nblk;
+  a.rows_per_cta = rows_per_cta;
+  a.seg_idx = seg_idx;
+  a.k = k;
+  a.status = status;
+  a.top = g.h_top;
+  a.stream = stream;
+  FastView& fv = a.fv;
+  fv = make_view(g, wait);
+  unsigned* d_mask = static_cast<unsigned*>(scratch);
+  uint8_t* d_rows = static_cast<uint8_t*>(scratch) + 256;
+  fv.cand_rows = d_rows;
+  MemoView memo{};
+  const int memo_batch = (memo_mem && !p_by_value && C > 0) ? fast_memo_batch(g, P) : 0;
+  if (memo_batch > 0) memo = memo_view(memo_mem, C);
+
+  // candidate-only rows for the type combinations in use
+  cudaError_t e = cudaSuccess;
+  unsigned mask_value = 0;
+  if (a.uv) {
+    mask_value = 1u << ((a.pv.dtype_ab & 3) * 4 + (a.pv.dtype_d & 3));
+  } else {
+    e = cudaMemsetAsync(d_mask, 0, sizeof(unsigned), stream);
     if (e != cudaSuccess) return e;
-    SliceArgs sl{};
-    sl.n_slices = 1;
-    sl.tiles = tiles;
-    sl.score_out = d_scores + first;
-    *launches += 2;
-#define KS_GO(LL, NN)                                                                                          \
-  e = launch_ln<LL, NN>(desc, nullptr, pv, 1, 1, nullptr, static_cast<int>(n), nblk, kFastRows, nullptr, nullptr, \
-                        fv, 0, nullptr, status, sl, top, stream)
-    if (g.top_compact && np == 5) e = launch_ln<3, 5, true>(desc, nullptr, pv, 1, 1, nullptr, static_cast<int>(n), nblk, kFastRows, nullptr, nullptr, fv, 0, nullptr, status, sl, top, stream);
-    else if (g.top_compact && np == 4) e = launch_ln<3, 4, true>(desc, nullptr, pv, 1, 1, nullptr, static_cast<int>(n), nblk, kFastRows, nullptr, nullptr, fv, 0, nullptr, status, sl, top, stream);
-    else if (g.top_compact) e = launch_ln<3, -1, true>(desc, nullptr, pv, 1, 1, nullptr, static_cast<int>(n), nblk, kFastRows, nullptr, nullptr, fv, 0, nullptr, status, sl, top, stream);
-    else if (L == 3 && np == 5) KS_GO(3, 5);
-    else if (L == 3 && np == 3) KS_GO(3, 3);
-    else if (L == 2 && np == 6) KS_GO(2, 6);
-    else if (L == 2 && np == 5) KS_GO(2, 5);
-    else if (L == 3 && np == 4) KS_GO(3, 4);
-    else if (L == 3) KS_GO(3, -1);
-    else if (L == 2) KS_GO(2, -1);
-    else if (L == 1) KS_GO(1, -1);
-    else KS_GO(0, -1);
-#undef KS_GO
+    combo_mask_kernel<<<P >= 4096 ? 16 : 1, 256, 0, stream>>>(d_p, P, d_mask);
+    ++*launches;
+  }
+  const bool tiles_mode = a.uv && slice && slice->n_slices > 1 && slice->tiles && P == 1 && !seg_off;
+  size_t pthr_bytes = 0;
+  const int pthr_cap = staged_floats(g.thr_cand0, &pthr_bytes);
+  if (tiles_mode) {
+    // one launch, two roles (blockIdx.y): the per-pair rows, and the candidate- / problem-only rows
+    size_t tthr = 0;
+    const int cap = staged_floats(std::max(g.thr_cand0, g.n_qthr - g.thr_cand0), &tthr);
+    e = ensure_dynamic_smem(reinterpret_cast<const void*>(&tile_one_kernel), tthr);
+    if (e != cudaSuccess) return e;
+    tile_one_kernel<<<dim3(nblk * (g.block_cands / 256), 2), 256, tthr, stream>>>(desc, a.pv, d_c, C, fv,
+                                                                                   g.block_cands, slice->tiles, cap);
+    ++*launches;
+  } else if (C > 0) {
+    size_t cthr = 0;
+    const int cap = staged_floats(g.thr_prob0 - g.thr_cand0, &cthr);
+    e = ensure_dynamic_smem(reinterpret_cast<const void*>(&cand_rows_kernel), cthr);
+    if (e != cudaSuccess) return e;
+    if (memo.keys) {
+      e = memo_clear(memo, stream);
+      if (e != cudaSuccess) return e;
+    }
+    cand_rows_kernel<<<dim3((C + 255) / 256, kCombos), 256, cthr, stream>>>(desc, d_c, C, a.uv ? nullptr : d_mask,
+                                                                            mask_value, fv, d_rows, memo, cap);
+    ++*launches;
+    if (memo.keys) {
+      e = ensure_dynamic_smem(reinterpret_cast<const void*>(&pair_table_kernel), pthr_bytes);
+      if (e != cudaSuccess) return e;
+      e = memo_compact(memo, stream);
+      if (e != cudaSuccess) return e;
+      ++*launches;
+      fv.pair_class = memo.cls;
+      fv.pair_tab = static_cast<const uint8_t*>(memo.tab);
+    }
+  }
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  if (ev_begin) cudaEventRecord(ev_begin, stream);
+
+  a.sl.n_slices = 1;
+  if (slice && slice->n_slices > 1) {
+    a.sl.n_slices = slice->n_slices;
+    a.sl.pairs = slice->pairs;
+    a.sl.scores = slice->scores;
+    a.sl.counters = slice->counters;
+    a.sl.out_idx = slice->out_idx;
+    a.sl.out_score = slice->out_score;
+    a.sl.tiles = tiles_mode ? slice->tiles : nullptr;
+    a.sl.out_seq = slice->out_seq;
+    a.sl.seq = slice->seq;
+  }
+  // problems in batches when the memo's table does not hold them all at once
+  const int step = memo.keys ? memo_batch : P;
+  for (int first = 0; first < P; first += step) {
+    const int n = P - first < step ? P - first : step;
+    if (memo.keys) {
+      pair_table_kernel<<<dim3(kMemoCap / 256, n), 256, pthr_bytes, stream>>>(desc, d_p + first, d_c, fv, memo,
+                                                                              pthr_cap);
+      ++*launches;
+    }
+    a.d_p = d_p ? d_p + first : nullptr;
+    a.P = n;
+    a.seg_off = seg_off ? seg_off + first : nullptr;
+    a.partial = partial + static_cast<size_t>(first) * nblk * k;
+    e = launch_walk(g, a);
+    ++*launches;
     if (e != cudaSuccess) return e;
   }
   return cudaSuccess;
 }
+
+// ks_score on the quantised path. Rows are taken in batches so that the tiles (n_rows bytes per
+// row) stay a bounded workspace; every batch is one tile launch and one walk launch.
+constexpr int64_t kScoreBatchRows = 4096 * 1024;
+
+size_t score_fast_scratch_bytes(const GbdtModel& g, int64_t rows) {
+  int64_t blocks = (std::min(rows, kScoreBatchRows) + g.block_cands - 1) / g.block_cands;
+  return static_cast<size_t>(blocks) * g.n_qrows * g.block_cands;
+}
+
+cudaError_t launch_score_fast(const ks_gpu_desc& desc, const GbdtModel& g, const float* d_feat, int64_t rows,
+                              float* d_scores, void* scratch, int* status, cudaStream_t stream,
+                              int64_t* launches, const FastWait* wait) {
+  WalkArgs a{};
+  a.desc = desc;
+  a.uv = 1;
+  a.P = 1;
+  a.rows_per_cta = g.block_cands;
+  a.status = status;
+  a.top = g.h_top;
+  a.stream = stream;
+  a.fv = make_view(g, wait);
+  uint8_t* tiles = static_cast<uint8_t*>(scratch);
+  size_t tthr = 0;
+  const int cap = staged_floats(g.n_qthr, &tthr);
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(&tile_rows_kernel), tthr);
+  if (e != cudaSuccess) return e;
+  for (int64_t first = 0; first < rows; first += kScoreBatchRows) {
+    const int64_t n = rows - first < kScoreBatchRows ? rows - first : kScoreBatchRows;
+    const int nblk = static_cast<int>((n + g.block_cands - 1) / g.block_cands);
+    tile_rows_kernel<<<nblk, g.block_cands / 4, tthr, stream>>>(d_feat + first * KS_F_PAD, n, a.fv, tiles, cap);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    a.C = static_cast<int>(n);
+    a.nblk = nblk;
+    a.sl = SliceArgs{};
+    a.sl.n_slices = 1;
+    a.sl.tiles = tiles;
+    a.sl.score_out = d_scores + first;
+    *launches += 2;
+    e = launch_walk(g, a);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
+#ifdef KS_DEBUG_BOUNDS
+int fast_bounds_line() {
+  int v = 0;
+  cudaMemcpyFromSymbol(&v, g_bounds_line, sizeof(int));
+  return v;
+}
+void fast_bounds_clear() {
+  const int z = 0;
+  cudaMemcpyToSymbol(g_bounds_line, &z, sizeof(int));
+}
+#else
+int fast_bounds_line() { return -1; }
+void fast_bounds_clear() {}
+#endif
 
 }  // namespace ks

@@ -47,6 +47,23 @@ struct DevNode {
   uint16_t left;  // left child (right = left + 1)
 };
 
+// Rows and thresholds of one feature column in the quantised form: its sorted distinct
+// thresholds are thr[thr0 .. thr0 + nthr), cut into nslice rows of at most 127, followed by
+// nrank rank rows (categorical columns with partition splits; rank[r][level] = rank of the level
+// in the row's ordering).
+struct FeatQ {
+  uint32_t thr0;
+  uint16_t nthr, row0, nslice, nrank;
+  uint8_t rank[3][4];
+};
+
+// Probe budget of the quantised kernel's chunk waits (0: the default) and the test hook that
+// starves a wait (the barrier is armed for more bytes than its copy brings).
+struct FastWait {
+  int limit;
+  int starve;
+};
+
 struct GbdtModel {
   int n_trees = 0;
   int max_depth = 0;
@@ -57,7 +74,12 @@ struct GbdtModel {
   // quantised fast form (complete trees, chunked level-order layout), see ks_gbdt_fast.cu
   bool fast = false;
   int fast_depth = 0;          // every tree padded to this depth
-  int n_qrows = 0;             // quantised feature rows (a feature, or a 127-threshold slice)
+  int fast_threads = 0;        // tile geometry: threads per CTA (512 or 1,024) ...
+  int block_cands = 0;         // ... and candidates per CTA = bytes per tile row (1,024 or 512)
+  int buf_bytes = 0;           // size of one of the two chunk buffers in shared memory
+  int ctas_per_sm = 1;         // CTAs of this geometry that share an SM
+  int n_qrows = 0;             // quantised feature rows (127-threshold slices and rank rows)
+  int n_qthr = 0, thr_cand0 = 0, thr_prob0 = 0;  // thresholds in all; first of the candidate-only / problem-only features
   int n_pair_rows = 0, n_cand_rows = 0, n_prob_rows = 0;  // rows by what their feature depends on
   int top_levels = 0;          // levels whose nodes also live in h_top
   bool top_compact = false;    // h_top holds one 32-bit word per node instead of a pair
@@ -66,9 +88,8 @@ struct GbdtModel {
   int n_chunks = 0;
   int chunk_bytes = 0;
   uint32_t* d_qnodes = nullptr;  // [n_chunks][chunk_bytes / 4]
-  float* d_qthr = nullptr;       // [n_qrows][256] sorted thresholds padded with +inf
-  uint8_t* d_qrow0 = nullptr;    // [64] first row of each feature column
-  uint8_t* d_qrowcnt = nullptr;  // [64] rows of each feature column
+  float* d_qthr = nullptr;       // [n_qthr] sorted thresholds, feature after feature
+  FeatQ* d_qfeat = nullptr;      // [64] rows and thresholds of each feature column
 };
 
 struct MlpModel {
@@ -114,6 +135,7 @@ struct ks_ctx {
   int* d_status = nullptr;  // bounded waits give up; d_status is its device alias
   int64_t launches = 0;
   int select_one_seq = 0;  // sequence number of the last single-problem call
+  ks::FastWait wait{0, 0};  // probe budget of bounded device waits (0: default) and the starve hook (tests)
   char err[256] = {0};
   // optional timing of the dominant kernel of the last ks_select* call (ks_profile_enable)
   bool profile = false;
@@ -132,10 +154,12 @@ namespace ks {
 
 constexpr int kBlock = 256;            // threads per block of the pair kernels
 constexpr int kSubTilesMax = 8;        // sub-tiles of kBlock rows one block ranks
-constexpr int kFastThreads = 512;      // threads per block of the quantised tree kernel
-constexpr int kFastR = 2;              // candidates per thread there
-constexpr int kFastRows = kFastThreads * kFastR;
 constexpr int kFastMaxDepth = 10;
+constexpr int kFastMaxProbRows = 256;  // rows of problem-only features
+constexpr int kFastMaxCandRec = 256;   // rows of candidate-only features (bytes of a per-call record)
+constexpr int kFastMaxPairRec = 256;   // rows of per-pair features a memoised model may have
+constexpr size_t kMemoTableBytes = size_t(256) << 20;  // per-(problem, class) records held at a time
+constexpr int kFastWaitLimit = 1 << 17;  // probes of a chunk wait (a sleep ends early, ~0.2 us measured): tens of ms
 constexpr int kMlpThreads = 512;        // threads per block of the tensor-core MLP kernel
 constexpr int kMaxSliceBlocks = 1024;  // candidate blocks the slice mode supports
 
@@ -166,7 +190,7 @@ struct FastSlice {
   int* counters;     // [blocks + 1], zero between calls
   int32_t* out_idx;  // single-problem form: [k], device-visible; else null (a merge kernel follows)
   float* out_score;
-  uint8_t* tiles;    // single-problem form: scratch for the prepared tiles [blocks][rows][kFastRows], or null
+  uint8_t* tiles;    // single-problem form: scratch for the prepared tiles [blocks][rows][block_cands], or null
   int* out_seq;      // single-problem form: device-visible word that receives `seq` after the results
   int seq;
 };
@@ -183,8 +207,8 @@ cudaError_t launch_remap_indices(int32_t* d_idx, long long n, const int32_t* d_m
                                  cudaStream_t stream, int64_t* launches);
 
 // Quantised tree path: blocks per problem for `per_problem` rows, and the launch itself.
-void fast_tiling(int P, int64_t per_problem, int* nblk, int* rows_per_cta);
-size_t fast_scratch_bytes(int C);  // per-call table of candidate-only rows
+void fast_tiling(const GbdtModel& g, int P, int64_t per_problem, int* nblk, int* rows_per_cta);
+size_t fast_scratch_bytes(const GbdtModel& g, int C);  // per-call table of candidate-only rows
 size_t fast_memo_bytes(const GbdtModel& g, int P, int C);  // memo of the per-pair rows (0: not used)
 void free_fast_gbdt(GbdtModel& m);
 cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, const ks_problem* d_p,
@@ -192,13 +216,18 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
                                int nblk, int rows_per_cta, const int64_t* seg_off, const int32_t* seg_idx,
                                int k, unsigned long long* partial, void* scratch, int* status,
                                cudaStream_t stream, int64_t* launches, cudaEvent_t ev_begin,
-                               const FastSlice* slice = nullptr, void* memo_mem = nullptr);
+                               const FastSlice* slice = nullptr, void* memo_mem = nullptr,
+                               const FastWait* wait = nullptr);
 int fast_slices(const GbdtModel& g, int64_t blocks);
 // ks_score with a qualifying ensemble: tiles quantised from the feature rows, then the same walk.
 size_t score_fast_scratch_bytes(const GbdtModel& g, int64_t rows);
 cudaError_t launch_score_fast(const ks_gpu_desc& desc, const GbdtModel& g, const float* d_feat, int64_t rows,
                               float* d_scores, void* scratch, int* status, cudaStream_t stream,
-                              int64_t* launches);
+                              int64_t* launches, const FastWait* wait = nullptr);
+// checked build (KS_DEBUG_BOUNDS): source line of the first index found out of range (0: none;
+// -1: not a checked build), and its reset
+int fast_bounds_line();
+void fast_bounds_clear();
 
 // Tensor-core MLP path.
 cudaError_t build_fast_mlp(MlpModel& m, const uint16_t* const* h_w, const float* const* h_b, const float* h_mu,
@@ -243,6 +272,7 @@ cudaError_t launch_select(const ks_gpu_desc& desc, const ks_model& model, const 
                           const int64_t* d_seg_off, const int32_t* d_seg_idx, int64_t pairs, int k,
                           void* d_partial, int32_t* d_topk_idx, float* d_topk_score,
                           cudaStream_t stream, int64_t* launches, int* d_status,
-                          cudaEvent_t ev_begin = nullptr, cudaEvent_t ev_end = nullptr, int* d_counters = nullptr);
+                          cudaEvent_t ev_begin = nullptr, cudaEvent_t ev_end = nullptr, int* d_counters = nullptr,
+                          const FastWait* wait = nullptr);
 
 }  // namespace ks

@@ -740,11 +740,11 @@ size_t select_partial_bytes(const ks_model& model, int P, int C, int64_t pairs, 
   const int64_t per = per_problem_rows(P, C, pairs, segmented);
   if (model.kind == 0 && model.gbdt.fast) {
     int nblk, rows;
-    fast_tiling(P, per, &nblk, &rows);
+    fast_tiling(model.gbdt, P, per, &nblk, &rows);
     const size_t part = (static_cast<size_t>(P) * nblk * k * sizeof(unsigned long long) + 255) / 256 * 256;
     const int S = segmented ? 1 : fast_slices(model.gbdt, static_cast<int64_t>(P) * nblk);
     const size_t planes = S > 1 ? (sizeof(float) * S * static_cast<size_t>(pairs) + 255) / 256 * 256 : 0;
-    return part + (fast_scratch_bytes(C) + 255) / 256 * 256 + planes + (S > 1 ? 0 : fast_memo_bytes(model.gbdt, P, C));
+    return part + (fast_scratch_bytes(model.gbdt, C) + 255) / 256 * 256 + planes + (S > 1 ? 0 : fast_memo_bytes(model.gbdt, P, C));
   }
   if (model.kind == 1 && model.mlp.tc) {
     const int nblk = mlp_tc_blocks_per_problem(P, per);
@@ -765,12 +765,12 @@ cudaError_t launch_select(const ks_gpu_desc& desc, const ks_model& model, const 
                           const int64_t* d_seg_off, const int32_t* d_seg_idx, int64_t pairs, int k,
                           void* d_partial, int32_t* d_topk_idx, float* d_topk_score,
                           cudaStream_t stream, int64_t* launches, int* d_status, cudaEvent_t ev_begin,
-                          cudaEvent_t ev_end, int* d_counters) {
+                          cudaEvent_t ev_end, int* d_counters, const FastWait* wait) {
   if (P == 0) return cudaSuccess;
   const int64_t per = per_problem_rows(P, C, pairs, d_seg_off != nullptr);
   if (model.kind == 0 && model.gbdt.fast) {
     int nblk, rows;
-    fast_tiling(P, per, &nblk, &rows);
+    fast_tiling(model.gbdt, P, per, &nblk, &rows);
     unsigned long long* part = static_cast<unsigned long long*>(d_partial);
     const size_t part_bytes = (static_cast<size_t>(P) * nblk * k * sizeof(unsigned long long) + 255) / 256 * 256;
     // an under-filled machine: split the trees over several CTAs per block (dense form only,
@@ -780,17 +780,17 @@ cudaError_t launch_select(const ks_gpu_desc& desc, const ks_model& model, const 
     if (sl.n_slices > 1) {
       sl.pairs = pairs;
       sl.scores = reinterpret_cast<float*>(static_cast<char*>(d_partial) + part_bytes +
-                                           (fast_scratch_bytes(C) + 255) / 256 * 256);
+                                           (fast_scratch_bytes(model.gbdt, C) + 255) / 256 * 256);
       sl.counters = d_counters;
     }
     // the memo of the per-pair rows sits behind the per-call table (batches of whole-ensemble CTAs only)
     const int sized_slices = d_seg_off ? 1 : fast_slices(model.gbdt, static_cast<int64_t>(P) * nblk);  // as sized
     void* memo_mem = (sized_slices > 1 || p_by_value || fast_memo_bytes(model.gbdt, P, C) == 0)
                          ? nullptr
-                         : static_cast<char*>(d_partial) + part_bytes + (fast_scratch_bytes(C) + 255) / 256 * 256;
+                         : static_cast<char*>(d_partial) + part_bytes + (fast_scratch_bytes(model.gbdt, C) + 255) / 256 * 256;
     cudaError_t e = launch_select_fast(desc, model.gbdt, d_p, p_by_value, P, d_c, C, nblk, rows, d_seg_off,
                                        d_seg_idx, k, part, static_cast<char*>(d_partial) + part_bytes, d_status,
-                                       stream, launches, ev_begin, sl.n_slices > 1 ? &sl : nullptr, memo_mem);
+                                       stream, launches, ev_begin, sl.n_slices > 1 ? &sl : nullptr, memo_mem, wait);
     if (e != cudaSuccess) return e;
     if (ev_end) cudaEventRecord(ev_end, stream);
     topk_merge_kernel<<<(P * 32 + kBlock - 1) / kBlock, kBlock, 0, stream>>>(part, P, nblk * k, k, d_topk_idx,

@@ -531,6 +531,82 @@ def test_select_other_model_shapes(ks, ctx, case):
     assert np.array_equal(hi_.numpy(), idx[2])
 
 
+@pytest.mark.parametrize("case", ["cfg1_slots128", "cfg1_hist256", "cfg1_pernode", "cfg2_pernode", "continuous"])
+def test_select_tile_geometries(ks, ctx, case):
+    """The quantised kernel's tile geometries, picked by the number of rows: the slot-table
+    ensemble (<= 72 rows: two CTAs of 512 threads x 1,024 candidates per SM), the 256-bin and the
+    quantile-per-node ensembles of config 1 (<= 149 rows: two CTAs of 512 threads x 512
+    candidates), the quantile-per-node ensemble of config 2 (<= 367 rows: one CTA of 1,024 threads x
+    512 candidates), and an ensemble with a continuous threshold at every node of 3,000 trees (more
+    rows than any geometry holds: the general kernel). Each: a batch (ks_select), the single-problem call (tree slices
+    over prepared tiles), the scoring call on given feature rows, and a batch of 33 problems or
+    more that takes the per-(problem, class) memo."""
+    if case == "continuous":
+        prob, cand, _, _ = wl.make_inputs(1, P=3, C=2500)
+        x = oracle.featurize(prob, cand, DESC)
+        lo, hi = x.min(axis=0), x.max(axis=0)
+        off, nodes = random_trees(5, 3000, 5, 0.95, lambda f, rng: np.float32(lo[f] + (hi[f] - lo[f]) * rng.random()))
+        w = wl.Workload(case, DESC, prob, cand, 10, gbdt=(off, nodes, 0.0))
+        want = "select_generic_kernel"
+    elif case == "cfg2_pernode":
+        w = wl.make_workload(2, P=6, seg=2500, law="pernode")
+        want = "threads=1024 block=512"
+    else:
+        law = case.split("_")[1]
+        w = wl.make_workload(1, P=5, C=3000, law=law)
+        want = "threads=512 block=1024" if law == "slots128" else "threads=512 block=512"
+    model = ctx.model_create_gbdt(*w.gbdt)
+    assert want in model.describe(), model.describe()
+    idx, sc = run_select(ks, ctx, w, model)
+    check_select(w, idx, sc, TOL_GBDT)
+    if case == "continuous":
+        return
+    # single-problem call against the dense pool, and the scoring call on given rows
+    C = min(len(w.candidates), 2600)
+    cand = w.candidates[:C]
+    d_c = dev(ks, cand)
+    for i in (0, len(w.problems) - 1):
+        hi_, hs_ = ctx.select_one(w.problems[i:i + 1], d_c, C, model, 10)
+        _, _, allsc = oracle.select(w.problems[i:i + 1], cand, DESC, 10, gbdt=w.gbdt, want_scores=True)
+        ok, msg = topk_accept(hi_.numpy(), hs_.numpy(), allsc, np.arange(C, dtype=np.int32), 10, TOL_GBDT)
+        assert ok, msg
+    x = oracle.featurize(w.problems[:2], cand, DESC)
+    rs = oracle.score_gbdt(x, *w.gbdt)
+    s = ctx.score(dev(ks, x), model).cpu().numpy()
+    assert np.all(np.abs(s - rs) <= TOL_GBDT * np.maximum(1, np.abs(rs)))
+    # memo path: 40 problems, few candidates
+    cfg = 2 if case.startswith("cfg2") else 1
+    wm = wl.make_workload(cfg, P=40, C=None if cfg == 2 else 700, seg=600 if cfg == 2 else None, law=w.meta["law"])
+    idx, sc = run_select(ks, ctx, wm, model)
+    check_select(wm, idx, sc, TOL_GBDT, sample=range(0, 40, 3))
+
+
+@pytest.mark.parametrize("geometry", ["1024,1024,32", "1024,1024,16", "1024,512,32", "512,512,16"])
+def test_select_forced_tile_geometry(ks, ctx, geometry, monkeypatch):
+    """Every tile geometry on the same ensemble (config 1, a quantile per node, 143 rows), forced
+    through KS_FAST_GEOMETRY = threads, candidates per CTA, chunk-buffer KiB."""
+    monkeypatch.setenv("KS_FAST_GEOMETRY", geometry)
+    w = wl.make_workload(1, P=4, C=2700, law="pernode")
+    model = ctx.model_create_gbdt(*w.gbdt)
+    t, c, _ = geometry.split(",")
+    assert f"threads={t} block={c}" in model.describe(), model.describe()
+    idx, sc = run_select(ks, ctx, w, model)
+    check_select(w, idx, sc, TOL_GBDT)
+    hi_, hs_ = ctx.select_one(w.problems[1:2], dev(ks, w.candidates), len(w.candidates), model, 10)
+    assert np.array_equal(hi_.numpy(), idx[1])
+
+
+def test_select_memo_table_in_batches(ks, ctx):
+    """The per-(problem, class) table holds 256 MiB of records; a batch of more problems than that
+    is served in several launches that reuse it (here 80-byte records: 409 problems at a time)."""
+    w = wl.make_workload(1, P=900, C=300, law="pernode")
+    model = ctx.model_create_gbdt(*w.gbdt)
+    n0 = ctx.launch_count()
+    idx, sc = run_select(ks, ctx, w, model)
+    assert ctx.launch_count() - n0 == 2 + 1 + 3 * 2 + 1  # mask, candidate rows, compaction, 3 x (table, walk), merge
+    check_select(w, idx, sc, TOL_GBDT, sample=list(range(0, 900, 37)) + [408, 409, 817, 818, 899])
+
+
 def test_select_pair_row_memo_paths(ks, ctx):
     """Batches of 32 problems or more copy the per-pair tile rows from a per-(problem, class)
     table, a class being (T_M, T_N, T_K, S, c_M, c_N, resident blocks). Cases: mixed element
