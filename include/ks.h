@@ -18,6 +18,13 @@
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream). Batch
  *     calls only enqueue work on that stream; they do not synchronise.
  *   - A context is bound to one device and is not thread-safe: use one per host thread.
+ *   - Every batch call of a context (ks_featurize, ks_score, ks_select, ks_valid_catalogue, ...)
+ *     uses the context's one device workspace, which is grown on demand: calls on one context
+ *     must go on one stream, or be serialised by the caller.
+ *   - A kernel whose bounded device-side wait gives up sets the context's status word and the
+ *     call's results are void. ks_select_one and ks_select_host report it themselves
+ *     (KS_ERR_TIMEOUT); after an asynchronous call, ks_device_status reports and clears it, and
+ *     must be called before the context's next call once a failure is suspected.
  *   - All structs are plain little-endian PODs with exactly the fields shown.
  */
 #ifndef KS_H_
@@ -171,6 +178,8 @@ ks_status ks_model_create_mlp(ks_ctx* ctx, int n_layers, const int* h_widths,
  * score is a function of (p, c), not of the feature row. */
 ks_status ks_model_create_static(ks_ctx* ctx, ks_model** out_model);
 
+/* Frees the model's device buffers. A model may be destroyed before or after its context, but
+ * must not be used in a call once the context is gone. */
 ks_status ks_model_destroy(ks_model* model);
 
 /* ---- search space and validity (the steps in front of the path) --------------------------- */
@@ -184,9 +193,14 @@ ks_status ks_model_destroy(ks_model* model);
  * mainloop schedule that the schedule names imply but the paper's table does not list
  * (TMA-Cooperative epilogue <=> cooperative mainloop; TMA epilogue => non-cooperative mainloop).
  * KS_VALID_WASTEFUL adds the rule of section "Validity Constraints" that drops candidates with
- * T_N > 2M or T_N > 2N. */
+ * T_N > 2M or T_N > 2N. KS_VALID_PRINTED_CAPACITY applies the capacity rule exactly as Table
+ * "Static validity constraints" prints it, mainloop + epilogue + reserve <= capacity for every
+ * schedule; without it the schedule-specific footprint of feature column 49 is compared
+ * (warp-specialised mainloops reuse their buffers for the epilogue), the reading that
+ * reproduces the paper's between-layout count differences. */
 #define KS_VALID_COUPLED 1u
 #define KS_VALID_WASTEFUL 2u
+#define KS_VALID_PRINTED_CAPACITY 4u
 
 /* Writes the candidates with linear ids first .. first+count-1 of the search space to
  * d_out[0..count) (device, 16-byte aligned, caller-owned). The id is a mixed-radix number whose
@@ -309,7 +323,9 @@ ks_status ks_select_host(ks_ctx* ctx, const ks_problem* h_p, int P, const ks_can
  *     KS_STATIC_MAX_KEYS is always sufficient. Larger requests return KS_ERR_UNSUPPORTED and
  *     launch nothing.
  *   - The first call on a device looks up the array's device address (cudaGetSymbolAddress);
- *     make that first call outside any stream capture.
+ *     make that first call outside any stream capture. With CUDA's lazy module loading that
+ *     first call is also what places the kernels' code and the 4 MiB array on the device: a
+ *     caller whose own pool takes all remaining memory must make it BEFORE the pool does.
  *   - All calls share the one array, which keeps the previous call's contents. The kernels
  *     write every entry they later read, so nothing has to be cleared, but two calls whose
  *     kernels overlap on the GPU (different streams, or different host threads) race on it:

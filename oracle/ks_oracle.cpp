@@ -253,8 +253,10 @@ void enumerate_one(int64_t id, OCandidate* c) {
 
 // Shared-memory footprint of one CTA as the feature map counts it (section "Resource Pressure
 // and Occupancy", same reading as columns 47-49): warp-specialised mainloops may reuse the
-// mainloop buffers for the epilogue, ping-pong and cooperative ones hold both.
-int64_t smem_total(const OProblem& p, const OCandidate& c, const OGpuDesc& h) {
+// mainloop buffers for the epilogue, ping-pong and cooperative ones hold both. With `printed` the
+// sum as Table "Static validity constraints" prints it: mainloop + epilogue + reserve, whatever
+// the schedule.
+int64_t smem_total(const OProblem& p, const OCandidate& c, const OGpuDesc& h, bool printed) {
   static const int64_t kBytes[4] = {2, 2, 1, 4};
   const int64_t bA = kBytes[p.dtype_ab & 3], bD = kBytes[p.dtype_d & 3];
   const int64_t TM = c.tile_m, TN = c.tile_n, TK = c.tile_k, S = c.stages;
@@ -263,20 +265,21 @@ int64_t smem_total(const OProblem& p, const OCandidate& c, const OGpuDesc& h) {
   const int64_t E = (ks == 2) ? 128 : 64;
   const int64_t B_epi =
       (c.epi_sched == 0) ? 0 : 2 * std::min<int64_t>(TM, E) * std::min<int64_t>(TN, 32) * bD;
+  if (printed) return smem_main + B_epi + h.smem_reserved;
   return ((ks == 0 || ks == 3) ? std::max(smem_main, B_epi) : smem_main + B_epi) + h.smem_reserved;
 }
 
 // Table "Static validity constraints", rule by rule. flags bit 0 adds the two couplings between
 // epilogue and mainloop schedule that CUTLASS's naming implies (TMA-Cooperative epilogue <=>
 // cooperative mainloop; TMA epilogue => non-cooperative mainloop); bit 1 adds the section's
-// "wasteful candidate" rule T_N > 2M or T_N > 2N.
+// "wasteful candidate" rule T_N > 2M or T_N > 2N; bit 2 takes the capacity rule as printed.
 bool is_valid(const OProblem& p, const OCandidate& c, const OGpuDesc& h, unsigned flags) {
   const bool coop = c.kernel_sched == 2;
   const bool a_col_major = p.layout == 2 || p.layout == 3;  // NN, NT
   const bool b_row_major = p.layout == 1 || p.layout == 3;  // TT, NT
   if (c.tile_sched == 1 && !coop) return false;             // Stream-K => cooperative mainloop
   if (coop && c.tile_m % 128 != 0) return false;            // cooperative => T_M = 0 mod 128
-  if (smem_total(p, c, h) > static_cast<int64_t>(h.smem_per_cta_max)) return false;  // capacity
+  if (smem_total(p, c, h, (flags & 4u) != 0) > static_cast<int64_t>(h.smem_per_cta_max)) return false;  // capacity
   if (a_col_major && c.tile_k > 256 * c.cluster_n) return false;  // A column-major: T_K <= 256 C_N
   if (b_row_major && c.tile_k > 256 * c.cluster_m) return false;  // B row-major: T_K <= 256 C_M
   if (flags & 1u) {

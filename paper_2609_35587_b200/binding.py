@@ -18,7 +18,7 @@ LIB_PATH = os.environ.get("KS_LIBRARY") or os.path.join(_HERE, "libks.so")
 
 KS_F, KS_F_PAD, KS_MAX_K, KS_MAX_DEPTH = 63, 64, 32, 15
 KS_CATALOGUE_SIZE = 534600
-KS_VALID_COUPLED, KS_VALID_WASTEFUL = 1, 2
+KS_VALID_COUPLED, KS_VALID_WASTEFUL, KS_VALID_PRINTED_CAPACITY = 1, 2, 4
 KS_OK, KS_ERR_INVALID_ARG, KS_ERR_UNSUPPORTED, KS_ERR_CUDA, KS_ERR_TIMEOUT, KS_ERR_OOM = range(6)
 
 EXPORTS = ("ks_create", "ks_destroy", "ks_last_cuda_error", "ks_model_create_gbdt",

@@ -63,6 +63,16 @@ ks_status ensure_workspace(ks_ctx* ctx, size_t bytes) {
 }  // namespace
 
 namespace ks {
+bool valid_desc(const ks_gpu_desc& d) {
+  if (!d.num_sms || !d.smem_per_sm || !d.smem_per_cta_max || !d.regs_per_sm || !d.max_threads_per_sm ||
+      !d.max_ctas_per_sm || !d.l2_bytes || !d.tma_bytes_per_us || d.reserved0)
+    return false;
+  if (d.max_threads_per_sm < 384) return false;
+  for (int i = 0; i < 4; ++i)
+    if (!d.tc_flops_per_us_per_sm[i]) return false;
+  return true;
+}
+
 cudaError_t ensure_dynamic_smem(const void* kernel, size_t bytes) {
   struct Entry {
     const void* kernel;
@@ -113,16 +123,6 @@ cudaError_t upload(T** dst, const T* src, size_t n) {
   return cudaMemcpy(*dst, src, n * sizeof(T), cudaMemcpyHostToDevice);
 }
 
-bool valid_desc(const ks_gpu_desc& d) {
-  if (!d.num_sms || !d.smem_per_sm || !d.smem_per_cta_max || !d.regs_per_sm || !d.max_threads_per_sm ||
-      !d.max_ctas_per_sm || !d.l2_bytes || !d.tma_bytes_per_us || d.reserved0)
-    return false;
-  if (d.max_threads_per_sm < 384) return false;
-  for (int i = 0; i < 4; ++i)
-    if (!d.tc_flops_per_us_per_sm[i]) return false;
-  return true;
-}
-
 // Checks one tree; returns its depth or -1.
 int validate_tree(const ks_node_host* t, int64_t n) {
   if (n < 1 || n > 65535) return -1;
@@ -158,7 +158,7 @@ int validate_tree(const ks_node_host* t, int64_t n) {
 
 void free_model(ks_model* m) {
   if (!m) return;
-  DeviceGuard g(m->ctx->device);
+  DeviceGuard g(m->device);  // not m->ctx: a model may be destroyed after its context
   cudaFree(m->gbdt.d_nodes);
   cudaFree(m->gbdt.d_roots);
   cudaFree(m->gbdt.d_qnodes);
@@ -213,7 +213,7 @@ const char* ks_feature_name(int index) {
 ks_status ks_create(ks_ctx** out_ctx, int cuda_device, const ks_gpu_desc* desc) {
   if (!out_ctx) return KS_ERR_INVALID_ARG;
   *out_ctx = nullptr;
-  if (!desc || !valid_desc(*desc)) return KS_ERR_INVALID_ARG;
+  if (!desc || !ks::valid_desc(*desc)) return KS_ERR_INVALID_ARG;
   int n_dev = 0;
   if (cudaGetDeviceCount(&n_dev) != cudaSuccess) {
     cudaGetLastError();
@@ -384,6 +384,7 @@ ks_status ks_model_create_gbdt(ks_ctx* ctx, int n_trees, const int64_t* h_tree_o
   ks_model* m = new (std::nothrow) ks_model();
   if (!m) return KS_ERR_OOM;
   m->ctx = ctx;
+  m->device = ctx->device;
   m->kind = 0;
   m->gbdt.n_trees = n_trees;
   m->gbdt.max_depth = max_depth;
@@ -424,6 +425,7 @@ ks_status ks_model_create_mlp(ks_ctx* ctx, int n_layers, const int* h_widths,
   ks_model* m = new (std::nothrow) ks_model();
   if (!m) return KS_ERR_OOM;
   m->ctx = ctx;
+  m->device = ctx->device;
   m->kind = 1;
   m->mlp.n_layers = n_layers;
   m->mlp.max_width = max_width;
@@ -454,6 +456,7 @@ ks_status ks_model_create_static(ks_ctx* ctx, ks_model** out_model) {
   ks_model* m = new (std::nothrow) ks_model();
   if (!m) return KS_ERR_OOM;
   m->ctx = ctx;
+  m->device = ctx->device;
   m->kind = 2;
   *out_model = m;
   return KS_OK;
@@ -478,7 +481,7 @@ ks_status ks_valid_catalogue(ks_ctx* ctx, const ks_problem* problem, unsigned fl
                              const ks_candidate* d_candidates, int C, ks_candidate* d_out,
                              int32_t* d_out_index, int32_t* d_count, int32_t* h_count, void* stream) {
   if (!ctx || !problem || !d_count || C < 0) return KS_ERR_INVALID_ARG;
-  if (flags & ~(KS_VALID_COUPLED | KS_VALID_WASTEFUL)) return KS_ERR_INVALID_ARG;
+  if (flags & ~(KS_VALID_COUPLED | KS_VALID_WASTEFUL | KS_VALID_PRINTED_CAPACITY)) return KS_ERR_INVALID_ARG;
   if (problem->layout > 3 || problem->dtype_ab > 3 || problem->dtype_d > 3) return KS_ERR_INVALID_ARG;
   if (!d_candidates && C > KS_CATALOGUE_SIZE) return KS_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(d_candidates) & 15u) || (reinterpret_cast<uintptr_t>(d_out) & 15u))
@@ -542,7 +545,7 @@ ks_status ks_score(ks_ctx* ctx, const float* d_features, int64_t rows, const ks_
   }
   if (model->kind == 1 && ks::score_mlp_tc_ok(model->mlp)) {
     cudaError_t e = ks::launch_score_mlp_tc(ctx->desc, model->mlp, d_features, rows, d_scores, ctx->d_status,
-                                            static_cast<cudaStream_t>(stream), &ctx->launches);
+                                            static_cast<cudaStream_t>(stream), &ctx->launches, &ctx->wait);
     return e == cudaSuccess ? KS_OK : cuda_fail(ctx, e, "ks_score");
   }
   cudaError_t e =

@@ -67,7 +67,7 @@ __device__ __forceinline__ bool is_valid(const ValidArgs& a, const ks_candidate&
   bool ok = !(c.tile_sched == 1 && !coop);                       // Stream-K => cooperative mainloop
   ok = ok && !(coop && (c.tile_m % 128u) != 0);                  // cooperative => T_M = 0 mod 128
   const SmemTerms sm = smem_terms(a.bA, a.bD, c, h);
-  ok = ok && sm.B_smem <= static_cast<long long>(h.smem_per_cta_max);  // capacity per CTA
+  ok = ok && ((a.flags & KS_VALID_PRINTED_CAPACITY) ? sm.both : sm.B_smem) <= static_cast<long long>(h.smem_per_cta_max);  // capacity per CTA
   ok = ok && !(a.a_col_major && c.tile_k > 256u * c.cluster_n);  // A column-major: T_K <= 256 C_N
   ok = ok && !(a.b_row_major && c.tile_k > 256u * c.cluster_m);  // B row-major: T_K <= 256 C_M
   if (a.flags & KS_VALID_COUPLED) {

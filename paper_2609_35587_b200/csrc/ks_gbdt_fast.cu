@@ -840,7 +840,8 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
     block_topk<5>(keys, k, s_warp, s_list);
   }
   if (sl.score_out) return;
-  if (tid < k) partial[(static_cast<size_t>(prob) * nblk + chunk) * k + tid] = s_list[tid];
+  if (tid < k)
+    partial[KS_IDX((static_cast<size_t>(prob) * nblk + chunk) * k + tid, static_cast<size_t>(P) * nblk * k)] = s_list[tid];
   if (S > 1 && sl.out_idx) {
     // single-problem form: the last block to finish merges the per-block lists (one warp)
     __threadfence();

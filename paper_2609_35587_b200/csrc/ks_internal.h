@@ -29,6 +29,8 @@ struct alignas(16) MlpTcParams {
   uint16_t ind0[8], ind1[8];           // bf16 of an indicator's standardised value when 0 / 1 (kernel sched 0..3, epilogue sched 0..2)
   float p_scale[18], p_shift[18];      // standardisation of the folded inputs
   const float* w1_prob;                // device, [18][256]: first-layer weights of the folded inputs
+  int wait_limit;                      // tries a barrier wait may take (set at every launch)
+  int starve;                          // test hook: the weight image is never copied, so the first wait runs out
 };
 
 // Linear scorer (one weight layer) in a form the fused ridge kernel consumes: per feature column
@@ -145,6 +147,7 @@ struct ks_ctx {
 
 struct ks_model {
   ks_ctx* ctx = nullptr;
+  int device = 0;  // the context's device (kept here: the model may outlive the context)
   int kind = 0;  // 0 tree ensemble, 1 MLP, 2 static sampling score
   ks::GbdtModel gbdt;
   ks::MlpModel mlp;
@@ -177,6 +180,8 @@ inline int categorical_levels(int col) {
 // cudaFuncSetAttribute(MaxDynamicSharedMemorySize) costs a driver call; remembers, per kernel and
 // device, the largest size already granted (ks_api.cu).
 cudaError_t ensure_dynamic_smem(const void* kernel, size_t bytes);
+// A descriptor every entry point accepts: no zero capacity or rate, reserved word zero.
+bool valid_desc(const ks_gpu_desc& d);
 
 // Builds the quantised fast form of a validated ensemble when it qualifies (m.fast).
 cudaError_t build_fast_gbdt(GbdtModel& m, int n_trees, const int64_t* h_tree_offsets,
@@ -243,12 +248,14 @@ size_t mlp_tc_scratch_bytes(int C);
 // ks_score on the tensor-core kernel (ordinal input form only): the given rows are the input.
 bool score_mlp_tc_ok(const MlpModel& m);
 cudaError_t launch_score_mlp_tc(const ks_gpu_desc& desc, const MlpModel& m, const float* d_feat, int64_t rows,
-                                float* d_scores, int* status, cudaStream_t stream, int64_t* launches);
+                                float* d_scores, int* status, cudaStream_t stream, int64_t* launches,
+                                const FastWait* wait = nullptr);
+constexpr int kMlpWaitLimit = 1 << 14;  // tries of a barrier wait of the tensor-core kernel (each blocks for up to a few microseconds): tens of ms
 cudaError_t launch_select_mlp_tc(const ks_gpu_desc& desc, const MlpModel& m, const ks_problem* d_p,
                                  const ks_problem* p_by_value, int P, const ks_candidate* d_c, int C, int nblk,
                                  const int64_t* seg_off, const int32_t* seg_idx, int k,
                                  unsigned long long* partial, void* scratch, int* status, cudaStream_t stream,
-                                 int64_t* launches, cudaEvent_t ev_begin);
+                                 int64_t* launches, cudaEvent_t ev_begin, const FastWait* wait = nullptr);
 
 // ---- launchers (each enqueues on `stream`, returns the cudaError of the launch) -----------
 cudaError_t launch_featurize(const ks_gpu_desc& desc, const ks_problem* d_p, int P,

@@ -804,7 +804,7 @@ cudaError_t launch_select(const ks_gpu_desc& desc, const ks_model& model, const 
     const size_t part_bytes = (static_cast<size_t>(P) * nblk * k * sizeof(unsigned long long) + 255) / 256 * 256;
     cudaError_t e = launch_select_mlp_tc(desc, model.mlp, d_p, p_by_value, P, d_c, C, nblk, d_seg_off, d_seg_idx, k,
                                          part, static_cast<char*>(d_partial) + part_bytes, d_status, stream,
-                                         launches, ev_begin);
+                                         launches, ev_begin, wait);
     if (e != cudaSuccess) return e;
     if (ev_end) cudaEventRecord(ev_end, stream);
     topk_merge_kernel<<<(P * 32 + kBlock - 1) / kBlock, kBlock, 0, stream>>>(part, P, nblk * k, k, d_topk_idx,

@@ -50,7 +50,6 @@ constexpr int kOffA = kW1Bytes + kW2Bytes;
 constexpr int kSmemBytes = kOffA + kABytes;           // 224 KB
 constexpr int kPlaneA = kTileRows * 16;               // bytes per 8-column plane of an A operand
 constexpr int kPlaneB = kH * 16;                      // ... of a B operand
-constexpr int kSpinLimit = 1 << 22;
 constexpr int kCandRec = 64;                          // bytes per (combination, candidate) record
 constexpr int kCombos = 16;
 constexpr int kNC = 29, kNPair = 21;                  // candidate-only and per-pair columns (13 are problem-only)
@@ -443,8 +442,9 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
     // both weight matrices, resident for the CTA's lifetime
     fence_async_proxy();
     mbar_expect_tx(bar_w, kW1Bytes + kW2Bytes);
-    for (int off = 0; off < kW1Bytes + kW2Bytes; off += 32768)
-      bulk_copy_g2s(sbase + kOffW1 + off, w_image + off, 32768, bar_w);
+    if (!prm.starve)  // test hook: without the copies the wait on this barrier runs out
+      for (int off = 0; off < kW1Bytes + kW2Bytes; off += 32768)
+        bulk_copy_g2s(sbase + kOffW1 + off, w_image + off, 32768, bar_w);
   }
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(512)
@@ -469,7 +469,7 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
   // Bounded wait. After the first one that runs out, every later wait of the CTA gives up after a
   // few probes, and the CTAs that start later leave at once (device flag).
   auto wait_ok = [&](uint32_t bar, uint32_t parity) {
-    for (int i = 0; i < kSpinLimit; ++i) {
+    for (int i = 0; i < prm.wait_limit; ++i) {
       if (mbar_try_wait(bar, parity)) return true;
       if ((i & 255) == 255 && *reinterpret_cast<volatile int*>(&s_fail)) break;
     }
@@ -487,7 +487,8 @@ select_mlp_tc_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_prob
   // The tile pipeline runs through all of them without draining in between.
   const int64_t problem_tiles = (len + kTileRows - 1) / kTileRows;
   const int64_t tile_first = problem_tiles * chunk / nblk;
-  const int total_tiles = static_cast<int>(problem_tiles * (chunk + 1) / nblk - tile_first);
+  // a CTA whose weights never arrived runs no tile at all: nothing is issued to the tensor cores
+  const int total_tiles = failed ? 0 : static_cast<int>(problem_tiles * (chunk + 1) / nblk - tile_first);
   auto tile_row0 = [&](int tile) { return (tile_first + tile) * kTileRows; };
   unsigned long long top = 0ull;  // second-epilogue warps: lane j holds the warp's j-th best key
 
@@ -832,7 +833,9 @@ cudaError_t launch_select_mlp_tc(const ks_gpu_desc& desc, const MlpModel& m, con
                                  const ks_problem* p_by_value, int P, const ks_candidate* d_c, int C, int nblk,
                                  const int64_t* seg_off, const int32_t* seg_idx, int k,
                                  unsigned long long* partial, void* scratch, int* status, cudaStream_t stream,
-                                 int64_t* launches, cudaEvent_t ev_begin) {
+                                 int64_t* launches, cudaEvent_t ev_begin, const FastWait* wait) {
+  m.h_tc_params->wait_limit = wait && wait->limit > 0 ? wait->limit : kMlpWaitLimit;
+  m.h_tc_params->starve = wait ? wait->starve : 0;
   ks_problem pv{};
   if (p_by_value) pv = *p_by_value;
   const int uv = p_by_value != nullptr;
@@ -880,7 +883,10 @@ cudaError_t launch_select_mlp_tc(const ks_gpu_desc& desc, const MlpModel& m, con
 bool score_mlp_tc_ok(const MlpModel& m) { return m.tc && m.h_tc_params && !m.h_tc_params->onehot; }
 
 cudaError_t launch_score_mlp_tc(const ks_gpu_desc& desc, const MlpModel& m, const float* d_feat, int64_t rows,
-                                float* d_scores, int* status, cudaStream_t stream, int64_t* launches) {
+                                float* d_scores, int* status, cudaStream_t stream, int64_t* launches,
+                                const FastWait* wait) {
+  m.h_tc_params->wait_limit = wait && wait->limit > 0 ? wait->limit : kMlpWaitLimit;
+  m.h_tc_params->starve = wait ? wait->starve : 0;
   cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(&select_mlp_tc_kernel<2>), kSmemBytes);
   if (e != cudaSuccess) return e;
   const uint8_t* image = reinterpret_cast<const uint8_t*>(m.d_tc_image);

@@ -53,10 +53,13 @@ extern "C" ks_status ks_select_trees_static(int cuda_device, const ks_gpu_desc* 
   static_assert(sizeof(ks_node_dev) == sizeof(ks::DevNode), "device node layout");
   if (!desc || P < 0 || C < 0 || n_trees < 0 || k < 1 || k > KS_MAX_K) return KS_ERR_INVALID_ARG;
   if (cuda_device < 0 || cuda_device >= kMaxDevices) return KS_ERR_INVALID_ARG;
-  if (!desc->num_sms || !desc->smem_per_sm || !desc->regs_per_sm || desc->max_threads_per_sm < 384 ||
-      !desc->max_ctas_per_sm || !desc->l2_bytes || !desc->tma_bytes_per_us || !desc->tc_flops_per_us_per_sm[0] ||
-      !desc->tc_flops_per_us_per_sm[1] || !desc->tc_flops_per_us_per_sm[2] || !desc->tc_flops_per_us_per_sm[3])
-    return KS_ERR_INVALID_ARG;
+  if (!ks::valid_desc(*desc)) return KS_ERR_INVALID_ARG;
+  int n_dev = 0;
+  if (cudaGetDeviceCount(&n_dev) != cudaSuccess) {
+    cudaGetLastError();
+    return KS_ERR_CUDA;
+  }
+  if (cuda_device >= n_dev) return KS_ERR_INVALID_ARG;
   if (P == 0) return KS_OK;
   if (!d_p || !d_topk_idx || !d_topk_score || (C > 0 && !d_c) || (n_trees > 0 && (!d_nodes || !d_tree_offsets)))
     return KS_ERR_INVALID_ARG;

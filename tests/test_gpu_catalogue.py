@@ -48,7 +48,7 @@ def test_enumerate_whole_space_and_windows(ks, ctx):
         assert ei.value.status == ks.KS_ERR_INVALID_ARG
 
 
-@pytest.mark.parametrize("flags", [0, 1, 2, 3])
+@pytest.mark.parametrize("flags", [0, 1, 2, 3, 5, 7])
 def test_valid_catalogue_of_the_search_space(ks, ctx, flags):
     cases = [problem(4096, 4096, 4096, lay, 1, 1) for lay in range(4)]
     cases += [problem(64, 64, 64, 0, 1, 1), problem(32, 128, 4096, 3, 1, 1),

@@ -1,12 +1,18 @@
-"""Full-size parity: the benchmark's workloads in the launch configuration bench.py times,
-checked on sampled problems the oracle can rank one by one, plus properties that hold for
-every problem."""
+"""Full-size parity: the benchmark's workloads in the launch configuration bench.py times. EVERY
+problem's top-k list is compared with the oracle's: the oracle's lists come from
+tests/golden/full_size.npz (written by tests/golden/make_full_size.py, which calls only the
+oracle) when the stored checksum matches the generated inputs, and are recomputed otherwise
+(minutes of host time per configuration). A row that differs from the oracle's row is not a
+failure by itself (two candidates whose oracle scores lie within the tolerance may swap): it is
+re-examined against the oracle's scores of the problem's whole candidate set with the
+acceptance rule of tests/helpers.topk_accept, and such rows must stay rare."""
 import numpy as np
 import pytest
 import torch
 
 import oracle
 from paper_2609_35587_b200 import workloads as wl
+from tests.golden import make_full_size as golden
 from tests.helpers import topk_accept
 
 pytestmark = pytest.mark.gpu
@@ -53,6 +59,34 @@ def check_properties(w, idx, sc):
             assert np.all(np.isin(idx[i], seg))
 
 
+def oracle_rows(name, w):
+    """The oracle's [P, k] lists of case `name`: stored, or computed now."""
+    store = golden.load()
+    if f"{name}_crc" in store and int(store[f"{name}_crc"][0]) == golden.checksum(w):
+        return store[f"{name}_idx"], store[f"{name}_score"]
+    return golden.oracle_topk(w)
+
+
+def check_every_problem(name, w, idx, sc, tol, exact_indices=True):
+    """All P rows against the oracle's rows. A row with the oracle's indices and scores within
+    the tolerance passes at once. Every other row must at least carry, rank by rank, the
+    oracle's j-th best score within the tolerance; it is then re-examined with the full
+    acceptance rule against the oracle's scores of the whole candidate set - all such rows
+    where indices are expected to be exact (tree ensembles: they must be rare), a sample of 48
+    where near-ties are the norm (the bf16 ranker)."""
+    ridx, rsc = oracle_rows(name, w)
+    assert ridx.shape == idx.shape
+    close = np.abs(sc - rsc) <= tol * np.maximum(1.0, np.abs(rsc))
+    assert close.all(), f"rank-wise scores differ from the oracle's in {np.count_nonzero(~close.all(axis=1))} rows"
+    redo = np.nonzero(~np.all(idx == ridx, axis=1))[0]
+    if exact_indices:
+        assert len(redo) <= max(8, len(idx) // 50), f"{len(redo)} of {len(idx)} rows differ from the oracle's rows"
+    elif len(redo) > 48:
+        redo = redo[wl.randint(11, 3, np.arange(48), len(redo))]
+    check_sampled(w, idx, sc, redo.tolist(), tol)
+    return len(redo)
+
+
 def check_sampled(w, idx, sc, sample, tol):
     for i in sample:
         p1 = w.problems[i:i + 1]
@@ -68,26 +102,27 @@ def check_sampled(w, idx, sc, sample, tol):
         assert ok, f"problem {i}: {msg}"
 
 
-def test_config1_full_space(ks, ctx):
-    w = wl.make_workload(1)
+@pytest.mark.parametrize("law", ["pernode", "hist256", "slots128"])
+def test_config1_full_space(ks, ctx, law):
+    w = wl.make_workload(1, law=law)
     assert w.pairs == 61_440_000
     model = ctx.model_create_gbdt(*w.gbdt)
+    assert "select_fast_kernel" in model.describe()
     idx, sc = run_full(ks, ctx, w, model)
     check_properties(w, idx, sc)
-    sample = wl.randint(7, 1, np.arange(12), len(w.problems))
-    check_sampled(w, idx, sc, [0, len(w.problems) - 1] + sample.tolist(), TOL_GBDT)
+    check_every_problem(f"cfg1_{law}", w, idx, sc, TOL_GBDT)
     idx2, sc2 = run_full(ks, ctx, w, model)
     assert np.array_equal(idx, idx2) and np.array_equal(sc.view(np.uint32), sc2.view(np.uint32))
 
 
 def test_config2_cross_precision(ks, ctx):
-    w = wl.make_workload(2)
+    w = wl.make_workload(2, law="pernode")
     assert w.pairs == 67_108_864
     model = ctx.model_create_gbdt(*w.gbdt)
+    assert "select_fast_kernel" in model.describe()
     idx, sc = run_full(ks, ctx, w, model)
     check_properties(w, idx, sc)
-    sample = wl.randint(7, 2, np.arange(10), len(w.problems))
-    check_sampled(w, idx, sc, [0, len(w.problems) - 1] + sample.tolist(), TOL_GBDT)
+    check_every_problem("cfg2_pernode", w, idx, sc, TOL_GBDT)
 
 
 def test_config4_neural_ranker(ks, ctx):
@@ -96,30 +131,38 @@ def test_config4_neural_ranker(ks, ctx):
     model = ctx.model_create_mlp(w.mlp)
     idx, sc = run_full(ks, ctx, w, model)
     check_properties(w, idx, sc)
-    check_sampled(w, idx, sc, [0, 517, len(w.problems) - 1], TOL_MLP)
+    # bf16 rounding points differ in order of summation: near-ties swap, so most rows take the full rule
+    check_every_problem("cfg4", w, idx, sc, TOL_MLP, exact_indices=False)
     idx2, sc2 = run_full(ks, ctx, w, model)
     assert np.array_equal(idx, idx2) and np.array_equal(sc.view(np.uint32), sc2.view(np.uint32))
 
 
-def test_config3_latency_stream_sample(ks, ctx):
-    """Calls drawn from the 100,000-call stream (first, last and a few in between)."""
+def test_config3_latency_stream(ks, ctx):
+    """The first 1,000 calls of the 100,000-call stream, every one against the oracle; then calls
+    from the rest of the stream (last and a few in between)."""
     w = wl.make_workload(3, P=100_000)
     model = ctx.model_create_gbdt(*w.gbdt)
     dev = torch.device("cuda", 0)
     d_c = ks.to_device(w.candidates, dev)
     C = len(w.candidates)
-    for i in [0, 1, 49_999, 77_777, 99_999]:
+    call = ctx.select_one_caller(d_c, C, model, w.k)
+    structs = ks.problem_structs(w.problems[:1000])
+    idx, sc = np.empty((1000, w.k), np.int32), np.empty((1000, w.k), np.float32)
+    for i in range(1000):
+        ci, cs = call(structs[i])
+        idx[i], sc[i] = ci.numpy(), cs.numpy()
+    w1000 = wl.make_workload(3, P=1000)
+    assert np.array_equal(w1000.problems, w.problems[:1000])
+    check_every_problem("cfg3_pernode", w1000, idx, sc, TOL_GBDT)
+    for i in [49_999, 77_777, 99_999]:
         hi, hs = ctx.select_one(w.problems[i:i + 1], d_c, C, model, w.k)
         _, _, allsc = oracle.select(w.problems[i:i + 1], w.candidates, w.desc, w.k, gbdt=w.gbdt, want_scores=True)
         ok, msg = topk_accept(hi.numpy(), hs.numpy(), allsc, np.arange(C, dtype=np.int32), w.k, TOL_GBDT)
         assert ok, f"call {i}: {msg}"
-    # the prepared caller (the form bench.py times) is the same call
-    call = ctx.select_one_caller(d_c, C, model, w.k)
-    structs = ks.problem_structs(w.problems[:300])
+    # the plain call is the same call as the prepared caller
     for i in [0, 7, 299]:
         hi, hs = ctx.select_one(w.problems[i:i + 1], d_c, C, model, w.k)
-        ci, cs = call(structs[i])
-        assert np.array_equal(ci.numpy(), hi.numpy()) and np.array_equal(cs.numpy(), hs.numpy())
+        assert np.array_equal(hi.numpy(), idx[i]) and np.array_equal(hs.numpy(), sc[i])
 
 
 def test_full_size_paper_forms(ks, ctx):

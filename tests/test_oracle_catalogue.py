@@ -31,6 +31,29 @@ def is_valid(p, c, flags=COUPLED):
     return len(oracle.valid_catalogue(p, DESC, flags, candidates=c)[0]) == len(c)
 
 
+PRINTED = 4      # flag bit 2: the capacity rule exactly as the table prints it
+
+
+def test_capacity_rule_as_printed_and_as_read():
+    """bf16, tile 128 x 96 x 128, four stages: mainloop 4 * 128 * (128 + 96) * 2 = 229,376 B, TMA
+    epilogue 2 * 64 * 32 * 2 = 8,192 B, reserve 2,048 B, capacity 232,448 B. A warp-specialised
+    mainloop reuses its buffers for the epilogue (229,376 + 2,048 fits); the printed sum
+    mainloop + epilogue + reserve = 239,616 does not. A cooperative mainloop holds both at once
+    under either reading. Over the whole space the printed form keeps fewer candidates, and its
+    between-layout differences are 50 / 50 / 90 instead of the paper's 55 / 55 / 99."""
+    ws = candidate(128, 96, 128, 4, kernel_sched=0, epi_sched=1)
+    assert is_valid(bf16(), ws, flags=COUPLED) and not is_valid(bf16(), ws, flags=COUPLED | PRINTED)
+    coop = candidate(128, 96, 128, 4, kernel_sched=2, epi_sched=2)
+    assert not is_valid(bf16(), coop, flags=COUPLED) and not is_valid(bf16(), coop, flags=COUPLED | PRINTED)
+    small = candidate(128, 96, 128, 3, kernel_sched=0, epi_sched=1)
+    assert is_valid(bf16(), small, flags=COUPLED | PRINTED)
+    n_read = [len(oracle.valid_catalogue(bf16(lay), DESC, COUPLED, dtype=DT)[1]) for lay in range(4)]
+    n_printed = [len(oracle.valid_catalogue(bf16(lay), DESC, COUPLED | PRINTED, dtype=DT)[1]) for lay in range(4)]
+    assert all(a < b for a, b in zip(n_printed, n_read))
+    assert (n_read[0] - n_read[1], n_read[0] - n_read[2], n_read[0] - n_read[3]) == (55, 55, 99)
+    assert (n_printed[0] - n_printed[1], n_printed[0] - n_printed[2], n_printed[0] - n_printed[3]) == (50, 50, 90)
+
+
 def test_size_is_the_papers_534600():
     assert oracle.catalogue_size() == 534600 == 4 * 9 * 5 * 11 * 15 * 3 * 3 * 2
 

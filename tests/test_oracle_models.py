@@ -28,7 +28,7 @@ def test_tiny_scoring_example():
     """Two depth-1 trees on the worked examples: T1 splits the wave count (column 30) at 3.5
     into (+0.1 | -0.2); T2 splits eta_last (column 31) at 0.5 into (-0.3 | +0.3).
     A: 7 waves, eta 0.988 -> -0.2 + 0.3; B: 1 wave, eta 0.108 -> 0.1 - 0.3; C: 1 wave,
-    eta 0.541 -> 0.1 + 0.3."""
+    eta 0.541 -> 0.1 + 0.3; D: 1 wave, eta 0.065 -> 0.1 - 0.3."""
     ex = read_worked_examples(GOLDEN)
     x = np.concatenate([oracle.featurize(p, c, DESC) for _, p, c, _ in ex])
     t1 = make_tree([(30, 3.5, 1), (None, 0.1, 0), (None, -0.2, 0)])
@@ -36,10 +36,10 @@ def test_tiny_scoring_example():
     nodes = np.concatenate([t1, t2])
     off = np.array([0, 3, 6])
     s, leaf = oracle.score_gbdt(x, off, nodes, want_leaf_idx=True)
-    np.testing.assert_allclose(s, [0.1, -0.2, 0.4], rtol=1e-6)
-    assert leaf.tolist() == [[2, 2], [1, 1], [1, 2]]
+    np.testing.assert_allclose(s, [0.1, -0.2, 0.4, -0.2], rtol=1e-6)
+    assert leaf.tolist() == [[2, 2], [1, 1], [1, 2], [1, 1]]
     s2 = oracle.score_gbdt(x, off, nodes, base_score=1.5)
-    np.testing.assert_allclose(s2, [1.6, 1.3, 1.9], rtol=1e-6)
+    np.testing.assert_allclose(s2, [1.6, 1.3, 1.9, 1.3], rtol=1e-6)
 
 
 def test_depth0_trees_give_a_constant():

@@ -1,7 +1,9 @@
 """ks_select_trees_static, the entry point for callers that may not allocate device memory
 (their pool owns the whole GPU, or a synchronising cudaMalloc is off-limits where they run):
-its results must match the regular ks_select on the same inputs, on two calls in a row that
-share the library's fixed scratch array, and oversize requests must be refused up front.
+its results must match the CPU oracle and the regular ks_select on the same inputs, on calls in
+a row that share the library's fixed scratch array; a call must leave the device's free memory
+as it found it (measured with cudaMemGetInfo, which sees every allocation on the device, not
+only torch's); and oversize requests must be refused up front.
 
 The file name sorts last on purpose, so that a run that stops at the first failure has
 already run every other test."""
@@ -9,7 +11,9 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2609_35587_b200 import workloads as wl
+from tests.helpers import topk_accept
 
 pytestmark = pytest.mark.gpu
 
@@ -39,12 +43,22 @@ def run_case(ks, ctx, w):
     d_off = torch.from_numpy(off.astype(np.int32)).to(dev)
     out_idx = torch.full((P, k), -7, dtype=torch.int32, device=dev)
     out_sc = torch.zeros((P, k), dtype=torch.float32, device=dev)
-    before = torch.cuda.memory_allocated()
-    st = ks.ks_select_trees_static(w.desc, d_p, P, d_c, C, d_nodes, d_off, len(off) - 1, base, k, out_idx, out_sc)
+    call = lambda: ks.ks_select_trees_static(w.desc, d_p, P, d_c, C, d_nodes, d_off, len(off) - 1, base, k,
+                                             out_idx, out_sc)
+    assert call() == ks.KS_OK       # warm call: module and array are on the device after it
     torch.cuda.synchronize()
-    assert st == ks.KS_OK
-    assert torch.cuda.memory_allocated() == before
+    free_before = torch.cuda.mem_get_info()[0]
+    out_idx.fill_(-7)
+    assert call() == ks.KS_OK
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before, "the call changed the device's free memory"
     got_idx, got_sc = out_idx.cpu().numpy(), out_sc.cpu().numpy()
+    # checker: the CPU oracle (every problem, full acceptance rule)
+    for i in range(P):
+        _, _, allsc = oracle.select(w.problems[i:i + 1], w.candidates, w.desc, k, gbdt=w.gbdt, want_scores=True)
+        ok, msg = topk_accept(got_idx[i], got_sc[i], allsc, np.arange(C, dtype=np.int32), k, TOL)
+        assert ok, f"problem {i}: {msg}"
+    # and the regular entry point
     assert np.array_equal(got_idx, ref_idx)
     assert np.all(np.abs(got_sc - ref_sc) <= TOL * np.maximum(1, np.abs(ref_sc)))
 
