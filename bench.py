@@ -4,8 +4,10 @@ full configuration space (1,024 problems x 60,000 candidates, 500 trees of depth
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload 1]
 
-One step = one pass of the whole path over the batch. With N > 1 (torchrun) every rank ranks
-its own batch of problems (no data-path collective; weak scaling) and rank 0 prints the line.
+One step = one pass of the whole path over the batch. With N > 1 (under torchrun, or started
+here when no launcher is around) every rank ranks its own batch of problems (weak scaling; the
+only exchange is the all-gather of the [P, k] result blocks) and rank 0 prints the line. The
+default N = 1 line also carries short runs of the other configurations under "extra".
 `--impl reference` times the CPU oracle on a bounded sample of the same workload instead.
 """
 from __future__ import annotations
@@ -352,6 +354,130 @@ def run_stages(args, rank, local_rank, dev):
     print(json.dumps(line), flush=True)
 
 
+def measure_select(ks, ctx, w, model, steps, warm, dev, flush, world=1, gather=None):
+    """K timed passes of ks_select over workload `w` (inputs resident on the device), each
+    bracketed by CUDA events on the launching stream with an L2 flush in front. Returns the
+    per-step times, the dominant kernel's own times, and the launches counted."""
+    import torch
+    import torch.distributed as dist
+    P, C, k = len(w.problems), len(w.candidates), w.k
+    d_p, d_c = ks.to_device(w.problems, dev), ks.to_device(w.candidates, dev)
+    d_so = None if w.seg_offsets is None else ks.to_device(w.seg_offsets, dev)
+    d_si = None if w.seg_index is None else ks.to_device(w.seg_index, dev)
+    out_idx = torch.empty((P, k), dtype=torch.int32, device=dev)
+    out_sc = torch.empty((P, k), dtype=torch.float32, device=dev)
+
+    def step():
+        ctx.select(d_p, P, d_c, C, model, k, d_so, d_si, w.pairs, out_idx, out_sc)
+        if gather is not None:  # N > 1: the one exchange of the sharded path
+            gather(out_idx, out_sc)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(warm):
+        step()
+    barrier()
+    ctx.profile_enable(True)
+    launches0 = ctx.launch_count()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    kern_ms = []
+    barrier()
+    for i in range(steps):
+        flush.fill_(i & 0xFF)
+        ev[i][0].record()
+        step()
+        ev[i][1].record()
+        kern_ms.append(ctx.profile_last_ms())
+    barrier()
+    ctx.profile_enable(False)
+    return {"step_ms": [a.elapsed_time(b) for a, b in ev], "kernel_ms": kern_ms,
+            "launches": int(ctx.launch_count() - launches0)}
+
+
+def tree_roofline(pairs, trees, depth, kms):
+    achieved = pairs * trees * depth * INSTR_PER_VISIT / (kms * 1e-3)
+    return achieved, achieved / ISSUE_PEAK
+
+
+def extra_runs(ks, ctx, dev, flush, args, peaks):
+    """Short runs of the other configurations and threshold laws, so that one default line carries
+    them: config 1 under the other two laws, config 2, config 4 (5 / 3 timed steps each), a
+    short latency stream, and the oracle on one host thread."""
+    import torch
+    from paper_2609_35587_b200 import workloads as wl
+    out = {}
+    for law in [l for l in wl.LAWS if l != args.law]:
+        w = wl.make_workload(1, law=law)
+        model = ctx.model_create_gbdt(*w.gbdt)
+        m = measure_select(ks, ctx, w, model, 5, 3, dev, flush)
+        kms = float(np.mean(m["kernel_ms"]))
+        out[f"config1_{law}"] = {"pairs_per_s": w.pairs / (np.mean(m["step_ms"]) * 1e-3), "ms_per_step": float(np.mean(m["step_ms"])),
+                                 "kernel_ms": kms, "frac": tree_roofline(w.pairs, 500, 8, kms)[1], "kernel": model.describe()}
+        model.close()
+    w = wl.make_workload(2, law=args.law)
+    model = ctx.model_create_gbdt(*w.gbdt)
+    m = measure_select(ks, ctx, w, model, 3, 3, dev, flush)
+    kms = float(np.mean(m["kernel_ms"]))
+    out[f"config2_{args.law}"] = {"pairs_per_s": w.pairs / (np.mean(m["step_ms"]) * 1e-3), "ms_per_step": float(np.mean(m["step_ms"])),
+                                  "kernel_ms": kms, "frac": tree_roofline(w.pairs, 1000, 8, kms)[1], "kernel": model.describe()}
+    model.close()
+    del w
+    w = wl.make_workload(4)
+    model = ctx.model_create_mlp(w.mlp)
+    m = measure_select(ks, ctx, w, model, 5, 3, dev, flush)
+    kms = float(np.mean(m["kernel_ms"]))
+    tflops = w.pairs * 2.0 * (64 * 256 + 256 * 256) / (kms * 1e-3) / 1e12
+    out["config4"] = {"pairs_per_s": w.pairs / (np.mean(m["step_ms"]) * 1e-3), "ms_per_step": float(np.mean(m["step_ms"])),
+                      "kernel_ms": kms, "tflops": tflops, "frac_of_sustained_bf16": tflops / peaks["bf16_tflops_sustained"],
+                      "frac_of_burst_bf16": tflops / peaks["bf16_tflops"], "kernel": model.describe()}
+    model.close()
+    # latency stream, short
+    w = wl.make_workload(3, P=2200, law=args.law)
+    model = ctx.model_create_gbdt(*w.gbdt)
+    d_c = ks.to_device(w.candidates, dev)
+    call = ctx.select_one_caller(d_c, len(w.candidates), model, w.k)
+    structs = ks.problem_structs(w.problems)
+    for i in range(200):
+        call(structs[i])
+    lat = np.empty(2000)
+    t_all = time.perf_counter()
+    for i in range(2000):
+        t0 = time.perf_counter()
+        call(structs[200 + i])
+        lat[i] = time.perf_counter() - t0
+    total = time.perf_counter() - t_all
+    out[f"config3_{args.law}"] = {"problems_per_s": 2000 / total, "p50_us": float(np.percentile(lat, 50) * 1e6),
+                                  "p99_us": float(np.percentile(lat, 99) * 1e6), "calls": 2000}
+    model.close()
+    # the oracle on one host thread (config 1, first two problems)
+    import oracle
+    w = wl.make_workload(1, P=2, law=args.law)
+    n_thr = oracle.threads()
+    oracle.set_threads(1)
+    t0 = time.perf_counter()
+    oracle.select(w.problems, w.candidates, w.desc, w.k, gbdt=w.gbdt)
+    dt = time.perf_counter() - t0
+    oracle.set_threads(n_thr)
+    out["oracle_1_thread"] = {"value": w.pairs / dt, "unit": UNIT, "cores": 1, "sample": f"2 problems x 60000 candidates of config 1, {dt:.1f} s"}
+    return out
+
+
+def spawn_ranks(args):
+    """`python bench.py --gpus N` with N > 1 and no launcher around it: start the N ranks here, one
+    process per GPU, the way the multi-rank launch line does."""
+    import socket
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -364,6 +490,8 @@ def main():
     ap.add_argument("--calls", type=int, default=100000, help="latency stream (workload 3): timed calls")
     ap.add_argument("--ref-problems", type=int, default=16)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extra", action="store_true",
+                    help="leave out the short runs of the other configurations that the default line carries")
     ap.add_argument("--problems", type=int, default=None,
                     help="profiling aid: rank only the first N problems of the workload (not a bench line)")
     ap.add_argument("--skip-e2e", action="store_true", help="profiling aid: skip the host-buffer leg")
@@ -373,6 +501,8 @@ def main():
                     help="time the unfused calls (ks_featurize, ks_score) one at a time instead of ks_select")
     args = ap.parse_args()
 
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -401,23 +531,17 @@ def main():
     if cfg == 3:
         run_latency_stream(args, rank, local_rank, dev)
         return
-    # weak scaling: every rank ranks its own batch of problems against the shared catalogue
+    # weak scaling: every rank ranks its own batch of problems against the shared catalogue; with
+    # N > 1 the [P, k] result blocks are all-gathered at the end of every step (the only exchange)
     w = wl.make_workload(cfg, P=args.problems, seed=wl.BASE_SEED, law=args.law)
     if rank != 0:
         w.problems = wl.make_inputs(cfg, P=args.problems, seed=wl.BASE_SEED + 7919 * rank)[0]
     P, C, k = len(w.problems), len(w.candidates), w.k
     ctx = ks.Context(w.desc, local_rank)
     model = ctx.model_create_gbdt(*w.gbdt) if w.gbdt is not None else ctx.model_create_mlp(w.mlp)
-    d_p, d_c = ks.to_device(w.problems, dev), ks.to_device(w.candidates, dev)
-    d_so = None if w.seg_offsets is None else ks.to_device(w.seg_offsets, dev)
-    d_si = None if w.seg_index is None else ks.to_device(w.seg_index, dev)
-    out_idx = torch.empty((P, k), dtype=torch.int32, device=dev)
-    out_sc = torch.empty((P, k), dtype=torch.float32, device=dev)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     pairs = w.pairs
-
-    def step():
-        ctx.select(d_p, P, d_c, C, model, k, d_so, d_si, pairs, out_idx, out_sc)
+    gather = (lambda i, s: sharding.all_gather_topk(i, s, P * world, k)) if world > 1 else None
 
     def barrier():
         if world > 1:
@@ -425,30 +549,12 @@ def main():
         torch.cuda.synchronize()
 
     n_warm = args.warmup if args.problems else max(args.warmup, 3)
-    for _ in range(n_warm):
-        step()
-    barrier()
-
-    # ---- device-resident timing: K steps, each bracketed by events, L2 flushed in between ----
-    ctx.profile_enable(True)
     sampler = ClockSampler(local_rank)
     sampler.start()
-    launches0 = ctx.launch_count()
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-          for _ in range(args.steps)]
-    kern_ms = []
-    barrier()
-    for i in range(args.steps):
-        flush.fill_(i & 0xFF)
-        ev[i][0].record()
-        step()
-        ev[i][1].record()
-        kern_ms.append(ctx.profile_last_ms())
-    barrier()
-    launches = ctx.launch_count() - launches0
+    m = measure_select(ks, ctx, w, model, args.steps, n_warm, dev, flush, world, gather)
     clocks = sampler.stop()
-    step_ms = [a.elapsed_time(b) for a, b in ev]
-    total_ms = float(sum(step_ms))
+    launches, kern_ms = m["launches"], m["kernel_ms"]
+    total_ms = float(sum(m["step_ms"]))
     if world > 1:
         total_ms = sharding.max_over_ranks(total_ms, dev)
     ms_per_step = total_ms / args.steps
@@ -461,13 +567,13 @@ def main():
     h_si = None if w.seg_index is None else torch.from_numpy(w.seg_index.copy()).pin_memory()
     h_idx = torch.empty((P, k), dtype=torch.int32).pin_memory()
     h_sc = torch.empty((P, k), dtype=torch.float32).pin_memory()
-    ctx.profile_enable(False)
     e2e_steps = 0 if args.skip_e2e else max(3, min(args.steps, 10))
     for _ in range(0 if args.skip_e2e else 2):
         ctx.select_host(h_p, P, h_c, C, model, k, h_so, h_si, pairs, h_idx, h_sc)
     barrier()
     t0 = time.perf_counter()
-    for _ in range(e2e_steps):
+    for i in range(e2e_steps):
+        flush.fill_(i & 0xFF)
         ctx.select_host(h_p, P, h_c, C, model, k, h_so, h_si, pairs, h_idx, h_sc)
     barrier()
     e2e_s = (time.perf_counter() - t0) / max(e2e_steps, 1)
@@ -480,22 +586,23 @@ def main():
     if rank == 0:
         peaks = load_peaks()
         kms = float(np.mean(kern_ms))
+        cfgd = config_dict(cfg, spec, args)
+        cfgd["l2"] = "flushed before every step of both legs (256 MiB write)"
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": n_warm, "ms_per_step": ms_per_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "data": "synthetic",
-                "config": config_dict(cfg, spec, args), "clocks": clocks, "gpu_launches": int(launches),
+                "config": cfgd, "clocks": clocks, "gpu_launches": int(launches),
                 "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
                         "d2h_bytes_per_step": int(d2h)}}
         if w.gbdt is not None:
-            visits = pairs * spec["trees"] * spec["depth"]
-            achieved = visits * INSTR_PER_VISIT / (kms * 1e-3)
+            achieved, frac = tree_roofline(pairs, spec["trees"], spec["depth"], kms)
             line["dtype"] = "f32"
             line["roofline"] = {"bound": "alu", "kernel": model.describe(),
                                 "achieved": achieved / 1e12, "peak": ISSUE_PEAK / 1e12,
                                 "unit": "T thread-instr/s (4 per node visit)",
-                                "frac": achieved / ISSUE_PEAK, "kernel_ms": kms,
+                                "frac": frac, "kernel_ms": kms,
                                 "peak_source": "derived: 148 SMs x 4 schedulers x 32 lanes x 1.965 GHz",
-                                "traffic": TRAFFIC_BYTES.get(cfg)}
+                                "traffic": TRAFFIC_BYTES.get((cfg, args.law))}
         else:
             flops = pairs * 2.0 * (64 * 256 + 256 * 256)
             achieved = flops / (kms * 1e-3)
@@ -503,10 +610,14 @@ def main():
             line["roofline"] = {"bound": "tensor", "kernel": model.describe(),
                                 "achieved": achieved / 1e12, "peak": peaks["bf16_tflops_sustained"],
                                 "unit": "TFLOP/s", "frac": achieved / 1e12 / peaks["bf16_tflops_sustained"],
+                                "frac_of_burst": achieved / 1e12 / peaks["bf16_tflops"],
                                 "kernel_ms": kms, "peak_source": peaks["source"] + " (sustained bf16)",
-                                "traffic": TRAFFIC_BYTES.get(cfg)}
+                                "traffic": TRAFFIC_BYTES.get((cfg, None))}
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = cpu_baseline(cfg, args.law)
+        if world == 1 and cfg == 1 and not args.problems and not args.no_extra:
+            model.close()
+            line["extra"] = extra_runs(ks, ctx, dev, flush, args, peaks)
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -517,7 +628,7 @@ def main():
 # 48-problem capture (17.6 MB) splits into 7.4 MB that do not depend on the number of problems
 # and 0.21 MB per problem (the problem's table of per-pair tile rows, read back through L2),
 # plus the partial lists of the full-size launch (9.7 MB): 7.4 + 1,024 x 0.21 + 9.7.
-TRAFFIC_BYTES = {1: 234e6, 4: 5.7e6}
+TRAFFIC_BYTES = {(1, "slots128"): 234e6, (4, None): 5.7e6}
 
 if __name__ == "__main__":
     main()

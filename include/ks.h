@@ -297,6 +297,16 @@ ks_status ks_select_host(ks_ctx* ctx, const ks_problem* h_p, int P, const ks_can
                          int64_t pairs, const ks_model* model, int k, int32_t* h_topk_idx,
                          float* h_topk_score, void* stream);
 
+/* Merge of partial top-k lists (Eq. "selection" over a candidate set that was split: the best k
+ * of a union are among the best k of its parts). For each of P problems, d_idx / d_score hold n
+ * gathered (pool index, score) entries, row-major [P, n], an index of -1 marking an empty
+ * entry; d_topk_idx / d_topk_score [P, k] receive the k best by (score descending, index
+ * ascending), padded with -1 / -inf. This is the one exchange step of the multi-GPU forms: ranks
+ * that each ranked a share of the candidates gather their lists and merge them here.
+ * Asynchronous on `stream`. */
+ks_status ks_merge_topk(ks_ctx* ctx, const int32_t* d_idx, const float* d_score, int P, int n, int k,
+                        int32_t* d_topk_idx, float* d_topk_score, void* stream);
+
 /* ---- selection without any allocation ------------------------------------------------------- */
 
 /* (The paper has no counterpart: this entry point exists for deployment reasons only.)

@@ -25,7 +25,7 @@ EXPORTS = ("ks_create", "ks_destroy", "ks_last_cuda_error", "ks_model_create_gbd
            "ks_model_create_mlp", "ks_model_create_static", "ks_model_destroy", "ks_featurize", "ks_score", "ks_select",
            "ks_select_one", "ks_select_host", "ks_status_string", "ks_feature_count",
            "ks_feature_name", "ks_launch_count", "ks_profile_enable", "ks_profile_last_ms", "ks_device_status", "ks_select_trees_static",
-           "ks_enumerate", "ks_valid_catalogue", "ks_remap_indices", "ks_model_describe",
+           "ks_enumerate", "ks_valid_catalogue", "ks_remap_indices", "ks_model_describe", "ks_merge_topk",
            "ks_debug_set_wait", "ks_debug_bounds_line", "ks_debug_bounds_clear")
 
 
@@ -77,6 +77,7 @@ def _load() -> ctypes.CDLL:
                                        ctypes.POINTER(ctypes.c_int32), vp]
     lib.ks_remap_indices.argtypes = [vp, vp, i64, vp, i32, vp]
     lib.ks_model_describe.argtypes = [vp, ctypes.c_char_p, i32]
+    lib.ks_merge_topk.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, vp]
     lib.ks_debug_set_wait.argtypes = [vp, i32, i32]
     lib.ks_debug_bounds_line.restype = i32
     lib.ks_debug_bounds_clear.restype = None
@@ -305,6 +306,17 @@ class Context:
         st = _lib.ks_select(self._h, _dptr(d_p), P, _dptr(d_c), C, _dptr(d_seg_off), _dptr(d_seg_idx),
                             pairs, model._h, k, _dptr(out_idx), _dptr(out_score), _stream())
         self._check(st, "ks_select")
+        return out_idx, out_score
+
+    def merge_topk(self, d_idx, d_score, k, out_idx=None, out_score=None):
+        """[P, n] gathered (index, score) entries -> the k best per problem, [P, k]."""
+        P, n = d_idx.shape
+        if out_idx is None:
+            out_idx = torch.empty((P, k), dtype=torch.int32, device=self.device)
+            out_score = torch.empty((P, k), dtype=torch.float32, device=self.device)
+        st = _lib.ks_merge_topk(self._h, _dptr(d_idx), _dptr(d_score), P, n, k, _dptr(out_idx), _dptr(out_score),
+                                _stream())
+        self._check(st, "ks_merge_topk")
         return out_idx, out_score
 
     def select_one_caller(self, d_c, C, model: Model, k, h_idx=None, h_score=None):

@@ -315,6 +315,17 @@ ks_status ks_profile_last_ms(ks_ctx* ctx, float* out_ms) {
   return e == cudaSuccess ? KS_OK : cuda_fail(ctx, e, "ks_profile_last_ms");
 }
 
+ks_status ks_merge_topk(ks_ctx* ctx, const int32_t* d_idx, const float* d_score, int P, int n, int k,
+                        int32_t* d_topk_idx, float* d_topk_score, void* stream) {
+  if (!ctx || P < 0 || n < 0 || k < 1 || k > KS_MAX_K) return KS_ERR_INVALID_ARG;
+  if (P == 0) return KS_OK;
+  if (!d_topk_idx || !d_topk_score || (n > 0 && (!d_idx || !d_score))) return KS_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  cudaError_t e = ks::launch_merge_lists(d_idx, d_score, P, n, k, d_topk_idx, d_topk_score,
+                                         static_cast<cudaStream_t>(stream), &ctx->launches);
+  return e == cudaSuccess ? KS_OK : cuda_fail(ctx, e, "ks_merge_topk");
+}
+
 ks_status ks_model_describe(const ks_model* model, char* buf, int len) {
   if (!model || !buf || len < 1) return KS_ERR_INVALID_ARG;
   if (model->kind == 0 && model->gbdt.fast) {

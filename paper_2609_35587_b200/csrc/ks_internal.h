@@ -257,6 +257,10 @@ cudaError_t launch_select_mlp_tc(const ks_gpu_desc& desc, const MlpModel& m, con
                                  unsigned long long* partial, void* scratch, int* status, cudaStream_t stream,
                                  int64_t* launches, cudaEvent_t ev_begin, const FastWait* wait = nullptr);
 
+// k-way merge of gathered partial lists (multi-GPU candidate split).
+cudaError_t launch_merge_lists(const int32_t* d_idx, const float* d_score, int P, int n, int k, int32_t* d_out_idx,
+                               float* d_out_score, cudaStream_t stream, int64_t* launches);
+
 // ---- launchers (each enqueues on `stream`, returns the cudaError of the launch) -----------
 cudaError_t launch_featurize(const ks_gpu_desc& desc, const ks_problem* d_p, int P,
                              const ks_candidate* d_c, int C, const int64_t* d_seg_off,

@@ -569,6 +569,40 @@ topk_merge_kernel(const unsigned long long* __restrict__ partial, int P, int n_k
   }
 }
 
+// Merge of ranked lists (the exchange step of a candidate-split selection): per problem, n
+// (index, score) entries gathered from several partial top-k lists, index -1 = empty; the k best
+// by (score descending, index ascending) go to the output. One warp per problem.
+__global__ void __launch_bounds__(kBlock)
+merge_lists_kernel(const int32_t* __restrict__ in_idx, const float* __restrict__ in_score, int P, int n, int k,
+                   int32_t* __restrict__ out_idx, float* __restrict__ out_score) {
+  const int warp = (blockIdx.x * kBlock + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (warp >= P) return;
+  const int32_t* idx = in_idx + static_cast<size_t>(warp) * n;
+  const float* sc = in_score + static_cast<size_t>(warp) * n;
+  unsigned long long prev = ~0ull;
+  for (int j = 0; j < k; ++j) {
+    unsigned long long best = 0ull;
+    for (int i = lane; i < n; i += 32) {
+      const unsigned long long v = idx[i] >= 0 ? make_key(sc[i] + 0.0f, idx[i]) : 0ull;
+      if (v < prev && v > best) best = v;
+    }
+    best = warp_max_u64(best);
+    if (lane == 0) {
+      out_idx[static_cast<size_t>(warp) * k + j] = key_index(best);
+      out_score[static_cast<size_t>(warp) * k + j] = key_score(best);
+    }
+    prev = best;
+  }
+}
+
+cudaError_t launch_merge_lists(const int32_t* d_idx, const float* d_score, int P, int n, int k, int32_t* d_out_idx,
+                               float* d_out_score, cudaStream_t stream, int64_t* launches) {
+  merge_lists_kernel<<<(P * 32 + kBlock - 1) / kBlock, kBlock, 0, stream>>>(d_idx, d_score, P, n, k, d_out_idx,
+                                                                           d_out_score);
+  ++*launches;
+  return cudaGetLastError();
+}
+
 // ------------------------------------------------------------------------------------------
 // launchers
 // ------------------------------------------------------------------------------------------

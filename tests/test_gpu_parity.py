@@ -596,6 +596,39 @@ def test_select_forced_tile_geometry(ks, ctx, geometry, monkeypatch):
     assert np.array_equal(hi_.numpy(), idx[1])
 
 
+def test_merge_topk_of_candidate_shares(ks, ctx):
+    """The exchange step of the candidate-split form: three shares of a pool are ranked separately
+    (per-share segments), their lists are concatenated as a gather would, and ks_merge_topk must
+    give the ranking of the whole pool; plus padding entries and exact ties."""
+    w = wl.make_workload(1, P=4, C=2000, trees=30, depth=6)
+    model = ctx.model_create_gbdt(*w.gbdt)
+    k, C, P = 10, 2000, 4
+    d_p, d_c = dev(ks, w.problems), dev(ks, w.candidates)
+    parts_i, parts_s = [], []
+    for lo, hi in ((0, 700), (700, 707), (707, 2000)):   # the middle share has fewer than k members
+        so = np.arange(P + 1, dtype=np.int64) * (hi - lo)
+        si = np.tile(np.arange(lo, hi, dtype=np.int32), P)
+        i, s = ctx.select(d_p, P, d_c, C, model, k, dev(ks, so), dev(ks, si), int(so[-1]))
+        parts_i.append(i)
+        parts_s.append(s)
+    gi, gs = ctx.merge_topk(torch.cat(parts_i, dim=1).contiguous(), torch.cat(parts_s, dim=1).contiguous(), k)
+    torch.cuda.synchronize()
+    check_select(w, gi.cpu().numpy(), gs.cpu().numpy(), TOL_GBDT)
+    # ties and padding against the plain definition
+    rng = np.random.default_rng(5)
+    idx = rng.permutation(400).astype(np.int32).reshape(2, 200)
+    sc = rng.integers(0, 6, (2, 200)).astype(np.float32)
+    idx[:, ::7] = -1
+    gi, gs = ctx.merge_topk(dev(ks, idx), dev(ks, sc), 32)
+    for r in range(2):
+        live = idx[r] >= 0
+        order = np.lexsort((idx[r][live], -sc[r][live]))[:32]
+        assert np.array_equal(gi[r].cpu().numpy(), idx[r][live][order])
+        assert np.array_equal(gs[r].cpu().numpy(), sc[r][live][order])
+    few = ctx.merge_topk(dev(ks, idx[:, :7]), dev(ks, sc[:, :7]), 10)[0].cpu().numpy()
+    assert np.all(few[:, 6:] == -1)
+
+
 def test_select_memo_table_in_batches(ks, ctx):
     """The per-(problem, class) table holds 256 MiB of records; a batch of more problems than that
     is served in several launches that reuse it (here 80-byte records: 409 problems at a time)."""

@@ -45,8 +45,28 @@ def _worker(rank, world, port, P, q):
 
     idx, sc = sharding.select_sharded(select_fn, w.problems, w.k, torch.device("cpu"))
     t = sharding.max_over_ranks(10.0 + rank, torch.device("cpu"))
+
+    # candidate split of the single-problem call: each rank ranks its share of the pool, the
+    # world x k pairs are gathered and merged (the oracle's top-k stands in for ks_merge_topk)
+    def select_part(lo, hi):
+        pool = np.arange(lo, hi, dtype=np.int32)
+        i1, s1 = oracle.select(w.problems[:1], w.candidates, w.desc, w.k, gbdt=w.gbdt,
+                               seg_off=np.array([0, hi - lo], np.int64), seg_idx=pool)
+        return torch.from_numpy(i1[0]), torch.from_numpy(s1[0])
+
+    def merge(i_all, s_all, k):
+        live = np.nonzero(i_all.numpy()[0] >= 0)[0]
+        mi, ms = oracle.topk(s_all.numpy()[0][live], 1, k, seg_off=np.array([0, len(live)], np.int64),
+                             seg_idx=i_all.numpy()[0][live].astype(np.int32))
+        return torch.from_numpy(mi), torch.from_numpy(ms)
+
+    one_i, one_s = [], []
+    for C in (300, 1):   # the second: a rank with no candidates at all
+        oi, os_ = sharding.select_one_sharded(select_part, merge, C, w.k, torch.device("cpu"))
+        one_i.append(oi.numpy())
+        one_s.append(os_.numpy())
     if rank == 0:
-        q.put((idx.numpy(), sc.numpy(), t))
+        q.put((idx.numpy(), sc.numpy(), t, one_i, one_s))
     dist.barrier()
     dist.destroy_process_group()
 
@@ -61,7 +81,7 @@ def test_two_ranks_match_the_unsharded_ranking():
         procs = [ctx.Process(target=_worker, args=(r, 2, port, P, q)) for r in range(2)]
         for p in procs:
             p.start()
-        idx, sc, t = q.get(timeout=120)
+        idx, sc, t, one_i, one_s = q.get(timeout=120)
         for p in procs:
             p.join(timeout=120)
             assert p.exitcode == 0
@@ -69,3 +89,6 @@ def test_two_ranks_match_the_unsharded_ranking():
         ridx, rsc = oracle.select(w.problems, w.candidates, w.desc, w.k, gbdt=w.gbdt)
         assert np.array_equal(idx, ridx) and np.array_equal(sc, rsc)
         assert t == 11.0
+        for C, oi, os_ in zip((300, 1), one_i, one_s):
+            r1i, r1s = oracle.select(w.problems[:1], w.candidates[:C], w.desc, w.k, gbdt=w.gbdt)
+            assert np.array_equal(oi, r1i[0]) and np.array_equal(os_, r1s[0])
