@@ -193,7 +193,8 @@ def run_latency_stream(args, rank, local_rank, dev):
     h_idx = torch.empty(k, dtype=torch.int32).pin_memory()
     h_sc = torch.empty(k, dtype=torch.float32).pin_memory()
     # the C call itself is what is timed: pointers and the by-value structs are prepared once
-    call = ctx.select_one_caller(d_c, C, model, k, h_idx, h_sc)
+    cat = None if args.unprepared else ctx.catalogue_prepare(d_c, C, model)
+    call = ctx.select_one_caller(d_c, C, model, k, h_idx, h_sc, catalogue=cat)
     structs = ks.problem_structs(w.problems)
     for i in range(n_warm):
         call(structs[i])
@@ -213,7 +214,8 @@ def run_latency_stream(args, rank, local_rank, dev):
             "value": n / total, "unit": "problems/s", "n_gpus": 1, "steps": n, "warmup": n_warm,
             "ms_per_step": total / n * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
-            "config": {"workload": "config 3 (dynamic)", "candidates": C, "trees": 500, "depth": 8, "k": k,
+            "config": {"workload": f"config 3 (dynamic), thresholds: {args.law}", "candidates": C, "trees": 500, "depth": 8, "k": k,
+                       "call": "ks_select_one" if args.unprepared else "ks_select_one_prepared", "kernel": model.describe(),
                        "l2": "catalogue and model are L2-resident by design (re-used every call)"},
             "latency_us": {"p50": float(np.percentile(lat, 50) * 1e6), "p99": float(np.percentile(lat, 99) * 1e6),
                            "mean": float(lat.mean() * 1e6)},
@@ -438,7 +440,8 @@ def extra_runs(ks, ctx, dev, flush, args, peaks):
     w = wl.make_workload(3, P=2200, law=args.law)
     model = ctx.model_create_gbdt(*w.gbdt)
     d_c = ks.to_device(w.candidates, dev)
-    call = ctx.select_one_caller(d_c, len(w.candidates), model, w.k)
+    cat = ctx.catalogue_prepare(d_c, len(w.candidates), model)
+    call = ctx.select_one_caller(d_c, len(w.candidates), model, w.k, catalogue=cat)
     structs = ks.problem_structs(w.problems)
     for i in range(200):
         call(structs[i])
@@ -488,6 +491,8 @@ def main():
     ap.add_argument("--law", default="pernode", choices=["pernode", "hist256", "slots128"],
                     help="threshold law of the synthetic tree ensemble (workloads.LAWS)")
     ap.add_argument("--calls", type=int, default=100000, help="latency stream (workload 3): timed calls")
+    ap.add_argument("--unprepared", action="store_true",
+                    help="latency stream: plain ks_select_one instead of the prepared-catalogue call")
     ap.add_argument("--ref-problems", type=int, default=16)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra", action="store_true",

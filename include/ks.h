@@ -128,6 +128,7 @@ typedef struct {
 
 typedef struct ks_ctx ks_ctx;
 typedef struct ks_model ks_model;
+typedef struct ks_catalogue ks_catalogue;
 
 /* ---- context ------------------------------------------------------------------------- */
 
@@ -288,6 +289,24 @@ ks_status ks_select(ks_ctx* ctx, const ks_problem* d_p, int P, const ks_candidat
 ks_status ks_select_one(ks_ctx* ctx, ks_problem p, const ks_candidate* d_c, int C,
                         const ks_model* model, int k, int32_t* h_topk_idx,
                         float* h_topk_score, void* stream);
+
+/* A candidate catalogue prepared for a stream of single-problem calls with one model (the
+ * dynamic-selection setting: problems arrive one at a time, the catalogue and the ranker stay).
+ * Everything about a call that depends only on (catalogue, model) is computed here, once: for a
+ * tree ensemble on the quantised path, every candidate's quantised candidate-only columns under
+ * each of the 16 element-type combinations and the classes of candidates that look alike to
+ * the per-pair columns. ks_select_one_prepared then evaluates the per-pair columns once per class
+ * for the problem at hand and runs the fused walk + top-k: two launches per call instead of
+ * building the candidates' tiles anew. The handle owns its device memory (a few hundred bytes
+ * per candidate), refers to d_c and the model (both must outlive it and stay unchanged) and
+ * belongs to the context. For models the quantised path does not serve, the handle is a plain
+ * reference and ks_select_one_prepared is ks_select_one. Synchronises `stream`. */
+ks_status ks_catalogue_prepare(ks_ctx* ctx, const ks_candidate* d_c, int C, const ks_model* model,
+                               ks_catalogue** out_catalogue, void* stream);
+ks_status ks_catalogue_destroy(ks_catalogue* catalogue);
+/* ks_select_one against a prepared catalogue: same results, same conventions. */
+ks_status ks_select_one_prepared(ks_ctx* ctx, const ks_catalogue* catalogue, ks_problem p, int k,
+                                 int32_t* h_topk_idx, float* h_topk_score, void* stream);
 
 /* ks_select for callers whose inputs live in HOST memory: copies problems, candidates and
  * segment arrays to the device, runs ks_select, copies the [P, k] results back and

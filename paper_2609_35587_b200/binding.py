@@ -25,7 +25,8 @@ EXPORTS = ("ks_create", "ks_destroy", "ks_last_cuda_error", "ks_model_create_gbd
            "ks_model_create_mlp", "ks_model_create_static", "ks_model_destroy", "ks_featurize", "ks_score", "ks_select",
            "ks_select_one", "ks_select_host", "ks_status_string", "ks_feature_count",
            "ks_feature_name", "ks_launch_count", "ks_profile_enable", "ks_profile_last_ms", "ks_device_status", "ks_select_trees_static",
-           "ks_enumerate", "ks_valid_catalogue", "ks_remap_indices", "ks_model_describe", "ks_merge_topk",
+           "ks_enumerate", "ks_valid_catalogue", "ks_remap_indices", "ks_model_describe", "ks_merge_topk", "ks_catalogue_prepare", "ks_catalogue_destroy",
+           "ks_select_one_prepared",
            "ks_debug_set_wait", "ks_debug_bounds_line", "ks_debug_bounds_clear")
 
 
@@ -78,6 +79,9 @@ def _load() -> ctypes.CDLL:
     lib.ks_remap_indices.argtypes = [vp, vp, i64, vp, i32, vp]
     lib.ks_model_describe.argtypes = [vp, ctypes.c_char_p, i32]
     lib.ks_merge_topk.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp, vp]
+    lib.ks_catalogue_prepare.argtypes = [vp, vp, i32, vp, ctypes.POINTER(vp), vp]
+    lib.ks_catalogue_destroy.argtypes = [vp]
+    lib.ks_select_one_prepared.argtypes = [vp, vp, _Problem, i32, vp, vp, vp]
     lib.ks_debug_set_wait.argtypes = [vp, i32, i32]
     lib.ks_debug_bounds_line.restype = i32
     lib.ks_debug_bounds_clear.restype = None
@@ -183,6 +187,24 @@ class Model:
     def close(self):
         if self._h:
             _lib.ks_model_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class Catalogue:
+    """ks_catalogue: a candidate pool prepared for single-problem calls with one model."""
+
+    def __init__(self, ctx: "Context", handle, d_c, C: int, model: Model):
+        self.ctx, self._h, self.d_c, self.C, self.model = ctx, handle, d_c, C, model
+
+    def close(self):
+        if self._h:
+            _lib.ks_catalogue_destroy(self._h)
             self._h = None
 
     def __del__(self):
@@ -319,15 +341,45 @@ class Context:
         self._check(st, "ks_merge_topk")
         return out_idx, out_score
 
-    def select_one_caller(self, d_c, C, model: Model, k, h_idx=None, h_score=None):
-        """For a stream of single problems: resolves the pointers, the model handle and the
-        current stream once and returns f(p) -> (h_idx, h_score), where p is one element of
-        `problem_structs(...)`. Per call only ks_select_one itself runs; the result tensors are
-        reused from call to call."""
+    def catalogue_prepare(self, d_c, C, model: Model) -> Catalogue:
+        h = ctypes.c_void_p()
+        st = _lib.ks_catalogue_prepare(self._h, _dptr(d_c), C, model._h, ctypes.byref(h), _stream())
+        self._check(st, "ks_catalogue_prepare")
+        return Catalogue(self, h, d_c, C, model)
+
+    def select_one_prepared(self, catalogue: Catalogue, problem: np.ndarray, k, h_idx=None, h_score=None):
+        r = np.ascontiguousarray(problem).reshape(-1)[0]
+        p = _Problem(int(r["m"]), int(r["n"]), int(r["k"]), int(r["layout"]), int(r["dtype_ab"]),
+                     int(r["dtype_d"]), int(r["epi_flags"]))
         if h_idx is None:
             h_idx = torch.empty(k, dtype=torch.int32).pin_memory()
             h_score = torch.empty(k, dtype=torch.float32).pin_memory()
-        fn, check = _lib.ks_select_one, self._check
+        st = _lib.ks_select_one_prepared(self._h, catalogue._h, p, k, _hptr(h_idx), _hptr(h_score), _stream())
+        self._check(st, "ks_select_one_prepared")
+        return h_idx, h_score
+
+    def select_one_caller(self, d_c, C, model: Model, k, h_idx=None, h_score=None, catalogue: Catalogue = None):
+        """For a stream of single problems: resolves the pointers, the model handle and the
+        current stream once and returns f(p) -> (h_idx, h_score), where p is one element of
+        `problem_structs(...)`. Per call only ks_select_one (ks_select_one_prepared when a prepared
+        catalogue is given) itself runs; the result tensors are reused from call to call."""
+        if h_idx is None:
+            h_idx = torch.empty(k, dtype=torch.int32).pin_memory()
+            h_score = torch.empty(k, dtype=torch.float32).pin_memory()
+        check = self._check
+        if catalogue is not None:
+            fn = _lib.ks_select_one_prepared
+            args = (k, _hptr(h_idx), _hptr(h_score), _stream())
+            ctx_h, cat_h = self._h, catalogue._h
+            keep = (catalogue, None, h_idx, h_score)
+
+            def call_prepared(p):
+                st = fn(ctx_h, cat_h, p, *args)
+                if st != KS_OK:
+                    check(st, "ks_select_one_prepared")
+                return keep[2], keep[3]
+            return call_prepared
+        fn = _lib.ks_select_one
         args = (_dptr(d_c), C, model._h, k, _hptr(h_idx), _hptr(h_score), _stream())
         ctx_h = self._h
         keep = (d_c, model, h_idx, h_score)  # the closure keeps the buffers alive

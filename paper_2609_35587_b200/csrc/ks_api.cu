@@ -666,6 +666,101 @@ ks_status ks_select_one(ks_ctx* ctx, ks_problem p, const ks_candidate* d_c, int 
   return read_status(ctx);
 }
 
+ks_status ks_catalogue_prepare(ks_ctx* ctx, const ks_candidate* d_c, int C, const ks_model* model,
+                               ks_catalogue** out_catalogue, void* stream) {
+  if (!out_catalogue) return KS_ERR_INVALID_ARG;
+  *out_catalogue = nullptr;
+  if (!ctx || !model || model->ctx != ctx || C < 0 || (C > 0 && !d_c) || !aligned16(d_c)) return KS_ERR_INVALID_ARG;
+  ks_catalogue* cat = new (std::nothrow) ks_catalogue();
+  if (!cat) return KS_ERR_OOM;
+  cat->ctx = ctx;
+  cat->model = model;
+  cat->d_c = d_c;
+  cat->C = C;
+  cat->device = ctx->device;
+  const ks::GbdtModel& g = model->gbdt;
+  if (model->kind == 0 && g.fast && C > 0) {
+    const int nblk = (C + g.block_cands - 1) / g.block_cands;
+    const int S = ks::fast_slices(g, nblk);
+    const size_t b_memo = ks::fast_prepared_memo_bytes(g, C);
+    if (S > 1 && b_memo > 0) {
+      DeviceGuard guard(ctx->device);
+      const size_t b_rows = align_up(ks::fast_prepared_rows_bytes(g, C));
+      const size_t b_part = align_up(sizeof(unsigned long long) * nblk * KS_MAX_K);
+      const size_t b_scores = align_up(sizeof(float) * static_cast<size_t>(S) * C);
+      cat->off_memo = b_rows;
+      cat->off_part = b_rows + align_up(b_memo);
+      cat->off_scores = cat->off_part + b_part;
+      cudaError_t e = cudaMalloc(&cat->d_mem, cat->off_scores + b_scores);
+      if (e == cudaSuccess)
+        e = ks::fast_prepare(ctx->desc, g, d_c, C, cat->d_mem, static_cast<char*>(cat->d_mem) + cat->off_memo,
+                             static_cast<cudaStream_t>(stream), &ctx->launches);
+      if (e == cudaSuccess) e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+      if (e != cudaSuccess) {
+        cudaFree(cat->d_mem);
+        delete cat;
+        return cuda_fail(ctx, e, "ks_catalogue_prepare");
+      }
+      cat->nblk = nblk;
+      cat->slices = S;
+      cat->prepared = true;
+    }
+  }
+  *out_catalogue = cat;
+  return KS_OK;
+}
+
+ks_status ks_catalogue_destroy(ks_catalogue* cat) {
+  if (!cat) return KS_OK;
+  DeviceGuard g(cat->device);
+  cudaFree(cat->d_mem);
+  delete cat;
+  return KS_OK;
+}
+
+ks_status ks_select_one_prepared(ks_ctx* ctx, const ks_catalogue* cat, ks_problem p, int k, int32_t* h_topk_idx,
+                                 float* h_topk_score, void* stream) {
+  if (!ctx || !cat || cat->ctx != ctx || k < 1 || k > KS_MAX_K || !h_topk_idx || !h_topk_score)
+    return KS_ERR_INVALID_ARG;
+  if (!cat->prepared) return ks_select_one(ctx, p, cat->d_c, cat->C, cat->model, k, h_topk_idx, h_topk_score, stream);
+  if (p.m < 1 || p.n < 1 || p.k < 1 || p.m > KS_MAX_DIM || p.n > KS_MAX_DIM || p.k > KS_MAX_DIM ||
+      p.layout > 3 || p.dtype_ab > 3 || p.dtype_d > 3 || p.epi_flags > 5)
+    return KS_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int32_t* pin_idx = static_cast<int32_t*>(ctx->pinned);
+  float* pin_sc = reinterpret_cast<float*>(pin_idx + KS_MAX_K);
+  char* base = static_cast<char*>(cat->d_mem);
+  const ks::GbdtModel& gm = cat->model->gbdt;
+  ks::FastSlice sl{};
+  sl.n_slices = cat->slices;
+  sl.pairs = cat->C;
+  sl.scores = reinterpret_cast<float*>(base + cat->off_scores);
+  sl.counters = ctx->d_counters;
+  sl.out_idx = ctx->d_pinned_idx;
+  sl.out_score = ctx->d_pinned_score;
+  sl.tiles = nullptr;
+  int* h_seq = reinterpret_cast<int*>(pin_sc + KS_MAX_K);
+  sl.out_seq = reinterpret_cast<int*>(ctx->d_pinned_score + KS_MAX_K);
+  sl.seq = ++ctx->select_one_seq;
+  ks::FastPrepared prep{reinterpret_cast<const uint8_t*>(base), base + cat->off_memo};
+  cudaError_t e = ks::launch_select_fast(ctx->desc, gm, nullptr, &p, 1, cat->d_c, cat->C, cat->nblk, gm.block_cands,
+                                         nullptr, nullptr, k, reinterpret_cast<unsigned long long*>(base + cat->off_part),
+                                         nullptr, ctx->d_status, st, &ctx->launches, nullptr, &sl, nullptr, &ctx->wait,
+                                         &prep);
+  if (e == cudaSuccess) {
+    bool seen = false;
+    for (int spin = 0; spin < (1 << 22) && !seen; ++spin) seen = *static_cast<volatile int*>(h_seq) == sl.seq;
+    if (!seen) e = cudaStreamSynchronize(st);  // a failed launch never writes the word: wait the regular way
+  }
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "ks_select_one_prepared");
+  ks_status s = read_status(ctx);
+  if (s != KS_OK) return s;
+  std::memcpy(h_topk_idx, pin_idx, k * sizeof(int32_t));
+  std::memcpy(h_topk_score, pin_sc, k * sizeof(float));
+  return KS_OK;
+}
+
 ks_status ks_select_host(ks_ctx* ctx, const ks_problem* h_p, int P, const ks_candidate* h_c, int C,
                          const int64_t* h_seg_offsets, const int32_t* h_seg_index, int64_t pairs,
                          const ks_model* model, int k, int32_t* h_topk_idx, float* h_topk_score,

@@ -204,6 +204,7 @@ struct FastView {
   const uint8_t* cand_rows;    // [kCombos][C][cand_rec] quantised candidate-only rows
   const unsigned* pair_class;  // [kCombos][C] class of every candidate, or null (no memo)
   const uint8_t* pair_tab;     // [P][kMemoCap][pair_rec] per-pair tile bytes of every (problem, class)
+  const uint8_t* prob_tab;     // [P][kFastMaxProbRows] tile bytes of the problem-only rows, or null
 };
 
 // ------------------------------------------------------------------------------------------
@@ -280,16 +281,44 @@ memo_compact_kernel(MemoView memo) {
 // grid (kMemoCap / 256, batch of problems); blocks past the number of classes leave at once.
 // `p` points at the batch's first problem, and record (problem within the batch, slot) is written.
 __global__ void __launch_bounds__(256)
-pair_table_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, const ks_candidate* __restrict__ c,
-                  FastView fv, MemoView memo, int thr_cap) {
+pair_table_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_problem p_value, int use_value,
+                  const ks_candidate* __restrict__ c, FastView fv, MemoView memo, int thr_cap) {
   extern __shared__ float s_pthr[];  // thresholds of the per-pair features
   __shared__ ProblemTerms s_pt;
   __shared__ FeatQ s_fq[64];
   const int prob = blockIdx.y, j = blockIdx.x * 256 + threadIdx.x;
-  const ks_problem pr = load_problem(p + prob);
+  // the select kernel that follows may start its own set-up now (it waits for this grid to finish
+  // before it reads the tables)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const ks_problem pr = use_value ? p_value : load_problem(p + prob);
   const int combo = (pr.dtype_ab & 3) * 4 + (pr.dtype_d & 3);
+  if (blockIdx.x == 0 && prob == 0 && threadIdx.x == 0) g_fast_abort = 0;  // (also) precedes the select kernel
   const int n_classes = memo.count[combo];
-  if (blockIdx.x * 256 >= n_classes) return;
+  if (blockIdx.x * 256 >= n_classes && blockIdx.x != gridDim.x - 1) return;
+  if (blockIdx.x == gridDim.x - 1) {
+    // the last block of the row: the problem-only rows of this problem, once for all its CTAs
+    __shared__ ProblemTerms s_pt0;
+    __shared__ float s_pf[64];
+    if (threadIdx.x == 0) {
+      problem_terms(pr, desc, s_pt0);
+      ks_candidate dummy{};
+      dummy.tile_m = dummy.tile_n = dummy.tile_k = 64;
+      dummy.stages = dummy.cluster_m = dummy.cluster_n = 1;
+      featurize_pair(s_pt0, dummy, desc, [&](int col, float v) {
+        if (col < KS_F && feat_class(col) == 0) s_pf[col] = v;
+      });
+    }
+    __syncthreads();
+    if (threadIdx.x < KS_F && feat_class(threadIdx.x) == 0) {
+      const FeatQ q = fv.feat[threadIdx.x];
+      const int first = fv.n_pair_rows + fv.n_cand_rows;
+      uint8_t* out = const_cast<uint8_t*>(fv.prob_tab) + static_cast<size_t>(prob) * kFastMaxProbRows;
+      quantise(q, fv.thr + q.thr0, s_pf[threadIdx.x], false,
+               [&](int row, uint8_t b) { out[KS_IDX(row - first, kFastMaxProbRows)] = b; });
+    }
+    if (blockIdx.x * 256 >= n_classes) return;
+    __syncthreads();
+  }
   const int slot = j < n_classes ? memo.dense[static_cast<size_t>(combo) * kMemoCap + j] : 0;
   const float* T = stage_thresholds(fv, 0, fv.thr_cand0, s_pthr, thr_cap);
   if (threadIdx.x < 64) s_fq[threadIdx.x] = fv.feat[threadIdx.x];
@@ -561,12 +590,6 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
   const int kOffTile = kNBuf * fv.buf_bytes;
   const int S = sl.n_slices;
   const int prob = blockIdx.x / (nblk * S), chunk = (blockIdx.x / S) % nblk, slice = blockIdx.x % S;
-  if (tid == 0) s_abort = *reinterpret_cast<volatile int*>(&g_fast_abort);
-  __syncthreads();
-  if (s_abort) {  // a wait ran out in an earlier CTA of this launch: the call fails, leave at once
-    if (tid < k && slice == 0 && partial) partial[(static_cast<size_t>(prob) * nblk + chunk) * k + tid] = 0ull;
-    return;
-  }
   int64_t lo, len;
   if (seg_off) {
     lo = seg_off[prob];
@@ -584,13 +607,15 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
   if (tid == 0) {
     if (!tiles_given) {
       problem_terms(use_value ? p_value : load_problem(p + prob), desc, s_pt);
-      // problem-only columns do not look at the candidate: evaluate them on a dummy one
-      ks_candidate dummy{};
-      dummy.tile_m = dummy.tile_n = dummy.tile_k = 64;
-      dummy.stages = dummy.cluster_m = dummy.cluster_n = 1;
-      featurize_pair(s_pt, dummy, desc, [&](int col, float v) {
-        if (feat_class(col) == 0) s_pfeat[col] = v;
-      });
+      if (!fv.prob_tab) {
+        // problem-only columns do not look at the candidate: evaluate them on a dummy one
+        ks_candidate dummy{};
+        dummy.tile_m = dummy.tile_n = dummy.tile_k = 64;
+        dummy.stages = dummy.cluster_m = dummy.cluster_n = 1;
+        featurize_pair(s_pt, dummy, desc, [&](int col, float v) {
+          if (feat_class(col) == 0) s_pfeat[col] = v;
+        });
+      }
     }
     for (int b = 0; b < kNBuf; ++b) mbar_init(bar0 + 8u * b, 1);
     s_fail = 0;
@@ -600,7 +625,19 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
   if (tid < 64) s_fq[tid] = fv.feat[tid];
   if (tid < KS_MAX_K) s_list[tid] = 0ull;
   __syncthreads();
-  if (!tiles_given && tid < KS_F && feat_class(tid) == 0) {
+  // everything above is independent of the kernel in front (the per-problem tables): when this
+  // grid was launched as its programmatic dependent, wait for that grid here
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (tid == 0) s_abort = *reinterpret_cast<volatile int*>(&g_fast_abort);
+  __syncthreads();
+  if (s_abort) {  // a wait ran out in an earlier CTA of this launch: the call fails, leave at once
+    if (tid < k && slice == 0 && partial) partial[(static_cast<size_t>(prob) * nblk + chunk) * k + tid] = 0ull;
+    return;
+  }
+  if (!tiles_given && fv.prob_tab) {
+    for (int i = tid; i < fv.n_prob_rows; i += THREADS)
+      s_pbin[i] = __ldcg(fv.prob_tab + static_cast<size_t>(prob) * kFastMaxProbRows + i);
+  } else if (!tiles_given && tid < KS_F && feat_class(tid) == 0) {
     const int first = fv.n_pair_rows + fv.n_cand_rows;
     const FeatQ& q = s_fq[tid];
     quantise(q, fv.thr + q.thr0, s_pfeat[tid], false,
@@ -1219,16 +1256,35 @@ int fast_memo_batch(const GbdtModel& g, int P) {
 size_t fast_memo_bytes(const GbdtModel& g, int P, int C) {
   const int batch = fast_memo_batch(g, P);
   if (batch == 0 || C < 1) return 0;
-  return memo_fixed_bytes(C) + static_cast<size_t>(batch) * kMemoCap * pair_rec_bytes(g);
+  return memo_fixed_bytes(C) + static_cast<size_t>(batch) * (static_cast<size_t>(kMemoCap) * pair_rec_bytes(g) + kFastMaxProbRows);
 }
 
-// Slice count of the single-problem call: as many tree slices as keep every CTA in the first wave.
+// Slice count of the single-problem call: the trees are split over S CTAs per candidate block.
+// A CTA costs its tile fill (about 0.15 of a whole-ensemble walk of its block) plus 1 / S of that
+// walk, and blocks x S CTAs run in waves of the CTAs the machine holds at once: the S with the
+// shortest estimated makespan wins.
 int fast_slices(const GbdtModel& g, int64_t blocks) {
   if (blocks < 1) blocks = 1;
   if (blocks > kMaxSliceBlocks) return 1;
-  int64_t s = (g.ctas_per_sm * 148) / blocks;
-  if (s > g.n_chunks) s = g.n_chunks;
-  return static_cast<int>(s < 1 ? 1 : s);
+  const int64_t slots = static_cast<int64_t>(g.ctas_per_sm) * 148;
+  if (blocks >= slots) return 1;  // the machine is full without slices
+  int best = 1;
+  double best_cost = 1e30;
+  for (int s = 1; s <= g.n_chunks && s <= 32; ++s) {
+    const int64_t waves = (blocks * s + slots - 1) / slots;
+    const double cost = static_cast<double>(waves) * (0.15 + 1.0 / s);
+    if (cost < best_cost - 1e-9) {
+      best_cost = cost;
+      best = s;
+    }
+  }
+  return best;
+}
+
+size_t fast_prepared_rows_bytes(const GbdtModel& g, int C) { return static_cast<size_t>(kCombos) * C * cand_rec_bytes(g); }
+size_t fast_prepared_memo_bytes(const GbdtModel& g, int C) {
+  if (g.n_pair_rows < 1 || g.n_pair_rows > kFastMaxPairRec || C < 1) return 0;
+  return memo_fixed_bytes(C) + static_cast<size_t>(kMemoCap) * pair_rec_bytes(g) + kFastMaxProbRows;
 }
 
 namespace {
@@ -1249,6 +1305,7 @@ struct WalkArgs {
   SliceArgs sl;
   const FastTopParams* top;
   cudaStream_t stream;
+  int dependent;  // launched right behind the kernel whose tables it reads
 };
 
 template <int L, int NP, bool kCompact, int THREADS, int NC>
@@ -1257,10 +1314,21 @@ cudaError_t launch_ln(const WalkArgs& a) {
   auto kernel = &select_fast_kernel<L, NP, kCompact, THREADS, NC>;
   cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), smem);
   if (e != cudaSuccess) return e;
-  kernel<<<static_cast<unsigned>(static_cast<int64_t>(a.P) * a.nblk * a.sl.n_slices), THREADS, smem, a.stream>>>(
-      a.desc, a.d_p, a.pv, a.uv, a.d_c, a.P, a.C, a.nblk, a.rows_per_cta, a.seg_off, a.seg_idx, a.fv, a.k, a.partial,
-      a.status, a.sl, *a.top);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(static_cast<unsigned>(static_cast<int64_t>(a.P) * a.nblk * a.sl.n_slices));
+  cfg.blockDim = dim3(THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = a.stream;
+  // behind a table kernel the grid is launched as its programmatic dependent: its CTAs may start
+  // their set-up while that kernel still runs, and wait for it (griddepcontrol.wait) before they
+  // read its tables
+  cudaLaunchAttribute attr{};
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = a.dependent ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, a.desc, a.d_p, a.pv, a.uv, a.d_c, a.P, a.C, a.nblk, a.rows_per_cta,
+                            a.seg_off, a.seg_idx, a.fv, a.k, a.partial, a.status, a.sl, *a.top);
 }
 
 // the instantiation for a model's top levels and depth, within one tile geometry
@@ -1328,12 +1396,39 @@ int staged_floats(int count, size_t* bytes) {
 
 }  // namespace
 
+// Prepared catalogue: the candidate-only rows of every candidate under every element-type
+// combination, and the candidates' classes, computed once for a (catalogue, model) pair.
+cudaError_t fast_prepare(const ks_gpu_desc& desc, const GbdtModel& g, const ks_candidate* d_c, int C, void* d_rows,
+                         void* memo_mem, cudaStream_t stream, int64_t* launches) {
+  FastView fv = make_view(g, nullptr);
+  MemoView memo{};
+  if (memo_mem) memo = memo_view(memo_mem, C);
+  size_t cthr = 0;
+  const int cap = staged_floats(g.thr_prob0 - g.thr_cand0, &cthr);
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(&cand_rows_kernel), cthr);
+  if (e != cudaSuccess) return e;
+  if (memo.keys) {
+    e = memo_clear(memo, stream);
+    if (e != cudaSuccess) return e;
+  }
+  cand_rows_kernel<<<dim3((C + 255) / 256, kCombos), 256, cthr, stream>>>(desc, d_c, C, nullptr, 0xFFFFu, fv,
+                                                                          static_cast<uint8_t*>(d_rows), memo, cap);
+  ++*launches;
+  if (memo.keys) {
+    e = memo_compact(memo, stream);
+    if (e != cudaSuccess) return e;
+    ++*launches;
+  }
+  return cudaGetLastError();
+}
+
 cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, const ks_problem* d_p,
                                const ks_problem* p_by_value, int P, const ks_candidate* d_c, int C,
                                int nblk, int rows_per_cta, const int64_t* seg_off, const int32_t* seg_idx,
                                int k, unsigned long long* partial, void* scratch, int* status,
                                cudaStream_t stream, int64_t* launches, cudaEvent_t ev_begin,
-                               const FastSlice* slice, void* memo_mem, const FastWait* wait) {
+                               const FastSlice* slice, void* memo_mem, const FastWait* wait,
+                               const FastPrepared* prep) {
   WalkArgs a{};
   a.desc = desc;
   if (p_by_value) a.pv = *p_by_value;
@@ -1353,13 +1448,22 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
   uint8_t* d_rows = static_cast<uint8_t*>(scratch) + 256;
   fv.cand_rows = d_rows;
   MemoView memo{};
-  const int memo_batch = (memo_mem && !p_by_value && C > 0) ? fast_memo_batch(g, P) : 0;
+  int memo_batch = (memo_mem && !p_by_value && C > 0) ? fast_memo_batch(g, P) : 0;
   if (memo_batch > 0) memo = memo_view(memo_mem, C);
+  if (prep) {  // prepared catalogue: candidate-only rows and classes were made once, for every type combination
+    fv.cand_rows = prep->cand_rows;
+    if (prep->memo_mem) {
+      memo = memo_view(prep->memo_mem, C);
+      memo_batch = 1;
+    }
+  }
 
   // candidate-only rows for the type combinations in use
   cudaError_t e = cudaSuccess;
   unsigned mask_value = 0;
-  if (a.uv) {
+  if (prep) {
+    // nothing to do per call
+  } else if (a.uv) {
     mask_value = 1u << ((a.pv.dtype_ab & 3) * 4 + (a.pv.dtype_d & 3));
   } else {
     e = cudaMemsetAsync(d_mask, 0, sizeof(unsigned), stream);
@@ -1370,7 +1474,15 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
   const bool tiles_mode = a.uv && slice && slice->n_slices > 1 && slice->tiles && P == 1 && !seg_off;
   size_t pthr_bytes = 0;
   const int pthr_cap = staged_floats(g.thr_cand0, &pthr_bytes);
-  if (tiles_mode) {
+  if (prep) {
+    if (memo.keys) {
+      e = ensure_dynamic_smem(reinterpret_cast<const void*>(&pair_table_kernel), pthr_bytes);
+      if (e != cudaSuccess) return e;
+      fv.pair_class = memo.cls;
+      fv.pair_tab = static_cast<const uint8_t*>(memo.tab);
+      fv.prob_tab = fv.pair_tab + static_cast<size_t>(kMemoCap) * pair_rec_bytes(g);
+    }
+  } else if (tiles_mode) {
     // one launch, two roles (blockIdx.y): the per-pair rows, and the candidate- / problem-only rows
     size_t tthr = 0;
     const int cap = staged_floats(std::max(g.thr_cand0, g.n_qthr - g.thr_cand0), &tthr);
@@ -1399,6 +1511,7 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
       ++*launches;
       fv.pair_class = memo.cls;
       fv.pair_tab = static_cast<const uint8_t*>(memo.tab);
+      fv.prob_tab = fv.pair_tab + static_cast<size_t>(memo_batch) * kMemoCap * pair_rec_bytes(g);
     }
   }
   e = cudaGetLastError();
@@ -1422,10 +1535,11 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
   for (int first = 0; first < P; first += step) {
     const int n = P - first < step ? P - first : step;
     if (memo.keys) {
-      pair_table_kernel<<<dim3(kMemoCap / 256, n), 256, pthr_bytes, stream>>>(desc, d_p + first, d_c, fv, memo,
-                                                                              pthr_cap);
+      pair_table_kernel<<<dim3(kMemoCap / 256, n), 256, pthr_bytes, stream>>>(desc, d_p ? d_p + first : nullptr, a.pv, a.uv,
+                                                                              d_c, fv, memo, pthr_cap);
       ++*launches;
     }
+    a.dependent = memo.keys != nullptr;
     a.d_p = d_p ? d_p + first : nullptr;
     a.P = n;
     a.seg_off = seg_off ? seg_off + first : nullptr;

@@ -145,6 +145,19 @@ struct ks_ctx {
   cudaEvent_t ev_begin = nullptr, ev_end = nullptr;
 };
 
+// A candidate catalogue prepared for single-problem calls with one model (ks_catalogue_prepare).
+struct ks_catalogue {
+  ks_ctx* ctx = nullptr;
+  const ks_model* model = nullptr;
+  const ks_candidate* d_c = nullptr;
+  int C = 0;
+  int device = 0;
+  bool prepared = false;   // false: calls go through ks_select_one
+  int nblk = 0, slices = 1, max_k = KS_MAX_K;
+  void* d_mem = nullptr;   // one block: rows | memo | partial lists | partial-score planes
+  size_t off_memo = 0, off_part = 0, off_scores = 0;
+};
+
 struct ks_model {
   ks_ctx* ctx = nullptr;
   int device = 0;  // the context's device (kept here: the model may outlive the context)
@@ -200,6 +213,12 @@ struct FastSlice {
   int seq;
 };
 
+// What a prepared catalogue hands to the quantised tree kernel instead of per-call work.
+struct FastPrepared {
+  const uint8_t* cand_rows;  // [16 type combinations][C][record] candidate-only rows
+  void* memo_mem;            // class tables and ids of every combination + one problem's record table, or null
+};
+
 // Search-space enumeration and validity filtering (ks_catalogue.cu).
 cudaError_t launch_enumerate(long long first, long long count, ks_candidate* d_out, cudaStream_t stream,
                              int64_t* launches);
@@ -222,7 +241,12 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
                                int k, unsigned long long* partial, void* scratch, int* status,
                                cudaStream_t stream, int64_t* launches, cudaEvent_t ev_begin,
                                const FastSlice* slice = nullptr, void* memo_mem = nullptr,
-                               const FastWait* wait = nullptr);
+                               const FastWait* wait = nullptr, const FastPrepared* prep = nullptr);
+// Prepared catalogue (single-problem calls against a fixed catalogue and model).
+size_t fast_prepared_rows_bytes(const GbdtModel& g, int C);
+size_t fast_prepared_memo_bytes(const GbdtModel& g, int C);  // 0: the model's per-pair rows do not fit a record
+cudaError_t fast_prepare(const ks_gpu_desc& desc, const GbdtModel& g, const ks_candidate* d_c, int C, void* d_rows,
+                         void* memo_mem, cudaStream_t stream, int64_t* launches);
 int fast_slices(const GbdtModel& g, int64_t blocks);
 // ks_score with a qualifying ensemble: tiles quantised from the feature rows, then the same walk.
 size_t score_fast_scratch_bytes(const GbdtModel& g, int64_t rows);

@@ -54,7 +54,10 @@ def topk_accept(gpu_idx, gpu_score, oracle_scores_row, pool_idx_row, k, tol):
 
     Accepts iff no duplicates, every index is in the segment, every returned score matches the
     oracle's score of that candidate within tol, the j-th pick is as good as the oracle's j-th
-    up to tol, and among oracle-exact ties the indices ascend. Returns (ok, message)."""
+    up to tol, and among exact ties the indices ascend. An exact tie is one on both sides: two
+    candidates whose oracle scores are equal but whose returned scores differ (another order of
+    the fp32 additions moved one of them by an ulp) are a tie within the tolerance, which may
+    come out in either order. Returns (ok, message)."""
     n = len(oracle_scores_row)
     kk = min(k, n)
     order = np.lexsort((pool_idx_row, -oracle_scores_row.astype(np.float64)))
@@ -84,6 +87,6 @@ def topk_accept(gpu_idx, gpu_score, oracle_scores_row, pool_idx_row, k, tol):
         if j > 0:
             prev = int(gpu_idx[j - 1])
             rp = pos[prev] if pos is not None else int(np.searchsorted(pool_idx_row, prev))
-            if float(oracle_scores_row[rp]) == so and prev > gi:
+            if float(oracle_scores_row[rp]) == so and float(gpu_score[j - 1]) == float(gpu_score[j]) and prev > gi:
                 return False, f"rank {j}: tie not in ascending index order ({prev} before {gi})"
     return True, ""

@@ -95,7 +95,7 @@ def test_valid_catalogue_of_explicit_lists(ks, ctx):
 def test_valid_catalogue_rejects_bad_arguments(ks, ctx):
     p = problem(64, 64, 64, 0, 1, 1)
     with pytest.raises(ks.KsError) as ei:
-        ctx.valid_catalogue(p, 4)
+        ctx.valid_catalogue(p, 8)
     assert ei.value.status == ks.KS_ERR_INVALID_ARG
     with pytest.raises(ks.KsError):
         ctx.valid_catalogue(p, 1, None, C=SIZE + 1)

@@ -596,6 +596,50 @@ def test_select_forced_tile_geometry(ks, ctx, geometry, monkeypatch):
     assert np.array_equal(hi_.numpy(), idx[1])
 
 
+@pytest.mark.parametrize("law", ["slots128", "pernode"])
+def test_select_one_prepared_catalogue(ks, ctx, law):
+    """The single-problem call against a prepared catalogue (candidate-only rows and classes made
+    once per catalogue and model): every call must give the oracle's ranking and the same result
+    as the unprepared call; mixed element types use different slices of the prepared tables; a
+    model the quantised path does not serve goes through the plain call."""
+    w = wl.make_workload(3, P=12, C=7000, law=law)
+    probs = w.problems.copy()
+    probs["dtype_ab"][3:6] = [1, 2, 3]
+    probs["dtype_d"][3:6] = [1, 1, 3]
+    probs["epi_flags"][6:8] = [3, 4]
+    model = ctx.model_create_gbdt(*w.gbdt)
+    C = len(w.candidates)
+    d_c = dev(ks, w.candidates)
+    cat = ctx.catalogue_prepare(d_c, C, model)
+    n0 = ctx.launch_count()
+    hi, hs = ctx.select_one_prepared(cat, probs[:1], 10)
+    assert ctx.launch_count() - n0 == 2   # the per-class table of the problem, then the fused walk + top-k
+    for i in range(len(probs)):
+        hi, hs = ctx.select_one_prepared(cat, probs[i:i + 1], 10)
+        hi, hs = hi.numpy().copy(), hs.numpy().copy()
+        _, _, allsc = oracle.select(probs[i:i + 1], w.candidates, DESC, 10, gbdt=w.gbdt, want_scores=True)
+        ok, msg = topk_accept(hi, hs, allsc, np.arange(C, dtype=np.int32), 10, TOL_GBDT)
+        assert ok, f"problem {i}: {msg}"
+        pi, ps = ctx.select_one(probs[i:i + 1], d_c, C, model, 10)
+        assert np.array_equal(pi.numpy(), hi) and np.array_equal(ps.numpy(), hs)
+    call = ctx.select_one_caller(d_c, C, model, 10, catalogue=cat)
+    ci, cs = call(ks.problem_structs(probs[2:3])[0])
+    pi, ps = ctx.select_one(probs[2:3], d_c, C, model, 10)
+    assert np.array_equal(ci.numpy(), pi.numpy())
+    cat.close()
+    # other k, a tiny pool (a single block: no slices, plain call), and an MLP
+    small = ctx.catalogue_prepare(d_c, 40, model)
+    hi, hs = ctx.select_one_prepared(small, probs[:1], 32)
+    pi, ps = ctx.select_one(probs[:1], d_c, 40, model, 32)
+    assert np.array_equal(hi.numpy(), pi.numpy())
+    w4 = wl.make_workload(4, P=1, C=16)
+    mlp = ctx.model_create_mlp(w4.mlp)
+    mcat = ctx.catalogue_prepare(d_c, C, mlp)
+    hi, hs = ctx.select_one_prepared(mcat, probs[:1], 10)
+    pi, ps = ctx.select_one(probs[:1], d_c, C, mlp, 10)
+    assert np.array_equal(hi.numpy(), pi.numpy())
+
+
 def test_merge_topk_of_candidate_shares(ks, ctx):
     """The exchange step of the candidate-split form: three shares of a pool are ranked separately
     (per-share segments), their lists are concatenated as a gather would, and ks_merge_topk must
