@@ -567,7 +567,7 @@ __device__ __forceinline__ uint32_t path_step(uint32_t a, uint32_t cb_r, uint32_
 // (row offset, replicated j + 1) pair, so that twice as many trees keep their word-wise levels.
 // THREADS threads rank NC candidates: NC / 4 words times THREADS / (NC / 4) tree groups.
 template <int L, int NP, bool kCompact, int THREADS, int NC>
-__global__ void __launch_bounds__(THREADS, THREADS == 512 ? 2 : 1)
+__global__ void __launch_bounds__(THREADS, THREADS <= 512 ? 2 : 1)
 select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_problem p_value, int use_value,
                    const ks_candidate* __restrict__ c, int P, int C, int nblk, int rows_per_cta,
                    const int64_t* __restrict__ seg_off, const int32_t* __restrict__ seg_idx, FastView fv,
@@ -949,18 +949,22 @@ static std::vector<PartitionCode> partition_codes(int L) {
 
 // Tile geometry by the number of rows: the [row][candidate] tile and the two chunk buffers have to
 // fit the shared memory of one SM (228 KiB, 1 KiB of it reserved per CTA; a CTA's own limit is
-// 227 KiB including its static part). Two CTAs of 512 threads per SM are preferred, since one
-// CTA's tile fill and ranking then overlap the other's walk: with 1,024 candidates each up to 72
-// rows, with 512 candidates up to 149. Beyond that one CTA of 1,024 threads: 1,024 candidates up
-// to 183 rows, 512 candidates up to 367. Every CTA streams the whole ensemble, so a halved block
-// doubles that traffic. More rows than that: the general kernel. A single CTA per SM takes
-// 32 KB chunk buffers when they fit. KS_FAST_GEOMETRY="threads,candidates,buffer KiB" overrides
-// the choice (a tuning aid; a geometry that does not fit is refused).
+// 227 KiB including its static part). Measured on one ensemble: what matters is (i) two CTAs per
+// SM, so that one CTA's tile fill and ranking overlap the other's walk (15 %), and (ii) four trees
+// or more per thread and chunk, which the compiler interleaves (13 %); sixteen walking warps per
+// SM already saturate the walk. Hence, in order of preference: two CTAs of 512 threads x 1,024
+// candidates (up to 72 rows), two CTAs of 256 threads x 512 candidates (up to 149 rows), then one
+// CTA of 512 threads with 1,024 candidates (up to 183 rows) or 512 candidates (up to 376 rows),
+// with 32 KB chunk buffers where they fit. Every CTA streams the whole ensemble, so a halved block
+// doubles that traffic (two CTAs of 256 threads x 256 candidates measured slower than one CTA of
+// 512 x 512). More rows than that: the general kernel.
+// KS_FAST_GEOMETRY="threads,candidates,buffer KiB" overrides the choice (a tuning aid; a geometry
+// that does not fit is refused).
 struct Geometry {
   int threads, cands, buf_bytes, ctas_per_sm;
 };
 static size_t geometry_smem(const Geometry& g, int n_rows) {
-  const size_t stat = g.threads == 512 ? 6656 + 256 : 10752 + 256;  // static shared memory of the kernel, with slack
+  const size_t stat = 2560 + static_cast<size_t>(g.threads) / 32 * KS_MAX_K * 8 + 256;  // static shared memory of the kernel, with slack
   return static_cast<size_t>(kNBuf) * g.buf_bytes + static_cast<size_t>(n_rows) * g.cands + stat;
 }
 static bool geometry_fits(const Geometry& g, int n_rows) {
@@ -968,12 +972,12 @@ static bool geometry_fits(const Geometry& g, int n_rows) {
   if (per_cta > 227 * 1024) return false;
   return g.ctas_per_sm * (per_cta + 1024) <= 228 * 1024;
 }
+static bool geometry_known(int t, int c) { return (t == 512 && c == 1024) || (t == 256 && c == 512) || (t == 512 && c == 512); }
 static bool pick_geometry(int n_rows, Geometry* out) {
   if (const char* env = std::getenv("KS_FAST_GEOMETRY")) {
     int t = 0, c = 0, kb = 0;
-    if (std::sscanf(env, "%d,%d,%d", &t, &c, &kb) == 3 && (t == 512 || t == 1024) && (c == 512 || c == 1024) &&
-        (kb == 16 || kb == 32)) {
-      Geometry g{t, c, kb * 1024, t == 512 ? 2 : 1};
+    if (std::sscanf(env, "%d,%d,%d", &t, &c, &kb) == 3 && geometry_known(t, c) && (kb == 16 || kb == 32)) {
+      Geometry g{t, c, kb * 1024, 2};
       if (!geometry_fits(g, n_rows)) g.ctas_per_sm = 1;
       if (geometry_fits(g, n_rows)) {
         *out = g;
@@ -981,8 +985,8 @@ static bool pick_geometry(int n_rows, Geometry* out) {
       }
     }
   }
-  const Geometry order[] = {{512, 1024, kBufBytes, 2},      {512, 512, kBufBytes, 2},  {1024, 1024, 2 * kBufBytes, 1},
-                            {1024, 1024, kBufBytes, 1},     {1024, 512, 2 * kBufBytes, 1}, {1024, 512, kBufBytes, 1}};
+  const Geometry order[] = {{512, 1024, kBufBytes, 2},     {256, 512, kBufBytes, 2}, {512, 1024, 2 * kBufBytes, 1},
+                            {512, 1024, kBufBytes, 1},     {512, 512, 2 * kBufBytes, 1}, {512, 512, kBufBytes, 1}};
   for (const Geometry& g : order)
     if (geometry_fits(g, n_rows)) {
       *out = g;
@@ -1356,8 +1360,7 @@ cudaError_t launch_walk_geom(const GbdtModel& g, const WalkArgs& a) {
 cudaError_t launch_walk(const GbdtModel& g, const WalkArgs& a) {
   if (g.fast_threads == 512 && g.block_cands == 1024) return launch_walk_geom<512, 1024>(g, a);
   if (g.fast_threads == 512) return launch_walk_geom<512, 512>(g, a);
-  if (g.block_cands == 1024) return launch_walk_geom<1024, 1024>(g, a);
-  return launch_walk_geom<1024, 512>(g, a);
+  return launch_walk_geom<256, 512>(g, a);
 }
 
 FastView make_view(const GbdtModel& g, const FastWait* wait) {

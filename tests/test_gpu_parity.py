@@ -535,8 +535,8 @@ def test_select_other_model_shapes(ks, ctx, case):
 def test_select_tile_geometries(ks, ctx, case):
     """The quantised kernel's tile geometries, picked by the number of rows: the slot-table
     ensemble (<= 72 rows: two CTAs of 512 threads x 1,024 candidates per SM), the 256-bin and the
-    quantile-per-node ensembles of config 1 (<= 149 rows: two CTAs of 512 threads x 512
-    candidates), the quantile-per-node ensemble of config 2 (<= 367 rows: one CTA of 1,024 threads x
+    quantile-per-node ensembles of config 1 (<= 149 rows: two CTAs of 256 threads x 512
+    candidates), the quantile-per-node ensemble of config 2 (<= 376 rows: one CTA of 512 threads x
     512 candidates), and an ensemble with a continuous threshold at every node of 3,000 trees (more
     rows than any geometry holds: the general kernel). Each: a batch (ks_select), the single-problem call (tree slices
     over prepared tiles), the scoring call on given feature rows, and a batch of 33 problems or
@@ -550,11 +550,11 @@ def test_select_tile_geometries(ks, ctx, case):
         want = "select_generic_kernel"
     elif case == "cfg2_pernode":
         w = wl.make_workload(2, P=6, seg=2500, law="pernode")
-        want = "threads=1024 block=512"
+        want = "threads=512 block=512"
     else:
         law = case.split("_")[1]
         w = wl.make_workload(1, P=5, C=3000, law=law)
-        want = "threads=512 block=1024" if law == "slots128" else "threads=512 block=512"
+        want = "threads=512 block=1024" if law == "slots128" else "threads=256 block=512"
     model = ctx.model_create_gbdt(*w.gbdt)
     assert want in model.describe(), model.describe()
     idx, sc = run_select(ks, ctx, w, model)
@@ -581,7 +581,7 @@ def test_select_tile_geometries(ks, ctx, case):
     check_select(wm, idx, sc, TOL_GBDT, sample=range(0, 40, 3))
 
 
-@pytest.mark.parametrize("geometry", ["1024,1024,32", "1024,1024,16", "1024,512,32", "512,512,16"])
+@pytest.mark.parametrize("geometry", ["512,1024,32", "512,1024,16", "512,512,32", "512,512,16", "256,512,16"])
 def test_select_forced_tile_geometry(ks, ctx, geometry, monkeypatch):
     """Every tile geometry on the same ensemble (config 1, a quantile per node, 143 rows), forced
     through KS_FAST_GEOMETRY = threads, candidates per CTA, chunk-buffer KiB."""
