@@ -628,12 +628,12 @@ def main():
         dist.destroy_process_group()
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel, per launch, from the
-# ncu summaries under profiles/ (None until a capture exists for that workload). Config 1: the
-# 48-problem capture (17.6 MB) splits into 7.4 MB that do not depend on the number of problems
-# and 0.21 MB per problem (the problem's table of per-pair tile rows, read back through L2),
-# plus the partial lists of the full-size launch (9.7 MB): 7.4 + 1,024 x 0.21 + 9.7.
-TRAFFIC_BYTES = {(1, "slots128"): 234e6, (4, None): 5.7e6}
+# dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel per full-size step, from the
+# ncu captures of the 48-problem case under profiles/, scaled by the problems (None: no capture
+# for that workload). Config 1, per-node law: 15.4 MB read in the small case (catalogue, model,
+# per-call tables, the class records of 48 problems) + 0.24 MB of class records per further
+# problem (written by the table kernel, read once) + 9.7 MB of partial lists written.
+TRAFFIC_BYTES = {(1, "pernode"): 260e6, (1, "slots128"): 234e6, (4, None): 5.7e6}
 
 if __name__ == "__main__":
     main()
