@@ -277,61 +277,78 @@ memo_compact_kernel(MemoView memo) {
   if (threadIdx.x == 0) memo.count[combo] = s_n;
 }
 
-// Per problem: the tile bytes of the per-pair rows of every class, from the class's member.
-// grid (kMemoCap / 256, batch of problems); blocks past the number of classes leave at once.
-// `p` points at the batch's first problem, and record (problem within the batch, slot) is written.
+// Per problem: the tile bytes of the per-pair rows of every class, from the class's member, plus
+// (last block of a row) the problem's own terms and the tile bytes of its problem-only rows.
+// grid (kMemoCap / 256, problem lanes): block (x, y) serves classes 256 x .. 256 x + 255 of the
+// problems y, y + gridDim.y, ... of the batch, so the thresholds are staged once per block.
+// `p` points at the batch's first problem; record (problem within the batch, slot) is written.
+// Dynamic shared memory: the staged thresholds (thr_cap floats), then 256 records.
+constexpr int kProbRec = kFastMaxProbRows + 128;  // problem-only rows, then the ProblemTerms
+static_assert(sizeof(ProblemTerms) <= 128, "problem record");
+
 __global__ void __launch_bounds__(256)
-pair_table_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_problem p_value, int use_value,
+pair_table_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_problem p_value, int use_value, int n_prob,
                   const ks_candidate* __restrict__ c, FastView fv, MemoView memo, int thr_cap) {
-  extern __shared__ float s_pthr[];  // thresholds of the per-pair features
+  extern __shared__ __align__(16) float s_pthr[];  // thresholds of the per-pair features, then the records
   __shared__ ProblemTerms s_pt;
   __shared__ FeatQ s_fq[64];
-  const int prob = blockIdx.y, j = blockIdx.x * 256 + threadIdx.x;
+  __shared__ float s_pf[64];
+  const int tid = threadIdx.x, j = blockIdx.x * 256 + tid;
+  const bool last_x = blockIdx.x == gridDim.x - 1;
   // the select kernel that follows may start its own set-up now (it waits for this grid to finish
   // before it reads the tables)
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  const ks_problem pr = use_value ? p_value : load_problem(p + prob);
-  const int combo = (pr.dtype_ab & 3) * 4 + (pr.dtype_d & 3);
-  if (blockIdx.x == 0 && prob == 0 && threadIdx.x == 0) g_fast_abort = 0;  // (also) precedes the select kernel
-  const int n_classes = memo.count[combo];
-  if (blockIdx.x * 256 >= n_classes && blockIdx.x != gridDim.x - 1) return;
-  if (blockIdx.x == gridDim.x - 1) {
-    // the last block of the row: the problem-only rows of this problem, once for all its CTAs
-    __shared__ ProblemTerms s_pt0;
-    __shared__ float s_pf[64];
-    if (threadIdx.x == 0) {
-      problem_terms(pr, desc, s_pt0);
-      ks_candidate dummy{};
-      dummy.tile_m = dummy.tile_n = dummy.tile_k = 64;
-      dummy.stages = dummy.cluster_m = dummy.cluster_n = 1;
-      featurize_pair(s_pt0, dummy, desc, [&](int col, float v) {
-        if (col < KS_F && feat_class(col) == 0) s_pf[col] = v;
-      });
-    }
-    __syncthreads();
-    if (threadIdx.x < KS_F && feat_class(threadIdx.x) == 0) {
-      const FeatQ q = fv.feat[threadIdx.x];
-      const int first = fv.n_pair_rows + fv.n_cand_rows;
-      uint8_t* out = const_cast<uint8_t*>(fv.prob_tab) + static_cast<size_t>(prob) * kFastMaxProbRows;
-      quantise(q, fv.thr + q.thr0, s_pf[threadIdx.x], false,
-               [&](int row, uint8_t b) { out[KS_IDX(row - first, kFastMaxProbRows)] = b; });
-    }
-    if (blockIdx.x * 256 >= n_classes) return;
-    __syncthreads();
-  }
-  const int slot = j < n_classes ? memo.dense[static_cast<size_t>(combo) * kMemoCap + j] : 0;
+  if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) g_fast_abort = 0;  // (also) precedes the select kernel
+  int most = 0;
+  for (int q = 0; q < kMemoCombos; ++q) most = max(most, memo.count[q]);
+  if (blockIdx.x * 256 >= most && !last_x) return;
   const float* T = stage_thresholds(fv, 0, fv.thr_cand0, s_pthr, thr_cap);
-  if (threadIdx.x < 64) s_fq[threadIdx.x] = fv.feat[threadIdx.x];
-  if (threadIdx.x == 0) problem_terms(pr, desc, s_pt);
-  __syncthreads();
-  if (j >= n_classes) return;
-  const ks_candidate cand = load_candidate(c + memo.reps[static_cast<size_t>(combo) * kMemoCap + slot]);
-  const long long b_eff = resources(s_pt, cand, desc).b_eff;
-  uint8_t* rec = static_cast<uint8_t*>(memo.tab) + (static_cast<size_t>(prob) * kMemoCap + slot) * fv.pair_rec;
-  pair_columns<true>(s_pt, cand, desc, b_eff, [&](int col, float v) {
-    const FeatQ& q = s_fq[col];
-    quantise(q, T + q.thr0, v, false, [&](int row, uint8_t b) { rec[KS_IDX(row, fv.pair_rec)] = b; });
-  });
+  uint8_t* my_rec = reinterpret_cast<uint8_t*>(s_pthr + (thr_cap > 0 ? (thr_cap + 3) / 4 * 4 : 0)) +
+                    static_cast<size_t>(tid) * fv.pair_rec;
+  if (tid < 64) s_fq[tid] = fv.feat[tid];
+  for (int prob = blockIdx.y; prob < n_prob; prob += gridDim.y) {
+    const ks_problem pr = use_value ? p_value : load_problem(p + prob);
+    const int combo = (pr.dtype_ab & 3) * 4 + (pr.dtype_d & 3);
+    const int n_classes = memo.count[combo];
+    __syncthreads();  // the previous problem's terms are no longer read (and the staging is complete)
+    if (tid == 0) {
+      problem_terms(pr, desc, s_pt);
+      if (last_x) {
+        ks_candidate dummy{};
+        dummy.tile_m = dummy.tile_n = dummy.tile_k = 64;
+        dummy.stages = dummy.cluster_m = dummy.cluster_n = 1;
+        featurize_pair(s_pt, dummy, desc, [&](int col, float v) {
+          if (col < KS_F && feat_class(col) == 0) s_pf[col] = v;
+        });
+      }
+    }
+    __syncthreads();
+    if (last_x) {
+      // once per problem, for all its CTAs: the problem-only rows and the problem's terms
+      uint8_t* out = const_cast<uint8_t*>(fv.prob_tab) + static_cast<size_t>(prob) * kProbRec;
+      if (tid < KS_F && feat_class(tid) == 0) {
+        const FeatQ& q = s_fq[tid];
+        const int first = fv.n_pair_rows + fv.n_cand_rows;
+        quantise(q, fv.thr + q.thr0, s_pf[tid], false,
+                 [&](int row, uint8_t b) { out[KS_IDX(row - first, kFastMaxProbRows)] = b; });
+      }
+      if (tid < static_cast<int>(sizeof(ProblemTerms) / 4))
+        reinterpret_cast<uint32_t*>(out + kFastMaxProbRows)[tid] = reinterpret_cast<const uint32_t*>(&s_pt)[tid];
+    }
+    if (j >= n_classes) continue;
+    const int slot = memo.dense[static_cast<size_t>(combo) * kMemoCap + j];
+    const ks_candidate cand = load_candidate(c + memo.reps[static_cast<size_t>(combo) * kMemoCap + slot]);
+    const long long b_eff = resources(s_pt, cand, desc).b_eff;
+    pair_columns<true>(s_pt, cand, desc, b_eff, [&](int col, float v) {
+      const FeatQ& q = s_fq[col];
+      quantise(q, T + q.thr0, v, false, [&](int row, uint8_t b) { my_rec[KS_IDX(row, fv.pair_rec)] = b; });
+    });
+    // the record leaves as whole 16-byte words (it is a multiple of 16 bytes, and so is its place)
+    uint4* dst = reinterpret_cast<uint4*>(static_cast<uint8_t*>(memo.tab) +
+                                          (static_cast<size_t>(prob) * kMemoCap + slot) * fv.pair_rec);
+    const uint4* src = reinterpret_cast<const uint4*>(my_rec);
+    for (int q = 0; q < fv.pair_rec / 16; ++q) dst[q] = src[q];
+  }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -493,6 +510,8 @@ __device__ __noinline__ void fill_tile(const ks_gpu_desc& desc, const ProblemTer
       continue;
     }
     const int ci = seg_off ? seg_idx[lo + row] : static_cast<int>(row);
+    // the candidate's class, fetched before the other loads that depend on ci only
+    const unsigned cid = fv.pair_class ? __ldg(fv.pair_class + static_cast<size_t>(combo) * C + ci) : kNoClass;
     // candidate-only rows
     scatter_record(fv.cand_rows + (static_cast<size_t>(combo) * C + KS_IDX(ci, C)) * fv.cand_rec, fv.n_cand_rows,
                    my + fv.n_pair_rows * NC, NC);
@@ -501,7 +520,6 @@ __device__ __noinline__ void fill_tile(const ks_gpu_desc& desc, const ProblemTer
     for (int q = 0; q < fv.n_prob_rows; ++q) dst[q * NC] = s_pbin[q];
     // per-pair rows: the record of the candidate's class, when there is one
     if (fv.pair_class) {
-      const unsigned cid = __ldg(fv.pair_class + static_cast<size_t>(combo) * C + ci);
       if (cid != kNoClass) {
         scatter_record(fv.pair_tab + (static_cast<size_t>(prob) * kMemoCap + KS_IDX(cid, kMemoCap)) * fv.pair_rec,
                        fv.n_pair_rows, my, NC);
@@ -605,9 +623,9 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
   const uint32_t bar0 = smem_u32(&s_bar[0]);  // barrier of buffer b: bar0 + 8 b
   const bool tiles_given = sl.tiles != nullptr;  // the tiles were built in front: no feature work here
   if (tid == 0) {
-    if (!tiles_given) {
+    if (!tiles_given && !fv.prob_tab) {
       problem_terms(use_value ? p_value : load_problem(p + prob), desc, s_pt);
-      if (!fv.prob_tab) {
+      {
         // problem-only columns do not look at the candidate: evaluate them on a dummy one
         ks_candidate dummy{};
         dummy.tile_m = dummy.tile_n = dummy.tile_k = 64;
@@ -635,8 +653,10 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
     return;
   }
   if (!tiles_given && fv.prob_tab) {
-    for (int i = tid; i < fv.n_prob_rows; i += THREADS)
-      s_pbin[i] = __ldcg(fv.prob_tab + static_cast<size_t>(prob) * kFastMaxProbRows + i);
+    const uint8_t* rec = fv.prob_tab + static_cast<size_t>(prob) * kProbRec;
+    for (int i = tid; i < fv.n_prob_rows; i += THREADS) s_pbin[i] = __ldcg(rec + i);
+    if (tid < static_cast<int>(sizeof(ProblemTerms) / 4))
+      reinterpret_cast<uint32_t*>(&s_pt)[tid] = __ldcg(reinterpret_cast<const uint32_t*>(rec + kFastMaxProbRows) + tid);
   } else if (!tiles_given && tid < KS_F && feat_class(tid) == 0) {
     const int first = fv.n_pair_rows + fv.n_cand_rows;
     const FeatQ& q = s_fq[tid];
@@ -1260,7 +1280,7 @@ int fast_memo_batch(const GbdtModel& g, int P) {
 size_t fast_memo_bytes(const GbdtModel& g, int P, int C) {
   const int batch = fast_memo_batch(g, P);
   if (batch == 0 || C < 1) return 0;
-  return memo_fixed_bytes(C) + static_cast<size_t>(batch) * (static_cast<size_t>(kMemoCap) * pair_rec_bytes(g) + kFastMaxProbRows);
+  return memo_fixed_bytes(C) + static_cast<size_t>(batch) * (static_cast<size_t>(kMemoCap) * pair_rec_bytes(g) + kProbRec);
 }
 
 // Slice count of the single-problem call: the trees are split over S CTAs per candidate block.
@@ -1288,7 +1308,7 @@ int fast_slices(const GbdtModel& g, int64_t blocks) {
 size_t fast_prepared_rows_bytes(const GbdtModel& g, int C) { return static_cast<size_t>(kCombos) * C * cand_rec_bytes(g); }
 size_t fast_prepared_memo_bytes(const GbdtModel& g, int C) {
   if (g.n_pair_rows < 1 || g.n_pair_rows > kFastMaxPairRec || C < 1) return 0;
-  return memo_fixed_bytes(C) + static_cast<size_t>(kMemoCap) * pair_rec_bytes(g) + kFastMaxProbRows;
+  return memo_fixed_bytes(C) + static_cast<size_t>(kMemoCap) * pair_rec_bytes(g) + kProbRec;
 }
 
 namespace {
@@ -1475,8 +1495,18 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
     ++*launches;
   }
   const bool tiles_mode = a.uv && slice && slice->n_slices > 1 && slice->tiles && P == 1 && !seg_off;
+  // shared memory of the table kernel: the per-pair thresholds when they fit beside its 256 records
   size_t pthr_bytes = 0;
-  const int pthr_cap = staged_floats(g.thr_cand0, &pthr_bytes);
+  int pthr_cap = staged_floats(g.thr_cand0, &pthr_bytes);
+  {
+    const size_t rec_bytes = static_cast<size_t>(256) * pair_rec_bytes(g);
+    size_t thr_part = pthr_cap > 0 ? static_cast<size_t>((pthr_cap + 3) / 4 * 4) * sizeof(float) : 0;
+    if (thr_part + rec_bytes > 200 * 1024) {
+      pthr_cap = 0;
+      thr_part = 0;
+    }
+    pthr_bytes = thr_part + rec_bytes + 16;
+  }
   if (prep) {
     if (memo.keys) {
       e = ensure_dynamic_smem(reinterpret_cast<const void*>(&pair_table_kernel), pthr_bytes);
@@ -1538,8 +1568,8 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
   for (int first = 0; first < P; first += step) {
     const int n = P - first < step ? P - first : step;
     if (memo.keys) {
-      pair_table_kernel<<<dim3(kMemoCap / 256, n), 256, pthr_bytes, stream>>>(desc, d_p ? d_p + first : nullptr, a.pv, a.uv,
-                                                                              d_c, fv, memo, pthr_cap);
+      pair_table_kernel<<<dim3(kMemoCap / 256, n < 32 ? n : 32), 256, pthr_bytes, stream>>>(
+          desc, d_p ? d_p + first : nullptr, a.pv, a.uv, n, d_c, fv, memo, pthr_cap);
       ++*launches;
     }
     a.dependent = memo.keys != nullptr;
