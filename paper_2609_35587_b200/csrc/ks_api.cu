@@ -691,10 +691,15 @@ ks_status ks_catalogue_prepare(ks_ctx* ctx, const ks_candidate* d_c, int C, cons
       cat->off_memo = b_rows;
       cat->off_part = b_rows + align_up(b_memo);
       cat->off_scores = cat->off_part + b_part;
-      cudaError_t e = cudaMalloc(&cat->d_mem, cat->off_scores + b_scores);
+      cat->off_order = cat->off_scores + b_scores;
+      cudaError_t e = cudaMalloc(&cat->d_mem, cat->off_order + ks::order_scratch_bytes(C));
       if (e == cudaSuccess)
         e = ks::fast_prepare(ctx->desc, g, d_c, C, cat->d_mem, static_cast<char*>(cat->d_mem) + cat->off_memo,
                              static_cast<cudaStream_t>(stream), &ctx->launches);
+      // the catalogue is ranked in similarity order (neighbouring candidates take similar paths)
+      if (e == cudaSuccess)
+        e = ks::launch_catalogue_order(d_c, C, static_cast<char*>(cat->d_mem) + cat->off_order,
+                                       static_cast<cudaStream_t>(stream), &ctx->launches);
       if (e == cudaSuccess) e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
       if (e != cudaSuccess) {
         cudaFree(cat->d_mem);
@@ -747,7 +752,7 @@ ks_status ks_select_one_prepared(ks_ctx* ctx, const ks_catalogue* cat, ks_proble
   cudaError_t e = ks::launch_select_fast(ctx->desc, gm, nullptr, &p, 1, cat->d_c, cat->C, cat->nblk, gm.block_cands,
                                          nullptr, nullptr, k, reinterpret_cast<unsigned long long*>(base + cat->off_part),
                                          nullptr, ctx->d_status, st, &ctx->launches, nullptr, &sl, nullptr, &ctx->wait,
-                                         &prep);
+                                         &prep, reinterpret_cast<const int32_t*>(base + cat->off_order));
   if (e == cudaSuccess) {
     bool seen = false;
     for (int spin = 0; spin < (1 << 22) && !seen; ++spin) seen = *static_cast<volatile int*>(h_seq) == sl.seq;

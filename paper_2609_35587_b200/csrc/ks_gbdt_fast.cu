@@ -169,9 +169,10 @@ __device__ __forceinline__ void quantise(const FeatQ& q, const float* T, float v
   }
 }
 
-// Byte of candidate i (0 .. 4 W - 1) of a block within one tile row of W words: the four
-// candidates of a word are i, i + W, i + 2 W, i + 3 W.
-__device__ __forceinline__ int tile_byte(int i, int W) { return (i % W) * 4 + i / W; }
+// Byte of row i (0 .. 4 W - 1) of a block within one tile row of W words: the four rows of a
+// word are consecutive, so that in a catalogue ranked in similarity order a thread's four
+// candidates are near-duplicates.
+__device__ __forceinline__ int tile_byte(int i, int) { return i; }
 
 // Slice mode (single-problem latency call): the trees are split over n_slices CTAs per
 // candidate block. Every CTA stores its partial scores; the last CTA to arrive for a block
@@ -204,7 +205,7 @@ struct FastView {
   const uint8_t* cand_rows;    // [kCombos][C][cand_rec] quantised candidate-only rows
   const unsigned* pair_class;  // [kCombos][C] class of every candidate, or null (no memo)
   const uint8_t* pair_tab;     // [P][kMemoCap][pair_rec] per-pair tile bytes of every (problem, class)
-  const uint8_t* prob_tab;     // [P][kFastMaxProbRows] tile bytes of the problem-only rows, or null
+  const uint8_t* prob_tab;     // [P][kProbRec] tile bytes of the problem-only rows and the problem's terms, or null
 };
 
 // ------------------------------------------------------------------------------------------
@@ -421,13 +422,13 @@ tile_rows_kernel(const float* __restrict__ feat, int64_t rows, FastView fv, uint
   const float* T = stage_thresholds(fv, 0, fv.n_thr, s_thr, thr_cap);
   if (word < 64) s_fq[word] = fv.feat[word];
   __syncthreads();
-  // byte b of the word is row b W + word of the block
+  // byte b of the word is row 4 word + b of the block
   const int64_t base = static_cast<int64_t>(blockIdx.x) * NC;
   const float4* src[4];
   bool live[4];
 #pragma unroll
   for (int b = 0; b < 4; ++b) {
-    const int64_t slot = base + b * W + word;
+    const int64_t slot = base + 4 * word + b;
     live[b] = slot < rows;
     src[b] = reinterpret_cast<const float4*>(feat + (live[b] ? slot : 0) * KS_F_PAD);
   }
@@ -509,7 +510,7 @@ __device__ __noinline__ void fill_tile(const ks_gpu_desc& desc, const ProblemTer
       for (int q = 0; q < fv.n_rows; ++q) my[q * NC] = 0x80;
       continue;
     }
-    const int ci = seg_off ? seg_idx[lo + row] : static_cast<int>(row);
+    const int ci = seg_idx ? seg_idx[lo + row] : static_cast<int>(row);
     // the candidate's class, fetched before the other loads that depend on ci only
     const unsigned cid = fv.pair_class ? __ldg(fv.pair_class + static_cast<size_t>(combo) * C + ci) : kNoClass;
     // candidate-only rows
@@ -608,12 +609,16 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
   const int kOffTile = kNBuf * fv.buf_bytes;
   const int S = sl.n_slices;
   const int prob = blockIdx.x / (nblk * S), chunk = (blockIdx.x / S) % nblk, slice = blockIdx.x % S;
-  int64_t lo, len;
+  // rows of this problem: lo = where its scores sit in per-row arrays; lo_idx = where its pool
+  // indices start in seg_idx (per-problem segments, or - without offsets - one ranking order of
+  // the whole catalogue shared by every problem)
+  int64_t lo, len, lo_idx;
   if (seg_off) {
-    lo = seg_off[prob];
+    lo = lo_idx = seg_off[prob];
     len = seg_off[prob + 1] - lo;
   } else {
     lo = static_cast<int64_t>(prob) * C;
+    lo_idx = 0;
     len = C;
   }
   // chunks of the ensemble this CTA walks
@@ -682,7 +687,7 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
       const float* T = stage_thresholds(fv, 0, fv.thr_cand0, reinterpret_cast<float*>(smem + kOffBuf0),
                                         fv.pair_class ? 0 : kNBuf * fv.buf_bytes / 4);
       __syncthreads();
-      fill_tile<THREADS, NC>(desc, s_pt, c, fv, seg_off, seg_idx, C, lo, start, stop, T, s_fq, s_pbin,
+      fill_tile<THREADS, NC>(desc, s_pt, c, fv, seg_off, seg_idx, C, lo_idx, start, stop, T, s_fq, s_pbin,
                              smem + kOffTile, prob);
     }
     __syncthreads();  // tile complete; the threshold table is no longer needed
@@ -852,7 +857,7 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
       // scoring call: the scores are the result (same order of additions as the ranking path)
 #pragma unroll
       for (int r = 0; r < 4; ++r) {
-        const int64_t row = start + r * W + word;
+        const int64_t row = start + 4 * word + r;
         if (grp == 0 && row < stop) sl.score_out[lo + row] = (fv.base + total[r]) + 0.0f;
       }
       continue;
@@ -861,7 +866,7 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
       // slice mode: publish this CTA's partial scores, let the last arrival finish the block
 #pragma unroll
       for (int r = 0; r < 4; ++r) {
-        const int64_t row = start + r * W + word;
+        const int64_t row = start + 4 * word + r;
         if (grp == 0 && row < stop) __stcg(sl.scores + static_cast<size_t>(slice) * sl.pairs + lo + row, total[r]);
       }
       __threadfence();
@@ -879,8 +884,8 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
       keys[r] = 0ull;
-      // byte r of word `word` is row r W + word of the block
-      const int64_t row = start + r * W + word;
+      // byte r of word `word` is row 4 word + r of the block
+      const int64_t row = start + 4 * word + r;
       if (grp == 0 && row < stop) {
         float s;
         if (S > 1) {
@@ -889,7 +894,7 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
         } else {
           s = fv.base + total[r];
         }
-        keys[r] = make_key(s + 0.0f, seg_off ? seg_idx[lo + row] : static_cast<int>(row));
+        keys[r] = make_key(s + 0.0f, seg_idx ? seg_idx[lo_idx + row] : static_cast<int>(row));
       }
     }
     keys[4] = tid < k ? s_list[tid] : 0ull;
@@ -972,12 +977,16 @@ static std::vector<PartitionCode> partition_codes(int L) {
 // 227 KiB including its static part). Measured on one ensemble: what matters is (i) two CTAs per
 // SM, so that one CTA's tile fill and ranking overlap the other's walk (15 %), and (ii) four trees
 // or more per thread and chunk, which the compiler interleaves (13 %); sixteen walking warps per
-// SM already saturate the walk. Hence, in order of preference: two CTAs of 512 threads x 1,024
-// candidates (up to 72 rows), two CTAs of 256 threads x 512 candidates (up to 149 rows), then one
-// CTA of 512 threads with 1,024 candidates (up to 183 rows) or 512 candidates (up to 376 rows),
-// with 32 KB chunk buffers where they fit. Every CTA streams the whole ensemble, so a halved block
-// doubles that traffic (two CTAs of 256 threads x 256 candidates measured slower than one CTA of
-// 512 x 512). More rows than that: the general kernel.
+// SM already saturate the walk, eight do not. Hence, in order of preference: two CTAs of 256
+// threads x 1,024 candidates (eight trees per thread and chunk, up to 128 registers per thread;
+// up to 74 rows), two CTAs of 256 threads x 512 candidates (up to 149 rows), then one CTA of 512
+// threads with 1,024 candidates (up to 183 rows) or 512 candidates (up to 376 rows), with 32 KB
+// chunk buffers where they fit. Every CTA streams the whole ensemble, so a halved block doubles
+// that traffic (two CTAs of 256 threads x 256 candidates measured slower than one CTA of
+// 512 x 512; two CTAs of 128 x 512 and one CTA of 256 x 1,024 have too few warps). Two CTAs of
+// 512 threads x 1,024 candidates (64 registers per thread) measured 54 to 63 ms on the same
+// ensemble depending on how unrelated code around the loop happened to be compiled; the
+// 256-thread form, 51.6 ms, does not depend on that. More rows than 376: the general kernel.
 // KS_FAST_GEOMETRY="threads,candidates,buffer KiB" overrides the choice (a tuning aid; a geometry
 // that does not fit is refused).
 struct Geometry {
@@ -992,7 +1001,9 @@ static bool geometry_fits(const Geometry& g, int n_rows) {
   if (per_cta > 227 * 1024) return false;
   return g.ctas_per_sm * (per_cta + 1024) <= 228 * 1024;
 }
-static bool geometry_known(int t, int c) { return (t == 512 && c == 1024) || (t == 256 && c == 512) || (t == 512 && c == 512); }
+static bool geometry_known(int t, int c) {
+  return (t == 512 && c == 1024) || (t == 256 && c == 512) || (t == 512 && c == 512) || (t == 256 && c == 1024);
+}
 static bool pick_geometry(int n_rows, Geometry* out) {
   if (const char* env = std::getenv("KS_FAST_GEOMETRY")) {
     int t = 0, c = 0, kb = 0;
@@ -1005,7 +1016,7 @@ static bool pick_geometry(int n_rows, Geometry* out) {
       }
     }
   }
-  const Geometry order[] = {{512, 1024, kBufBytes, 2},     {256, 512, kBufBytes, 2}, {512, 1024, 2 * kBufBytes, 1},
+  const Geometry order[] = {{256, 1024, kBufBytes, 2},     {256, 512, kBufBytes, 2}, {512, 1024, 2 * kBufBytes, 1},
                             {512, 1024, kBufBytes, 1},     {512, 512, 2 * kBufBytes, 1}, {512, 512, kBufBytes, 1}};
   for (const Geometry& g : order)
     if (geometry_fits(g, n_rows)) {
@@ -1380,7 +1391,8 @@ cudaError_t launch_walk_geom(const GbdtModel& g, const WalkArgs& a) {
 cudaError_t launch_walk(const GbdtModel& g, const WalkArgs& a) {
   if (g.fast_threads == 512 && g.block_cands == 1024) return launch_walk_geom<512, 1024>(g, a);
   if (g.fast_threads == 512) return launch_walk_geom<512, 512>(g, a);
-  return launch_walk_geom<256, 512>(g, a);
+  if (g.block_cands == 512) return launch_walk_geom<256, 512>(g, a);
+  return launch_walk_geom<256, 1024>(g, a);
 }
 
 FastView make_view(const GbdtModel& g, const FastWait* wait) {
@@ -1451,7 +1463,7 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
                                int k, unsigned long long* partial, void* scratch, int* status,
                                cudaStream_t stream, int64_t* launches, cudaEvent_t ev_begin,
                                const FastSlice* slice, void* memo_mem, const FastWait* wait,
-                               const FastPrepared* prep) {
+                               const FastPrepared* prep, const int32_t* perm) {
   WalkArgs a{};
   a.desc = desc;
   if (p_by_value) a.pv = *p_by_value;
@@ -1470,6 +1482,7 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
   unsigned* d_mask = static_cast<unsigned*>(scratch);
   uint8_t* d_rows = static_cast<uint8_t*>(scratch) + 256;
   fv.cand_rows = d_rows;
+  if (!seg_off && perm) a.seg_idx = perm;  // dense form ranked in the given order of the catalogue
   MemoView memo{};
   int memo_batch = (memo_mem && !p_by_value && C > 0) ? fast_memo_batch(g, P) : 0;
   if (memo_batch > 0) memo = memo_view(memo_mem, C);

@@ -154,8 +154,8 @@ struct ks_catalogue {
   int device = 0;
   bool prepared = false;   // false: calls go through ks_select_one
   int nblk = 0, slices = 1, max_k = KS_MAX_K;
-  void* d_mem = nullptr;   // one block: rows | memo | partial lists | partial-score planes
-  size_t off_memo = 0, off_part = 0, off_scores = 0;
+  void* d_mem = nullptr;   // one block: rows | memo | partial lists | partial-score planes | similarity order
+  size_t off_memo = 0, off_part = 0, off_scores = 0, off_order = 0;
 };
 
 struct ks_model {
@@ -219,6 +219,13 @@ struct FastPrepared {
   void* memo_mem;            // class tables and ids of every combination + one problem's record table, or null
 };
 
+// Similarity order of a catalogue (ks_order.cu): positions sorted so that neighbours differ in as
+// few knobs as possible; written to the front of `scratch` as C int32.
+constexpr int kOrderMinProblems = 16;  // batches of at least this many problems are ranked in similarity order
+size_t order_scratch_bytes(int C);
+cudaError_t launch_catalogue_order(const ks_candidate* d_c, int C, void* scratch, cudaStream_t stream,
+                                   int64_t* launches);
+
 // Search-space enumeration and validity filtering (ks_catalogue.cu).
 cudaError_t launch_enumerate(long long first, long long count, ks_candidate* d_out, cudaStream_t stream,
                              int64_t* launches);
@@ -241,7 +248,8 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
                                int k, unsigned long long* partial, void* scratch, int* status,
                                cudaStream_t stream, int64_t* launches, cudaEvent_t ev_begin,
                                const FastSlice* slice = nullptr, void* memo_mem = nullptr,
-                               const FastWait* wait = nullptr, const FastPrepared* prep = nullptr);
+                               const FastWait* wait = nullptr, const FastPrepared* prep = nullptr,
+                               const int32_t* perm = nullptr);
 // Prepared catalogue (single-problem calls against a fixed catalogue and model).
 size_t fast_prepared_rows_bytes(const GbdtModel& g, int C);
 size_t fast_prepared_memo_bytes(const GbdtModel& g, int C);  // 0: the model's per-pair rows do not fit a record

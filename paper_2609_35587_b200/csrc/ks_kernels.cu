@@ -4,6 +4,7 @@
 // in ks_gbdt_fast.cu.
 #include <cuda_bf16.h>
 
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -778,7 +779,10 @@ size_t select_partial_bytes(const ks_model& model, int P, int C, int64_t pairs, 
     const size_t part = (static_cast<size_t>(P) * nblk * k * sizeof(unsigned long long) + 255) / 256 * 256;
     const int S = segmented ? 1 : fast_slices(model.gbdt, static_cast<int64_t>(P) * nblk);
     const size_t planes = S > 1 ? (sizeof(float) * S * static_cast<size_t>(pairs) + 255) / 256 * 256 : 0;
-    return part + (fast_scratch_bytes(model.gbdt, C) + 255) / 256 * 256 + planes + (S > 1 ? 0 : fast_memo_bytes(model.gbdt, P, C));
+    const size_t memo = S > 1 ? 0 : (fast_memo_bytes(model.gbdt, P, C) + 255) / 256 * 256;
+    // a dense batch is ranked in similarity order of the catalogue (ks_order.cu)
+    const size_t order = (memo > 0 && !segmented && P >= kOrderMinProblems) ? order_scratch_bytes(C) : 0;
+    return part + (fast_scratch_bytes(model.gbdt, C) + 255) / 256 * 256 + planes + memo + order;
   }
   if (model.kind == 1 && model.mlp.tc) {
     const int nblk = mlp_tc_blocks_per_problem(P, per);
@@ -822,9 +826,19 @@ cudaError_t launch_select(const ks_gpu_desc& desc, const ks_model& model, const 
     void* memo_mem = (sized_slices > 1 || p_by_value || fast_memo_bytes(model.gbdt, P, C) == 0)
                          ? nullptr
                          : static_cast<char*>(d_partial) + part_bytes + (fast_scratch_bytes(model.gbdt, C) + 255) / 256 * 256;
+    // a dense batch of problems: rank the catalogue in similarity order (neighbouring candidates
+    // then take similar paths through the trees); the order sits behind the memo
+    const int32_t* perm = nullptr;
+    if (memo_mem && !d_seg_off && P >= kOrderMinProblems && C > 0) {
+      void* order_mem = static_cast<char*>(memo_mem) + (fast_memo_bytes(model.gbdt, P, C) + 255) / 256 * 256;
+      cudaError_t eo = launch_catalogue_order(d_c, C, order_mem, stream, launches);
+      if (eo != cudaSuccess) return eo;
+      perm = static_cast<const int32_t*>(order_mem);
+    }
     cudaError_t e = launch_select_fast(desc, model.gbdt, d_p, p_by_value, P, d_c, C, nblk, rows, d_seg_off,
                                        d_seg_idx, k, part, static_cast<char*>(d_partial) + part_bytes, d_status,
-                                       stream, launches, ev_begin, sl.n_slices > 1 ? &sl : nullptr, memo_mem, wait);
+                                       stream, launches, ev_begin, sl.n_slices > 1 ? &sl : nullptr, memo_mem, wait,
+                                       nullptr, perm);
     if (e != cudaSuccess) return e;
     if (ev_end) cudaEventRecord(ev_end, stream);
     topk_merge_kernel<<<(P * 32 + kBlock - 1) / kBlock, kBlock, 0, stream>>>(part, P, nblk * k, k, d_topk_idx,

@@ -534,7 +534,7 @@ def test_select_other_model_shapes(ks, ctx, case):
 @pytest.mark.parametrize("case", ["cfg1_slots128", "cfg1_hist256", "cfg1_pernode", "cfg2_pernode", "continuous"])
 def test_select_tile_geometries(ks, ctx, case):
     """The quantised kernel's tile geometries, picked by the number of rows: the slot-table
-    ensemble (<= 72 rows: two CTAs of 512 threads x 1,024 candidates per SM), the 256-bin and the
+    ensemble (<= 74 rows: two CTAs of 256 threads x 1,024 candidates per SM), the 256-bin and the
     quantile-per-node ensembles of config 1 (<= 149 rows: two CTAs of 256 threads x 512
     candidates), the quantile-per-node ensemble of config 2 (<= 376 rows: one CTA of 512 threads x
     512 candidates), and an ensemble with a continuous threshold at every node of 3,000 trees (more
@@ -554,7 +554,7 @@ def test_select_tile_geometries(ks, ctx, case):
     else:
         law = case.split("_")[1]
         w = wl.make_workload(1, P=5, C=3000, law=law)
-        want = "threads=512 block=1024" if law == "slots128" else "threads=256 block=512"
+        want = "threads=256 block=1024" if law == "slots128" else "threads=256 block=512"
     model = ctx.model_create_gbdt(*w.gbdt)
     assert want in model.describe(), model.describe()
     idx, sc = run_select(ks, ctx, w, model)
@@ -581,7 +581,7 @@ def test_select_tile_geometries(ks, ctx, case):
     check_select(wm, idx, sc, TOL_GBDT, sample=range(0, 40, 3))
 
 
-@pytest.mark.parametrize("geometry", ["512,1024,32", "512,1024,16", "512,512,32", "512,512,16", "256,512,16"])
+@pytest.mark.parametrize("geometry", ["512,1024,32", "512,1024,16", "512,512,32", "512,512,16", "256,512,16", "256,1024,16"])
 def test_select_forced_tile_geometry(ks, ctx, geometry, monkeypatch):
     """Every tile geometry on the same ensemble (config 1, a quantile per node, 143 rows), forced
     through KS_FAST_GEOMETRY = threads, candidates per CTA, chunk-buffer KiB."""
@@ -680,7 +680,8 @@ def test_select_memo_table_in_batches(ks, ctx):
     model = ctx.model_create_gbdt(*w.gbdt)
     n0 = ctx.launch_count()
     idx, sc = run_select(ks, ctx, w, model)
-    assert ctx.launch_count() - n0 == 2 + 1 + 3 * 2 + 1  # mask, candidate rows, compaction, 3 x (table, walk), merge
+    # mask, candidate rows, compaction, the catalogue's similarity order (key kernel + sort), 3 x (table, walk), merge
+    assert ctx.launch_count() - n0 == 2 + 1 + 4 + 3 * 2 + 1
     check_select(w, idx, sc, TOL_GBDT, sample=list(range(0, 900, 37)) + [408, 409, 817, 818, 899])
 
 
