@@ -586,7 +586,7 @@ __device__ __forceinline__ uint32_t path_step(uint32_t a, uint32_t cb_r, uint32_
 // (row offset, replicated j + 1) pair, so that twice as many trees keep their word-wise levels.
 // THREADS threads rank NC candidates: NC / 4 words times THREADS / (NC / 4) tree groups.
 template <int L, int NP, bool kCompact, int THREADS, int NC>
-__global__ void __launch_bounds__(THREADS, THREADS <= 512 ? 2 : 1)
+__global__ void __launch_bounds__(THREADS, THREADS <= 256 ? 2 : 1)
 select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_problem p_value, int use_value,
                    const ks_candidate* __restrict__ c, int P, int C, int nblk, int rows_per_cta,
                    const int64_t* __restrict__ seg_off, const int32_t* __restrict__ seg_idx, FastView fv,
@@ -974,19 +974,20 @@ static std::vector<PartitionCode> partition_codes(int L) {
 
 // Tile geometry by the number of rows: the [row][candidate] tile and the two chunk buffers have to
 // fit the shared memory of one SM (228 KiB, 1 KiB of it reserved per CTA; a CTA's own limit is
-// 227 KiB including its static part). Measured on one ensemble: what matters is (i) two CTAs per
-// SM, so that one CTA's tile fill and ranking overlap the other's walk (15 %), and (ii) four trees
-// or more per thread and chunk, which the compiler interleaves (13 %); sixteen walking warps per
-// SM already saturate the walk, eight do not. Hence, in order of preference: two CTAs of 256
-// threads x 1,024 candidates (eight trees per thread and chunk, up to 128 registers per thread;
-// up to 74 rows), two CTAs of 256 threads x 512 candidates (up to 149 rows), then one CTA of 512
-// threads with 1,024 candidates (up to 183 rows) or 512 candidates (up to 376 rows), with 32 KB
-// chunk buffers where they fit. Every CTA streams the whole ensemble, so a halved block doubles
-// that traffic (two CTAs of 256 threads x 256 candidates measured slower than one CTA of
-// 512 x 512; two CTAs of 128 x 512 and one CTA of 256 x 1,024 have too few warps). Two CTAs of
-// 512 threads x 1,024 candidates (64 registers per thread) measured 54 to 63 ms on the same
-// ensemble depending on how unrelated code around the loop happened to be compiled; the
-// 256-thread form, 51.6 ms, does not depend on that. More rows than 376: the general kernel.
+// 227 KiB including its static part). What was measured to matter on one ensemble: (i) four trees
+// or more per thread and chunk, which the compiler interleaves (13 %); (ii) up to 128 registers
+// per thread - the 64-register forms (two CTAs of 512 threads) ran 54 to 63 ms on the same
+// ensemble depending on how unrelated code around the loop happened to be compiled, and one CTA
+// of 512 threads gained 15 % from the larger budget; (iii) two CTAs per SM, so that one CTA's
+// tile fill and ranking overlap the other's walk, when the tile leaves room for them; sixteen
+// walking warps per SM saturate the walk, eight do not. Hence, in order of preference: two CTAs
+// of 256 threads x 1,024 candidates (eight trees per thread and chunk; up to 74 rows); one CTA of
+// 512 threads x 1,024 candidates with 32 KB chunk buffers (eight trees per thread and chunk; up
+// to 156 rows); two CTAs of 256 threads x 512 candidates; one CTA of 512 threads x 1,024
+// candidates with 16 KB buffers (up to 188 rows) or x 512 candidates (up to 376 rows). Every CTA
+// streams the whole ensemble, so a halved block doubles that traffic (two CTAs of 256 threads x
+// 256 candidates measured slower than one CTA of 512 x 512; two CTAs of 128 x 512 and one CTA of
+// 256 x 1,024 have too few warps). More rows than 376: the general kernel.
 // KS_FAST_GEOMETRY="threads,candidates,buffer KiB" overrides the choice (a tuning aid; a geometry
 // that does not fit is refused).
 struct Geometry {
@@ -1016,8 +1017,8 @@ static bool pick_geometry(int n_rows, Geometry* out) {
       }
     }
   }
-  const Geometry order[] = {{256, 1024, kBufBytes, 2},     {256, 512, kBufBytes, 2}, {512, 1024, 2 * kBufBytes, 1},
-                            {512, 1024, kBufBytes, 1},     {512, 512, 2 * kBufBytes, 1}, {512, 512, kBufBytes, 1}};
+  const Geometry order[] = {{256, 1024, kBufBytes, 2},     {512, 1024, 2 * kBufBytes, 1}, {256, 512, kBufBytes, 2},
+                            {512, 1024, kBufBytes, 1},     {512, 512, 2 * kBufBytes, 1},  {512, 512, kBufBytes, 1}};
   for (const Geometry& g : order)
     if (geometry_fits(g, n_rows)) {
       *out = g;

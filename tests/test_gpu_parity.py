@@ -535,9 +535,9 @@ def test_select_other_model_shapes(ks, ctx, case):
 def test_select_tile_geometries(ks, ctx, case):
     """The quantised kernel's tile geometries, picked by the number of rows: the slot-table
     ensemble (<= 74 rows: two CTAs of 256 threads x 1,024 candidates per SM), the 256-bin and the
-    quantile-per-node ensembles of config 1 (<= 149 rows: two CTAs of 256 threads x 512
-    candidates), the quantile-per-node ensemble of config 2 (<= 376 rows: one CTA of 512 threads x
-    512 candidates), and an ensemble with a continuous threshold at every node of 3,000 trees (more
+    quantile-per-node ensembles of config 1 (<= 156 rows: one CTA of 512 threads x 1,024
+    candidates with 32 KB chunk buffers), the quantile-per-node ensemble of config 2 (<= 376 rows:
+    one CTA of 512 threads x 512 candidates), and an ensemble with a continuous threshold at every node of 3,000 trees (more
     rows than any geometry holds: the general kernel). Each: a batch (ks_select), the single-problem call (tree slices
     over prepared tiles), the scoring call on given feature rows, and a batch of 33 problems or
     more that takes the per-(problem, class) memo."""
@@ -554,7 +554,7 @@ def test_select_tile_geometries(ks, ctx, case):
     else:
         law = case.split("_")[1]
         w = wl.make_workload(1, P=5, C=3000, law=law)
-        want = "threads=256 block=1024" if law == "slots128" else "threads=256 block=512"
+        want = "threads=256 block=1024" if law == "slots128" else "threads=512 block=1024"
     model = ctx.model_create_gbdt(*w.gbdt)
     assert want in model.describe(), model.describe()
     idx, sc = run_select(ks, ctx, w, model)
