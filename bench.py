@@ -630,10 +630,10 @@ def main():
 
 # dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel per full-size step, from the
 # ncu captures of the 48-problem case under profiles/, scaled by the problems (None: no capture
-# for that workload). Config 1, per-node law: 15.4 MB read in the small case (catalogue, model,
+# for that workload). Config 1, per-node law: 15.7 MB read in the small case (catalogue, model,
 # per-call tables, the class records of 48 problems) + 0.24 MB of class records per further
-# problem (written by the table kernel, read once) + 9.7 MB of partial lists written.
-TRAFFIC_BYTES = {(1, "pernode"): 260e6, (1, "slots128"): 234e6, (4, None): 5.7e6}
+# problem (written by the table kernel, read once) + 4.8 MB of partial lists written.
+TRAFFIC_BYTES = {(1, "pernode"): 255e6, (1, "slots128"): 229e6, (4, None): 5.7e6}
 
 if __name__ == "__main__":
     main()
