@@ -404,6 +404,40 @@ def tree_roofline(pairs, trees, depth, kms):
     return achieved, achieved / ISSUE_PEAK
 
 
+def walk_floor(ks, ctx, w, model, dev):
+    """The tree walk stripped to its gather and instruction stream (ks_debug_walk_floor): feature
+    rows of the workload's first problems, 592 blocks of 1,024 rows (whole waves of 148 or 296
+    CTAs); the time of one pass over the ensemble is the difference of two calls that differ in
+    their number of passes only, so tile building, launches and the first copies cancel."""
+    import torch
+    rows = 592 * 1024
+    C = len(w.candidates)
+    P = -(-rows // C)
+    d_p, d_c = ks.to_device(w.problems[:P], dev), ks.to_device(w.candidates, dev)
+    feat = ctx.featurize(d_p, P, d_c, C)[:rows]
+    out = torch.empty(rows, dtype=torch.float32, device=dev)
+    lo, hi = 2, 10
+
+    def timed(repeat):
+        best = float("inf")
+        for _ in range(4):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            ctx.debug_walk_floor(feat, model, repeat, out)
+            e1.record()
+            torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        return best
+
+    timed(lo)
+    t_lo, t_hi = timed(lo), timed(hi)
+    pass_ms = (t_hi - t_lo) / (hi - lo)
+    trees, depth = len(w.gbdt[0]) - 1, 8  # config 1's ensemble: complete trees of depth 8
+    return {"rows": rows, "pass_ms": pass_ms, "passes": [lo, hi], "call_ms": [t_lo, t_hi],
+            "frac": tree_roofline(rows, trees, depth, pass_ms)[1], "kernel": model.describe()}
+
+
 def extra_runs(ks, ctx, dev, flush, args, peaks):
     """Short runs of the other configurations and threshold laws, so that one default line carries
     them: config 1 under the other two laws, config 2, config 4 (5 / 3 timed steps each), a
@@ -418,7 +452,12 @@ def extra_runs(ks, ctx, dev, flush, args, peaks):
         kms = float(np.mean(m["kernel_ms"]))
         out[f"config1_{law}"] = {"pairs_per_s": w.pairs / (np.mean(m["step_ms"]) * 1e-3), "ms_per_step": float(np.mean(m["step_ms"])),
                                  "kernel_ms": kms, "frac": tree_roofline(w.pairs, 500, 8, kms)[1], "kernel": model.describe()}
+        out[f"walk_floor_{law}"] = walk_floor(ks, ctx, w, model, dev)
         model.close()
+    w = wl.make_workload(1, law=args.law)
+    model = ctx.model_create_gbdt(*w.gbdt)
+    out[f"walk_floor_{args.law}"] = walk_floor(ks, ctx, w, model, dev)
+    model.close()
     w = wl.make_workload(2, law=args.law)
     model = ctx.model_create_gbdt(*w.gbdt)
     m = measure_select(ks, ctx, w, model, 3, 3, dev, flush)

@@ -396,6 +396,20 @@ ks_status ks_model_describe(const ks_model* model, char* buf, int len);
  * runs out, the kernel sets the status word and returns, and the call reports KS_ERR_TIMEOUT
  * without any fault: the failure path can be tested on a healthy GPU. */
 ks_status ks_debug_set_wait(ks_ctx* ctx, int probe_limit, int starve);
+/* Measurement aid, no counterpart in the paper: the tree walk of ks_score stripped of everything
+ * but its gather and instruction stream, to measure the floor that stream sets for the tree
+ * kernel. Tiles are built from the `rows` feature rows (device, [rows][64] floats) exactly as
+ * ks_score builds them; every CTA then copies the first two chunks of the ensemble once and
+ * walks them `repeat` x n_chunks times (as many chunk walks as `repeat` passes over the whole
+ * ensemble) without waiting for, releasing or refilling a chunk buffer, and stores the sums it
+ * accumulated to d_scores (device, [rows]; with c0, c1 the sums of the two chunks' leaves for a
+ * row and n = repeat x n_chunks: base + ceil(n / 2) c0 + floor(n / 2) c1). The time of a pass is
+ * the difference of two calls with different `repeat`, divided by the difference. Tree models on
+ * the quantised kernel with 1,024-candidate tiles, three word-wise and five path levels only
+ * (the benchmark's ensemble); anything else returns KS_ERR_UNSUPPORTED. 1 <= repeat <= 4096.
+ * Asynchronous on `stream`; uses the context's workspace like ks_score. */
+ks_status ks_debug_walk_floor(ks_ctx* ctx, const float* d_features, int64_t rows, const ks_model* model,
+                              int repeat, float* d_scores, void* stream);
 /* Checked build only (libks_debug.so, compiled with KS_DEBUG_BOUNDS): the kernels compare
  * every index they form from data with its range and, instead of touching memory out of range,
  * record the source line of the first violation. Returns that line, 0 when there was none,

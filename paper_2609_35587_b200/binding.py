@@ -27,7 +27,7 @@ EXPORTS = ("ks_create", "ks_destroy", "ks_last_cuda_error", "ks_model_create_gbd
            "ks_feature_name", "ks_launch_count", "ks_profile_enable", "ks_profile_last_ms", "ks_device_status", "ks_select_trees_static",
            "ks_enumerate", "ks_valid_catalogue", "ks_remap_indices", "ks_model_describe", "ks_merge_topk", "ks_catalogue_prepare", "ks_catalogue_destroy",
            "ks_select_one_prepared",
-           "ks_debug_set_wait", "ks_debug_bounds_line", "ks_debug_bounds_clear")
+           "ks_debug_set_wait", "ks_debug_bounds_line", "ks_debug_bounds_clear", "ks_debug_walk_floor")
 
 
 class KsError(RuntimeError):
@@ -83,6 +83,7 @@ def _load() -> ctypes.CDLL:
     lib.ks_catalogue_destroy.argtypes = [vp]
     lib.ks_select_one_prepared.argtypes = [vp, vp, _Problem, i32, vp, vp, vp]
     lib.ks_debug_set_wait.argtypes = [vp, i32, i32]
+    lib.ks_debug_walk_floor.argtypes = [vp, vp, i64, vp, i32, vp, vp]
     lib.ks_debug_bounds_line.restype = i32
     lib.ks_debug_bounds_clear.restype = None
     for name in EXPORTS:
@@ -317,6 +318,15 @@ class Context:
                            _stream())
         self._check(st, "ks_score")
         return (scores, leaf) if want_leaf_idx else scores
+
+    def debug_walk_floor(self, d_features, model: Model, repeat: int, out=None):
+        """Measurement aid: the tree walk stripped to its gather stream (see ks_debug_walk_floor)."""
+        rows = d_features.shape[0]
+        if out is None:
+            out = torch.empty(rows, dtype=torch.float32, device=self.device)
+        st = _lib.ks_debug_walk_floor(self._h, _dptr(d_features), rows, model._h, int(repeat), _dptr(out), _stream())
+        self._check(st, "ks_debug_walk_floor")
+        return out
 
     def select(self, d_p, P, d_c, C, model: Model, k, d_seg_off=None, d_seg_idx=None, pairs=None,
                out_idx=None, out_score=None):

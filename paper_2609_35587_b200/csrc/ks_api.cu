@@ -330,9 +330,11 @@ ks_status ks_model_describe(const ks_model* model, char* buf, int len) {
   if (!model || !buf || len < 1) return KS_ERR_INVALID_ARG;
   if (model->kind == 0 && model->gbdt.fast) {
     const ks::GbdtModel& g = model->gbdt;
-    std::snprintf(buf, len, "select_fast_kernel threads=%d block=%d rows=%d thresholds=%d top_levels=%d%s trees=%d depth=%d",
+    std::snprintf(buf, len,
+                  "select_fast_kernel threads=%d block=%d rows=%d thresholds=%d top_levels=%d%s trees=%d depth=%d "
+                  "chunks=%d chunk_trees=%d",
                   g.fast_threads, g.block_cands, g.n_qrows, g.n_qthr, g.top_levels, g.top_compact ? "c" : "",
-                  g.n_trees, g.fast_depth);
+                  g.n_trees, g.fast_depth, g.n_chunks, g.tpc);
   } else if (model->kind == 0) {
     std::snprintf(buf, len, "select_generic_kernel trees=%d depth=%d", model->gbdt.n_trees, model->gbdt.max_depth);
   } else if (model->kind == 1 && model->mlp.tc) {
@@ -535,6 +537,20 @@ ks_status ks_featurize(ks_ctx* ctx, const ks_problem* d_p, int P, const ks_candi
   cudaError_t e = ks::launch_featurize(ctx->desc, d_p, P, d_c, C, d_seg_offsets, d_seg_index, pairs,
                                        d_features, ctx->ws, static_cast<cudaStream_t>(stream), &ctx->launches);
   return e == cudaSuccess ? KS_OK : cuda_fail(ctx, e, "ks_featurize");
+}
+
+ks_status ks_debug_walk_floor(ks_ctx* ctx, const float* d_features, int64_t rows, const ks_model* model,
+                              int repeat, float* d_scores, void* stream) {
+  if (!ctx || !model || model->ctx != ctx || rows < 1 || repeat < 1 || repeat > 4096) return KS_ERR_INVALID_ARG;
+  if (!d_features || !d_scores) return KS_ERR_INVALID_ARG;
+  if (model->kind != 0 || !model->gbdt.fast) return KS_ERR_UNSUPPORTED;
+  DeviceGuard g(ctx->device);
+  ks_status s = ensure_workspace(ctx, ks::score_fast_scratch_bytes(model->gbdt, rows));
+  if (s != KS_OK) return s;
+  cudaError_t e = ks::launch_score_fast(ctx->desc, model->gbdt, d_features, rows, d_scores, ctx->ws, ctx->d_status,
+                                        static_cast<cudaStream_t>(stream), &ctx->launches, &ctx->wait, repeat);
+  if (e == cudaErrorNotSupported) return KS_ERR_UNSUPPORTED;
+  return e == cudaSuccess ? KS_OK : cuda_fail(ctx, e, "ks_debug_walk_floor");
 }
 
 ks_status ks_score(ks_ctx* ctx, const float* d_features, int64_t rows, const ks_model* model,

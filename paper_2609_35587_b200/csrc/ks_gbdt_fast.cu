@@ -66,6 +66,7 @@ constexpr unsigned kSleepNs = 1200;    // asked-for sleep between two probes of 
 constexpr int kCombos = 16;            // dtype_ab x dtype_d
 
 // shared memory map (byte offsets from the dynamic shared base): the chunk buffers, then the tile
+constexpr int kSmCount = 148;           // SMs of the one device this library is built for (sm_100a)
 constexpr int kNBuf = 2;                // tree-chunk buffers (a ring; four of 8 KB and three of 12 KB measured slower)
 constexpr int kOffBuf0 = 0;
 
@@ -189,6 +190,7 @@ struct SliceArgs {
   int* out_seq;            // single-problem form: receives `seq` once the k results are written
   int seq;
   float* score_out;        // scoring call (ks_score): the scores of the block's rows go here, no ranking
+  int repeat;              // floor measurement only: passes over the resident chunks
 };
 
 struct FastView {
@@ -478,59 +480,113 @@ tile_rows_kernel(const float* __restrict__ feat, int64_t rows, FastView fv, uint
 // phase A
 // ------------------------------------------------------------------------------------------
 
-// Scatters a 16-byte-aligned record of `n` row bytes into a tile column.
-__device__ __forceinline__ void scatter_record(const uint8_t* __restrict__ rec, int n, unsigned char* dst, int NC) {
-  const uint4* src = reinterpret_cast<const uint4*>(rec);
-  for (int v = 0; v * 16 < n; ++v) {
-    const uint4 q = __ldg(src + v);
-    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+// Sixteen rows of four neighbouring candidates: q[r] holds candidate r's bytes of rows row0 ..
+// row0 + 15 (a 16-byte vector of its record). Byte r of a tile word is candidate r, so every
+// group of four rows is a 4 x 4 byte transpose (eight byte permutes) and four word stores.
+__device__ __forceinline__ void scatter_vectors(const uint4 (&q)[4], int row0, int n, unsigned char* word0, int NC) {
+  const uint32_t w[4][4] = {{q[0].x, q[0].y, q[0].z, q[0].w},
+                            {q[1].x, q[1].y, q[1].z, q[1].w},
+                            {q[2].x, q[2].y, q[2].z, q[2].w},
+                            {q[3].x, q[3].y, q[3].z, q[3].w}};
 #pragma unroll
-    for (int b = 0; b < 16; ++b)
-      if (v * 16 + b < n) dst[(v * 16 + b) * NC] = static_cast<unsigned char>(w[b >> 2] >> (8 * (b & 3)));
+  for (int g = 0; g < 4; ++g) {
+    const int row = row0 + 4 * g;
+    if (row >= n) break;
+    const uint32_t lo_ab = __byte_perm(w[0][g], w[1][g], 0x5140u), lo_cd = __byte_perm(w[2][g], w[3][g], 0x5140u);
+    const uint32_t hi_ab = __byte_perm(w[0][g], w[1][g], 0x7362u), hi_cd = __byte_perm(w[2][g], w[3][g], 0x7362u);
+    const uint32_t out[4] = {__byte_perm(lo_ab, lo_cd, 0x5410u), __byte_perm(lo_ab, lo_cd, 0x7632u),
+                             __byte_perm(hi_ab, hi_cd, 0x5410u), __byte_perm(hi_ab, hi_cd, 0x7632u)};
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      if (row + j < n) *reinterpret_cast<uint32_t*>(word0 + static_cast<size_t>(row + j) * NC) = out[j];
   }
 }
 
-// Fills the tile bytes of the candidates this thread owns in phase A: candidate-only rows
-// from the per-call table, problem-only rows from s_pbin, per-pair rows from the memo record of
-// the candidate's class or computed here. Slots past the end of the segment get a neutral byte
-// so that word-wise arithmetic on the tile never borrows across bytes.
+// Fills the tile: candidate-only rows from the per-call table, problem-only rows from s_pbin,
+// per-pair rows from the memo record of the candidate's class or computed here. Slots past the
+// end of the segment get a neutral byte so that word-wise arithmetic on the tile never borrows
+// across bytes. A thread serves the four candidates of one tile word (byte r of the word is
+// candidate r): it fetches their records sixteen rows at a time and stores whole words; the
+// THREADS / (NC / 4) threads that share a word deal the records' vectors among themselves.
 template <int THREADS, int NC>
 __device__ __noinline__ void fill_tile(const ks_gpu_desc& desc, const ProblemTerms& pt,
                                        const ks_candidate* __restrict__ c, const FastView& fv,
                                        const int64_t* __restrict__ seg_off, const int32_t* __restrict__ seg_idx,
                                        int C, int64_t lo, int64_t start, int64_t stop, const float* T,
                                        const FeatQ* s_fq, const uint8_t* s_pbin, unsigned char* tile, int prob) {
+  constexpr int W = NC / 4, PARTS = THREADS / W;
   const int tid = threadIdx.x;
   const int combo = pt.dtype_ab * 4 + pt.dtype_d;
-#pragma unroll 1
-  for (int i = tid; i < NC; i += THREADS) {
-    const int64_t row = start + i;
-    unsigned char* my = tile + tile_byte(i, NC / 4);
-    if (row >= stop) {
-      for (int q = 0; q < fv.n_rows; ++q) my[q * NC] = 0x80;
-      continue;
+  // problem-only rows: one byte for the whole row
+  {
+    unsigned char* dst = tile + static_cast<size_t>(fv.n_pair_rows + fv.n_cand_rows) * NC;
+    for (int i = tid; i < fv.n_prob_rows * (NC / 16); i += THREADS) {
+      const uint32_t b = s_pbin[i / (NC / 16)] * 0x01010101u;
+      reinterpret_cast<uint4*>(dst)[i] = make_uint4(b, b, b, b);
     }
-    const int ci = seg_idx ? seg_idx[lo + row] : static_cast<int>(row);
-    // the candidate's class, fetched before the other loads that depend on ci only
-    const unsigned cid = fv.pair_class ? __ldg(fv.pair_class + static_cast<size_t>(combo) * C + ci) : kNoClass;
-    // candidate-only rows
-    scatter_record(fv.cand_rows + (static_cast<size_t>(combo) * C + KS_IDX(ci, C)) * fv.cand_rec, fv.n_cand_rows,
-                   my + fv.n_pair_rows * NC, NC);
-    // problem-only rows
-    unsigned char* dst = my + (fv.n_pair_rows + fv.n_cand_rows) * NC;
-    for (int q = 0; q < fv.n_prob_rows; ++q) dst[q * NC] = s_pbin[q];
-    // per-pair rows: the record of the candidate's class, when there is one
-    if (fv.pair_class) {
-      if (cid != kNoClass) {
-        scatter_record(fv.pair_tab + (static_cast<size_t>(prob) * kMemoCap + KS_IDX(cid, kMemoCap)) * fv.pair_rec,
-                       fv.n_pair_rows, my, NC);
-        continue;
+  }
+  const int word = tid % W, part = tid / W;
+  unsigned char* word0 = tile + 4 * word;
+  int ci[4];
+  unsigned cid[4];
+  bool lone = false;  // one of this word's candidates has no record of per-pair rows
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    const int64_t row = start + 4 * word + r;
+    ci[r] = row < stop ? (seg_idx ? seg_idx[lo + row] : static_cast<int>(row)) : -1;
+  }
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    cid[r] = (ci[r] >= 0 && fv.pair_class) ? __ldg(fv.pair_class + static_cast<size_t>(combo) * C + ci[r]) : kNoClass;
+    lone |= ci[r] >= 0 && cid[r] == kNoClass;
+  }
+  const uint4 neutral = make_uint4(0x80808080u, 0x80808080u, 0x80808080u, 0x80808080u);
+  const int cand_vecs = (fv.n_cand_rows + 15) / 16, pair_vecs = (fv.n_pair_rows + 15) / 16;
+  const uint8_t* cand_rec[4];
+  const uint8_t* pair_rec[4];
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    cand_rec[r] = ci[r] >= 0 ? fv.cand_rows + (static_cast<size_t>(combo) * C + KS_IDX(ci[r], C)) * fv.cand_rec : nullptr;
+    pair_rec[r] = cid[r] != kNoClass
+                      ? fv.pair_tab + (static_cast<size_t>(prob) * kMemoCap + KS_IDX(cid[r], kMemoCap)) * fv.pair_rec
+                      : nullptr;
+  }
+  // kBatch vectors of the four candidates are fetched before the first is stored, so that a thread
+  // waits for the memory once per batch, not once per vector
+  constexpr int kBatch = 1;
+#pragma unroll 1
+  for (int v0 = part; v0 < cand_vecs + pair_vecs; v0 += kBatch * PARTS) {
+    uint4 q[kBatch][4];
+#pragma unroll
+    for (int j = 0; j < kBatch; ++j) {
+      const int v = v0 + j * PARTS;
+      if (v >= cand_vecs + pair_vecs) break;
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        const uint8_t* rec = v < cand_vecs ? cand_rec[r] : pair_rec[r];
+        q[j][r] = rec ? __ldg(reinterpret_cast<const uint4*>(rec) + (v < cand_vecs ? v : v - cand_vecs)) : neutral;
       }
     }
-    const ks_candidate cand = load_candidate(c + ci);
+#pragma unroll
+    for (int j = 0; j < kBatch; ++j) {
+      const int v = v0 + j * PARTS;
+      if (v >= cand_vecs + pair_vecs) break;
+      if (v < cand_vecs) scatter_vectors(q[j], 16 * v, fv.n_cand_rows, word0 + static_cast<size_t>(fv.n_pair_rows) * NC, NC);
+      else scatter_vectors(q[j], 16 * (v - cand_vecs), fv.n_pair_rows, word0, NC);
+    }
+  }
+  // candidates without a record (no memo in this call, or a class table that was full): their
+  // per-pair columns are computed here, after the word stores that cover their bytes
+  if (!__syncthreads_or(lone)) return;
+  if (!lone) return;
+#pragma unroll 1
+  for (int r = part % 4; r < 4; r += (PARTS < 4 ? PARTS : 4)) {
+    if (ci[r] < 0 || cid[r] != kNoClass) continue;
+    unsigned char* my = word0 + r;
+    const ks_candidate cand = load_candidate(c + ci[r]);
     pair_columns<true>(pt, cand, desc, resources(pt, cand, desc).b_eff, [&](int col, float v) {
       const FeatQ& q = s_fq[col];
-      quantise(q, T + q.thr0, v, false, [&](int r, uint8_t b) { my[KS_IDX(r, fv.n_pair_rows) * NC] = b; });
+      quantise(q, T + q.thr0, v, false, [&](int row, uint8_t b) { my[KS_IDX(row, fv.n_pair_rows) * NC] = b; });
     });
   }
 }
@@ -585,13 +641,17 @@ __device__ __forceinline__ uint32_t path_step(uint32_t a, uint32_t cb_r, uint32_
 // levels' constants travel as one 32-bit word per node (row offset << 8 | j + 1) instead of a
 // (row offset, replicated j + 1) pair, so that twice as many trees keep their word-wise levels.
 // THREADS threads rank NC candidates: NC / 4 words times THREADS / (NC / 4) tree groups.
-template <int L, int NP, bool kCompact, int THREADS, int NC>
+// kFloor (measurement only): the walk without its chunk ring. The first kNBuf chunks are copied
+// once and stay resident; the CTA walks them again and again (sl.repeat passes of n_chunks chunk
+// walks each), never waits, releases or refills, so the time per pass is that of the gather and
+// instruction stream of the walk alone, at the occupancy and tile size of the real kernel.
+template <int L, int NP, bool kCompact, int THREADS, int NC, bool kFloor = false>
 __global__ void __launch_bounds__(THREADS, THREADS <= 256 ? 2 : 1)
 select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_problem p_value, int use_value,
                    const ks_candidate* __restrict__ c, int P, int C, int nblk, int rows_per_cta,
                    const int64_t* __restrict__ seg_off, const int32_t* __restrict__ seg_idx, FastView fv,
                    int k, unsigned long long* __restrict__ partial, int* __restrict__ status,
-                   SliceArgs sl, const __grid_constant__ FastTopParams top) {
+                   SliceArgs sl, int n_items, const __grid_constant__ FastTopParams top) {
   constexpr int W = NC / 4;        // words per tile row = lane slots
   constexpr int G = THREADS / W;   // tree groups
   static_assert(THREADS % W == 0 && W % 32 == 0 && G >= 1, "tile geometry");
@@ -608,7 +668,32 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
   const int tid = threadIdx.x;
   const int kOffTile = kNBuf * fv.buf_bytes;
   const int S = sl.n_slices;
-  const int prob = blockIdx.x / (nblk * S), chunk = (blockIdx.x / S) % nblk, slice = blockIdx.x % S;
+  const uint32_t sbase = smem_u32(smem);
+  const uint32_t bar0 = smem_u32(&s_bar[0]);  // barrier of buffer b: bar0 + 8 b
+  const bool tiles_given = sl.tiles != nullptr;  // the tiles were built in front: no feature work here
+  if (tid == 0) {
+    for (int b = 0; b < kNBuf; ++b) mbar_init(bar0 + 8u * b, 1);
+    s_fail = 0;
+    for (int b = 0; b < kNBuf; ++b) s_done[b] = s_pending[b] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (tid < 64) s_fq[tid] = fv.feat[tid];
+  __syncthreads();
+  // everything above is independent of the kernel in front (the per-problem tables): when this
+  // grid was launched as its programmatic dependent, wait for that grid here
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  uint32_t phases = 0;  // bit b: parity of buffer b's barrier
+  const int word = tid % W, grp = tid / W;
+  volatile int* v_fail = &s_fail;
+
+  // A CTA serves the items blockIdx.x, blockIdx.x + gridDim.x, ...: an item is one (problem,
+  // candidate block, tree slice). The batch form of a geometry that holds one CTA per SM is
+  // launched with one CTA per SM, so that a CTA's set-up and the gap between two CTAs are paid
+  // once, not per item; everything else (two CTAs per SM, which hide each other's gaps; tree
+  // slices and scoring, which leave an item early) is launched with one CTA per item.
+#pragma unroll 1
+  for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+  const int prob = item / (nblk * S), chunk = (item / S) % nblk, slice = item % S;
   // rows of this problem: lo = where its scores sit in per-row arrays; lo_idx = where its pool
   // indices start in seg_idx (per-problem segments, or - without offsets - one ranking order of
   // the whole catalogue shared by every problem)
@@ -624,9 +709,7 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
   // chunks of the ensemble this CTA walks
   const int ch_begin = static_cast<int>(static_cast<int64_t>(fv.n_chunks) * slice / S);
   const int ch_end = static_cast<int>(static_cast<int64_t>(fv.n_chunks) * (slice + 1) / S);
-  const uint32_t sbase = smem_u32(smem);
-  const uint32_t bar0 = smem_u32(&s_bar[0]);  // barrier of buffer b: bar0 + 8 b
-  const bool tiles_given = sl.tiles != nullptr;  // the tiles were built in front: no feature work here
+  __syncthreads();  // the item before this one is finished with the shared state
   if (tid == 0) {
     if (!tiles_given && !fv.prob_tab) {
       problem_terms(use_value ? p_value : load_problem(p + prob), desc, s_pt);
@@ -640,37 +723,26 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
         });
       }
     }
-    for (int b = 0; b < kNBuf; ++b) mbar_init(bar0 + 8u * b, 1);
-    s_fail = 0;
-    for (int b = 0; b < kNBuf; ++b) s_done[b] = s_pending[b] = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    s_abort = *reinterpret_cast<volatile int*>(&g_fast_abort);
   }
-  if (tid < 64) s_fq[tid] = fv.feat[tid];
   if (tid < KS_MAX_K) s_list[tid] = 0ull;
-  __syncthreads();
-  // everything above is independent of the kernel in front (the per-problem tables): when this
-  // grid was launched as its programmatic dependent, wait for that grid here
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  if (tid == 0) s_abort = *reinterpret_cast<volatile int*>(&g_fast_abort);
-  __syncthreads();
-  if (s_abort) {  // a wait ran out in an earlier CTA of this launch: the call fails, leave at once
-    if (tid < k && slice == 0 && partial) partial[(static_cast<size_t>(prob) * nblk + chunk) * k + tid] = 0ull;
-    return;
-  }
   if (!tiles_given && fv.prob_tab) {
     const uint8_t* rec = fv.prob_tab + static_cast<size_t>(prob) * kProbRec;
     for (int i = tid; i < fv.n_prob_rows; i += THREADS) s_pbin[i] = __ldcg(rec + i);
     if (tid < static_cast<int>(sizeof(ProblemTerms) / 4))
       reinterpret_cast<uint32_t*>(&s_pt)[tid] = __ldcg(reinterpret_cast<const uint32_t*>(rec + kFastMaxProbRows) + tid);
-  } else if (!tiles_given && tid < KS_F && feat_class(tid) == 0) {
+  }
+  __syncthreads();
+  if (s_abort) {  // a wait ran out in an earlier CTA of this launch: the call fails, leave at once
+    if (tid < k && slice == 0 && partial) partial[(static_cast<size_t>(prob) * nblk + chunk) * k + tid] = 0ull;
+    return;
+  }
+  if (!tiles_given && !fv.prob_tab && tid < KS_F && feat_class(tid) == 0) {
     const int first = fv.n_pair_rows + fv.n_cand_rows;
     const FeatQ& q = s_fq[tid];
     quantise(q, fv.thr + q.thr0, s_pfeat[tid], false,
              [&](int row, uint8_t b) { s_pbin[KS_IDX(row - first, kFastMaxProbRows)] = b; });
   }
-  uint32_t phases = 0;  // bit b: parity of buffer b's barrier
-  const int word = tid % W, grp = tid / W;
-  volatile int* v_fail = &s_fail;
 
   for (int64_t start = static_cast<int64_t>(chunk) * rows_per_cta; start < len;
        start += static_cast<int64_t>(nblk) * rows_per_cta) {
@@ -716,22 +788,26 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
 #else
     constexpr uint32_t tile0 = 0, tile_bytes = 0;
 #endif
+    const int ch_stop = kFloor ? ch_begin + (ch_end - ch_begin) * sl.repeat : ch_end;
 #pragma unroll 1
-    for (int ch = ch_begin; ch < ch_end; ++ch) {
-      const int b = (ch - ch_begin) % kNBuf;
+    for (int ch_it = ch_begin; ch_it < ch_stop; ++ch_it) {
+      const int b = (ch_it - ch_begin) % kNBuf;
+      const int ch = kFloor ? ch_begin + b : ch_it;  // the chunk whose trees are walked
       const uint32_t bar = bar0 + 8u * b;
       const uint32_t par = (phases >> b) & 1u;
       // A wait that runs out ends the walk of this CTA: the buffer was never filled, so it is not
       // read; the call fails, and the CTAs that start later leave at once.
-      if (*v_fail || !mbar_wait_bounded(bar, par, fv.wait_limit, v_fail)) {
-        if (!*v_fail) {
-          s_fail = 1;
-          atomicExch(&g_fast_abort, 1);
-          if (status) atomicExch(status, KS_ERR_TIMEOUT);
+      if (!kFloor || ch_it - ch_begin < kNBuf) {
+        if (*v_fail || !mbar_wait_bounded(bar, par, fv.wait_limit, v_fail)) {
+          if (!*v_fail) {
+            s_fail = 1;
+            atomicExch(&g_fast_abort, 1);
+            if (status) atomicExch(status, KS_ERR_TIMEOUT);
+          }
+          break;
         }
-        break;
+        phases ^= 1u << b;
       }
-      phases ^= 1u << b;
       const uint32_t buf = sbase + kOffBuf0 + b * fv.buf_bytes;
       // With A_l the shared address of a walk's node at level l, A_{l+1} = 2 A_l + (4 tpc - buf)
       // + 4 bit for every level, and after the last level A points at the walk's leaf.
@@ -751,14 +827,14 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
           uint32_t d[kTop > 0 ? kTop : 1];
           if (kCompact) {
             const uint32_t* tw = reinterpret_cast<const uint32_t*>(top.w) +
-                                 static_cast<size_t>(KS_IDX(ch * tpc + t, 2 * kFastTopPairs / kTop)) * kTop;
+                                 static_cast<size_t>(KS_IDX(ch * tpc + t, 2 * kFastTopPairs / (kTop > 0 ? kTop : 1))) * kTop;
 #pragma unroll
             for (int n = 0; n < kTop; ++n) {
               const uint32_t v = tw[n];
               d[n] = lds_u32(cb + static_cast<uint32_t>(KS_IDX(v >> 8, fv.n_rows * NC))) - __byte_perm(v, 0u, 0u);
             }
           } else {
-            const uint2* tw = top.w + static_cast<size_t>(KS_IDX(ch * tpc + t, kFastTopPairs / kTop)) * kTop;
+            const uint2* tw = top.w + static_cast<size_t>(KS_IDX(ch * tpc + t, kFastTopPairs / (kTop > 0 ? kTop : 1))) * kTop;
 #pragma unroll
             for (int n = 0; n < kTop; ++n)
               d[n] = lds_u32(cb + static_cast<uint32_t>(KS_IDX(tw[n].x, fv.n_rows * NC))) - tw[n].y;
@@ -803,7 +879,7 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
       // Release the buffer without a block-wide barrier: every warp counts itself out, and the
       // last one to leave refills the buffer (nobody waits; warps may run a chunk ahead).
       __syncwarp();
-      if ((tid & 31) == 0) {
+      if (!kFloor && (tid & 31) == 0) {
         if (atomicAdd(&s_done[b], 1) == THREADS / 32 - 1) {
           s_done[b] = 0;
           s_pending[b] = 0;
@@ -819,6 +895,7 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
       }
     }
     __syncthreads();  // all walks are done: the buffers are free
+    if (kFloor && tid < kNBuf && !*v_fail) s_pending[tid] = 0;  // copied once, landed, never refilled
     if (*v_fail) {
       // The call has failed. Before this CTA gives its shared memory back, give the copies that
       // may still be in flight the time to land (bounded again); the test hook's copies land in
@@ -937,6 +1014,7 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
       }
     }
   }
+  }  // items
 }
 
 }  // namespace
@@ -1008,7 +1086,7 @@ static bool geometry_known(int t, int c) {
 static bool pick_geometry(int n_rows, Geometry* out) {
   if (const char* env = std::getenv("KS_FAST_GEOMETRY")) {
     int t = 0, c = 0, kb = 0;
-    if (std::sscanf(env, "%d,%d,%d", &t, &c, &kb) == 3 && geometry_known(t, c) && (kb == 16 || kb == 32)) {
+    if (std::sscanf(env, "%d,%d,%d", &t, &c, &kb) == 3 && geometry_known(t, c) && kb >= 8 && kb <= 32) {
       Geometry g{t, c, kb * 1024, 2};
       if (!geometry_fits(g, n_rows)) g.ctas_per_sm = 1;
       if (geometry_fits(g, n_rows)) {
@@ -1302,7 +1380,7 @@ size_t fast_memo_bytes(const GbdtModel& g, int P, int C) {
 int fast_slices(const GbdtModel& g, int64_t blocks) {
   if (blocks < 1) blocks = 1;
   if (blocks > kMaxSliceBlocks) return 1;
-  const int64_t slots = static_cast<int64_t>(g.ctas_per_sm) * 148;
+  const int64_t slots = static_cast<int64_t>(g.ctas_per_sm) * kSmCount;
   if (blocks >= slots) return 1;  // the machine is full without slices
   int best = 1;
   double best_cost = 1e30;
@@ -1344,14 +1422,20 @@ struct WalkArgs {
   int dependent;  // launched right behind the kernel whose tables it reads
 };
 
-template <int L, int NP, bool kCompact, int THREADS, int NC>
+template <int L, int NP, bool kCompact, int THREADS, int NC, bool kFloor = false>
 cudaError_t launch_ln(const WalkArgs& a) {
   const size_t smem = static_cast<size_t>(kNBuf) * a.fv.buf_bytes + static_cast<size_t>(a.fv.n_rows) * NC;
-  auto kernel = &select_fast_kernel<L, NP, kCompact, THREADS, NC>;
+  auto kernel = &select_fast_kernel<L, NP, kCompact, THREADS, NC, kFloor>;
   cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), smem);
   if (e != cudaSuccess) return e;
   cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3(static_cast<unsigned>(static_cast<int64_t>(a.P) * a.nblk * a.sl.n_slices));
+  // One CTA per item, or - batch form of the geometries that hold one CTA per SM - one CTA per SM,
+  // each serving many items. (Two persistent CTAs on an SM run in step, so that both fill and rank
+  // at the same time and neither hides the other's: measured 6 % slower than one CTA per item.)
+  const int64_t n_items = static_cast<int64_t>(a.P) * a.nblk * a.sl.n_slices;
+  const bool persistent = THREADS > 256 && a.sl.n_slices == 1 && !a.sl.score_out && !a.sl.tiles;
+  const int64_t slots = kSmCount;
+  cfg.gridDim = dim3(static_cast<unsigned>(persistent && n_items > slots ? slots : n_items));
   cfg.blockDim = dim3(THREADS);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = a.stream;
@@ -1364,7 +1448,8 @@ cudaError_t launch_ln(const WalkArgs& a) {
   cfg.attrs = &attr;
   cfg.numAttrs = a.dependent ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, kernel, a.desc, a.d_p, a.pv, a.uv, a.d_c, a.P, a.C, a.nblk, a.rows_per_cta,
-                            a.seg_off, a.seg_idx, a.fv, a.k, a.partial, a.status, a.sl, *a.top);
+                            a.seg_off, a.seg_idx, a.fv, a.k, a.partial, a.status, a.sl, static_cast<int>(n_items),
+                            *a.top);
 }
 
 // the instantiation for a model's top levels and depth, within one tile geometry
@@ -1387,6 +1472,15 @@ cudaError_t launch_walk_geom(const GbdtModel& g, const WalkArgs& a) {
   if (L == 2) return launch_ln<2, -1, false, THREADS, NC>(a);
   if (L == 1) return launch_ln<1, -1, false, THREADS, NC>(a);
   return launch_ln<0, -1, false, THREADS, NC>(a);
+}
+
+// The floor measurement exists for the two geometries and the ensemble shape of the benchmark's
+// first configuration (three word-wise levels, five path levels, top constants as pairs).
+cudaError_t launch_walk_floor(const GbdtModel& g, const WalkArgs& a) {
+  if (g.top_compact || g.top_levels != 3 || g.fast_depth != 8 || g.n_chunks < kNBuf || g.block_cands != 1024)
+    return cudaErrorNotSupported;
+  if (g.fast_threads == 512) return launch_ln<3, 5, false, 512, 1024, true>(a);
+  return launch_ln<3, 5, false, 256, 1024, true>(a);
 }
 
 cudaError_t launch_walk(const GbdtModel& g, const WalkArgs& a) {
@@ -1609,7 +1703,7 @@ size_t score_fast_scratch_bytes(const GbdtModel& g, int64_t rows) {
 
 cudaError_t launch_score_fast(const ks_gpu_desc& desc, const GbdtModel& g, const float* d_feat, int64_t rows,
                               float* d_scores, void* scratch, int* status, cudaStream_t stream,
-                              int64_t* launches, const FastWait* wait) {
+                              int64_t* launches, const FastWait* wait, int floor_repeat) {
   WalkArgs a{};
   a.desc = desc;
   a.uv = 1;
@@ -1636,8 +1730,9 @@ cudaError_t launch_score_fast(const ks_gpu_desc& desc, const GbdtModel& g, const
     a.sl.n_slices = 1;
     a.sl.tiles = tiles;
     a.sl.score_out = d_scores + first;
+    a.sl.repeat = floor_repeat;
     *launches += 2;
-    e = launch_walk(g, a);
+    e = floor_repeat > 0 ? launch_walk_floor(g, a) : launch_walk(g, a);
     if (e != cudaSuccess) return e;
   }
   return cudaSuccess;

@@ -260,7 +260,7 @@ int fast_slices(const GbdtModel& g, int64_t blocks);
 size_t score_fast_scratch_bytes(const GbdtModel& g, int64_t rows);
 cudaError_t launch_score_fast(const ks_gpu_desc& desc, const GbdtModel& g, const float* d_feat, int64_t rows,
                               float* d_scores, void* scratch, int* status, cudaStream_t stream,
-                              int64_t* launches, const FastWait* wait = nullptr);
+                              int64_t* launches, const FastWait* wait = nullptr, int floor_repeat = 0);
 // checked build (KS_DEBUG_BOUNDS): source line of the first index found out of range (0: none;
 // -1: not a checked build), and its reset
 int fast_bounds_line();

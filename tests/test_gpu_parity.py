@@ -163,6 +163,35 @@ def test_score_gbdt_quantised_path(ks, ctx):
         assert np.all(np.abs(s - rs[:n]) <= TOL_GBDT * np.maximum(1, np.abs(rs[:n])))
 
 
+def test_walk_floor_sums(ks, ctx):
+    """The measurement form of the walk (ks_debug_walk_floor) walks real trees on real tiles:
+    its sums are those of the ensemble's first two chunks, repeated as the header says."""
+    import re
+    w = wl.make_workload(1, P=1, C=2500, trees=60, depth=8)
+    x = oracle.featurize(w.problems, w.candidates, DESC)
+    off, nodes, base = w.gbdt
+    model = ctx.model_create_gbdt(off, nodes, base)
+    m = re.search(r"chunks=(\d+) chunk_trees=(\d+)", model.describe())
+    assert "block=1024" in model.describe() and m, model.describe()
+    n_chunks, tpc = int(m.group(1)), int(m.group(2))
+    assert n_chunks >= 2
+    part = [oracle.score_gbdt(x, off[c * tpc:(c + 1) * tpc + 1] - off[c * tpc],
+                              nodes[off[c * tpc]:off[(c + 1) * tpc]], 0.0) for c in (0, 1)]
+    d_x = dev(ks, x)
+    for repeat in (1, 3):
+        n = repeat * n_chunks
+        got = ctx.debug_walk_floor(d_x, model, repeat).cpu().numpy()
+        want = base + ((n + 1) // 2) * part[0].astype(np.float64) + (n // 2) * part[1].astype(np.float64)
+        assert np.all(np.abs(got - want) <= 4 * TOL_GBDT * n * np.maximum(1, np.abs(want)))
+    assert np.std(part[0]) > 1e-2
+    # an ensemble in another tile geometry or shape is refused
+    w2 = wl.make_workload(0, P=1, C=300)
+    model2 = ctx.model_create_gbdt(*w2.gbdt)
+    with pytest.raises(ks.KsError) as e:
+        ctx.debug_walk_floor(dev(ks, oracle.featurize(w2.problems, w2.candidates, DESC)), model2, 2)
+    assert e.value.status == ks.KS_ERR_UNSUPPORTED
+
+
 def test_score_mlp(ks, ctx):
     w = wl.make_workload(4, P=3, C=411)
     x = oracle.featurize(w.problems, w.candidates, DESC)
