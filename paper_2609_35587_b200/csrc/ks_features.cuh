@@ -305,25 +305,34 @@ __device__ __forceinline__ float static_score(const ProblemTerms& t, const ks_ca
   return __fmul_rn(s, __fsqrt_rn(F64i(TM * TN * TK)));
 }
 
-// Writes the 64 columns of one pair through `put(column, value)`.
+// The columns that depend on the problem alone (class 0 of feat_class), straight from its terms.
 template <typename Put>
-__device__ __forceinline__ void featurize_pair(const ProblemTerms& t, const ks_candidate& c,
-                                               const ks_gpu_desc& h, Put put) {
-  const int TM = c.tile_m, TN = c.tile_n, TK = c.tile_k, S = c.stages;
-  const int cM = c.cluster_m, cN = c.cluster_n;
-  const int bA = t.bA, bD = t.bD;
-
-  // ---- structural core ------------------------------------------------------------------
+__device__ __forceinline__ void problem_columns(const ProblemTerms& t, Put put) {
   put(0, t.log2m);
   put(1, t.log2n);
   put(2, t.log2k);
   put(3, F32i(t.layout == 2 || t.layout == 3));
   put(4, F32i(t.layout == 1 || t.layout == 3));
   put(5, F32i(t.dtype_ab));
-  put(6, F32i(bA));
-  put(7, F32i(bD));
+  put(6, F32i(t.bA));
+  put(7, F32i(t.bD));
   put(8, F32i(t.has_bias));
   put(9, F32i(t.act));
+  put(37, t.i_problem);
+  put(40, t.ws_frac_l2);
+  put(45, t.f_traffic_epi);
+}
+
+// Writes the 64 columns of one pair through `put(column, value)`.
+template <typename Put>
+__device__ __forceinline__ void featurize_pair(const ProblemTerms& t, const ks_candidate& c,
+                                               const ks_gpu_desc& h, Put put) {
+  const int TM = c.tile_m, TN = c.tile_n, TK = c.tile_k, S = c.stages;
+  const int cM = c.cluster_m, cN = c.cluster_n;
+  const int bA = t.bA;
+
+  // ---- structural core ------------------------------------------------------------------
+  problem_columns(t, put);
   put(10, F32i(TM));
   put(11, F32i(TN));
   put(12, F32i(TK));
@@ -341,11 +350,8 @@ __device__ __forceinline__ void featurize_pair(const ProblemTerms& t, const ks_c
   const Resources r = resources(t, c, h);
   pair_columns<true>(t, c, h, r.b_eff, put);
 
-  // ---- memory behaviour (problem-only and candidate-only columns) ---------------------------
-  put(37, t.i_problem);
+  // ---- memory behaviour (candidate-only column) -----------------------------------------------
   put(38, __fdiv_rn(F64i(2 * r.area), F64i(static_cast<long long>(TM) * bA + static_cast<long long>(TN) * bA)));
-  put(40, t.ws_frac_l2);
-  put(45, t.f_traffic_epi);
 
   // ---- resource pressure columns ------------------------------------------------------------
   put(46, F64i(r.B_stage));

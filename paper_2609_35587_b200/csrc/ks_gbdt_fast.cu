@@ -229,7 +229,10 @@ __global__ void combo_mask_kernel(const ks_problem* __restrict__ p, int P, unsig
 __device__ __forceinline__ const float* stage_thresholds(const FastView& fv, int first, int count, float* s_thr,
                                                          int cap) {
   if (count > cap) return fv.thr + first;
-  for (int i = threadIdx.x; i < count; i += blockDim.x) s_thr[i] = __ldg(fv.thr + first + i);
+  const int vec = (first & 3) == 0 ? count / 4 : 0;  // whole 16-byte words when the source is aligned like s_thr
+  for (int i = threadIdx.x; i < vec; i += blockDim.x)
+    reinterpret_cast<float4*>(s_thr)[i] = __ldg(reinterpret_cast<const float4*>(fv.thr + first) + i);
+  for (int i = 4 * vec + threadIdx.x; i < count; i += blockDim.x) s_thr[i] = __ldg(fv.thr + first + i);
   return s_thr;
 }
 
@@ -316,14 +319,7 @@ pair_table_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_problem
     __syncthreads();  // the previous problem's terms are no longer read (and the staging is complete)
     if (tid == 0) {
       problem_terms(pr, desc, s_pt);
-      if (last_x) {
-        ks_candidate dummy{};
-        dummy.tile_m = dummy.tile_n = dummy.tile_k = 64;
-        dummy.stages = dummy.cluster_m = dummy.cluster_n = 1;
-        featurize_pair(s_pt, dummy, desc, [&](int col, float v) {
-          if (col < KS_F && feat_class(col) == 0) s_pf[col] = v;
-        });
-      }
+      if (last_x) problem_columns(s_pt, [&](int col, float v) { s_pf[col] = v; });
     }
     __syncthreads();
     if (last_x) {
@@ -713,15 +709,7 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
   if (tid == 0) {
     if (!tiles_given && !fv.prob_tab) {
       problem_terms(use_value ? p_value : load_problem(p + prob), desc, s_pt);
-      {
-        // problem-only columns do not look at the candidate: evaluate them on a dummy one
-        ks_candidate dummy{};
-        dummy.tile_m = dummy.tile_n = dummy.tile_k = 64;
-        dummy.stages = dummy.cluster_m = dummy.cluster_n = 1;
-        featurize_pair(s_pt, dummy, desc, [&](int col, float v) {
-          if (feat_class(col) == 0) s_pfeat[col] = v;
-        });
-      }
+      problem_columns(s_pt, [&](int col, float v) { s_pfeat[col] = v; });
     }
     s_abort = *reinterpret_cast<volatile int*>(&g_fast_abort);
   }
@@ -982,30 +970,32 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
   if (tid < k)
     partial[KS_IDX((static_cast<size_t>(prob) * nblk + chunk) * k + tid, static_cast<size_t>(P) * nblk * k)] = s_list[tid];
   if (S > 1 && sl.out_idx) {
-    // single-problem form: the last block to finish merges the per-block lists (one warp)
+    // single-problem form: the last block to finish merges the per-block lists
     __threadfence();
     __syncthreads();
     if (tid == 0) s_last = atomicAdd(sl.counters + nblk, 1) == nblk - 1;
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    if (tid < 32) {
-      const int n_keys = nblk * k;
-      unsigned long long prev = ~0ull;
-      for (int j = 0; j < k; ++j) {
-        unsigned long long best = 0ull;
-        for (int i = tid; i < n_keys; i += 32) {
-          const unsigned long long v = __ldcg(partial + i);
-          if (v < prev && v > best) best = v;
-        }
-        best = warp_max_u64(best);
-        if (tid == 0) {
-          sl.out_idx[j] = key_index(best);
-          sl.out_score[j] = key_score(best);
-        }
-        prev = best;
-      }
+    // the whole CTA ranks the nblk * k keys (each key is read once)
+    const int n_keys = nblk * k;
+    __syncthreads();
+    if (tid < KS_MAX_K) s_list[tid] = 0ull;
+    for (int base = 0; base < n_keys; base += 2 * THREADS) {
+      unsigned long long keys[3];
+      keys[0] = base + tid < n_keys ? __ldcg(partial + base + tid) : 0ull;
+      keys[1] = base + THREADS + tid < n_keys ? __ldcg(partial + base + THREADS + tid) : 0ull;
+      __syncthreads();
+      keys[2] = tid < k ? s_list[tid] : 0ull;
+      __syncthreads();
+      block_topk<3>(keys, k, s_warp, s_list);
     }
+    if (tid < k) {
+      sl.out_idx[tid] = key_index(s_list[tid]);
+      sl.out_score[tid] = key_score(s_list[tid]);
+      __threadfence_system();
+    }
+    __syncthreads();
     if (tid == 0) {
       sl.counters[nblk] = 0;
       if (sl.out_seq) {  // the results are in place: tell the host, which polls this word

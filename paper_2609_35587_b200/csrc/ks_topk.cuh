@@ -53,9 +53,11 @@ __device__ __forceinline__ void warp_topk_insert(unsigned long long& mine, unsig
 }
 
 // The k largest of the block's keys (N per thread), descending, into s_list[0..k).
-// Two levels: every warp first ranks its own keys (k rounds of warp-wide max, no block
-// barrier), then warp 0 ranks the n_warps * k survivors. All threads of the block must call;
-// s_warp needs n_warps * KS_MAX_K slots.
+// Two levels: every warp first ranks its own keys (k rounds of warp-wide max, no block barrier;
+// a warp that runs out of keys stops), then warp 0 merges the warps' sorted lists: lane w holds
+// the head of warp w's list, a round takes the largest head and its lane moves on to the next
+// entry. Equal keys (the same candidate listed twice) leave in the same round, so they are
+// reported once. All threads of the block must call; s_warp needs n_warps * KS_MAX_K slots.
 template <int N>
 __device__ __forceinline__ void block_topk(const unsigned long long (&keys)[N], int k,
                                            unsigned long long* s_warp, unsigned long long* s_list) {
@@ -69,22 +71,28 @@ __device__ __forceinline__ void block_topk(const unsigned long long (&keys)[N], 
       if (v < prev && v > best) best = v;
     }
     best = warp_max_u64(best);
+    if (best == 0ull) {  // nothing left in this warp
+      if (lane < k - j) s_warp[warp * k + j + lane] = 0ull;
+      break;
+    }
     if (lane == 0) s_warp[warp * k + j] = best;
     prev = best;
   }
   __syncthreads();
   if (warp == 0) {
-    const int n = n_warps * k;
-    prev = ~0ull;
+    int next = 1;
+    unsigned long long head = lane < n_warps ? s_warp[lane * k] : 0ull;
     for (int j = 0; j < k; ++j) {
-      unsigned long long best = 0ull;
-      for (int i = lane; i < n; i += 32) {
-        const unsigned long long v = s_warp[i];
-        if (v < prev && v > best) best = v;
+      const unsigned long long m = warp_max_u64(head);
+      if (lane == 0) s_list[j] = m;
+      if (m == 0ull) {
+        if (lane > j && lane < k) s_list[lane] = 0ull;
+        break;
       }
-      best = warp_max_u64(best);
-      if (lane == 0) s_list[j] = best;
-      prev = best;
+      if (head == m) {
+        head = next < k ? s_warp[lane * k + next] : 0ull;
+        ++next;
+      }
     }
   }
   __syncthreads();
