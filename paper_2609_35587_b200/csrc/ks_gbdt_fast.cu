@@ -153,10 +153,10 @@ __device__ __forceinline__ int count_le(const float* T, int n, float v) {
 // thresholds that are <= v, i.e. the overall count less 127 s clamped to 0..127; a rank row gets
 // the rank of the level code v. `T` is the feature's own sorted threshold array. With
 // `nan_right` a NaN takes the last bin of every slice (x < t is false: it goes right).
+// `pos` is the count of the feature's thresholds that are <= v (unused for a feature without slices).
 template <typename Put>
-__device__ __forceinline__ void quantise(const FeatQ& q, const float* T, float v, bool nan_right, Put put) {
+__device__ __forceinline__ void emit_rows(const FeatQ& q, int pos, float v, Put put) {
   if (q.nslice) {
-    const int pos = (nan_right && v != v) ? q.nthr : count_le(T, q.nthr, v);
     for (int s = 0; s < q.nslice; ++s) {
       int b = pos - kSlice * s;
       b = b < 0 ? 0 : (b > kSlice ? kSlice : b);
@@ -168,6 +168,51 @@ __device__ __forceinline__ void quantise(const FeatQ& q, const float* T, float v
     for (int r = 0; r < q.nrank; ++r)
       put(q.row0 + q.nslice + r, static_cast<uint8_t>(0x80 | ((code >= 0 && code < 4) ? q.rank[r][code] : 0)));
   }
+}
+template <typename Put>
+__device__ __forceinline__ void quantise(const FeatQ& q, const float* T, float v, bool nan_right, Put put) {
+  const int pos = q.nslice ? ((nan_right && v != v) ? q.nthr : count_le(T, q.nthr, v)) : 0;
+  emit_rows(q, pos, v, put);
+}
+
+// The per-pair columns (class 2 of feat_class) in ascending order, and a column's place among them.
+constexpr int kPairCols = 21;
+__host__ __device__ constexpr int pair_slot(int col) {
+  return col <= 36 ? col - 23 : (col == 39 ? 14 : (col <= 44 ? col - 26 : col - 41));
+}
+__host__ __device__ constexpr int pair_col(int slot) {
+  return slot <= 13 ? slot + 23 : (slot == 14 ? 39 : (slot <= 18 ? slot + 26 : slot + 41));
+}
+constexpr bool pair_slots_match_classes() {
+  int n = 0;
+  for (int c = 0; c < KS_F; ++c)
+    if (feat_class(c) == 2) {
+      if (pair_slot(c) != n || pair_col(n) != c) return false;
+      ++n;
+    }
+  return n == kPairCols;
+}
+static_assert(pair_slots_match_classes(), "per-pair columns");
+
+// All per-pair columns of one pair at once: the binary searches advance in step (one probe of
+// every column per round), so that a thread has 21 independent loads in flight instead of one
+// dependent chain after the other. `T` is the staged (or global) array of per-pair thresholds.
+template <typename Put>
+__device__ __forceinline__ void quantise_pair_columns(const FeatQ* s_fq, const float* T, const float (&v)[kPairCols],
+                                                      int max_thr, Put put) {
+  int pos[kPairCols];
+#pragma unroll
+  for (int i = 0; i < kPairCols; ++i) pos[i] = 0;
+  for (int s = max_thr > 0 ? 1 << (31 - __clz(max_thr)) : 0; s >= 1; s >>= 1) {
+#pragma unroll
+    for (int i = 0; i < kPairCols; ++i) {
+      const FeatQ& q = s_fq[pair_col(i)];
+      const int np = pos[i] + s;
+      if (np <= q.nthr && T[q.thr0 + np - 1] <= v[i]) pos[i] = np;
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < kPairCols; ++i) emit_rows(s_fq[pair_col(i)], pos[i], v[i], put);
 }
 
 // Byte of row i (0 .. 4 W - 1) of a block within one tile row of W words: the four rows of a
@@ -312,6 +357,7 @@ pair_table_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_problem
   uint8_t* my_rec = reinterpret_cast<uint8_t*>(s_pthr + (thr_cap > 0 ? (thr_cap + 3) / 4 * 4 : 0)) +
                     static_cast<size_t>(tid) * fv.pair_rec;
   if (tid < 64) s_fq[tid] = fv.feat[tid];
+  int max_thr = -1;  // the longest threshold list among the per-pair columns (found after the first barrier)
   for (int prob = blockIdx.y; prob < n_prob; prob += gridDim.y) {
     const ks_problem pr = use_value ? p_value : load_problem(p + prob);
     const int combo = (pr.dtype_ab & 3) * 4 + (pr.dtype_d & 3);
@@ -335,13 +381,17 @@ pair_table_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_problem
         reinterpret_cast<uint32_t*>(out + kFastMaxProbRows)[tid] = reinterpret_cast<const uint32_t*>(&s_pt)[tid];
     }
     if (j >= n_classes) continue;
+    if (max_thr < 0) {
+      max_thr = 0;
+#pragma unroll
+      for (int i = 0; i < kPairCols; ++i) max_thr = max(max_thr, static_cast<int>(s_fq[pair_col(i)].nthr));
+    }
     const int slot = memo.dense[static_cast<size_t>(combo) * kMemoCap + j];
     const ks_candidate cand = load_candidate(c + memo.reps[static_cast<size_t>(combo) * kMemoCap + slot]);
     const long long b_eff = resources(s_pt, cand, desc).b_eff;
-    pair_columns<true>(s_pt, cand, desc, b_eff, [&](int col, float v) {
-      const FeatQ& q = s_fq[col];
-      quantise(q, T + q.thr0, v, false, [&](int row, uint8_t b) { my_rec[KS_IDX(row, fv.pair_rec)] = b; });
-    });
+    float vals[kPairCols];
+    pair_columns<true>(s_pt, cand, desc, b_eff, [&](int col, float v) { vals[pair_slot(col)] = v; });
+    quantise_pair_columns(s_fq, T, vals, max_thr, [&](int row, uint8_t b) { my_rec[KS_IDX(row, fv.pair_rec)] = b; });
     // the record leaves as whole 16-byte words (it is a multiple of 16 bytes, and so is its place)
     uint4* dst = reinterpret_cast<uint4*>(static_cast<uint8_t*>(memo.tab) +
                                           (static_cast<size_t>(prob) * kMemoCap + slot) * fv.pair_rec);
