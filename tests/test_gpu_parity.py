@@ -625,6 +625,26 @@ def test_select_forced_tile_geometry(ks, ctx, geometry, monkeypatch):
     assert np.array_equal(hi_.numpy(), idx[1])
 
 
+@pytest.mark.parametrize("geometry,segments", [("512,1024,32", False), ("512,512,16", False), ("512,512,32", True)])
+def test_select_more_items_than_sms(ks, ctx, geometry, segments, monkeypatch):
+    """The one-CTA-per-SM geometries launch one CTA per SM and let it serve many (problem,
+    candidate block) items: here 330 to 660 items, not a multiple of the 148 CTAs, so that some
+    CTAs take one item more than others, with a ragged last block per problem; dense catalogue
+    (ranked in similarity order) and per-problem segments."""
+    monkeypatch.setenv("KS_FAST_GEOMETRY", geometry)
+    if segments:
+        w = wl.make_workload(2, P=110, seg=1300, trees=24, depth=8, law="pernode")
+    else:
+        w = wl.make_workload(1, P=110, C=2700, trees=24, depth=8, law="pernode")
+    model = ctx.model_create_gbdt(*w.gbdt)
+    t, c, _ = geometry.split(",")
+    assert f"threads={t} block={c}" in model.describe(), model.describe()
+    idx, sc = run_select(ks, ctx, w, model)
+    check_select(w, idx, sc, TOL_GBDT, sample=range(0, 110, 2))
+    idx2, sc2 = run_select(ks, ctx, w, model)     # the barriers' parities carry over from call to call
+    assert np.array_equal(idx, idx2) and np.array_equal(sc, sc2)
+
+
 @pytest.mark.parametrize("law", ["slots128", "pernode"])
 def test_select_one_prepared_catalogue(ks, ctx, law):
     """The single-problem call against a prepared catalogue (candidate-only rows and classes made
