@@ -408,12 +408,18 @@ def walk_floor(ks, ctx, w, model, dev):
     """The tree walk stripped to its gather and instruction stream (ks_debug_walk_floor): feature
     rows of the workload's first problems, 592 blocks of 1,024 rows (whole waves of 148 or 296
     CTAs); the time of one pass over the ensemble is the difference of two calls that differ in
-    their number of passes only, so tile building, launches and the first copies cancel."""
+    their number of passes only, so tile building, launches and the first copies cancel. The rows
+    are those of the catalogue in similarity order, as the product kernel's tiles are."""
     import torch
     rows = 592 * 1024
     C = len(w.candidates)
     P = -(-rows // C)
-    d_p, d_c = ks.to_device(w.problems[:P], dev), ks.to_device(w.candidates, dev)
+    # the catalogue in the similarity order the product ranks it in (the same sort keys), so that a
+    # warp's lanes hold neighbouring candidates here as they do there
+    c = w.candidates
+    order = np.lexsort((c["instr_n"] != c["tile_n"], c["tile_sched"], c["epi_sched"], c["kernel_sched"],
+                        c["cluster_n"], c["cluster_m"], c["stages"], c["tile_k"], c["tile_n"], c["tile_m"]))
+    d_p, d_c = ks.to_device(w.problems[:P], dev), ks.to_device(np.ascontiguousarray(c[order]), dev)
     feat = ctx.featurize(d_p, P, d_c, C)[:rows]
     out = torch.empty(rows, dtype=torch.float32, device=dev)
     lo, hi = 2, 10
@@ -543,6 +549,8 @@ def main():
                     help="measure the search-space enumeration + validity filter instead of a selection workload")
     ap.add_argument("--stages", action="store_true",
                     help="time the unfused calls (ks_featurize, ks_score) one at a time instead of ks_select")
+    ap.add_argument("--floor", action="store_true",
+                    help="measure the tree walk's gather stream alone (ks_debug_walk_floor) on config 1's ensemble")
     args = ap.parse_args()
 
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
@@ -564,13 +572,23 @@ def main():
     dev = torch.device("cuda", local_rank)
     cfg = args.workload
     spec = wl.CONFIGS[cfg]
-    if world > 1 and cfg != 3 and not args.catalogue and not args.stages:
+    if world > 1 and cfg != 3 and not args.catalogue and not args.stages and not args.floor:
         dist.init_process_group("nccl", device_id=dev)
     if args.catalogue:
         run_catalogue(args, rank, local_rank, dev)
         return
     if args.stages:
         run_stages(args, rank, local_rank, dev)
+        return
+    if args.floor:
+        if rank == 0:
+            w = wl.make_workload(1, P=12, law=args.law)
+            ctx = ks.Context(w.desc, local_rank)
+            model = ctx.model_create_gbdt(*w.gbdt)
+            f = walk_floor(ks, ctx, w, model, dev)
+            print(json.dumps({"metric": "tree walk, gather stream alone (fraction of the issue roofline)", "value": f["frac"],
+                              "unit": "fraction", "n_gpus": 1, "higher_is_better": True, "data": "synthetic",
+                              "config": {"workload": f"config 1 ensemble, thresholds: {args.law}", **f}}), flush=True)
         return
     if cfg == 3:
         run_latency_stream(args, rank, local_rank, dev)
