@@ -246,7 +246,9 @@ ks_status ks_remap_indices(ks_ctx* ctx, int32_t* d_idx, int64_t n, const int32_t
 /* Candidate sets: with d_seg_offsets == NULL every problem is ranked against the whole pool
  * d_c[0..C) (dense P x C; pairs = P*C, pair (i, j) is row i*C + j). Otherwise problem i is
  * ranked against d_c[d_seg_index[j]] for j in [d_seg_offsets[i], d_seg_offsets[i+1])
- * (d_seg_offsets has P+1 non-decreasing entries starting at 0; row j belongs to pair j). */
+ * (d_seg_offsets has P+1 non-decreasing entries starting at 0; row j belongs to pair j).
+ * A problem's candidate set is a set: the indices of one segment must be distinct (for the
+ * ranking calls; an index listed twice is reported once by some kernels and twice by others). */
 
 /* x = phi(p, c, h) for every pair (Table "Feature groups"; the column list is
  * ks_feature_name). Writes pairs x 64 fp32, row-major. `pairs` must equal P*C or
