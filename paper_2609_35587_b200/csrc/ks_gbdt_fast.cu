@@ -1592,6 +1592,31 @@ cudaError_t fast_prepare(const ks_gpu_desc& desc, const GbdtModel& g, const ks_c
   return cudaGetLastError();
 }
 
+// Problems per launch when a call is served in batches of at most `cap`. In the launch form
+// with one CTA per SM every launch runs its items in rounds of kSmCount, and a last round that
+// is nearly empty still takes a whole item's time; a batch a little below the cap can save a
+// round per launch (4,096 problems x 32 blocks in batches of 226 instead of 227: 889 rounds
+// instead of 903: 134.9 -> 130.7 ms). Picks the size within an eighth below the cap that needs
+// the fewest rounds. (With two CTAs per SM, one per item, the hardware hands out the items and
+// the same rule measured 0.6 % slower: not applied there.)
+static int balanced_step(const GbdtModel& g, int P, int cap, int nblk) {
+  if (P <= cap || g.ctas_per_sm != 1 || cap < 16) return cap;
+  int best = cap;
+  int64_t best_rounds = INT64_MAX;
+  for (int n = cap; n >= cap - cap / 8; --n) {
+    int64_t rounds = 0;
+    for (int first = 0; first < P; first += n) {
+      const int64_t items = static_cast<int64_t>(P - first < n ? P - first : n) * nblk;
+      rounds += (items + kSmCount - 1) / kSmCount;
+    }
+    if (rounds < best_rounds) {
+      best_rounds = rounds;
+      best = n;
+    }
+  }
+  return best;
+}
+
 cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, const ks_problem* d_p,
                                const ks_problem* p_by_value, int P, const ks_candidate* d_c, int C,
                                int nblk, int rows_per_cta, const int64_t* seg_off, const int32_t* seg_idx,
@@ -1712,7 +1737,7 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
     a.sl.seq = slice->seq;
   }
   // problems in batches when the memo's table does not hold them all at once
-  const int step = memo.keys ? memo_batch : P;
+  const int step = memo.keys ? balanced_step(g, P, memo_batch, nblk) : P;
   for (int first = 0; first < P; first += step) {
     const int n = P - first < step ? P - first : step;
     if (memo.keys) {
