@@ -344,31 +344,37 @@ pair_table_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_problem
   __shared__ ProblemTerms s_pt;
   __shared__ FeatQ s_fq[64];
   __shared__ float s_pf[64];
-  const int tid = threadIdx.x, j = blockIdx.x * 256 + tid;
-  const bool last_x = blockIdx.x == gridDim.x - 1;
+  const int tid = threadIdx.x;
   // the select kernel that follows may start its own set-up now (it waits for this grid to finish
   // before it reads the tables)
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  if (blockIdx.x == 0 && blockIdx.y == 0 && tid == 0) g_fast_abort = 0;  // (also) precedes the select kernel
+  if (blockIdx.x == 0 && tid == 0) g_fast_abort = 0;  // (also) precedes the select kernel
   int most = 0;
   for (int q = 0; q < kMemoCombos; ++q) most = max(most, memo.count[q]);
-  if (blockIdx.x * 256 >= most && !last_x) return;
+  // An item is (block of 256 classes, problem); the blocks of the grid deal the items among
+  // themselves, so that the work is even whatever the number of classes. The item of class
+  // block 0 also writes its problem's own record (problem-only rows and terms).
+  const int class_blocks = most > 0 ? (most + 255) / 256 : 1;
+  const int n_items = class_blocks * n_prob;
+  if (static_cast<int>(blockIdx.x) >= n_items) return;
   const float* T = stage_thresholds(fv, 0, fv.thr_cand0, s_pthr, thr_cap);
   uint8_t* my_rec = reinterpret_cast<uint8_t*>(s_pthr + (thr_cap > 0 ? (thr_cap + 3) / 4 * 4 : 0)) +
                     static_cast<size_t>(tid) * fv.pair_rec;
   if (tid < 64) s_fq[tid] = fv.feat[tid];
   int max_thr = -1;  // the longest threshold list among the per-pair columns (found after the first barrier)
-  for (int prob = blockIdx.y; prob < n_prob; prob += gridDim.y) {
+  for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+    const int prob = item / class_blocks, j = (item % class_blocks) * 256 + tid;
+    const bool first_block = item % class_blocks == 0;
     const ks_problem pr = use_value ? p_value : load_problem(p + prob);
     const int combo = (pr.dtype_ab & 3) * 4 + (pr.dtype_d & 3);
     const int n_classes = memo.count[combo];
-    __syncthreads();  // the previous problem's terms are no longer read (and the staging is complete)
+    __syncthreads();  // the previous item's terms are no longer read (and the staging is complete)
     if (tid == 0) {
       problem_terms(pr, desc, s_pt);
-      if (last_x) problem_columns(s_pt, [&](int col, float v) { s_pf[col] = v; });
+      if (first_block) problem_columns(s_pt, [&](int col, float v) { s_pf[col] = v; });
     }
     __syncthreads();
-    if (last_x) {
+    if (first_block) {
       // once per problem, for all its CTAs: the problem-only rows and the problem's terms
       uint8_t* out = const_cast<uint8_t*>(fv.prob_tab) + static_cast<size_t>(prob) * kProbRec;
       if (tid < KS_F && feat_class(tid) == 0) {
@@ -1596,7 +1602,7 @@ cudaError_t fast_prepare(const ks_gpu_desc& desc, const GbdtModel& g, const ks_c
 // with one CTA per SM every launch runs its items in rounds of kSmCount, and a last round that
 // is nearly empty still takes a whole item's time; a batch a little below the cap can save a
 // round per launch (4,096 problems x 32 blocks in batches of 226 instead of 227: 889 rounds
-// instead of 903: 134.9 -> 130.7 ms). Picks the size within an eighth below the cap that needs
+// instead of 903: 133.3 -> 130.7 ms). Picks the size within an eighth below the cap that needs
 // the fewest rounds. (With two CTAs per SM, one per item, the hardware hands out the items and
 // the same rule measured 0.6 % slower: not applied there.)
 static int balanced_step(const GbdtModel& g, int P, int cap, int nblk) {
@@ -1741,7 +1747,12 @@ cudaError_t launch_select_fast(const ks_gpu_desc& desc, const GbdtModel& g, cons
   for (int first = 0; first < P; first += step) {
     const int n = P - first < step ? P - first : step;
     if (memo.keys) {
-      pair_table_kernel<<<dim3(kMemoCap / 256, n < 32 ? n : 32), 256, pthr_bytes, stream>>>(
+      // as many blocks as the machine holds at once (two per SM by registers, fewer when the staged
+      // thresholds take more than half an SM's shared memory); never more blocks than items
+      const int64_t table_items = static_cast<int64_t>(kMemoCap / 256) * n;
+      const int64_t table_slots = static_cast<int64_t>(kSmCount) * (2 * (pthr_bytes + 4096) <= 227 * 1024 ? 2 : 1);
+      pair_table_kernel<<<static_cast<unsigned>(table_items < table_slots ? table_items : table_slots), 256, pthr_bytes,
+                          stream>>>(
           desc, d_p ? d_p + first : nullptr, a.pv, a.uv, n, d_c, fv, memo, pthr_cap);
       ++*launches;
     }
