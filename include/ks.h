@@ -401,10 +401,12 @@ ks_status ks_debug_set_wait(ks_ctx* ctx, int probe_limit, int starve);
 /* Measurement aid, no counterpart in the paper: the tree walk of ks_score stripped of everything
  * but its gather and instruction stream, to measure the floor that stream sets for the tree
  * kernel. Tiles are built from the `rows` feature rows (device, [rows][64] floats) exactly as
- * ks_score builds them; every CTA then copies the first two chunks of the ensemble once and
- * walks them `repeat` x n_chunks times (as many chunk walks as `repeat` passes over the whole
- * ensemble) without waiting for, releasing or refilling a chunk buffer, and stores the sums it
- * accumulated to d_scores (device, [rows]; with c0, c1 the sums of the two chunks' leaves for a
+ * ks_score builds them; every CTA then copies the first chunks of the ensemble once (two per
+ * tree group: the CTA's threads / 256 groups deal the chunks among themselves, group g taking
+ * chunks g, g + G, ...) and every group walks its two resident chunks as often as `repeat` passes
+ * over the whole ensemble would make it walk chunks, without waiting for, releasing or refilling
+ * a chunk buffer; the sums go to d_scores (device, [rows]; with one group, c0 and c1 the sums of
+ * the two chunks' leaves for a
  * row and n = repeat x n_chunks: base + ceil(n / 2) c0 + floor(n / 2) c1). The time of a pass is
  * the difference of two calls with different `repeat`, divided by the difference. Tree models on
  * the quantised kernel with 1,024-candidate tiles, three word-wise and five path levels only

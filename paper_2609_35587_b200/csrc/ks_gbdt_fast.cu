@@ -67,6 +67,12 @@ constexpr int kCombos = 16;            // dtype_ab x dtype_d
 
 // shared memory map (byte offsets from the dynamic shared base): the chunk buffers, then the tile
 constexpr int kSmCount = 148;           // SMs of the one device this library is built for (sm_100a)
+// Chunk rings of a CTA with G tree groups: every ring has kNBuf buffers and serves G / rings groups,
+// which share out the trees of its chunks; ring r takes the chunks r, r + rings, ... A ring of
+// its own per group means that only the group's warps meet at a buffer's release, for the same
+// shared memory and the same trees per thread and chunk (config 1, two groups: 55.3 -> 54.4 ms);
+// four groups do best with two rings (config 2: 132.4 ms with four rings, 131.6 with one, 129.3 with two).
+__host__ __device__ constexpr int ring_count(int groups) { return groups <= 2 ? groups : 2; }
 constexpr int kNBuf = 2;                // tree-chunk buffers (a ring; four of 8 KB and three of 12 KB measured slower)
 constexpr int kOffBuf0 = 0;
 
@@ -693,10 +699,11 @@ __device__ __forceinline__ uint32_t path_step(uint32_t a, uint32_t cb_r, uint32_
 // levels' constants travel as one 32-bit word per node (row offset << 8 | j + 1) instead of a
 // (row offset, replicated j + 1) pair, so that twice as many trees keep their word-wise levels.
 // THREADS threads rank NC candidates: NC / 4 words times THREADS / (NC / 4) tree groups.
-// kFloor (measurement only): the walk without its chunk ring. The first kNBuf chunks are copied
-// once and stay resident; the CTA walks them again and again (sl.repeat passes of n_chunks chunk
-// walks each), never waits, releases or refills, so the time per pass is that of the gather and
-// instruction stream of the walk alone, at the occupancy and tile size of the real kernel.
+// kFloor (measurement only): the walk without its chunk rings. Every tree group's first kNBuf
+// chunks are copied once and stay resident; the group walks them again and again (sl.repeat
+// times as many chunk walks as it has chunks), never waits, releases or refills, so the time per
+// pass is that of the gather and instruction stream of the walk alone, at the occupancy and tile
+// size of the real kernel.
 template <int L, int NP, bool kCompact, int THREADS, int NC, bool kFloor = false>
 __global__ void __launch_bounds__(THREADS, THREADS <= 256 ? 2 : 1)
 select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_problem p_value, int use_value,
@@ -706,27 +713,29 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
                    SliceArgs sl, int n_items, const __grid_constant__ FastTopParams top) {
   constexpr int W = NC / 4;        // words per tile row = lane slots
   constexpr int G = THREADS / W;   // tree groups
+  constexpr int RG = ring_count(G);  // chunk rings
+  constexpr int GPR = G / RG;        // groups that share a ring (and split the trees of its chunks)
   static_assert(THREADS % W == 0 && W % 32 == 0 && G >= 1, "tile geometry");
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ ProblemTerms s_pt;
   __shared__ unsigned long long s_warp[THREADS / 32 * KS_MAX_K];
   __shared__ unsigned long long s_list[KS_MAX_K];
-  __shared__ __align__(8) unsigned long long s_bar[kNBuf];
+  __shared__ __align__(8) unsigned long long s_bar[kNBuf * RG];  // [ring][buffer]
   __shared__ FeatQ s_fq[64];
   __shared__ uint8_t s_pbin[kFastMaxProbRows];
   __shared__ float s_pfeat[64];
-  __shared__ int s_fail, s_last, s_done[kNBuf], s_abort, s_pending[kNBuf];
+  __shared__ int s_fail, s_last, s_done[kNBuf * RG], s_abort, s_pending[kNBuf * RG];
 
   const int tid = threadIdx.x;
-  const int kOffTile = kNBuf * fv.buf_bytes;
+  const int kOffTile = kNBuf * RG * fv.buf_bytes;  // every ring has kNBuf buffers
   const int S = sl.n_slices;
   const uint32_t sbase = smem_u32(smem);
   const uint32_t bar0 = smem_u32(&s_bar[0]);  // barrier of buffer b: bar0 + 8 b
   const bool tiles_given = sl.tiles != nullptr;  // the tiles were built in front: no feature work here
   if (tid == 0) {
-    for (int b = 0; b < kNBuf; ++b) mbar_init(bar0 + 8u * b, 1);
+    for (int b = 0; b < kNBuf * RG; ++b) mbar_init(bar0 + 8u * b, 1);
     s_fail = 0;
-    for (int b = 0; b < kNBuf; ++b) s_done[b] = s_pending[b] = 0;
+    for (int b = 0; b < kNBuf * RG; ++b) s_done[b] = s_pending[b] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (tid < 64) s_fq[tid] = fv.feat[tid];
@@ -801,7 +810,7 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
     } else {
       // thresholds of the per-pair features: into the idle chunk buffers when they fit
       const float* T = stage_thresholds(fv, 0, fv.thr_cand0, reinterpret_cast<float*>(smem + kOffBuf0),
-                                        fv.pair_class ? 0 : kNBuf * fv.buf_bytes / 4);
+                                        fv.pair_class ? 0 : kNBuf * RG * fv.buf_bytes / 4);
       __syncthreads();
       fill_tile<THREADS, NC>(desc, s_pt, c, fv, seg_off, seg_idx, C, lo_idx, start, stop, T, s_fq, s_pbin,
                              smem + kOffTile, prob);
@@ -811,37 +820,44 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
     // ---- phase B ---------------------------------------------------------------------------------
     if (tid == 0) {
       fence_async_proxy();
-      const char* src = reinterpret_cast<const char*>(fv.chunks) + static_cast<size_t>(ch_begin) * fv.chunk_bytes;
-      for (int b = 0; b < kNBuf && ch_begin + b < ch_end; ++b) {
-        // test hook: a barrier armed for more bytes than its copy brings never completes
-        mbar_expect_tx(bar0 + 8u * b, fv.chunk_bytes + (fv.starve ? 16 : 0));
-        bulk_copy_g2s(sbase + kOffBuf0 + b * fv.buf_bytes, src + static_cast<size_t>(b) * fv.chunk_bytes,
-                      fv.chunk_bytes, bar0 + 8u * b);
-        s_pending[b] = 1;
-      }
+      // ring g takes the chunks ch_begin + g, ch_begin + g + RG, ... through its own buffers
+      for (int g = 0; g < RG; ++g)
+        for (int b = 0; b < kNBuf && ch_begin + g + b * RG < ch_end; ++b) {
+          const int rb = g * kNBuf + b;
+          // test hook: a barrier armed for more bytes than its copy brings never completes
+          mbar_expect_tx(bar0 + 8u * rb, fv.chunk_bytes + (fv.starve ? 16 : 0));
+          bulk_copy_g2s(sbase + kOffBuf0 + rb * fv.buf_bytes,
+                        reinterpret_cast<const char*>(fv.chunks) + static_cast<size_t>(ch_begin + g + b * RG) * fv.chunk_bytes,
+                        fv.chunk_bytes, bar0 + 8u * rb);
+          s_pending[rb] = 1;
+        }
     }
     float score[4] = {0.0f, 0.0f, 0.0f, 0.0f};
     const uint32_t cb = sbase + kOffTile + word * 4;
-    const int tpc = fv.tpc, grp_trees = (tpc + G - 1) / G;
+    const int tpc = fv.tpc, grp_trees = (tpc + GPR - 1) / GPR;
     const int np = NP >= 0 ? NP : fv.depth - L;
     constexpr int kTop = (1 << L) - 1;
-    const int t_first = grp * grp_trees;
+    const int ring = grp / GPR;
+    // the groups of a ring share out the trees of its chunks
+    const int t_first = (grp % GPR) * grp_trees;
     const int t_count = t_first + grp_trees <= tpc ? grp_trees : (tpc > t_first ? tpc - t_first : 0);
 #ifdef KS_DEBUG_BOUNDS
     const uint32_t tile0 = sbase + kOffTile, tile_bytes = static_cast<uint32_t>(fv.n_rows) * NC;
 #else
     constexpr uint32_t tile0 = 0, tile_bytes = 0;
 #endif
-    const int ch_stop = kFloor ? ch_begin + (ch_end - ch_begin) * sl.repeat : ch_end;
+    // this ring's chunks: n_mine of them; the floor form walks its first kNBuf again and again
+    const int n_mine = ch_end - ch_begin > ring ? (ch_end - ch_begin - ring + RG - 1) / RG : 0;
+    const int n_walks = kFloor ? n_mine * sl.repeat : n_mine;
 #pragma unroll 1
-    for (int ch_it = ch_begin; ch_it < ch_stop; ++ch_it) {
-      const int b = (ch_it - ch_begin) % kNBuf;
-      const int ch = kFloor ? ch_begin + b : ch_it;  // the chunk whose trees are walked
-      const uint32_t bar = bar0 + 8u * b;
+    for (int it = 0; it < n_walks; ++it) {
+      const int b = it % kNBuf, rb = ring * kNBuf + b;
+      const int ch = ch_begin + ring + (kFloor ? b : it) * RG;  // the chunk whose trees are walked
+      const uint32_t bar = bar0 + 8u * rb;
       const uint32_t par = (phases >> b) & 1u;
       // A wait that runs out ends the walk of this CTA: the buffer was never filled, so it is not
       // read; the call fails, and the CTAs that start later leave at once.
-      if (!kFloor || ch_it - ch_begin < kNBuf) {
+      if (!kFloor || it < kNBuf) {
         if (*v_fail || !mbar_wait_bounded(bar, par, fv.wait_limit, v_fail)) {
           if (!*v_fail) {
             s_fail = 1;
@@ -852,7 +868,7 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
         }
         phases ^= 1u << b;
       }
-      const uint32_t buf = sbase + kOffBuf0 + b * fv.buf_bytes;
+      const uint32_t buf = sbase + kOffBuf0 + rb * fv.buf_bytes;
       // With A_l the shared address of a walk's node at level l, A_{l+1} = 2 A_l + (4 tpc - buf)
       // + 4 bit for every level, and after the last level A points at the walk's leaf.
       const uint32_t k0 = 4u * tpc - buf;  // modulo 2^32, like the additions it enters
@@ -920,37 +936,37 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
           score[r] += lds_f32(a[r]);
         }
       }
-      // Release the buffer without a block-wide barrier: every warp counts itself out, and the
-      // last one to leave refills the buffer (nobody waits; warps may run a chunk ahead).
+      // Release the buffer without a block-wide barrier: every warp of the group counts itself
+      // out, and the last one to leave refills the buffer (nobody waits; warps may run a chunk ahead).
       __syncwarp();
       if (!kFloor && (tid & 31) == 0) {
-        if (atomicAdd(&s_done[b], 1) == THREADS / 32 - 1) {
-          s_done[b] = 0;
-          s_pending[b] = 0;
-          if (ch + kNBuf < ch_end && !*v_fail) {
+        if (atomicAdd(&s_done[rb], 1) == THREADS / 32 / RG - 1) {
+          s_done[rb] = 0;
+          s_pending[rb] = 0;
+          if (ch + kNBuf * RG < ch_end && !*v_fail) {
             fence_async_proxy();
             mbar_expect_tx(bar, fv.chunk_bytes + (fv.starve ? 16 : 0));
             bulk_copy_g2s(buf, reinterpret_cast<const char*>(fv.chunks) +
-                                   static_cast<size_t>(KS_IDX(ch + kNBuf, fv.n_chunks)) * fv.chunk_bytes,
+                                   static_cast<size_t>(KS_IDX(ch + kNBuf * RG, fv.n_chunks)) * fv.chunk_bytes,
                           fv.chunk_bytes, bar);
-            s_pending[b] = 1;
+            s_pending[rb] = 1;
           }
         }
       }
     }
     __syncthreads();  // all walks are done: the buffers are free
-    if (kFloor && tid < kNBuf && !*v_fail) s_pending[tid] = 0;  // copied once, landed, never refilled
+    if (kFloor && tid < kNBuf * RG && !*v_fail) s_pending[tid] = 0;  // copied once, landed, never refilled
     if (*v_fail) {
       // The call has failed. Before this CTA gives its shared memory back, give the copies that
       // may still be in flight the time to land (bounded again); the test hook's copies land in
       // full although their barriers never complete, so there a short pause stands in for it.
-      if (tid == 0) {
+      if (word == 0 && grp % GPR == 0) {  // one thread per ring, for its ring's buffers (it knows their parities)
         for (int b = 0; b < kNBuf; ++b) {
-          if (!s_pending[b]) continue;
+          if (!s_pending[ring * kNBuf + b]) continue;
           if (fv.starve) {
             for (int i = 0; i < 64; ++i) __nanosleep(kSleepNs);
           } else {
-            mbar_wait_bounded(bar0 + 8u * b, (phases >> b) & 1u, fv.wait_limit, &s_abort /* stays 0 */);
+            mbar_wait_bounded(bar0 + 8u * (ring * kNBuf + b), (phases >> b) & 1u, fv.wait_limit, &s_abort /* stays 0 */);
           }
         }
       }
@@ -1224,13 +1240,16 @@ cudaError_t build_fast_gbdt(GbdtModel& m, int n_trees, const int64_t* off, const
   if (table.empty()) table.push_back(0.0f);
   const int G = threads / (NC / 4);
   const int per_tree_words = (2 << D) - 1;
-  int tpc = geom.buf_bytes / (per_tree_words * 4) / 2 * 2;  // even: the two groups of the smallest geometry share a chunk's trees
-  if (tpc < 2) return cudaSuccess;
-  if (tpc >= G) tpc = tpc / G * G;  // whole groups (fewer trees than groups: the spare groups idle)
-  if (tpc > (n_trees + G - 1) / G * G) tpc = (n_trees + G - 1) / G * G;  // a small ensemble is one short chunk
+  // A chunk is what one ring's buffer holds (the geometry's buffer size is shared out among the
+  // rings); ring r takes the chunks r, r + rings, ..., and the groups of a ring split a chunk's trees.
+  const int rings = ring_count(G), gpr = G / rings;
+  const int group_buf = geom.buf_bytes / rings / 16 * 16;
+  int tpc = group_buf / (per_tree_words * 4) / gpr * gpr;
+  if (tpc < gpr) return cudaSuccess;
+  if (tpc > (n_trees + G - 1) / G * gpr) tpc = (n_trees + G - 1) / G * gpr;  // a small ensemble: one short chunk per ring
   const int n_chunks = (n_trees + tpc - 1) / tpc;
   const int chunk_words = (tpc * per_tree_words + 3) / 4 * 4;  // bulk copies move multiples of 16 bytes
-  if (chunk_words * 4 > geom.buf_bytes) return cudaSuccess;
+  if (chunk_words * 4 > group_buf) return cudaSuccess;
   int L = D < 3 ? D : 3;  // levels whose nodes travel as kernel-parameter constants
   while (L > 0 && static_cast<int64_t>(n_chunks) * tpc * ((1 << L) - 1) > kFastTopPairs) --L;
   // three levels in the compact form (one word per node) when the pair form would leave fewer
@@ -1336,7 +1355,7 @@ cudaError_t build_fast_gbdt(GbdtModel& m, int n_trees, const int64_t* off, const
   m.fast_depth = D;
   m.fast_threads = threads;
   m.block_cands = NC;
-  m.buf_bytes = geom.buf_bytes;
+  m.buf_bytes = group_buf;
   m.ctas_per_sm = geom.ctas_per_sm;
   m.n_qrows = n_rows;
   m.n_pair_rows = n_class[2];
@@ -1470,7 +1489,8 @@ struct WalkArgs {
 
 template <int L, int NP, bool kCompact, int THREADS, int NC, bool kFloor = false>
 cudaError_t launch_ln(const WalkArgs& a) {
-  const size_t smem = static_cast<size_t>(kNBuf) * a.fv.buf_bytes + static_cast<size_t>(a.fv.n_rows) * NC;
+  const size_t smem = static_cast<size_t>(kNBuf) * ring_count(THREADS / (NC / 4)) * a.fv.buf_bytes +
+                      static_cast<size_t>(a.fv.n_rows) * NC;
   auto kernel = &select_fast_kernel<L, NP, kCompact, THREADS, NC, kFloor>;
   cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kernel), smem);
   if (e != cudaSuccess) return e;
@@ -1523,7 +1543,8 @@ cudaError_t launch_walk_geom(const GbdtModel& g, const WalkArgs& a) {
 // The floor measurement exists for the two geometries and the ensemble shape of the benchmark's
 // first configuration (three word-wise levels, five path levels, top constants as pairs).
 cudaError_t launch_walk_floor(const GbdtModel& g, const WalkArgs& a) {
-  if (g.top_compact || g.top_levels != 3 || g.fast_depth != 8 || g.n_chunks < kNBuf || g.block_cands != 1024)
+  if (g.top_compact || g.top_levels != 3 || g.fast_depth != 8 || g.block_cands != 1024 ||
+      g.n_chunks < kNBuf * ring_count(g.fast_threads / 256))  // every ring needs its kNBuf resident chunks
     return cudaErrorNotSupported;
   if (g.fast_threads == 512) return launch_ln<3, 5, false, 512, 1024, true>(a);
   return launch_ln<3, 5, false, 256, 1024, true>(a);

@@ -171,18 +171,23 @@ def test_walk_floor_sums(ks, ctx):
     x = oracle.featurize(w.problems, w.candidates, DESC)
     off, nodes, base = w.gbdt
     model = ctx.model_create_gbdt(off, nodes, base)
-    m = re.search(r"chunks=(\d+) chunk_trees=(\d+)", model.describe())
-    assert "block=1024" in model.describe() and m, model.describe()
-    n_chunks, tpc = int(m.group(1)), int(m.group(2))
-    assert n_chunks >= 2
+    m = re.search(r"threads=(\d+) block=1024 .*chunks=(\d+) chunk_trees=(\d+)", model.describe())
+    assert m, model.describe()
+    G, n_chunks, tpc = int(m.group(1)) // 256, int(m.group(2)), int(m.group(3))
+    assert n_chunks >= 2 * G
+    # tree group g walks chunks g, g + G, ...; its first two stay resident
     part = [oracle.score_gbdt(x, off[c * tpc:(c + 1) * tpc + 1] - off[c * tpc],
-                              nodes[off[c * tpc]:off[(c + 1) * tpc]], 0.0) for c in (0, 1)]
+                              nodes[off[c * tpc]:off[(c + 1) * tpc]], 0.0).astype(np.float64) for c in range(2 * G)]
     d_x = dev(ks, x)
     for repeat in (1, 3):
-        n = repeat * n_chunks
         got = ctx.debug_walk_floor(d_x, model, repeat).cpu().numpy()
-        want = base + ((n + 1) // 2) * part[0].astype(np.float64) + (n // 2) * part[1].astype(np.float64)
-        assert np.all(np.abs(got - want) <= 4 * TOL_GBDT * n * np.maximum(1, np.abs(want)))
+        want = np.full(len(x), np.float64(base))
+        walks = 0
+        for g in range(G):
+            n = repeat * len(range(g, n_chunks, G))
+            want += ((n + 1) // 2) * part[g] + (n // 2) * part[g + G]
+            walks += n
+        assert np.all(np.abs(got - want) <= 4 * TOL_GBDT * walks * np.maximum(1, np.abs(want)))
     assert np.std(part[0]) > 1e-2
     # an ensemble in another tile geometry or shape is refused
     w2 = wl.make_workload(0, P=1, C=300)
