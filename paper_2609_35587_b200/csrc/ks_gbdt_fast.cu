@@ -1148,7 +1148,7 @@ static bool geometry_known(int t, int c) {
 static bool pick_geometry(int n_rows, Geometry* out) {
   if (const char* env = std::getenv("KS_FAST_GEOMETRY")) {
     int t = 0, c = 0, kb = 0;
-    if (std::sscanf(env, "%d,%d,%d", &t, &c, &kb) == 3 && geometry_known(t, c) && kb >= 8 && kb <= 32) {
+    if (std::sscanf(env, "%d,%d,%d", &t, &c, &kb) == 3 && geometry_known(t, c) && kb >= 8 && kb <= 64) {
       Geometry g{t, c, kb * 1024, 2};
       if (!geometry_fits(g, n_rows)) g.ctas_per_sm = 1;
       if (geometry_fits(g, n_rows)) {
