@@ -27,6 +27,8 @@ def main() -> int:
     cases.append(("cfg1 pernode", wl.make_workload(1, P=2, C=2100, law="pernode"), 10))
     cases.append(("cfg2 pernode segments", wl.make_workload(2, P=3, seg=1100, law="pernode"), 10))
     cases.append(("cfg2 memo", wl.make_workload(2, P=40, seg=90, trees=30, depth=6), 10))
+    # more (problem, candidate block) items than SMs: the launch form in which a CTA serves many items
+    cases.append(("many items", wl.make_workload(1, P=90, C=2100, trees=24, depth=8, law="pernode"), 10))
     for name, w, k in cases:
         model = ctx.model_create_gbdt(*w.gbdt)
         assert "select_fast_kernel" in model.describe(), (name, model.describe())
