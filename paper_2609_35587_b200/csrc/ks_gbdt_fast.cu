@@ -31,13 +31,15 @@
 //   the tiles are built once by tile_one_kernel; scoring call (ks_score): tiles are quantised
 //   from given feature rows by tile_rows_kernel and the scores are stored instead of ranked.
 //
-// Kernel (one CTA = one problem x up to NC candidates, THREADS threads)
+// Kernel (an item = one problem x up to NC candidates; a CTA of THREADS threads serves one item,
+// or - batch form of the geometries with one CTA per SM - the items blockIdx.x, + gridDim.x, ...)
 //   phase A  fill the [row][candidate] byte tile. A 32-bit word of a row holds the four
 //            candidates that share a lane slot, so a warp's byte loads of any mix of rows
 //            touch 32 distinct banks and one word load serves four candidates;
-//   phase B  stream the ensemble through two shared-memory buffers (cp.async.bulk + mbarrier,
-//            bounded waits). Thread (w, g) owns the four candidates of word w and walks the
-//            trees of group g of every chunk. The top levels are evaluated for all four
+//   phase B  stream the ensemble through rings of two shared-memory buffers (cp.async.bulk +
+//            mbarrier, bounded waits). Thread (w, g) owns the four candidates of word w and
+//            walks group g's share of the trees: the chunks of its ring (see ring_count), and of
+//            those the trees that fall to it when two groups share a ring. The top levels are evaluated for all four
 //            candidates at once, node by node, with byte-parallel arithmetic on whole words;
 //            below that each candidate follows its own path: a' = 2 a + k0 (+ 4 to go right), a
 //            multiply-add plus a predicated add;
@@ -65,7 +67,6 @@ constexpr int kSlice = 127;            // thresholds per row: a byte is 0x80 | (
 constexpr unsigned kSleepNs = 1200;    // asked-for sleep between two probes of a chunk barrier (400 to 2500 measured alike)
 constexpr int kCombos = 16;            // dtype_ab x dtype_d
 
-// shared memory map (byte offsets from the dynamic shared base): the chunk buffers, then the tile
 constexpr int kSmCount = 148;           // SMs of the one device this library is built for (sm_100a)
 // Chunk rings of a CTA with G tree groups: every ring has kNBuf buffers and serves G / rings groups,
 // which share out the trees of its chunks; ring r takes the chunks r, r + rings, ... A ring of
@@ -73,7 +74,8 @@ constexpr int kSmCount = 148;           // SMs of the one device this library is
 // shared memory and the same trees per thread and chunk (config 1, two groups: 55.3 -> 54.4 ms);
 // four groups do best with two rings (config 2: 132.4 ms with four rings, 131.6 with one, 129.3 with two).
 __host__ __device__ constexpr int ring_count(int groups) { return groups <= 2 ? groups : 2; }
-constexpr int kNBuf = 2;                // tree-chunk buffers (a ring; four of 8 KB and three of 12 KB measured slower)
+constexpr int kNBuf = 2;                // buffers of a ring (four of 8 KB and three of 12 KB measured slower)
+// shared memory map (byte offsets from the dynamic shared base): the rings' chunk buffers, then the tile
 constexpr int kOffBuf0 = 0;
 
 #ifdef KS_DEBUG_BOUNDS
