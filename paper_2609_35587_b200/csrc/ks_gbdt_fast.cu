@@ -32,7 +32,8 @@
 //   from given feature rows by tile_rows_kernel and the scores are stored instead of ranked.
 //
 // Kernel (an item = one problem x up to NC candidates; a CTA of THREADS threads serves one item,
-// or - batch form of the geometries with one CTA per SM - the items blockIdx.x, + gridDim.x, ...)
+// or - batch form of the geometries with one CTA per SM - a run of items: one candidate block
+// for problem after problem, whose candidate-only rows it keeps in the tile)
 //   phase A  fill the [row][candidate] byte tile. A 32-bit word of a row holds the four
 //            candidates that share a lane slot, so a warp's byte loads of any mix of rows
 //            touch 32 distinct banks and one word load serves four candidates;
@@ -573,10 +574,13 @@ __device__ __noinline__ void fill_tile(const ks_gpu_desc& desc, const ProblemTer
                                        const ks_candidate* __restrict__ c, const FastView& fv,
                                        const int64_t* __restrict__ seg_off, const int32_t* __restrict__ seg_idx,
                                        int C, int64_t lo, int64_t start, int64_t stop, const float* T,
-                                       const FeatQ* s_fq, const uint8_t* s_pbin, unsigned char* tile, int prob) {
+                                       const FeatQ* s_fq, const uint8_t* s_pbin, unsigned char* tile, int prob,
+                                       unsigned* s_cid, bool reuse) {
   constexpr int W = NC / 4, PARTS = THREADS / W;
   const int tid = threadIdx.x;
   const int combo = pt.dtype_ab * 4 + pt.dtype_d;
+  // `reuse`: the tile still holds the candidate-only rows of these very candidates (the CTA's last
+  // item was the same candidate block under the same element types), and s_cid their classes.
   // problem-only rows: one byte for the whole row
   {
     unsigned char* dst = tile + static_cast<size_t>(fv.n_pair_rows + fv.n_cand_rows) * NC;
@@ -590,15 +594,25 @@ __device__ __noinline__ void fill_tile(const ks_gpu_desc& desc, const ProblemTer
   int ci[4];
   unsigned cid[4];
   bool lone = false;  // one of this word's candidates has no record of per-pair rows
+  if (reuse) {
 #pragma unroll
-  for (int r = 0; r < 4; ++r) {
-    const int64_t row = start + 4 * word + r;
-    ci[r] = row < stop ? (seg_idx ? seg_idx[lo + row] : static_cast<int>(row)) : -1;
-  }
+    for (int r = 0; r < 4; ++r) {
+      ci[r] = start + 4 * word + r < stop ? 0 : -1;  // (the pool index itself is not needed again)
+      cid[r] = s_cid[4 * word + r];
+      lone |= ci[r] >= 0 && cid[r] == kNoClass;
+    }
+  } else {
 #pragma unroll
-  for (int r = 0; r < 4; ++r) {
-    cid[r] = (ci[r] >= 0 && fv.pair_class) ? __ldg(fv.pair_class + static_cast<size_t>(combo) * C + ci[r]) : kNoClass;
-    lone |= ci[r] >= 0 && cid[r] == kNoClass;
+    for (int r = 0; r < 4; ++r) {
+      const int64_t row = start + 4 * word + r;
+      ci[r] = row < stop ? (seg_idx ? seg_idx[lo + row] : static_cast<int>(row)) : -1;
+    }
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      cid[r] = (ci[r] >= 0 && fv.pair_class) ? __ldg(fv.pair_class + static_cast<size_t>(combo) * C + ci[r]) : kNoClass;
+      lone |= ci[r] >= 0 && cid[r] == kNoClass;
+      if (s_cid && part == 0) s_cid[4 * word + r] = cid[r];
+    }
   }
   const uint4 neutral = make_uint4(0x80808080u, 0x80808080u, 0x80808080u, 0x80808080u);
   const int cand_vecs = (fv.n_cand_rows + 15) / 16, pair_vecs = (fv.n_pair_rows + 15) / 16;
@@ -615,7 +629,7 @@ __device__ __noinline__ void fill_tile(const ks_gpu_desc& desc, const ProblemTer
   // waits for the memory once per batch, not once per vector
   constexpr int kBatch = 1;
 #pragma unroll 1
-  for (int v0 = part; v0 < cand_vecs + pair_vecs; v0 += kBatch * PARTS) {
+  for (int v0 = (reuse ? cand_vecs : 0) + part; v0 < cand_vecs + pair_vecs; v0 += kBatch * PARTS) {
     uint4 q[kBatch][4];
 #pragma unroll
     for (int j = 0; j < kBatch; ++j) {
@@ -643,7 +657,8 @@ __device__ __noinline__ void fill_tile(const ks_gpu_desc& desc, const ProblemTer
   for (int r = part % 4; r < 4; r += (PARTS < 4 ? PARTS : 4)) {
     if (ci[r] < 0 || cid[r] != kNoClass) continue;
     unsigned char* my = word0 + r;
-    const ks_candidate cand = load_candidate(c + ci[r]);
+    const int64_t row = start + 4 * word + r;
+    const ks_candidate cand = load_candidate(c + (seg_idx ? seg_idx[lo + row] : static_cast<int>(row)));
     pair_columns<true>(pt, cand, desc, resources(pt, cand, desc).b_eff, [&](int col, float v) {
       const FeatQ& q = s_fq[col];
       quantise(q, T + q.thr0, v, false, [&](int row, uint8_t b) { my[KS_IDX(row, fv.n_pair_rows) * NC] = b; });
@@ -727,6 +742,9 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
   __shared__ uint8_t s_pbin[kFastMaxProbRows];
   __shared__ float s_pfeat[64];
   __shared__ int s_fail, s_last, s_done[kNBuf * RG], s_abort, s_pending[kNBuf * RG];
+  // the classes of the candidates whose candidate-only rows the tile holds (one-CTA forms only:
+  // there a CTA serves one candidate block for many problems in a row, see below)
+  __shared__ unsigned s_cid[THREADS > 256 ? NC : 1];
 
   const int tid = threadIdx.x;
   const int kOffTile = kNBuf * RG * fv.buf_bytes;  // every ring has kNBuf buffers
@@ -749,14 +767,23 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
   const int word = tid % W, grp = tid / W;
   volatile int* v_fail = &s_fail;
 
-  // A CTA serves the items blockIdx.x, blockIdx.x + gridDim.x, ...: an item is one (problem,
-  // candidate block, tree slice). The batch form of a geometry that holds one CTA per SM is
+  // An item is one (problem, candidate block, tree slice). The batch form of a geometry that holds one CTA per SM is
   // launched with one CTA per SM, so that a CTA's set-up and the gap between two CTAs are paid
   // once, not per item; everything else (two CTAs per SM, which hide each other's gaps; tree
   // slices and scoring, which leave an item early) is launched with one CTA per item.
+  // A CTA that serves many items of a dense batch takes a run of consecutive items in the order
+  // (candidate block, problem): successive items then are the same candidates for another problem,
+  // and while the element types stay the same their candidate-only rows (and classes) stay in place.
+  const int grid = static_cast<int>(gridDim.x), cta = static_cast<int>(blockIdx.x);
+  const bool block_major = grid < n_items && !seg_off && S == 1;
+  const int per_cta = (n_items + grid - 1) / grid;
+  const int first_item = block_major ? cta * per_cta : cta, item_step = block_major ? 1 : grid;
+  const int last_item = block_major ? (first_item + per_cta < n_items ? first_item + per_cta : n_items) : n_items;
+  int held_chunk = -1, held_combo = -1;  // what the tile's candidate-only rows belong to
 #pragma unroll 1
-  for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
-  const int prob = item / (nblk * S), chunk = (item / S) % nblk, slice = item % S;
+  for (int item = first_item; item < last_item; item += item_step) {
+  const int prob = block_major ? item % P : item / (nblk * S);
+  const int chunk = block_major ? item / P : (item / S) % nblk, slice = item % S;
   // rows of this problem: lo = where its scores sit in per-row arrays; lo_idx = where its pool
   // indices start in seg_idx (per-problem segments, or - without offsets - one ranking order of
   // the whole catalogue shared by every problem)
@@ -814,8 +841,12 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
       const float* T = stage_thresholds(fv, 0, fv.thr_cand0, reinterpret_cast<float*>(smem + kOffBuf0),
                                         fv.pair_class ? 0 : kNBuf * RG * fv.buf_bytes / 4);
       __syncthreads();
+      const int combo = s_pt.dtype_ab * 4 + s_pt.dtype_d;
+      const bool reuse = THREADS > 256 && block_major && fv.pair_class && chunk == held_chunk && combo == held_combo;
       fill_tile<THREADS, NC>(desc, s_pt, c, fv, seg_off, seg_idx, C, lo_idx, start, stop, T, s_fq, s_pbin,
-                             smem + kOffTile, prob);
+                             smem + kOffTile, prob, THREADS > 256 && block_major ? s_cid : nullptr, reuse);
+      held_chunk = chunk;
+      held_combo = combo;
     }
     __syncthreads();  // tile complete; the threshold table is no longer needed
 
@@ -1136,7 +1167,8 @@ struct Geometry {
   int threads, cands, buf_bytes, ctas_per_sm;
 };
 static size_t geometry_smem(const Geometry& g, int n_rows) {
-  const size_t stat = 2560 + static_cast<size_t>(g.threads) / 32 * KS_MAX_K * 8 + 256;  // static shared memory of the kernel, with slack
+  // static shared memory of the kernel, with slack (the one-CTA forms keep a class per candidate)
+  const size_t stat = 2560 + static_cast<size_t>(g.threads) / 32 * KS_MAX_K * 8 + 256 + (g.threads > 256 ? 4 * g.cands : 0);
   return static_cast<size_t>(kNBuf) * g.buf_bytes + static_cast<size_t>(n_rows) * g.cands + stat;
 }
 static bool geometry_fits(const Geometry& g, int n_rows) {

@@ -648,6 +648,17 @@ def test_select_more_items_than_sms(ks, ctx, geometry, segments, monkeypatch):
     check_select(w, idx, sc, TOL_GBDT, sample=range(0, 110, 2))
     idx2, sc2 = run_select(ks, ctx, w, model)     # the barriers' parities carry over from call to call
     assert np.array_equal(idx, idx2) and np.array_equal(sc, sc2)
+    if not segments:
+        # a CTA keeps a candidate block's candidate-only rows from one problem to the next while
+        # the element types stay the same: runs of equal types of every length, and switches
+        rng = np.random.default_rng(11)
+        w.problems = w.problems.copy()
+        kinds = [(0, 0), (1, 1), (2, 1), (3, 3)]       # (dtype_ab, dtype_d)
+        pick = np.repeat(rng.integers(0, 4, 40), rng.integers(1, 6, 40))[:110]
+        w.problems["dtype_ab"] = [kinds[i][0] for i in pick]
+        w.problems["dtype_d"] = [kinds[i][1] for i in pick]
+        idx, sc = run_select(ks, ctx, w, model)
+        check_select(w, idx, sc, TOL_GBDT, sample=range(0, 110, 3))
 
 
 @pytest.mark.parametrize("law", ["slots128", "pernode"])
