@@ -744,7 +744,7 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
   __shared__ int s_fail, s_last, s_done[kNBuf * RG], s_abort, s_pending[kNBuf * RG];
   // the classes of the candidates whose candidate-only rows the tile holds (one-CTA forms only:
   // there a CTA serves one candidate block for many problems in a row, see below)
-  __shared__ unsigned s_cid[THREADS > 256 ? NC : 1];
+  __shared__ unsigned s_cid[THREADS > 256 && NC == 1024 ? NC : 1];
 
   const int tid = threadIdx.x;
   const int kOffTile = kNBuf * RG * fv.buf_bytes;  // every ring has kNBuf buffers
@@ -771,11 +771,14 @@ select_fast_kernel(ks_gpu_desc desc, const ks_problem* __restrict__ p, ks_proble
   // launched with one CTA per SM, so that a CTA's set-up and the gap between two CTAs are paid
   // once, not per item; everything else (two CTAs per SM, which hide each other's gaps; tree
   // slices and scoring, which leave an item early) is launched with one CTA per item.
-  // A CTA that serves many items of a dense batch takes a run of consecutive items in the order
-  // (candidate block, problem): successive items then are the same candidates for another problem,
-  // and while the element types stay the same their candidate-only rows (and classes) stay in place.
+  // A CTA (of the 1,024-candidate forms) that serves many items of a dense batch takes a run of
+  // consecutive items in the order (candidate block, problem): successive items then are the same
+  // candidates for another problem, and while the element types stay the same their
+  // candidate-only rows (and classes) stay in place. (The 512-candidate form serves segmented
+  // batches in the benchmark; compiled with this path it ran them 2 % slower, so it keeps the
+  // plain order.)
   const int grid = static_cast<int>(gridDim.x), cta = static_cast<int>(blockIdx.x);
-  const bool block_major = grid < n_items && !seg_off && S == 1;
+  const bool block_major = NC == 1024 && grid < n_items && !seg_off && S == 1;
   const int per_cta = (n_items + grid - 1) / grid;
   const int first_item = block_major ? cta * per_cta : cta, item_step = block_major ? 1 : grid;
   const int last_item = block_major ? (first_item + per_cta < n_items ? first_item + per_cta : n_items) : n_items;
@@ -1168,7 +1171,7 @@ struct Geometry {
 };
 static size_t geometry_smem(const Geometry& g, int n_rows) {
   // static shared memory of the kernel, with slack (the one-CTA forms keep a class per candidate)
-  const size_t stat = 2560 + static_cast<size_t>(g.threads) / 32 * KS_MAX_K * 8 + 256 + (g.threads > 256 ? 4 * g.cands : 0);
+  const size_t stat = 2560 + static_cast<size_t>(g.threads) / 32 * KS_MAX_K * 8 + 256 + (g.threads > 256 && g.cands == 1024 ? 4 * g.cands : 0);
   return static_cast<size_t>(kNBuf) * g.buf_bytes + static_cast<size_t>(n_rows) * g.cands + stat;
 }
 static bool geometry_fits(const Geometry& g, int n_rows) {
